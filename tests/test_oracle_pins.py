@@ -1,0 +1,449 @@
+"""CPU-only tests that pin the oracle to what the paper and the mathematics fix.
+
+Each test names the passage it checks.  None of them re-types the oracle's own formula: they use
+the paper's printed values (Table II, Theorem 1), invariants stated in the Appendix proof, closed
+forms, special cases that reduce to a library routine, and brute-force search over the explicit
+set of representable values with exact rational arithmetic.
+"""
+import itertools
+import math
+import os
+from fractions import Fraction
+
+import numpy as np
+import pytest
+
+from oracle import oracle as orc
+from paper_2302_08007_b200 import synth
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+Cfg = orc.Config
+
+GRID = [Cfg(k1, 8, k2, d2, m) for k1 in (1, 2, 4, 8, 16, 32, 64, 1024) for k2 in (1, 2, 4, 8)
+        for d2 in (0, 1, 2, 3) for m in (1, 2, 4, 7, 8) if k2 <= k1]
+SMALL_GRID = GRID[::7]
+
+
+def _golden_rows(name):
+    with open(os.path.join(GOLDEN, name)) as f:
+        return [ln.strip() for ln in f if ln.strip() and not ln.startswith("#")]
+
+
+# ---- Table II: bits per element -----------------------------------------------------------------
+def test_table2_bits_per_element_formula_and_packed_bytes():
+    for row in _golden_rows("table2_formats.txt"):
+        name, k1, k2, d1, d2, m, bits = row.split()
+        cfg = Cfg(int(k1), int(d1), int(k2), int(d2), int(m))
+        assert orc.bits_per_element(cfg) == float(bits)
+        # the packed planes spend exactly that many bits when the line needs no padding
+        rows, cols = 3, 1024
+        _, nbytes = orc.packed_sizes(cfg, rows, cols, axis=1)
+        assert sum(nbytes) * 8 == int(bits) * rows * cols
+        _, nbytes = orc.packed_sizes(cfg, cols, rows, axis=0)
+        assert sum(nbytes) * 8 == int(bits) * rows * cols
+
+
+def test_bits_per_element_general():
+    # Section III: (m+1) + d1/k1 + d2/k2, e.g. MSFP16-like k1=16, d2=0, m=7 -> 8.5 bits
+    assert orc.bits_per_element(Cfg(16, 8, 1, 0, 7)) == 8.5
+    assert orc.bits_per_element(Cfg(8, 8, 8, 2, 3)) == 4 + 1 + 0.25
+
+
+# ---- Theorem 1 -----------------------------------------------------------------------------------
+def test_theorem1_closed_form_values():
+    for row in _golden_rows("theorem1_bounds.txt"):
+        name, m, bound = row.split()
+        cfg = Cfg(16, 8, 2, 1, int(m))
+        assert abs(orc.theorem1_bound_db(cfg, 1 << 20) - float(bound)) < 1e-3
+    # N < k1 replaces k1 by N (end of the proof)
+    assert orc.theorem1_bound_db(Cfg(16, 8, 2, 1, 4), 4) > orc.theorem1_bound_db(Cfg(16, 8, 2, 1, 4), 16)
+
+
+def test_theorem1_holds_on_random_and_adversarial_inputs():
+    rng = np.random.default_rng(5)
+    inputs = [synth.normal(4096, 1), synth.laplace(4096, 2), synth.student_t(4096, 3),
+              synth.normal_with_outliers(4096, 4, frac=0.01),
+              (rng.standard_normal(4096) * np.exp2(rng.integers(-6, 6, 4096))).astype(np.float32)]
+    for cfg in GRID:
+        if cfg.m < 2:
+            continue
+        for x in inputs:
+            assert orc.qsnr(cfg, x) >= orc.theorem1_bound_db(cfg, x.size) - 1e-9, cfg
+
+
+def test_theorem1_worst_case_search_tiny_blocks():
+    # every block from a grid of magnitudes in a few binades; k1=4, k2=2
+    vals = np.array([0.0] + [m * 2.0 ** e for e in (-3, -2, -1, 0) for m in (1.0, 1.24, 1.26, 1.5, 1.74, 1.99)],
+                    dtype=np.float32)
+    blocks = np.array(list(itertools.product(vals, repeat=4)), dtype=np.float32)
+    blocks = blocks[np.abs(blocks).max(axis=1) > 0]
+    for d2 in (0, 1, 2):
+        for m in (2, 3):
+            cfg = Cfg(4, 8, 2, d2, m)
+            y, _ = orc.quant_dequant(cfg, blocks)
+            e2 = ((y.astype(np.float64) - blocks) ** 2).sum(axis=1)
+            s2 = (blocks.astype(np.float64) ** 2).sum(axis=1)
+            worst = (-10 * np.log10(np.maximum(e2, 1e-300) / s2)).min()
+            assert worst >= orc.theorem1_bound_db(cfg, 4) - 1e-9
+
+
+# ---- hand-worked blocks ---------------------------------------------------------------------------
+def test_hand_worked_blocks():
+    for row in _golden_rows("hand_blocks.txt"):
+        rnd, xs, qs, F, taus, codes = [f.strip() for f in row.split("|")]
+        cfg = Cfg(8, 8, 2, 1, 4, orc.POW2, int(rnd))
+        x = np.array([float(v) for v in xs.split()], dtype=np.float32)
+        want = np.array([float(v) for v in qs.split()], dtype=np.float32)
+        y, _ = orc.quant_dequant(cfg, x)
+        assert y.view(np.uint32).tolist() == want.view(np.uint32).tolist()
+        Fo, tauo, codeo = orc.encode(cfg, x)
+        assert Fo.ravel().tolist() == [int(F)]
+        assert tauo.ravel().tolist() == [int(t) for t in taus.split()]
+        assert codeo.ravel().tolist() == [int(c, 16) for c in codes.split()]
+
+
+def test_hand_worked_packed_bytes():
+    # 5-bit codes 08 16 05 04 02 11 0f 04, LSB first: bits written out by hand
+    x = np.array([1.0, -0.75, 0.3, 0.26, 0.124, -0.06, 1.9, 0.49], dtype=np.float32)
+    exps, micro, elems = orc.pack(Cfg(8, 8, 2, 1, 4), x)
+    bits = "".join(format(c, "05b")[::-1] for c in (0x08, 0x16, 0x05, 0x04, 0x02, 0x11, 0x0F, 0x04))
+    want = bytes(int(bits[i:i + 8][::-1], 2) for i in range(0, 40, 8))
+    assert bytes(elems[0, :5]) == want == bytes.fromhex("c81622e223")
+    assert exps[0, 0] == 127 and micro[0, 0] == 0b0110
+    assert not elems[0, 5:].any() and not exps[0, 1:].any() and not micro[0, 1:].any()
+
+
+# ---- Appendix invariants ---------------------------------------------------------------------------
+def _fields(cfg, x):
+    F, tau, code = orc.encode(cfg, x)
+    y, _ = orc.quant_dequant(cfg, x)
+    n = x.size
+    nb = F.shape[1]
+    q = (code & ((1 << cfg.m) - 1)).astype(np.int64).ravel()[:n]
+    s = (code >> cfg.m).astype(np.int64).ravel()[:n]
+    Fe = np.repeat(F.ravel().astype(np.int64), cfg.k1)[:n]
+    te = np.repeat(tau.ravel().astype(np.int64), cfg.k2)[:n]
+    return F, tau, q, s, Fe, te, y, nb
+
+
+@pytest.mark.parametrize("cfg", SMALL_GRID, ids=str)
+def test_representation_form_and_error_bounds(cfg):
+    """Q(x) = +-q * 2^(E-tau-m+1) with integer q < 2^m; |Q(x)-x| <= 2^(E-tau-m) unless clamped."""
+    for x in (synth.normal(2048, 7), synth.edge_case_values(2048, 8)):
+        F, tau, q, s, Fe, te, y, nb = _fields(cfg, x)
+        assert q.max() < (1 << cfg.m) and tau.max() <= (1 << cfg.d2) - 1
+        p = Fe - 127 - te - (cfg.m - 1)
+        recon = np.ldexp(q.astype(np.float64), p) * np.where(s == 1, -1.0, 1.0)
+        assert np.array_equal(recon.astype(np.float32).view(np.uint32), y.view(np.uint32))
+        assert np.array_equal(s, (x.view(np.uint32) >> 31).astype(np.int64))      # sign kept, also for zeros
+        err = np.abs(y.astype(np.float64) - x.astype(np.float64))
+        half = np.ldexp(1.0, p - 1)
+        clamped = np.abs(x.astype(np.float64)) > np.ldexp(float((1 << cfg.m) - 1), p)
+        assert (err[~clamped] <= half[~clamped]).all()
+        assert (err[clamped] <= 2 * half[clamped]).all()
+        assert (q[clamped] == (1 << cfg.m) - 1).all()
+
+
+@pytest.mark.parametrize("cfg", SMALL_GRID, ids=str)
+def test_shared_exponent_and_microexponent_structure(cfg):
+    """E is the largest private exponent; the block's largest element sits in a sub-block with
+    tau = 0; a sub-block with tau < beta holds an element whose private exponent is E - tau."""
+    x = synth.edge_case_values(4096, 11)
+    F, tau, q, s, Fe, te, y, nb = _fields(cfg, x)
+    f = ((x.view(np.uint32) >> 23) & 0xFF).astype(np.int64)
+    beta = (1 << cfg.d2) - 1
+    fb = f.reshape(-1, cfg.k1)
+    assert np.array_equal(F.ravel(), fb.max(axis=1))
+    fs = f.reshape(-1, cfg.k2).max(axis=1)
+    t = tau.ravel().astype(np.int64)
+    Fs = np.repeat(F.ravel().astype(np.int64), cfg.k1 // cfg.k2)
+    assert (t.reshape(-1, cfg.k1 // cfg.k2).min(axis=1) == 0).all()
+    assert np.array_equal(fs[t < beta], (Fs - t)[t < beta])
+    assert (fs[t == beta] <= (Fs - beta)[t == beta]).all()
+
+
+@pytest.mark.parametrize("cfg", SMALL_GRID, ids=str)
+def test_idempotence_values_and_bytes(cfg):
+    for x in (synth.laplace(1536, 3), synth.edge_case_values(1536, 4)):
+        y, _ = orc.quant_dequant(cfg, x)
+        y2, (e2, _) = orc.quant_dequant(cfg, y)
+        assert np.array_equal(y.view(np.uint32), y2.view(np.uint32)) and e2 == 0.0
+        for a, b in zip(orc.pack(cfg, x), orc.pack(cfg, y)):
+            assert np.array_equal(a, b)
+
+
+def test_powers_of_two_inside_the_window_are_exact():
+    for cfg in (orc.MX4, orc.MX6, orc.MX9, Cfg(32, 8, 4, 2, 3)):
+        for E in (-126, -20, 0, 100):
+            x = np.zeros(cfg.k1, dtype=np.float32)
+            x[0] = np.ldexp(1.5, E)                       # pins the shared exponent, tau_0 = 0
+            for t in range(E - cfg.m + 1, E + 1):
+                x[1] = np.ldexp(1.0, t)                   # same sub-block (k2 >= 2) -> tau = 0
+                y, _ = orc.quant_dequant(cfg, x)
+                assert y[1] == x[1], (cfg, E, t)
+            x[1] = np.ldexp(1.0, E - cfg.m - 1)           # below half a step: flushed to zero
+            assert orc.quant_dequant(cfg, x)[0][1] == 0.0
+
+
+@pytest.mark.parametrize("cfg", SMALL_GRID, ids=str)
+def test_power_of_two_scale_equivariance(cfg):
+    x = synth.student_t(2048, 9)
+    y, (e2, s2) = orc.quant_dequant(cfg, x)
+    for t in (-40, -3, 5, 60):
+        yt, (e2t, s2t) = orc.quant_dequant(cfg, np.ldexp(x, t))
+        assert np.array_equal(yt, np.ldexp(y, t))
+        assert orc.qsnr_db(e2t, s2t) == pytest.approx(orc.qsnr_db(e2, s2), abs=1e-9)
+
+
+def test_qsnr_monotone_in_m_and_six_db_per_bit():
+    x = synth.normal(1 << 16, 0)
+    for k1, k2, d2 in ((16, 2, 1), (16, 1, 0), (64, 8, 2), (8, 1, 1)):
+        q = [orc.qsnr(Cfg(k1, 8, k2, d2, m), x) for m in range(1, 9)]
+        assert all(b > a for a, b in zip(q, q[1:]))
+        steps = np.diff(q[2:])
+        assert np.all(np.abs(steps - 6.02) < 0.35), steps
+
+
+def test_d2_zero_is_plain_block_floating_point():
+    """d2 = 0 is conventional BFP: the result cannot depend on k2 and every element of a block
+    shares one step."""
+    x = synth.laplace(4096, 12)
+    base, _ = orc.quant_dequant(Cfg(16, 8, 1, 0, 5), x)
+    for k2 in (2, 4, 8, 16):
+        y, _ = orc.quant_dequant(Cfg(16, 8, k2, 0, 5), x)
+        assert np.array_equal(y.view(np.uint32), base.view(np.uint32))
+    blk = base.reshape(-1, 16).astype(np.float64)
+    E = np.floor(np.log2(np.abs(x.reshape(-1, 16)).max(axis=1)))
+    ratio = blk / np.ldexp(1.0, (E - 4).astype(int))[:, None]
+    assert np.array_equal(ratio, np.round(ratio))
+
+
+def test_scalar_case_matches_bf16_rounding_except_binade_carries():
+    """k1 = k2 = 1, d2 = 0, m = 8 is a scalar float with 8 significant bits, i.e. bf16 rounding
+    (a library routine here: torch's cast), except that BDR never bumps the exponent."""
+    import torch
+    x = synth.normal(1 << 16, 21)
+    y, _ = orc.quant_dequant(Cfg(1, 8, 1, 0, 8), x)
+    ref = torch.from_numpy(x).to(torch.bfloat16).to(torch.float32).numpy()
+    differs = y != ref
+    assert 0 < differs.mean() < 0.01
+    # where they differ, bf16 carried into the next binade and BDR clamped to the top code
+    assert np.array_equal(np.abs(ref[differs]), np.exp2(np.floor(np.log2(np.abs(x[differs]))) + 1))
+    assert np.array_equal(np.abs(y[differs]), np.abs(ref[differs]) * (1 - 2.0 ** -8))
+
+
+# ---- brute force against the explicit value set -----------------------------------------------------
+def _brute_block(cfg, xs):
+    """Nearest representable value by exact rational search over the explicit code set."""
+    def pexp(v):
+        v = abs(Fraction(float(v)))
+        if v < Fraction(1, 2 ** 126):
+            return -127
+        e = math.floor(math.log2(v))
+        while Fraction(2) ** e > v:
+            e -= 1
+        while Fraction(2) ** (e + 1) <= v:
+            e += 1
+        return e
+    E = max(pexp(v) for v in xs)
+    beta = 2 ** cfg.d2 - 1
+    out = []
+    for j in range(0, len(xs), cfg.k2):
+        sub = xs[j:j + cfg.k2]
+        tau = min(E - max(pexp(v) for v in sub), beta)
+        step = Fraction(2) ** (E - tau - cfg.m + 1)
+        for v in sub:
+            a = abs(Fraction(float(v)))
+            best = min(range(2 ** cfg.m), key=lambda q: (abs(q * step - a), q % 2 if cfg.rounding == 0 else -q))
+            out.append(float(best * step) * (-1.0 if math.copysign(1.0, float(v)) < 0 else 1.0))
+    return out
+
+
+@pytest.mark.parametrize("rounding", [orc.RNE, orc.RNA])
+def test_brute_force_all_bf16_values_in_a_few_binades(rounding):
+    # every bf16 value with exponent in [-3, 1] (plus zero), paired with fixed companions
+    mags = [0.0] + [(1 + k / 128.0) * 2.0 ** e for e in range(-3, 2) for k in range(128)]
+    comps = [0.0, 0.3, -1.0, 1.99, 0.06]
+    for m, d2, k1, k2 in ((1, 1, 2, 1), (2, 1, 2, 2), (3, 0, 2, 1), (3, 2, 4, 2), (2, 1, 4, 1)):
+        cfg = Cfg(k1, 8, k2, d2, m, orc.POW2, rounding)
+        blocks = []
+        for v in mags:
+            for c in comps:
+                blk = [v, c] + [0.25, -0.01][: k1 - 2]
+                blocks.append(blk)
+        x = np.array(blocks, dtype=np.float32)
+        y, _ = orc.quant_dequant(cfg, x)
+        ya, _ = orc.quant_dequant(cfg, x, alt=True)
+        assert np.array_equal(y.view(np.uint32), ya.view(np.uint32))
+        want = np.array([_brute_block(cfg, list(b)) for b in x], dtype=np.float32)
+        assert np.array_equal(y.view(np.uint32), want.view(np.uint32)), cfg
+
+
+def test_two_formulations_agree_everywhere():
+    for cfg in GRID[::3]:
+        for rounding in (orc.RNE, orc.RNA):
+            c = Cfg(cfg.k1, 8, cfg.k2, cfg.d2, cfg.m, orc.POW2, rounding)
+            for x in (synth.edge_case_values(2048, 31), synth.f32_to_bf16_bits(synth.normal(2048, 32))):
+                if x.dtype == np.uint16:
+                    x = synth.bf16_bits_to_f32(x)        # bf16-valued inputs: ties are common
+                a, _ = orc.quant_dequant(c, x)
+                b, _ = orc.quant_dequant(c, x, alt=True)
+                assert np.array_equal(a.view(np.uint32), b.view(np.uint32)), c
+
+
+# ---- layout, axes, tails ------------------------------------------------------------------------------
+@pytest.mark.parametrize("cfg", [orc.MX4, orc.MX6, orc.MX9, Cfg(8, 8, 4, 2, 3), Cfg(32, 8, 1, 3, 6), Cfg(16, 8, 16, 0, 7)], ids=str)
+def test_pack_unpack_round_trip(cfg):
+    x = synth.edge_case_values(5 * 200, 40).reshape(5, 200)        # 200 is not a multiple of 16 or 32
+    for axis in (0, 1):
+        y, _ = orc.quant_dequant(cfg, x, axis=axis)
+        planes = orc.pack(cfg, x, axis=axis)
+        back = orc.unpack(cfg, planes, 5, 200, axis=axis)
+        assert np.array_equal(back.view(np.uint32), y.view(np.uint32))
+        again = orc.pack(cfg, back, axis=axis)
+        for a, b in zip(planes, again):
+            assert np.array_equal(a, b)
+
+
+def test_column_direction_is_row_direction_of_the_transpose():
+    x = synth.normal_matrix(48, 80, 50)
+    for cfg in (orc.MX6, Cfg(32, 8, 8, 2, 3)):
+        y0, s0 = orc.quant_dequant(cfg, x, axis=0)
+        y1, s1 = orc.quant_dequant(cfg, np.ascontiguousarray(x.T), axis=1)
+        assert np.array_equal(y0, y1.T) and s0 == pytest.approx(s1, rel=1e-12)
+        for a, b in zip(orc.pack(cfg, x, axis=0), orc.pack(cfg, np.ascontiguousarray(x.T), axis=1)):
+            assert np.array_equal(a, b)
+
+
+def test_short_last_block_behaves_as_zero_padded():
+    x = synth.normal(100, 60)
+    for cfg in (orc.MX6, Cfg(64, 8, 8, 2, 5)):
+        pad = np.zeros(-(-100 // cfg.k1) * cfg.k1, dtype=np.float32)
+        pad[:100] = x
+        y, s = orc.quant_dequant(cfg, x)
+        yp, sp = orc.quant_dequant(cfg, pad)
+        assert np.array_equal(y, yp[:100]) and s == pytest.approx(sp, rel=1e-12)
+        for a, b in zip(orc.pack(cfg, x), orc.pack(cfg, pad)):
+            assert np.array_equal(a, b)
+
+
+def test_nonfinite_block_becomes_nan_block():
+    x = synth.normal(64, 61)
+    x[17] = np.inf
+    y, (e2, s2) = orc.quant_dequant(orc.MX6, x)
+    assert np.isnan(y[16:32]).all() and np.isfinite(y[:16]).all() and np.isfinite(y[32:]).all()
+    assert np.isnan(orc.qsnr_db(e2, s2))
+    exps, _, _ = orc.pack(orc.MX6, x)
+    assert exps[0, 1] == 0xFF
+    assert np.isnan(orc.unpack(orc.MX6, orc.pack(orc.MX6, x), 1, 64)[0, 16:32]).all()
+
+
+# ---- QSNR (Eq. 3) ---------------------------------------------------------------------------------------
+def test_qsnr_definition_closed_forms():
+    assert orc.qsnr_db(1.0, 100.0) == pytest.approx(20.0, abs=1e-12)
+    assert orc.qsnr_db(0.5, 0.5) == 0.0
+    assert math.isinf(orc.qsnr_db(0.0, 1.0)) and math.isnan(orc.qsnr_db(0.0, 0.0))
+    # an input made of representable values has infinite QSNR; sums are plain fp64 sums
+    x = np.array([1.0, 0.5, -0.25, 1.75] * 4, dtype=np.float32)
+    _, (e2, s2) = orc.quant_dequant(orc.MX6, x)
+    assert e2 == 0.0 and s2 == 4 * (1 + 0.25 + 0.0625 + 3.0625)
+    # one element off by exactly half a step: err^2 known in closed form
+    x = np.zeros(16, dtype=np.float32); x[0] = 1.0; x[1] = 1.0 + 1.0 / 16           # MX6 step at E=0 is 1/8
+    _, (e2, s2) = orc.quant_dequant(orc.MX6, x)
+    assert e2 == (1.0 / 16) ** 2 and s2 == 1.0 + (17.0 / 16) ** 2
+
+
+def test_soft_pins_from_the_pareto_discussion():
+    """Section IV-C quotes approximate QSNR gaps on X ~ N(0,|N(0,1)|); hold them to +-1 dB."""
+    x = synth.variable_variance_vectors(2048, 1024, seed=3)
+    q = lambda *a, **k: orc.qsnr(Cfg(*a, **k), x)
+    mx9, mx6, msfp16 = q(16, 8, 2, 1, 7), q(16, 8, 2, 1, 4), q(16, 8, 1, 0, 7)
+    assert abs((mx9 - msfp16) - 3.6) < 1.0
+    for m in (2, 4, 7):
+        assert abs((q(16, 8, 2, 2, m) - q(16, 8, 2, 1, m)) - 0.5) < 0.5
+        assert abs((q(16, 8, 2, 1, m) - q(16, 8, 8, 1, m)) - 2.0) < 1.0
+        assert abs((q(16, 8, 1, 1, m) - q(16, 8, 2, 1, m)) - 0.7) < 0.5
+    e4m3 = q(0, 32, 1, 4, 3, scale_kind=orc.FP32_FP)
+    e5m2 = q(0, 32, 1, 5, 2, scale_kind=orc.FP32_FP)
+    assert e5m2 < mx6 < e4m3
+    assert 13.0 < mx9 - e4m3 < 18.0
+
+
+# ---- comparator kinds --------------------------------------------------------------------------------------
+def test_fp8_casts_match_library_casts():
+    import torch
+    x = np.concatenate([synth.normal(20000, 70) * 30, synth.edge_case_values(4000, 71),
+                        np.array([0.0, -0.0, 448.0, 463.9, -448.0, 2 ** -9, 2 ** -10, 1.5 * 2 ** -10, 57344.0, 6e4,
+                                  2 ** -16, 2 ** -17, 3 * 2 ** -17], dtype=np.float32)]).astype(np.float32)
+    for (eb, mb, dt, lim) in ((4, 3, torch.float8_e4m3fn, 464.0), (5, 2, torch.float8_e5m2, 61440.0)):
+        xs = x[np.abs(x) < lim]
+        want = torch.from_numpy(xs).to(dt).to(torch.float32).numpy()
+        got = orc.minifloat_round(xs, eb, mb)
+        assert np.array_equal(got.view(np.uint32), want.view(np.uint32))
+    # saturation beyond the largest finite value
+    assert orc.minifloat_round(np.array([1e9, -1e9], dtype=np.float32), 4, 3).tolist() == [448.0, -448.0]
+    assert orc.minifloat_round(np.array([1e9], dtype=np.float32), 5, 2).tolist() == [57344.0]
+
+
+def test_fp8_kind_is_scale_then_cast():
+    import torch
+    x = synth.normal(4096, 72)
+    x[0] = 448.0                                       # amax = 448 -> s = 1 -> the kind is the bare cast
+    x = np.clip(x, -448, 448)
+    y, _ = orc.quant_dequant(Cfg(0, 32, 1, 4, 3, orc.FP32_FP), x)
+    want = torch.from_numpy(x).to(torch.float8_e4m3fn).to(torch.float32).numpy()
+    assert np.array_equal(y.view(np.uint32), want.view(np.uint32))
+    assert orc.bits_per_element(Cfg(0, 32, 1, 4, 3, orc.FP32_FP)) == 8.0
+
+
+def test_int_kind_reduces_to_integer_rounding_when_scale_is_one():
+    # Eq. 1: s = max/(2^(b-1)-1); with max = 127 (INT8) s = 1 and Eq. 2 is RoundToInt(x)
+    x = (synth.normal(4096, 73) * 40).clip(-127, 127).astype(np.float32)
+    x[0] = 127.0
+    y, _ = orc.quant_dequant(Cfg(0, 32, 1, 0, 7, orc.FP32_INT), x)
+    assert np.array_equal(y, np.rint(x))
+    # and is scale-equivariant under powers of two (s scales exactly)
+    y2, _ = orc.quant_dequant(Cfg(0, 32, 1, 0, 7, orc.FP32_INT), x * np.float32(2.0 ** -9))
+    assert np.array_equal(y2, y * np.float32(2.0 ** -9))
+    # INT4: values are multiples of max/7
+    x4 = synth.normal(1024, 74)
+    y4, _ = orc.quant_dequant(Cfg(0, 32, 1, 0, 3, orc.FP32_INT), x4)
+    k = y4 / (np.abs(x4).max() / np.float32(7))
+    assert np.allclose(k, np.round(k), atol=1e-5) and np.abs(k).max() <= 7 + 1e-5
+
+
+def test_vsq_reductions():
+    # all 16-vectors share the same maximum -> every integer sub-scale is 2^d2-1 -> per-tensor INT
+    x = synth.normal(2048, 75).reshape(-1, 16)
+    x = (x / np.abs(x).max(axis=1, keepdims=True)).astype(np.float32)
+    x[:, 0] = 1.0
+    x = x.ravel()
+    for m in (3, 7):
+        yv, _ = orc.quant_dequant(Cfg(0, 32, 16, 8, m, orc.FP32_VSQ), x)
+        yi, _ = orc.quant_dequant(Cfg(0, 32, 1, 0, m, orc.FP32_INT), x)
+        assert np.allclose(yv, yi, rtol=3e-7, atol=0)
+    # a finer sub-scale can only help on data with varied per-vector maxima
+    x = synth.variable_variance_vectors(256, 16, 76).ravel()
+    qs = [orc.qsnr(Cfg(0, 32, 16, d2, 3, orc.FP32_VSQ), x) for d2 in (4, 6, 8, 10)]
+    assert qs[-1] > orc.qsnr(Cfg(0, 32, 1, 0, 3, orc.FP32_INT), x)
+    assert qs == sorted(qs) or max(qs) - min(qs) < 1.0
+
+
+# ---- GEMM reference ---------------------------------------------------------------------------------------------
+def test_gemm_reference_is_the_plain_definition():
+    rng = np.random.default_rng(80)
+    a = rng.integers(-8, 9, (7, 33)).astype(np.float32)
+    b = rng.integers(-8, 9, (5, 33)).astype(np.float32)
+    c = orc.gemm_nt_f64(a, b)
+    assert np.array_equal(c, (a.astype(np.int64) @ b.astype(np.int64).T).astype(np.float64))
+    assert np.array_equal(orc.gemm_nt_f64(a, b, nthreads=3), c)
+    ri, ci = np.array([0, 6, 3]), np.array([4, 0, 2])
+    assert np.array_equal(orc.gemm_nt_f64_sampled(a, b, ri, ci), c[ri, ci])
+
+
+def test_multithreaded_oracle_is_the_same_function():
+    x = synth.normal_matrix(64, 256, 81)
+    for axis in (0, 1):
+        a, sa = orc.quant_dequant(orc.MX6, x, axis=axis)
+        b, sb = orc.quant_dequant(orc.MX6, x, axis=axis, nthreads=4)
+        assert np.array_equal(a, b) and sa == sb
