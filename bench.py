@@ -1,0 +1,368 @@
+#!/usr/bin/env python
+"""Benchmark of the BDR/MX hot path on B200.
+
+One "step" = one pass of the whole quantization path over one 8192 x 8192 bf16 activation tensor
+(Laplace(0,1), 1% outlier columns x50): for each of MX4 / MX6 / MX9 and each direction (row-wise,
+column-wise) a quantize-dequantize with fused QSNR sums, a quantize+pack with fused QSNR sums, and
+an unpack+dequantize -- 18 kernel launches.  `value` is the algorithmic bytes those 18 operations
+must move divided by the device time (GB/s); the MX-GEMM and design-sweep legs are measured
+separately after the timed steps and reported in the same JSON line.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+ROWS, COLS = 8192, 8192
+FORMATS = (("MX4", 2), ("MX6", 4), ("MX9", 7))  # name, m  (k1=16, d1=8, k2=2, d2=1: Table II)
+METRIC = "MX quant-dequant GB/s"
+FALLBACK_HBM_GBS = 6650.0
+
+# dram__bytes_read.sum + dram__bytes_write.sum per launch from the committed ncu captures
+# (profiles/*.md), scaled to the 8192 x 8192 launch; None where no capture exists yet.
+NCU_TRAFFIC_BYTES: dict[str, float | None] = {}
+
+
+def bits_per_element(m: int) -> float:
+    return (m + 1) + 8 / 16 + 1 / 2
+
+
+def op_bytes(op: str, m: int, n_elems: int) -> float:
+    """Algorithmic bytes of one operation on bf16 data: what the method itself must move."""
+    packed = bits_per_element(m) / 8.0
+    per_elem = {"quant_dequant": 2.0 + 2.0, "pack": 2.0 + packed, "unpack": packed + 2.0}[op]
+    return per_elem * n_elems
+
+
+def step_bytes(n_elems: int) -> float:
+    return sum(op_bytes(op, m, n_elems) for _, m in FORMATS for _axis in (1, 0) for op in ("quant_dequant", "pack", "unpack"))
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            d = json.load(f)
+        return float(d["hbm_gbs"]), "measured", d
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback", {}
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.proc = None
+        self.lines: list[str] = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.gpu), "--query-gpu=" + self.QUERY,
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._pump, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _pump(self):
+        for ln in self.proc.stdout:
+            self.lines.append(ln.strip())
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, smax, reasons = [], [], set()
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        for ln in self.lines:
+            f = [t.strip() for t in ln.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1]))
+                smax.append(float(f[2]))
+            except ValueError:
+                continue
+            for name, val in zip(names, f[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        return {"sm_mhz": float(np.median(sm)), "sm_max_mhz": float(max(smax)), "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+# ---------------------------------------------------------------------------------------------------
+# CPU baseline: the oracle as it stands, on a bounded sample of the same workload
+# ---------------------------------------------------------------------------------------------------
+def oracle_step(x_f32: np.ndarray, nthreads: int) -> float:
+    """Runs the step's 18 operations with the oracle on x_f32 (rows split over threads for axis 1,
+    columns for axis 0; ctypes releases the GIL).  Returns seconds."""
+    from concurrent.futures import ThreadPoolExecutor
+    from oracle import oracle as orc
+
+    rows, cols = x_f32.shape
+
+    def one(cfg, axis, part):
+        xs = np.ascontiguousarray(x_f32[part, :] if axis == 1 else x_f32[:, part])
+        r, c = xs.shape
+        orc.quant_dequant(cfg, xs, axis=axis)
+        planes = orc.pack(cfg, xs, axis=axis)
+        orc.unpack(cfg, planes, r, c, axis=axis)
+
+    t0 = time.perf_counter()
+    with ThreadPoolExecutor(max_workers=nthreads) as ex:
+        for _, m in FORMATS:
+            cfg = orc.Config(16, 8, 2, 1, m)
+            for axis in (1, 0):
+                n = rows if axis == 1 else cols
+                chunk = -(-n // nthreads)
+                chunk = -(-chunk // 16) * 16
+                parts = [slice(i, min(n, i + chunk)) for i in range(0, n, chunk)]
+                list(ex.map(lambda p: one(cfg, axis, p), parts))
+    return time.perf_counter() - t0
+
+
+def cpu_sample(x_bits: np.ndarray, sample_rows: int) -> np.ndarray:
+    from paper_2302_08007_b200 import synth
+    return synth.bf16_bits_to_f32(x_bits[:sample_rows]).reshape(sample_rows, -1)
+
+
+def run_reference(args):
+    """--impl reference: the oracle on the host cores, each step a bounded sample of the workload."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import oracle as orc
+    from paper_2302_08007_b200 import synth
+    orc.build()
+    cores = len(os.sched_getaffinity(0))
+    sample_rows = 1024
+    x = synth.outlier_channel_matrix(sample_rows, COLS, seed=0, stream=3, frac=0.01, gain=50.0)
+    xs = synth.bf16_bits_to_f32(synth.f32_to_bf16_bits(x)).reshape(sample_rows, COLS)
+    for _ in range(args.warmup):
+        oracle_step(xs, cores)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle_step(xs, cores)
+    dt = time.perf_counter() - t0
+    gbs = step_bytes(xs.size) * args.steps / dt / 1e9
+    sample = "%d x %d slice of the 8192 x 8192 tensor per step, all 18 operations" % (sample_rows, COLS)
+    line = {"impl": "reference", "metric": METRIC, "value": gbs, "unit": "GB/s", "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": "C3: 8192x8192 bf16 Laplace(0,1), 1% outlier columns x50; MX4/MX6/MX9 x row/column x "
+                                   "(quant-dequant, pack, unpack); CPU oracle on a bounded sample"},
+            "cpu_baseline": {"value": gbs, "unit": "GB/s", "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": gbs, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+# ---------------------------------------------------------------------------------------------------
+# GPU arm
+# ---------------------------------------------------------------------------------------------------
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2302_08007_b200 import binding as bdr
+    from paper_2302_08007_b200 import synth
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    bdr.lib()  # fail loudly if the CUDA library is missing
+
+    # every rank quantizes its own tensor (independent replicas of the path: no data-path collective)
+    x_host = synth.outlier_channel_matrix(ROWS, COLS, seed=rank, stream=3, frac=0.01, gain=50.0)
+    x_bits = synth.f32_to_bf16_bits(x_host)
+    del x_host
+    x_pinned = torch.from_numpy(x_bits.view(np.int16)).view(torch.bfloat16).pin_memory()
+    x = x_pinned.cuda()
+    n_elems = x.numel()
+
+    cfgs = {name: bdr.Config(16, 8, 2, 1, m) for name, m in FORMATS}
+    y = torch.empty_like(x)
+    planes = {(name, axis): bdr.alloc_planes(cfgs[name], ROWS, COLS, axis) for name, _ in FORMATS for axis in (1, 0)}
+    ops = [(name, m, axis, op) for name, m in FORMATS for axis in (1, 0) for op in ("quant_dequant", "pack", "unpack")]
+    sums = torch.zeros((len(ops), 2), dtype=torch.float64, device="cuda")
+    sums_host = torch.empty((len(ops), 2), dtype=torch.float64).pin_memory()
+
+    def run_op(i, name, axis, op):
+        if op == "quant_dequant":
+            bdr.bdr_quant_dequant(cfgs[name], x, y, axis=axis, qsnr_sums=sums[i])
+        elif op == "pack":
+            bdr.bdr_pack(cfgs[name], x, planes[(name, axis)], axis=axis, qsnr_sums=sums[i])
+        else:
+            bdr.bdr_unpack(cfgs[name], planes[(name, axis)], y, axis=axis)
+
+    def step():
+        for i, (name, _m, axis, op) in enumerate(ops):
+            run_op(i, name, axis, op)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        step()
+    barrier()
+
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.3)
+    sums.zero_()
+    barrier()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record()
+    for _ in range(args.steps):
+        step()
+    ev1.record()
+    barrier()
+    ms = ev0.elapsed_time(ev1)
+    clocks = sampler.stop() if rank == 0 else {}
+    if world > 1:
+        t = torch.tensor([ms], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    ms_per_step = ms / args.steps
+    value = step_bytes(n_elems) * world / (ms_per_step * 1e-3) / 1e9
+    qsnr = {}
+    sums_np = (sums / args.steps).cpu().numpy()
+    for i, (name, _m, axis, op) in enumerate(ops):
+        if op == "pack":
+            qsnr["%s_axis%d" % (name, axis)] = float(-10.0 * np.log10(sums_np[i, 0] / sums_np[i, 1]))
+
+    # ---- per-kernel timing on the launching stream (roofline of the dominant kernel) ----
+    kernels = {}
+    reps = max(5, args.steps)
+    for i, (name, m, axis, op) in enumerate(ops):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        run_op(i, name, axis, op)
+        torch.cuda.synchronize()
+        a.record()
+        for _ in range(reps):
+            run_op(i, name, axis, op)
+        b.record()
+        torch.cuda.synchronize()
+        dur_ms = a.elapsed_time(b) / reps
+        key = "%s_%s_%s" % (op, name, "row" if axis == 1 else "col")
+        kernels[key] = {"ms": dur_ms, "GBps": op_bytes(op, m, n_elems) / (dur_ms * 1e-3) / 1e9}
+    peak, peak_kind, _ = measured_peaks()
+    dom = max(kernels, key=lambda k: kernels[k]["ms"])
+    for k in kernels.values():
+        k["frac"] = k["GBps"] / peak
+    roofline = {"bound": "hbm", "kernel": dom, "achieved": kernels[dom]["GBps"], "peak": peak, "unit": "GB/s",
+                "frac": kernels[dom]["GBps"] / peak, "peak_source": peak_kind,
+                "traffic": NCU_TRAFFIC_BYTES.get(dom)}
+
+    # ---- end to end through the C ABI with host buffers: H2D of the step's input, D2H of its result ----
+    e2e_steps = max(1, min(args.steps, 5))
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(e2e_steps):
+        x.copy_(x_pinned, non_blocking=True)
+        step()
+        sums_host.copy_(sums, non_blocking=True)
+    e1.record()
+    barrier()
+    e2e_ms = e0.elapsed_time(e1)
+    if world > 1:
+        t = torch.tensor([e2e_ms], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_ms = float(t.item())
+    e2e = {"value": step_bytes(n_elems) * world / (e2e_ms / e2e_steps * 1e-3) / 1e9, "unit": "GB/s",
+           "h2d_bytes_per_step": x.numel() * x.element_size(), "d2h_bytes_per_step": sums.numel() * 8,
+           "steps": e2e_steps}
+
+    extra = {}
+    if rank == 0:
+        extra = secondary_legs(args, bdr, synth, torch)
+
+    cpu_baseline = None
+    if rank == 0 and world == 1:
+        from oracle import oracle as orc
+        orc.build()
+        cores = len(os.sched_getaffinity(0))
+        sample_rows = 4096
+        xs = cpu_sample(x_bits, sample_rows)
+        sec = oracle_step(xs, cores)
+        cpu_baseline = {"value": step_bytes(xs.size) / sec / 1e9, "unit": "GB/s", "cores": cores, "kind": "oracle",
+                        "sample": "first %d of %d rows, all 18 operations once (%.1f s)" % (sample_rows, ROWS, sec)}
+
+    if rank == 0:
+        line = {"metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
+                "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+                "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+                "config": {"workload": "C3: 8192x8192 bf16 Laplace(0,1), 1% outlier columns x50; MX4/MX6/MX9 x "
+                                       "row/column x (quant-dequant+QSNR, pack+QSNR, unpack)",
+                           "l2": "inputs larger than L2 (134 MB tensor, >=168 MB streamed per launch)",
+                           "replicas": "independent tensor per rank, no collective"},
+                "frac_of_hbm_peak": value / world / peak, "roofline": roofline, "kernels": kernels,
+                "cpu_baseline": cpu_baseline, "e2e": e2e, "gpu_launches": len(ops) * args.steps, "clocks": clocks,
+                "qsnr_db": qsnr}
+        line.update(extra)
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def secondary_legs(args, bdr, synth, torch) -> dict:
+    """MX-GEMM TFLOP/s and design-sweep configs/s, when those entry points are built."""
+    out = {}
+    try:
+        from paper_2302_08007_b200 import legs
+    except ImportError:
+        return out
+    for fn in (legs.gemm_leg, legs.sweep_leg):
+        try:
+            out.update(fn(args))
+        except bdr.BdrError as e:
+            out[fn.__name__] = {"unavailable": str(e)}
+    return out
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,137 @@
+/*
+ * bdr.h -- C ABI of the B200 (sm_100a) Block Data Representations / shared-microexponent library.
+ *
+ * Every entry point takes plain pointers and sizes.  Unless a parameter says "host", a pointer is
+ * a DEVICE pointer to memory that the caller allocated and keeps alive until the work queued on
+ * `stream` has finished.  The library allocates no device memory, never synchronises a stream and
+ * leaves every result on the device.  `stream` is a cudaStream_t passed as void* (NULL = the
+ * legacy default stream).  Return value: BDR_OK (0) or a negative bdr_status_t; all argument
+ * validation happens on the host before anything is launched, so a failing call has queued no work
+ * (BDR_ERR_CUDA reports a failed launch).
+ *
+ * Layout conventions
+ *   A tensor is a row-major 2-D array [rows, cols] with a row pitch of `ld` ELEMENTS (ld >= cols).
+ *   `axis` is the quantization (= reduction) direction: axis 1 = along the contiguous dimension
+ *   ("row-wise"), axis 0 = along the strided dimension ("column-wise").  A "line" is one row
+ *   (axis 1) or one column (axis 0); lines are cut into ceil(len/k1) blocks of k1 consecutive
+ *   elements; a short last block behaves as if it were zero padded.  Blocks never span lines.
+ *
+ * Packed layout (three planes per tensor, line-major: line l starts at plane + l*ld_plane bytes)
+ *   exps  : one byte per block, the biased shared exponent F (0xFF marks a block that held Inf/NaN)
+ *   micro : little-endian, LSB-first stream of d2-bit fields, field j = shift tau of sub-block j of
+ *           the line (empty when d2 = 0)
+ *   elems : little-endian, LSB-first stream of (m+1)-bit codes, code i = (sign << m) | magnitude of
+ *           element i of the line; positions of the zero padding hold code 0
+ *   This spends exactly (m+1) + d1/k1 + d2/k2 bits per element (Section III) whenever a line needs
+ *   no padding.  For axis 0 the planes are laid out column by column, i.e. they are byte-identical
+ *   to the axis-1 planes of the transposed tensor (the "transpose, then quantize" copy that the
+ *   backward pass needs, Section V).
+ */
+#ifndef BDR_H_
+#define BDR_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* How the two scale levels are encoded (Section III, Table I). */
+typedef enum {
+    BDR_SCALE_POW2 = 0,     /* MX / BFP / MSFP: block scale 2^E (d1 = 8 bits), sub-block scale 2^-tau */
+    BDR_SCALE_FP32_INT = 1, /* INT: FP32 scale from the maximum (Section II, Eq. 1-2); m = bits - 1   */
+    BDR_SCALE_FP32_FP = 2,  /* FP8-like: FP32 scale + per-element d2-bit exponent, m explicit bits    */
+    BDR_SCALE_FP32_VSQ = 3  /* VSQ: FP32 scale + unsigned d2-bit integer sub-scale per k2 elements    */
+} bdr_scale_kind_t;
+
+typedef enum { BDR_ROUND_NEAREST_EVEN = 0, BDR_ROUND_NEAREST_AWAY = 1 } bdr_rounding_t;
+typedef enum { BDR_F32 = 0, BDR_BF16 = 1 } bdr_dtype_t;
+
+/* The BDR parameter tuple of Section III (k1, d1, k2, d2, m) plus scale kind and tie rule.
+ * POW2 kind: d1 must be 8, k2 divides k1, 0 <= d2 <= 3, 1 <= m <= 8; the CUDA kernels additionally
+ * need k1 and k2 to be powers of two with k1 <= 1024 (else BDR_ERR_UNSUPPORTED).
+ * FP32_* kinds are accepted by bdr_qsnr only, with k1 = 0 meaning one scale for the whole tensor. */
+typedef struct {
+    int32_t k1, d1, k2, d2, m, scale_kind, rounding;
+} bdr_config_t;
+
+/* Device pointers to the three packed planes and their line pitches in bytes.  Pitches must be
+ * multiples of 16 and plane bases 16-byte aligned.  `micro` may be NULL when d2 = 0. */
+typedef struct {
+    uint8_t *exps, *micro, *elems;
+    int64_t ld_exps, ld_micro, ld_elems;
+} bdr_planes_t;
+
+typedef enum {
+    BDR_OK = 0,
+    BDR_ERR_NULL = -1,        /* a required pointer is NULL                                          */
+    BDR_ERR_BAD_CONFIG = -2,  /* parameter tuple outside the definition (k2 does not divide k1, ...)  */
+    BDR_ERR_UNSUPPORTED = -3, /* valid, but no kernel for it (non power-of-two k1, FP32 kind in pack) */
+    BDR_ERR_MISALIGNED = -4,  /* pointer or pitch breaks a stated alignment rule                      */
+    BDR_ERR_SIZE = -5,        /* negative size, ld < cols, size over the stated maximum               */
+    BDR_ERR_WORKSPACE = -6,   /* workspace missing or too small                                       */
+    BDR_ERR_CUDA = -7,        /* a CUDA call or kernel launch failed                                  */
+    BDR_ERR_TIMEOUT = -8      /* a bounded device-side wait ran out (reported by mx_gemm_status)      */
+} bdr_status_t;
+
+/* Text for a status code (host; never NULL). */
+const char* bdr_strerror(int status);
+
+/* Section III bits-per-element formula realised as plane sizes (host only).  ld_out / bytes_out
+ * (host arrays of 3: exps, micro, elems) receive the default line pitches (rounded up to 16 bytes)
+ * and total plane sizes for a [rows, cols] tensor quantized along `axis`. */
+int bdr_packed_sizes(const bdr_config_t* cfg /*host*/, int64_t rows, int64_t cols, int axis,
+                     int64_t ld_out[3] /*host*/, int64_t bytes_out[3] /*host*/);
+
+/* Q(x): quantize to the format and write the dequantized values back in the input's dtype and
+ * layout (Appendix: shared exponent = private exponent of the block's largest element; sub-block
+ * shift tau <= 2^d2-1; m-digit magnitude rounded to nearest, clamped at 2^m-1).
+ *   x, y          [rows, ld] of `dt`; y may alias x; y may be NULL when only the sums are wanted
+ *   qsnr_sums_dev NULL, or 2 doubles that this call ADDS {sum (Q(x)-x)^2, sum x^2} to (Eq. 3);
+ *                 the caller zeroes them
+ * POW2 kind only.  Fast path: axis 1, 16-byte aligned x/y, ld*sizeof(dt) and cols multiples of
+ * what a 16-element slice needs; anything else runs a slower general kernel with the same result. */
+int bdr_quant_dequant(const bdr_config_t* cfg /*host*/, const void* x, void* y, bdr_dtype_t dt,
+                      int64_t rows, int64_t cols, int64_t ld, int axis, double* qsnr_sums_dev,
+                      void* stream);
+
+/* Quantize and write the packed planes (layout above); optionally also the dequantized tensor
+ * (y_dq, same dtype/pitch as x, may be NULL) and the Eq. 3 sums.  Every byte of every plane line
+ * up to its pitch is written (padding bytes are zero). */
+int bdr_pack(const bdr_config_t* cfg /*host*/, const void* x, bdr_dtype_t dt, int64_t rows, int64_t cols,
+             int64_t ld, int axis, const bdr_planes_t* out /*host struct of device pointers*/, void* y_dq,
+             double* qsnr_sums_dev, void* stream);
+
+/* Decode packed planes to values (-1)^s * q * 2^(F-127-tau-(m-1)) of dtype `dt` in a [rows, ld]
+ * tensor; the inverse of bdr_pack's planes -> Q(x). */
+int bdr_unpack(const bdr_config_t* cfg /*host*/, const bdr_planes_t* in /*host struct*/, void* y, bdr_dtype_t dt,
+               int64_t rows, int64_t cols, int64_t ld, int axis, void* stream);
+
+/* Bytes of device scratch that bdr_qsnr needs for n_cfgs configurations (host only). */
+int64_t bdr_qsnr_workspace_bytes(int n_cfgs);
+
+/* The design-space sweep of Section IV: QSNR (Eq. 3, in dB, ratio of whole-tensor sums) of one
+ * tensor under n_cfgs configurations, reading the tensor once per group of configurations.
+ *   cfgs         host array; POW2 entries as above; FP32_INT / FP32_FP (d2 = 4,m = 3 or d2 = 5,m = 2)
+ *                / FP32_VSQ entries need k1 = 0 (per-tensor FP32 scale from the current amax)
+ *   qsnr_db_dev  n_cfgs doubles, written (not accumulated)
+ *   workspace    device scratch of at least bdr_qsnr_workspace_bytes(n_cfgs) bytes, 16-byte aligned;
+ *                contents are overwritten
+ * axis 1 only for n_cfgs > 1. */
+int bdr_qsnr(const bdr_config_t* cfgs /*host*/, int n_cfgs, const void* x, bdr_dtype_t dt, int64_t rows,
+             int64_t cols, int64_t ld, int axis, double* qsnr_db_dev, void* workspace, int64_t workspace_bytes,
+             void* stream);
+
+/* C[M,N] (fp32, row pitch ldc elements) = deq(A)[M,K] * deq(B)[N,K]^T with both operands given as
+ * packed planes quantized along K (axis 1 planes of A and of B), decoded to bf16 inside the kernel
+ * and accumulated in fp32 on the tensor cores (Section V: both inputs of a tensor operation are
+ * MX-quantized along the reduction dimension).
+ * Needs k1 = 16, k2 = 2, d2 = 1, m <= 7 for both operands, K a multiple of 64. */
+int mx_gemm(const bdr_config_t* cfg_a /*host*/, const bdr_planes_t* a /*host struct*/,
+            const bdr_config_t* cfg_b /*host*/, const bdr_planes_t* b /*host struct*/, int64_t M, int64_t N,
+            int64_t K, float* c, int64_t ldc, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* BDR_H_ */

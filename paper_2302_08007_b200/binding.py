@@ -1,0 +1,210 @@
+"""Thin ctypes binding over the C ABI declared in ``include/bdr.h``.
+
+Argument marshalling only: torch tensors provide device memory and streams, every step of the
+method runs inside the CUDA library.  There is no CPU fallback: if the library is missing, loading
+raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from dataclasses import dataclass
+
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libbdr_b200.so")
+
+SCALE_POW2, SCALE_FP32_INT, SCALE_FP32_FP, SCALE_FP32_VSQ = 0, 1, 2, 3
+ROUND_NEAREST_EVEN, ROUND_NEAREST_AWAY = 0, 1
+F32, BF16 = 0, 1
+
+EXPORTS = ("bdr_strerror", "bdr_packed_sizes", "bdr_quant_dequant", "bdr_pack", "bdr_unpack",
+           "bdr_qsnr_workspace_bytes", "bdr_qsnr", "mx_gemm")
+
+
+class BdrError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__("%s failed: %s (status %d)" % (where, strerror(status), status))
+
+
+class _Config(C.Structure):
+    _fields_ = [(n, C.c_int32) for n in ("k1", "d1", "k2", "d2", "m", "scale_kind", "rounding")]
+
+
+class _Planes(C.Structure):
+    _fields_ = [("exps", C.c_void_p), ("micro", C.c_void_p), ("elems", C.c_void_p),
+                ("ld_exps", C.c_int64), ("ld_micro", C.c_int64), ("ld_elems", C.c_int64)]
+
+
+@dataclass(frozen=True)
+class Config:
+    """bdr_config_t: the (k1, d1, k2, d2, m) tuple of Section III plus scale kind and tie rule."""
+    k1: int
+    d1: int
+    k2: int
+    d2: int
+    m: int
+    scale_kind: int = SCALE_POW2
+    rounding: int = ROUND_NEAREST_EVEN
+
+    def c(self) -> _Config:
+        return _Config(self.k1, self.d1, self.k2, self.d2, self.m, self.scale_kind, self.rounding)
+
+
+MX9 = Config(16, 8, 2, 1, 7)
+MX6 = Config(16, 8, 2, 1, 4)
+MX4 = Config(16, 8, 2, 1, 2)
+
+
+@dataclass
+class Planes:
+    """Device tensors (uint8, [nlines, ld]) holding the three packed planes."""
+    exps: torch.Tensor
+    micro: torch.Tensor
+    elems: torch.Tensor
+
+    def c(self) -> _Planes:
+        return _Planes(self.exps.data_ptr(), self.micro.data_ptr() if self.micro.numel() else None,
+                       self.elems.data_ptr(), self.exps.stride(0), self.micro.stride(0) if self.micro.numel() else 0,
+                       self.elems.stride(0))
+
+
+_lib = None
+
+
+def lib():
+    """Load the CUDA library; raises if it has not been built (there is no fallback)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError("CUDA library %s is missing: run paper_2302_08007_b200/build.py "
+                              "(or __graft_entry__.build())" % LIB_PATH)
+        L = C.CDLL(LIB_PATH)
+        L.bdr_strerror.restype = C.c_char_p
+        L.bdr_strerror.argtypes = [C.c_int]
+        L.bdr_packed_sizes.argtypes = [C.c_void_p, C.c_int64, C.c_int64, C.c_int, C.c_void_p, C.c_void_p]
+        L.bdr_quant_dequant.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int64, C.c_int64, C.c_int64,
+                                        C.c_int, C.c_void_p, C.c_void_p]
+        L.bdr_pack.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int64, C.c_int64, C.c_int64, C.c_int, C.c_void_p,
+                               C.c_void_p, C.c_void_p, C.c_void_p]
+        L.bdr_unpack.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int64, C.c_int64, C.c_int64, C.c_int,
+                                 C.c_void_p]
+        L.bdr_qsnr_workspace_bytes.restype = C.c_int64
+        L.bdr_qsnr_workspace_bytes.argtypes = [C.c_int]
+        L.bdr_qsnr.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_int, C.c_int64, C.c_int64, C.c_int64, C.c_int,
+                               C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p]
+        L.mx_gemm.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_int64, C.c_int64,
+                              C.c_void_p, C.c_int64, C.c_void_p]
+        for fn in (L.bdr_packed_sizes, L.bdr_quant_dequant, L.bdr_pack, L.bdr_unpack, L.bdr_qsnr, L.mx_gemm):
+            fn.restype = C.c_int
+        _lib = L
+    return _lib
+
+
+def strerror(status: int) -> str:
+    return lib().bdr_strerror(int(status)).decode()
+
+
+def _check(status: int, where: str):
+    if status != 0:
+        raise BdrError(status, where)
+
+
+def _dt(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return F32
+    if t.dtype == torch.bfloat16:
+        return BF16
+    raise TypeError("tensor dtype must be float32 or bfloat16")
+
+
+def _stream(stream) -> C.c_void_p:
+    s = stream if stream is not None else torch.cuda.current_stream()
+    return C.c_void_p(s.cuda_stream)
+
+
+def _as2d(t: torch.Tensor):
+    if t.dim() == 1:
+        t = t.unsqueeze(0)
+    if t.dim() != 2 or t.stride(1) != 1:
+        raise ValueError("expected a 1-D or row-major 2-D tensor")
+    return t
+
+
+def _ptr(t):
+    return C.c_void_p(t.data_ptr()) if t is not None else None
+
+
+def bdr_packed_sizes(cfg: Config, rows: int, cols: int, axis: int = 1):
+    """Default line pitches and plane sizes in bytes: ([ld_exps, ld_micro, ld_elems], [bytes...])."""
+    ld = (C.c_int64 * 3)()
+    nb = (C.c_int64 * 3)()
+    c = cfg.c()
+    _check(lib().bdr_packed_sizes(C.addressof(c), rows, cols, axis, C.addressof(ld), C.addressof(nb)),
+           "bdr_packed_sizes")
+    return list(ld), list(nb)
+
+
+def alloc_planes(cfg: Config, rows: int, cols: int, axis: int = 1, device="cuda") -> Planes:
+    ld, _ = bdr_packed_sizes(cfg, rows, cols, axis)
+    nlines = rows if axis == 1 else cols
+    mk = lambda l: torch.empty((nlines, l), dtype=torch.uint8, device=device)
+    return Planes(mk(ld[0]), mk(ld[1]), mk(ld[2]))
+
+
+def bdr_quant_dequant(cfg: Config, x: torch.Tensor, y: torch.Tensor | None = None, axis: int = 1,
+                      qsnr_sums: torch.Tensor | None = None, stream=None) -> torch.Tensor | None:
+    """Q(x) into ``y`` (same dtype/shape/pitch as x; may be x itself).  ``qsnr_sums`` (2 float64 on
+    the device) is accumulated into."""
+    x2 = _as2d(x)
+    y2 = _as2d(y) if y is not None else None
+    if y2 is not None and (y2.shape != x2.shape or y2.stride(0) != x2.stride(0) or y2.dtype != x2.dtype):
+        raise ValueError("y must match x in shape, pitch and dtype")
+    c = cfg.c()
+    _check(lib().bdr_quant_dequant(C.addressof(c), _ptr(x2), _ptr(y2), _dt(x2), x2.shape[0], x2.shape[1], x2.stride(0),
+                                   axis, _ptr(qsnr_sums), _stream(stream)), "bdr_quant_dequant")
+    return y
+
+
+def bdr_pack(cfg: Config, x: torch.Tensor, planes: Planes, axis: int = 1, y_dq: torch.Tensor | None = None,
+             qsnr_sums: torch.Tensor | None = None, stream=None) -> Planes:
+    x2 = _as2d(x)
+    y2 = _as2d(y_dq) if y_dq is not None else None
+    if y2 is not None and (y2.shape != x2.shape or y2.stride(0) != x2.stride(0) or y2.dtype != x2.dtype):
+        raise ValueError("y_dq must match x in shape, pitch and dtype")
+    c, p = cfg.c(), planes.c()
+    _check(lib().bdr_pack(C.addressof(c), _ptr(x2), _dt(x2), x2.shape[0], x2.shape[1], x2.stride(0), axis,
+                          C.addressof(p), _ptr(y2), _ptr(qsnr_sums), _stream(stream)), "bdr_pack")
+    return planes
+
+
+def bdr_unpack(cfg: Config, planes: Planes, y: torch.Tensor, axis: int = 1, stream=None) -> torch.Tensor:
+    y2 = _as2d(y)
+    c, p = cfg.c(), planes.c()
+    _check(lib().bdr_unpack(C.addressof(c), C.addressof(p), _ptr(y2), _dt(y2), y2.shape[0], y2.shape[1], y2.stride(0),
+                            axis, _stream(stream)), "bdr_unpack")
+    return y
+
+
+def bdr_qsnr_workspace_bytes(n_cfgs: int) -> int:
+    return int(lib().bdr_qsnr_workspace_bytes(int(n_cfgs)))
+
+
+def bdr_qsnr(cfgs, x: torch.Tensor, out_db: torch.Tensor, workspace: torch.Tensor, axis: int = 1, stream=None):
+    """QSNR in dB of x under every configuration of ``cfgs`` into out_db (float64, len(cfgs))."""
+    x2 = _as2d(x)
+    arr = (_Config * len(cfgs))(*[c.c() for c in cfgs])
+    _check(lib().bdr_qsnr(C.addressof(arr), len(cfgs), _ptr(x2), _dt(x2), x2.shape[0], x2.shape[1], x2.stride(0), axis,
+                          _ptr(out_db), _ptr(workspace), workspace.numel() * workspace.element_size(),
+                          _stream(stream)), "bdr_qsnr")
+    return out_db
+
+
+def mx_gemm(cfg_a: Config, a: Planes, cfg_b: Config, b: Planes, M: int, N: int, K: int, c: torch.Tensor, stream=None):
+    """c[M,N] (float32) = deq(a)[M,K] @ deq(b)[N,K]^T from packed operands quantized along K."""
+    ca, cb, pa, pb = cfg_a.c(), cfg_b.c(), a.c(), b.c()
+    _check(lib().mx_gemm(C.addressof(ca), C.addressof(pa), C.addressof(cb), C.addressof(pb), M, N, K, _ptr(c),
+                         c.stride(0), _stream(stream)), "mx_gemm")
+    return c

@@ -1,0 +1,188 @@
+// C-ABI entry points: argument validation on the host, then dispatch to the kernels.
+#include <mutex>
+
+#include "bdr_device.cuh"
+#include "bdr_host.h"
+
+namespace bdr {
+
+int sm_count() {
+    static int cached[64];
+    static std::mutex mu;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 148;
+    std::lock_guard<std::mutex> lock(mu);
+    if (cached[dev] == 0) {
+        int n = 0;
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
+        cached[dev] = n;
+    }
+    return cached[dev];
+}
+
+static bool is_pow2(int v) { return v > 0 && (v & (v - 1)) == 0; }
+
+// Definition-level check of a POW2 tuple, then what the kernels can run.
+int check_pow2_config(const bdr_config_t* c, QParams* qp) {
+    if (!c) return BDR_ERR_NULL;
+    if (c->scale_kind != BDR_SCALE_POW2) {
+        if (c->scale_kind < 0 || c->scale_kind > BDR_SCALE_FP32_VSQ) return BDR_ERR_BAD_CONFIG;
+        return BDR_ERR_UNSUPPORTED;
+    }
+    if (c->rounding != BDR_ROUND_NEAREST_EVEN && c->rounding != BDR_ROUND_NEAREST_AWAY) return BDR_ERR_BAD_CONFIG;
+    if (c->d1 != 8 || c->k1 < 1 || c->k2 < 1 || c->k1 % c->k2 != 0 || c->d2 < 0 || c->d2 > 3 || c->m < 1 || c->m > 8)
+        return BDR_ERR_BAD_CONFIG;
+    if (!is_pow2(c->k1) || !is_pow2(c->k2) || c->k1 > 1024) return BDR_ERR_UNSUPPORTED;
+    if (qp) {
+        qp->k1 = c->k1; qp->k2 = c->k2; qp->d2 = c->d2; qp->m = c->m; qp->rounding = c->rounding;
+        qp->beta = (1 << c->d2) - 1;
+        qp->qmax = (1u << c->m) - 1u;
+    }
+    return BDR_OK;
+}
+
+static int check_tensor(const void* x, int dt, int64_t rows, int64_t cols, int64_t ld, int axis) {
+    if (dt != BDR_F32 && dt != BDR_BF16) return BDR_ERR_UNSUPPORTED;
+    if (axis != 0 && axis != 1) return BDR_ERR_BAD_CONFIG;
+    if (rows < 0 || cols < 0 || ld < cols) return BDR_ERR_SIZE;
+    if (!x) return (rows == 0 || cols == 0) ? BDR_OK : BDR_ERR_NULL;  // an empty tensor has no storage
+    if ((uintptr_t)x % (dt == BDR_F32 ? 4 : 2)) return BDR_ERR_MISALIGNED;
+    return BDR_OK;
+}
+
+static void line_bytes(const bdr_config_t* c, int64_t len, int64_t out[3]) {
+    const int64_t nb = (len + c->k1 - 1) / c->k1;
+    out[0] = nb;
+    out[1] = (nb * (c->k1 / c->k2) * c->d2 + 7) / 8;
+    out[2] = (nb * c->k1 * (c->m + 1) + 7) / 8;
+}
+
+static int check_planes(const bdr_config_t* c, const bdr_planes_t* p, int64_t len) {
+    if (!p || !p->exps || !p->elems || (c->d2 > 0 && !p->micro)) return BDR_ERR_NULL;
+    int64_t need[3];
+    line_bytes(c, len, need);
+    if (p->ld_exps < need[0] || p->ld_elems < need[2] || (c->d2 > 0 && p->ld_micro < need[1])) return BDR_ERR_SIZE;
+    if (((uintptr_t)p->exps | (uintptr_t)p->elems | (uintptr_t)(c->d2 ? p->micro : nullptr)) % 16) return BDR_ERR_MISALIGNED;
+    if ((p->ld_exps | p->ld_elems | (c->d2 ? p->ld_micro : 0)) % 16) return BDR_ERR_MISALIGNED;
+    return BDR_OK;
+}
+
+// True when every plane line is filled exactly by its natural bytes (no pitch padding to zero).
+static bool planes_tight(const bdr_config_t* c, const bdr_planes_t* p, int64_t len) {
+    int64_t need[3];
+    line_bytes(c, len, need);
+    return p->ld_exps == need[0] && p->ld_elems == need[2] && (c->d2 == 0 || p->ld_micro == need[1]);
+}
+
+template <typename T>
+static int quant_dispatch(const QParams& qp, const T* x, T* y, int64_t rows, int64_t cols, int64_t ld, int axis,
+                          const bdr_planes_t* out, bool tight, double* sums, cudaStream_t st) {
+    if (rows == 0 || cols == 0) return BDR_OK;
+    int rc = BDR_ERR_UNSUPPORTED;
+    if (axis == 1) {
+        if (out) { if (tight) rc = pack_rowwise_mx<T>(x, y, rows, cols, ld, *out, qp, sums, st); }
+        else rc = quant_rowwise<T>(x, y, rows, cols, ld, qp, sums, st);
+    } else {
+        if (!out || tight) rc = quant_colwise_mx<T>(x, y, rows, cols, ld, out, qp, sums, st);
+    }
+    if (rc == BDR_ERR_UNSUPPORTED) rc = quant_general<T>(x, y, rows, cols, ld, axis, out, qp, sums, st);
+    return rc;
+}
+
+}  // namespace bdr
+
+using namespace bdr;
+
+extern "C" {
+
+const char* bdr_strerror(int status) {
+    switch (status) {
+        case BDR_OK: return "ok";
+        case BDR_ERR_NULL: return "a required pointer is NULL";
+        case BDR_ERR_BAD_CONFIG: return "configuration outside the BDR definition";
+        case BDR_ERR_UNSUPPORTED: return "valid request that no kernel of this library covers";
+        case BDR_ERR_MISALIGNED: return "pointer or pitch breaks an alignment rule";
+        case BDR_ERR_SIZE: return "bad size or pitch";
+        case BDR_ERR_WORKSPACE: return "workspace missing or too small";
+        case BDR_ERR_CUDA: return "CUDA call or kernel launch failed";
+        case BDR_ERR_TIMEOUT: return "bounded device-side wait ran out";
+    }
+    return "unknown status";
+}
+
+int bdr_packed_sizes(const bdr_config_t* cfg, int64_t rows, int64_t cols, int axis, int64_t ld_out[3],
+                     int64_t bytes_out[3]) {
+    if (!cfg || !ld_out || !bytes_out) return BDR_ERR_NULL;
+    if (cfg->scale_kind != BDR_SCALE_POW2) return BDR_ERR_UNSUPPORTED;
+    if (cfg->d1 != 8 || cfg->k1 < 1 || cfg->k2 < 1 || cfg->k1 % cfg->k2 != 0 || cfg->d2 < 0 || cfg->d2 > 3 ||
+        cfg->m < 1 || cfg->m > 8)
+        return BDR_ERR_BAD_CONFIG;
+    if (axis != 0 && axis != 1) return BDR_ERR_BAD_CONFIG;
+    if (rows < 0 || cols < 0) return BDR_ERR_SIZE;
+    const int64_t nlines = axis == 1 ? rows : cols, len = axis == 1 ? cols : rows;
+    int64_t need[3];
+    line_bytes(cfg, len, need);
+    for (int i = 0; i < 3; ++i) {
+        ld_out[i] = (need[i] + 15) / 16 * 16;
+        bytes_out[i] = ld_out[i] * nlines;
+    }
+    return BDR_OK;
+}
+
+int bdr_quant_dequant(const bdr_config_t* cfg, const void* x, void* y, bdr_dtype_t dt, int64_t rows, int64_t cols,
+                      int64_t ld, int axis, double* qsnr_sums_dev, void* stream) {
+    QParams qp;
+    int rc = check_pow2_config(cfg, &qp);
+    if (rc) return rc;
+    if ((rc = check_tensor(x, dt, rows, cols, ld, axis))) return rc;
+    if (rows == 0 || cols == 0) return BDR_OK;
+    if (!y && !qsnr_sums_dev) return BDR_ERR_NULL;
+    if (y && (uintptr_t)y % (dt == BDR_F32 ? 4 : 2)) return BDR_ERR_MISALIGNED;
+    if (qsnr_sums_dev && (uintptr_t)qsnr_sums_dev % 8) return BDR_ERR_MISALIGNED;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (dt == BDR_F32)
+        return quant_dispatch<float>(qp, (const float*)x, (float*)y, rows, cols, ld, axis, nullptr, false, qsnr_sums_dev, st);
+    return quant_dispatch<__nv_bfloat16>(qp, (const __nv_bfloat16*)x, (__nv_bfloat16*)y, rows, cols, ld, axis, nullptr,
+                                         false, qsnr_sums_dev, st);
+}
+
+int bdr_pack(const bdr_config_t* cfg, const void* x, bdr_dtype_t dt, int64_t rows, int64_t cols, int64_t ld, int axis,
+             const bdr_planes_t* out, void* y_dq, double* qsnr_sums_dev, void* stream) {
+    QParams qp;
+    int rc = check_pow2_config(cfg, &qp);
+    if (rc) return rc;
+    if ((rc = check_tensor(x, dt, rows, cols, ld, axis))) return rc;
+    if (rows == 0 || cols == 0) return BDR_OK;
+    if ((rc = check_planes(cfg, out, axis == 1 ? cols : rows))) return rc;
+    if (y_dq && (uintptr_t)y_dq % (dt == BDR_F32 ? 4 : 2)) return BDR_ERR_MISALIGNED;
+    if (qsnr_sums_dev && (uintptr_t)qsnr_sums_dev % 8) return BDR_ERR_MISALIGNED;
+    const bool tight = planes_tight(cfg, out, axis == 1 ? cols : rows);
+    cudaStream_t st = (cudaStream_t)stream;
+    if (dt == BDR_F32)
+        return quant_dispatch<float>(qp, (const float*)x, (float*)y_dq, rows, cols, ld, axis, out, tight, qsnr_sums_dev, st);
+    return quant_dispatch<__nv_bfloat16>(qp, (const __nv_bfloat16*)x, (__nv_bfloat16*)y_dq, rows, cols, ld, axis, out,
+                                         tight, qsnr_sums_dev, st);
+}
+
+int bdr_unpack(const bdr_config_t* cfg, const bdr_planes_t* in, void* y, bdr_dtype_t dt, int64_t rows, int64_t cols,
+               int64_t ld, int axis, void* stream) {
+    QParams qp;
+    int rc = check_pow2_config(cfg, &qp);
+    if (rc) return rc;
+    if ((rc = check_tensor(y, dt, rows, cols, ld, axis))) return rc;
+    if (rows == 0 || cols == 0) return BDR_OK;
+    if ((rc = check_planes(cfg, in, axis == 1 ? cols : rows))) return rc;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (dt == BDR_F32) {
+        rc = axis == 1 ? unpack_rowwise_mx<float>(*in, (float*)y, rows, cols, ld, qp, st)
+                       : unpack_colwise_mx<float>(*in, (float*)y, rows, cols, ld, qp, st);
+        if (rc == BDR_ERR_UNSUPPORTED) rc = unpack_general<float>(*in, (float*)y, rows, cols, ld, axis, qp, st);
+    } else {
+        rc = axis == 1 ? unpack_rowwise_mx<__nv_bfloat16>(*in, (__nv_bfloat16*)y, rows, cols, ld, qp, st)
+                       : unpack_colwise_mx<__nv_bfloat16>(*in, (__nv_bfloat16*)y, rows, cols, ld, qp, st);
+        if (rc == BDR_ERR_UNSUPPORTED) rc = unpack_general<__nv_bfloat16>(*in, (__nv_bfloat16*)y, rows, cols, ld, axis, qp, st);
+    }
+    return rc;
+}
+
+}  // extern "C"

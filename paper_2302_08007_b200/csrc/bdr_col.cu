@@ -1,0 +1,254 @@
+// Column-direction (axis 0) fast paths for the k1 = 16, k2 = 2 family: blocks run down the strided
+// dimension, and the packed planes come out in the transposed (column-major, reduction-contiguous)
+// layout that the backward-pass GEMMs consume (Section V: "transpose, then quantize").
+//
+// A CTA owns a tile of 64 columns x 32 row-blocks (512 rows).  Each warp takes one 16-row block at a
+// time; a lane owns two adjacent columns, so every row access of the warp is one contiguous,
+// fully coalesced segment.  The lane's codes are staged in shared memory as [row-block][column]
+// items; the CTA then gathers them per column and writes each column's 32 row-blocks as one
+// contiguous run of 64*W bytes (and 32 exponent bytes, 32*d2 microexponent bytes), so the transposed
+// planes are written with whole 16-byte vectors and whole 32-byte sectors.
+#include "bdr_device.cuh"
+#include "bdr_host.h"
+
+namespace bdr {
+
+constexpr int kColThreads = 256;
+constexpr int kColWarps = kColThreads / 32;
+constexpr int kTileCols = 64;
+constexpr int kTileBlocks = 32;  // 16-row blocks per tile
+
+// two adjacent columns of one row, as fp32 bit patterns
+__device__ __forceinline__ void load_pair(const float* p, uint32_t& a, uint32_t& b) {
+    const uint2 v = __ldg(reinterpret_cast<const uint2*>(p));
+    a = v.x; b = v.y;
+}
+__device__ __forceinline__ void load_pair(const __nv_bfloat16* p, uint32_t& a, uint32_t& b) {
+    const uint32_t v = __ldg(reinterpret_cast<const uint32_t*>(p));
+    a = v << 16; b = v & 0xFFFF0000u;
+}
+__device__ __forceinline__ void store_pair(float* p, uint32_t a, uint32_t b) {
+    *reinterpret_cast<uint2*>(p) = make_uint2(a, b);
+}
+__device__ __forceinline__ void store_pair(__nv_bfloat16* p, uint32_t a, uint32_t b) {
+    *reinterpret_cast<uint32_t*>(p) = (a >> 16) | (b & 0xFFFF0000u);
+}
+
+template <int W>
+struct ColStage {
+    static constexpr int kW = W > 0 ? W : 1;
+    uint16_t elems[kTileBlocks][kTileCols][kW];  // 2W bytes per (row-block, column)
+    uint8_t exps[kTileBlocks][kTileCols];
+    uint8_t micro[kTileBlocks][kTileCols][3];
+};
+
+template <typename T, int W>  // W = m + 1 when packing, 0 when only y / sums are wanted
+__global__ void __launch_bounds__(kColThreads)
+quant_colwise_mx_kernel(const T* x, T* y, int64_t rows, int64_t cols, int64_t ld, bdr_planes_t out, QParams qp,
+                        double* sums) {
+    __shared__ __align__(16) ColStage<W> st;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int64_t c0 = (int64_t)blockIdx.x * kTileCols;
+    const int64_t tb0 = (int64_t)blockIdx.y * kTileBlocks;
+    const int64_t nblocks = rows / kSlice;
+    const int64_t c = c0 + 2 * lane;
+    double e2 = 0.0, s2 = 0.0;
+    for (int bl = warp; bl < kTileBlocks; bl += kColWarps) {
+        const int64_t b = tb0 + bl;
+        if (b >= nblocks) break;
+        uint32_t u[2][kSlice];
+        const T* px = x + b * kSlice * ld + c;
+#pragma unroll
+        for (int r = 0; r < kSlice; ++r) load_pair(px + r * ld, u[0][r], u[1][r]);
+        uint32_t yb[2][kSlice];
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            uint32_t code[kSlice], tau[kSlice / 2];
+            int fj[kSlice / 2], fb[1];
+            subblock_exponents<2>(u[h], fj);
+            int F = 0;
+#pragma unroll
+            for (int j = 0; j < kSlice / 2; ++j) F = max(F, fj[j]);
+            fb[0] = F;
+            if (sums) quantize_slice<2, kSlice, true>(u[h], fj, fb, qp, yb[h], code, tau, e2, s2);
+            else quantize_slice<2, kSlice, false>(u[h], fj, fb, qp, yb[h], code, tau, e2, s2);
+            if (W > 0) {
+                uint32_t words[(kSlice * ColStage<W>::kW + 31) / 32];
+                codes_to_words<ColStage<W>::kW>(code, words);
+#pragma unroll
+                for (int k = 0; k < ColStage<W>::kW; ++k)
+                    st.elems[bl][2 * lane + h][k] = (uint16_t)(words[k >> 1] >> ((k & 1) * 16));
+                st.exps[bl][2 * lane + h] = (uint8_t)F;
+                uint32_t mbits = 0;
+#pragma unroll
+                for (int j = 0; j < kSlice / 2; ++j) mbits |= tau[j] << (j * qp.d2);
+                for (int k = 0; k < qp.d2; ++k) st.micro[bl][2 * lane + h][k] = (uint8_t)(mbits >> (8 * k));
+            }
+        }
+        if (y) {
+            T* py = y + b * kSlice * ld + c;
+#pragma unroll
+            for (int r = 0; r < kSlice; ++r) store_pair(py + r * ld, yb[0][r], yb[1][r]);
+        }
+    }
+    if (W > 0) {
+        constexpr int kW = ColStage<W>::kW;
+        __syncthreads();
+        // elems: each column's run is kTileBlocks * 2W = 64W bytes = 4W vectors of 16 bytes
+        for (int idx = threadIdx.x; idx < kTileCols * 4 * kW; idx += kColThreads) {
+            const int ci = idx % kTileCols, v = idx / kTileCols;
+            uint32_t w4[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int h0 = 8 * v + 2 * i, h1 = h0 + 1;
+                w4[i] = (uint32_t)st.elems[h0 / kW][ci][h0 % kW] | ((uint32_t)st.elems[h1 / kW][ci][h1 % kW] << 16);
+            }
+            *reinterpret_cast<uint4*>(out.elems + (c0 + ci) * out.ld_elems + tb0 * 2 * kW + v * 16) =
+                make_uint4(w4[0], w4[1], w4[2], w4[3]);
+        }
+        // exps: 32 bytes per column; micro: 32*d2 bytes per column
+        for (int idx = threadIdx.x; idx < kTileCols * 2; idx += kColThreads) {
+            const int ci = idx % kTileCols, v = idx / kTileCols;
+            uint32_t w4[4] = {0, 0, 0, 0};
+#pragma unroll
+            for (int i = 0; i < 16; ++i) w4[i >> 2] |= (uint32_t)st.exps[16 * v + i][ci] << ((i & 3) * 8);
+            *reinterpret_cast<uint4*>(out.exps + (c0 + ci) * out.ld_exps + tb0 + v * 16) =
+                make_uint4(w4[0], w4[1], w4[2], w4[3]);
+        }
+        for (int idx = threadIdx.x; idx < kTileCols * 2 * qp.d2; idx += kColThreads) {
+            const int ci = idx % kTileCols, v = idx / kTileCols;
+            uint32_t w4[4] = {0, 0, 0, 0};
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+                const int t = 16 * v + i;
+                w4[i >> 2] |= (uint32_t)st.micro[t / qp.d2][ci][t % qp.d2] << ((i & 3) * 8);
+            }
+            *reinterpret_cast<uint4*>(out.micro + (c0 + ci) * out.ld_micro + tb0 * qp.d2 + v * 16) =
+                make_uint4(w4[0], w4[1], w4[2], w4[3]);
+        }
+    }
+    if (sums) block_accumulate_sums(e2, s2, sums);
+}
+
+// Mirror image: gather each column's packed run with coalesced 16-byte loads, scatter it into
+// [row-block][column] items in shared memory, then decode with lanes on adjacent column pairs.
+template <typename T, int W>
+__global__ void __launch_bounds__(kColThreads)
+unpack_colwise_mx_kernel(bdr_planes_t in, T* y, int64_t rows, int64_t cols, int64_t ld, QParams qp) {
+    __shared__ __align__(16) ColStage<W> st;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int64_t c0 = (int64_t)blockIdx.x * kTileCols;
+    const int64_t tb0 = (int64_t)blockIdx.y * kTileBlocks;
+    for (int idx = threadIdx.x; idx < kTileCols * 4 * W; idx += kColThreads) {
+        const int v = idx % (4 * W), ci = idx / (4 * W);  // consecutive threads walk one column's run
+        const uint4 q4 = __ldg(reinterpret_cast<const uint4*>(in.elems + (c0 + ci) * in.ld_elems + tb0 * 2 * W + v * 16));
+        const uint32_t w4[4] = {q4.x, q4.y, q4.z, q4.w};
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const int h = 8 * v + i;
+            st.elems[h / W][ci][h % W] = (uint16_t)(w4[i >> 1] >> ((i & 1) * 16));
+        }
+    }
+    for (int idx = threadIdx.x; idx < kTileCols * 2; idx += kColThreads) {
+        const int v = idx % 2, ci = idx / 2;
+        const uint4 q4 = __ldg(reinterpret_cast<const uint4*>(in.exps + (c0 + ci) * in.ld_exps + tb0 + v * 16));
+        const uint32_t w4[4] = {q4.x, q4.y, q4.z, q4.w};
+#pragma unroll
+        for (int i = 0; i < 16; ++i) st.exps[16 * v + i][ci] = (uint8_t)(w4[i >> 2] >> ((i & 3) * 8));
+    }
+    for (int idx = threadIdx.x; idx < kTileCols * 2 * qp.d2; idx += kColThreads) {
+        const int v = idx % (2 * qp.d2), ci = idx / (2 * qp.d2);
+        const uint4 q4 = __ldg(reinterpret_cast<const uint4*>(in.micro + (c0 + ci) * in.ld_micro + tb0 * qp.d2 + v * 16));
+        const uint32_t w4[4] = {q4.x, q4.y, q4.z, q4.w};
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+            const int t = 16 * v + i;
+            st.micro[t / qp.d2][ci][t % qp.d2] = (uint8_t)(w4[i >> 2] >> ((i & 3) * 8));
+        }
+    }
+    __syncthreads();
+    const int64_t c = c0 + 2 * lane;
+    for (int bl = warp; bl < kTileBlocks; bl += kColWarps) {
+        const int64_t b = tb0 + bl;
+        uint32_t yb[2][kSlice];
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            uint32_t words[(kSlice * W + 31) / 32 + 1];
+#pragma unroll
+            for (int i = 0; i < (kSlice * W + 31) / 32 + 1; ++i) words[i] = 0;
+#pragma unroll
+            for (int k = 0; k < W; ++k) words[k >> 1] |= (uint32_t)st.elems[bl][2 * lane + h][k] << ((k & 1) * 16);
+            uint32_t mbits = 0;
+            for (int k = 0; k < qp.d2; ++k) mbits |= (uint32_t)st.micro[bl][2 * lane + h][k] << (8 * k);
+            decode_slice<W>(words, st.exps[bl][2 * lane + h], mbits, qp, yb[h]);
+        }
+        T* py = y + b * kSlice * ld + c;
+#pragma unroll
+        for (int r = 0; r < kSlice; ++r) store_pair(py + r * ld, yb[0][r], yb[1][r]);
+    }
+}
+
+template <typename T, int W>
+static int launch_col(const T* x, T* y, int64_t rows, int64_t cols, int64_t ld, const bdr_planes_t* out,
+                      const QParams& qp, double* sums, cudaStream_t st) {
+    const dim3 grid((unsigned)(cols / kTileCols), (unsigned)((rows / kSlice + kTileBlocks - 1) / kTileBlocks));
+    bdr_planes_t pl = {};
+    if (out) pl = *out;
+    quant_colwise_mx_kernel<T, W><<<grid, kColThreads, 0, st>>>(x, y, rows, cols, ld, pl, qp, sums);
+    return cudaGetLastError() == cudaSuccess ? BDR_OK : BDR_ERR_CUDA;
+}
+
+template <typename T>
+int quant_colwise_mx(const T* x, T* y, int64_t rows, int64_t cols, int64_t ld, const bdr_planes_t* out,
+                     const QParams& qp, double* sums, cudaStream_t st) {
+    if (qp.k1 != 16 || qp.k2 != 2 || cols % kTileCols != 0 || rows % kSlice != 0) return BDR_ERR_UNSUPPORTED;
+    if (out && rows % (kSlice * kTileBlocks) != 0) return BDR_ERR_UNSUPPORTED;
+    if ((((uintptr_t)x | (uintptr_t)y) % 16) || (ld * sizeof(T)) % 16) return BDR_ERR_UNSUPPORTED;
+    if (rows / kSlice / kTileBlocks > 65535) return BDR_ERR_UNSUPPORTED;
+    if (!out) return launch_col<T, 0>(x, y, rows, cols, ld, out, qp, sums, st);
+    switch (qp.m + 1) {
+        case 2: return launch_col<T, 2>(x, y, rows, cols, ld, out, qp, sums, st);
+        case 3: return launch_col<T, 3>(x, y, rows, cols, ld, out, qp, sums, st);
+        case 4: return launch_col<T, 4>(x, y, rows, cols, ld, out, qp, sums, st);
+        case 5: return launch_col<T, 5>(x, y, rows, cols, ld, out, qp, sums, st);
+        case 6: return launch_col<T, 6>(x, y, rows, cols, ld, out, qp, sums, st);
+        case 7: return launch_col<T, 7>(x, y, rows, cols, ld, out, qp, sums, st);
+        case 8: return launch_col<T, 8>(x, y, rows, cols, ld, out, qp, sums, st);
+        case 9: return launch_col<T, 9>(x, y, rows, cols, ld, out, qp, sums, st);
+    }
+    return BDR_ERR_UNSUPPORTED;
+}
+
+template <typename T, int W>
+static int launch_unpack_col(const bdr_planes_t& in, T* y, int64_t rows, int64_t cols, int64_t ld, const QParams& qp,
+                             cudaStream_t st) {
+    const dim3 grid((unsigned)(cols / kTileCols), (unsigned)(rows / (kSlice * kTileBlocks)));
+    unpack_colwise_mx_kernel<T, W><<<grid, kColThreads, 0, st>>>(in, y, rows, cols, ld, qp);
+    return cudaGetLastError() == cudaSuccess ? BDR_OK : BDR_ERR_CUDA;
+}
+
+template <typename T>
+int unpack_colwise_mx(const bdr_planes_t& in, T* y, int64_t rows, int64_t cols, int64_t ld, const QParams& qp,
+                      cudaStream_t st) {
+    if (qp.k1 != 16 || qp.k2 != 2 || cols % kTileCols != 0 || rows % (kSlice * kTileBlocks) != 0) return BDR_ERR_UNSUPPORTED;
+    if (((uintptr_t)y % 16) || (ld * sizeof(T)) % 16) return BDR_ERR_UNSUPPORTED;
+    if (rows / (kSlice * kTileBlocks) > 65535) return BDR_ERR_UNSUPPORTED;
+    switch (qp.m + 1) {
+        case 2: return launch_unpack_col<T, 2>(in, y, rows, cols, ld, qp, st);
+        case 3: return launch_unpack_col<T, 3>(in, y, rows, cols, ld, qp, st);
+        case 4: return launch_unpack_col<T, 4>(in, y, rows, cols, ld, qp, st);
+        case 5: return launch_unpack_col<T, 5>(in, y, rows, cols, ld, qp, st);
+        case 6: return launch_unpack_col<T, 6>(in, y, rows, cols, ld, qp, st);
+        case 7: return launch_unpack_col<T, 7>(in, y, rows, cols, ld, qp, st);
+        case 8: return launch_unpack_col<T, 8>(in, y, rows, cols, ld, qp, st);
+        case 9: return launch_unpack_col<T, 9>(in, y, rows, cols, ld, qp, st);
+    }
+    return BDR_ERR_UNSUPPORTED;
+}
+
+template int quant_colwise_mx<float>(const float*, float*, int64_t, int64_t, int64_t, const bdr_planes_t*, const QParams&, double*, cudaStream_t);
+template int quant_colwise_mx<__nv_bfloat16>(const __nv_bfloat16*, __nv_bfloat16*, int64_t, int64_t, int64_t, const bdr_planes_t*, const QParams&, double*, cudaStream_t);
+template int unpack_colwise_mx<float>(const bdr_planes_t&, float*, int64_t, int64_t, int64_t, const QParams&, cudaStream_t);
+template int unpack_colwise_mx<__nv_bfloat16>(const bdr_planes_t&, __nv_bfloat16*, int64_t, int64_t, int64_t, const QParams&, cudaStream_t);
+
+}  // namespace bdr

@@ -1,0 +1,284 @@
+// Device-side building blocks shared by the quantize / pack / unpack / sweep kernels.
+//
+// Notation follows the paper's Appendix: F is the biased shared exponent of a k1-block (the fp32
+// exponent field of its largest element, E = F - 127), tau the shift of a k2-sub-block
+// (tau = min(F - F_sub, beta), beta = 2^d2 - 1), m the number of magnitude digits, q the integer
+// magnitude (0 .. 2^m - 1) and p = E - tau - (m - 1) the exponent of one unit of q.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "bdr.h"
+
+namespace bdr {
+
+// Launch-time constants of one POW2 configuration.
+struct QParams {
+    int k1, k2, d2, m, rounding;
+    int beta;       // 2^d2 - 1
+    uint32_t qmax;  // 2^m - 1
+};
+
+constexpr int kSlice = 16;  // elements a thread keeps in registers at a time
+
+__device__ __forceinline__ int exp_field(uint32_t u) { return (int)((u >> 23) & 0xFFu); }
+
+// 2^p as fp32 bits for -149 <= p <= 127 (subnormal powers included).
+__device__ __forceinline__ uint32_t pow2_bits(int p) {
+    return p >= -126 ? (uint32_t)(p + 127) << 23 : 1u << (p + 149);
+}
+
+// Exact integer formulation of one element (any tie rule, any exponent): |x| = M * 2^(fe-150),
+// |x| / 2^p = M / 2^sh.  Returns q (clamped) and the dequantized bit pattern.
+__device__ __forceinline__ void quant_elem_exact(uint32_t u, int F, int tau, const QParams& qp, uint32_t& q,
+                                                 uint32_t& ybits) {
+    const int f = exp_field(u);
+    const uint32_t M = (u & 0x7FFFFFu) | (f ? 0x800000u : 0u);
+    const int fe = f ? f : 1;
+    const int sh = 24 - qp.m - tau - (fe - F);  // >= 8 for every legal configuration
+    uint32_t qq = 0;
+    if (sh <= 25) {
+        const uint32_t fl = M >> sh;
+        const uint32_t rem = M & ((1u << sh) - 1u);
+        const uint32_t half = 1u << (sh - 1);
+        qq = fl + ((rem > half) || (rem == half && (qp.rounding == BDR_ROUND_NEAREST_AWAY || (fl & 1u))) ? 1u : 0u);
+    }
+    qq = min(qq, qp.qmax);
+    q = qq;
+    const int p = F - 127 - tau - (qp.m - 1);
+    const float mag = __fmul_rn(__uint2float_rn(qq), __uint_as_float(pow2_bits(p)));  // exact
+    ybits = __float_as_uint(mag) | (u & 0x80000000u);
+}
+
+// Fast formulation for ties-to-even: adding C = 1.5 * 2^(p+23) makes the fp32 adder round |x| to a
+// multiple of 2^p (nearest, ties to even) and leaves q in the low mantissa bits of the sum.
+// Valid while C is finite, i.e. F <= kFastMaxF.
+constexpr int kFastMaxF = 230;
+
+struct SubScale {
+    uint32_t Cbits;  // bits of C
+    float C;
+};
+
+__device__ __forceinline__ SubScale make_subscale(int F, int tau, int m) {
+    SubScale s;
+    s.Cbits = ((uint32_t)(F - tau - m + 24) << 23) | 0x400000u;
+    s.C = __uint_as_float(s.Cbits);
+    return s;
+}
+
+__device__ __forceinline__ void quant_elem_fast(uint32_t u, const SubScale& s, uint32_t qmax, uint32_t& q,
+                                                uint32_t& ybits, float& abs_x, float& abs_q) {
+    abs_x = __uint_as_float(u & 0x7FFFFFFFu);
+    const float t = __fadd_rn(abs_x, s.C);
+    q = min(__float_as_uint(t) - s.Cbits, qmax);
+    abs_q = __fsub_rn(__uint_as_float(s.Cbits + q), s.C);
+    ybits = __float_as_uint(abs_q) | (u & 0x80000000u);
+}
+
+// ---- element I/O --------------------------------------------------------------------------------
+template <typename T> struct Elem;
+template <> struct Elem<float> {
+    static constexpr int kBytes = 4;
+    __device__ static __forceinline__ uint32_t load_bits(const float* p) { return __float_as_uint(*p); }
+    __device__ static __forceinline__ void store_bits(float* p, uint32_t b) { *p = __uint_as_float(b); }
+};
+template <> struct Elem<__nv_bfloat16> {
+    static constexpr int kBytes = 2;
+    __device__ static __forceinline__ uint32_t load_bits(const __nv_bfloat16* p) {
+        return (uint32_t)(*reinterpret_cast<const uint16_t*>(p)) << 16;
+    }
+    // every value this library produces from bf16 inputs (or from m <= 8 codes within bf16's
+    // exponent range) has its low 16 fp32 bits clear, so truncation is exact
+    __device__ static __forceinline__ void store_bits(__nv_bfloat16* p, uint32_t b) {
+        *reinterpret_cast<uint16_t*>(p) = (uint16_t)(b >> 16);
+    }
+};
+
+// Load / store one 16-element slice as fp32 bit patterns with 128-bit accesses.
+__device__ __forceinline__ void load_slice_vec(const float* p, uint32_t (&u)[kSlice]) {
+    const uint4* v = reinterpret_cast<const uint4*>(p);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const uint4 w = __ldg(v + i);
+        u[4 * i] = w.x; u[4 * i + 1] = w.y; u[4 * i + 2] = w.z; u[4 * i + 3] = w.w;
+    }
+}
+__device__ __forceinline__ void load_slice_vec(const __nv_bfloat16* p, uint32_t (&u)[kSlice]) {
+    const uint4* v = reinterpret_cast<const uint4*>(p);
+#pragma unroll
+    for (int i = 0; i < 2; ++i) {
+        const uint4 w = __ldg(v + i);
+        const uint32_t ws[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            u[8 * i + 2 * k] = ws[k] << 16;
+            u[8 * i + 2 * k + 1] = ws[k] & 0xFFFF0000u;
+        }
+    }
+}
+__device__ __forceinline__ void store_slice_vec(float* p, const uint32_t (&y)[kSlice]) {
+    uint4* v = reinterpret_cast<uint4*>(p);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) v[i] = make_uint4(y[4 * i], y[4 * i + 1], y[4 * i + 2], y[4 * i + 3]);
+}
+__device__ __forceinline__ void store_slice_vec(__nv_bfloat16* p, const uint32_t (&y)[kSlice]) {
+    uint4* v = reinterpret_cast<uint4*>(p);
+#pragma unroll
+    for (int i = 0; i < 2; ++i) {
+        uint32_t ws[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) ws[k] = (y[8 * i + 2 * k] >> 16) | (y[8 * i + 2 * k + 1] & 0xFFFF0000u);
+        v[i] = make_uint4(ws[0], ws[1], ws[2], ws[3]);
+    }
+}
+
+// Guarded scalar versions for ragged tails and unaligned tensors: elements at index >= n read as +0.
+template <typename T>
+__device__ __forceinline__ void load_slice_guarded(const T* p, int64_t stride, int n, uint32_t (&u)[kSlice]) {
+#pragma unroll
+    for (int i = 0; i < kSlice; ++i) u[i] = i < n ? Elem<T>::load_bits(p + i * stride) : 0u;
+}
+template <typename T>
+__device__ __forceinline__ void store_slice_guarded(T* p, int64_t stride, int n, const uint32_t (&y)[kSlice]) {
+#pragma unroll
+    for (int i = 0; i < kSlice; ++i)
+        if (i < n) Elem<T>::store_bits(p + i * stride, y[i]);
+}
+
+// ---- block reduction of the two Eq. 3 sums ------------------------------------------------------
+__device__ __forceinline__ double warp_sum(double v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
+    return v;
+}
+
+// Every thread of the CTA calls this once; adds the CTA totals to sums[0..1] with two atomics.
+__device__ __forceinline__ void block_accumulate_sums(double err2, double sig2, double* sums) {
+    __shared__ double sh[2][32];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarp = (blockDim.x + 31) >> 5;
+    err2 = warp_sum(err2);
+    sig2 = warp_sum(sig2);
+    if (lane == 0) { sh[0][warp] = err2; sh[1][warp] = sig2; }
+    __syncthreads();
+    if (warp == 0) {
+        double e = lane < nwarp ? sh[0][lane] : 0.0, s = lane < nwarp ? sh[1][lane] : 0.0;
+        e = warp_sum(e);
+        s = warp_sum(s);
+        if (lane == 0) { atomicAdd(sums, e); atomicAdd(sums + 1, s); }
+    }
+}
+
+}  // namespace bdr
+
+namespace bdr {
+
+// ---- one 16-element slice ------------------------------------------------------------------------
+// Sub-block maxima of the exponent fields (k2 <= 16) and, for k1 < 16, block maxima.
+template <int K2>
+__device__ __forceinline__ void subblock_exponents(const uint32_t (&u)[kSlice], int (&fj)[kSlice / K2]) {
+#pragma unroll
+    for (int j = 0; j < kSlice / K2; ++j) {
+        int f = 0;
+#pragma unroll
+        for (int i = 0; i < K2; ++i) f = max(f, exp_field(u[j * K2 + i]));
+        fj[j] = f;
+    }
+}
+
+// Quantize the slice.  fb[] holds the shared exponent of each k1-block touching the slice
+// (K1S = min(k1,16) elements each; for k1 >= 16 the single entry is the block's exponent after
+// any cross-lane reduction).  Produces dequantized bit patterns, element codes (sign<<m | q),
+// sub-block shifts, and adds this slice's Eq. 3 terms to e2 / s2 when WANT_SUMS.
+template <int K2, int K1S, bool WANT_SUMS>
+__device__ __forceinline__ void quantize_slice(const uint32_t (&u)[kSlice], const int (&fj)[kSlice / K2],
+                                               const int (&fb)[kSlice / K1S], const QParams& qp,
+                                               uint32_t (&yb)[kSlice], uint32_t (&code)[kSlice],
+                                               uint32_t (&tau)[kSlice / K2], double& e2, double& s2) {
+#pragma unroll
+    for (int j = 0; j < kSlice / K2; ++j) {
+        const int F = fb[(j * K2) / K1S];
+        const int t = min(F - fj[j], qp.beta);
+        tau[j] = (uint32_t)t;
+        if (F == 255) {  // Inf/NaN somewhere in the block: the whole block decodes to NaN
+            tau[j] = 0;
+#pragma unroll
+            for (int i = 0; i < K2; ++i) {
+                yb[j * K2 + i] = 0x7FC00000u;
+                code[j * K2 + i] = 0;
+                if (WANT_SUMS) { e2 = __longlong_as_double(0x7FF8000000000000ll); s2 = e2; }
+            }
+        } else if (qp.rounding == BDR_ROUND_NEAREST_EVEN && F <= kFastMaxF) {
+            const SubScale ss = make_subscale(F, t, qp.m);
+#pragma unroll
+            for (int i = 0; i < K2; ++i) {
+                const int k = j * K2 + i;
+                uint32_t q;
+                float ax, aq;
+                quant_elem_fast(u[k], ss, qp.qmax, q, yb[k], ax, aq);
+                code[k] = ((u[k] >> 31) << qp.m) | q;
+                if (WANT_SUMS) {
+                    const double de = (double)__fsub_rn(aq, ax), dx = (double)ax;  // difference is exact in fp32
+                    e2 = fma(de, de, e2);
+                    s2 = fma(dx, dx, s2);
+                }
+            }
+        } else {
+#pragma unroll
+            for (int i = 0; i < K2; ++i) {
+                const int k = j * K2 + i;
+                uint32_t q;
+                quant_elem_exact(u[k], F, t, qp, q, yb[k]);
+                code[k] = ((u[k] >> 31) << qp.m) | q;
+                if (WANT_SUMS) {
+                    const double de = (double)__uint_as_float(yb[k]) - (double)__uint_as_float(u[k]);
+                    const double dx = (double)__uint_as_float(u[k]);
+                    e2 = fma(de, de, e2);
+                    s2 = fma(dx, dx, s2);
+                }
+            }
+        }
+    }
+}
+
+// ---- bit-stream helpers for one slice (code width W = m + 1 known at compile time) -----------------
+// Pack 16 codes into the little-endian LSB-first stream of the slice (2W bytes).
+template <int W>
+__device__ __forceinline__ void codes_to_words(const uint32_t (&code)[kSlice], uint32_t (&words)[(kSlice * W + 31) / 32]) {
+#pragma unroll
+    for (int i = 0; i < (kSlice * W + 31) / 32; ++i) words[i] = 0;
+#pragma unroll
+    for (int i = 0; i < kSlice; ++i) {
+        const int bit = i * W, wi = bit >> 5, sh = bit & 31;
+        words[wi] |= code[i] << sh;
+        if (sh + W > 32) words[wi + 1] |= code[i] >> (32 - sh);
+    }
+}
+
+
+// Decode one slice: codes are W-bit fields of the little-endian stream in `words`.
+template <int W>
+__device__ __forceinline__ void decode_slice(const uint32_t (&words)[(kSlice * W + 31) / 32 + 1], int F, uint32_t mbits,
+                                             const QParams& qp, uint32_t (&yb)[kSlice]) {
+    constexpr uint32_t kMask = (1u << W) - 1u;
+#pragma unroll
+    for (int j = 0; j < kSlice / 2; ++j) {
+        const int tau = (int)((mbits >> (j * qp.d2)) & (uint32_t)qp.beta);
+        const float scale = __uint_as_float(pow2_bits(max(F - 127 - tau - (qp.m - 1), -149)));
+#pragma unroll
+        for (int i = 0; i < 2; ++i) {
+            const int k = 2 * j + i, bit = k * W, wi = bit >> 5, sh = bit & 31;
+            uint32_t code = words[wi] >> sh;
+            if (sh + W > 32) code |= words[wi + 1] << (32 - sh);
+            code &= kMask;
+            const uint32_t q = code & qp.qmax;
+            // 2^23 + q is exact in fp32; subtracting 2^23 converts q without the conversion pipe
+            const float qf = __fsub_rn(__uint_as_float(0x4B000000u | q), 8388608.0f);
+            yb[k] = F == 255 ? 0x7FC00000u : (__float_as_uint(__fmul_rn(qf, scale)) | ((code >> qp.m) << 31));
+        }
+    }
+}
+
+}  // namespace bdr

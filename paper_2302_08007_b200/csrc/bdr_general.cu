@@ -1,0 +1,141 @@
+// General kernels: any axis, any POW2 configuration, any pitch or alignment, ragged tails.
+// Correctness first; the fast paths in bdr_row.cu / bdr_col.cu / bdr_unpack.cu cover the shapes
+// that matter for throughput and produce identical bytes.
+#include "bdr_device.cuh"
+#include "bdr_host.h"
+
+namespace bdr {
+
+constexpr int kGenThreads = 128;
+
+// OR a field into an LSB-first bit stream whose line starts 4-byte aligned (planes are zeroed first).
+__device__ __forceinline__ void or_bits(uint8_t* line, int64_t bitpos, int nbits, uint32_t val) {
+    if (!val) return;
+    uint32_t* w = reinterpret_cast<uint32_t*>(line) + (bitpos >> 5);
+    const int sh = (int)(bitpos & 31);
+    atomicOr(w, val << sh);
+    if (sh + nbits > 32) atomicOr(w + 1, val >> (32 - sh));
+}
+
+__device__ __forceinline__ uint32_t get_bits(const uint8_t* line, int64_t bitpos, int nbits) {
+    const uint32_t* w = reinterpret_cast<const uint32_t*>(line) + (bitpos >> 5);
+    const int sh = (int)(bitpos & 31);
+    uint32_t v = w[0] >> sh;
+    if (sh + nbits > 32) v |= w[1] << (32 - sh);
+    return v & ((1u << nbits) - 1u);
+}
+
+// One thread per (line, k1-block).
+template <typename T>
+__global__ void __launch_bounds__(kGenThreads)
+quant_general_kernel(const T* x, T* y, int64_t nlines, int64_t len, int64_t line_stride, int64_t elem_stride,
+                     int64_t nblocks, int64_t total_rounded, bdr_planes_t out, bool pack, QParams qp, double* sums) {
+    double e2 = 0.0, s2 = 0.0;
+    const int nsub = qp.k1 / qp.k2;
+    for (int64_t g = (int64_t)blockIdx.x * kGenThreads + threadIdx.x; g < total_rounded;
+         g += (int64_t)gridDim.x * kGenThreads) {
+        if (g >= nlines * nblocks) continue;
+        const int64_t line = g / nblocks, b = g - line * nblocks;
+        const int64_t i0 = b * qp.k1;
+        const int n = (int)min((int64_t)qp.k1, len - i0);
+        const T* px = x + line * line_stride + i0 * elem_stride;
+        T* py = y ? y + line * line_stride + i0 * elem_stride : nullptr;
+        int F = 0;
+        for (int i = 0; i < n; ++i) F = max(F, exp_field(Elem<T>::load_bits(px + i * elem_stride)));
+        if (pack) out.exps[line * out.ld_exps + b] = (uint8_t)F;
+        for (int j = 0; j < nsub; ++j) {
+            int Fj = 0;
+            for (int i = j * qp.k2; i < (j + 1) * qp.k2 && i < n; ++i)
+                Fj = max(Fj, exp_field(Elem<T>::load_bits(px + i * elem_stride)));
+            const int tau = F == 255 ? 0 : min(F - Fj, qp.beta);
+            if (pack && qp.d2) or_bits(out.micro + line * out.ld_micro, (b * nsub + j) * (int64_t)qp.d2, qp.d2, (uint32_t)tau);
+            for (int i = j * qp.k2; i < (j + 1) * qp.k2 && i < n; ++i) {
+                const uint32_t u = Elem<T>::load_bits(px + i * elem_stride);
+                uint32_t q = 0, yb = 0x7FC00000u;
+                if (F != 255) quant_elem_exact(u, F, tau, qp, q, yb);
+                const uint32_t code = F == 255 ? 0u : (((u >> 31) << qp.m) | q);
+                if (py) Elem<T>::store_bits(py + i * elem_stride, yb);
+                if (pack) or_bits(out.elems + line * out.ld_elems, (i0 + i) * (int64_t)(qp.m + 1), qp.m + 1, code);
+                if (sums) {
+                    const double de = (double)__uint_as_float(yb) - (double)__uint_as_float(u);
+                    const double dx = (double)__uint_as_float(u);
+                    e2 = fma(de, de, e2);
+                    s2 = fma(dx, dx, s2);
+                }
+            }
+        }
+    }
+    if (sums) block_accumulate_sums(e2, s2, sums);
+}
+
+// One thread per element.
+template <typename T>
+__global__ void __launch_bounds__(kGenThreads)
+unpack_general_kernel(bdr_planes_t in, T* y, int64_t nlines, int64_t len, int64_t line_stride, int64_t elem_stride,
+                      int axis, QParams qp) {
+    const int nsub = qp.k1 / qp.k2;
+    const int64_t total = nlines * len;
+    for (int64_t g = (int64_t)blockIdx.x * kGenThreads + threadIdx.x; g < total; g += (int64_t)gridDim.x * kGenThreads) {
+        // consecutive threads walk the contiguous dimension of y
+        const int64_t line = axis == 1 ? g / len : g % nlines;
+        const int64_t i = axis == 1 ? g % len : g / nlines;
+        const int64_t b = i / qp.k1;
+        const int F = in.exps[line * in.ld_exps + b];
+        uint32_t yb = 0x7FC00000u;
+        if (F != 255) {
+            const int64_t j = b * nsub + (i - b * qp.k1) / qp.k2;
+            const int tau = qp.d2 ? (int)get_bits(in.micro + line * in.ld_micro, j * (int64_t)qp.d2, qp.d2) : 0;
+            const uint32_t code = get_bits(in.elems + line * in.ld_elems, i * (int64_t)(qp.m + 1), qp.m + 1);
+            const uint32_t q = code & qp.qmax;
+            const int p = max(F - 127 - tau - (qp.m - 1), -149);
+            yb = __float_as_uint(__fmul_rn(__uint2float_rn(q), __uint_as_float(pow2_bits(p)))) | ((code >> qp.m) << 31);
+        }
+        Elem<T>::store_bits(y + line * line_stride + i * elem_stride, yb);
+    }
+}
+
+template <typename T>
+int quant_general(const T* x, T* y, int64_t rows, int64_t cols, int64_t ld, int axis, const bdr_planes_t* out,
+                  const QParams& qp, double* sums, cudaStream_t st) {
+    const int64_t nlines = axis == 1 ? rows : cols, len = axis == 1 ? cols : rows;
+    const int64_t line_stride = axis == 1 ? ld : 1, elem_stride = axis == 1 ? 1 : ld;
+    const int64_t nblocks = (len + qp.k1 - 1) / qp.k1;
+    bdr_planes_t pl = {};
+    if (out) {
+        pl = *out;
+        if (cudaMemsetAsync(pl.exps, 0, (size_t)(nlines * pl.ld_exps), st) != cudaSuccess) return BDR_ERR_CUDA;
+        if (qp.d2 && pl.micro && cudaMemsetAsync(pl.micro, 0, (size_t)(nlines * pl.ld_micro), st) != cudaSuccess)
+            return BDR_ERR_CUDA;
+        if (cudaMemsetAsync(pl.elems, 0, (size_t)(nlines * pl.ld_elems), st) != cudaSuccess) return BDR_ERR_CUDA;
+    }
+    const int64_t total = nlines * nblocks;
+    if (total == 0) return BDR_OK;
+    const int64_t rounded = (total + kGenThreads - 1) / kGenThreads * kGenThreads;
+    const int grid = (int)max((int64_t)1, min(rounded / kGenThreads, (int64_t)sm_count() * 16));
+    quant_general_kernel<T><<<grid, kGenThreads, 0, st>>>(x, y, nlines, len, line_stride, elem_stride, nblocks, rounded,
+                                                          pl, out != nullptr, qp, sums);
+    return cudaGetLastError() == cudaSuccess ? BDR_OK : BDR_ERR_CUDA;
+}
+
+template <typename T>
+int unpack_general(const bdr_planes_t& in, T* y, int64_t rows, int64_t cols, int64_t ld, int axis, const QParams& qp,
+                   cudaStream_t st) {
+    const int64_t nlines = axis == 1 ? rows : cols, len = axis == 1 ? cols : rows;
+    const int64_t line_stride = axis == 1 ? ld : 1, elem_stride = axis == 1 ? 1 : ld;
+    const int64_t total = nlines * len;
+    if (total == 0) return BDR_OK;
+    const int grid = (int)max((int64_t)1, min((total + kGenThreads - 1) / kGenThreads, (int64_t)sm_count() * 16));
+    unpack_general_kernel<T><<<grid, kGenThreads, 0, st>>>(in, y, nlines, len, line_stride, elem_stride, axis, qp);
+    return cudaGetLastError() == cudaSuccess ? BDR_OK : BDR_ERR_CUDA;
+}
+
+template int quant_general<float>(const float*, float*, int64_t, int64_t, int64_t, int, const bdr_planes_t*,
+                                  const QParams&, double*, cudaStream_t);
+template int quant_general<__nv_bfloat16>(const __nv_bfloat16*, __nv_bfloat16*, int64_t, int64_t, int64_t, int,
+                                          const bdr_planes_t*, const QParams&, double*, cudaStream_t);
+template int unpack_general<float>(const bdr_planes_t&, float*, int64_t, int64_t, int64_t, int, const QParams&,
+                                   cudaStream_t);
+template int unpack_general<__nv_bfloat16>(const bdr_planes_t&, __nv_bfloat16*, int64_t, int64_t, int64_t, int,
+                                           const QParams&, cudaStream_t);
+
+}  // namespace bdr

@@ -1,0 +1,45 @@
+// Host-side declarations shared by the translation units of the library (not part of the ABI).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "bdr.h"
+
+namespace bdr {
+
+struct QParams;
+
+int sm_count();  // SMs of the current device (cached per device)
+
+// axis-1 kernels (bdr_row.cu); BDR_ERR_UNSUPPORTED = not covered, use the general kernel
+template <typename T>
+int quant_rowwise(const T* x, T* y, int64_t rows, int64_t cols, int64_t ld, const QParams& qp, double* sums,
+                  cudaStream_t st);
+template <typename T>
+int pack_rowwise_mx(const T* x, T* y, int64_t rows, int64_t cols, int64_t ld, const bdr_planes_t& out,
+                    const QParams& qp, double* sums, cudaStream_t st);
+
+// axis-0 fast path for k1 = 16, k2 = 2 (bdr_col.cu)
+template <typename T>
+int quant_colwise_mx(const T* x, T* y, int64_t rows, int64_t cols, int64_t ld, const bdr_planes_t* out,
+                     const QParams& qp, double* sums, cudaStream_t st);
+
+// general kernels: any axis, any POW2 configuration, any alignment (bdr_general.cu)
+template <typename T>
+int quant_general(const T* x, T* y, int64_t rows, int64_t cols, int64_t ld, int axis, const bdr_planes_t* out,
+                  const QParams& qp, double* sums, cudaStream_t st);
+template <typename T>
+int unpack_general(const bdr_planes_t& in, T* y, int64_t rows, int64_t cols, int64_t ld, int axis, const QParams& qp,
+                   cudaStream_t st);
+
+// unpack fast paths for k1 = 16, k2 = 2 (bdr_unpack.cu)
+template <typename T>
+int unpack_rowwise_mx(const bdr_planes_t& in, T* y, int64_t rows, int64_t cols, int64_t ld, const QParams& qp,
+                      cudaStream_t st);
+template <typename T>
+int unpack_colwise_mx(const bdr_planes_t& in, T* y, int64_t rows, int64_t cols, int64_t ld, const QParams& qp,
+                      cudaStream_t st);
+
+}  // namespace bdr

@@ -1,0 +1,193 @@
+"""GPU parity: the CUDA path through the C ABI against the oracle, element by element.
+
+Bit-exact for dequantized tensors and packed bytes; QSNR within 1e-6 dB relative.
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import oracle as orc
+from paper_2302_08007_b200 import binding as bdr
+from paper_2302_08007_b200 import synth
+from tests import helpers as H
+
+pytestmark = pytest.mark.gpu
+
+Cfg = bdr.Config
+
+# every (k1, k2, d2) family the sweep uses plus the degenerate corners, a few m each
+ROW_CONFIGS = [Cfg(k1, 8, k2, d2, m) for (k1, k2, d2) in
+               [(1, 1, 0), (2, 1, 1), (2, 2, 2), (4, 2, 1), (8, 1, 2), (8, 8, 1), (16, 2, 1), (16, 1, 0), (16, 4, 2),
+                (16, 8, 3), (16, 16, 1), (32, 2, 1), (64, 8, 2), (128, 1, 1), (256, 4, 2), (512, 2, 1), (1024, 8, 1),
+                (1024, 1, 2)]
+               for m in (1, 4, 8)]
+MX = {"MX4": bdr.MX4, "MX6": bdr.MX6, "MX9": bdr.MX9}
+
+
+def run_quant(cfg, x_host, dtype, axis=1, ld=None, want_y=True, inplace=False):
+    x = H.host_to_device(x_host, dtype, ld)
+    y = x if inplace else (torch.empty_like(x) if ld is None else H.host_to_device(np.zeros_like(x_host), dtype, ld))
+    sums = torch.zeros(2, dtype=torch.float64, device="cuda")
+    bdr.bdr_quant_dequant(cfg, x, y if want_y else None, axis=axis, qsnr_sums=sums)
+    torch.cuda.synchronize()
+    return (H.device_to_host_f32(y) if want_y else None), sums.cpu().numpy()
+
+
+@pytest.mark.parametrize("cfg", ROW_CONFIGS, ids=str)
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_rowwise_quant_dequant_matches_oracle(cfg, dtype):
+    # 3 rows x 2560 columns spans several CTAs' worth of slices; 2560 is a multiple of every k1 <= 512
+    for kind, rows, cols in (("normal", 3, 2560), ("edge", 5, 2048), ("laplace_outliers", 2, 1024)):
+        x = H.make_input(kind, rows, cols, dtype, seed=11)
+        y, sums = run_quant(cfg, x, dtype)
+        want, so = orc.quant_dequant(H.to_orc(cfg), x)
+        H.assert_bits_equal(y, want, "%s %s %s" % (cfg, dtype, kind))
+        H.assert_qsnr_close(sums, so, "%s %s %s" % (cfg, dtype, kind))
+
+
+@pytest.mark.parametrize("cfg", [bdr.MX6, bdr.MX9, Cfg(64, 8, 4, 2, 3), Cfg(1024, 8, 2, 1, 5), Cfg(8, 8, 2, 1, 4)], ids=str)
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_rowwise_ragged_shapes_and_pitches(cfg, dtype):
+    for rows, cols, ld in ((1, 1, None), (7, 100, None), (4, 1000, 1003), (3, 16, 24), (2, 1037, 1040), (1, 5000, None)):
+        x = H.make_input("normal", rows, cols, dtype, seed=rows * 1000 + cols)
+        y, sums = run_quant(cfg, x, dtype, ld=ld)
+        want, so = orc.quant_dequant(H.to_orc(cfg), x)
+        H.assert_bits_equal(y, want, "%s %s %dx%d ld=%s" % (cfg, dtype, rows, cols, ld))
+        H.assert_qsnr_close(sums, so)
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_extreme_exponents_signed_zeros_and_ties_away(dtype):
+    for kind in ("tiny", "huge", "edge"):
+        x = H.make_input(kind, 4, 1024, dtype, seed=5)
+        for cfg in (bdr.MX4, bdr.MX9, Cfg(16, 8, 2, 3, 8), Cfg(32, 8, 1, 2, 6, bdr.SCALE_POW2, bdr.ROUND_NEAREST_AWAY),
+                    Cfg(16, 8, 2, 1, 4, bdr.SCALE_POW2, bdr.ROUND_NEAREST_AWAY)):
+            y, sums = run_quant(cfg, x, dtype)
+            want, so = orc.quant_dequant(H.to_orc(cfg), x)
+            H.assert_bits_equal(y, want, "%s %s %s" % (cfg, dtype, kind))
+            H.assert_qsnr_close(sums, so, "%s %s %s" % (cfg, dtype, kind))
+
+
+def test_nonfinite_inputs_poison_only_their_block():
+    x = H.make_input("normal", 2, 512, "f32", seed=9)
+    x[0, 37] = np.inf
+    x[1, 300] = np.nan
+    for cfg in (bdr.MX6, Cfg(64, 8, 2, 1, 4)):
+        y, sums = run_quant(cfg, x, "f32")
+        want, _ = orc.quant_dequant(H.to_orc(cfg), x)
+        assert np.array_equal(np.isnan(y), np.isnan(want))
+        ok = ~np.isnan(want)
+        H.assert_bits_equal(y[ok], want[ok])
+        assert np.isnan(sums).any()
+
+
+def test_in_place_and_sums_only():
+    x = H.make_input("normal", 8, 2048, "f32", seed=3)
+    want, so = orc.quant_dequant(H.to_orc(bdr.MX6), x)
+    y, sums = run_quant(bdr.MX6, x, "f32", inplace=True)
+    H.assert_bits_equal(y, want)
+    _, sums2 = run_quant(bdr.MX6, x, "f32", want_y=False)
+    H.assert_qsnr_close(sums2, so)
+    assert np.array_equal(sums, sums2) or np.allclose(sums, sums2, rtol=1e-12)
+
+
+def test_empty_tensors_are_no_ops():
+    for rows, cols in ((0, 64), (4, 0)):
+        x = torch.empty((rows, cols), device="cuda")
+        bdr.bdr_quant_dequant(bdr.MX6, x, torch.empty_like(x))
+    torch.cuda.synchronize()
+
+
+# ---- the first BASELINE configuration, complete -------------------------------------------------------
+def test_config1_mx6_vector_of_65536():
+    x = synth.normal(65536, seed=0).reshape(1, -1)
+    xd = torch.from_numpy(x).cuda()
+    planes = bdr.alloc_planes(bdr.MX6, 1, 65536)
+    assert [p.shape[1] for p in (planes.exps, planes.micro, planes.elems)] == [4096, 4096, 40960]
+    y = torch.empty_like(xd)
+    sums = torch.zeros(2, dtype=torch.float64, device="cuda")
+    bdr.bdr_pack(bdr.MX6, xd, planes, y_dq=y, qsnr_sums=sums)
+    torch.cuda.synchronize()
+    want, so = orc.quant_dequant(orc.MX6, x)
+    H.assert_bits_equal(y.cpu().numpy(), want)
+    H.assert_planes_equal(H.planes_to_host(planes), orc.pack(orc.MX6, x))
+    H.assert_qsnr_close(sums.cpu().numpy(), so)
+    assert abs(orc.qsnr_db(*sums.cpu().numpy()) - 28.3) < 0.1
+
+
+# ---- pack / unpack -----------------------------------------------------------------------------------------
+@pytest.mark.parametrize("name", list(MX))
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("axis", [1, 0])
+def test_pack_and_unpack_mx_formats(name, dtype, axis):
+    cfg = MX[name]
+    # fast-path shapes (multiples of 512) and shapes that force the general kernels
+    for kind, rows, cols in (("laplace_outliers", 512, 1024), ("edge", 1024, 512), ("normal", 40, 100), ("normal", 33, 512)):
+        x = H.make_input(kind, rows, cols, dtype, seed=21)
+        xd = H.host_to_device(x, dtype)
+        planes = bdr.alloc_planes(cfg, rows, cols, axis)
+        y = torch.empty_like(xd)
+        sums = torch.zeros(2, dtype=torch.float64, device="cuda")
+        bdr.bdr_pack(cfg, xd, planes, axis=axis, y_dq=y, qsnr_sums=sums)
+        back = torch.full_like(xd, 7.0)
+        bdr.bdr_unpack(cfg, planes, back, axis=axis)
+        torch.cuda.synchronize()
+        what = "%s %s axis=%d %s %dx%d" % (name, dtype, axis, kind, rows, cols)
+        want, so = orc.quant_dequant(H.to_orc(cfg), x, axis=axis)
+        H.assert_bits_equal(H.device_to_host_f32(y), want, what + " y_dq")
+        H.assert_planes_equal(H.planes_to_host(planes), orc.pack(H.to_orc(cfg), x, axis=axis), what)
+        H.assert_bits_equal(H.device_to_host_f32(back), want, what + " unpack")
+        H.assert_qsnr_close(sums.cpu().numpy(), so, what)
+
+
+@pytest.mark.parametrize("cfg", [Cfg(8, 8, 4, 2, 3), Cfg(32, 8, 1, 3, 6), Cfg(16, 8, 16, 0, 7), Cfg(16, 8, 2, 2, 8),
+                                 Cfg(16, 8, 2, 0, 3), Cfg(1024, 8, 8, 1, 1), Cfg(1, 8, 1, 0, 8)], ids=str)
+def test_pack_and_unpack_general_configs(cfg):
+    for axis in (1, 0):
+        for rows, cols in ((6, 200), (512, 512)):
+            x = H.make_input("edge", rows, cols, "f32", seed=31)
+            xd = H.host_to_device(x, "f32")
+            planes = bdr.alloc_planes(cfg, rows, cols, axis)
+            for t in (planes.exps, planes.micro, planes.elems):
+                t.fill_(0xAB)                                   # every byte up to the pitch must be rewritten
+            bdr.bdr_pack(cfg, xd, planes, axis=axis)
+            back = torch.empty_like(xd)
+            bdr.bdr_unpack(cfg, planes, back, axis=axis)
+            torch.cuda.synchronize()
+            want, _ = orc.quant_dequant(H.to_orc(cfg), x, axis=axis)
+            H.assert_planes_equal(H.planes_to_host(planes), orc.pack(H.to_orc(cfg), x, axis=axis), str(cfg))
+            H.assert_bits_equal(back.cpu().numpy(), want, str(cfg))
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_columnwise_quant_dequant(dtype):
+    for cfg in (bdr.MX6, bdr.MX9, Cfg(32, 8, 4, 2, 3), Cfg(8, 8, 1, 1, 5)):
+        for rows, cols, ld in ((512, 256, None), (100, 72, None), (64, 200, 208)):
+            x = H.make_input("laplace_outliers", rows, cols, dtype, seed=41)
+            y, sums = run_quant(cfg, x, dtype, axis=0, ld=ld)
+            want, so = orc.quant_dequant(H.to_orc(cfg), x, axis=0)
+            H.assert_bits_equal(y, want, "%s %s %dx%d" % (cfg, dtype, rows, cols))
+            H.assert_qsnr_close(sums, so)
+
+
+# ---- host-side error paths: nothing is launched -----------------------------------------------------------
+def test_argument_errors_are_reported_not_launched():
+    x = torch.zeros((4, 64), device="cuda")
+    with pytest.raises(bdr.BdrError) as e:
+        bdr.bdr_quant_dequant(Cfg(16, 8, 3, 1, 4), x, x)                 # k2 does not divide k1
+    assert e.value.status == -2
+    with pytest.raises(bdr.BdrError) as e:
+        bdr.bdr_quant_dequant(Cfg(16, 7, 2, 1, 4), x, x)                 # d1 must be 8
+    assert e.value.status == -2
+    with pytest.raises(bdr.BdrError) as e:
+        bdr.bdr_quant_dequant(Cfg(24, 8, 2, 1, 4), x, x)                 # legal BDR, no kernel
+    assert e.value.status == -3
+    with pytest.raises(bdr.BdrError) as e:
+        bdr.bdr_quant_dequant(bdr.MX6, x, None)                          # nothing to produce
+    assert e.value.status == -1
+    planes = bdr.alloc_planes(bdr.MX6, 4, 64)
+    small = bdr.Planes(planes.exps, planes.micro, torch.empty((4, 16), dtype=torch.uint8, device="cuda"))
+    with pytest.raises(bdr.BdrError) as e:
+        bdr.bdr_pack(bdr.MX6, x, small)
+    assert e.value.status == -5
+    torch.cuda.synchronize()
