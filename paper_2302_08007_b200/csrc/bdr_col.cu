@@ -42,31 +42,66 @@ struct ColStage {
     uint8_t micro[kTileBlocks][kTileCols][3];
 };
 
+// one row's pair of columns as fetched (4 bytes of bf16, 8 bytes of fp32)
+template <typename T> struct PairWord;
+template <> struct PairWord<float> {
+    using type = uint2;
+    __device__ static __forceinline__ void fetch(type* smem, const float* g) { cp_async8(smem, g); }
+    __device__ static __forceinline__ void split(type w, uint32_t& a, uint32_t& b) { a = w.x; b = w.y; }
+};
+template <> struct PairWord<__nv_bfloat16> {
+    using type = uint32_t;
+    __device__ static __forceinline__ void fetch(type* smem, const __nv_bfloat16* g) { cp_async4(smem, g); }
+    __device__ static __forceinline__ void split(type w, uint32_t& a, uint32_t& b) { a = w << 16; b = w & 0xFFFF0000u; }
+};
+template <typename T> struct ColRing {
+    static constexpr int kStages = sizeof(T) == 2 ? 3 : 2;
+    static constexpr size_t kBytes = (size_t)kStages * kSlice * kColThreads * sizeof(typename PairWord<T>::type);
+};
+
 template <typename T, int W>  // W = m + 1 when packing, 0 when only y / sums are wanted
-__global__ void __launch_bounds__(kColThreads)
+__global__ void __launch_bounds__(kColThreads, 2)
 quant_colwise_mx_kernel(const T* x, T* y, int64_t rows, int64_t cols, int64_t ld, bdr_planes_t out, QParams qp,
                         double* sums) {
-    __shared__ __align__(16) ColStage<W> st;
+    using PW = typename PairWord<T>::type;
+    constexpr int kStages = ColRing<T>::kStages;
+    extern __shared__ __align__(16) uint8_t dyn_smem[];
+    PW* ring = reinterpret_cast<PW*>(dyn_smem);  // [stage][row of the block][thread]
+    ColStage<W>& st = *reinterpret_cast<ColStage<W>*>(dyn_smem + ColRing<T>::kBytes);
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int64_t c0 = (int64_t)blockIdx.x * kTileCols;
     const int64_t tb0 = (int64_t)blockIdx.y * kTileBlocks;
     const int64_t nblocks = rows / kSlice;
     const int64_t c = c0 + 2 * lane;
     double e2 = 0.0, s2 = 0.0;
+    auto issue = [&](int bl, int stg) {
+        if (bl < kTileBlocks && tb0 + bl < nblocks) {
+            const T* px = x + (tb0 + bl) * kSlice * ld + c;
+#pragma unroll
+            for (int r = 0; r < kSlice; ++r) PairWord<T>::fetch(&ring[(stg * kSlice + r) * kColThreads + threadIdx.x], px + r * ld);
+        }
+        cp_async_commit();
+    };
+#pragma unroll
+    for (int s = 0; s < kStages - 1; ++s) issue(warp + s * kColWarps, s);
+    int rs = 0;
     for (int bl = warp; bl < kTileBlocks; bl += kColWarps) {
         const int64_t b = tb0 + bl;
         if (b >= nblocks) break;
+        issue(bl + (kStages - 1) * kColWarps, (rs + kStages - 1) % kStages);
+        cp_async_wait<kStages - 1>();
         uint32_t u[2][kSlice];
-        const T* px = x + b * kSlice * ld + c;
 #pragma unroll
-        for (int r = 0; r < kSlice; ++r) load_pair(px + r * ld, u[0][r], u[1][r]);
+        for (int r = 0; r < kSlice; ++r)
+            PairWord<T>::split(ring[(rs * kSlice + r) * kColThreads + threadIdx.x], u[0][r], u[1][r]);
+        rs = (rs + 1) % kStages;
         uint32_t yb[2][kSlice];
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
             uint32_t code[kSlice], tau[kSlice / 2];
-            int fj[kSlice / 2], fb[1];
+            uint32_t fj[kSlice / 2], fb[1];
             subblock_exponents<2>(u[h], fj);
-            int F = 0;
+            uint32_t F = 0;
 #pragma unroll
             for (int j = 0; j < kSlice / 2; ++j) F = max(F, fj[j]);
             fb[0] = F;
@@ -78,7 +113,7 @@ quant_colwise_mx_kernel(const T* x, T* y, int64_t rows, int64_t cols, int64_t ld
 #pragma unroll
                 for (int k = 0; k < ColStage<W>::kW; ++k)
                     st.elems[bl][2 * lane + h][k] = (uint16_t)(words[k >> 1] >> ((k & 1) * 16));
-                st.exps[bl][2 * lane + h] = (uint8_t)F;
+                st.exps[bl][2 * lane + h] = (uint8_t)(F >> 23);
                 uint32_t mbits = 0;
 #pragma unroll
                 for (int j = 0; j < kSlice / 2; ++j) mbits |= tau[j] << (j * qp.d2);
@@ -194,7 +229,14 @@ static int launch_col(const T* x, T* y, int64_t rows, int64_t cols, int64_t ld, 
     const dim3 grid((unsigned)(cols / kTileCols), (unsigned)((rows / kSlice + kTileBlocks - 1) / kTileBlocks));
     bdr_planes_t pl = {};
     if (out) pl = *out;
-    quant_colwise_mx_kernel<T, W><<<grid, kColThreads, 0, st>>>(x, y, rows, cols, ld, pl, qp, sums);
+    auto kern = quant_colwise_mx_kernel<T, W>;
+    const size_t smem = ColRing<T>::kBytes + (W > 0 ? sizeof(ColStage<W>) : 16);
+    static bool attr_done = false;
+    if (!attr_done) {
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return BDR_ERR_CUDA;
+        attr_done = true;
+    }
+    kern<<<grid, kColThreads, smem, st>>>(x, y, rows, cols, ld, pl, qp, sums);
     return cudaGetLastError() == cudaSuccess ? BDR_OK : BDR_ERR_CUDA;
 }
 

@@ -56,6 +56,8 @@ __device__ __forceinline__ void quant_elem_exact(uint32_t u, int F, int tau, con
 // multiple of 2^p (nearest, ties to even) and leaves q in the low mantissa bits of the sum.
 // Valid while C is finite, i.e. F <= kFastMaxF.
 constexpr int kFastMaxF = 230;
+// shared-exponent range in which the Eq. 3 terms of a block are summed in fp32 before widening
+constexpr int kSumMinF = 96, kSumMaxF = 158;
 
 struct SubScale {
     uint32_t Cbits;  // bits of C
@@ -148,6 +150,47 @@ __device__ __forceinline__ void store_slice_guarded(T* p, int64_t stride, int n,
         if (i < n) Elem<T>::store_bits(p + i * stride, y[i]);
 }
 
+// ---- per-thread asynchronous prefetch ring (global -> shared, read back by the issuing thread) --------
+// A thread queues 16-byte copies several loop iterations ahead and later reads only what it queued
+// itself, so a wait_group is all the synchronisation needed and the bytes in flight per SM no longer
+// depend on how many registers the kernel uses.
+__device__ __forceinline__ void cp_async16(void* smem, const void* gmem) {
+    const uint32_t s = (uint32_t)__cvta_generic_to_shared(smem);
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(s), "l"(gmem) : "memory");
+}
+__device__ __forceinline__ void cp_async8(void* smem, const void* gmem) {
+    const uint32_t s = (uint32_t)__cvta_generic_to_shared(smem);
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"(s), "l"(gmem) : "memory");
+}
+__device__ __forceinline__ void cp_async4(void* smem, const void* gmem) {
+    const uint32_t s = (uint32_t)__cvta_generic_to_shared(smem);
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(s), "l"(gmem) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
+// 16-byte words of one slice (as fetched) -> fp32 bit patterns
+template <typename T> struct SliceWords;
+template <> struct SliceWords<float> {
+    static constexpr int kVecs = 4;
+    __device__ static __forceinline__ void expand(const uint4 (&w)[4], uint32_t (&u)[kSlice]) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) { u[4 * i] = w[i].x; u[4 * i + 1] = w[i].y; u[4 * i + 2] = w[i].z; u[4 * i + 3] = w[i].w; }
+    }
+};
+template <> struct SliceWords<__nv_bfloat16> {
+    static constexpr int kVecs = 2;
+    __device__ static __forceinline__ void expand(const uint4 (&w)[2], uint32_t (&u)[kSlice]) {
+#pragma unroll
+        for (int i = 0; i < 2; ++i) {
+            const uint32_t ws[4] = {w[i].x, w[i].y, w[i].z, w[i].w};
+#pragma unroll
+            for (int k = 0; k < 4; ++k) { u[8 * i + 2 * k] = ws[k] << 16; u[8 * i + 2 * k + 1] = ws[k] & 0xFFFF0000u; }
+        }
+    }
+};
+
 // ---- block reduction of the two Eq. 3 sums ------------------------------------------------------
 __device__ __forceinline__ double warp_sum(double v) {
 #pragma unroll
@@ -176,71 +219,127 @@ __device__ __forceinline__ void block_accumulate_sums(double err2, double sig2, 
 namespace bdr {
 
 // ---- one 16-element slice ------------------------------------------------------------------------
-// Sub-block maxima of the exponent fields (k2 <= 16) and, for k1 < 16, block maxima.
+// Exponent fields are kept in place (bits 30..23, "e23" values) so no per-element shift is needed.
+constexpr uint32_t kExpMask = 0x7F800000u;
+
+// Sub-block maxima of the exponent fields (k2 <= 16), as e23 values.
 template <int K2>
-__device__ __forceinline__ void subblock_exponents(const uint32_t (&u)[kSlice], int (&fj)[kSlice / K2]) {
+__device__ __forceinline__ void subblock_exponents(const uint32_t (&u)[kSlice], uint32_t (&ej)[kSlice / K2]) {
 #pragma unroll
     for (int j = 0; j < kSlice / K2; ++j) {
-        int f = 0;
+        uint32_t e = 0;
 #pragma unroll
-        for (int i = 0; i < K2; ++i) f = max(f, exp_field(u[j * K2 + i]));
-        fj[j] = f;
+        for (int i = 0; i < K2; ++i) e = max(e, u[j * K2 + i] & kExpMask);
+        ej[j] = e;
     }
 }
 
-// Quantize the slice.  fb[] holds the shared exponent of each k1-block touching the slice
-// (K1S = min(k1,16) elements each; for k1 >= 16 the single entry is the block's exponent after
-// any cross-lane reduction).  Produces dequantized bit patterns, element codes (sign<<m | q),
-// sub-block shifts, and adds this slice's Eq. 3 terms to e2 / s2 when WANT_SUMS.
+// Exact path for one slice: ties-away rounding, or a block that holds Inf/NaN.
 template <int K2, int K1S, bool WANT_SUMS>
-__device__ __forceinline__ void quantize_slice(const uint32_t (&u)[kSlice], const int (&fj)[kSlice / K2],
-                                               const int (&fb)[kSlice / K1S], const QParams& qp,
-                                               uint32_t (&yb)[kSlice], uint32_t (&code)[kSlice],
-                                               uint32_t (&tau)[kSlice / K2], double& e2, double& s2) {
+__device__ __forceinline__ void quantize_slice_exact(const uint32_t (&u)[kSlice], const uint32_t (&ej)[kSlice / K2],
+                                                  const uint32_t (&eb)[kSlice / K1S], const QParams& qp,
+                                                  uint32_t (&yb)[kSlice], uint32_t (&code)[kSlice],
+                                                  uint32_t (&tau)[kSlice / K2], double& e2, double& s2) {
 #pragma unroll
     for (int j = 0; j < kSlice / K2; ++j) {
-        const int F = fb[(j * K2) / K1S];
-        const int t = min(F - fj[j], qp.beta);
+        const int F = (int)(eb[(j * K2) / K1S] >> 23);
+        const int t = F == 255 ? 0 : min(F - (int)(ej[j] >> 23), qp.beta);
         tau[j] = (uint32_t)t;
-        if (F == 255) {  // Inf/NaN somewhere in the block: the whole block decodes to NaN
-            tau[j] = 0;
 #pragma unroll
-            for (int i = 0; i < K2; ++i) {
-                yb[j * K2 + i] = 0x7FC00000u;
-                code[j * K2 + i] = 0;
-                if (WANT_SUMS) { e2 = __longlong_as_double(0x7FF8000000000000ll); s2 = e2; }
-            }
-        } else if (qp.rounding == BDR_ROUND_NEAREST_EVEN && F <= kFastMaxF) {
-            const SubScale ss = make_subscale(F, t, qp.m);
-#pragma unroll
-            for (int i = 0; i < K2; ++i) {
-                const int k = j * K2 + i;
-                uint32_t q;
-                float ax, aq;
-                quant_elem_fast(u[k], ss, qp.qmax, q, yb[k], ax, aq);
-                code[k] = ((u[k] >> 31) << qp.m) | q;
-                if (WANT_SUMS) {
-                    const double de = (double)__fsub_rn(aq, ax), dx = (double)ax;  // difference is exact in fp32
-                    e2 = fma(de, de, e2);
-                    s2 = fma(dx, dx, s2);
-                }
-            }
-        } else {
-#pragma unroll
-            for (int i = 0; i < K2; ++i) {
-                const int k = j * K2 + i;
-                uint32_t q;
-                quant_elem_exact(u[k], F, t, qp, q, yb[k]);
-                code[k] = ((u[k] >> 31) << qp.m) | q;
-                if (WANT_SUMS) {
-                    const double de = (double)__uint_as_float(yb[k]) - (double)__uint_as_float(u[k]);
-                    const double dx = (double)__uint_as_float(u[k]);
-                    e2 = fma(de, de, e2);
-                    s2 = fma(dx, dx, s2);
-                }
+        for (int i = 0; i < K2; ++i) {
+            const int k = j * K2 + i;
+            uint32_t q = 0, y = 0x7FC00000u;
+            if (F != 255) quant_elem_exact(u[k], F, t, qp, q, y);
+            yb[k] = y;
+            code[k] = F == 255 ? 0u : (((u[k] >> 31) << qp.m) | q);
+            if (WANT_SUMS) {
+                const double de = (double)__uint_as_float(y) - (double)__uint_as_float(u[k]);
+                const double dx = (double)__uint_as_float(u[k]);
+                e2 = fma(de, de, e2);
+                s2 = fma(dx, dx, s2);
             }
         }
     }
+}
+
+// Quantize the slice.  eb[] holds the shared exponent (e23) of each k1-block touching the slice
+// (K1S = min(k1,16) elements each; for k1 >= 16 the single entry is the block's exponent after any
+// cross-lane reduction).  Produces dequantized bit patterns, element codes (sign<<m | q), sub-block
+// shifts, and adds this slice's Eq. 3 terms to e2 / s2 when WANT_SUMS.
+//
+// Fast path (ties-to-even, finite block): work in the block-normalised domain a = |x| * 2^(127-F),
+// a < 2.  There the unit of q is 2^(-(m-1)-tau), so adding C = 1.5 * 2^(23-(m-1)-tau) makes the fp32
+// adder round a to a multiple of that unit (nearest, ties to even) and leaves q in the low
+// mantissa bits; C depends on tau only.  Every scaling is by a power of two and therefore exact
+// (an element so small that a underflows rounds to q = 0 either way).  The Eq. 3 terms are summed
+// in fp32 in the normalised domain (at most 16 terms of magnitude <= 4) and widened once per block
+// with the exact factor 2^(2F-254).
+template <int K2, int K1S, bool WANT_SUMS>
+__device__ __forceinline__ void quantize_slice(const uint32_t (&u)[kSlice], const uint32_t (&ej)[kSlice / K2],
+                                               const uint32_t (&eb)[kSlice / K1S], const QParams& qp,
+                                               uint32_t (&yb)[kSlice], uint32_t (&code)[kSlice],
+                                               uint32_t (&tau)[kSlice / K2], double& e2, double& s2) {
+    uint32_t emax = eb[0];
+#pragma unroll
+    for (int b = 1; b < kSlice / K1S; ++b) emax = max(emax, eb[b]);
+    if (qp.rounding != BDR_ROUND_NEAREST_EVEN || emax == kExpMask) {
+        quantize_slice_exact<K2, K1S, WANT_SUMS>(u, ej, eb, qp, yb, code, tau, e2, s2);
+        return;
+    }
+    const uint32_t c_base = ((uint32_t)(127 + 23 - (qp.m - 1)) << 23) | 0x400000u;
+    const uint32_t beta23 = (uint32_t)qp.beta << 23;
+#pragma unroll
+    for (int b = 0; b < kSlice / K1S; ++b) {
+        const uint32_t F23 = eb[b];
+        const float K = __uint_as_float(max(0x7F000000u - F23, 0x00400000u));  // 2^(127-F)
+        const float Kinv = __uint_as_float(max(F23, 0x00400000u));            // 2^(F-127)
+        float pe = 0.f, ps = 0.f;
+#pragma unroll
+        for (int jj = 0; jj < K1S / K2; ++jj) {
+            const int j = b * (K1S / K2) + jj;
+            const uint32_t dm = min(F23 - ej[j], beta23);  // tau << 23
+            tau[j] = dm >> 23;
+            const uint32_t c_bits = c_base - dm;
+            const float C = __uint_as_float(c_bits);
+            const float Cmax = __uint_as_float(c_bits + qp.qmax);
+#pragma unroll
+            for (int i = 0; i < K2; ++i) {
+                const int k = j * K2 + i;
+                const float a = __fmul_rn(fabsf(__uint_as_float(u[k])), K);
+                const float r = fminf(__fadd_rn(a, C), Cmax);
+                const float aq = __fsub_rn(r, C);
+                code[k] = (__float_as_uint(r) - c_bits) | ((u[k] >> (31 - qp.m)) & (qp.qmax + 1u));
+                yb[k] = __float_as_uint(__fmul_rn(aq, Kinv)) | (u[k] & 0x80000000u);
+                if (WANT_SUMS) {
+                    const float de = __fsub_rn(aq, a);  // exact
+                    pe = fmaf(de, de, pe);
+                    ps = fmaf(a, a, ps);
+                }
+            }
+        }
+        if (WANT_SUMS) {
+            const double w = __hiloint2double((int)((F23 >> 2) + 0x30100000u), 0);  // 2^(2F-254)
+            e2 = fma((double)pe, w, e2);
+            s2 = fma((double)ps, w, s2);
+        }
+    }
+}
+
+// Division by a launch-time constant without the 64-bit divide sequence (n, d < 2^31).
+struct FastDiv {
+    uint32_t d, mul, shift;
+};
+inline FastDiv make_fastdiv(uint32_t d) {
+    FastDiv f;
+    f.d = d;
+    uint32_t s = 0;
+    while ((1ull << s) < d) ++s;
+    f.shift = s;
+    f.mul = (uint32_t)(((1ull << 32) * ((1ull << s) - d)) / d + 1);
+    return f;
+}
+__device__ __forceinline__ uint32_t fastdiv(uint32_t n, const FastDiv& f) {
+    return (uint32_t)(((uint64_t)__umulhi(n, f.mul) + n) >> f.shift);
 }
 
 // ---- bit-stream helpers for one slice (code width W = m + 1 known at compile time) -----------------

@@ -12,54 +12,134 @@ namespace bdr {
 
 constexpr int kThreads = 256;
 
+// Prefetch ring.  Per iteration a warp consumes one contiguous run of 32 * kVecs 16-byte words (lane
+// l owns words [l*kVecs, (l+1)*kVecs)).  The warp copies the run cooperatively -- instruction v
+// moves words v*32 .. v*32+31, i.e. 512 contiguous bytes -- so every 32-byte sector is requested
+// once, and stores word c at position c ^ ((c >> 3) & (kVecs-1)) so that the later per-lane 16-byte
+// reads (stride kVecs words) hit eight different bank groups per quarter-warp.
+template <typename T, int SPT> struct Ring {
+    static constexpr int kVecs = SliceWords<T>::kVecs * SPT;  // 16-byte words per thread per iteration
+    static constexpr int kStages = kVecs >= 8 ? 2 : (kVecs >= 4 ? 3 : 4);  // ~128 bytes ahead per thread
+    static constexpr size_t kBytes = (size_t)kStages * kVecs * kThreads * 16;
+    __device__ static __forceinline__ uint32_t swz(uint32_t c) { return c ^ ((c >> 3) & (kVecs >= 8 ? 7u : (uint32_t)(kVecs - 1))); }
+    // warp_stage: this warp's 32*kVecs words of one stage; src: start of the warp's run in global memory
+    __device__ static __forceinline__ void issue(uint4* warp_stage, const T* src, int lane) {
+#pragma unroll
+        for (int v = 0; v < kVecs; ++v) {
+            const uint32_t c = v * 32 + lane;
+            cp_async16(warp_stage + swz(c), reinterpret_cast<const uint4*>(src) + c);
+        }
+    }
+    __device__ static __forceinline__ uint4 read(const uint4* warp_stage, int lane, int v) {
+        return warp_stage[swz(lane * kVecs + v)];
+    }
+};
+
+// Quantize the SPT slices a thread holds (shared exponents across lanes when k1 spans them).
+template <int K2, int K1S, int SPT>
+__device__ __forceinline__ void quantize_unit(const uint32_t (&u)[SPT][kSlice], const QParams& qp, int group_lanes,
+                                              bool want_sums, uint32_t (&yb)[SPT][kSlice], double& e2, double& s2) {
+    uint32_t fj[SPT][kSlice / K2];
+    uint32_t fb[SPT][kSlice / K1S];
+#pragma unroll
+    for (int s = 0; s < SPT; ++s) {
+        subblock_exponents<K2>(u[s], fj[s]);
+#pragma unroll
+        for (int b = 0; b < kSlice / K1S; ++b) {
+            uint32_t f = 0;
+#pragma unroll
+            for (int j = 0; j < K1S / K2; ++j) f = max(f, fj[s][b * (K1S / K2) + j]);
+            fb[s][b] = f;
+        }
+    }
+    if (K1S == kSlice && qp.k1 > kSlice) {  // block spans the thread's slices and maybe lanes
+        uint32_t F = fb[0][0];
+#pragma unroll
+        for (int s = 1; s < SPT; ++s) F = max(F, fb[s][0]);
+        for (int o = group_lanes >> 1; o > 0; o >>= 1) F = max(F, __shfl_xor_sync(0xFFFFFFFFu, F, o));
+#pragma unroll
+        for (int s = 0; s < SPT; ++s) fb[s][0] = F;
+    }
+#pragma unroll
+    for (int s = 0; s < SPT; ++s) {
+        uint32_t code[kSlice], tau[kSlice / K2];
+        if (want_sums) quantize_slice<K2, K1S, true>(u[s], fj[s], fb[s], qp, yb[s], code, tau, e2, s2);
+        else quantize_slice<K2, K1S, false>(u[s], fj[s], fb[s], qp, yb[s], code, tau, e2, s2);
+    }
+}
+
 template <typename T, int K2, int K1S, int SPT>
 __global__ void __launch_bounds__(kThreads)
-quant_rowwise_kernel(const T* x, T* y, int64_t rows, int64_t cols, int64_t ld, int64_t units_per_row,
-                     int64_t total_units, int group_lanes, QParams qp, bool vec_ok, double* sums) {
+quant_rowwise_kernel(const T* x, T* y, int64_t rows, int64_t cols, int64_t ld, FastDiv units_per_row,
+                     uint32_t total_units, int group_lanes, QParams qp, bool vec_ok, bool all_full, double* sums) {
     constexpr int kUnit = kSlice * SPT;  // elements per thread per iteration
+    constexpr int kVecs = Ring<T, SPT>::kVecs, kStages = Ring<T, SPT>::kStages;
+    extern __shared__ __align__(16) uint4 ring[];  // [stage][warp][32*kVecs words]
     double e2 = 0.0, s2 = 0.0;
+    const uint32_t stride = gridDim.x * kThreads;
+    const uint32_t g0 = blockIdx.x * kThreads + threadIdx.x;
     // total_units is a multiple of 32, so whole warps iterate together (shuffles need every lane)
-    for (int64_t g = (int64_t)blockIdx.x * kThreads + threadIdx.x; g < total_units;
-         g += (int64_t)gridDim.x * kThreads) {
-        const int64_t row = g / units_per_row;
-        const int64_t col0 = (g - row * units_per_row) * kUnit;
-        const bool live = row < rows;
-        uint32_t u[SPT][kSlice];
-        int fj[SPT][kSlice / K2];
-        int fb[SPT][kSlice / K1S];
-#pragma unroll
-        for (int s = 0; s < SPT; ++s) {
-            const int64_t c0 = col0 + s * kSlice;
-            const int n = live ? (int)max((int64_t)0, min((int64_t)kSlice, cols - c0)) : 0;
-            if (n == kSlice && vec_ok) load_slice_vec(x + row * ld + c0, u[s]);
-            else load_slice_guarded(x + row * ld + c0, 1, n, u[s]);
-            subblock_exponents<K2>(u[s], fj[s]);
-#pragma unroll
-            for (int b = 0; b < kSlice / K1S; ++b) {
-                int f = 0;
-#pragma unroll
-                for (int j = 0; j < K1S / K2; ++j) f = max(f, fj[s][b * (K1S / K2) + j]);
-                fb[s][b] = f;
+    if (all_full) {
+        // every unit is a full, 16-byte aligned run of the tensor and a warp's 32 units are contiguous
+        // (units_per_row % 32 == 0): feed them through the prefetch ring
+        const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+        const uint32_t gw0 = g0 - lane;  // the warp's first unit
+        auto stage_ptr = [&](int stage) { return ring + ((size_t)stage * (kThreads / 32) + warp) * 32 * kVecs; };
+        auto issue = [&](uint32_t gw, int stage) {
+            if (gw < total_units) {
+                const uint32_t row = fastdiv(gw, units_per_row);
+                Ring<T, SPT>::issue(stage_ptr(stage), x + (int64_t)row * ld + (int64_t)(gw - row * units_per_row.d) * kUnit, lane);
             }
-        }
-        if (K1S == kSlice && qp.k1 > kSlice) {  // block spans the thread's slices and maybe lanes
-            int F = fb[0][0];
+            cp_async_commit();
+        };
 #pragma unroll
-            for (int s = 1; s < SPT; ++s) F = max(F, fb[s][0]);
-            for (int o = group_lanes >> 1; o > 0; o >>= 1) F = max(F, __shfl_xor_sync(0xFFFFFFFFu, F, o));
+        for (int s = 0; s < kStages - 1; ++s) issue(gw0 + s * stride, s);
+        int stage = 0;
+        for (uint32_t g = g0; g < total_units; g += stride) {
+            __syncwarp();  // all lanes are done with the stage that is refilled next
+            issue(g - lane + (kStages - 1) * stride, (stage + kStages - 1) % kStages);
+            cp_async_wait<kStages - 1>();
+            __syncwarp();  // a lane's words were fetched by other lanes
+            uint32_t u[SPT][kSlice], yb[SPT][kSlice];
 #pragma unroll
-            for (int s = 0; s < SPT; ++s) fb[s][0] = F;
-        }
+            for (int s = 0; s < SPT; ++s) {
+                uint4 w[SliceWords<T>::kVecs];
 #pragma unroll
-        for (int s = 0; s < SPT; ++s) {
-            uint32_t yb[kSlice], code[kSlice], tau[kSlice / K2];
-            if (sums) quantize_slice<K2, K1S, true>(u[s], fj[s], fb[s], qp, yb, code, tau, e2, s2);
-            else quantize_slice<K2, K1S, false>(u[s], fj[s], fb[s], qp, yb, code, tau, e2, s2);
+                for (int v = 0; v < SliceWords<T>::kVecs; ++v)
+                    w[v] = Ring<T, SPT>::read(stage_ptr(stage), lane, s * SliceWords<T>::kVecs + v);
+                SliceWords<T>::expand(w, u[s]);
+            }
+            quantize_unit<K2, K1S, SPT>(u, qp, group_lanes, sums != nullptr, yb, e2, s2);
             if (y) {
+                const uint32_t row = fastdiv(g, units_per_row);
+                T* dst = y + (int64_t)row * ld + (int64_t)(g - row * units_per_row.d) * kUnit;
+#pragma unroll
+                for (int s = 0; s < SPT; ++s) store_slice_vec(dst + s * kSlice, yb[s]);
+            }
+            stage = (stage + 1) % kStages;
+        }
+    } else {
+        for (uint32_t g = g0; g < total_units; g += stride) {
+            const int64_t row = fastdiv(g, units_per_row);
+            const int64_t col0 = (int64_t)(g - (uint32_t)row * units_per_row.d) * kUnit;
+            const bool live = row < rows;
+            uint32_t u[SPT][kSlice], yb[SPT][kSlice];
+#pragma unroll
+            for (int s = 0; s < SPT; ++s) {
                 const int64_t c0 = col0 + s * kSlice;
                 const int n = live ? (int)max((int64_t)0, min((int64_t)kSlice, cols - c0)) : 0;
-                if (n == kSlice && vec_ok) store_slice_vec(y + row * ld + c0, yb);
-                else store_slice_guarded(y + row * ld + c0, 1, n, yb);
+                if (n == kSlice && vec_ok) load_slice_vec(x + row * ld + c0, u[s]);
+                else load_slice_guarded(x + row * ld + c0, 1, n, u[s]);
+            }
+            quantize_unit<K2, K1S, SPT>(u, qp, group_lanes, sums != nullptr, yb, e2, s2);
+            if (y) {
+#pragma unroll
+                for (int s = 0; s < SPT; ++s) {
+                    const int64_t c0 = col0 + s * kSlice;
+                    const int n = live ? (int)max((int64_t)0, min((int64_t)kSlice, cols - c0)) : 0;
+                    if (n == kSlice && vec_ok) store_slice_vec(y + row * ld + c0, yb[s]);
+                    else store_slice_guarded(y + row * ld + c0, 1, n, yb[s]);
+                }
             }
         }
     }
@@ -67,34 +147,57 @@ quant_rowwise_kernel(const T* x, T* y, int64_t rows, int64_t cols, int64_t ld, i
 }
 
 // ---- packing fast path: k1 = 16, k2 = 2, code width W = m + 1 -------------------------------------
-// One warp handles 32 consecutive slices (512 elements) of one row per iteration.  Each lane
-// assembles its slice's 2W bytes of codes in registers, the warp stages them in shared memory and
-// writes whole 16-byte vectors, so every plane is written with full-width coalesced stores.
+// One warp handles 32 consecutive slices (512 elements) of one row per iteration; the input comes
+// through the per-thread prefetch ring.  Each lane assembles its slice's 2W bytes of codes in
+// registers, the warp stages them in shared memory and writes whole 16-byte vectors, so every
+// plane is written with full-width coalesced stores.
 template <typename T, int W>
 __global__ void __launch_bounds__(kThreads)
-pack_rowwise_mx_kernel(const T* x, T* y_dq, int64_t rows, int64_t cols, int64_t ld, bdr_planes_t out, QParams qp,
-                       double* sums) {
+pack_rowwise_mx_kernel(const T* x, T* y_dq, FastDiv warps_per_row, uint32_t total, int64_t ld, bdr_planes_t out,
+                       QParams qp, double* sums) {
     constexpr int kWarps = kThreads / 32;
     constexpr int kElemBytes = 2 * W;                  // per slice
-    constexpr int kStage = 32 * kElemBytes + 32 + 96;  // elems | exps | micro (<= 3 bytes per slice)
-    __shared__ __align__(16) uint8_t stage_all[kWarps][(kStage + 15) / 16 * 16];
+    constexpr int kStage = (32 * kElemBytes + 32 + 96 + 15) / 16 * 16;  // elems | exps | micro (<= 3 B per slice)
+    constexpr int kVecs = Ring<T, 1>::kVecs, kStages = Ring<T, 1>::kStages;
+    extern __shared__ __align__(16) uint4 ring[];  // [stage][warp][32*kVecs words], then the per-warp staging
+    uint8_t* stage_base = reinterpret_cast<uint8_t*>(ring + kStages * kVecs * kThreads);
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    uint8_t* stage = stage_all[warp];
+    uint8_t* stage = stage_base + warp * kStage;
     uint8_t* st_exps = stage + 32 * kElemBytes;
     uint8_t* st_micro = st_exps + 32;
 
-    const int64_t warps_per_row = cols / 512;
-    const int64_t total = rows * warps_per_row;
+    const uint32_t stride = gridDim.x * kWarps;
+    const uint32_t w0 = blockIdx.x * kWarps + warp;
+    auto stage_ptr = [&](int st) { return ring + ((size_t)st * kWarps + warp) * 32 * kVecs; };
+    auto issue = [&](uint32_t wi, int st) {
+        if (wi < total) {
+            const uint32_t row = fastdiv(wi, warps_per_row);
+            Ring<T, 1>::issue(stage_ptr(st), x + (int64_t)row * ld + (int64_t)(wi - row * warps_per_row.d) * 512, lane);
+        }
+        cp_async_commit();
+    };
+#pragma unroll
+    for (int s = 0; s < kStages - 1; ++s) issue(w0 + s * stride, s);
+    int rs = 0;
     double e2 = 0.0, s2 = 0.0;
-    for (int64_t wi = (int64_t)blockIdx.x * kWarps + warp; wi < total; wi += (int64_t)gridDim.x * kWarps) {
-        const int64_t row = wi / warps_per_row;
-        const int64_t slice0 = (wi - row * warps_per_row) * 32;  // first slice of the warp in its row
+    for (uint32_t wi = w0; wi < total; wi += stride) {
+        issue(wi + (kStages - 1) * stride, (rs + kStages - 1) % kStages);  // trailing __syncwarp below covers reuse
+        cp_async_wait<kStages - 1>();
+        __syncwarp();  // a lane's words were fetched by other lanes
+        const int64_t row = fastdiv(wi, warps_per_row);
+        const int64_t slice0 = (int64_t)(wi - (uint32_t)row * warps_per_row.d) * 32;  // first slice of the warp in its row
         const int64_t col = (slice0 + lane) * kSlice;
         uint32_t u[kSlice], yb[kSlice], code[kSlice], tau[kSlice / 2];
-        int fj[kSlice / 2], fb[1];
-        load_slice_vec(x + row * ld + col, u);
+        uint32_t fj[kSlice / 2], fb[1];
+        {
+            uint4 w[kVecs];
+#pragma unroll
+            for (int v = 0; v < kVecs; ++v) w[v] = Ring<T, 1>::read(stage_ptr(rs), lane, v);
+            SliceWords<T>::expand(w, u);
+        }
+        rs = (rs + 1) % kStages;
         subblock_exponents<2>(u, fj);
-        int F = 0;
+        uint32_t F = 0;
 #pragma unroll
         for (int j = 0; j < kSlice / 2; ++j) F = max(F, fj[j]);
         fb[0] = F;
@@ -104,14 +207,14 @@ pack_rowwise_mx_kernel(const T* x, T* y_dq, int64_t rows, int64_t cols, int64_t 
 
         uint32_t words[(kSlice * W + 31) / 32];
         codes_to_words<W>(code, words);
-        if (W % 2 == 0 && W % 8 == 0) {  // 16 bytes per slice
+        if (W == 8) {  // 16 bytes per slice
             *reinterpret_cast<uint4*>(stage + lane * kElemBytes) = make_uint4(words[0], words[1], words[2], words[3]);
         } else {
             uint16_t* dst = reinterpret_cast<uint16_t*>(stage + lane * kElemBytes);
 #pragma unroll
             for (int h = 0; h < W; ++h) dst[h] = (uint16_t)(words[h >> 1] >> ((h & 1) * 16));
         }
-        st_exps[lane] = (uint8_t)F;
+        st_exps[lane] = (uint8_t)(F >> 23);
         uint32_t mbits = 0;
 #pragma unroll
         for (int j = 0; j < kSlice / 2; ++j) mbits |= tau[j] << (j * qp.d2);
@@ -149,9 +252,18 @@ static int launch_quant_row(const T* x, T* y, int64_t rows, int64_t cols, int64_
     total = (total + 31) / 32 * 32;
     const int group = qp.k1 > kUnit ? qp.k1 / kUnit : 1;
     const bool vec_ok = (((uintptr_t)x | (uintptr_t)y) % 16 == 0) && (ld * sizeof(T)) % 16 == 0;
+    const bool all_full = vec_ok && padded == cols && cols % kUnit == 0 && upr % 32 == 0;
     if (total == 0) return BDR_OK;
-    quant_rowwise_kernel<T, K2, K1S, SPT><<<grid_for(total, kThreads), kThreads, 0, st>>>(
-        x, y, rows, cols, ld, upr, total, group, qp, vec_ok, sums);
+    if (total >= (1ll << 31) - (1ll << 24)) return BDR_ERR_UNSUPPORTED;  // 32-bit unit indices (incl. prefetch look-ahead)
+    auto kern = quant_rowwise_kernel<T, K2, K1S, SPT>;
+    const size_t smem = Ring<T, SPT>::kBytes;
+    static bool attr_done = false;  // per instantiation; the attribute is idempotent, so a race is harmless
+    if (!attr_done) {
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return BDR_ERR_CUDA;
+        attr_done = true;
+    }
+    kern<<<grid_for(total, kThreads), kThreads, smem, st>>>(x, y, rows, cols, ld, make_fastdiv((uint32_t)upr), (uint32_t)total, group, qp,
+                                                            vec_ok, all_full, sums);
     return cudaGetLastError() == cudaSuccess ? BDR_OK : BDR_ERR_CUDA;
 }
 
@@ -191,7 +303,15 @@ static int launch_pack_row(const T* x, T* y, int64_t rows, int64_t cols, int64_t
                            const QParams& qp, double* sums, cudaStream_t st) {
     const int64_t total = rows * (cols / 512);
     if (total == 0) return BDR_OK;
-    pack_rowwise_mx_kernel<T, W><<<grid_for(total, kThreads / 32), kThreads, 0, st>>>(x, y, rows, cols, ld, out, qp, sums);
+    if (total >= (1ll << 31) - (1ll << 24)) return BDR_ERR_UNSUPPORTED;
+    auto kern = pack_rowwise_mx_kernel<T, W>;
+    const size_t smem = Ring<T, 1>::kBytes + (kThreads / 32) * ((32 * 2 * W + 32 + 96 + 15) / 16 * 16);
+    static bool attr_done = false;
+    if (!attr_done) {
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return BDR_ERR_CUDA;
+        attr_done = true;
+    }
+    kern<<<grid_for(total, kThreads / 32), kThreads, smem, st>>>(x, y, make_fastdiv((uint32_t)(cols / 512)), (uint32_t)total, ld, out, qp, sums);
     return cudaGetLastError() == cudaSuccess ? BDR_OK : BDR_ERR_CUDA;
 }
 

@@ -11,31 +11,47 @@ constexpr int kUnpackThreads = 256;
 
 template <typename T, int W>
 __global__ void __launch_bounds__(kUnpackThreads)
-unpack_rowwise_mx_kernel(bdr_planes_t in, T* y, int64_t rows, int64_t cols, int64_t ld, QParams qp) {
+unpack_rowwise_mx_kernel(bdr_planes_t in, T* y, FastDiv warps_per_row, uint32_t total, int64_t ld, QParams qp) {
     constexpr int kWarps = kUnpackThreads / 32;
     constexpr int kElemBytes = 2 * W;
     constexpr int kStage = (32 * kElemBytes + 32 + 96 + 15) / 16 * 16;
-    __shared__ __align__(16) uint8_t stage_all[kWarps][kStage];
+    constexpr int kStages = 3;  // packed bytes are prefetched two iterations ahead with cp.async
+    __shared__ __align__(16) uint8_t stage_all[kWarps][kStages][kStage];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    uint8_t* stage = stage_all[warp];
-    uint8_t* st_exps = stage + 32 * kElemBytes;
-    uint8_t* st_micro = st_exps + 32;
-    const int64_t warps_per_row = cols / 512;
-    const int64_t total = rows * warps_per_row;
-    for (int64_t wi = (int64_t)blockIdx.x * kWarps + warp; wi < total; wi += (int64_t)gridDim.x * kWarps) {
-        const int64_t row = wi / warps_per_row;
-        const int64_t slice0 = (wi - row * warps_per_row) * 32;
-        const uint4* g_elems = reinterpret_cast<const uint4*>(in.elems + row * in.ld_elems + slice0 * kElemBytes);
-        uint4* s4 = reinterpret_cast<uint4*>(stage);
-        for (int v = lane; v < 32 * kElemBytes / 16; v += 32) s4[v] = __ldg(g_elems + v);
-        if (lane < 2) {
-            reinterpret_cast<uint4*>(st_exps)[lane] =
-                __ldg(reinterpret_cast<const uint4*>(in.exps + row * in.ld_exps + slice0) + lane);
-        } else if (lane - 2 < 2 * qp.d2) {
-            reinterpret_cast<uint4*>(st_micro)[lane - 2] =
-                __ldg(reinterpret_cast<const uint4*>(in.micro + row * in.ld_micro + slice0 * qp.d2) + (lane - 2));
+    const uint32_t stride = gridDim.x * kWarps;
+    const uint32_t w0 = blockIdx.x * kWarps + warp;
+    const int n_elem_vecs = 32 * kElemBytes / 16, n_micro_vecs = 2 * qp.d2;
+    auto issue = [&](uint32_t wi, int st) {
+        if (wi < total) {
+            const int64_t row = fastdiv(wi, warps_per_row);
+            const int64_t slice0 = (int64_t)(wi - (uint32_t)row * warps_per_row.d) * 32;
+            uint8_t* stage = stage_all[warp][st];
+            for (int v = lane; v < n_elem_vecs + 2 + n_micro_vecs; v += 32) {
+                if (v < n_elem_vecs)
+                    cp_async16(stage + v * 16, in.elems + row * in.ld_elems + slice0 * kElemBytes + v * 16);
+                else if (v < n_elem_vecs + 2)
+                    cp_async16(stage + 32 * kElemBytes + (v - n_elem_vecs) * 16,
+                               in.exps + row * in.ld_exps + slice0 + (v - n_elem_vecs) * 16);
+                else
+                    cp_async16(stage + 32 * kElemBytes + 32 + (v - n_elem_vecs - 2) * 16,
+                               in.micro + row * in.ld_micro + slice0 * qp.d2 + (v - n_elem_vecs - 2) * 16);
+            }
         }
-        __syncwarp();
+        cp_async_commit();
+    };
+#pragma unroll
+    for (int s = 0; s < kStages - 1; ++s) issue(w0 + s * stride, s);
+    int rs = 0;
+    for (uint32_t wi = w0; wi < total; wi += stride) {
+        issue(wi + (kStages - 1) * stride, (rs + kStages - 1) % kStages);
+        cp_async_wait<kStages - 1>();
+        __syncwarp();  // the slice a lane decodes was fetched by other lanes
+        const uint8_t* stage = stage_all[warp][rs];
+        const uint8_t* st_exps = stage + 32 * kElemBytes;
+        const uint8_t* st_micro = st_exps + 32;
+        rs = (rs + 1) % kStages;
+        const int64_t row = fastdiv(wi, warps_per_row);
+        const int64_t slice0 = (int64_t)(wi - (uint32_t)row * warps_per_row.d) * 32;
         uint32_t words[(kSlice * W + 31) / 32 + 1];
 #pragma unroll
         for (int i = 0; i < (kSlice * W + 31) / 32 + 1; ++i) words[i] = 0;
@@ -53,7 +69,7 @@ unpack_rowwise_mx_kernel(bdr_planes_t in, T* y, int64_t rows, int64_t cols, int6
         uint32_t yb[kSlice];
         decode_slice<W>(words, F, mbits, qp, yb);
         store_slice_vec(y + row * ld + (slice0 + lane) * kSlice, yb);
-        __syncwarp();
+        __syncwarp();  // everyone is done with this stage before it is refilled
     }
 }
 
@@ -61,9 +77,10 @@ template <typename T, int W>
 static int launch_unpack_row(const bdr_planes_t& in, T* y, int64_t rows, int64_t cols, int64_t ld, const QParams& qp,
                              cudaStream_t st) {
     const int64_t total = rows * (cols / 512);
+    if (total >= (1ll << 31) - (1ll << 24)) return BDR_ERR_UNSUPPORTED;
     const int64_t need = (total + kUnpackThreads / 32 - 1) / (kUnpackThreads / 32);
     const int grid = (int)max((int64_t)1, min(need, (int64_t)sm_count() * 8));
-    unpack_rowwise_mx_kernel<T, W><<<grid, kUnpackThreads, 0, st>>>(in, y, rows, cols, ld, qp);
+    unpack_rowwise_mx_kernel<T, W><<<grid, kUnpackThreads, 0, st>>>(in, y, make_fastdiv((uint32_t)(cols / 512)), (uint32_t)total, ld, qp);
     return cudaGetLastError() == cudaSuccess ? BDR_OK : BDR_ERR_CUDA;
 }
 

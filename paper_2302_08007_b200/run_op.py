@@ -1,0 +1,52 @@
+"""Run one operation of the library a few times on a seeded synthetic tensor (for profilers and
+quick timing):  python -m paper_2302_08007_b200.run_op --op pack --fmt MX6 --axis 1 --dtype bf16"""
+from __future__ import annotations
+
+import argparse
+
+import numpy as np
+import torch
+
+from . import binding as bdr
+from . import synth
+
+FORMATS = {"MX4": bdr.MX4, "MX6": bdr.MX6, "MX9": bdr.MX9}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--op", default="pack", choices=["quant_dequant", "pack", "unpack"])
+    ap.add_argument("--fmt", default="MX6", choices=list(FORMATS))
+    ap.add_argument("--axis", type=int, default=1)
+    ap.add_argument("--dtype", default="bf16", choices=["bf16", "f32"])
+    ap.add_argument("--rows", type=int, default=8192)
+    ap.add_argument("--cols", type=int, default=8192)
+    ap.add_argument("--reps", type=int, default=3)
+    ap.add_argument("--no-sums", action="store_true")
+    a = ap.parse_args()
+    cfg = FORMATS[a.fmt]
+    x = torch.from_numpy(synth.outlier_channel_matrix(a.rows, a.cols, seed=0, stream=3)).cuda()
+    if a.dtype == "bf16":
+        x = x.to(torch.bfloat16)
+    y = torch.empty_like(x)
+    planes = bdr.alloc_planes(cfg, a.rows, a.cols, a.axis)
+    sums = None if a.no_sums else torch.zeros(2, dtype=torch.float64, device="cuda")
+    bdr.bdr_pack(cfg, x, planes, axis=a.axis)
+    torch.cuda.synchronize()
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+    ev[0].record()
+    for _ in range(a.reps):
+        if a.op == "quant_dequant":
+            bdr.bdr_quant_dequant(cfg, x, y, axis=a.axis, qsnr_sums=sums)
+        elif a.op == "pack":
+            bdr.bdr_pack(cfg, x, planes, axis=a.axis, qsnr_sums=sums)
+        else:
+            bdr.bdr_unpack(cfg, planes, y, axis=a.axis)
+    ev[1].record()
+    torch.cuda.synchronize()
+    print("%s %s axis=%d %s %dx%d: %.4f ms per launch" % (a.op, a.fmt, a.axis, a.dtype, a.rows, a.cols,
+                                                          ev[0].elapsed_time(ev[1]) / a.reps))
+
+
+if __name__ == "__main__":
+    main()
