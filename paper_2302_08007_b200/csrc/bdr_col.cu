@@ -59,7 +59,7 @@ template <typename T> struct ColRing {
     static constexpr size_t kBytes = (size_t)kStages * kSlice * kColThreads * sizeof(typename PairWord<T>::type);
 };
 
-template <typename T, int W>  // W = m + 1 when packing, 0 when only y / sums are wanted
+template <typename T, int W, bool SUMS, bool YOUT>  // W = m + 1 when packing, 0 when only y / sums are wanted
 __global__ void __launch_bounds__(kColThreads, 2)
 quant_colwise_mx_kernel(const T* x, T* y, int64_t rows, int64_t cols, int64_t ld, bdr_planes_t out, QParams qp,
                         double* sums) {
@@ -98,29 +98,28 @@ quant_colwise_mx_kernel(const T* x, T* y, int64_t rows, int64_t cols, int64_t ld
         uint32_t yb[2][kSlice];
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
-            uint32_t code[kSlice], tau[kSlice / 2];
+            uint32_t rq[kSlice], cb[kSlice / 2], tau[kSlice / 2];
             uint32_t fj[kSlice / 2], fb[1];
             subblock_exponents<2>(u[h], fj);
             uint32_t F = 0;
 #pragma unroll
             for (int j = 0; j < kSlice / 2; ++j) F = max(F, fj[j]);
             fb[0] = F;
-            if (sums) quantize_slice<2, kSlice, true>(u[h], fj, fb, qp, yb[h], code, tau, e2, s2);
-            else quantize_slice<2, kSlice, false>(u[h], fj, fb, qp, yb[h], code, tau, e2, s2);
+            quantize_slice<2, kSlice, SUMS, YOUT, (W > 0)>(u[h], fj, fb, qp, yb[h], rq, cb, tau, e2, s2);
             if (W > 0) {
                 uint32_t words[(kSlice * ColStage<W>::kW + 31) / 32];
-                codes_to_words<ColStage<W>::kW>(code, words);
+                pack_words<ColStage<W>::kW, kSlice, 2>(u[h], rq, cb, words);
 #pragma unroll
                 for (int k = 0; k < ColStage<W>::kW; ++k)
                     st.elems[bl][2 * lane + h][k] = (uint16_t)(words[k >> 1] >> ((k & 1) * 16));
                 st.exps[bl][2 * lane + h] = (uint8_t)(F >> 23);
-                uint32_t mbits = 0;
+                uint32_t mbits = 0;  // d2 = 1
 #pragma unroll
-                for (int j = 0; j < kSlice / 2; ++j) mbits |= tau[j] << (j * qp.d2);
-                for (int k = 0; k < qp.d2; ++k) st.micro[bl][2 * lane + h][k] = (uint8_t)(mbits >> (8 * k));
+                for (int j = 0; j < kSlice / 2; ++j) mbits |= tau[j] << j;
+                st.micro[bl][2 * lane + h][0] = (uint8_t)mbits;
             }
         }
-        if (y) {
+        if (YOUT) {
             T* py = y + b * kSlice * ld + c;
 #pragma unroll
             for (int r = 0; r < kSlice; ++r) store_pair(py + r * ld, yb[0][r], yb[1][r]);
@@ -162,7 +161,7 @@ quant_colwise_mx_kernel(const T* x, T* y, int64_t rows, int64_t cols, int64_t ld
                 make_uint4(w4[0], w4[1], w4[2], w4[3]);
         }
     }
-    if (sums) block_accumulate_sums(e2, s2, sums);
+    if (SUMS) block_accumulate_sums(e2, s2, sums);
 }
 
 // Mirror image: gather each column's packed run with coalesced 16-byte loads, scatter it into
@@ -223,13 +222,13 @@ unpack_colwise_mx_kernel(bdr_planes_t in, T* y, int64_t rows, int64_t cols, int6
     }
 }
 
-template <typename T, int W>
+template <typename T, int W, bool SUMS, bool YOUT>
 static int launch_col(const T* x, T* y, int64_t rows, int64_t cols, int64_t ld, const bdr_planes_t* out,
                       const QParams& qp, double* sums, cudaStream_t st) {
     const dim3 grid((unsigned)(cols / kTileCols), (unsigned)((rows / kSlice + kTileBlocks - 1) / kTileBlocks));
     bdr_planes_t pl = {};
     if (out) pl = *out;
-    auto kern = quant_colwise_mx_kernel<T, W>;
+    auto kern = quant_colwise_mx_kernel<T, W, SUMS, YOUT>;
     const size_t smem = ColRing<T>::kBytes + (W > 0 ? sizeof(ColStage<W>) : 16);
     static bool attr_done = false;
     if (!attr_done) {
@@ -240,23 +239,29 @@ static int launch_col(const T* x, T* y, int64_t rows, int64_t cols, int64_t ld, 
     return cudaGetLastError() == cudaSuccess ? BDR_OK : BDR_ERR_CUDA;
 }
 
+template <typename T, int W>
+static int col_flags(const T* x, T* y, int64_t rows, int64_t cols, int64_t ld, const bdr_planes_t* out,
+                     const QParams& qp, double* sums, cudaStream_t st) {
+    if (sums) return y ? launch_col<T, W, true, true>(x, y, rows, cols, ld, out, qp, sums, st)
+                       : launch_col<T, W, true, false>(x, y, rows, cols, ld, out, qp, sums, st);
+    if (y) return launch_col<T, W, false, true>(x, y, rows, cols, ld, out, qp, sums, st);
+    if constexpr (W > 0) return launch_col<T, W, false, false>(x, y, rows, cols, ld, out, qp, sums, st);
+    return BDR_ERR_NULL;
+}
+
+// Fast path for the Table II family (k1 = 16, k2 = 2, d2 = 1; packing: m = 2, 4, 7).
 template <typename T>
 int quant_colwise_mx(const T* x, T* y, int64_t rows, int64_t cols, int64_t ld, const bdr_planes_t* out,
                      const QParams& qp, double* sums, cudaStream_t st) {
-    if (qp.k1 != 16 || qp.k2 != 2 || cols % kTileCols != 0 || rows % kSlice != 0) return BDR_ERR_UNSUPPORTED;
+    if (qp.k1 != 16 || qp.k2 != 2 || qp.d2 != 1 || cols % kTileCols != 0 || rows % kSlice != 0) return BDR_ERR_UNSUPPORTED;
     if (out && rows % (kSlice * kTileBlocks) != 0) return BDR_ERR_UNSUPPORTED;
     if ((((uintptr_t)x | (uintptr_t)y) % 16) || (ld * sizeof(T)) % 16) return BDR_ERR_UNSUPPORTED;
     if (rows / kSlice / kTileBlocks > 65535) return BDR_ERR_UNSUPPORTED;
-    if (!out) return launch_col<T, 0>(x, y, rows, cols, ld, out, qp, sums, st);
-    switch (qp.m + 1) {
-        case 2: return launch_col<T, 2>(x, y, rows, cols, ld, out, qp, sums, st);
-        case 3: return launch_col<T, 3>(x, y, rows, cols, ld, out, qp, sums, st);
-        case 4: return launch_col<T, 4>(x, y, rows, cols, ld, out, qp, sums, st);
-        case 5: return launch_col<T, 5>(x, y, rows, cols, ld, out, qp, sums, st);
-        case 6: return launch_col<T, 6>(x, y, rows, cols, ld, out, qp, sums, st);
-        case 7: return launch_col<T, 7>(x, y, rows, cols, ld, out, qp, sums, st);
-        case 8: return launch_col<T, 8>(x, y, rows, cols, ld, out, qp, sums, st);
-        case 9: return launch_col<T, 9>(x, y, rows, cols, ld, out, qp, sums, st);
+    if (!out) return col_flags<T, 0>(x, y, rows, cols, ld, out, qp, sums, st);
+    switch (qp.m) {
+        case 2: return col_flags<T, 3>(x, y, rows, cols, ld, out, qp, sums, st);
+        case 4: return col_flags<T, 5>(x, y, rows, cols, ld, out, qp, sums, st);
+        case 7: return col_flags<T, 8>(x, y, rows, cols, ld, out, qp, sums, st);
     }
     return BDR_ERR_UNSUPPORTED;
 }
@@ -272,18 +277,14 @@ static int launch_unpack_col(const bdr_planes_t& in, T* y, int64_t rows, int64_t
 template <typename T>
 int unpack_colwise_mx(const bdr_planes_t& in, T* y, int64_t rows, int64_t cols, int64_t ld, const QParams& qp,
                       cudaStream_t st) {
-    if (qp.k1 != 16 || qp.k2 != 2 || cols % kTileCols != 0 || rows % (kSlice * kTileBlocks) != 0) return BDR_ERR_UNSUPPORTED;
+    if (qp.k1 != 16 || qp.k2 != 2 || qp.d2 != 1 || cols % kTileCols != 0 || rows % (kSlice * kTileBlocks) != 0)
+        return BDR_ERR_UNSUPPORTED;
     if (((uintptr_t)y % 16) || (ld * sizeof(T)) % 16) return BDR_ERR_UNSUPPORTED;
     if (rows / (kSlice * kTileBlocks) > 65535) return BDR_ERR_UNSUPPORTED;
-    switch (qp.m + 1) {
-        case 2: return launch_unpack_col<T, 2>(in, y, rows, cols, ld, qp, st);
-        case 3: return launch_unpack_col<T, 3>(in, y, rows, cols, ld, qp, st);
-        case 4: return launch_unpack_col<T, 4>(in, y, rows, cols, ld, qp, st);
-        case 5: return launch_unpack_col<T, 5>(in, y, rows, cols, ld, qp, st);
-        case 6: return launch_unpack_col<T, 6>(in, y, rows, cols, ld, qp, st);
-        case 7: return launch_unpack_col<T, 7>(in, y, rows, cols, ld, qp, st);
-        case 8: return launch_unpack_col<T, 8>(in, y, rows, cols, ld, qp, st);
-        case 9: return launch_unpack_col<T, 9>(in, y, rows, cols, ld, qp, st);
+    switch (qp.m) {
+        case 2: return launch_unpack_col<T, 3>(in, y, rows, cols, ld, qp, st);
+        case 4: return launch_unpack_col<T, 5>(in, y, rows, cols, ld, qp, st);
+        case 7: return launch_unpack_col<T, 8>(in, y, rows, cols, ld, qp, st);
     }
     return BDR_ERR_UNSUPPORTED;
 }

@@ -238,20 +238,22 @@ __device__ __forceinline__ void subblock_exponents(const uint32_t (&u)[kSlice], 
 template <int K2, int K1S, bool WANT_SUMS>
 __device__ __forceinline__ void quantize_slice_exact(const uint32_t (&u)[kSlice], const uint32_t (&ej)[kSlice / K2],
                                                   const uint32_t (&eb)[kSlice / K1S], const QParams& qp,
-                                                  uint32_t (&yb)[kSlice], uint32_t (&code)[kSlice],
-                                                  uint32_t (&tau)[kSlice / K2], double& e2, double& s2) {
+                                                  uint32_t (&yb)[kSlice], uint32_t (&rq)[kSlice],
+                                                  uint32_t (&cb)[kSlice / K2], uint32_t (&tau)[kSlice / K2],
+                                                  double& e2, double& s2) {
 #pragma unroll
     for (int j = 0; j < kSlice / K2; ++j) {
         const int F = (int)(eb[(j * K2) / K1S] >> 23);
         const int t = F == 255 ? 0 : min(F - (int)(ej[j] >> 23), qp.beta);
         tau[j] = (uint32_t)t;
+        cb[j] = 0;
 #pragma unroll
         for (int i = 0; i < K2; ++i) {
             const int k = j * K2 + i;
             uint32_t q = 0, y = 0x7FC00000u;
             if (F != 255) quant_elem_exact(u[k], F, t, qp, q, y);
             yb[k] = y;
-            code[k] = F == 255 ? 0u : (((u[k] >> 31) << qp.m) | q);
+            rq[k] = F == 255 ? 0u : q;
             if (WANT_SUMS) {
                 const double de = (double)__uint_as_float(y) - (double)__uint_as_float(u[k]);
                 const double dx = (double)__uint_as_float(u[k]);
@@ -264,8 +266,10 @@ __device__ __forceinline__ void quantize_slice_exact(const uint32_t (&u)[kSlice]
 
 // Quantize the slice.  eb[] holds the shared exponent (e23) of each k1-block touching the slice
 // (K1S = min(k1,16) elements each; for k1 >= 16 the single entry is the block's exponent after any
-// cross-lane reduction).  Produces dequantized bit patterns, element codes (sign<<m | q), sub-block
-// shifts, and adds this slice's Eq. 3 terms to e2 / s2 when WANT_SUMS.
+// cross-lane reduction).  Produces dequantized bit patterns (WANT_Y), and for packing (WANT_CODE)
+// the sub-block shifts tau plus the magnitudes in "raw" form: q of element k is rq[k] - cb[k / K2]
+// (the packer removes the per-sub-block offset cb after it has shifted the fields into place; the
+// sign comes from u).  Adds this slice's Eq. 3 terms to e2 / s2 when WANT_SUMS.
 //
 // Fast path (ties-to-even, finite block): work in the block-normalised domain a = |x| * 2^(127-F),
 // a < 2.  There the unit of q is 2^(-(m-1)-tau), so adding C = 1.5 * 2^(23-(m-1)-tau) makes the fp32
@@ -274,16 +278,17 @@ __device__ __forceinline__ void quantize_slice_exact(const uint32_t (&u)[kSlice]
 // (an element so small that a underflows rounds to q = 0 either way).  The Eq. 3 terms are summed
 // in fp32 in the normalised domain (at most 16 terms of magnitude <= 4) and widened once per block
 // with the exact factor 2^(2F-254).
-template <int K2, int K1S, bool WANT_SUMS>
+template <int K2, int K1S, bool WANT_SUMS, bool WANT_Y = true, bool WANT_CODE = true>
 __device__ __forceinline__ void quantize_slice(const uint32_t (&u)[kSlice], const uint32_t (&ej)[kSlice / K2],
                                                const uint32_t (&eb)[kSlice / K1S], const QParams& qp,
-                                               uint32_t (&yb)[kSlice], uint32_t (&code)[kSlice],
-                                               uint32_t (&tau)[kSlice / K2], double& e2, double& s2) {
+                                               uint32_t (&yb)[kSlice], uint32_t (&rq)[kSlice],
+                                               uint32_t (&cb)[kSlice / K2], uint32_t (&tau)[kSlice / K2], double& e2,
+                                               double& s2) {
     uint32_t emax = eb[0];
 #pragma unroll
     for (int b = 1; b < kSlice / K1S; ++b) emax = max(emax, eb[b]);
     if (qp.rounding != BDR_ROUND_NEAREST_EVEN || emax == kExpMask) {
-        quantize_slice_exact<K2, K1S, WANT_SUMS>(u, ej, eb, qp, yb, code, tau, e2, s2);
+        quantize_slice_exact<K2, K1S, WANT_SUMS>(u, ej, eb, qp, yb, rq, cb, tau, e2, s2);
         return;
     }
     const uint32_t c_base = ((uint32_t)(127 + 23 - (qp.m - 1)) << 23) | 0x400000u;
@@ -298,8 +303,8 @@ __device__ __forceinline__ void quantize_slice(const uint32_t (&u)[kSlice], cons
         for (int jj = 0; jj < K1S / K2; ++jj) {
             const int j = b * (K1S / K2) + jj;
             const uint32_t dm = min(F23 - ej[j], beta23);  // tau << 23
-            tau[j] = dm >> 23;
             const uint32_t c_bits = c_base - dm;
+            if (WANT_CODE) { tau[j] = dm >> 23; cb[j] = c_bits; }
             const float C = __uint_as_float(c_bits);
             const float Cmax = __uint_as_float(c_bits + qp.qmax);
 #pragma unroll
@@ -308,8 +313,8 @@ __device__ __forceinline__ void quantize_slice(const uint32_t (&u)[kSlice], cons
                 const float a = __fmul_rn(fabsf(__uint_as_float(u[k])), K);
                 const float r = fminf(__fadd_rn(a, C), Cmax);
                 const float aq = __fsub_rn(r, C);
-                code[k] = (__float_as_uint(r) - c_bits) | ((u[k] >> (31 - qp.m)) & (qp.qmax + 1u));
-                yb[k] = __float_as_uint(__fmul_rn(aq, Kinv)) | (u[k] & 0x80000000u);
+                if (WANT_CODE) rq[k] = __float_as_uint(r);
+                if (WANT_Y) yb[k] = __float_as_uint(__fmul_rn(aq, Kinv)) | (u[k] & 0x80000000u);
                 if (WANT_SUMS) {
                     const float de = __fsub_rn(aq, a);  // exact
                     pe = fmaf(de, de, pe);
@@ -322,6 +327,22 @@ __device__ __forceinline__ void quantize_slice(const uint32_t (&u)[kSlice], cons
             e2 = fma((double)pe, w, e2);
             s2 = fma((double)ps, w, s2);
         }
+    }
+}
+
+// Runtime-flag front end: picks the instantiation that computes only what the caller will use.
+template <int K2, int K1S, bool WANT_CODE>
+__device__ __forceinline__ void quantize_slice_rt(const uint32_t (&u)[kSlice], const uint32_t (&ej)[kSlice / K2],
+                                                  const uint32_t (&eb)[kSlice / K1S], const QParams& qp, bool want_sums,
+                                                  bool want_y, uint32_t (&yb)[kSlice], uint32_t (&rq)[kSlice],
+                                                  uint32_t (&cb)[kSlice / K2], uint32_t (&tau)[kSlice / K2], double& e2,
+                                                  double& s2) {
+    if (want_y) {
+        if (want_sums) quantize_slice<K2, K1S, true, true, WANT_CODE>(u, ej, eb, qp, yb, rq, cb, tau, e2, s2);
+        else quantize_slice<K2, K1S, false, true, WANT_CODE>(u, ej, eb, qp, yb, rq, cb, tau, e2, s2);
+    } else {
+        if (want_sums) quantize_slice<K2, K1S, true, false, WANT_CODE>(u, ej, eb, qp, yb, rq, cb, tau, e2, s2);
+        else quantize_slice<K2, K1S, false, false, WANT_CODE>(u, ej, eb, qp, yb, rq, cb, tau, e2, s2);
     }
 }
 
@@ -342,40 +363,73 @@ __device__ __forceinline__ uint32_t fastdiv(uint32_t n, const FastDiv& f) {
     return (uint32_t)(((uint64_t)__umulhi(n, f.mul) + n) >> f.shift);
 }
 
-// ---- bit-stream helpers for one slice (code width W = m + 1 known at compile time) -----------------
-// Pack 16 codes into the little-endian LSB-first stream of the slice (2W bytes).
-template <int W>
-__device__ __forceinline__ void codes_to_words(const uint32_t (&code)[kSlice], uint32_t (&words)[(kSlice * W + 31) / 32]) {
+// ---- bit-stream helpers (code width W = m + 1 known at compile time) -------------------------------
+// Pack N elements (raw magnitudes rq with per-sub-block offsets cb, signs from u) into the
+// little-endian LSB-first stream: code i = (sign << m) | q occupies bits [i*W, i*W + W).
+// A field that lies inside one word is placed with one multiply-add, rq * 2^sh, in wrap-around
+// arithmetic; the offsets are removed afterwards with one multiply-add per sub-block and word
+// (cb * -(sum of its 2^sh)), which leaves exactly q * 2^sh because q * 2^sh < 2^32.  Sign bits are
+// ORed into a second accumulator.  The few fields that straddle two words take the plain route.
+template <int W, int N, int K2>
+__device__ __forceinline__ void pack_words(const uint32_t (&u)[N], const uint32_t (&rq)[N], const uint32_t (&cb)[N / K2],
+                                           uint32_t (&words)[(N * W + 31) / 32]) {
+    constexpr int NW = (N * W + 31) / 32, M = W - 1;
+    uint32_t accq[NW], accs[NW];
 #pragma unroll
-    for (int i = 0; i < (kSlice * W + 31) / 32; ++i) words[i] = 0;
+    for (int w = 0; w < NW; ++w) { accq[w] = 0; accs[w] = 0; }
 #pragma unroll
-    for (int i = 0; i < kSlice; ++i) {
+    for (int i = 0; i < N; ++i) {
         const int bit = i * W, wi = bit >> 5, sh = bit & 31;
-        words[wi] |= code[i] << sh;
-        if (sh + W > 32) words[wi + 1] |= code[i] >> (32 - sh);
+        if (sh + W <= 32) {
+            accq[wi] += rq[i] * (1u << sh);
+            const int sp = sh + M;  // where the sign bit goes
+            accs[wi] |= (sp == 31 ? u[i] : (u[i] >> (31 - sp))) & (1u << sp);
+        } else {
+            const uint32_t code = (rq[i] - cb[i / K2]) | ((u[i] >> 31) << M);
+            accs[wi] |= code << sh;
+            accs[wi + 1] |= code >> (32 - sh);
+        }
     }
+#pragma unroll
+    for (int j = 0; j < N / K2; ++j) {
+#pragma unroll
+        for (int w = (j * K2 * W) >> 5; w <= (((j + 1) * K2 - 1) * W) >> 5; ++w) {
+            uint32_t kc = 0;  // folds to a constant
+#pragma unroll
+            for (int i = j * K2; i < (j + 1) * K2; ++i) {
+                const int bit = i * W, wi = bit >> 5, sh = bit & 31;
+                if (wi == w && sh + W <= 32) kc += 1u << sh;
+            }
+            if (kc) accq[w] -= cb[j] * kc;
+        }
+    }
+#pragma unroll
+    for (int w = 0; w < NW; ++w) words[w] = accq[w] | accs[w];
 }
 
-
-// Decode one slice: codes are W-bit fields of the little-endian stream in `words`.
+// Decode one slice (k2 = 2): codes are W-bit fields of the little-endian stream in `words`.
+// value = q * 2^p with p = F-127-tau-(m-1): the float 2^23 + q is built by ORing q into its
+// mantissa, and fma(2^23 + q, 2^p, -2^(p+23)) is then exactly q * 2^p (valid while 2^(p+23) is finite).
 template <int W>
 __device__ __forceinline__ void decode_slice(const uint32_t (&words)[(kSlice * W + 31) / 32 + 1], int F, uint32_t mbits,
                                              const QParams& qp, uint32_t (&yb)[kSlice]) {
-    constexpr uint32_t kMask = (1u << W) - 1u;
+    constexpr int M = W - 1;
+    constexpr uint32_t kQMask = (1u << M) - 1u;
+    const bool fma_ok = F <= kFastMaxF;
 #pragma unroll
     for (int j = 0; j < kSlice / 2; ++j) {
         const int tau = (int)((mbits >> (j * qp.d2)) & (uint32_t)qp.beta);
-        const float scale = __uint_as_float(pow2_bits(max(F - 127 - tau - (qp.m - 1), -149)));
+        const int p = max(F - 127 - tau - (M - 1), -149);
+        const float scale = __uint_as_float(pow2_bits(p));
+        const float bias = __uint_as_float(((uint32_t)(p + 150) << 23) | 0x80000000u);  // -2^(p+23)
 #pragma unroll
         for (int i = 0; i < 2; ++i) {
             const int k = 2 * j + i, bit = k * W, wi = bit >> 5, sh = bit & 31;
-            uint32_t code = words[wi] >> sh;
-            if (sh + W > 32) code |= words[wi + 1] << (32 - sh);
-            code &= kMask;
-            const uint32_t q = code & qp.qmax;
-            // 2^23 + q is exact in fp32; subtracting 2^23 converts q without the conversion pipe
-            const float qf = __fsub_rn(__uint_as_float(0x4B000000u | q), 8388608.0f);
-            yb[k] = F == 255 ? 0x7FC00000u : (__float_as_uint(__fmul_rn(qf, scale)) | ((code >> qp.m) << 31));
+            // 32 stream bits starting at this code
+            const uint32_t f = sh == 0 ? words[wi] : (sh + W > 32 ? __funnelshift_r(words[wi], words[wi + 1], sh) : words[wi] >> sh);
+            const float qf = __uint_as_float(0x4B000000u | (f & kQMask));
+            const float mag = fma_ok ? fmaf(qf, scale, bias) : __fmul_rn(__fsub_rn(qf, 8388608.0f), scale);
+            yb[k] = F == 255 ? 0x7FC00000u : (__float_as_uint(mag) | ((f << (31 - M)) & 0x80000000u));
         }
     }
 }

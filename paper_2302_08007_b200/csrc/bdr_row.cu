@@ -38,7 +38,8 @@ template <typename T, int SPT> struct Ring {
 // Quantize the SPT slices a thread holds (shared exponents across lanes when k1 spans them).
 template <int K2, int K1S, int SPT>
 __device__ __forceinline__ void quantize_unit(const uint32_t (&u)[SPT][kSlice], const QParams& qp, int group_lanes,
-                                              bool want_sums, uint32_t (&yb)[SPT][kSlice], double& e2, double& s2) {
+                                              bool want_sums, bool want_y, uint32_t (&yb)[SPT][kSlice], double& e2,
+                                              double& s2) {
     uint32_t fj[SPT][kSlice / K2];
     uint32_t fb[SPT][kSlice / K1S];
 #pragma unroll
@@ -62,9 +63,8 @@ __device__ __forceinline__ void quantize_unit(const uint32_t (&u)[SPT][kSlice], 
     }
 #pragma unroll
     for (int s = 0; s < SPT; ++s) {
-        uint32_t code[kSlice], tau[kSlice / K2];
-        if (want_sums) quantize_slice<K2, K1S, true>(u[s], fj[s], fb[s], qp, yb[s], code, tau, e2, s2);
-        else quantize_slice<K2, K1S, false>(u[s], fj[s], fb[s], qp, yb[s], code, tau, e2, s2);
+        uint32_t rq[kSlice], cb[kSlice / K2], tau[kSlice / K2];
+        quantize_slice_rt<K2, K1S, false>(u[s], fj[s], fb[s], qp, want_sums, want_y, yb[s], rq, cb, tau, e2, s2);
     }
 }
 
@@ -109,7 +109,7 @@ quant_rowwise_kernel(const T* x, T* y, int64_t rows, int64_t cols, int64_t ld, F
                     w[v] = Ring<T, SPT>::read(stage_ptr(stage), lane, s * SliceWords<T>::kVecs + v);
                 SliceWords<T>::expand(w, u[s]);
             }
-            quantize_unit<K2, K1S, SPT>(u, qp, group_lanes, sums != nullptr, yb, e2, s2);
+            quantize_unit<K2, K1S, SPT>(u, qp, group_lanes, sums != nullptr, y != nullptr, yb, e2, s2);
             if (y) {
                 const uint32_t row = fastdiv(g, units_per_row);
                 T* dst = y + (int64_t)row * ld + (int64_t)(g - row * units_per_row.d) * kUnit;
@@ -131,7 +131,7 @@ quant_rowwise_kernel(const T* x, T* y, int64_t rows, int64_t cols, int64_t ld, F
                 if (n == kSlice && vec_ok) load_slice_vec(x + row * ld + c0, u[s]);
                 else load_slice_guarded(x + row * ld + c0, 1, n, u[s]);
             }
-            quantize_unit<K2, K1S, SPT>(u, qp, group_lanes, sums != nullptr, yb, e2, s2);
+            quantize_unit<K2, K1S, SPT>(u, qp, group_lanes, sums != nullptr, y != nullptr, yb, e2, s2);
             if (y) {
 #pragma unroll
                 for (int s = 0; s < SPT; ++s) {
@@ -147,24 +147,32 @@ quant_rowwise_kernel(const T* x, T* y, int64_t rows, int64_t cols, int64_t ld, F
 }
 
 // ---- packing fast path: k1 = 16, k2 = 2, code width W = m + 1 -------------------------------------
-// One warp handles 32 consecutive slices (512 elements) of one row per iteration; the input comes
-// through the per-thread prefetch ring.  Each lane assembles its slice's 2W bytes of codes in
-// registers, the warp stages them in shared memory and writes whole 16-byte vectors, so every
-// plane is written with full-width coalesced stores.
-template <typename T, int W>
+// One warp handles 64 consecutive slices (1024 elements) per iteration, two adjacent slices per
+// lane; the input comes through the prefetch ring.  A lane's 32 codes are exactly W 32-bit words,
+// which it assembles in registers; the warp stages them in shared memory and writes whole
+// 16-byte vectors, so every plane is written with full-width coalesced stores.
+constexpr int kPackSPT = 2;
+template <int W> struct PackStage {
+    static constexpr int kElemBytes = 32 * kPackSPT * 2 * W;  // per warp iteration
+    static constexpr int kExpBytes = 32 * kPackSPT;
+    static constexpr int kMicroBytes = 32 * kPackSPT;         // d2 = 1: one byte per slice
+    static constexpr int kBytes = kElemBytes + kExpBytes + kMicroBytes;  // a multiple of 16
+};
+
+template <typename T, int W, bool SUMS, bool YDQ>
 __global__ void __launch_bounds__(kThreads)
 pack_rowwise_mx_kernel(const T* x, T* y_dq, FastDiv warps_per_row, uint32_t total, int64_t ld, bdr_planes_t out,
                        QParams qp, double* sums) {
     constexpr int kWarps = kThreads / 32;
-    constexpr int kElemBytes = 2 * W;                  // per slice
-    constexpr int kStage = (32 * kElemBytes + 32 + 96 + 15) / 16 * 16;  // elems | exps | micro (<= 3 B per slice)
-    constexpr int kVecs = Ring<T, 1>::kVecs, kStages = Ring<T, 1>::kStages;
+    using R = Ring<T, kPackSPT>;
+    constexpr int kVecs = R::kVecs, kStages = R::kStages, kSV = SliceWords<T>::kVecs;
+    constexpr int kWarpElems = 32 * kPackSPT * kSlice;  // 1024
     extern __shared__ __align__(16) uint4 ring[];  // [stage][warp][32*kVecs words], then the per-warp staging
     uint8_t* stage_base = reinterpret_cast<uint8_t*>(ring + kStages * kVecs * kThreads);
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    uint8_t* stage = stage_base + warp * kStage;
-    uint8_t* st_exps = stage + 32 * kElemBytes;
-    uint8_t* st_micro = st_exps + 32;
+    uint8_t* stage = stage_base + warp * PackStage<W>::kBytes;
+    uint8_t* st_exps = stage + PackStage<W>::kElemBytes;
+    uint8_t* st_micro = st_exps + PackStage<W>::kExpBytes;
 
     const uint32_t stride = gridDim.x * kWarps;
     const uint32_t w0 = blockIdx.x * kWarps + warp;
@@ -172,7 +180,7 @@ pack_rowwise_mx_kernel(const T* x, T* y_dq, FastDiv warps_per_row, uint32_t tota
     auto issue = [&](uint32_t wi, int st) {
         if (wi < total) {
             const uint32_t row = fastdiv(wi, warps_per_row);
-            Ring<T, 1>::issue(stage_ptr(st), x + (int64_t)row * ld + (int64_t)(wi - row * warps_per_row.d) * 512, lane);
+            R::issue(stage_ptr(st), x + (int64_t)row * ld + (int64_t)(wi - row * warps_per_row.d) * kWarpElems, lane);
         }
         cp_async_commit();
     };
@@ -185,54 +193,56 @@ pack_rowwise_mx_kernel(const T* x, T* y_dq, FastDiv warps_per_row, uint32_t tota
         cp_async_wait<kStages - 1>();
         __syncwarp();  // a lane's words were fetched by other lanes
         const int64_t row = fastdiv(wi, warps_per_row);
-        const int64_t slice0 = (int64_t)(wi - (uint32_t)row * warps_per_row.d) * 32;  // first slice of the warp in its row
-        const int64_t col = (slice0 + lane) * kSlice;
-        uint32_t u[kSlice], yb[kSlice], code[kSlice], tau[kSlice / 2];
-        uint32_t fj[kSlice / 2], fb[1];
-        {
-            uint4 w[kVecs];
+        const int64_t slice0 = (int64_t)(wi - (uint32_t)row * warps_per_row.d) * (32 * kPackSPT);  // warp's first slice in its row
 #pragma unroll
-            for (int v = 0; v < kVecs; ++v) w[v] = Ring<T, 1>::read(stage_ptr(rs), lane, v);
+        for (int s = 0; s < kPackSPT; ++s) {  // one slice at a time keeps the live register set small
+            uint32_t u[kSlice], yb[kSlice], rq[kSlice], cb[kSlice / 2], tau[kSlice / 2];
+            uint32_t fj[kSlice / 2], fb[1];
+            uint4 w[kSV];
+#pragma unroll
+            for (int v = 0; v < kSV; ++v) w[v] = R::read(stage_ptr(rs), lane, s * kSV + v);
             SliceWords<T>::expand(w, u);
+            subblock_exponents<2>(u, fj);
+            uint32_t F = 0;
+#pragma unroll
+            for (int j = 0; j < kSlice / 2; ++j) F = max(F, fj[j]);
+            fb[0] = F;
+            quantize_slice<2, kSlice, SUMS, YDQ, true>(u, fj, fb, qp, yb, rq, cb, tau, e2, s2);
+            if (YDQ) store_slice_vec(y_dq + row * ld + (slice0 + kPackSPT * lane + s) * kSlice, yb);
+            uint32_t words[(kSlice * W + 31) / 32];
+            pack_words<W, kSlice, 2>(u, rq, cb, words);
+            const int sl = kPackSPT * lane + s;  // slice index within the warp's run
+            if (W % 2 == 0) {
+                uint32_t* dst = reinterpret_cast<uint32_t*>(stage + sl * 2 * W);
+#pragma unroll
+                for (int h = 0; h < W / 2; ++h) dst[h] = words[h];
+            } else {
+                uint16_t* dst = reinterpret_cast<uint16_t*>(stage + sl * 2 * W);
+#pragma unroll
+                for (int h = 0; h < W; ++h) dst[h] = (uint16_t)(words[h >> 1] >> ((h & 1) * 16));
+            }
+            st_exps[sl] = (uint8_t)(F >> 23);
+            uint32_t mb = 0;  // d2 = 1: one bit per sub-block
+#pragma unroll
+            for (int j = 0; j < kSlice / 2; ++j) mb |= tau[j] << j;
+            st_micro[sl] = (uint8_t)mb;
         }
         rs = (rs + 1) % kStages;
-        subblock_exponents<2>(u, fj);
-        uint32_t F = 0;
-#pragma unroll
-        for (int j = 0; j < kSlice / 2; ++j) F = max(F, fj[j]);
-        fb[0] = F;
-        if (sums) quantize_slice<2, kSlice, true>(u, fj, fb, qp, yb, code, tau, e2, s2);
-        else quantize_slice<2, kSlice, false>(u, fj, fb, qp, yb, code, tau, e2, s2);
-        if (y_dq) store_slice_vec(y_dq + row * ld + col, yb);
-
-        uint32_t words[(kSlice * W + 31) / 32];
-        codes_to_words<W>(code, words);
-        if (W == 8) {  // 16 bytes per slice
-            *reinterpret_cast<uint4*>(stage + lane * kElemBytes) = make_uint4(words[0], words[1], words[2], words[3]);
-        } else {
-            uint16_t* dst = reinterpret_cast<uint16_t*>(stage + lane * kElemBytes);
-#pragma unroll
-            for (int h = 0; h < W; ++h) dst[h] = (uint16_t)(words[h >> 1] >> ((h & 1) * 16));
-        }
-        st_exps[lane] = (uint8_t)(F >> 23);
-        uint32_t mbits = 0;
-#pragma unroll
-        for (int j = 0; j < kSlice / 2; ++j) mbits |= tau[j] << (j * qp.d2);
-        for (int b = 0; b < qp.d2; ++b) st_micro[lane * qp.d2 + b] = (uint8_t)(mbits >> (8 * b));
         __syncwarp();
-        uint4* g_elems = reinterpret_cast<uint4*>(out.elems + row * out.ld_elems + slice0 * kElemBytes);
+        uint4* g_elems = reinterpret_cast<uint4*>(out.elems + row * out.ld_elems + slice0 * 2 * W);
         const uint4* s4 = reinterpret_cast<const uint4*>(stage);
-        for (int v = lane; v < 32 * kElemBytes / 16; v += 32) g_elems[v] = s4[v];
-        if (lane < 2) {
+        for (int v = lane; v < PackStage<W>::kElemBytes / 16; v += 32) g_elems[v] = s4[v];
+        constexpr int n_exp_vecs = PackStage<W>::kExpBytes / 16, n_micro_vecs = 32 * kPackSPT / 16;
+        if (lane < n_exp_vecs) {
             reinterpret_cast<uint4*>(out.exps + row * out.ld_exps + slice0)[lane] =
                 reinterpret_cast<const uint4*>(st_exps)[lane];
-        } else if (lane - 2 < 2 * qp.d2) {
-            reinterpret_cast<uint4*>(out.micro + row * out.ld_micro + slice0 * qp.d2)[lane - 2] =
-                reinterpret_cast<const uint4*>(st_micro)[lane - 2];
+        } else if (lane - n_exp_vecs < n_micro_vecs) {
+            reinterpret_cast<uint4*>(out.micro + row * out.ld_micro + slice0)[lane - n_exp_vecs] =
+                reinterpret_cast<const uint4*>(st_micro)[lane - n_exp_vecs];
         }
         __syncwarp();
     }
-    if (sums) block_accumulate_sums(e2, s2, sums);
+    if (SUMS) block_accumulate_sums(e2, s2, sums);
 }
 
 // ---- host launchers --------------------------------------------------------------------------------
@@ -246,6 +256,11 @@ template <typename T, int K2, int K1S, int SPT>
 static int launch_quant_row(const T* x, T* y, int64_t rows, int64_t cols, int64_t ld, const QParams& qp, double* sums,
                             cudaStream_t st) {
     constexpr int kUnit = kSlice * SPT;
+    if (ld == cols && cols % qp.k1 == 0) {  // contiguous tensor of whole blocks: one long row, no row arithmetic
+        cols *= rows;
+        ld = cols;
+        rows = 1;
+    }
     const int64_t padded = (cols + qp.k1 - 1) / qp.k1 * qp.k1;  // whole blocks
     const int64_t upr = (padded + kUnit - 1) / kUnit;
     int64_t total = rows * upr;
@@ -294,42 +309,55 @@ int quant_rowwise(const T* x, T* y, int64_t rows, int64_t cols, int64_t ld, cons
         case 4: return dispatch_k2<T, 4, 1>(k2, x, y, rows, cols, ld, qp, sums, st);
         case 8: return dispatch_k2<T, 8, 1>(k2, x, y, rows, cols, ld, qp, sums, st);
         case 1024: return dispatch_k2<T, 16, 2>(k2, x, y, rows, cols, ld, qp, sums, st);
-        default: return dispatch_k2<T, 16, 1>(k2, x, y, rows, cols, ld, qp, sums, st);  // 16 .. 512
+        default:  // 16 .. 512; two slices per thread for 2-byte elements (64 bytes per thread either way)
+            if (sizeof(T) == 2 && cols % 32 == 0) return dispatch_k2<T, 16, 2>(k2, x, y, rows, cols, ld, qp, sums, st);
+            return dispatch_k2<T, 16, 1>(k2, x, y, rows, cols, ld, qp, sums, st);
     }
 }
 
-template <typename T, int W>
+template <typename T, int W, bool SUMS, bool YDQ>
 static int launch_pack_row(const T* x, T* y, int64_t rows, int64_t cols, int64_t ld, const bdr_planes_t& out,
                            const QParams& qp, double* sums, cudaStream_t st) {
-    const int64_t total = rows * (cols / 512);
+    if (ld == cols) {  // contiguous tensor, tight planes: one long row
+        cols *= rows;
+        ld = cols;
+        rows = 1;
+    }
+    const int64_t total = rows * (cols / 1024);
     if (total == 0) return BDR_OK;
     if (total >= (1ll << 31) - (1ll << 24)) return BDR_ERR_UNSUPPORTED;
-    auto kern = pack_rowwise_mx_kernel<T, W>;
-    const size_t smem = Ring<T, 1>::kBytes + (kThreads / 32) * ((32 * 2 * W + 32 + 96 + 15) / 16 * 16);
+    auto kern = pack_rowwise_mx_kernel<T, W, SUMS, YDQ>;
+    const size_t smem = Ring<T, kPackSPT>::kBytes + (kThreads / 32) * PackStage<W>::kBytes;
     static bool attr_done = false;
     if (!attr_done) {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return BDR_ERR_CUDA;
         attr_done = true;
     }
-    kern<<<grid_for(total, kThreads / 32), kThreads, smem, st>>>(x, y, make_fastdiv((uint32_t)(cols / 512)), (uint32_t)total, ld, out, qp, sums);
+    kern<<<grid_for(total, kThreads / 32), kThreads, smem, st>>>(x, y, make_fastdiv((uint32_t)(cols / 1024)), (uint32_t)total, ld, out, qp, sums);
     return cudaGetLastError() == cudaSuccess ? BDR_OK : BDR_ERR_CUDA;
 }
 
-// Returns BDR_ERR_UNSUPPORTED when the shape / configuration is outside the fast path.
+template <typename T, int W>
+static int pack_row_flags(const T* x, T* y, int64_t rows, int64_t cols, int64_t ld, const bdr_planes_t& out,
+                          const QParams& qp, double* sums, cudaStream_t st) {
+    if (sums) return y ? launch_pack_row<T, W, true, true>(x, y, rows, cols, ld, out, qp, sums, st)
+                       : launch_pack_row<T, W, true, false>(x, y, rows, cols, ld, out, qp, sums, st);
+    return y ? launch_pack_row<T, W, false, true>(x, y, rows, cols, ld, out, qp, sums, st)
+             : launch_pack_row<T, W, false, false>(x, y, rows, cols, ld, out, qp, sums, st);
+}
+
+// Fast path for the Table II family (k1 = 16, k2 = 2, d2 = 1; m = 2, 4, 7).  Returns
+// BDR_ERR_UNSUPPORTED for every other configuration or shape (the general kernel covers those).
 template <typename T>
 int pack_rowwise_mx(const T* x, T* y, int64_t rows, int64_t cols, int64_t ld, const bdr_planes_t& out,
                     const QParams& qp, double* sums, cudaStream_t st) {
-    if (qp.k1 != 16 || qp.k2 != 2 || cols % 512 != 0) return BDR_ERR_UNSUPPORTED;
+    if (qp.k1 != 16 || qp.k2 != 2 || qp.d2 != 1) return BDR_ERR_UNSUPPORTED;
+    if (ld == cols ? (rows * cols) % 1024 != 0 || cols % 16 != 0 : cols % 1024 != 0) return BDR_ERR_UNSUPPORTED;
     if ((((uintptr_t)x | (uintptr_t)y) % 16) || (ld * sizeof(T)) % 16) return BDR_ERR_UNSUPPORTED;
-    switch (qp.m + 1) {
-        case 2: return launch_pack_row<T, 2>(x, y, rows, cols, ld, out, qp, sums, st);
-        case 3: return launch_pack_row<T, 3>(x, y, rows, cols, ld, out, qp, sums, st);
-        case 4: return launch_pack_row<T, 4>(x, y, rows, cols, ld, out, qp, sums, st);
-        case 5: return launch_pack_row<T, 5>(x, y, rows, cols, ld, out, qp, sums, st);
-        case 6: return launch_pack_row<T, 6>(x, y, rows, cols, ld, out, qp, sums, st);
-        case 7: return launch_pack_row<T, 7>(x, y, rows, cols, ld, out, qp, sums, st);
-        case 8: return launch_pack_row<T, 8>(x, y, rows, cols, ld, out, qp, sums, st);
-        case 9: return launch_pack_row<T, 9>(x, y, rows, cols, ld, out, qp, sums, st);
+    switch (qp.m) {
+        case 2: return pack_row_flags<T, 3>(x, y, rows, cols, ld, out, qp, sums, st);
+        case 4: return pack_row_flags<T, 5>(x, y, rows, cols, ld, out, qp, sums, st);
+        case 7: return pack_row_flags<T, 8>(x, y, rows, cols, ld, out, qp, sums, st);
     }
     return BDR_ERR_UNSUPPORTED;
 }

@@ -89,15 +89,10 @@ int unpack_rowwise_mx(const bdr_planes_t& in, T* y, int64_t rows, int64_t cols, 
                       cudaStream_t st) {
     if (qp.k1 != 16 || qp.k2 != 2 || cols % 512 != 0) return BDR_ERR_UNSUPPORTED;
     if (((uintptr_t)y % 16) || (ld * sizeof(T)) % 16) return BDR_ERR_UNSUPPORTED;
-    switch (qp.m + 1) {
-        case 2: return launch_unpack_row<T, 2>(in, y, rows, cols, ld, qp, st);
-        case 3: return launch_unpack_row<T, 3>(in, y, rows, cols, ld, qp, st);
-        case 4: return launch_unpack_row<T, 4>(in, y, rows, cols, ld, qp, st);
-        case 5: return launch_unpack_row<T, 5>(in, y, rows, cols, ld, qp, st);
-        case 6: return launch_unpack_row<T, 6>(in, y, rows, cols, ld, qp, st);
-        case 7: return launch_unpack_row<T, 7>(in, y, rows, cols, ld, qp, st);
-        case 8: return launch_unpack_row<T, 8>(in, y, rows, cols, ld, qp, st);
-        case 9: return launch_unpack_row<T, 9>(in, y, rows, cols, ld, qp, st);
+    switch (qp.m) {
+        case 2: return launch_unpack_row<T, 3>(in, y, rows, cols, ld, qp, st);
+        case 4: return launch_unpack_row<T, 5>(in, y, rows, cols, ld, qp, st);
+        case 7: return launch_unpack_row<T, 8>(in, y, rows, cols, ld, qp, st);
     }
     return BDR_ERR_UNSUPPORTED;
 }

@@ -23,6 +23,7 @@ def main():
     ap.add_argument("--cols", type=int, default=8192)
     ap.add_argument("--reps", type=int, default=3)
     ap.add_argument("--no-sums", action="store_true")
+    ap.add_argument("--no-y", action="store_true", help="quant_dequant: only the QSNR sums")
     a = ap.parse_args()
     cfg = FORMATS[a.fmt]
     x = torch.from_numpy(synth.outlier_channel_matrix(a.rows, a.cols, seed=0, stream=3)).cuda()
@@ -37,7 +38,7 @@ def main():
     ev[0].record()
     for _ in range(a.reps):
         if a.op == "quant_dequant":
-            bdr.bdr_quant_dequant(cfg, x, y, axis=a.axis, qsnr_sums=sums)
+            bdr.bdr_quant_dequant(cfg, x, None if a.no_y else y, axis=a.axis, qsnr_sums=sums)
         elif a.op == "pack":
             bdr.bdr_pack(cfg, x, planes, axis=a.axis, qsnr_sums=sums)
         else:

@@ -122,7 +122,8 @@ def test_config1_mx6_vector_of_65536():
 def test_pack_and_unpack_mx_formats(name, dtype, axis):
     cfg = MX[name]
     # fast-path shapes (multiples of 512) and shapes that force the general kernels
-    for kind, rows, cols in (("laplace_outliers", 512, 1024), ("edge", 1024, 512), ("normal", 40, 100), ("normal", 33, 512)):
+    for kind, rows, cols in (("laplace_outliers", 512, 1024), ("edge", 1024, 512), ("normal", 40, 100), ("normal", 33, 512),
+                             ("edge", 64, 2048)):
         x = H.make_input(kind, rows, cols, dtype, seed=21)
         xd = H.host_to_device(x, dtype)
         planes = bdr.alloc_planes(cfg, rows, cols, axis)
