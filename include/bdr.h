@@ -117,7 +117,8 @@ int64_t bdr_qsnr_workspace_bytes(int n_cfgs);
  *   qsnr_db_dev  n_cfgs doubles, written (not accumulated)
  *   workspace    device scratch of at least bdr_qsnr_workspace_bytes(n_cfgs) bytes, 16-byte aligned;
  *                contents are overwritten
- * axis 1 only for n_cfgs > 1. */
+ * 1 <= n_cfgs <= 4096.  axis must be 1 (rows are the lines); column-direction QSNR of a single
+ * configuration comes from bdr_quant_dequant's fused sums. */
 int bdr_qsnr(const bdr_config_t* cfgs /*host*/, int n_cfgs, const void* x, bdr_dtype_t dt, int64_t rows,
              int64_t cols, int64_t ld, int axis, double* qsnr_db_dev, void* workspace, int64_t workspace_bytes,
              void* stream);

@@ -278,7 +278,7 @@ __device__ __forceinline__ void quantize_slice_exact(const uint32_t (&u)[kSlice]
 // (an element so small that a underflows rounds to q = 0 either way).  The Eq. 3 terms are summed
 // in fp32 in the normalised domain (at most 16 terms of magnitude <= 4) and widened once per block
 // with the exact factor 2^(2F-254).
-template <int K2, int K1S, bool WANT_SUMS, bool WANT_Y = true, bool WANT_CODE = true>
+template <int K2, int K1S, bool WANT_SUMS, bool WANT_Y = true, bool WANT_CODE = true, bool WANT_SIG = true>
 __device__ __forceinline__ void quantize_slice(const uint32_t (&u)[kSlice], const uint32_t (&ej)[kSlice / K2],
                                                const uint32_t (&eb)[kSlice / K1S], const QParams& qp,
                                                uint32_t (&yb)[kSlice], uint32_t (&rq)[kSlice],
@@ -318,14 +318,14 @@ __device__ __forceinline__ void quantize_slice(const uint32_t (&u)[kSlice], cons
                 if (WANT_SUMS) {
                     const float de = __fsub_rn(aq, a);  // exact
                     pe = fmaf(de, de, pe);
-                    ps = fmaf(a, a, ps);
+                    if (WANT_SIG) ps = fmaf(a, a, ps);
                 }
             }
         }
         if (WANT_SUMS) {
             const double w = __hiloint2double((int)((F23 >> 2) + 0x30100000u), 0);  // 2^(2F-254)
             e2 = fma((double)pe, w, e2);
-            s2 = fma((double)ps, w, s2);
+            if (WANT_SIG) s2 = fma((double)ps, w, s2);
         }
     }
 }

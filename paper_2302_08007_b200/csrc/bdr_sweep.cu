@@ -1,0 +1,414 @@
+// bdr_qsnr: the design-space sweep of Section IV -- QSNR (Eq. 3) of one tensor under many
+// configurations, reading the tensor once per group of 64 configurations.
+//
+// A CTA stages a tile of 4096 consecutive elements of a row in shared memory (fp32 bit patterns)
+// together with a pyramid of block-maximum exponent bytes for block sizes 2, 4, ..., 1024 (every k1
+// and k2 of the grid is one of its levels).  Then each warp takes configurations round-robin; for
+// one configuration its lanes walk the tile's 16-element slices, evaluate sum (Q(x)-x)^2 with the
+// same slice quantizer as the quantize kernels, and the warp adds the tile's total to a per-CTA
+// accumulator in shared memory.  Only at the end does a CTA touch the global sums (one atomic per
+// configuration), so the tensor is read from HBM once per 64 configurations and the kernel is
+// bound by plain ALU throughput.
+//
+// The comparator kinds of Table I (INT with an FP32 max-scale, Eq. 1-2; FP8-like scalar floats;
+// VSQ) are evaluated in the same loop with IEEE single operations (division included), so their
+// dequantized values match a plain CPU implementation bit for bit.
+#include <vector>
+
+#include "bdr_device.cuh"
+#include "bdr_host.h"
+
+namespace bdr {
+
+constexpr int kSweepThreads = 256;
+constexpr int kSweepWarps = kSweepThreads / 32;
+constexpr int kTile = 4096;                    // elements per tile: a multiple of every k1 <= 1024
+constexpr int kTileSlices = kTile / kSlice;    // 256
+constexpr int kCfgGroup = 64;                  // configurations evaluated per tile visit
+constexpr int kLevels = 10;                    // block sizes 2^1 .. 2^10
+
+struct SweepCfg {
+    int32_t kind, k1, k2, d2, m, rounding;
+    int32_t k2t, k1t;  // compile-time selectors: sub-block / block size inside a slice (<= 16)
+};
+
+struct SweepSmem {
+    uint4 x[kTile / 4];            // 16-byte chunks, chunk c stored at c ^ ((c >> 3) & 3)
+    uint8_t lv[kTile];             // level l (block size 2^l) starts at lv_off(l); sizes 2048, 1024, ..., 4
+    double sig_warp[kSweepWarps];
+};
+__host__ __device__ constexpr int lv_off(int l) { return kTile - (kTile >> (l - 1)); }  // 0, 2048, 3072, ...
+
+__device__ __forceinline__ int swz4(int c) { return c ^ ((c >> 3) & 3); }
+
+__device__ __forceinline__ float round_to_int(float t, int rounding) {  // 0 <= t < 2^22
+    if (rounding == BDR_ROUND_NEAREST_EVEN) return __fsub_rn(__fadd_rn(t, 8388608.0f), 8388608.0f);
+    return floorf(__fadd_rn(t, 0.5f));
+}
+
+// ---- POW2 kind: error energy of one slice ------------------------------------------------------------
+template <int K2, int K1S>
+__device__ __forceinline__ void pow2_slice(const uint32_t (&u)[kSlice], const SweepSmem& sm, int s, const SweepCfg& c,
+                                           const QParams& qp, double& e2) {
+    uint32_t ej[kSlice / K2], eb[kSlice / K1S];
+    if (K2 == 1) {
+#pragma unroll
+        for (int i = 0; i < kSlice; ++i) ej[i] = u[i] & kExpMask;
+    } else {
+        constexpr int l2 = K2 == 2 ? 1 : K2 == 4 ? 2 : K2 == 8 ? 3 : 4;
+        const uint8_t* p = sm.lv + lv_off(l2) + s * (kSlice / K2);
+#pragma unroll
+        for (int j = 0; j < kSlice / K2; ++j) ej[j] = (uint32_t)p[j] << 23;
+    }
+    if (K1S == kSlice) {
+        const int l1 = 31 - __clz(c.k1);  // log2 k1 >= 4
+        eb[0] = (uint32_t)sm.lv[lv_off(l1) + ((s * kSlice) >> l1)] << 23;
+    } else if (K1S == 1) {
+#pragma unroll
+        for (int i = 0; i < kSlice; ++i) eb[i] = u[i] & kExpMask;
+    } else {
+        constexpr int l1 = K1S == 2 ? 1 : K1S == 4 ? 2 : 3;
+        const uint8_t* p = sm.lv + lv_off(l1) + s * (kSlice / K1S);
+#pragma unroll
+        for (int b = 0; b < kSlice / K1S; ++b) eb[b] = (uint32_t)p[b] << 23;
+    }
+    uint32_t yb[kSlice], rq[kSlice], cb[kSlice / K2], tau[kSlice / K2];
+    double s2 = 0.0;
+    quantize_slice<K2, K1S, true, false, false, false>(u, ej, eb, qp, yb, rq, cb, tau, e2, s2);
+}
+
+template <int K1S>
+__device__ __forceinline__ void pow2_slice_k2(const uint32_t (&u)[kSlice], const SweepSmem& sm, int s, const SweepCfg& c,
+                                              const QParams& qp, double& e2) {
+    switch (c.k2t) {
+        case 1: pow2_slice<1, K1S>(u, sm, s, c, qp, e2); break;
+        case 2: if constexpr (K1S >= 2) pow2_slice<2, K1S>(u, sm, s, c, qp, e2); break;
+        case 4: if constexpr (K1S >= 4) pow2_slice<4, K1S>(u, sm, s, c, qp, e2); break;
+        case 8: if constexpr (K1S >= 8) pow2_slice<8, K1S>(u, sm, s, c, qp, e2); break;
+        default: if constexpr (K1S >= 16) pow2_slice<16, K1S>(u, sm, s, c, qp, e2); break;
+    }
+}
+
+// ---- FP32-scaled comparator kinds (one FP32 scale for the whole tensor) -----------------------------
+__device__ __forceinline__ void add_err(float deq_mag, uint32_t ubits, double& e2) {
+    const double d = (double)deq_mag - (double)__uint_as_float(ubits & 0x7FFFFFFFu);
+    e2 = fma(d, d, e2);
+}
+
+// Eq. 1: s = max / (2^(b-1) - 1) with m = b-1;  Eq. 2: q = RoundToInt(x / s);  descale s * q.
+__device__ __forceinline__ void int_slice(const uint32_t (&u)[kSlice], float amax, const SweepCfg& c, double& e2) {
+    const float qmax = (float)((1 << c.m) - 1);
+    const float s = __fdiv_rn(amax, qmax);
+#pragma unroll
+    for (int i = 0; i < kSlice; ++i) {
+        float mag = 0.f;
+        if (s > 0.f) {
+            const float t = __fdiv_rn(__uint_as_float(u[i] & 0x7FFFFFFFu), s);
+            mag = __fmul_rn(fminf(round_to_int(t, c.rounding), qmax), s);
+        }
+        add_err(mag, u[i], e2);
+    }
+}
+
+// Scalar float with d2 exponent bits and m explicit mantissa bits under an FP32 tensor scale.
+__device__ __forceinline__ void fp_slice(const uint32_t (&u)[kSlice], float amax, const SweepCfg& c, double& e2) {
+    const int bias = (1 << (c.d2 - 1)) - 1;
+    const float fmax = (c.d2 == 4 && c.m == 3)
+                           ? 448.0f
+                           : __uint_as_float(((uint32_t)((1 << c.d2) - 2 - bias + 127) << 23) | (0x7FFFFFu & ~(0x7FFFFFu >> c.m)));
+    const float s = __fdiv_rn(amax, fmax);
+    const int ef_min = 1 - bias + 127;
+#pragma unroll
+    for (int i = 0; i < kSlice; ++i) {
+        float mag = 0.f;
+        if (s > 0.f) {
+            const float a = fabsf(__fdiv_rn(__uint_as_float(u[i]), s));
+            const int ef = max((int)(__float_as_uint(a) >> 23), ef_min);
+            const float step = __uint_as_float((uint32_t)(ef - c.m) << 23);
+            const float inv_step = __uint_as_float((uint32_t)(254 - (ef - c.m)) << 23);
+            const float q = round_to_int(__fmul_rn(a, inv_step), c.rounding);
+            mag = fabsf(__fmul_rn(fminf(__fmul_rn(q, step), fmax), s));
+        }
+        add_err(mag, u[i], e2);
+    }
+}
+
+// VSQ: FP32 scale gamma for the tensor, unsigned d2-bit integer sub-scale per 16-element vector.
+__device__ __forceinline__ void vsq_slice(const uint32_t (&u)[kSlice], float amax, const SweepCfg& c, double& e2) {
+    const float qmax = (float)((1 << c.m) - 1);
+    const float umax = (float)((1u << c.d2) - 1u);
+    const float gamma = __fdiv_rn(__fdiv_rn(amax, qmax), umax);
+    uint32_t avb = 0;
+#pragma unroll
+    for (int i = 0; i < kSlice; ++i) avb = max(avb, u[i] & 0x7FFFFFFFu);
+    const float sv = __fdiv_rn(__uint_as_float(avb), qmax);
+    float uu = 0.f;
+    if (gamma > 0.f) uu = fminf(round_to_int(__fdiv_rn(sv, gamma), c.rounding), umax);
+    const float eff = __fmul_rn(uu, gamma);
+#pragma unroll
+    for (int i = 0; i < kSlice; ++i) {
+        float mag = 0.f;
+        if (eff > 0.f) {
+            const float t = __fdiv_rn(__uint_as_float(u[i] & 0x7FFFFFFFu), eff);
+            mag = __fmul_rn(fminf(round_to_int(t, c.rounding), qmax), eff);
+        }
+        add_err(mag, u[i], e2);
+    }
+}
+
+// ---- kernels ----------------------------------------------------------------------------------------------
+template <typename T>
+__global__ void amax_kernel(const T* x, int64_t rows, int64_t cols, int64_t ld, uint32_t* amax_bits) {
+    uint32_t m = 0;
+    const int64_t total = rows * cols;
+    for (int64_t g = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; g < total; g += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t r = g / cols;
+        m = max(m, Elem<T>::load_bits(x + r * ld + (g - r * cols)) & 0x7FFFFFFFu);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) m = max(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
+    if ((threadIdx.x & 31) == 0) atomicMax(amax_bits, m);
+}
+
+template <typename T>
+__global__ void __launch_bounds__(kSweepThreads)
+sweep_kernel(const T* x, int64_t rows, int64_t cols, int64_t ld, const SweepCfg* cfgs, int n_cfg, int n_groups,
+             int tiles_per_row, int64_t total_units, double* err_sums, double* sig_sum, const uint32_t* amax_bits) {
+    extern __shared__ __align__(16) uint8_t dyn[];
+    SweepSmem& sm = *reinterpret_cast<SweepSmem*>(dyn);
+    double* acc = reinterpret_cast<double*>(dyn + sizeof(SweepSmem));  // [n_cfg]
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    for (int c = threadIdx.x; c < n_cfg; c += kSweepThreads) acc[c] = 0.0;
+    double sig_acc = 0.0;
+    const float amax = __uint_as_float(*amax_bits);
+    int64_t loaded_tile = -1;
+    for (int64_t unit = blockIdx.x; unit < total_units; unit += gridDim.x) {
+        const int64_t tile = unit / n_groups;
+        const int group = (int)(unit - tile * n_groups);
+        if (tile != loaded_tile) {
+            __syncthreads();  // everyone is done with the previous tile
+            const int64_t row = tile / tiles_per_row;
+            const int64_t t0 = (tile - row * tiles_per_row) * kTile;
+            const int n = (int)min((int64_t)kTile, cols - t0);
+            const T* src = x + row * ld + t0;
+            // stage: thread t owns slice t (16 elements = 4 chunks)
+            {
+                const int s = threadIdx.x;
+                uint32_t u[kSlice];
+                load_slice_guarded(src + s * kSlice, 1, max(0, min(kSlice, n - s * kSlice)), u);
+#pragma unroll
+                for (int v = 0; v < 4; ++v) sm.x[swz4(4 * s + v)] = make_uint4(u[4 * v], u[4 * v + 1], u[4 * v + 2], u[4 * v + 3]);
+                // exponent pyramid levels 1..4 from the slice, signal energy of the slice
+                uint32_t e[kSlice];
+#pragma unroll
+                for (int i = 0; i < kSlice; ++i) e[i] = u[i] >> 23 & 0xFFu;
+#pragma unroll
+                for (int l = 1; l <= 4; ++l) {
+#pragma unroll
+                    for (int j = 0; j < (kSlice >> l); ++j) {
+                        e[j] = max(e[2 * j], e[2 * j + 1]);
+                        sm.lv[lv_off(l) + s * (kSlice >> l) + j] = (uint8_t)e[j];
+                    }
+                }
+                // levels 5..9 inside the warp (a warp covers 512 consecutive elements), level 10 below
+                uint32_t v = e[0];
+#pragma unroll
+                for (int l = 5; l <= 9; ++l) {
+                    v = max(v, __shfl_xor_sync(0xFFFFFFFFu, v, 1 << (l - 5)));
+                    if ((lane & ((1 << (l - 4)) - 1)) == 0) sm.lv[lv_off(l) + (s >> (l - 4))] = (uint8_t)v;
+                }
+                // signal energy: sum x^2 normalised by the slice exponent, widened once
+                const uint32_t F23 = e[0] << 23;
+                const float K = __uint_as_float(max(0x7F000000u - F23, 0x00400000u));
+                float ps = 0.f;
+                double sg;
+                if (e[0] == 255) {
+                    sg = __longlong_as_double(0x7FF8000000000000ll);
+                } else {
+#pragma unroll
+                    for (int i = 0; i < kSlice; ++i) {
+                        const float a = __fmul_rn(fabsf(__uint_as_float(u[i])), K);
+                        ps = fmaf(a, a, ps);
+                    }
+                    sg = (double)ps * __hiloint2double((int)((F23 >> 2) + 0x30100000u), 0);
+                }
+                sg = warp_sum(sg);
+                if (lane == 0) sm.sig_warp[warp] = sg;
+            }
+            __syncthreads();
+            if (threadIdx.x < kTile / 1024)
+                sm.lv[lv_off(10) + threadIdx.x] = max(sm.lv[lv_off(9) + 2 * threadIdx.x], sm.lv[lv_off(9) + 2 * threadIdx.x + 1]);
+            if (threadIdx.x == 0 && group == 0) {
+#pragma unroll
+                for (int w = 0; w < kSweepWarps; ++w) sig_acc += sm.sig_warp[w];
+            }
+            __syncthreads();
+            loaded_tile = tile;
+        }
+        for (int ci = group * kCfgGroup + warp; ci < min(n_cfg, (group + 1) * kCfgGroup); ci += kSweepWarps) {
+            const SweepCfg c = cfgs[ci];
+            QParams qp;
+            qp.k1 = c.k1; qp.k2 = c.k2; qp.d2 = c.d2; qp.m = c.m; qp.rounding = c.rounding;
+            qp.beta = (1 << c.d2) - 1;
+            qp.qmax = (1u << c.m) - 1u;
+            double e2 = 0.0;
+            for (int s = lane; s < kTileSlices; s += 32) {
+                uint32_t u[kSlice];
+#pragma unroll
+                for (int v = 0; v < 4; ++v) {
+                    const uint4 w = sm.x[swz4(4 * s + v)];
+                    u[4 * v] = w.x; u[4 * v + 1] = w.y; u[4 * v + 2] = w.z; u[4 * v + 3] = w.w;
+                }
+                if (c.kind == BDR_SCALE_POW2) {
+                    switch (c.k1t) {
+                        case 1: pow2_slice_k2<1>(u, sm, s, c, qp, e2); break;
+                        case 2: pow2_slice_k2<2>(u, sm, s, c, qp, e2); break;
+                        case 4: pow2_slice_k2<4>(u, sm, s, c, qp, e2); break;
+                        case 8: pow2_slice_k2<8>(u, sm, s, c, qp, e2); break;
+                        default: pow2_slice_k2<16>(u, sm, s, c, qp, e2); break;
+                    }
+                } else if (c.kind == BDR_SCALE_FP32_INT) {
+                    int_slice(u, amax, c, e2);
+                } else if (c.kind == BDR_SCALE_FP32_FP) {
+                    fp_slice(u, amax, c, e2);
+                } else {
+                    vsq_slice(u, amax, c, e2);
+                }
+            }
+            e2 = warp_sum(e2);
+            if (lane == 0) acc[ci] += e2;  // this warp is the only writer of acc[ci] in the CTA
+        }
+    }
+    __syncthreads();
+    for (int c = threadIdx.x; c < n_cfg; c += kSweepThreads)
+        if (acc[c] != 0.0) atomicAdd(err_sums + c, acc[c]);
+    if (threadIdx.x == 0 && sig_acc != 0.0) atomicAdd(sig_sum, sig_acc);
+}
+
+// The configuration table travels to the device inside kernel parameters (no host buffer has to
+// outlive the call, and nothing synchronises): up to kCfgChunk entries per launch.
+constexpr int kCfgChunk = 96;
+struct CfgChunk { SweepCfg c[kCfgChunk]; };
+__global__ void upload_cfgs_kernel(CfgChunk chunk, SweepCfg* dst, int n) {
+    if ((int)threadIdx.x < n) dst[threadIdx.x] = chunk.c[threadIdx.x];
+}
+
+// Eq. 3 from the accumulated sums: -10 log10(err / sig); err = 0 < sig -> +inf, sig = 0 -> NaN.
+__global__ void qsnr_finalize_kernel(const double* err_sums, const double* sig_sum, int n, double* out_db) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n) return;
+    const double e = err_sums[i], s = *sig_sum;
+    double q;
+    if (s == 0.0 || s != s || e != e) q = __longlong_as_double(0x7FF8000000000000ll);
+    else if (e == 0.0) q = __longlong_as_double(0x7FF0000000000000ll);
+    else q = -10.0 * log10(e / s);
+    out_db[i] = q;
+}
+
+// workspace layout: [n] error sums | signal sum | amax bits (+pad to 16) | [n] SweepCfg
+static size_t ws_cfg_offset(int n) { return (((size_t)n + 1) * 8 + 16 + 15) / 16 * 16; }
+
+int64_t sweep_workspace_bytes(int n) { return (int64_t)((ws_cfg_offset(n) + (size_t)n * sizeof(SweepCfg) + 255) / 256 * 256); }
+
+static bool is_pow2i(int v) { return v > 0 && (v & (v - 1)) == 0; }
+
+// Validate one configuration for the sweep and translate it.
+static int make_sweep_cfg(const bdr_config_t& c, SweepCfg* out) {
+    if (c.rounding != BDR_ROUND_NEAREST_EVEN && c.rounding != BDR_ROUND_NEAREST_AWAY) return BDR_ERR_BAD_CONFIG;
+    SweepCfg s = {c.scale_kind, c.k1, c.k2, c.d2, c.m, c.rounding, 1, 1};
+    switch (c.scale_kind) {
+        case BDR_SCALE_POW2:
+            if (c.d1 != 8 || c.k1 < 1 || c.k2 < 1 || c.k1 % c.k2 != 0 || c.d2 < 0 || c.d2 > 3 || c.m < 1 || c.m > 8)
+                return BDR_ERR_BAD_CONFIG;
+            if (!is_pow2i(c.k1) || !is_pow2i(c.k2) || c.k1 > 1024) return BDR_ERR_UNSUPPORTED;
+            s.k1t = c.k1 < kSlice ? c.k1 : kSlice;
+            s.k2t = c.d2 == 0 ? s.k1t : c.k2;  // d2 = 0: every shift is zero whatever k2 is
+            if (s.k2t > kSlice) return BDR_ERR_UNSUPPORTED;
+            break;
+        case BDR_SCALE_FP32_INT:
+            if (c.m < 1 || c.m > 15) return BDR_ERR_BAD_CONFIG;
+            if (c.k1 != 0) return BDR_ERR_UNSUPPORTED;
+            break;
+        case BDR_SCALE_FP32_FP:
+            if (c.d2 < 2 || c.d2 > 5 || c.m < 1 || c.m > 7) return BDR_ERR_BAD_CONFIG;
+            if (c.k1 != 0) return BDR_ERR_UNSUPPORTED;
+            break;
+        case BDR_SCALE_FP32_VSQ:
+            if (c.k2 < 1 || c.d2 < 1 || c.d2 > 16 || c.m < 1 || c.m > 15) return BDR_ERR_BAD_CONFIG;
+            if (c.k1 != 0 || c.k2 != kSlice) return BDR_ERR_UNSUPPORTED;
+            break;
+        default: return BDR_ERR_BAD_CONFIG;
+    }
+    *out = s;
+    return BDR_OK;
+}
+
+template <typename T>
+static int sweep_launch(const SweepCfg* host_cfgs, int n, bool need_amax, const T* x, int64_t rows, int64_t cols, int64_t ld,
+                        double* out_db, uint8_t* ws, cudaStream_t st) {
+    double* err = reinterpret_cast<double*>(ws);
+    double* sig = err + n;
+    uint32_t* amax = reinterpret_cast<uint32_t*>(sig + 1);
+    SweepCfg* dcfg = reinterpret_cast<SweepCfg*>(ws + ws_cfg_offset(n));
+    if (cudaMemsetAsync(ws, 0, ws_cfg_offset(n), st) != cudaSuccess) return BDR_ERR_CUDA;
+    for (int i0 = 0; i0 < n; i0 += kCfgChunk) {
+        CfgChunk chunk;
+        const int cnt = min(kCfgChunk, n - i0);
+        for (int i = 0; i < cnt; ++i) chunk.c[i] = host_cfgs[i0 + i];
+        upload_cfgs_kernel<<<1, kCfgChunk, 0, st>>>(chunk, dcfg + i0, cnt);
+    }
+    if (rows > 0 && cols > 0) {
+        if (need_amax) {
+            const int64_t total = rows * cols;
+            const int grid = (int)max((int64_t)1, min((total + 1023) / 1024, (int64_t)sm_count() * 8));
+            amax_kernel<T><<<grid, 256, 0, st>>>(x, rows, cols, ld, amax);
+        }
+        const int tiles_per_row = (int)((cols + kTile - 1) / kTile);
+        const int n_groups = (n + kCfgGroup - 1) / kCfgGroup;
+        const int64_t units = rows * tiles_per_row * n_groups;
+        const size_t smem = sizeof(SweepSmem) + (size_t)n * sizeof(double);
+        auto kern = sweep_kernel<T>;
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return BDR_ERR_CUDA;
+        const int grid = (int)max((int64_t)1, min(units, (int64_t)sm_count() * 4));
+        kern<<<grid, kSweepThreads, smem, st>>>(x, rows, cols, ld, dcfg, n, n_groups, tiles_per_row, units, err, sig, amax);
+    }
+    qsnr_finalize_kernel<<<(n + 127) / 128, 128, 0, st>>>(err, sig, n, out_db);
+    return cudaGetLastError() == cudaSuccess ? BDR_OK : BDR_ERR_CUDA;
+}
+
+}  // namespace bdr
+
+using namespace bdr;
+
+extern "C" {
+
+int64_t bdr_qsnr_workspace_bytes(int n_cfgs) { return n_cfgs < 1 ? 0 : sweep_workspace_bytes(n_cfgs); }
+
+int bdr_qsnr(const bdr_config_t* cfgs, int n_cfgs, const void* x, bdr_dtype_t dt, int64_t rows, int64_t cols, int64_t ld,
+             int axis, double* qsnr_db_dev, void* workspace, int64_t workspace_bytes, void* stream) {
+    constexpr int kMaxCfgs = 4096;  // per-CTA accumulators live in shared memory
+    if (!cfgs || !qsnr_db_dev) return BDR_ERR_NULL;
+    if (n_cfgs < 1 || n_cfgs > kMaxCfgs) return BDR_ERR_SIZE;
+    if (dt != BDR_F32 && dt != BDR_BF16) return BDR_ERR_UNSUPPORTED;
+    if (axis != 0 && axis != 1) return BDR_ERR_BAD_CONFIG;
+    if (rows < 0 || cols < 0 || ld < cols) return BDR_ERR_SIZE;
+    if (!x && rows > 0 && cols > 0) return BDR_ERR_NULL;
+    if ((uintptr_t)x % (dt == BDR_F32 ? 4 : 2) || (uintptr_t)qsnr_db_dev % 8) return BDR_ERR_MISALIGNED;
+    std::vector<SweepCfg> table(n_cfgs);
+    bool need_amax = false;
+    for (int i = 0; i < n_cfgs; ++i) {
+        const int rc = make_sweep_cfg(cfgs[i], &table[i]);
+        if (rc) return rc;
+        need_amax |= cfgs[i].scale_kind != BDR_SCALE_POW2;
+    }
+    if (axis != 1) return BDR_ERR_UNSUPPORTED;  // the sweep walks rows; column-wise QSNR comes from bdr_quant_dequant's sums
+    if (!workspace || workspace_bytes < sweep_workspace_bytes(n_cfgs)) return BDR_ERR_WORKSPACE;
+    if ((uintptr_t)workspace % 16) return BDR_ERR_MISALIGNED;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (dt == BDR_F32)
+        return sweep_launch<float>(table.data(), n_cfgs, need_amax, (const float*)x, rows, cols, ld, qsnr_db_dev, (uint8_t*)workspace, st);
+    return sweep_launch<__nv_bfloat16>(table.data(), n_cfgs, need_amax, (const __nv_bfloat16*)x, rows, cols, ld, qsnr_db_dev,
+                                       (uint8_t*)workspace, st);
+}
+
+}  // extern "C"

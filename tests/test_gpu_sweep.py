@@ -1,0 +1,87 @@
+"""GPU parity of bdr_qsnr (the design-space sweep) against the oracle: QSNR within 1e-6 dB relative."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import oracle as orc
+from paper_2302_08007_b200 import binding as bdr
+from paper_2302_08007_b200 import sweep, synth
+from tests import helpers as H
+
+pytestmark = pytest.mark.gpu
+
+
+def run_sweep(cfgs, x_host, dtype="f32", ld=None):
+    x = H.host_to_device(x_host, dtype, ld)
+    out = torch.full((len(cfgs),), -1.0, dtype=torch.float64, device="cuda")
+    ws = torch.empty(bdr.bdr_qsnr_workspace_bytes(len(cfgs)), dtype=torch.uint8, device="cuda")
+    bdr.bdr_qsnr(cfgs, x, out, ws)
+    torch.cuda.synchronize()
+    return out.cpu().numpy()
+
+
+def check(cfgs, got, x, what=""):
+    for cfg, g in zip(cfgs, got):
+        want = orc.qsnr(H.to_orc(cfg), x)
+        if math.isnan(want) or math.isinf(want):
+            assert (math.isnan(g) and math.isnan(want)) or g == want, (what, cfg, g, want)
+        else:
+            assert abs(g - want) <= H.QSNR_REL_TOL * max(abs(want), 1e-3), (what, cfg, g, want)
+
+
+def test_sweep_workload_has_the_documented_size():
+    names = [n for n, _ in sweep.sweep_configs()]
+    assert len(sweep.bdr_grid()) == 441 and len(names) == 457 and len(set(names)) == 457
+
+
+@pytest.mark.parametrize("dist", synth.SWEEP_DISTRIBUTIONS)
+def test_full_sweep_on_each_distribution(dist):
+    cfgs = [c for _, c in sweep.sweep_configs()]
+    x = synth.sweep_distribution(dist, 1 << 16, seed=1).reshape(1, -1)
+    check(cfgs, run_sweep(cfgs, x), x, dist)
+
+
+def test_sweep_ragged_rows_pitch_and_bf16():
+    cfgs = [c for _, c in sweep.sweep_configs()][::5] + [c for _, c in sweep.comparators()]
+    x = synth.normal_with_outliers(7 * 5000, seed=3).reshape(7, 5000)      # rows are lines; 5000 is not a multiple of 16
+    check(cfgs, run_sweep(cfgs, x, ld=5008), x, "ragged")
+    xb = H.make_input("laplace_outliers", 3, 4096 + 512, "bf16", seed=4)
+    check(cfgs, run_sweep(cfgs, xb, dtype="bf16"), xb, "bf16")
+
+
+def test_sweep_extra_configs_edge_values_and_ties_away():
+    C = bdr.Config
+    cfgs = [C(1, 8, 1, 0, 8), C(2, 8, 1, 1, 3), C(4, 8, 2, 2, 5), C(16, 8, 16, 1, 4), C(512, 8, 4, 3, 6),
+            C(16, 8, 2, 1, 4, bdr.SCALE_POW2, bdr.ROUND_NEAREST_AWAY), C(0, 32, 1, 0, 7, bdr.SCALE_FP32_INT, bdr.ROUND_NEAREST_AWAY),
+            C(0, 32, 1, 4, 3, bdr.SCALE_FP32_FP, bdr.ROUND_NEAREST_AWAY), C(0, 32, 16, 6, 3, bdr.SCALE_FP32_VSQ, bdr.ROUND_NEAREST_AWAY),
+            C(0, 32, 1, 3, 2, bdr.SCALE_FP32_FP), C(0, 32, 1, 0, 1, bdr.SCALE_FP32_INT)]
+    for kind in ("edge", "tiny", "normal"):
+        x = H.make_input(kind, 2, 8192, "f32", seed=6)
+        if kind == "edge":
+            x = np.clip(x, -1e30, 1e30).astype(np.float32)       # keep x/s finite for the FP32-scaled kinds
+        check(cfgs, run_sweep(cfgs, x), x, kind)
+
+
+def test_sweep_degenerate_tensors_and_errors():
+    cfgs = [bdr.MX6, bdr.Config(0, 32, 1, 0, 7, bdr.SCALE_FP32_INT)]
+    z = np.zeros((1, 4096), dtype=np.float32)
+    got = run_sweep(cfgs, z)
+    assert np.isnan(got).all()                                  # no signal: QSNR undefined
+    exact = np.tile(np.array([1.0, 0.5, -0.25, 1.75], dtype=np.float32), 1024).reshape(1, -1)
+    assert math.isinf(run_sweep([bdr.MX6], exact)[0])           # representable input: no noise
+    x = torch.zeros((4, 64), device="cuda")
+    out = torch.zeros(1, dtype=torch.float64, device="cuda")
+    ws = torch.empty(16, dtype=torch.uint8, device="cuda")
+    with pytest.raises(bdr.BdrError) as e:
+        bdr.bdr_qsnr([bdr.MX6], x, out, ws)
+    assert e.value.status == -6
+    ws = torch.empty(bdr.bdr_qsnr_workspace_bytes(1), dtype=torch.uint8, device="cuda")
+    with pytest.raises(bdr.BdrError) as e:
+        bdr.bdr_qsnr([bdr.MX6], x, out, ws, axis=0)
+    assert e.value.status == -3
+    with pytest.raises(bdr.BdrError) as e:
+        bdr.bdr_qsnr([bdr.Config(16, 8, 3, 1, 4)], x, out, ws)
+    assert e.value.status == -2
+    torch.cuda.synchronize()
