@@ -126,11 +126,20 @@ int bdr_qsnr(const bdr_config_t* cfgs /*host*/, int n_cfgs, const void* x, bdr_d
 /* C[M,N] (fp32, row pitch ldc elements) = deq(A)[M,K] * deq(B)[N,K]^T with both operands given as
  * packed planes quantized along K (axis 1 planes of A and of B), decoded to bf16 inside the kernel
  * and accumulated in fp32 on the tensor cores (Section V: both inputs of a tensor operation are
- * MX-quantized along the reduction dimension).
- * Needs k1 = 16, k2 = 2, d2 = 1, m <= 7 for both operands, K a multiple of 64. */
+ * MX-quantized along the reduction dimension).  The result equals the fp32-accumulated product of
+ * the dequantized operands; only the summation order is unspecified.
+ * Needs the Table II formats (k1 = 16, k2 = 2, d2 = 1, m in {2, 4, 7}; A and B may differ), M a
+ * multiple of 128, N a multiple of 256, K a multiple of 64, c 16-byte aligned and ldc a multiple
+ * of 4; anything else is BDR_ERR_UNSUPPORTED.  Blocks whose shared exponent lies below 2^-120
+ * decode to zero (bf16 has no finer values).  A device-side wait that runs out is reported by
+ * mx_gemm_status(), not by this call. */
 int mx_gemm(const bdr_config_t* cfg_a /*host*/, const bdr_planes_t* a /*host struct*/,
             const bdr_config_t* cfg_b /*host*/, const bdr_planes_t* b /*host struct*/, int64_t M, int64_t N,
             int64_t K, float* c, int64_t ldc, void* stream);
+
+/* BDR_OK, or BDR_ERR_TIMEOUT if any mx_gemm launch on the current device gave up a bounded wait
+ * (sticky).  Host call; synchronises with the device (it copies one word back). */
+int mx_gemm_status(void);
 
 #ifdef __cplusplus
 }

@@ -20,7 +20,7 @@ ROUND_NEAREST_EVEN, ROUND_NEAREST_AWAY = 0, 1
 F32, BF16 = 0, 1
 
 EXPORTS = ("bdr_strerror", "bdr_packed_sizes", "bdr_quant_dequant", "bdr_pack", "bdr_unpack",
-           "bdr_qsnr_workspace_bytes", "bdr_qsnr", "mx_gemm")
+           "bdr_qsnr_workspace_bytes", "bdr_qsnr", "mx_gemm", "mx_gemm_status")
 
 
 class BdrError(RuntimeError):
@@ -97,6 +97,8 @@ def lib():
                                C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p]
         L.mx_gemm.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_int64, C.c_int64,
                               C.c_void_p, C.c_int64, C.c_void_p]
+        L.mx_gemm_status.restype = C.c_int
+        L.mx_gemm_status.argtypes = []
         for fn in (L.bdr_packed_sizes, L.bdr_quant_dequant, L.bdr_pack, L.bdr_unpack, L.bdr_qsnr, L.mx_gemm):
             fn.restype = C.c_int
         _lib = L
@@ -208,3 +210,8 @@ def mx_gemm(cfg_a: Config, a: Planes, cfg_b: Config, b: Planes, M: int, N: int, 
     _check(lib().mx_gemm(C.addressof(ca), C.addressof(pa), C.addressof(cb), C.addressof(pb), M, N, K, _ptr(c),
                          c.stride(0), _stream(stream)), "mx_gemm")
     return c
+
+
+def mx_gemm_status() -> int:
+    """0, or the (sticky) status of a launch whose bounded device-side wait ran out."""
+    return int(lib().mx_gemm_status())

@@ -1,0 +1,65 @@
+"""Secondary benchmark legs (argument marshalling + CUDA-event timing only): the design-space sweep
+(configs/s) and the MX GEMM (TFLOP/s).  bench.py calls these after its timed steps."""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+from . import binding as bdr
+from . import sweep, synth
+
+SWEEP_N = 1 << 24
+
+
+def _time(fn, reps: int, warmup: int = 1) -> float:
+    for _ in range(warmup):
+        fn()
+    torch.cuda.synchronize()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record()
+    for _ in range(reps):
+        fn()
+    b.record()
+    torch.cuda.synchronize()
+    return a.elapsed_time(b) / reps
+
+
+def sweep_leg(args) -> dict:
+    """QSNR of 2^24 fp32 values per distribution under the 457-configuration sweep."""
+    named = sweep.sweep_configs()
+    cfgs = [c for _, c in named]
+    names = [n for n, _ in named]
+    out = torch.empty(len(cfgs), dtype=torch.float64, device="cuda")
+    ws = torch.empty(bdr.bdr_qsnr_workspace_bytes(len(cfgs)), dtype=torch.uint8, device="cuda")
+    per_dist = {}
+    total_ms = 0.0
+    show = {"MX9": "bdr_k1=16_k2=2_d2=1_m=7", "MX6": "bdr_k1=16_k2=2_d2=1_m=4", "MX4": "bdr_k1=16_k2=2_d2=1_m=2",
+            "MSFP16": "bdr_k1=16_k2=1_d2=0_m=7", "INT8": "int8", "INT4": "int4", "FP8_E4M3": "fp8_e4m3",
+            "FP8_E5M2": "fp8_e5m2", "VSQ_INT4_d2=6": "vsq_int4_d2=6"}
+    for dist in synth.SWEEP_DISTRIBUTIONS:
+        x = torch.from_numpy(synth.sweep_distribution(dist, SWEEP_N, seed=0)).cuda().reshape(1, -1)
+        ms = _time(lambda: bdr.bdr_qsnr(cfgs, x, out, ws), reps=3)
+        q = out.cpu().numpy()
+        per_dist[dist] = {"ms": ms, "qsnr_db": {k: float(q[names.index(v)]) for k, v in show.items()}}
+        total_ms += ms
+        del x
+    n_eval = len(cfgs) * len(synth.SWEEP_DISTRIBUTIONS)
+    return {"sweep": {"metric": "BDR-sweep configs/s", "value": n_eval / (total_ms * 1e-3), "unit": "configs/s",
+                      "configs": len(cfgs), "distributions": list(synth.SWEEP_DISTRIBUTIONS),
+                      "elements_per_distribution": SWEEP_N, "ms_total": total_ms,
+                      "element_configs_per_s": n_eval * SWEEP_N / (total_ms * 1e-3), "bound": "alu",
+                      "per_distribution": per_dist}}
+
+
+def gemm_leg(args) -> dict:
+    """C[4096,4096] = A * B^T with MX6 operands packed along K (fp32 accumulate and output)."""
+    M = N = K = 4096
+    a = torch.from_numpy(synth.normal_matrix(M, K, seed=0, stream=10)).cuda()
+    b = torch.from_numpy(synth.normal_matrix(N, K, seed=0, stream=11, sigma=0.02)).cuda()
+    pa, pb = bdr.alloc_planes(bdr.MX6, M, K), bdr.alloc_planes(bdr.MX6, N, K)
+    bdr.bdr_pack(bdr.MX6, a, pa)
+    bdr.bdr_pack(bdr.MX6, b, pb)
+    c = torch.empty((M, N), dtype=torch.float32, device="cuda")
+    ms = _time(lambda: bdr.mx_gemm(bdr.MX6, pa, bdr.MX6, pb, M, N, K, c), reps=20, warmup=3)
+    return {"mx_gemm": {"metric": "MX-GEMM TFLOP/s", "value": 2.0 * M * N * K / (ms * 1e-3) / 1e12, "unit": "TFLOP/s",
+                        "ms": ms, "shape": [M, N, K], "format": "MX6 x MX6", "bound": "tensor"}}

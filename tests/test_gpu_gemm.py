@@ -1,0 +1,112 @@
+"""GPU parity of mx_gemm against the fp64 oracle product of the dequantized operands.
+
+Target: relative Frobenius error <= 1e-3.  The decoded operands are exact in bf16 and their products
+exact in fp32, so only the fp32 summation order separates the two; the observed error is ~1e-6.
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import oracle as orc
+from paper_2302_08007_b200 import binding as bdr
+from paper_2302_08007_b200 import synth
+from tests import helpers as H
+
+pytestmark = pytest.mark.gpu
+
+FMT = {"MX4": bdr.MX4, "MX6": bdr.MX6, "MX9": bdr.MX9}
+REL_FROB_TOL = 1e-3
+
+
+def gpu_gemm(cfg_a, a_host, cfg_b, b_host):
+    M, K = a_host.shape
+    N = b_host.shape[0]
+    a, b = torch.from_numpy(a_host).cuda(), torch.from_numpy(b_host).cuda()
+    pa, pb = bdr.alloc_planes(cfg_a, M, K), bdr.alloc_planes(cfg_b, N, K)
+    bdr.bdr_pack(cfg_a, a, pa)
+    bdr.bdr_pack(cfg_b, b, pb)
+    c = torch.full((M, N), float("nan"), dtype=torch.float32, device="cuda")
+    bdr.mx_gemm(cfg_a, pa, cfg_b, pb, M, N, K, c)
+    torch.cuda.synchronize()
+    assert bdr.mx_gemm_status() == 0
+    return c.cpu().numpy()
+
+
+def oracle_gemm(cfg_a, a_host, cfg_b, b_host):
+    aq, _ = orc.quant_dequant(H.to_orc(cfg_a), a_host)
+    bq, _ = orc.quant_dequant(H.to_orc(cfg_b), b_host)
+    return orc.gemm_nt_f64(aq, bq, nthreads=8)
+
+
+def rel_frob(c, ref):
+    return float(np.linalg.norm(c.astype(np.float64) - ref) / max(np.linalg.norm(ref), 1e-300))
+
+
+def test_exact_case_small_integers():
+    # operands that are representable in MX9 and whose dot products are small integers: any
+    # summation order gives the same fp32 result, so the match must be bit for bit
+    rng = np.random.default_rng(0)
+    a = rng.integers(-8, 9, (128, 64)).astype(np.float32)
+    b = rng.integers(-8, 9, (256, 64)).astype(np.float32)
+    a[:, ::16] = 8.0      # pin every block's shared exponent so all of -8..8 stay representable
+    b[:, ::16] = -8.0
+    c = gpu_gemm(bdr.MX9, a, bdr.MX9, b)
+    ref = oracle_gemm(bdr.MX9, a, bdr.MX9, b)
+    assert np.array_equal(ref, (a.astype(np.int64) @ b.astype(np.int64).T).astype(np.float64))
+    assert np.array_equal(c.astype(np.float64), ref)
+
+
+@pytest.mark.parametrize("fa,fb", [("MX6", "MX6"), ("MX9", "MX4"), ("MX4", "MX9"), ("MX9", "MX9"), ("MX4", "MX4")])
+def test_random_operands_match_the_oracle(fa, fb):
+    M, N, K = 256, 512, 320                              # several tiles in M and N, 5 K steps
+    a = synth.normal_matrix(M, K, seed=1, stream=1)
+    b = synth.normal_matrix(N, K, seed=1, stream=2, sigma=0.02)
+    c = gpu_gemm(FMT[fa], a, FMT[fb], b)
+    ref = oracle_gemm(FMT[fa], a, FMT[fb], b)
+    err = rel_frob(c, ref)
+    assert err <= REL_FROB_TOL, err
+    assert err <= 1e-5, err                              # what exact decoding should deliver
+
+
+def test_outlier_channels_and_extreme_scales():
+    M, N, K = 128, 256, 512
+    a = synth.outlier_channel_matrix(M, K, seed=2, gain=50.0)
+    for scale in (1.0, 1e-30, 1e25):
+        b = synth.normal_matrix(N, K, seed=3, sigma=0.02) * np.float32(scale)
+        c = gpu_gemm(bdr.MX6, a, bdr.MX9, b)
+        ref = oracle_gemm(bdr.MX6, a, bdr.MX9, b)
+        assert rel_frob(c, ref) <= 1e-5, scale
+    z = np.zeros((N, K), dtype=np.float32)
+    assert not gpu_gemm(bdr.MX6, a, bdr.MX6, z).any()
+
+
+def test_config4_shape_on_sampled_entries():
+    M = N = K = 4096
+    a = synth.normal_matrix(M, K, seed=0, stream=10)
+    b = synth.normal_matrix(N, K, seed=0, stream=11, sigma=0.02)
+    c = gpu_gemm(bdr.MX6, a, bdr.MX6, b)
+    aq, _ = orc.quant_dequant(orc.MX6, a, nthreads=8)
+    bq, _ = orc.quant_dequant(orc.MX6, b, nthreads=8)
+    rng = np.random.default_rng(4)
+    ri, ci = rng.integers(0, M, 4096), rng.integers(0, N, 4096)
+    ref = orc.gemm_nt_f64_sampled(aq, bq, ri, ci)
+    got = c[ri, ci].astype(np.float64)
+    assert np.linalg.norm(got - ref) / np.linalg.norm(ref) <= 1e-5
+    assert np.isfinite(c).all()
+    # a full row and a full column of tiles as well
+    assert rel_frob(c[:128], orc.gemm_nt_f64(aq[:128], bq, nthreads=8)) <= 1e-5
+
+
+def test_gemm_argument_errors():
+    pa, pb = bdr.alloc_planes(bdr.MX6, 128, 64), bdr.alloc_planes(bdr.MX6, 256, 64)
+    c = torch.empty((128, 256), device="cuda")
+    with pytest.raises(bdr.BdrError) as e:
+        bdr.mx_gemm(bdr.Config(16, 8, 2, 1, 3), pa, bdr.MX6, pb, 128, 256, 64, c)     # m = 3 has no gemm kernel
+    assert e.value.status == -3
+    with pytest.raises(bdr.BdrError) as e:
+        bdr.mx_gemm(bdr.MX6, pa, bdr.MX6, pb, 100, 256, 64, c)
+    assert e.value.status == -3
+    with pytest.raises(bdr.BdrError) as e:
+        bdr.mx_gemm(bdr.MX6, pa, bdr.MX6, pb, 128, 256, 128, c)                       # planes too narrow for K
+    assert e.value.status == -5
+    torch.cuda.synchronize()
