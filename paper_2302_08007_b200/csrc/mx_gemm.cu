@@ -4,13 +4,13 @@
 // with m <= 7 is exact in bf16 -- and multiplied on the 5th-generation tensor cores
 // (tcgen05.mma, kind::f16, fp32 accumulation in tensor memory).
 //
-// One CTA computes a 128 x 256 tile of C.  Warps 0-7 are decoders: per 64-wide K step they read the
-// packed codes / exponents / microexponents of the tile's 128 A rows and 256 B rows straight from
-// global memory (the operands live in L2), rebuild bf16 values with packed bf16x2 arithmetic and
-// store them in shared memory in the K-major, 128-byte-swizzled layout the tensor core reads.
-// Warp 8 issues the MMAs (4 x K=16 per stage) and signals stage reuse / accumulator completion
-// through tcgen05.commit on mbarriers.  After the last K step warps 0-7 read the accumulator from
-// tensor memory (tcgen05.ld) and store C.  Every wait is bounded: if one runs out the kernel
+// One CTA computes a 128 x 256 tile of C.  Warps 0-11 are decoders, one thread per tile row (128 A
+// rows + 256 B rows): per 64-wide K step a thread reads its row's packed codes / exponents /
+// microexponents from global memory (the operands live in L2) one step ahead of use, rebuilds bf16
+// values with packed bf16x2 arithmetic and stores them in shared memory in the K-major,
+// 128-byte-swizzled layout the tensor core reads.  Warp 12 issues the MMAs (4 x K=16 per stage) and
+// signals stage reuse / accumulator completion through tcgen05.commit on mbarriers.  After the last
+// K step warps 0-7 read the accumulator from tensor memory (tcgen05.ld) and store C.  Every wait is bounded: if one runs out the kernel
 // records BDR_ERR_TIMEOUT in a status word, skips the remaining work, frees its tensor memory and
 // returns.
 #include "bdr_device.cuh"
@@ -19,8 +19,11 @@
 namespace bdr {
 
 constexpr int kBM = 128, kBN = 256, kBK = 64;
-constexpr int kStages = 4;
-constexpr int kDecodeWarps = 8;
+constexpr int kStages = 3;       // bf16 operand stages (48 KB each)
+// packed-byte prefetch ring: K steps in flight per decode thread (shared memory budget decides)
+template <int W> struct RingDepth { static constexpr int value = W >= 8 ? 2 : 4; };
+constexpr int kDecodeWarps = (kBM + kBN) / 32;  // 12: one decode thread per tile row
+constexpr int kEpilogueWarps = 8;
 constexpr int kGemmThreads = (kDecodeWarps + 1) * 32;
 constexpr int kABytes = kBM * kBK * 2;  // 16 KB
 constexpr int kBBytes = kBN * kBK * 2;  // 32 KB
@@ -111,35 +114,59 @@ __device__ __forceinline__ uint32_t bf16_pow2(int e) {
     return e >= 1 ? (uint32_t)e << 7 : (e >= -6 ? 1u << (6 + e) : 0u);
 }
 
-// Decode one 16-element block (k1 = 16, k2 = 2, d2 = 1, code width W = m + 1) into 8 bf16x2 words.
-// A code pair t (2W stream bits) is spread to the two halves of a word, the magnitudes are ORed
-// into the mantissa of bf16 128.0 (0x4300 | q = 128 + q exactly, q < 128), 128 is subtracted and the
-// result multiplied by the sub-block's power-of-two scale with packed bf16x2 arithmetic; both steps
-// are exact.  The sign bit is ORed in last.
-template <int W>
-__device__ __forceinline__ void decode_block_bf16(const uint32_t (&words)[(kSlice * W + 31) / 32 + 1], uint32_t F, uint32_t micro,
-                                                  uint32_t (&out)[8]) {
+__device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+}
+__device__ __forceinline__ uint32_t bf16x2_fma(uint32_t a, uint32_t b, uint32_t c) {
+    uint32_t d;
+    asm("fma.rn.bf16x2 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+    return d;
+}
+__device__ __forceinline__ uint32_t bf16x2_mul(uint32_t a, uint32_t b) {
+    uint32_t d;
+    asm("mul.rn.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+    return d;
+}
+
+// Decode one 16-element block (k1 = 16, k2 = 2, d2 = 1, code width W = m + 1) that starts at stream
+// bit `bit0` of w[] into 8 bf16x2 words.  A code pair t (2W stream bits) is spread to the two halves
+// of a word; the magnitudes are ORed into the mantissa of bf16 128.0 (0x4300 | q = 128 + q exactly,
+// q < 128); one packed fused multiply-add with the sub-block's power-of-two scale s and the
+// constant -128 s then gives q * s exactly (the exact result is representable, so the single
+// rounding changes nothing).  The sign bit is ORed in last.
+template <int W, int NWORDS>
+__device__ __forceinline__ void decode_block_bf16(const uint32_t (&w)[NWORDS], int bit0, uint32_t F, uint32_t micro, uint32_t (&out)[8]) {
     constexpr int M = W - 1;
     constexpr uint32_t kQ2 = ((1u << M) - 1u) * 0x00010001u;
-    const int e0 = (int)F - (M - 1);  // biased exponent of one unit of q at tau = 0
-    uint32_t s0 = bf16_pow2(e0), s1 = bf16_pow2(e0 - 1);
-    if (F == 255) { s0 = 0x7FC0u; s1 = 0x7FC0u; }  // Inf/NaN block -> NaN
-    s0 *= 0x00010001u;
-    s1 *= 0x00010001u;
-    const __nv_bfloat162 k128 = __floats2bfloat162_rn(128.f, 128.f);
+    // scale of one unit of q: 2^(F-127-tau-(m-1)); the constant term -128 * scale needs exponent + 7
+    const int e0 = (int)F - (M - 1);
+    uint32_t s0 = bf16_pow2(e0) * 0x00010001u, s1 = bf16_pow2(e0 - 1) * 0x00010001u;
+    uint32_t n0, n1;
+    const bool safe = e0 >= 2 && e0 <= 247;  // both scales and both constants are normal bf16 numbers
+    if (safe) {
+        n0 = (s0 + 0x03800380u) | 0x80008000u;  // -(2^7 * s0)
+        n1 = (s1 + 0x03800380u) | 0x80008000u;
+    } else {
+        if (F == 255) { s0 = 0x7FC07FC0u; s1 = s0; }  // Inf/NaN block -> NaN
+        n0 = 0; n1 = 0;
+    }
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
-        const int bit = 2 * j * W, wi = bit >> 5, sh = bit & 31;
-        const uint32_t t = sh == 0 ? words[wi] : (sh + 2 * W > 32 ? __funnelshift_r(words[wi], words[wi + 1], sh) : words[wi] >> sh);
+        const int bit = bit0 + 2 * j * W, wi = bit >> 5, sh = bit & 31;
+        const uint32_t t = sh == 0 ? w[wi] : (sh + 2 * W > 32 ? __funnelshift_r(w[wi], wi + 1 < NWORDS ? w[wi + 1] : 0u, sh) : w[wi] >> sh);
         uint32_t u;
-        if (W == 8) u = __byte_perm(t, 0, 0x4140);                 // bytes [b0, 0, b1, 0]
-        else u = (t & ((1u << W) - 1u)) | ((t << (16 - W)) & (((1u << W) - 1u) << 16));
-        uint32_t mag = (u & kQ2) | 0x43004300u;
-        uint32_t sgn = (u << (15 - M)) & 0x80008000u;
-        uint32_t sc = (micro >> j) & 1u ? s1 : s0;
-        __nv_bfloat162 q = __hsub2(*reinterpret_cast<__nv_bfloat162*>(&mag), k128);
-        __nv_bfloat162 v = __hmul2(q, *reinterpret_cast<__nv_bfloat162*>(&sc));
-        out[j] = *reinterpret_cast<uint32_t*>(&v) | sgn;
+        if (W == 8) u = __byte_perm(t, 0, 0x4140);        // bytes [b0, 0, b1, 0]
+        else if (3 * W <= 16) u = (t & ((1u << (2 * W)) - 1u)) * ((1u << (16 - W)) + 1u);  // t | t << (16-W), no overlap
+        else u = (t & ((1u << W) - 1u)) | (t << (16 - W));
+        const uint32_t mag = (u & kQ2) | 0x43004300u;
+        const bool t1 = (micro >> j) & 1u;
+        uint32_t v;
+        if (safe) {
+            v = bf16x2_fma(mag, t1 ? s1 : s0, t1 ? n1 : n0);
+        } else {  // tiny / huge / NaN exponents: subtract first, then scale (both exact)
+            v = bf16x2_mul(bf16x2_fma(mag, 0x3F803F80u, 0xC300C300u), t1 ? s1 : s0);
+        }
+        out[j] = v | ((u << (15 - M)) & 0x80008000u);
     }
 }
 
@@ -149,6 +176,69 @@ struct GemmSmem {
     int failed;
 };
 
+// Bytes of one row's packed data for one K step, padded so that ring slots stay 8-byte aligned.
+template <int W> struct RowStep {
+    static constexpr int kElemBytes = kBK * W / 8;        // 24 / 40 / 64
+    static constexpr int kBytes = kElemBytes + 8;         // + 4 exponent bytes + 4 microexponent bytes
+    static constexpr int kRingBytes = kBytes * RingDepth<W>::value;  // one thread's ring
+};
+template <int WA, int WB> struct RingStride {
+    static constexpr int value = RowStep<WA>::kRingBytes > RowStep<WB>::kRingBytes ? RowStep<WA>::kRingBytes : RowStep<WB>::kRingBytes;
+};
+
+// The decode loop of one thread: its row's 64 elements (4 blocks) per K step.  The row's packed
+// bytes travel through a private ring in shared memory that cp.async fills kRing-1 steps ahead.
+template <int W>
+__device__ __forceinline__ bool decode_rows(const bdr_planes_t& pl, int64_t grow, int r, uint32_t tile_off, uint32_t tiles_addr,
+                                            uint8_t* ring_base, GemmSmem& gs, int nk, int lane) {
+    constexpr int NW = kBK * W / 32;  // 32-bit words of codes per K step: 6 / 10 / 16
+    constexpr int kSlot = RowStep<W>::kBytes;
+    constexpr int kRing = RingDepth<W>::value;
+    const uint8_t* ge = pl.elems + grow * pl.ld_elems;
+    const uint8_t* gx = pl.exps + grow * pl.ld_exps;
+    const uint8_t* gm = pl.micro + grow * pl.ld_micro;
+    uint8_t* ring = ring_base;  // this thread's private ring
+    auto issue = [&](int kk) {
+        if (kk < nk) {
+            uint8_t* slot = ring + (kk % kRing) * kSlot;
+#pragma unroll
+            for (int i = 0; i < RowStep<W>::kElemBytes / 8; ++i) cp_async8(slot + 8 * i, ge + (size_t)kk * RowStep<W>::kElemBytes + 8 * i);
+            cp_async4(slot + RowStep<W>::kElemBytes, gx + 4 * kk);
+            cp_async4(slot + RowStep<W>::kElemBytes + 4, gm + 4 * kk);
+        }
+        cp_async_commit();
+    };
+#pragma unroll
+    for (int i = 0; i < kRing - 1; ++i) issue(i);
+    for (int kk = 0; kk < nk; ++kk) {
+        issue(kk + kRing - 1);
+        cp_async_wait<kRing - 1>();
+        const uint32_t* slot = reinterpret_cast<const uint32_t*>(ring + (kk % kRing) * kSlot);
+        uint32_t w[NW];
+#pragma unroll
+        for (int i = 0; i < NW; ++i) w[i] = slot[i];
+        const uint32_t exps4 = slot[NW], micro4 = slot[NW + 1];
+        const int stage = kk % kStages;
+        if (kk >= kStages) {
+            bool ok = mbar_wait(&gs.empty[stage], ((kk / kStages) - 1) & 1);
+            ok = __all_sync(0xFFFFFFFFu, ok);
+            if (!ok) return false;
+        }
+        const uint32_t tile = tiles_addr + stage * kStageBytes + tile_off;
+#pragma unroll
+        for (int bb = 0; bb < kBK / kSlice; ++bb) {
+            uint32_t o[8];
+            decode_block_bf16<W, NW>(w, bb * kSlice * W, (exps4 >> (8 * bb)) & 0xFFu, (micro4 >> (8 * bb)) & 0xFFu, o);
+            st_shared_v4(tile + (((2 * bb) ^ (r & 7)) << 4), o[0], o[1], o[2], o[3]);
+            st_shared_v4(tile + (((2 * bb + 1) ^ (r & 7)) << 4), o[4], o[5], o[6], o[7]);
+        }
+        fence_proxy_async();  // make the generic-proxy stores visible to the tensor core's reads
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&gs.full[stage]);
+    }
+    return true;
+}
+
 template <int WA, int WB>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 mx_gemm_kernel(bdr_planes_t a, bdr_planes_t b, int64_t M, int64_t N, int64_t K, float* c, int64_t ldc) {
@@ -156,6 +246,7 @@ mx_gemm_kernel(bdr_planes_t a, bdr_planes_t b, int64_t M, int64_t N, int64_t K, 
     // tiles first (1024-byte aligned for the swizzle), bookkeeping after them
     uint8_t* tiles = reinterpret_cast<uint8_t*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     GemmSmem& gs = *reinterpret_cast<GemmSmem*>(tiles + kStages * kStageBytes);
+    uint8_t* ring_base = tiles + kStages * kStageBytes + 256 + (size_t)threadIdx.x * RingStride<WA, WB>::value;  // this thread's packed-byte ring
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int64_t m0 = (int64_t)blockIdx.y * kBM, n0 = (int64_t)blockIdx.x * kBN;
     const int nk = (int)(K / kBK);
@@ -174,84 +265,26 @@ mx_gemm_kernel(bdr_planes_t a, bdr_planes_t b, int64_t M, int64_t N, int64_t K, 
 
     if (warp < kDecodeWarps) {
         // ---------------- decoders ----------------
-        // Work item = half a row of the K step (2 blocks = 32 elements); 768 items, 3 per thread.
-        // Consecutive lanes take consecutive rows, so the eight 16-byte stores of a quarter-warp land
-        // in eight different swizzled positions (no bank conflicts).
+        // Thread t owns tile row t (A rows 0-127, then B rows 0-255).  Consecutive lanes hold
+        // consecutive rows, so the eight 16-byte stores of a quarter-warp land in eight different
+        // swizzled positions (no bank conflicts).  The packed bytes of K step kk+1 are fetched into
+        // registers before step kk is decoded.
+        const bool is_a = warp < kBM / 32;  // warp-uniform
+        const int r = is_a ? (int)threadIdx.x : (int)threadIdx.x - kBM;
+        const bdr_planes_t& pl = is_a ? a : b;
+        const int64_t grow = (is_a ? m0 : n0) + r;
+        const uint32_t tile_off = (uint32_t)((is_a ? 0 : kABytes) + (r >> 3) * 1024 + (r & 7) * 128);
         bool ok = true;
-        for (int kk = 0; kk < nk && ok; ++kk) {
-            const int stage = kk % kStages;
-            if (kk >= kStages) {
-                ok = mbar_wait(&gs.empty[stage], ((kk / kStages) - 1) & 1);
-                ok = __all_sync(0xFFFFFFFFu, ok);
-                if (!ok) break;
-            }
-            uint8_t* sa = tiles + stage * kStageBytes;
-#pragma unroll 1
-            for (int it = 0; it < 3; ++it) {
-                const int item = it * 256 + (int)threadIdx.x;  // 0..767
-                const int half = item / (kBM + kBN), row = item - half * (kBM + kBN);
-                const bool is_a = row < kBM;
-                const int r = is_a ? row : row - kBM;
-                const bdr_planes_t& pl = is_a ? a : b;
-                const int64_t grow = (is_a ? m0 : n0) + r;
-                const int64_t blk = (int64_t)kk * (kBK / kSlice) + half * 2;  // first of the item's two blocks
-                uint8_t* tile = sa + (is_a ? 0 : kABytes) + (r >> 3) * 1024 + (r & 7) * 128;
-                const uint32_t exps2 = *reinterpret_cast<const uint16_t*>(pl.exps + grow * pl.ld_exps + blk);
-                const uint32_t micro2 = *reinterpret_cast<const uint16_t*>(pl.micro + grow * pl.ld_micro + blk);
-                if (is_a) {
-                    constexpr int NW = (2 * kSlice * WA + 31) / 32;  // words of two blocks
-                    const uint32_t* src = reinterpret_cast<const uint32_t*>(pl.elems + grow * pl.ld_elems + blk * 2 * WA);
-                    uint32_t w[NW + 1];
-#pragma unroll
-                    for (int i = 0; i < NW; ++i) w[i] = __ldg(src + i);
-                    w[NW] = 0;
-#pragma unroll
-                    for (int bb = 0; bb < 2; ++bb) {
-                        uint32_t words[(kSlice * WA + 31) / 32 + 1];
-#pragma unroll
-                        for (int i = 0; i < (kSlice * WA + 31) / 32 + 1; ++i) {
-                            const int bit = bb * kSlice * WA + 32 * i, wi = bit >> 5, sh = bit & 31;
-                            words[i] = wi > NW ? 0u : (sh == 0 ? w[wi] : __funnelshift_r(w[wi], wi + 1 <= NW ? w[wi + 1] : 0u, sh));
-                        }
-                        uint32_t o[8];
-                        decode_block_bf16<WA>(words, (exps2 >> (8 * bb)) & 0xFFu, (micro2 >> (8 * bb)) & 0xFFu, o);
-                        const int chunk = (half * 2 + bb) * 2;  // 16-byte chunk index of the block's first 8 elements
-                        *reinterpret_cast<uint4*>(tile + ((chunk ^ (r & 7)) << 4)) = make_uint4(o[0], o[1], o[2], o[3]);
-                        *reinterpret_cast<uint4*>(tile + (((chunk + 1) ^ (r & 7)) << 4)) = make_uint4(o[4], o[5], o[6], o[7]);
-                    }
-                } else {
-                    constexpr int NW = (2 * kSlice * WB + 31) / 32;
-                    const uint32_t* src = reinterpret_cast<const uint32_t*>(pl.elems + grow * pl.ld_elems + blk * 2 * WB);
-                    uint32_t w[NW + 1];
-#pragma unroll
-                    for (int i = 0; i < NW; ++i) w[i] = __ldg(src + i);
-                    w[NW] = 0;
-#pragma unroll
-                    for (int bb = 0; bb < 2; ++bb) {
-                        uint32_t words[(kSlice * WB + 31) / 32 + 1];
-#pragma unroll
-                        for (int i = 0; i < (kSlice * WB + 31) / 32 + 1; ++i) {
-                            const int bit = bb * kSlice * WB + 32 * i, wi = bit >> 5, sh = bit & 31;
-                            words[i] = wi > NW ? 0u : (sh == 0 ? w[wi] : __funnelshift_r(w[wi], wi + 1 <= NW ? w[wi + 1] : 0u, sh));
-                        }
-                        uint32_t o[8];
-                        decode_block_bf16<WB>(words, (exps2 >> (8 * bb)) & 0xFFu, (micro2 >> (8 * bb)) & 0xFFu, o);
-                        const int chunk = (half * 2 + bb) * 2;
-                        *reinterpret_cast<uint4*>(tile + ((chunk ^ (r & 7)) << 4)) = make_uint4(o[0], o[1], o[2], o[3]);
-                        *reinterpret_cast<uint4*>(tile + (((chunk + 1) ^ (r & 7)) << 4)) = make_uint4(o[4], o[5], o[6], o[7]);
-                    }
-                }
-            }
-            fence_proxy_async();  // make the generic-proxy stores visible to the tensor core's reads
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&gs.full[stage]);
-        }
+        if (is_a) ok = decode_rows<WA>(pl, grow, r, tile_off, smem_u32(tiles), ring_base, gs, nk, lane);
+        else ok = decode_rows<WB>(pl, grow, r, tile_off, smem_u32(tiles), ring_base, gs, nk, lane);
         if (!ok) gs.failed = 1;
 
         // ---------------- epilogue ----------------
-        bool done = ok && mbar_wait(&gs.accum, 0);
+        bool done = ok && warp < kEpilogueWarps && mbar_wait(&gs.accum, 0);
         done = __all_sync(0xFFFFFFFFu, done);
-        if (done) {
+        if (warp >= kEpilogueWarps) {
+            // decoders 8-11 have no accumulator lanes to drain
+        } else if (done) {
             tc_fence_after();
             const int lane_base = (warp & 3) * 32;            // a warp may only touch its own 32 TMEM lanes
             const int col_base = (warp >> 2) * (kBN / 2);     // warps 0-3: columns 0-127, warps 4-7: 128-255
@@ -302,7 +335,7 @@ template <int WA, int WB>
 static int launch_gemm(const bdr_planes_t& a, const bdr_planes_t& b, int64_t M, int64_t N, int64_t K, float* c, int64_t ldc,
                        cudaStream_t st) {
     auto kern = mx_gemm_kernel<WA, WB>;
-    const size_t smem = (size_t)kStages * kStageBytes + sizeof(GemmSmem) + 1024;
+    const size_t smem = (size_t)kStages * kStageBytes + 256 + (size_t)(kBM + kBN) * RingStride<WA, WB>::value + 1024;
     static bool attr_done = false;
     if (!attr_done) {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return BDR_ERR_CUDA;
