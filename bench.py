@@ -3,8 +3,8 @@
 
 One "step" = one pass of the whole quantization path over one 8192 x 8192 bf16 activation tensor
 (Laplace(0,1), 1% outlier columns x50): for each of MX4 / MX6 / MX9 and each direction (row-wise,
-column-wise) a quantize-dequantize with fused QSNR sums, a quantize+pack with fused QSNR sums, and
-an unpack+dequantize -- 18 kernel launches.  `value` is the algorithmic bytes those 18 operations
+column-wise) a quantize-dequantize with fused QSNR sums, a quantize+pack, and an unpack+dequantize
+-- 18 kernel launches.  `value` is the algorithmic bytes those 18 operations
 must move divided by the device time (GB/s); the MX-GEMM and design-sweep legs are measured
 separately after the timed steps and reported in the same JSON line.
 
@@ -217,7 +217,7 @@ def run_ours(args):
         if op == "quant_dequant":
             bdr.bdr_quant_dequant(cfgs[name], x, y, axis=axis, qsnr_sums=sums[i])
         elif op == "pack":
-            bdr.bdr_pack(cfgs[name], x, planes[(name, axis)], axis=axis, qsnr_sums=sums[i])
+            bdr.bdr_pack(cfgs[name], x, planes[(name, axis)], axis=axis)
         else:
             bdr.bdr_unpack(cfgs[name], planes[(name, axis)], y, axis=axis)
 
@@ -257,7 +257,7 @@ def run_ours(args):
     qsnr = {}
     sums_np = (sums / args.steps).cpu().numpy()
     for i, (name, _m, axis, op) in enumerate(ops):
-        if op == "pack":
+        if op == "quant_dequant":
             qsnr["%s_axis%d" % (name, axis)] = float(-10.0 * np.log10(sums_np[i, 0] / sums_np[i, 1]))
 
     # ---- per-kernel timing on the launching stream (roofline of the dominant kernel) ----
@@ -323,7 +323,7 @@ def run_ours(args):
                 "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
                 "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
                 "config": {"workload": "C3: 8192x8192 bf16 Laplace(0,1), 1% outlier columns x50; MX4/MX6/MX9 x "
-                                       "row/column x (quant-dequant+QSNR, pack+QSNR, unpack)",
+                                       "row/column x (quant-dequant+QSNR, pack, unpack)",
                            "l2": "inputs larger than L2 (134 MB tensor, >=168 MB streamed per launch)",
                            "replicas": "independent tensor per rank, no collective"},
                 "frac_of_hbm_peak": value / world / peak, "roofline": roofline, "kernels": kernels,
@@ -337,11 +337,8 @@ def run_ours(args):
 
 def secondary_legs(args, bdr, synth, torch) -> dict:
     """MX-GEMM TFLOP/s and design-sweep configs/s, when those entry points are built."""
+    from paper_2302_08007_b200 import legs
     out = {}
-    try:
-        from paper_2302_08007_b200 import legs
-    except ImportError:
-        return out
     for fn in (legs.gemm_leg, legs.sweep_leg):
         try:
             out.update(fn(args))
