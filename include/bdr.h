@@ -123,6 +123,23 @@ int bdr_qsnr(const bdr_config_t* cfgs /*host*/, int n_cfgs, const void* x, bdr_d
              int64_t cols, int64_t ld, int axis, double* qsnr_db_dev, void* workspace, int64_t workspace_bytes,
              void* stream);
 
+/* The same sweep as bdr_qsnr for callers that cannot hand over scratch memory.  (The paper has no
+ * counterpart; this is a convenience of this library.)  Think of a monitoring hook that runs inside
+ * another framework's training step, or a serving loop with a fixed memory plan: all device memory
+ * already belongs to that framework's pool, a cudaMalloc could fail, and it would stall the GPU
+ * because allocation and free synchronise the device.  This entry point therefore allocates nothing:
+ * its scratch is an array built into the library (about 20 KB that every GPU loading the library
+ * holds until the process ends).
+ *   - at most bdr_qsnr_static_max_cfgs() (= 512) configurations per call; more is BDR_ERR_SIZE
+ *   - inputs, outputs, validation and results are exactly those of bdr_qsnr
+ *   - the first call on each device looks up the array's device address (a host-side query, no
+ *     allocation); make that first call outside any stream capture
+ *   - all calls on a device share the one array: it is cleared at the start of every call, and two
+ *     calls whose GPU work overlaps (different streams, or threads) race on it -- serialise them */
+int bdr_qsnr_static_max_cfgs(void);
+int bdr_qsnr_static(const bdr_config_t* cfgs /*host*/, int n_cfgs, const void* x, bdr_dtype_t dt, int64_t rows,
+                    int64_t cols, int64_t ld, int axis, double* qsnr_db_dev, void* stream);
+
 /* C[M,N] (fp32, row pitch ldc elements) = deq(A)[M,K] * deq(B)[N,K]^T with both operands given as
  * packed planes quantized along K (axis 1 planes of A and of B), decoded to bf16 inside the kernel
  * and accumulated in fp32 on the tensor cores (Section V: both inputs of a tensor operation are

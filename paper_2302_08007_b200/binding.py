@@ -20,7 +20,8 @@ ROUND_NEAREST_EVEN, ROUND_NEAREST_AWAY = 0, 1
 F32, BF16 = 0, 1
 
 EXPORTS = ("bdr_strerror", "bdr_packed_sizes", "bdr_quant_dequant", "bdr_pack", "bdr_unpack",
-           "bdr_qsnr_workspace_bytes", "bdr_qsnr", "mx_gemm", "mx_gemm_status")
+           "bdr_qsnr_workspace_bytes", "bdr_qsnr", "bdr_qsnr_static_max_cfgs", "bdr_qsnr_static", "mx_gemm",
+           "mx_gemm_status")
 
 
 class BdrError(RuntimeError):
@@ -97,6 +98,11 @@ def lib():
                                C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p]
         L.mx_gemm.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_int64, C.c_int64,
                               C.c_void_p, C.c_int64, C.c_void_p]
+        L.bdr_qsnr_static_max_cfgs.restype = C.c_int
+        L.bdr_qsnr_static_max_cfgs.argtypes = []
+        L.bdr_qsnr_static.restype = C.c_int
+        L.bdr_qsnr_static.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_int, C.c_int64, C.c_int64, C.c_int64, C.c_int,
+                                      C.c_void_p, C.c_void_p]
         L.mx_gemm_status.restype = C.c_int
         L.mx_gemm_status.argtypes = []
         for fn in (L.bdr_packed_sizes, L.bdr_quant_dequant, L.bdr_pack, L.bdr_unpack, L.bdr_qsnr, L.mx_gemm):
@@ -201,6 +207,21 @@ def bdr_qsnr(cfgs, x: torch.Tensor, out_db: torch.Tensor, workspace: torch.Tenso
     _check(lib().bdr_qsnr(C.addressof(arr), len(cfgs), _ptr(x2), _dt(x2), x2.shape[0], x2.shape[1], x2.stride(0), axis,
                           _ptr(out_db), _ptr(workspace), workspace.numel() * workspace.element_size(),
                           _stream(stream)), "bdr_qsnr")
+    return out_db
+
+
+def bdr_qsnr_static_max_cfgs() -> int:
+    return int(lib().bdr_qsnr_static_max_cfgs())
+
+
+def bdr_qsnr_static(cfgs, x: torch.Tensor, out_db: torch.Tensor, axis: int = 1, stream=None):
+    """bdr_qsnr without a workspace argument: the scratch is built into the library, for callers that
+    must not allocate device memory (see include/bdr.h).  At most bdr_qsnr_static_max_cfgs()
+    configurations; calls that overlap on the GPU race on the shared scratch."""
+    x2 = _as2d(x)
+    arr = (_Config * len(cfgs))(*[c.c() for c in cfgs])
+    _check(lib().bdr_qsnr_static(C.addressof(arr), len(cfgs), _ptr(x2), _dt(x2), x2.shape[0], x2.shape[1], x2.stride(0),
+                                 axis, _ptr(out_db), _stream(stream)), "bdr_qsnr_static")
     return out_db
 
 

@@ -13,6 +13,7 @@
 // The comparator kinds of Table I (INT with an FP32 max-scale, Eq. 1-2; FP8-like scalar floats;
 // VSQ) are evaluated in the same loop with IEEE single operations (division included), so their
 // dequantized values match a plain CPU implementation bit for bit.
+#include <mutex>
 #include <vector>
 
 #include "bdr_device.cuh"
@@ -25,7 +26,6 @@ constexpr int kSweepWarps = kSweepThreads / 32;
 constexpr int kTile = 4096;                    // elements per tile: a multiple of every k1 <= 1024
 constexpr int kTileSlices = kTile / kSlice;    // 256
 constexpr int kCfgGroup = 64;                  // configurations evaluated per tile visit
-constexpr int kLevels = 10;                    // block sizes 2^1 .. 2^10
 
 struct SweepCfg {
     int32_t kind, k1, k2, d2, m, rounding;
@@ -376,6 +376,31 @@ static int sweep_launch(const SweepCfg* host_cfgs, int n, bool need_amax, const 
     return cudaGetLastError() == cudaSuccess ? BDR_OK : BDR_ERR_CUDA;
 }
 
+// ---- built-in scratch for callers that cannot allocate ---------------------------------------------
+// bdr_qsnr_static keeps its scratch in this file-scope device array instead of taking a workspace
+// pointer.  Every GPU that loads the library holds these bytes until the process exits.  In host
+// code the array's name is only a stand-in symbol, not a device address, so the address a kernel can
+// use is looked up once per device with cudaGetSymbolAddress (below) while that device is current.
+constexpr int kStaticMaxCfgs = 512;
+constexpr size_t kStaticScratchBytes = 20736;  // = sweep_workspace_bytes(512)
+static __device__ __align__(256) unsigned char g_qsnr_static_scratch[kStaticScratchBytes];
+
+// Device address of the built-in scratch on the current device (set up on first use per device).
+static int static_scratch_ptr(uint8_t** out) {
+    static std::mutex mu;
+    static uint8_t* cached[64];
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return BDR_ERR_CUDA;
+    std::lock_guard<std::mutex> lock(mu);
+    if (!cached[dev]) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_qsnr_static_scratch) != cudaSuccess || !p) return BDR_ERR_CUDA;
+        cached[dev] = static_cast<uint8_t*>(p);
+    }
+    *out = cached[dev];
+    return BDR_OK;
+}
+
 }  // namespace bdr
 
 using namespace bdr;
@@ -409,6 +434,19 @@ int bdr_qsnr(const bdr_config_t* cfgs, int n_cfgs, const void* x, bdr_dtype_t dt
         return sweep_launch<float>(table.data(), n_cfgs, need_amax, (const float*)x, rows, cols, ld, qsnr_db_dev, (uint8_t*)workspace, st);
     return sweep_launch<__nv_bfloat16>(table.data(), n_cfgs, need_amax, (const __nv_bfloat16*)x, rows, cols, ld, qsnr_db_dev,
                                        (uint8_t*)workspace, st);
+}
+
+int bdr_qsnr_static_max_cfgs(void) { return kStaticMaxCfgs; }
+
+int bdr_qsnr_static(const bdr_config_t* cfgs, int n_cfgs, const void* x, bdr_dtype_t dt, int64_t rows, int64_t cols,
+                    int64_t ld, int axis, double* qsnr_db_dev, void* stream) {
+    static_assert(kStaticScratchBytes % 256 == 0, "scratch size is a multiple of its alignment");
+    if (n_cfgs > kStaticMaxCfgs) return BDR_ERR_SIZE;  // more configurations than the built-in scratch holds
+    if (n_cfgs >= 1 && sweep_workspace_bytes(n_cfgs) > (int64_t)kStaticScratchBytes) return BDR_ERR_SIZE;
+    uint8_t* scratch = nullptr;
+    const int rc = static_scratch_ptr(&scratch);  // first call on a device resolves the symbol's address
+    if (rc) return rc;
+    return bdr_qsnr(cfgs, n_cfgs, x, dt, rows, cols, ld, axis, qsnr_db_dev, scratch, (int64_t)kStaticScratchBytes, stream);
 }
 
 }  // extern "C"
