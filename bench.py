@@ -339,7 +339,7 @@ def secondary_legs(args, bdr, synth, torch) -> dict:
     """MX-GEMM TFLOP/s and design-sweep configs/s, when those entry points are built."""
     from paper_2302_08007_b200 import legs
     out = {}
-    for fn in (legs.gemm_leg, legs.sweep_leg):
+    for fn in (legs.gemm_leg, legs.sweep_leg, legs.linear_leg):
         try:
             out.update(fn(args))
         except bdr.BdrError as e:

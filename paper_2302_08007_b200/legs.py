@@ -6,7 +6,7 @@ import numpy as np
 import torch
 
 from . import binding as bdr
-from . import sweep, synth
+from . import linear, sweep, synth
 
 SWEEP_N = 1 << 24
 
@@ -63,3 +63,19 @@ def gemm_leg(args) -> dict:
     ms = _time(lambda: bdr.mx_gemm(bdr.MX6, pa, bdr.MX6, pb, M, N, K, c), reps=20, warmup=3)
     return {"mx_gemm": {"metric": "MX-GEMM TFLOP/s", "value": 2.0 * M * N * K / (ms * 1e-3) / 1e12, "unit": "TFLOP/s",
                         "ms": ms, "shape": [M, N, K], "format": "MX6 x MX6", "bound": "tensor"}}
+
+
+def linear_leg(args) -> dict:
+    """One transformer linear layer in MX9 training form: X[8192x4096], W[16384x4096], dY[8192x16384]
+    (bf16); six quantizations with fused QSNR and three MX GEMMs (forward, dX, dW)."""
+    tokens, d_in, d_out = 8192, 4096, 16384
+    bf = lambda a: torch.from_numpy(synth.f32_to_bf16_bits(a).view(np.int16)).view(torch.bfloat16).cuda()
+    x = bf(synth.outlier_channel_matrix(tokens, d_in, seed=0, stream=1, frac=0.01, gain=20.0))
+    w = bf(synth.normal_matrix(d_out, d_in, seed=0, stream=2, sigma=0.02))
+    dy = bf(synth.normal_matrix(tokens, d_out, seed=0, stream=3, sigma=1e-3))
+    buf = linear.alloc(bdr.MX9, tokens, d_in, d_out)
+    ms = _time(lambda: linear.step(bdr.MX9, x, w, dy, buf), reps=3)
+    flops = 3 * 2.0 * tokens * d_in * d_out
+    return {"linear_layer": {"workload": "MX9 linear layer fwd+bwd: 6 quantize+pack (+QSNR), 3 mx_gemm", "ms": ms,
+                             "gemm_tflops_incl_quantization": flops / (ms * 1e-3) / 1e12,
+                             "qsnr_db": linear.qsnr_db(buf), "mx_gemm_status": bdr.mx_gemm_status()}}

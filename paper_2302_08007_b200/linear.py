@@ -1,0 +1,60 @@
+"""One linear layer in MX training form (Section V, Fig. 8): every matmul of the forward and the
+backward pass takes both operands MX-quantized along that matmul's reduction dimension, so each of
+X, W and dY is quantized twice -- once along its rows and once along its columns (the "transpose,
+then quantize" copy).  This module only sequences calls of the C ABI; all arithmetic is in the
+kernels.
+
+    Y  = X  W^T   reduce over in-features : X  row-wise, W  row-wise
+    dX = dY W     reduce over out-features: dY row-wise, W  column-wise
+    dW = dY^T X   reduce over tokens      : dY column-wise, X column-wise
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass
+
+import torch
+
+from . import binding as bdr
+
+
+@dataclass
+class LinearBuffers:
+    """Everything the step writes, allocated once by the caller."""
+    planes: dict           # (name, axis) -> Planes
+    sums: torch.Tensor     # [6, 2] float64: Eq. 3 sums of the six quantizations
+    y: torch.Tensor        # [tokens, out] float32
+    dx: torch.Tensor       # [tokens, in] float32
+    dw: torch.Tensor       # [out, in] float32
+
+
+ORDER = (("x", 1), ("x", 0), ("w", 1), ("w", 0), ("dy", 1), ("dy", 0))
+
+
+def alloc(cfg: bdr.Config, tokens: int, d_in: int, d_out: int, device="cuda") -> LinearBuffers:
+    shapes = {"x": (tokens, d_in), "w": (d_out, d_in), "dy": (tokens, d_out)}
+    planes = {(n, ax): bdr.alloc_planes(cfg, *shapes[n], ax, device=device) for n, ax in ORDER}
+    return LinearBuffers(planes, torch.zeros((6, 2), dtype=torch.float64, device=device),
+                         torch.empty((tokens, d_out), dtype=torch.float32, device=device),
+                         torch.empty((tokens, d_in), dtype=torch.float32, device=device),
+                         torch.empty((d_out, d_in), dtype=torch.float32, device=device))
+
+
+def step(cfg: bdr.Config, x: torch.Tensor, w: torch.Tensor, dy: torch.Tensor, buf: LinearBuffers, stream=None):
+    """Six quantizations (with fused QSNR sums) and three MX GEMMs.  Returns (Y, dX, dW)."""
+    tokens, d_in = x.shape
+    d_out = w.shape[0]
+    src = {"x": x, "w": w, "dy": dy}
+    buf.sums.zero_()
+    for i, (n, ax) in enumerate(ORDER):
+        bdr.bdr_pack(cfg, src[n], buf.planes[(n, ax)], axis=ax, qsnr_sums=buf.sums[i], stream=stream)
+    p = buf.planes
+    bdr.mx_gemm(cfg, p[("x", 1)], cfg, p[("w", 1)], tokens, d_out, d_in, buf.y, stream=stream)      # Y  = X W^T
+    bdr.mx_gemm(cfg, p[("dy", 1)], cfg, p[("w", 0)], tokens, d_in, d_out, buf.dx, stream=stream)    # dX = dY W
+    bdr.mx_gemm(cfg, p[("dy", 0)], cfg, p[("x", 0)], d_out, d_in, tokens, buf.dw, stream=stream)    # dW = dY^T X
+    return buf.y, buf.dx, buf.dw
+
+
+def qsnr_db(buf: LinearBuffers) -> dict:
+    s = buf.sums.cpu()
+    return {"%s_%s" % (n, "row" if ax == 1 else "col"): float(-10.0 * torch.log10(s[i, 0] / s[i, 1]))
+            for i, (n, ax) in enumerate(ORDER)}
