@@ -13,6 +13,8 @@
 // K step warps 0-7 read the accumulator from tensor memory (tcgen05.ld) and store C.  Every wait is bounded: if one runs out the kernel
 // records BDR_ERR_TIMEOUT in a status word, skips the remaining work, frees its tensor memory and
 // returns.
+#include <cuda.h>
+
 #include "bdr_device.cuh"
 #include "bdr_host.h"
 
@@ -331,6 +333,12 @@ mx_gemm_kernel(bdr_planes_t a, bdr_planes_t b, int64_t M, int64_t N, int64_t K, 
     if (threadIdx.x == 0 && gs.failed) atomicExch(&g_gemm_status, (int)BDR_ERR_TIMEOUT);
 }
 
+}  // namespace bdr
+
+#include "mx_gemm_pair.cuh"
+
+namespace bdr {
+
 template <int WA, int WB>
 static int launch_gemm(const bdr_planes_t& a, const bdr_planes_t& b, int64_t M, int64_t N, int64_t K, float* c, int64_t ldc,
                        cudaStream_t st) {
@@ -349,10 +357,15 @@ static int launch_gemm(const bdr_planes_t& a, const bdr_planes_t& b, int64_t M, 
 template <int WA>
 static int gemm_pick_b(int mb, const bdr_planes_t& a, const bdr_planes_t& b, int64_t M, int64_t N, int64_t K, float* c,
                        int64_t ldc, cudaStream_t st) {
+    // 2-CTA kernel when the shape allows whole 256-row pairs and 256-element K chunks
+    const bool pair = M % 256 == 0 && K % kChunkK == 0 && M / 128 <= 0x7FFFFFFF && N / 256 <= 65535;
     switch (mb) {
-        case 2: return launch_gemm<WA, 3>(a, b, M, N, K, c, ldc, st);
-        case 4: return launch_gemm<WA, 5>(a, b, M, N, K, c, ldc, st);
-        case 7: return launch_gemm<WA, 8>(a, b, M, N, K, c, ldc, st);
+        case 2: { const int rc = pair ? launch_gemm_pair<WA, 3>(a, b, M, N, K, c, ldc, st) : BDR_ERR_UNSUPPORTED;
+                  return rc == BDR_ERR_UNSUPPORTED ? launch_gemm<WA, 3>(a, b, M, N, K, c, ldc, st) : rc; }
+        case 4: { const int rc = pair ? launch_gemm_pair<WA, 5>(a, b, M, N, K, c, ldc, st) : BDR_ERR_UNSUPPORTED;
+                  return rc == BDR_ERR_UNSUPPORTED ? launch_gemm<WA, 5>(a, b, M, N, K, c, ldc, st) : rc; }
+        case 7: { const int rc = pair ? launch_gemm_pair<WA, 8>(a, b, M, N, K, c, ldc, st) : BDR_ERR_UNSUPPORTED;
+                  return rc == BDR_ERR_UNSUPPORTED ? launch_gemm<WA, 8>(a, b, M, N, K, c, ldc, st) : rc; }
     }
     return BDR_ERR_UNSUPPORTED;
 }

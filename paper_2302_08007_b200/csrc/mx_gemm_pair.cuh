@@ -1,0 +1,327 @@
+// mx_gemm, 2-CTA version: a cluster of two CTAs computes a 256 x 256 tile of C with
+// tcgen05.mma.cta_group::2 (each CTA owns 128 rows of the accumulator in its own tensor memory and
+// supplies its 128 rows of A and its 128-row half of the B tile from its own shared memory).
+//
+// Per CTA:  one thread of warp 8 streams the packed bytes of the CTA's 256 operand rows into shared
+// memory with 2-D TMA tile loads (cp.async.bulk.tensor, one per plane: 128 rows x 256 K-elements of
+// codes, exponents or microexponents; no multicast; completion on an mbarrier), so no thread ever
+// waits on an uncoalesced global load;  warps 0-7 (one thread per row)
+// decode those bytes to bf16 and store them in the K-major 128-byte-swizzled operand stages;  in the
+// leader CTA one thread of warp 9 issues the MMAs once the decoders of BOTH CTAs have arrived on its
+// "full" barrier, and tcgen05.commit (multicast to both CTAs) releases the stage and, at the end,
+// signals the epilogue;  warps 0-7 then drain their CTA's accumulator with tcgen05.ld.
+// Every wait is bounded; a wait that runs out sets the status word and the CTA falls through to the
+// final cluster barrier, frees its tensor memory and returns.
+// (textually included by mx_gemm.cu, which defines the shared PTX wrappers, the decoder and the status word)
+#pragma once
+
+namespace bdr {
+
+constexpr int kPairRows = 128;                  // rows of A and of the B half per CTA
+constexpr int kChunkK = 256;                    // K elements per bulk-copy chunk (4 K steps)
+constexpr int kStepsPerChunk = kChunkK / kBK;   // 4
+constexpr int kPairDecodeWarps = 8;
+constexpr int kLoaderWarp = 8, kMmaWarp = 9;
+constexpr int kPairThreads = 10 * 32;
+constexpr int kPairStageBytes = 2 * kPairRows * kBK * 2;  // A 16 KB + B half 16 KB
+
+// Packed bytes of one chunk (256 K elements) for 128 rows, as the TMA writes them: dense row-major
+// arrays [128][codes], [128][16 exponent bytes], [128][16 microexponent bytes].
+template <int W> struct ChunkPlanes {
+    static constexpr int kElemRow = kChunkK * W / 8;  // 96 / 160 / 256 bytes of codes per row
+    static constexpr int kElems = 0;
+    static constexpr int kExps = kPairRows * kElemRow;
+    static constexpr int kMicro = kExps + kPairRows * 16;
+    static constexpr int kBytes = kMicro + kPairRows * 16;  // a multiple of 128
+};
+template <int WA, int WB> struct PairSmem {
+    static constexpr int kPackedBytes = ChunkPlanes<WA>::kBytes + ChunkPlanes<WB>::kBytes;  // one buffer
+    static constexpr int kBudget = 224 * 1024 - 2 * kPackedBytes - 1024;
+    static constexpr int kStages = kBudget / kPairStageBytes >= 4 ? 4 : kBudget / kPairStageBytes;
+    static_assert(kStages >= 2, "operand stages do not fit");
+    static constexpr size_t kBytes = (size_t)kStages * kPairStageBytes + 2 * kPackedBytes + 1024 /*bookkeeping*/ + 1024 /*alignment*/;
+};
+
+struct PairMaps {  // tensor maps of the three planes of A and of B (uint8 elements, rows x row bytes)
+    CUtensorMap a_elems, a_exps, a_micro, b_elems, b_exps, b_micro;
+};
+
+struct PairBars {
+    uint64_t full[4], empty[4], accum, pk_full[2], pk_empty[2];
+    uint32_t tmem_base;
+    int failed;
+};
+
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// arrive on the barrier at the same shared-memory offset in CTA `rank` of the cluster
+__device__ __forceinline__ void mbar_arrive_cluster(uint64_t* bar, uint32_t rank) {
+    uint32_t remote;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(smem_u32(bar)), "r"(rank));
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(remote) : "memory");
+}
+__device__ __forceinline__ bool mbar_wait_cluster(uint64_t* bar, uint32_t parity) {
+    const uint32_t addr = smem_u32(bar);
+    for (uint32_t it = 0; it < kSpinLimit; ++it) {
+        uint32_t done;
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(done)
+            : "r"(addr), "r"(parity)
+            : "memory");
+        if (done) return true;
+    }
+    return false;
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+// 2-D tile load: box starts at byte x of row y (x must be a multiple of 16)
+__device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, int x, int y, uint64_t* bar) {
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+                 ::"r"(smem_u32(dst)), "l"(map), "r"(x), "r"(y), "r"(smem_u32(bar))
+                 : "memory");
+}
+__device__ __forceinline__ void tmem_alloc2(uint32_t* dst_smem, uint32_t ncols) {
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(dst_smem)), "r"(ncols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc2(uint32_t taddr, uint32_t ncols) {
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+// arrive (once the issuing thread's earlier MMAs have completed) on the barrier at this offset in both CTAs
+__device__ __forceinline__ void umma_commit2(uint64_t* bar) {
+    const uint16_t mask = 3;
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                 ::"r"(smem_u32(bar)), "h"(mask)
+                 : "memory");
+}
+__device__ __forceinline__ void umma2_bf16(uint32_t tmem_d, uint64_t desc_a, uint64_t desc_b, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(tmem_d), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// D = fp32, A = B = bf16, both K-major, N = 256, M = 256 (128 rows per CTA)
+constexpr uint32_t kPairInstrDesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(256 >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
+
+// pk0 / pk1: this operand's ChunkPlanes in the two packed buffers
+template <int W>
+__device__ __forceinline__ bool pair_decode_rows(const uint8_t* pk0, const uint8_t* pk1, int r, uint32_t tile_off,
+                                                 uint32_t stages_addr, int n_stages, PairBars& bars, int nk, int lane) {
+    constexpr int NW = kBK * W / 32;  // code words per K step
+    for (int kk = 0; kk < nk; ++kk) {
+        const int chunk = kk / kStepsPerChunk, ks = kk % kStepsPerChunk, buf = chunk & 1;
+        if (ks == 0) {
+            bool ok = mbar_wait(&bars.pk_full[buf], (chunk >> 1) & 1);
+            ok = __all_sync(0xFFFFFFFFu, ok);
+            if (!ok) return false;
+        }
+        const uint8_t* pk = buf ? pk1 : pk0;
+        uint32_t w[NW];
+        const uint2* src = reinterpret_cast<const uint2*>(pk + ChunkPlanes<W>::kElems + r * ChunkPlanes<W>::kElemRow + ks * (kBK * W / 8));
+#pragma unroll
+        for (int i = 0; i < NW / 2; ++i) { const uint2 v = src[i]; w[2 * i] = v.x; w[2 * i + 1] = v.y; }
+        const uint32_t exps4 = *reinterpret_cast<const uint32_t*>(pk + ChunkPlanes<W>::kExps + r * 16 + 4 * ks);
+        const uint32_t micro4 = *reinterpret_cast<const uint32_t*>(pk + ChunkPlanes<W>::kMicro + r * 16 + 4 * ks);
+        const int stage = kk % n_stages;
+        if (kk >= n_stages) {
+            bool ok = mbar_wait(&bars.empty[stage], ((kk / n_stages) - 1) & 1);
+            ok = __all_sync(0xFFFFFFFFu, ok);
+            if (!ok) return false;
+        }
+        const uint32_t tile = stages_addr + stage * kPairStageBytes + tile_off;
+#pragma unroll
+        for (int bb = 0; bb < kBK / kSlice; ++bb) {
+            uint32_t o[8];
+            decode_block_bf16<W, NW>(w, bb * kSlice * W, (exps4 >> (8 * bb)) & 0xFFu, (micro4 >> (8 * bb)) & 0xFFu, o);
+            st_shared_v4(tile + (((2 * bb) ^ (r & 7)) << 4), o[0], o[1], o[2], o[3]);
+            st_shared_v4(tile + (((2 * bb + 1) ^ (r & 7)) << 4), o[4], o[5], o[6], o[7]);
+        }
+        fence_proxy_async();  // generic-proxy stores -> visible to the tensor core's (async proxy) reads
+        __syncwarp();
+        if (lane == 0) {
+            mbar_arrive_cluster(&bars.full[stage], 0);                            // the leader CTA counts both CTAs' decoders
+            if (ks == kStepsPerChunk - 1) mbar_arrive(&bars.pk_empty[buf]);       // this warp is done with the packed buffer
+        }
+    }
+    return true;
+}
+
+template <int WA, int WB>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kPairThreads, 1)
+mx_gemm_pair_kernel(const __grid_constant__ PairMaps maps, int64_t M, int64_t N, int64_t K, float* c, int64_t ldc) {
+    using SM = PairSmem<WA, WB>;
+    constexpr int kStages = SM::kStages;
+    extern __shared__ __align__(1024) uint8_t smem_raw[];
+    uint8_t* stages = reinterpret_cast<uint8_t*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    uint8_t* pk[2] = {stages + kStages * kPairStageBytes, stages + kStages * kPairStageBytes + SM::kPackedBytes};
+    PairBars& bars = *reinterpret_cast<PairBars*>(stages + kStages * kPairStageBytes + 2 * SM::kPackedBytes);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = cluster_ctarank();
+    const int64_t m0 = ((int64_t)(blockIdx.x >> 1) * 2 + rank) * kPairRows;  // this CTA's rows of A and C
+    const int64_t n0 = (int64_t)blockIdx.y * 256;                             // the pair's columns
+    const int64_t nb0 = n0 + (int64_t)rank * kPairRows;                       // this CTA's half of the B tile
+    const int nk = (int)(K / kBK), nchunks = (int)(K / kChunkK);
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < 4; ++s) { mbar_init(&bars.full[s], 2 * kPairDecodeWarps); mbar_init(&bars.empty[s], 1); }
+        mbar_init(&bars.accum, 1);
+        for (int i = 0; i < 2; ++i) { mbar_init(&bars.pk_full[i], 1); mbar_init(&bars.pk_empty[i], kPairDecodeWarps); }
+        bars.failed = 0;
+        fence_barrier_init();
+    }
+    if (warp == kMmaWarp) tmem_alloc2(&bars.tmem_base, 256);  // 256 fp32 columns x 128 lanes in each CTA
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();  // both CTAs' barriers are initialised before anyone signals across the cluster
+    tc_fence_after();
+    const uint32_t tmem_base = bars.tmem_base;
+
+    if (warp < kPairDecodeWarps) {
+        // ---------------- decoders: thread t owns row t (A rows 0-127, then the B half's 128 rows) ----------------
+        const bool is_a = warp < kPairRows / 32;
+        const int r = is_a ? (int)threadIdx.x : (int)threadIdx.x - kPairRows;
+        const uint32_t tile_off = (uint32_t)((is_a ? 0 : kPairRows * kBK * 2) + (r >> 3) * 1024 + (r & 7) * 128);
+        bool ok;
+        if (is_a) ok = pair_decode_rows<WA>(pk[0], pk[1], r, tile_off, smem_u32(stages), kStages, bars, nk, lane);
+        else ok = pair_decode_rows<WB>(pk[0] + ChunkPlanes<WA>::kBytes, pk[1] + ChunkPlanes<WA>::kBytes, r, tile_off,
+                                       smem_u32(stages), kStages, bars, nk, lane);
+        if (!ok) bars.failed = 1;
+
+        // ---------------- epilogue: this CTA's 128 x 256 block of C ----------------
+        bool done = ok && mbar_wait(&bars.accum, 0);
+        done = __all_sync(0xFFFFFFFFu, done);
+        if (done) {
+            tc_fence_after();
+            const int lane_base = (warp & 3) * 32, col_base = (warp >> 2) * 128;
+            float* crow = c + (m0 + lane_base + lane) * ldc + n0 + col_base;
+#pragma unroll 1
+            for (int cc = 0; cc < 128; cc += 32) {
+                uint32_t v[32];
+                tmem_ld32(tmem_base + ((uint32_t)lane_base << 16) + (uint32_t)(col_base + cc), v);
+#pragma unroll
+                for (int q = 0; q < 8; ++q)
+                    *reinterpret_cast<uint4*>(crow + cc + 4 * q) = make_uint4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
+            }
+        } else {
+            bars.failed = 1;
+        }
+        tc_fence_before();
+    } else if (warp == kLoaderWarp) {
+        // ---------------- loader: six TMA tile loads per chunk (256 K elements x 128 rows per plane) ----------------
+        if (lane == 0) {
+            bool ok = true;
+            for (int ch = 0; ch < nchunks; ++ch) {
+                const int buf = ch & 1;
+                if (ch >= 2) {
+                    ok = mbar_wait(&bars.pk_empty[buf], ((ch >> 1) - 1) & 1);
+                    if (!ok) break;
+                }
+                uint8_t* pa = pk[buf];
+                uint8_t* pb = pk[buf] + ChunkPlanes<WA>::kBytes;
+                mbar_expect_tx(&bars.pk_full[buf], (uint32_t)SM::kPackedBytes);
+                tma_load_2d(pa + ChunkPlanes<WA>::kElems, &maps.a_elems, ch * ChunkPlanes<WA>::kElemRow, (int)m0, &bars.pk_full[buf]);
+                tma_load_2d(pa + ChunkPlanes<WA>::kExps, &maps.a_exps, ch * 16, (int)m0, &bars.pk_full[buf]);
+                tma_load_2d(pa + ChunkPlanes<WA>::kMicro, &maps.a_micro, ch * 16, (int)m0, &bars.pk_full[buf]);
+                tma_load_2d(pb + ChunkPlanes<WB>::kElems, &maps.b_elems, ch * ChunkPlanes<WB>::kElemRow, (int)nb0, &bars.pk_full[buf]);
+                tma_load_2d(pb + ChunkPlanes<WB>::kExps, &maps.b_exps, ch * 16, (int)nb0, &bars.pk_full[buf]);
+                tma_load_2d(pb + ChunkPlanes<WB>::kMicro, &maps.b_micro, ch * 16, (int)nb0, &bars.pk_full[buf]);
+            }
+            if (!ok) bars.failed = 1;
+        }
+        __syncwarp();
+    } else {
+        // ---------------- MMA issuer: one lane of the leader CTA ----------------
+        if (rank == 0 && lane == 0) {
+            bool ok = true;
+            for (int kk = 0; kk < nk; ++kk) {
+                const int stage = kk % kStages;
+                ok = mbar_wait_cluster(&bars.full[stage], (kk / kStages) & 1);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t sa = smem_u32(stages + stage * kPairStageBytes);
+                const uint64_t da = make_smem_desc(sa), db = make_smem_desc(sa + kPairRows * kBK * 2);
+#pragma unroll
+                for (int k = 0; k < kBK / 16; ++k)
+                    umma2_bf16(tmem_base, da + (uint64_t)(2 * k), db + (uint64_t)(2 * k), kPairInstrDesc, (kk | k) != 0);
+                umma_commit2(&bars.empty[stage]);  // both CTAs may refill the stage once these MMAs have read it
+            }
+            if (ok) umma_commit2(&bars.accum);     // accumulators complete in both CTAs
+            else bars.failed = 1;
+        }
+        __syncwarp();
+        tc_fence_before();
+    }
+    __syncthreads();
+    cluster_sync_all();  // the peer may still be reading this CTA's shared memory / signalling its barriers
+    if (warp == kMmaWarp) {
+        tc_fence_after();
+        tmem_dealloc2(tmem_base, 256);
+    }
+    if (threadIdx.x == 0 && bars.failed) atomicExch(&g_gemm_status, (int)BDR_ERR_TIMEOUT);
+}
+
+// cuTensorMapEncodeTiled through the runtime's driver entry point (the library does not link libcuda)
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+static EncodeTiledFn encode_tiled_fn() {
+    static EncodeTiledFn fn = nullptr;
+    static bool tried = false;
+    if (!tried) {
+        tried = true;
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess && q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+// plane viewed as a [rows, row_bytes] byte matrix with pitch `ld`; box = 128 rows x box_bytes
+static bool make_plane_map(CUtensorMap* out, const uint8_t* base, int64_t rows, int64_t row_bytes, int64_t ld, int box_bytes) {
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[2] = {(cuuint64_t)row_bytes, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)ld};
+    const cuuint32_t box[2] = {(cuuint32_t)box_bytes, (cuuint32_t)kPairRows};
+    const cuuint32_t estr[2] = {1, 1};
+    return fn(out, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<uint8_t*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+              CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <int WA, int WB>
+int launch_gemm_pair(const bdr_planes_t& a, const bdr_planes_t& b, int64_t M, int64_t N, int64_t K, float* c, int64_t ldc,
+                     cudaStream_t st) {
+    auto kern = mx_gemm_pair_kernel<WA, WB>;
+    const size_t smem = PairSmem<WA, WB>::kBytes;
+    static bool attr_done = false;
+    if (!attr_done) {
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return BDR_ERR_CUDA;
+        attr_done = true;
+    }
+    PairMaps maps;
+    const bool ok = make_plane_map(&maps.a_elems, a.elems, M, K * WA / 8, a.ld_elems, ChunkPlanes<WA>::kElemRow) &&
+                    make_plane_map(&maps.a_exps, a.exps, M, K / 16, a.ld_exps, 16) &&
+                    make_plane_map(&maps.a_micro, a.micro, M, K / 16, a.ld_micro, 16) &&
+                    make_plane_map(&maps.b_elems, b.elems, N, K * WB / 8, b.ld_elems, ChunkPlanes<WB>::kElemRow) &&
+                    make_plane_map(&maps.b_exps, b.exps, N, K / 16, b.ld_exps, 16) &&
+                    make_plane_map(&maps.b_micro, b.micro, N, K / 16, b.ld_micro, 16);
+    if (!ok) return BDR_ERR_UNSUPPORTED;  // caller falls back to the single-CTA kernel
+    const dim3 grid((unsigned)(M / 128), (unsigned)(N / 256));  // x: CTAs (two per 256-row pair), y: column tiles
+    kern<<<grid, kPairThreads, smem, st>>>(maps, M, N, K, c, ldc);
+    return cudaGetLastError() == cudaSuccess ? BDR_OK : BDR_ERR_CUDA;
+}
+
+}  // namespace bdr

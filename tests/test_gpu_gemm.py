@@ -68,6 +68,17 @@ def test_random_operands_match_the_oracle(fa, fb):
     assert err <= 1e-5, err                              # what exact decoding should deliver
 
 
+@pytest.mark.parametrize("fa,fb", [("MX6", "MX6"), ("MX9", "MX4"), ("MX4", "MX6"), ("MX9", "MX9")])
+def test_two_cta_kernel_shapes(fa, fb):
+    # M a multiple of 256 and K a multiple of 256 select the 2-CTA (cta_group::2) kernel
+    M, N, K = 512, 768, 1024
+    a = synth.normal_matrix(M, K, seed=6, stream=1)
+    b = synth.outlier_channel_matrix(N, K, seed=6, stream=2, gain=20.0, dist="normal", sigma=0.02)
+    c = gpu_gemm(FMT[fa], a, FMT[fb], b)
+    ref = oracle_gemm(FMT[fa], a, FMT[fb], b)
+    assert rel_frob(c, ref) <= 1e-5
+
+
 def test_outlier_channels_and_extreme_scales():
     M, N, K = 128, 256, 512
     a = synth.outlier_channel_matrix(M, K, seed=2, gain=50.0)
