@@ -116,6 +116,16 @@ __device__ __forceinline__ uint32_t bf16_pow2(int e) {
     return e >= 1 ? (uint32_t)e << 7 : (e >= -6 ? 1u << (6 + e) : 0u);
 }
 
+__device__ __forceinline__ uint2 ld_shared_v2(uint32_t addr) {
+    uint2 v;
+    asm volatile("ld.shared.v2.b32 {%0, %1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(addr) : "memory");
+    return v;
+}
+__device__ __forceinline__ uint32_t ld_shared_b32(uint32_t addr) {
+    uint32_t v;
+    asm volatile("ld.shared.b32 %0, [%1];" : "=r"(v) : "r"(addr) : "memory");
+    return v;
+}
 __device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
     asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
 }
@@ -136,21 +146,24 @@ __device__ __forceinline__ uint32_t bf16x2_mul(uint32_t a, uint32_t b) {
 // q < 128); one packed fused multiply-add with the sub-block's power-of-two scale s and the
 // constant -128 s then gives q * s exactly (the exact result is representable, so the single
 // rounding changes nothing).  The sign bit is ORed in last.
-template <int W, int NWORDS>
+template <int W, int NWORDS, bool SAFE>
 __device__ __forceinline__ void decode_block_bf16(const uint32_t (&w)[NWORDS], int bit0, uint32_t F, uint32_t micro, uint32_t (&out)[8]) {
     constexpr int M = W - 1;
     constexpr uint32_t kQ2 = ((1u << M) - 1u) * 0x00010001u;
-    // scale of one unit of q: 2^(F-127-tau-(m-1)); the constant term -128 * scale needs exponent + 7
+    // scale of one unit of q: 2^(F-127-tau-(m-1)); the constant term -128 * scale needs exponent + 7.
+    // SAFE (decided by the caller for the whole warp): 2 <= e0 <= 247, so both scales and both
+    // constants are normal bf16 numbers and one fused multiply-add per pair does the job.
     const int e0 = (int)F - (M - 1);
-    uint32_t s0 = bf16_pow2(e0) * 0x00010001u, s1 = bf16_pow2(e0 - 1) * 0x00010001u;
-    uint32_t n0, n1;
-    const bool safe = e0 >= 2 && e0 <= 247;  // both scales and both constants are normal bf16 numbers
-    if (safe) {
+    uint32_t s0, s1, n0 = 0, n1 = 0;
+    if (SAFE) {
+        s0 = ((uint32_t)e0 << 7) * 0x00010001u;
+        s1 = s0 - 0x00800080u;
         n0 = (s0 + 0x03800380u) | 0x80008000u;  // -(2^7 * s0)
-        n1 = (s1 + 0x03800380u) | 0x80008000u;
+        n1 = n0 - 0x00800080u;
     } else {
+        s0 = bf16_pow2(e0) * 0x00010001u;
+        s1 = bf16_pow2(e0 - 1) * 0x00010001u;
         if (F == 255) { s0 = 0x7FC07FC0u; s1 = s0; }  // Inf/NaN block -> NaN
-        n0 = 0; n1 = 0;
     }
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
@@ -163,13 +176,23 @@ __device__ __forceinline__ void decode_block_bf16(const uint32_t (&w)[NWORDS], i
         const uint32_t mag = (u & kQ2) | 0x43004300u;
         const bool t1 = (micro >> j) & 1u;
         uint32_t v;
-        if (safe) {
-            v = bf16x2_fma(mag, t1 ? s1 : s0, t1 ? n1 : n0);
-        } else {  // tiny / huge / NaN exponents: subtract first, then scale (both exact)
-            v = bf16x2_mul(bf16x2_fma(mag, 0x3F803F80u, 0xC300C300u), t1 ? s1 : s0);
-        }
+        if (SAFE) v = bf16x2_fma(mag, t1 ? s1 : s0, t1 ? n1 : n0);
+        else v = bf16x2_mul(bf16x2_fma(mag, 0x3F803F80u, 0xC300C300u), t1 ? s1 : s0);  // subtract 128, then scale: both exact
         out[j] = v | ((u << (15 - M)) & 0x80008000u);
     }
+}
+
+// true when every block exponent in the word (4 bytes, one per block) allows the SAFE decoder
+template <int W>
+__device__ __forceinline__ bool exps_safe(uint32_t exps4) {
+    constexpr int M = W - 1;
+    bool ok = true;
+#pragma unroll
+    for (int b = 0; b < 4; ++b) {
+        const int e0 = (int)((exps4 >> (8 * b)) & 0xFFu) - (M - 1);
+        ok = ok && e0 >= 2 && e0 <= 247;
+    }
+    return ok;
 }
 
 struct GemmSmem {
@@ -227,10 +250,12 @@ __device__ __forceinline__ bool decode_rows(const bdr_planes_t& pl, int64_t grow
             if (!ok) return false;
         }
         const uint32_t tile = tiles_addr + stage * kStageBytes + tile_off;
+        const bool safe = __all_sync(0xFFFFFFFFu, exps_safe<W>(exps4));  // warp-uniform choice of decoder
 #pragma unroll
         for (int bb = 0; bb < kBK / kSlice; ++bb) {
             uint32_t o[8];
-            decode_block_bf16<W, NW>(w, bb * kSlice * W, (exps4 >> (8 * bb)) & 0xFFu, (micro4 >> (8 * bb)) & 0xFFu, o);
+            if (safe) decode_block_bf16<W, NW, true>(w, bb * kSlice * W, (exps4 >> (8 * bb)) & 0xFFu, (micro4 >> (8 * bb)) & 0xFFu, o);
+            else decode_block_bf16<W, NW, false>(w, bb * kSlice * W, (exps4 >> (8 * bb)) & 0xFFu, (micro4 >> (8 * bb)) & 0xFFu, o);
             st_shared_v4(tile + (((2 * bb) ^ (r & 7)) << 4), o[0], o[1], o[2], o[3]);
             st_shared_v4(tile + (((2 * bb + 1) ^ (r & 7)) << 4), o[4], o[5], o[6], o[7]);
         }

@@ -20,9 +20,9 @@ namespace bdr {
 constexpr int kPairRows = 128;                  // rows of A and of the B half per CTA
 constexpr int kChunkK = 256;                    // K elements per bulk-copy chunk (4 K steps)
 constexpr int kStepsPerChunk = kChunkK / kBK;   // 4
-constexpr int kPairDecodeWarps = 8;
-constexpr int kLoaderWarp = 8, kMmaWarp = 9;
-constexpr int kPairThreads = 10 * 32;
+constexpr int kPairDecodeWarps = 16;            // two threads per row: each decodes two of the row's four blocks per K step
+constexpr int kLoaderWarp = 16, kMmaWarp = 17;
+constexpr int kPairThreads = 18 * 32;
 constexpr int kPairStageBytes = 2 * kPairRows * kBK * 2;  // A 16 KB + B half 16 KB
 
 // Packed bytes of one chunk (256 K elements) for 128 rows, as the TMA writes them: dense row-major
@@ -65,7 +65,7 @@ __device__ __forceinline__ void cluster_sync_all() {
 __device__ __forceinline__ void mbar_arrive_cluster(uint64_t* bar, uint32_t rank) {
     uint32_t remote;
     asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(smem_u32(bar)), "r"(rank));
-    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(remote) : "memory");
+    asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(remote) : "memory");
 }
 __device__ __forceinline__ bool mbar_wait_cluster(uint64_t* bar, uint32_t parity) {
     const uint32_t addr = smem_u32(bar);
@@ -73,7 +73,7 @@ __device__ __forceinline__ bool mbar_wait_cluster(uint64_t* bar, uint32_t parity
         uint32_t done;
         asm volatile(
             "{\n\t.reg .pred p;\n\t"
-            "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
             "selp.u32 %0, 1, 0, p;\n\t}"
             : "=r"(done)
             : "r"(addr), "r"(parity)
@@ -116,11 +116,13 @@ __device__ __forceinline__ void umma2_bf16(uint32_t tmem_d, uint64_t desc_a, uin
 // D = fp32, A = B = bf16, both K-major, N = 256, M = 256 (128 rows per CTA)
 constexpr uint32_t kPairInstrDesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(256 >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
 
-// pk0 / pk1: this operand's ChunkPlanes in the two packed buffers
+// pk0 / pk1: shared-memory addresses of this operand's ChunkPlanes in the two packed buffers.
+// `half` selects which two of the row's four 16-element blocks of a K step this thread decodes.
 template <int W>
-__device__ __forceinline__ bool pair_decode_rows(const uint8_t* pk0, const uint8_t* pk1, int r, uint32_t tile_off,
+__device__ __forceinline__ bool pair_decode_rows(uint32_t pk0, uint32_t pk1, int r, int half, uint32_t tile_off,
                                                  uint32_t stages_addr, int n_stages, PairBars& bars, int nk, int lane) {
-    constexpr int NW = kBK * W / 32;  // code words per K step
+    constexpr int NW = 2 * kSlice * W / 32;  // code words of two blocks: 3 / 5 / 8
+    constexpr int NLD = (NW + 1) / 2;        // 8-byte loads that cover them (the run starts 4-byte aligned)
     for (int kk = 0; kk < nk; ++kk) {
         const int chunk = kk / kStepsPerChunk, ks = kk % kStepsPerChunk, buf = chunk & 1;
         if (ks == 0) {
@@ -128,13 +130,20 @@ __device__ __forceinline__ bool pair_decode_rows(const uint8_t* pk0, const uint8
             ok = __all_sync(0xFFFFFFFFu, ok);
             if (!ok) return false;
         }
-        const uint8_t* pk = buf ? pk1 : pk0;
-        uint32_t w[NW];
-        const uint2* src = reinterpret_cast<const uint2*>(pk + ChunkPlanes<W>::kElems + r * ChunkPlanes<W>::kElemRow + ks * (kBK * W / 8));
+        const uint32_t pk = buf ? pk1 : pk0;
+        // the two blocks' codes: 4W bytes starting at byte ks*8W + half*4W of the row (4-byte aligned)
+        const uint32_t ebase = pk + ChunkPlanes<W>::kElems + r * ChunkPlanes<W>::kElemRow + ks * (kBK * W / 8) + half * (4 * W);
+        uint32_t w[NW + 1];
+        if ((4 * W) % 8 == 0) {
 #pragma unroll
-        for (int i = 0; i < NW / 2; ++i) { const uint2 v = src[i]; w[2 * i] = v.x; w[2 * i + 1] = v.y; }
-        const uint32_t exps4 = *reinterpret_cast<const uint32_t*>(pk + ChunkPlanes<W>::kExps + r * 16 + 4 * ks);
-        const uint32_t micro4 = *reinterpret_cast<const uint32_t*>(pk + ChunkPlanes<W>::kMicro + r * 16 + 4 * ks);
+            for (int i = 0; i < NW / 2; ++i) { const uint2 v = ld_shared_v2(ebase + 8 * i); w[2 * i] = v.x; w[2 * i + 1] = v.y; }
+        } else {
+#pragma unroll
+            for (int i = 0; i < NW; ++i) w[i] = ld_shared_b32(ebase + 4 * i);
+        }
+        w[NW] = 0;
+        const uint32_t exps2 = (ld_shared_b32(pk + ChunkPlanes<W>::kExps + r * 16 + 4 * ks) >> (16 * half)) & 0xFFFFu;
+        const uint32_t micro2 = (ld_shared_b32(pk + ChunkPlanes<W>::kMicro + r * 16 + 4 * ks) >> (16 * half)) & 0xFFFFu;
         const int stage = kk % n_stages;
         if (kk >= n_stages) {
             bool ok = mbar_wait(&bars.empty[stage], ((kk / n_stages) - 1) & 1);
@@ -142,12 +151,17 @@ __device__ __forceinline__ bool pair_decode_rows(const uint8_t* pk0, const uint8
             if (!ok) return false;
         }
         const uint32_t tile = stages_addr + stage * kPairStageBytes + tile_off;
+        constexpr int M = W - 1;
+        const int ea = (int)(exps2 & 0xFFu) - (M - 1), eb = (int)(exps2 >> 8) - (M - 1);
+        const bool safe = __all_sync(0xFFFFFFFFu, ea >= 2 && ea <= 247 && eb >= 2 && eb <= 247);  // warp-uniform decoder choice
 #pragma unroll
-        for (int bb = 0; bb < kBK / kSlice; ++bb) {
+        for (int bb = 0; bb < 2; ++bb) {
             uint32_t o[8];
-            decode_block_bf16<W, NW>(w, bb * kSlice * W, (exps4 >> (8 * bb)) & 0xFFu, (micro4 >> (8 * bb)) & 0xFFu, o);
-            st_shared_v4(tile + (((2 * bb) ^ (r & 7)) << 4), o[0], o[1], o[2], o[3]);
-            st_shared_v4(tile + (((2 * bb + 1) ^ (r & 7)) << 4), o[4], o[5], o[6], o[7]);
+            if (safe) decode_block_bf16<W, NW + 1, true>(w, bb * kSlice * W, (exps2 >> (8 * bb)) & 0xFFu, (micro2 >> (8 * bb)) & 0xFFu, o);
+            else decode_block_bf16<W, NW + 1, false>(w, bb * kSlice * W, (exps2 >> (8 * bb)) & 0xFFu, (micro2 >> (8 * bb)) & 0xFFu, o);
+            const int chunk16 = 2 * (2 * half + bb);  // 16-byte chunk of the block's first 8 elements within the 128-byte row
+            st_shared_v4(tile + ((chunk16 ^ (r & 7)) << 4), o[0], o[1], o[2], o[3]);
+            st_shared_v4(tile + (((chunk16 + 1) ^ (r & 7)) << 4), o[4], o[5], o[6], o[7]);
         }
         fence_proxy_async();  // generic-proxy stores -> visible to the tensor core's (async proxy) reads
         __syncwarp();
@@ -190,14 +204,16 @@ mx_gemm_pair_kernel(const __grid_constant__ PairMaps maps, int64_t M, int64_t N,
     const uint32_t tmem_base = bars.tmem_base;
 
     if (warp < kPairDecodeWarps) {
-        // ---------------- decoders: thread t owns row t (A rows 0-127, then the B half's 128 rows) ----------------
-        const bool is_a = warp < kPairRows / 32;
-        const int r = is_a ? (int)threadIdx.x : (int)threadIdx.x - kPairRows;
+        // ---------------- decoders: threads t and t+256 share row t (A rows 0-127, then the B half's 128 rows) ----------------
+        const int half = warp >> 3;                 // warps 0-7: blocks 0,1 of each K step; warps 8-15: blocks 2,3
+        const int row256 = (int)threadIdx.x & 255;  // consecutive lanes hold consecutive rows (conflict-free swizzled stores)
+        const bool is_a = row256 < kPairRows;
+        const int r = is_a ? row256 : row256 - kPairRows;
         const uint32_t tile_off = (uint32_t)((is_a ? 0 : kPairRows * kBK * 2) + (r >> 3) * 1024 + (r & 7) * 128);
         bool ok;
-        if (is_a) ok = pair_decode_rows<WA>(pk[0], pk[1], r, tile_off, smem_u32(stages), kStages, bars, nk, lane);
-        else ok = pair_decode_rows<WB>(pk[0] + ChunkPlanes<WA>::kBytes, pk[1] + ChunkPlanes<WA>::kBytes, r, tile_off,
-                                       smem_u32(stages), kStages, bars, nk, lane);
+        if (is_a) ok = pair_decode_rows<WA>(smem_u32(pk[0]), smem_u32(pk[1]), r, half, tile_off, smem_u32(stages), kStages, bars, nk, lane);
+        else ok = pair_decode_rows<WB>(smem_u32(pk[0]) + ChunkPlanes<WA>::kBytes, smem_u32(pk[1]) + ChunkPlanes<WA>::kBytes, r, half,
+                                       tile_off, smem_u32(stages), kStages, bars, nk, lane);
         if (!ok) bars.failed = 1;
 
         // ---------------- epilogue: this CTA's 128 x 256 block of C ----------------
@@ -205,10 +221,10 @@ mx_gemm_pair_kernel(const __grid_constant__ PairMaps maps, int64_t M, int64_t N,
         done = __all_sync(0xFFFFFFFFu, done);
         if (done) {
             tc_fence_after();
-            const int lane_base = (warp & 3) * 32, col_base = (warp >> 2) * 128;
+            const int lane_base = (warp & 3) * 32, col_base = (warp >> 2) * 64;  // 16 warps: 4 lane groups x 4 column quarters
             float* crow = c + (m0 + lane_base + lane) * ldc + n0 + col_base;
 #pragma unroll 1
-            for (int cc = 0; cc < 128; cc += 32) {
+            for (int cc = 0; cc < 64; cc += 32) {
                 uint32_t v[32];
                 tmem_ld32(tmem_base + ((uint32_t)lane_base << 16) + (uint32_t)(col_base + cc), v);
 #pragma unroll
