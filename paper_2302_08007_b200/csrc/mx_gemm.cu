@@ -30,7 +30,8 @@ constexpr int kGemmThreads = (kDecodeWarps + 1) * 32;
 constexpr int kABytes = kBM * kBK * 2;  // 16 KB
 constexpr int kBBytes = kBN * kBK * 2;  // 32 KB
 constexpr int kStageBytes = kABytes + kBBytes;
-constexpr uint32_t kSpinLimit = 1u << 20;  // bounded waits (each try_wait itself blocks for a while)
+constexpr uint32_t kSpinLimit = 1u << 18;     // bounded waits: this many polls ...
+constexpr uint32_t kSuspendHintNs = 2000;     // ... each of which may sleep about this long in hardware
 
 __device__ int g_gemm_status = 0;  // sticky: first failing launch leaves BDR_ERR_TIMEOUT here
 
@@ -49,10 +50,10 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
         uint32_t done;
         asm volatile(
             "{\n\t.reg .pred p;\n\t"
-            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
             "selp.u32 %0, 1, 0, p;\n\t}"
             : "=r"(done)
-            : "r"(addr), "r"(parity)
+            : "r"(addr), "r"(parity), "r"(kSuspendHintNs)
             : "memory");
         if (done) return true;
     }

@@ -34,12 +34,15 @@ template <int W> struct ChunkPlanes {
     static constexpr int kMicro = kExps + kPairRows * 16;
     static constexpr int kBytes = kMicro + kPairRows * 16;  // a multiple of 128
 };
+constexpr int kMaxPk = 3;  // packed-chunk buffers (TMA runs up to kPk-1 chunks ahead of the decoders)
 template <int WA, int WB> struct PairSmem {
     static constexpr int kPackedBytes = ChunkPlanes<WA>::kBytes + ChunkPlanes<WB>::kBytes;  // one buffer
-    static constexpr int kBudget = 224 * 1024 - 2 * kPackedBytes - 1024;
+    // three packed buffers when two operand stages still fit beside them, else two
+    static constexpr int kPk = (224 * 1024 - 3 * kPackedBytes - 1024) / kPairStageBytes >= 2 ? 3 : 2;
+    static constexpr int kBudget = 224 * 1024 - kPk * kPackedBytes - 1024;
     static constexpr int kStages = kBudget / kPairStageBytes >= 4 ? 4 : kBudget / kPairStageBytes;
     static_assert(kStages >= 2, "operand stages do not fit");
-    static constexpr size_t kBytes = (size_t)kStages * kPairStageBytes + 2 * kPackedBytes + 1024 /*bookkeeping*/ + 1024 /*alignment*/;
+    static constexpr size_t kBytes = (size_t)kStages * kPairStageBytes + kPk * kPackedBytes + 1024 /*bookkeeping*/ + 1024 /*alignment*/;
 };
 
 struct PairMaps {  // tensor maps of the three planes of A and of B (uint8 elements, rows x row bytes)
@@ -47,7 +50,7 @@ struct PairMaps {  // tensor maps of the three planes of A and of B (uint8 eleme
 };
 
 struct PairBars {
-    uint64_t full[4], empty[4], accum, pk_full[2], pk_empty[2];
+    uint64_t full[4], empty[4], accum, pk_full[kMaxPk], pk_empty[kMaxPk];
     uint32_t tmem_base;
     int failed;
 };
@@ -73,10 +76,10 @@ __device__ __forceinline__ bool mbar_wait_cluster(uint64_t* bar, uint32_t parity
         uint32_t done;
         asm volatile(
             "{\n\t.reg .pred p;\n\t"
-            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
             "selp.u32 %0, 1, 0, p;\n\t}"
             : "=r"(done)
-            : "r"(addr), "r"(parity)
+            : "r"(addr), "r"(parity), "r"(kSuspendHintNs)
             : "memory");
         if (done) return true;
     }
@@ -119,18 +122,18 @@ constexpr uint32_t kPairInstrDesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint3
 // pk0 / pk1: shared-memory addresses of this operand's ChunkPlanes in the two packed buffers.
 // `half` selects which two of the row's four 16-element blocks of a K step this thread decodes.
 template <int W>
-__device__ __forceinline__ bool pair_decode_rows(uint32_t pk0, uint32_t pk1, int r, int half, uint32_t tile_off,
+__device__ __forceinline__ bool pair_decode_rows(uint32_t pk0, uint32_t pk_stride, int n_pk, int r, int half, uint32_t tile_off,
                                                  uint32_t stages_addr, int n_stages, PairBars& bars, int nk, int lane) {
     constexpr int NW = 2 * kSlice * W / 32;  // code words of two blocks: 3 / 5 / 8
     constexpr int NLD = (NW + 1) / 2;        // 8-byte loads that cover them (the run starts 4-byte aligned)
     for (int kk = 0; kk < nk; ++kk) {
-        const int chunk = kk / kStepsPerChunk, ks = kk % kStepsPerChunk, buf = chunk & 1;
+        const int chunk = kk / kStepsPerChunk, ks = kk % kStepsPerChunk, buf = chunk % n_pk;
         if (ks == 0) {
-            bool ok = mbar_wait(&bars.pk_full[buf], (chunk >> 1) & 1);
+            bool ok = mbar_wait(&bars.pk_full[buf], (chunk / n_pk) & 1);
             ok = __all_sync(0xFFFFFFFFu, ok);
             if (!ok) return false;
         }
-        const uint32_t pk = buf ? pk1 : pk0;
+        const uint32_t pk = pk0 + buf * pk_stride;
         // the two blocks' codes: 4W bytes starting at byte ks*8W + half*4W of the row (4-byte aligned)
         const uint32_t ebase = pk + ChunkPlanes<W>::kElems + r * ChunkPlanes<W>::kElemRow + ks * (kBK * W / 8) + half * (4 * W);
         uint32_t w[NW + 1];
@@ -180,8 +183,9 @@ mx_gemm_pair_kernel(const __grid_constant__ PairMaps maps, int64_t M, int64_t N,
     constexpr int kStages = SM::kStages;
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     uint8_t* stages = reinterpret_cast<uint8_t*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-    uint8_t* pk[2] = {stages + kStages * kPairStageBytes, stages + kStages * kPairStageBytes + SM::kPackedBytes};
-    PairBars& bars = *reinterpret_cast<PairBars*>(stages + kStages * kPairStageBytes + 2 * SM::kPackedBytes);
+    constexpr int kPk = SM::kPk;
+    uint8_t* pk_base = stages + kStages * kPairStageBytes;  // kPk packed buffers of SM::kPackedBytes each
+    PairBars& bars = *reinterpret_cast<PairBars*>(pk_base + kPk * SM::kPackedBytes);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = cluster_ctarank();
     const int64_t m0 = ((int64_t)(blockIdx.x >> 1) * 2 + rank) * kPairRows;  // this CTA's rows of A and C
@@ -192,7 +196,7 @@ mx_gemm_pair_kernel(const __grid_constant__ PairMaps maps, int64_t M, int64_t N,
     if (threadIdx.x == 0) {
         for (int s = 0; s < 4; ++s) { mbar_init(&bars.full[s], 2 * kPairDecodeWarps); mbar_init(&bars.empty[s], 1); }
         mbar_init(&bars.accum, 1);
-        for (int i = 0; i < 2; ++i) { mbar_init(&bars.pk_full[i], 1); mbar_init(&bars.pk_empty[i], kPairDecodeWarps); }
+        for (int i = 0; i < kMaxPk; ++i) { mbar_init(&bars.pk_full[i], 1); mbar_init(&bars.pk_empty[i], kPairDecodeWarps); }
         bars.failed = 0;
         fence_barrier_init();
     }
@@ -211,9 +215,9 @@ mx_gemm_pair_kernel(const __grid_constant__ PairMaps maps, int64_t M, int64_t N,
         const int r = is_a ? row256 : row256 - kPairRows;
         const uint32_t tile_off = (uint32_t)((is_a ? 0 : kPairRows * kBK * 2) + (r >> 3) * 1024 + (r & 7) * 128);
         bool ok;
-        if (is_a) ok = pair_decode_rows<WA>(smem_u32(pk[0]), smem_u32(pk[1]), r, half, tile_off, smem_u32(stages), kStages, bars, nk, lane);
-        else ok = pair_decode_rows<WB>(smem_u32(pk[0]) + ChunkPlanes<WA>::kBytes, smem_u32(pk[1]) + ChunkPlanes<WA>::kBytes, r, half,
-                                       tile_off, smem_u32(stages), kStages, bars, nk, lane);
+        if (is_a) ok = pair_decode_rows<WA>(smem_u32(pk_base), SM::kPackedBytes, kPk, r, half, tile_off, smem_u32(stages), kStages, bars, nk, lane);
+        else ok = pair_decode_rows<WB>(smem_u32(pk_base) + ChunkPlanes<WA>::kBytes, SM::kPackedBytes, kPk, r, half, tile_off,
+                                       smem_u32(stages), kStages, bars, nk, lane);
         if (!ok) bars.failed = 1;
 
         // ---------------- epilogue: this CTA's 128 x 256 block of C ----------------
@@ -240,13 +244,13 @@ mx_gemm_pair_kernel(const __grid_constant__ PairMaps maps, int64_t M, int64_t N,
         if (lane == 0) {
             bool ok = true;
             for (int ch = 0; ch < nchunks; ++ch) {
-                const int buf = ch & 1;
-                if (ch >= 2) {
-                    ok = mbar_wait(&bars.pk_empty[buf], ((ch >> 1) - 1) & 1);
+                const int buf = ch % kPk;
+                if (ch >= kPk) {
+                    ok = mbar_wait(&bars.pk_empty[buf], ((ch / kPk) - 1) & 1);
                     if (!ok) break;
                 }
-                uint8_t* pa = pk[buf];
-                uint8_t* pb = pk[buf] + ChunkPlanes<WA>::kBytes;
+                uint8_t* pa = pk_base + (size_t)buf * SM::kPackedBytes;
+                uint8_t* pb = pa + ChunkPlanes<WA>::kBytes;
                 mbar_expect_tx(&bars.pk_full[buf], (uint32_t)SM::kPackedBytes);
                 tma_load_2d(pa + ChunkPlanes<WA>::kElems, &maps.a_elems, ch * ChunkPlanes<WA>::kElemRow, (int)m0, &bars.pk_full[buf]);
                 tma_load_2d(pa + ChunkPlanes<WA>::kExps, &maps.a_exps, ch * 16, (int)m0, &bars.pk_full[buf]);
