@@ -61,6 +61,22 @@ def measured_peaks():
         return FALLBACK_HBM_GBS, "fallback", {}
 
 
+def max_over_ranks(ms: float, world: int, device="cuda") -> float:
+    """The job's time is the slowest rank's time (all-reduce MAX); identity for one rank."""
+    if world <= 1:
+        return float(ms)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def aggregate_value(bytes_per_rank: float, world: int, ms_per_step: float) -> float:
+    """Whole-job GB/s of `world` independent replicas that each move bytes_per_rank per step."""
+    return bytes_per_rank * world / (ms_per_step * 1e-3) / 1e9
+
+
 class ClockSampler:
     """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
     QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
@@ -248,12 +264,9 @@ def run_ours(args):
     barrier()
     ms = ev0.elapsed_time(ev1)
     clocks = sampler.stop() if rank == 0 else {}
-    if world > 1:
-        t = torch.tensor([ms], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
+    ms = max_over_ranks(ms, world)
     ms_per_step = ms / args.steps
-    value = step_bytes(n_elems) * world / (ms_per_step * 1e-3) / 1e9
+    value = aggregate_value(step_bytes(n_elems), world, ms_per_step)
     qsnr = {}
     sums_np = (sums / args.steps).cpu().numpy()
     for i, (name, _m, axis, op) in enumerate(ops):
@@ -295,11 +308,8 @@ def run_ours(args):
     e1.record()
     barrier()
     e2e_ms = e0.elapsed_time(e1)
-    if world > 1:
-        t = torch.tensor([e2e_ms], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t.item())
-    e2e = {"value": step_bytes(n_elems) * world / (e2e_ms / e2e_steps * 1e-3) / 1e9, "unit": "GB/s",
+    e2e_ms = max_over_ranks(e2e_ms, world)
+    e2e = {"value": aggregate_value(step_bytes(n_elems), world, e2e_ms / e2e_steps), "unit": "GB/s",
            "h2d_bytes_per_step": x.numel() * x.element_size(), "d2h_bytes_per_step": sums.numel() * 8,
            "steps": e2e_steps}
 

@@ -149,15 +149,12 @@ quant_colwise_mx_kernel(const T* x, T* y, int64_t rows, int64_t cols, int64_t ld
             *reinterpret_cast<uint4*>(out.exps + (c0 + ci) * out.ld_exps + tb0 + v * 16) =
                 make_uint4(w4[0], w4[1], w4[2], w4[3]);
         }
-        for (int idx = threadIdx.x; idx < kTileCols * 2 * qp.d2; idx += kColThreads) {
+        for (int idx = threadIdx.x; idx < kTileCols * 2; idx += kColThreads) {  // d2 = 1
             const int ci = idx % kTileCols, v = idx / kTileCols;
             uint32_t w4[4] = {0, 0, 0, 0};
 #pragma unroll
-            for (int i = 0; i < 16; ++i) {
-                const int t = 16 * v + i;
-                w4[i >> 2] |= (uint32_t)st.micro[t / qp.d2][ci][t % qp.d2] << ((i & 3) * 8);
-            }
-            *reinterpret_cast<uint4*>(out.micro + (c0 + ci) * out.ld_micro + tb0 * qp.d2 + v * 16) =
+            for (int i = 0; i < 16; ++i) w4[i >> 2] |= (uint32_t)st.micro[16 * v + i][ci][0] << ((i & 3) * 8);
+            *reinterpret_cast<uint4*>(out.micro + (c0 + ci) * out.ld_micro + tb0 + v * 16) =
                 make_uint4(w4[0], w4[1], w4[2], w4[3]);
         }
     }
@@ -190,14 +187,14 @@ unpack_colwise_mx_kernel(bdr_planes_t in, T* y, int64_t rows, int64_t cols, int6
 #pragma unroll
         for (int i = 0; i < 16; ++i) st.exps[16 * v + i][ci] = (uint8_t)(w4[i >> 2] >> ((i & 3) * 8));
     }
-    for (int idx = threadIdx.x; idx < kTileCols * 2 * qp.d2; idx += kColThreads) {
-        const int v = idx % (2 * qp.d2), ci = idx / (2 * qp.d2);
-        const uint4 q4 = __ldg(reinterpret_cast<const uint4*>(in.micro + (c0 + ci) * in.ld_micro + tb0 * qp.d2 + v * 16));
+    for (int idx = threadIdx.x; idx < kTileCols * 2; idx += kColThreads) {
+        const int v = idx % 2, ci = idx / 2;
+        const uint4 q4 = __ldg(reinterpret_cast<const uint4*>(in.micro + (c0 + ci) * in.ld_micro + tb0 + v * 16));
         const uint32_t w4[4] = {q4.x, q4.y, q4.z, q4.w};
 #pragma unroll
         for (int i = 0; i < 16; ++i) {
             const int t = 16 * v + i;
-            st.micro[t / qp.d2][ci][t % qp.d2] = (uint8_t)(w4[i >> 2] >> ((i & 3) * 8));
+            st.micro[t][ci][0] = (uint8_t)(w4[i >> 2] >> ((i & 3) * 8));
         }
     }
     __syncthreads();
@@ -212,9 +209,8 @@ unpack_colwise_mx_kernel(bdr_planes_t in, T* y, int64_t rows, int64_t cols, int6
             for (int i = 0; i < (kSlice * W + 31) / 32 + 1; ++i) words[i] = 0;
 #pragma unroll
             for (int k = 0; k < W; ++k) words[k >> 1] |= (uint32_t)st.elems[bl][2 * lane + h][k] << ((k & 1) * 16);
-            uint32_t mbits = 0;
-            for (int k = 0; k < qp.d2; ++k) mbits |= (uint32_t)st.micro[bl][2 * lane + h][k] << (8 * k);
-            decode_slice<W>(words, st.exps[bl][2 * lane + h], mbits, qp, yb[h]);
+            const uint32_t mbits = st.micro[bl][2 * lane + h][0];
+            decode_slice<W>(words, st.exps[bl][2 * lane + h], mbits, yb[h]);
         }
         T* py = y + b * kSlice * ld + c;
 #pragma unroll

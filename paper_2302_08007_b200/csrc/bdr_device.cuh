@@ -407,31 +407,51 @@ __device__ __forceinline__ void pack_words(const uint32_t (&u)[N], const uint32_
     for (int w = 0; w < NW; ++w) words[w] = accq[w] | accs[w];
 }
 
-// Decode one slice (k2 = 2): codes are W-bit fields of the little-endian stream in `words`.
+// Decode one slice of the Table II family (k2 = 2, d2 = 1): codes are W-bit fields of the
+// little-endian stream in `words`, `mbits` holds the eight sub-block shifts (one bit each).
 // value = q * 2^p with p = F-127-tau-(m-1): the float 2^23 + q is built by ORing q into its
-// mantissa, and fma(2^23 + q, 2^p, -2^(p+23)) is then exactly q * 2^p (valid while 2^(p+23) is finite).
-template <int W>
-__device__ __forceinline__ void decode_slice(const uint32_t (&words)[(kSlice * W + 31) / 32 + 1], int F, uint32_t mbits,
-                                             const QParams& qp, uint32_t (&yb)[kSlice]) {
+// mantissa, and fma(2^23 + q, 2^p, -2^(p+23)) is then exactly q * 2^p.  FAST requires every scale
+// and constant to be a normal fp32 number (the caller checks 16 <= F <= 230 for the whole warp);
+// otherwise the magnitude is converted and scaled in two exact steps, which also covers subnormal
+// results and NaN blocks.
+template <int W, bool FAST>
+__device__ __forceinline__ void decode_slice_impl(const uint32_t (&words)[(kSlice * W + 31) / 32 + 1], int F, uint32_t mbits,
+                                                  uint32_t (&yb)[kSlice]) {
     constexpr int M = W - 1;
     constexpr uint32_t kQMask = (1u << M) - 1u;
-    const bool fma_ok = F <= kFastMaxF;
+    // tau = 0 / 1: scale 2^p and bias -2^(p+23)
+    const uint32_t s0 = (uint32_t)(F - (M - 1)) << 23, s1 = s0 - 0x00800000u;
+    const uint32_t b0 = (s0 + (23u << 23)) | 0x80000000u, b1 = b0 - 0x00800000u;
 #pragma unroll
     for (int j = 0; j < kSlice / 2; ++j) {
-        const int tau = (int)((mbits >> (j * qp.d2)) & (uint32_t)qp.beta);
-        const int p = max(F - 127 - tau - (M - 1), -149);
-        const float scale = __uint_as_float(pow2_bits(p));
-        const float bias = __uint_as_float(((uint32_t)(p + 150) << 23) | 0x80000000u);  // -2^(p+23)
+        const bool t1 = (mbits >> j) & 1u;
+        float scale, bias;
+        if (FAST) {
+            scale = __uint_as_float(t1 ? s1 : s0);
+            bias = __uint_as_float(t1 ? b1 : b0);
+        } else {
+            scale = __uint_as_float(pow2_bits(max(F - 127 - (t1 ? 1 : 0) - (M - 1), -149)));
+            bias = 0.f;
+        }
 #pragma unroll
         for (int i = 0; i < 2; ++i) {
             const int k = 2 * j + i, bit = k * W, wi = bit >> 5, sh = bit & 31;
             // 32 stream bits starting at this code
             const uint32_t f = sh == 0 ? words[wi] : (sh + W > 32 ? __funnelshift_r(words[wi], words[wi + 1], sh) : words[wi] >> sh);
             const float qf = __uint_as_float(0x4B000000u | (f & kQMask));
-            const float mag = fma_ok ? fmaf(qf, scale, bias) : __fmul_rn(__fsub_rn(qf, 8388608.0f), scale);
-            yb[k] = F == 255 ? 0x7FC00000u : (__float_as_uint(mag) | ((f << (31 - M)) & 0x80000000u));
+            const float mag = FAST ? fmaf(qf, scale, bias) : __fmul_rn(__fsub_rn(qf, 8388608.0f), scale);
+            const uint32_t v = __float_as_uint(mag) | ((f << (31 - M)) & 0x80000000u);
+            yb[k] = (!FAST && F == 255) ? 0x7FC00000u : v;
         }
     }
+}
+
+// Warp-uniform choice between the two decoders (all 32 lanes must call this).
+template <int W>
+__device__ __forceinline__ void decode_slice(const uint32_t (&words)[(kSlice * W + 31) / 32 + 1], int F, uint32_t mbits,
+                                             uint32_t (&yb)[kSlice]) {
+    if (__all_sync(0xFFFFFFFFu, F >= 16 && F <= kFastMaxF)) decode_slice_impl<W, true>(words, F, mbits, yb);
+    else decode_slice_impl<W, false>(words, F, mbits, yb);
 }
 
 }  // namespace bdr

@@ -20,7 +20,7 @@ unpack_rowwise_mx_kernel(bdr_planes_t in, T* y, FastDiv warps_per_row, uint32_t 
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const uint32_t stride = gridDim.x * kWarps;
     const uint32_t w0 = blockIdx.x * kWarps + warp;
-    const int n_elem_vecs = 32 * kElemBytes / 16, n_micro_vecs = 2 * qp.d2;
+    const int n_elem_vecs = 32 * kElemBytes / 16, n_micro_vecs = 2;  // d2 = 1: one byte per slice
     auto issue = [&](uint32_t wi, int st) {
         if (wi < total) {
             const int64_t row = fastdiv(wi, warps_per_row);
@@ -34,7 +34,7 @@ unpack_rowwise_mx_kernel(bdr_planes_t in, T* y, FastDiv warps_per_row, uint32_t 
                                in.exps + row * in.ld_exps + slice0 + (v - n_elem_vecs) * 16);
                 else
                     cp_async16(stage + 32 * kElemBytes + 32 + (v - n_elem_vecs - 2) * 16,
-                               in.micro + row * in.ld_micro + slice0 * qp.d2 + (v - n_elem_vecs - 2) * 16);
+                               in.micro + row * in.ld_micro + slice0 + (v - n_elem_vecs - 2) * 16);
             }
         }
         cp_async_commit();
@@ -64,10 +64,9 @@ unpack_rowwise_mx_kernel(bdr_planes_t in, T* y, FastDiv warps_per_row, uint32_t 
             for (int h = 0; h < W; ++h) words[h >> 1] |= (uint32_t)src[h] << ((h & 1) * 16);
         }
         const int F = st_exps[lane];
-        uint32_t mbits = 0;
-        for (int b = 0; b < qp.d2; ++b) mbits |= (uint32_t)st_micro[lane * qp.d2 + b] << (8 * b);
+        const uint32_t mbits = st_micro[lane];
         uint32_t yb[kSlice];
-        decode_slice<W>(words, F, mbits, qp, yb);
+        decode_slice<W>(words, F, mbits, yb);
         store_slice_vec(y + row * ld + (slice0 + lane) * kSlice, yb);
         __syncwarp();  // everyone is done with this stage before it is refilled
     }
@@ -87,7 +86,7 @@ static int launch_unpack_row(const bdr_planes_t& in, T* y, int64_t rows, int64_t
 template <typename T>
 int unpack_rowwise_mx(const bdr_planes_t& in, T* y, int64_t rows, int64_t cols, int64_t ld, const QParams& qp,
                       cudaStream_t st) {
-    if (qp.k1 != 16 || qp.k2 != 2 || cols % 512 != 0) return BDR_ERR_UNSUPPORTED;
+    if (qp.k1 != 16 || qp.k2 != 2 || qp.d2 != 1 || cols % 512 != 0) return BDR_ERR_UNSUPPORTED;
     if (((uintptr_t)y % 16) || (ld * sizeof(T)) % 16) return BDR_ERR_UNSUPPORTED;
     switch (qp.m) {
         case 2: return launch_unpack_row<T, 3>(in, y, rows, cols, ld, qp, st);
