@@ -30,6 +30,19 @@ def _newest_header() -> float:
     return max(os.path.getmtime(h) for h in hs)
 
 
+def _included_sources(path: str) -> float:
+    """Newest mtime among the file and any local .cu file it includes textually."""
+    newest = os.path.getmtime(path)
+    with open(path) as f:
+        for line in f:
+            line = line.strip()
+            if line.startswith('#include "') and line.endswith('.cu"'):
+                dep = os.path.join(CSRC, line[len('#include "'):-1])
+                if os.path.exists(dep):
+                    newest = max(newest, os.path.getmtime(dep))
+    return newest
+
+
 def build(force: bool = False, verbose: bool = False) -> str:
     os.makedirs(OBJ, exist_ok=True)
     srcs = sorted(glob.glob(os.path.join(CSRC, "*.cu")))
@@ -39,7 +52,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
     for s in srcs:
         o = os.path.join(OBJ, os.path.basename(s)[:-3] + ".o")
         objs.append(o)
-        if force or not os.path.exists(o) or os.path.getmtime(o) < max(os.path.getmtime(s), hdr):
+        if force or not os.path.exists(o) or os.path.getmtime(o) < max(_included_sources(s), hdr):
             jobs.append([_nvcc(), *NVCC_FLAGS, "-c", s, "-o", o] + (["-Xptxas", "-v"] if verbose else []))
 
     def run(cmd):

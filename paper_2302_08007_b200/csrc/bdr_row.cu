@@ -33,13 +33,40 @@ template <typename T, int SPT> struct Ring {
     __device__ static __forceinline__ uint4 read(const uint4* warp_stage, int lane, int v) {
         return warp_stage[swz(lane * kVecs + v)];
     }
+    // Write the warp's results through the (already consumed) stage so that global stores are as
+    // coalesced as the loads: each lane drops its kVecs words at their swizzled positions, then
+    // instruction v stores words v*32 .. v*32+31 (512 contiguous bytes) of the run at dst.
+    __device__ static __forceinline__ void store_run(uint4* warp_stage, T* dst, int lane, const uint4 (&mine)[kVecs]) {
+#pragma unroll
+        for (int v = 0; v < kVecs; ++v) warp_stage[swz(lane * kVecs + v)] = mine[v];
+        __syncwarp();
+#pragma unroll
+        for (int v = 0; v < kVecs; ++v) {
+            const uint32_t c = v * 32 + lane;
+            reinterpret_cast<uint4*>(dst)[c] = warp_stage[swz(c)];
+        }
+    }
 };
 
+// dequantized bit patterns of one slice -> the 16-byte words of the output tensor
+__device__ __forceinline__ void slice_to_words(const uint32_t (&y)[kSlice], uint4 (&w)[4], const float*) {
+#pragma unroll
+    for (int i = 0; i < 4; ++i) w[i] = make_uint4(y[4 * i], y[4 * i + 1], y[4 * i + 2], y[4 * i + 3]);
+}
+__device__ __forceinline__ void slice_to_words(const uint32_t (&y)[kSlice], uint4 (&w)[2], const __nv_bfloat16*) {
+#pragma unroll
+    for (int i = 0; i < 2; ++i) {
+        uint32_t ws[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) ws[k] = (y[8 * i + 2 * k] >> 16) | (y[8 * i + 2 * k + 1] & 0xFFFF0000u);
+        w[i] = make_uint4(ws[0], ws[1], ws[2], ws[3]);
+    }
+}
+
 // Quantize the SPT slices a thread holds (shared exponents across lanes when k1 spans them).
-template <int K2, int K1S, int SPT>
+template <int K2, int K1S, int SPT, bool SUMS, bool YOUT>
 __device__ __forceinline__ void quantize_unit(const uint32_t (&u)[SPT][kSlice], const QParams& qp, int group_lanes,
-                                              bool want_sums, bool want_y, uint32_t (&yb)[SPT][kSlice], double& e2,
-                                              double& s2) {
+                                              uint32_t (&yb)[SPT][kSlice], double& e2, double& s2) {
     uint32_t fj[SPT][kSlice / K2];
     uint32_t fb[SPT][kSlice / K1S];
 #pragma unroll
@@ -64,11 +91,11 @@ __device__ __forceinline__ void quantize_unit(const uint32_t (&u)[SPT][kSlice], 
 #pragma unroll
     for (int s = 0; s < SPT; ++s) {
         uint32_t rq[kSlice], cb[kSlice / K2], tau[kSlice / K2];
-        quantize_slice_rt<K2, K1S, false>(u[s], fj[s], fb[s], qp, want_sums, want_y, yb[s], rq, cb, tau, e2, s2);
+        quantize_slice<K2, K1S, SUMS, YOUT, false>(u[s], fj[s], fb[s], qp, yb[s], rq, cb, tau, e2, s2);
     }
 }
 
-template <typename T, int K2, int K1S, int SPT>
+template <typename T, int K2, int K1S, int SPT, bool SUMS, bool YOUT>
 __global__ void __launch_bounds__(kThreads)
 quant_rowwise_kernel(const T* x, T* y, int64_t rows, int64_t cols, int64_t ld, FastDiv units_per_row,
                      uint32_t total_units, int group_lanes, QParams qp, bool vec_ok, bool all_full, double* sums) {
@@ -109,12 +136,21 @@ quant_rowwise_kernel(const T* x, T* y, int64_t rows, int64_t cols, int64_t ld, F
                     w[v] = Ring<T, SPT>::read(stage_ptr(stage), lane, s * SliceWords<T>::kVecs + v);
                 SliceWords<T>::expand(w, u[s]);
             }
-            quantize_unit<K2, K1S, SPT>(u, qp, group_lanes, sums != nullptr, y != nullptr, yb, e2, s2);
-            if (y) {
-                const uint32_t row = fastdiv(g, units_per_row);
-                T* dst = y + (int64_t)row * ld + (int64_t)(g - row * units_per_row.d) * kUnit;
+            quantize_unit<K2, K1S, SPT, SUMS, YOUT>(u, qp, group_lanes, yb, e2, s2);
+            if (YOUT) {
+                const uint32_t gw = g - lane;  // the warp's first unit: its 32 units are one contiguous run
+                const uint32_t row = fastdiv(gw, units_per_row);
+                T* dst = y + (int64_t)row * ld + (int64_t)(gw - row * units_per_row.d) * kUnit;
+                uint4 mine[kVecs];
 #pragma unroll
-                for (int s = 0; s < SPT; ++s) store_slice_vec(dst + s * kSlice, yb[s]);
+                for (int s = 0; s < SPT; ++s) {
+                    uint4 w[SliceWords<T>::kVecs];
+                    slice_to_words(yb[s], w, (const T*)nullptr);
+#pragma unroll
+                    for (int v = 0; v < SliceWords<T>::kVecs; ++v) mine[s * SliceWords<T>::kVecs + v] = w[v];
+                }
+                __syncwarp();  // every lane has read its input words from this stage
+                Ring<T, SPT>::store_run(stage_ptr(stage), dst, lane, mine);
             }
             stage = (stage + 1) % kStages;
         }
@@ -131,8 +167,8 @@ quant_rowwise_kernel(const T* x, T* y, int64_t rows, int64_t cols, int64_t ld, F
                 if (n == kSlice && vec_ok) load_slice_vec(x + row * ld + c0, u[s]);
                 else load_slice_guarded(x + row * ld + c0, 1, n, u[s]);
             }
-            quantize_unit<K2, K1S, SPT>(u, qp, group_lanes, sums != nullptr, y != nullptr, yb, e2, s2);
-            if (y) {
+            quantize_unit<K2, K1S, SPT, SUMS, YOUT>(u, qp, group_lanes, yb, e2, s2);
+            if (YOUT) {
 #pragma unroll
                 for (int s = 0; s < SPT; ++s) {
                     const int64_t c0 = col0 + s * kSlice;
@@ -143,7 +179,7 @@ quant_rowwise_kernel(const T* x, T* y, int64_t rows, int64_t cols, int64_t ld, F
             }
         }
     }
-    if (sums) block_accumulate_sums(e2, s2, sums);
+    if (SUMS) block_accumulate_sums(e2, s2, sums);
 }
 
 // ---- packing fast path: k1 = 16, k2 = 2, code width W = m + 1 -------------------------------------
@@ -194,6 +230,7 @@ pack_rowwise_mx_kernel(const T* x, T* y_dq, FastDiv warps_per_row, uint32_t tota
         __syncwarp();  // a lane's words were fetched by other lanes
         const int64_t row = fastdiv(wi, warps_per_row);
         const int64_t slice0 = (int64_t)(wi - (uint32_t)row * warps_per_row.d) * (32 * kPackSPT);  // warp's first slice in its row
+        uint4 ymine[YDQ ? kVecs : 1];
 #pragma unroll
         for (int s = 0; s < kPackSPT; ++s) {  // one slice at a time keeps the live register set small
             uint32_t u[kSlice], yb[kSlice], rq[kSlice], cb[kSlice / 2], tau[kSlice / 2];
@@ -208,7 +245,12 @@ pack_rowwise_mx_kernel(const T* x, T* y_dq, FastDiv warps_per_row, uint32_t tota
             for (int j = 0; j < kSlice / 2; ++j) F = max(F, fj[j]);
             fb[0] = F;
             quantize_slice<2, kSlice, SUMS, YDQ, true>(u, fj, fb, qp, yb, rq, cb, tau, e2, s2);
-            if (YDQ) store_slice_vec(y_dq + row * ld + (slice0 + kPackSPT * lane + s) * kSlice, yb);
+            if (YDQ) {
+                uint4 wy[kSV];
+                slice_to_words(yb, wy, (const T*)nullptr);
+#pragma unroll
+                for (int v = 0; v < kSV; ++v) ymine[s * kSV + v] = wy[v];
+            }
             uint32_t words[(kSlice * W + 31) / 32];
             pack_words<W, kSlice, 2>(u, rq, cb, words);
             const int sl = kPackSPT * lane + s;  // slice index within the warp's run
@@ -226,6 +268,10 @@ pack_rowwise_mx_kernel(const T* x, T* y_dq, FastDiv warps_per_row, uint32_t tota
 #pragma unroll
             for (int j = 0; j < kSlice / 2; ++j) mb |= tau[j] << j;
             st_micro[sl] = (uint8_t)mb;
+        }
+        if (YDQ) {
+            __syncwarp();  // every lane has read its input words from this stage
+            R::store_run(stage_ptr(rs), y_dq + row * ld + slice0 * kSlice, lane, reinterpret_cast<const uint4(&)[kVecs]>(ymine));
         }
         rs = (rs + 1) % kStages;
         __syncwarp();
@@ -252,9 +298,9 @@ static int grid_for(int64_t units, int per_cta) {
     return (int)max((int64_t)1, min(need, cap));
 }
 
-template <typename T, int K2, int K1S, int SPT>
-static int launch_quant_row(const T* x, T* y, int64_t rows, int64_t cols, int64_t ld, const QParams& qp, double* sums,
-                            cudaStream_t st) {
+template <typename T, int K2, int K1S, int SPT, bool SUMS, bool YOUT>
+static int launch_quant_row_flags(const T* x, T* y, int64_t rows, int64_t cols, int64_t ld, const QParams& qp, double* sums,
+                                  cudaStream_t st) {
     constexpr int kUnit = kSlice * SPT;
     if (ld == cols && cols % qp.k1 == 0) {  // contiguous tensor of whole blocks: one long row, no row arithmetic
         cols *= rows;
@@ -270,7 +316,7 @@ static int launch_quant_row(const T* x, T* y, int64_t rows, int64_t cols, int64_
     const bool all_full = vec_ok && padded == cols && cols % kUnit == 0 && upr % 32 == 0;
     if (total == 0) return BDR_OK;
     if (total >= (1ll << 31) - (1ll << 24)) return BDR_ERR_UNSUPPORTED;  // 32-bit unit indices (incl. prefetch look-ahead)
-    auto kern = quant_rowwise_kernel<T, K2, K1S, SPT>;
+    auto kern = quant_rowwise_kernel<T, K2, K1S, SPT, SUMS, YOUT>;
     const size_t smem = Ring<T, SPT>::kBytes;
     static bool attr_done = false;  // per instantiation; the attribute is idempotent, so a race is harmless
     if (!attr_done) {
@@ -280,6 +326,14 @@ static int launch_quant_row(const T* x, T* y, int64_t rows, int64_t cols, int64_
     kern<<<grid_for(total, kThreads), kThreads, smem, st>>>(x, y, rows, cols, ld, make_fastdiv((uint32_t)upr), (uint32_t)total, group, qp,
                                                             vec_ok, all_full, sums);
     return cudaGetLastError() == cudaSuccess ? BDR_OK : BDR_ERR_CUDA;
+}
+
+template <typename T, int K2, int K1S, int SPT>
+static int launch_quant_row(const T* x, T* y, int64_t rows, int64_t cols, int64_t ld, const QParams& qp, double* sums,
+                            cudaStream_t st) {
+    if (sums) return y ? launch_quant_row_flags<T, K2, K1S, SPT, true, true>(x, y, rows, cols, ld, qp, sums, st)
+                       : launch_quant_row_flags<T, K2, K1S, SPT, true, false>(x, y, rows, cols, ld, qp, sums, st);
+    return launch_quant_row_flags<T, K2, K1S, SPT, false, true>(x, y, rows, cols, ld, qp, sums, st);
 }
 
 template <typename T, int K1S, int SPT>
@@ -362,12 +416,12 @@ int pack_rowwise_mx(const T* x, T* y, int64_t rows, int64_t cols, int64_t ld, co
     return BDR_ERR_UNSUPPORTED;
 }
 
-template int quant_rowwise<float>(const float*, float*, int64_t, int64_t, int64_t, const QParams&, double*, cudaStream_t);
-template int quant_rowwise<__nv_bfloat16>(const __nv_bfloat16*, __nv_bfloat16*, int64_t, int64_t, int64_t,
-                                          const QParams&, double*, cudaStream_t);
-template int pack_rowwise_mx<float>(const float*, float*, int64_t, int64_t, int64_t, const bdr_planes_t&,
-                                    const QParams&, double*, cudaStream_t);
-template int pack_rowwise_mx<__nv_bfloat16>(const __nv_bfloat16*, __nv_bfloat16*, int64_t, int64_t, int64_t,
-                                            const bdr_planes_t&, const QParams&, double*, cudaStream_t);
+#ifndef BDR_ROW_DTYPE
+#define BDR_ROW_DTYPE float
+#endif
+template int quant_rowwise<BDR_ROW_DTYPE>(const BDR_ROW_DTYPE*, BDR_ROW_DTYPE*, int64_t, int64_t, int64_t, const QParams&, double*,
+                                          cudaStream_t);
+template int pack_rowwise_mx<BDR_ROW_DTYPE>(const BDR_ROW_DTYPE*, BDR_ROW_DTYPE*, int64_t, int64_t, int64_t, const bdr_planes_t&,
+                                            const QParams&, double*, cudaStream_t);
 
 }  // namespace bdr
