@@ -454,4 +454,58 @@ __device__ __forceinline__ void decode_slice(const uint32_t (&words)[(kSlice * W
     else decode_slice_impl<W, false>(words, F, mbits, yb);
 }
 
+// ---- warp-cooperative staging shared by the row-direction kernels ---------------------------------
+constexpr int kRowThreads = 256;
+
+// Prefetch ring.  Per iteration a warp consumes one contiguous run of 32 * kVecs 16-byte words (lane
+// l owns words [l*kVecs, (l+1)*kVecs)).  The warp copies the run cooperatively -- instruction v
+// moves words v*32 .. v*32+31, i.e. 512 contiguous bytes -- so every 32-byte sector is requested
+// once, and stores word c at position c ^ ((c >> 3) & (kVecs-1)) so that the later per-lane 16-byte
+// reads (stride kVecs words) hit eight different bank groups per quarter-warp.
+template <typename T, int SPT> struct Ring {
+    static constexpr int kVecs = SliceWords<T>::kVecs * SPT;  // 16-byte words per thread per iteration
+    static constexpr int kStages = kVecs >= 8 ? 2 : (kVecs >= 4 ? 3 : 4);  // ~128 bytes ahead per thread
+    static constexpr size_t kBytes = (size_t)kStages * kVecs * kRowThreads * 16;
+    __device__ static __forceinline__ uint32_t swz(uint32_t c) { return c ^ ((c >> 3) & (kVecs >= 8 ? 7u : (uint32_t)(kVecs - 1))); }
+    // warp_stage: this warp's 32*kVecs words of one stage; src: start of the warp's run in global memory
+    __device__ static __forceinline__ void issue(uint4* warp_stage, const T* src, int lane) {
+#pragma unroll
+        for (int v = 0; v < kVecs; ++v) {
+            const uint32_t c = v * 32 + lane;
+            cp_async16(warp_stage + swz(c), reinterpret_cast<const uint4*>(src) + c);
+        }
+    }
+    __device__ static __forceinline__ uint4 read(const uint4* warp_stage, int lane, int v) {
+        return warp_stage[swz(lane * kVecs + v)];
+    }
+    // Write the warp's results through the (already consumed) stage so that global stores are as
+    // coalesced as the loads: each lane drops its kVecs words at their swizzled positions, then
+    // instruction v stores words v*32 .. v*32+31 (512 contiguous bytes) of the run at dst.
+    __device__ static __forceinline__ void store_run(uint4* warp_stage, T* dst, int lane, const uint4 (&mine)[kVecs]) {
+#pragma unroll
+        for (int v = 0; v < kVecs; ++v) warp_stage[swz(lane * kVecs + v)] = mine[v];
+        __syncwarp();
+#pragma unroll
+        for (int v = 0; v < kVecs; ++v) {
+            const uint32_t c = v * 32 + lane;
+            reinterpret_cast<uint4*>(dst)[c] = warp_stage[swz(c)];
+        }
+    }
+};
+
+// dequantized bit patterns of one slice -> the 16-byte words of the output tensor
+__device__ __forceinline__ void slice_to_words(const uint32_t (&y)[kSlice], uint4 (&w)[4], const float*) {
+#pragma unroll
+    for (int i = 0; i < 4; ++i) w[i] = make_uint4(y[4 * i], y[4 * i + 1], y[4 * i + 2], y[4 * i + 3]);
+}
+__device__ __forceinline__ void slice_to_words(const uint32_t (&y)[kSlice], uint4 (&w)[2], const __nv_bfloat16*) {
+#pragma unroll
+    for (int i = 0; i < 2; ++i) {
+        uint32_t ws[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) ws[k] = (y[8 * i + 2 * k] >> 16) | (y[8 * i + 2 * k + 1] & 0xFFFF0000u);
+        w[i] = make_uint4(ws[0], ws[1], ws[2], ws[3]);
+    }
+}
+
 }  // namespace bdr

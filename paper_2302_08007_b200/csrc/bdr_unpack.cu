@@ -17,6 +17,8 @@ unpack_rowwise_mx_kernel(bdr_planes_t in, T* y, FastDiv warps_per_row, uint32_t 
     constexpr int kStage = (32 * kElemBytes + 32 + 96 + 15) / 16 * 16;
     constexpr int kStages = 3;  // packed bytes are prefetched two iterations ahead with cp.async
     __shared__ __align__(16) uint8_t stage_all[kWarps][kStages][kStage];
+    using R = Ring<T, 1>;  // only its swizzled, coalesced store path is used here
+    __shared__ __align__(16) uint4 out_stage[kWarps][32 * R::kVecs];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const uint32_t stride = gridDim.x * kWarps;
     const uint32_t w0 = blockIdx.x * kWarps + warp;
@@ -67,8 +69,10 @@ unpack_rowwise_mx_kernel(bdr_planes_t in, T* y, FastDiv warps_per_row, uint32_t 
         const uint32_t mbits = st_micro[lane];
         uint32_t yb[kSlice];
         decode_slice<W>(words, F, mbits, yb);
-        store_slice_vec(y + row * ld + (slice0 + lane) * kSlice, yb);
-        __syncwarp();  // everyone is done with this stage before it is refilled
+        uint4 mine[R::kVecs];
+        slice_to_words(yb, mine, (const T*)nullptr);
+        R::store_run(out_stage[warp], y + row * ld + slice0 * kSlice, lane, mine);  // 512 contiguous bytes per store instruction
+        __syncwarp();  // everyone is done with both stages before they are refilled
     }
 }
 
