@@ -25,17 +25,26 @@ constexpr int kSweepThreads = 256;
 constexpr int kSweepWarps = kSweepThreads / 32;
 constexpr int kTile = 4096;                    // elements per tile: a multiple of every k1 <= 1024
 constexpr int kTileSlices = kTile / kSlice;    // 256
-constexpr int kCfgGroup = 64;                  // configurations evaluated per tile visit
+constexpr int kFamGroup = 16;                  // families (up to 8 configurations each) evaluated per tile visit
 
-struct SweepCfg {
-    int32_t kind, k1, k2, d2, m, rounding;
-    int32_t k2t, k1t;  // compile-time selectors: sub-block / block size inside a slice (<= 16)
+constexpr int kFamMax = 8;  // configurations (mantissa widths) per family
+struct SweepCfg {            // one family, 32 bytes
+    int32_t k1;
+    uint8_t kind, k2, d2, rounding;
+    uint8_t k2t, k1t;        // compile-time selectors: sub-block / block size inside a slice (<= 16)
+    uint8_t nm, pad;
+    uint32_t m_packed;       // nm mantissa widths, 4 bits each
+    uint16_t idx[kFamMax];   // where each member's result goes
+    __host__ __device__ int m(int i) const { return (int)((m_packed >> (4 * i)) & 0xFu); }
 };
+static_assert(sizeof(SweepCfg) == 32, "family record size");
+static_assert(kTileSlices == kSweepThreads, "one slice per thread");
 
 struct SweepSmem {
     uint4 x[kTile / 4];            // 16-byte chunks, chunk c stored at c ^ ((c >> 3) & 3)
     uint8_t lv[kTile];             // level l (block size 2^l) starts at lv_off(l); sizes 2048, 1024, ..., 4
     double sig_warp[kSweepWarps];
+    double fam_acc[kSweepWarps][8][32];  // per-lane error sums of the family a warp is working on, one row per member
 };
 __host__ __device__ constexpr int lv_off(int l) { return kTile - (kTile >> (l - 1)); }  // 0, 2048, 3072, ...
 
@@ -46,10 +55,10 @@ __device__ __forceinline__ float round_to_int(float t, int rounding) {  // 0 <= 
     return floorf(__fadd_rn(t, 0.5f));
 }
 
-// ---- POW2 kind: error energy of one slice ------------------------------------------------------------
+// ---- POW2 kind: error energy of one slice for every mantissa width of a family -----------------------
 template <int K2, int K1S>
 __device__ __forceinline__ void pow2_slice(const uint32_t (&u)[kSlice], const SweepSmem& sm, int s, const SweepCfg& c,
-                                           const QParams& qp, double& e2) {
+                                           double* lane_acc /* member mi at lane_acc[32 * mi] */) {
     uint32_t ej[kSlice / K2], eb[kSlice / K1S];
     if (K2 == 1) {
 #pragma unroll
@@ -72,20 +81,69 @@ __device__ __forceinline__ void pow2_slice(const uint32_t (&u)[kSlice], const Sw
 #pragma unroll
         for (int b = 0; b < kSlice / K1S; ++b) eb[b] = (uint32_t)p[b] << 23;
     }
-    uint32_t yb[kSlice], rq[kSlice], cb[kSlice / K2], tau[kSlice / K2];
-    double s2 = 0.0;
-    quantize_slice<K2, K1S, true, false, false, false>(u, ej, eb, qp, yb, rq, cb, tau, e2, s2);
+    uint32_t emax = eb[0];
+#pragma unroll
+    for (int b = 1; b < kSlice / K1S; ++b) emax = max(emax, eb[b]);
+    if (c.rounding != BDR_ROUND_NEAREST_EVEN || emax == kExpMask) {
+        // ties-away or an Inf/NaN block: exact path, one member at a time
+#pragma unroll 1
+        for (int mi = 0; mi < c.nm; ++mi) {
+            QParams qp;
+            qp.k1 = c.k1; qp.k2 = c.k2; qp.d2 = c.d2; qp.m = c.m(mi); qp.rounding = c.rounding;
+            qp.beta = (1 << c.d2) - 1;
+            qp.qmax = (1u << qp.m) - 1u;
+            uint32_t yb[kSlice], rq[kSlice], cb[kSlice / K2], tau[kSlice / K2];
+            double e2 = 0.0, s2 = 0.0;
+            quantize_slice_exact<K2, K1S, true>(u, ej, eb, qp, yb, rq, cb, tau, e2, s2);
+            lane_acc[32 * mi] += e2;
+        }
+        return;
+    }
+    // Fast path, as in quantize_slice: a = |x| * 2^(127-F) and the shifts are computed once; each
+    // mantissa width only changes the rounding constant C = 1.5 * 2^(23-(m-1)-tau) and the clamp.
+    const uint32_t beta23 = (uint32_t)((1 << c.d2) - 1) << 23;
+#pragma unroll
+    for (int b = 0; b < kSlice / K1S; ++b) {
+        const uint32_t F23 = eb[b];
+        const float K = __uint_as_float(max(0x7F000000u - F23, 0x00400000u));
+        const double w = __hiloint2double((int)((F23 >> 2) + 0x30100000u), 0);  // 2^(2F-254)
+        float a[K1S];
+        uint32_t dm[K1S / K2];
+#pragma unroll
+        for (int i = 0; i < K1S; ++i) a[i] = __fmul_rn(fabsf(__uint_as_float(u[b * K1S + i])), K);
+#pragma unroll
+        for (int jj = 0; jj < K1S / K2; ++jj) dm[jj] = min(F23 - ej[b * (K1S / K2) + jj], beta23);
+#pragma unroll 1
+        for (int mi = 0; mi < c.nm; ++mi) {  // not unrolled: keeps the instruction footprint of the 15 shapes small
+            const int m = c.m(mi);
+            const uint32_t c_base = ((uint32_t)(127 + 23 - (m - 1)) << 23) | 0x400000u;
+            const uint32_t qmax = (1u << m) - 1u;
+            float pe = 0.f;
+#pragma unroll
+            for (int jj = 0; jj < K1S / K2; ++jj) {
+                const uint32_t c_bits = c_base - dm[jj];
+                const float C = __uint_as_float(c_bits), Cmax = __uint_as_float(c_bits + qmax);
+#pragma unroll
+                for (int i = 0; i < K2; ++i) {
+                    const float ai = a[jj * K2 + i];
+                    const float de = __fsub_rn(__fsub_rn(fminf(__fadd_rn(ai, C), Cmax), C), ai);  // exact
+                    pe = fmaf(de, de, pe);
+                }
+            }
+            lane_acc[32 * mi] = fma((double)pe, w, lane_acc[32 * mi]);
+        }
+    }
 }
 
 template <int K1S>
 __device__ __forceinline__ void pow2_slice_k2(const uint32_t (&u)[kSlice], const SweepSmem& sm, int s, const SweepCfg& c,
-                                              const QParams& qp, double& e2) {
+                                              double* e2) {
     switch (c.k2t) {
-        case 1: pow2_slice<1, K1S>(u, sm, s, c, qp, e2); break;
-        case 2: if constexpr (K1S >= 2) pow2_slice<2, K1S>(u, sm, s, c, qp, e2); break;
-        case 4: if constexpr (K1S >= 4) pow2_slice<4, K1S>(u, sm, s, c, qp, e2); break;
-        case 8: if constexpr (K1S >= 8) pow2_slice<8, K1S>(u, sm, s, c, qp, e2); break;
-        default: if constexpr (K1S >= 16) pow2_slice<16, K1S>(u, sm, s, c, qp, e2); break;
+        case 1: pow2_slice<1, K1S>(u, sm, s, c, e2); break;
+        case 2: if constexpr (K1S >= 2) pow2_slice<2, K1S>(u, sm, s, c, e2); break;
+        case 4: if constexpr (K1S >= 4) pow2_slice<4, K1S>(u, sm, s, c, e2); break;
+        case 8: if constexpr (K1S >= 8) pow2_slice<8, K1S>(u, sm, s, c, e2); break;
+        default: if constexpr (K1S >= 16) pow2_slice<16, K1S>(u, sm, s, c, e2); break;
     }
 }
 
@@ -97,7 +155,7 @@ __device__ __forceinline__ void add_err(float deq_mag, uint32_t ubits, double& e
 
 // Eq. 1: s = max / (2^(b-1) - 1) with m = b-1;  Eq. 2: q = RoundToInt(x / s);  descale s * q.
 __device__ __forceinline__ void int_slice(const uint32_t (&u)[kSlice], float amax, const SweepCfg& c, double& e2) {
-    const float qmax = (float)((1 << c.m) - 1);
+    const float qmax = (float)((1 << c.m(0)) - 1);
     const float s = __fdiv_rn(amax, qmax);
 #pragma unroll
     for (int i = 0; i < kSlice; ++i) {
@@ -112,10 +170,11 @@ __device__ __forceinline__ void int_slice(const uint32_t (&u)[kSlice], float ama
 
 // Scalar float with d2 exponent bits and m explicit mantissa bits under an FP32 tensor scale.
 __device__ __forceinline__ void fp_slice(const uint32_t (&u)[kSlice], float amax, const SweepCfg& c, double& e2) {
+    const int cm = c.m(0);
     const int bias = (1 << (c.d2 - 1)) - 1;
-    const float fmax = (c.d2 == 4 && c.m == 3)
+    const float fmax = (c.d2 == 4 && cm == 3)
                            ? 448.0f
-                           : __uint_as_float(((uint32_t)((1 << c.d2) - 2 - bias + 127) << 23) | (0x7FFFFFu & ~(0x7FFFFFu >> c.m)));
+                           : __uint_as_float(((uint32_t)((1 << c.d2) - 2 - bias + 127) << 23) | (0x7FFFFFu & ~(0x7FFFFFu >> cm)));
     const float s = __fdiv_rn(amax, fmax);
     const int ef_min = 1 - bias + 127;
 #pragma unroll
@@ -124,8 +183,8 @@ __device__ __forceinline__ void fp_slice(const uint32_t (&u)[kSlice], float amax
         if (s > 0.f) {
             const float a = fabsf(__fdiv_rn(__uint_as_float(u[i]), s));
             const int ef = max((int)(__float_as_uint(a) >> 23), ef_min);
-            const float step = __uint_as_float((uint32_t)(ef - c.m) << 23);
-            const float inv_step = __uint_as_float((uint32_t)(254 - (ef - c.m)) << 23);
+            const float step = __uint_as_float((uint32_t)(ef - cm) << 23);
+            const float inv_step = __uint_as_float((uint32_t)(254 - (ef - cm)) << 23);
             const float q = round_to_int(__fmul_rn(a, inv_step), c.rounding);
             mag = fabsf(__fmul_rn(fminf(__fmul_rn(q, step), fmax), s));
         }
@@ -135,7 +194,7 @@ __device__ __forceinline__ void fp_slice(const uint32_t (&u)[kSlice], float amax
 
 // VSQ: FP32 scale gamma for the tensor, unsigned d2-bit integer sub-scale per 16-element vector.
 __device__ __forceinline__ void vsq_slice(const uint32_t (&u)[kSlice], float amax, const SweepCfg& c, double& e2) {
-    const float qmax = (float)((1 << c.m) - 1);
+    const float qmax = (float)((1 << c.m(0)) - 1);
     const float umax = (float)((1u << c.d2) - 1u);
     const float gamma = __fdiv_rn(__fdiv_rn(amax, qmax), umax);
     uint32_t avb = 0;
@@ -172,7 +231,7 @@ __global__ void amax_kernel(const T* x, int64_t rows, int64_t cols, int64_t ld, 
 
 template <typename T>
 __global__ void __launch_bounds__(kSweepThreads)
-sweep_kernel(const T* x, int64_t rows, int64_t cols, int64_t ld, const SweepCfg* cfgs, int n_cfg, int n_groups,
+sweep_kernel(const T* x, int64_t rows, int64_t cols, int64_t ld, const SweepCfg* fams, int n_fam, int n_cfg, int n_groups,
              int tiles_per_row, int64_t total_units, double* err_sums, double* sig_sum, const uint32_t* amax_bits) {
     extern __shared__ __align__(16) uint8_t dyn[];
     SweepSmem& sm = *reinterpret_cast<SweepSmem*>(dyn);
@@ -245,14 +304,14 @@ sweep_kernel(const T* x, int64_t rows, int64_t cols, int64_t ld, const SweepCfg*
             __syncthreads();
             loaded_tile = tile;
         }
-        for (int ci = group * kCfgGroup + warp; ci < min(n_cfg, (group + 1) * kCfgGroup); ci += kSweepWarps) {
-            const SweepCfg c = cfgs[ci];
-            QParams qp;
-            qp.k1 = c.k1; qp.k2 = c.k2; qp.d2 = c.d2; qp.m = c.m; qp.rounding = c.rounding;
-            qp.beta = (1 << c.d2) - 1;
-            qp.qmax = (1u << c.m) - 1u;
-            double e2 = 0.0;
-            for (int s = lane; s < kTileSlices; s += 32) {
+        // All warps work on the same family at the same time (one slice per thread), so the whole CTA
+        // runs one instantiation of the slice code at a time and stays inside the instruction cache.
+        for (int fi = group * kFamGroup; fi < min(n_fam, (group + 1) * kFamGroup); ++fi) {
+            const SweepCfg c = fams[fi];
+            double* e2 = &sm.fam_acc[warp][0][lane];  // this lane's sums, member mi at e2[32 * mi]
+            for (int mi = 0; mi < c.nm; ++mi) e2[32 * mi] = 0.0;
+            {
+                const int s = threadIdx.x;  // kTileSlices == kSweepThreads
                 uint32_t u[kSlice];
 #pragma unroll
                 for (int v = 0; v < 4; ++v) {
@@ -261,22 +320,24 @@ sweep_kernel(const T* x, int64_t rows, int64_t cols, int64_t ld, const SweepCfg*
                 }
                 if (c.kind == BDR_SCALE_POW2) {
                     switch (c.k1t) {
-                        case 1: pow2_slice_k2<1>(u, sm, s, c, qp, e2); break;
-                        case 2: pow2_slice_k2<2>(u, sm, s, c, qp, e2); break;
-                        case 4: pow2_slice_k2<4>(u, sm, s, c, qp, e2); break;
-                        case 8: pow2_slice_k2<8>(u, sm, s, c, qp, e2); break;
-                        default: pow2_slice_k2<16>(u, sm, s, c, qp, e2); break;
+                        case 1: pow2_slice_k2<1>(u, sm, s, c, e2); break;
+                        case 2: pow2_slice_k2<2>(u, sm, s, c, e2); break;
+                        case 4: pow2_slice_k2<4>(u, sm, s, c, e2); break;
+                        case 8: pow2_slice_k2<8>(u, sm, s, c, e2); break;
+                        default: pow2_slice_k2<16>(u, sm, s, c, e2); break;
                     }
                 } else if (c.kind == BDR_SCALE_FP32_INT) {
-                    int_slice(u, amax, c, e2);
+                    int_slice(u, amax, c, e2[0]);
                 } else if (c.kind == BDR_SCALE_FP32_FP) {
-                    fp_slice(u, amax, c, e2);
+                    fp_slice(u, amax, c, e2[0]);
                 } else {
-                    vsq_slice(u, amax, c, e2);
+                    vsq_slice(u, amax, c, e2[0]);
                 }
             }
-            e2 = warp_sum(e2);
-            if (lane == 0) acc[ci] += e2;  // this warp is the only writer of acc[ci] in the CTA
+            for (int mi = 0; mi < c.nm; ++mi) {
+                const double t = warp_sum(e2[32 * mi]);
+                if (lane == 0) atomicAdd(&acc[c.idx[mi]], t);  // eight warps share the slot
+            }
         }
     }
     __syncthreads();
@@ -312,18 +373,20 @@ int64_t sweep_workspace_bytes(int n) { return (int64_t)((ws_cfg_offset(n) + (siz
 
 static bool is_pow2i(int v) { return v > 0 && (v & (v - 1)) == 0; }
 
-// Validate one configuration for the sweep and translate it.
-static int make_sweep_cfg(const bdr_config_t& c, SweepCfg* out) {
+// Validate one configuration for the sweep and translate it into a one-member family.
+static int make_sweep_cfg(const bdr_config_t& c, int index, SweepCfg* out) {
     if (c.rounding != BDR_ROUND_NEAREST_EVEN && c.rounding != BDR_ROUND_NEAREST_AWAY) return BDR_ERR_BAD_CONFIG;
-    SweepCfg s = {c.scale_kind, c.k1, c.k2, c.d2, c.m, c.rounding, 1, 1};
+    SweepCfg s = {};
+    s.k1 = c.k1; s.kind = (uint8_t)c.scale_kind; s.rounding = (uint8_t)c.rounding;
+    s.k2t = 1; s.k1t = 1; s.nm = 1;
     switch (c.scale_kind) {
         case BDR_SCALE_POW2:
             if (c.d1 != 8 || c.k1 < 1 || c.k2 < 1 || c.k1 % c.k2 != 0 || c.d2 < 0 || c.d2 > 3 || c.m < 1 || c.m > 8)
                 return BDR_ERR_BAD_CONFIG;
             if (!is_pow2i(c.k1) || !is_pow2i(c.k2) || c.k1 > 1024) return BDR_ERR_UNSUPPORTED;
-            s.k1t = c.k1 < kSlice ? c.k1 : kSlice;
-            s.k2t = c.d2 == 0 ? s.k1t : c.k2;  // d2 = 0: every shift is zero whatever k2 is
-            if (s.k2t > kSlice) return BDR_ERR_UNSUPPORTED;
+            s.k1t = (uint8_t)(c.k1 < kSlice ? c.k1 : kSlice);
+            s.k2t = (uint8_t)(c.d2 == 0 ? s.k1t : c.k2);  // d2 = 0: every shift is zero whatever k2 is
+            if (c.d2 != 0 && c.k2 > kSlice) return BDR_ERR_UNSUPPORTED;
             break;
         case BDR_SCALE_FP32_INT:
             if (c.m < 1 || c.m > 15) return BDR_ERR_BAD_CONFIG;
@@ -339,22 +402,45 @@ static int make_sweep_cfg(const bdr_config_t& c, SweepCfg* out) {
             break;
         default: return BDR_ERR_BAD_CONFIG;
     }
+    s.k2 = (uint8_t)(c.scale_kind == BDR_SCALE_POW2 ? s.k2t : c.k2);  // the effective sub-block size
+    s.d2 = (uint8_t)c.d2;
+    s.m_packed = (uint32_t)c.m;
+    s.idx[0] = (uint16_t)index;
     *out = s;
     return BDR_OK;
 }
 
+// Merge configurations that differ only in m into families of up to kFamMax members.
+static void build_families(const std::vector<SweepCfg>& singles, std::vector<SweepCfg>* fams) {
+    for (const SweepCfg& c : singles) {
+        bool merged = false;
+        if (c.kind == BDR_SCALE_POW2) {
+            for (SweepCfg& f : *fams) {
+                if (f.kind == c.kind && f.k1 == c.k1 && f.k2 == c.k2 && f.d2 == c.d2 && f.rounding == c.rounding && f.nm < kFamMax) {
+                    f.m_packed |= c.m_packed << (4 * f.nm);
+                    f.idx[f.nm] = c.idx[0];
+                    f.nm++;
+                    merged = true;
+                    break;
+                }
+            }
+        }
+        if (!merged) fams->push_back(c);
+    }
+}
+
 template <typename T>
-static int sweep_launch(const SweepCfg* host_cfgs, int n, bool need_amax, const T* x, int64_t rows, int64_t cols, int64_t ld,
-                        double* out_db, uint8_t* ws, cudaStream_t st) {
+static int sweep_launch(const SweepCfg* host_fams, int n_fam, int n, bool need_amax, const T* x, int64_t rows, int64_t cols,
+                        int64_t ld, double* out_db, uint8_t* ws, cudaStream_t st) {
     double* err = reinterpret_cast<double*>(ws);
     double* sig = err + n;
     uint32_t* amax = reinterpret_cast<uint32_t*>(sig + 1);
     SweepCfg* dcfg = reinterpret_cast<SweepCfg*>(ws + ws_cfg_offset(n));
     if (cudaMemsetAsync(ws, 0, ws_cfg_offset(n), st) != cudaSuccess) return BDR_ERR_CUDA;
-    for (int i0 = 0; i0 < n; i0 += kCfgChunk) {
+    for (int i0 = 0; i0 < n_fam; i0 += kCfgChunk) {
         CfgChunk chunk;
-        const int cnt = min(kCfgChunk, n - i0);
-        for (int i = 0; i < cnt; ++i) chunk.c[i] = host_cfgs[i0 + i];
+        const int cnt = min(kCfgChunk, n_fam - i0);
+        for (int i = 0; i < cnt; ++i) chunk.c[i] = host_fams[i0 + i];
         upload_cfgs_kernel<<<1, kCfgChunk, 0, st>>>(chunk, dcfg + i0, cnt);
     }
     if (rows > 0 && cols > 0) {
@@ -364,13 +450,13 @@ static int sweep_launch(const SweepCfg* host_cfgs, int n, bool need_amax, const 
             amax_kernel<T><<<grid, 256, 0, st>>>(x, rows, cols, ld, amax);
         }
         const int tiles_per_row = (int)((cols + kTile - 1) / kTile);
-        const int n_groups = (n + kCfgGroup - 1) / kCfgGroup;
+        const int n_groups = (n_fam + kFamGroup - 1) / kFamGroup;
         const int64_t units = rows * tiles_per_row * n_groups;
         const size_t smem = sizeof(SweepSmem) + (size_t)n * sizeof(double);
         auto kern = sweep_kernel<T>;
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return BDR_ERR_CUDA;
         const int grid = (int)max((int64_t)1, min(units, (int64_t)sm_count() * 4));
-        kern<<<grid, kSweepThreads, smem, st>>>(x, rows, cols, ld, dcfg, n, n_groups, tiles_per_row, units, err, sig, amax);
+        kern<<<grid, kSweepThreads, smem, st>>>(x, rows, cols, ld, dcfg, n_fam, n, n_groups, tiles_per_row, units, err, sig, amax);
     }
     qsnr_finalize_kernel<<<(n + 127) / 128, 128, 0, st>>>(err, sig, n, out_db);
     return cudaGetLastError() == cudaSuccess ? BDR_OK : BDR_ERR_CUDA;
@@ -419,20 +505,22 @@ int bdr_qsnr(const bdr_config_t* cfgs, int n_cfgs, const void* x, bdr_dtype_t dt
     if (rows < 0 || cols < 0 || ld < cols) return BDR_ERR_SIZE;
     if (!x && rows > 0 && cols > 0) return BDR_ERR_NULL;
     if ((uintptr_t)x % (dt == BDR_F32 ? 4 : 2) || (uintptr_t)qsnr_db_dev % 8) return BDR_ERR_MISALIGNED;
-    std::vector<SweepCfg> table(n_cfgs);
+    std::vector<SweepCfg> singles(n_cfgs), table;
     bool need_amax = false;
     for (int i = 0; i < n_cfgs; ++i) {
-        const int rc = make_sweep_cfg(cfgs[i], &table[i]);
+        const int rc = make_sweep_cfg(cfgs[i], i, &singles[i]);
         if (rc) return rc;
         need_amax |= cfgs[i].scale_kind != BDR_SCALE_POW2;
     }
+    build_families(singles, &table);
+    const int n_fam = (int)table.size();
     if (axis != 1) return BDR_ERR_UNSUPPORTED;  // the sweep walks rows; column-wise QSNR comes from bdr_quant_dequant's sums
     if (!workspace || workspace_bytes < sweep_workspace_bytes(n_cfgs)) return BDR_ERR_WORKSPACE;
     if ((uintptr_t)workspace % 16) return BDR_ERR_MISALIGNED;
     cudaStream_t st = (cudaStream_t)stream;
     if (dt == BDR_F32)
-        return sweep_launch<float>(table.data(), n_cfgs, need_amax, (const float*)x, rows, cols, ld, qsnr_db_dev, (uint8_t*)workspace, st);
-    return sweep_launch<__nv_bfloat16>(table.data(), n_cfgs, need_amax, (const __nv_bfloat16*)x, rows, cols, ld, qsnr_db_dev,
+        return sweep_launch<float>(table.data(), n_fam, n_cfgs, need_amax, (const float*)x, rows, cols, ld, qsnr_db_dev, (uint8_t*)workspace, st);
+    return sweep_launch<__nv_bfloat16>(table.data(), n_fam, n_cfgs, need_amax, (const __nv_bfloat16*)x, rows, cols, ld, qsnr_db_dev,
                                        (uint8_t*)workspace, st);
 }
 
