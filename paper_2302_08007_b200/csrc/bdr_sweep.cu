@@ -40,9 +40,13 @@ struct SweepCfg {            // one family, 32 bytes
 static_assert(sizeof(SweepCfg) == 32, "family record size");
 static_assert(kTileSlices == kSweepThreads, "one slice per thread");
 
-struct SweepSmem {
+constexpr int kTilesPerUnit = 4;  // tiles a CTA keeps resident while it walks a group of families
+struct SweepTile {
     uint4 x[kTile / 4];            // 16-byte chunks, chunk c stored at c ^ ((c >> 3) & 3)
     uint8_t lv[kTile];             // level l (block size 2^l) starts at lv_off(l); sizes 2048, 1024, ..., 4
+};
+struct SweepSmem {
+    SweepTile t[kTilesPerUnit];
     double sig_warp[kSweepWarps];
     double fam_acc[kSweepWarps][8][32];  // per-lane error sums of the family a warp is working on, one row per member
 };
@@ -57,7 +61,7 @@ __device__ __forceinline__ float round_to_int(float t, int rounding) {  // 0 <= 
 
 // ---- POW2 kind: error energy of one slice for every mantissa width of a family -----------------------
 template <int K2, int K1S>
-__device__ __forceinline__ void pow2_slice(const uint32_t (&u)[kSlice], const SweepSmem& sm, int s, const SweepCfg& c,
+__device__ __forceinline__ void pow2_slice(const uint32_t (&u)[kSlice], const SweepTile& sm, int s, const SweepCfg& c,
                                            double* lane_acc /* member mi at lane_acc[32 * mi] */) {
     uint32_t ej[kSlice / K2], eb[kSlice / K1S];
     if (K2 == 1) {
@@ -136,7 +140,7 @@ __device__ __forceinline__ void pow2_slice(const uint32_t (&u)[kSlice], const Sw
 }
 
 template <int K1S>
-__device__ __forceinline__ void pow2_slice_k2(const uint32_t (&u)[kSlice], const SweepSmem& sm, int s, const SweepCfg& c,
+__device__ __forceinline__ void pow2_slice_k2(const uint32_t (&u)[kSlice], const SweepTile& sm, int s, const SweepCfg& c,
                                               double* e2) {
     switch (c.k2t) {
         case 1: pow2_slice<1, K1S>(u, sm, s, c, e2); break;
@@ -240,43 +244,47 @@ sweep_kernel(const T* x, int64_t rows, int64_t cols, int64_t ld, const SweepCfg*
     for (int c = threadIdx.x; c < n_cfg; c += kSweepThreads) acc[c] = 0.0;
     double sig_acc = 0.0;
     const float amax = __uint_as_float(*amax_bits);
-    int64_t loaded_tile = -1;
+    const int64_t total_tiles = rows * tiles_per_row;
     for (int64_t unit = blockIdx.x; unit < total_units; unit += gridDim.x) {
-        const int64_t tile = unit / n_groups;
-        const int group = (int)(unit - tile * n_groups);
-        if (tile != loaded_tile) {
-            __syncthreads();  // everyone is done with the previous tile
+        const int64_t tgroup = unit / n_groups;              // kTilesPerUnit consecutive tiles
+        const int group = (int)(unit - tgroup * n_groups);   // kFamGroup consecutive families
+        const int64_t tile0 = tgroup * kTilesPerUnit;
+        const int ntiles = (int)min((int64_t)kTilesPerUnit, total_tiles - tile0);
+        __syncthreads();  // everyone is done with the previous unit's tiles
+        for (int ti = 0; ti < ntiles; ++ti) {
+            SweepTile& tl = sm.t[ti];
+            const int64_t tile = tile0 + ti;
             const int64_t row = tile / tiles_per_row;
             const int64_t t0 = (tile - row * tiles_per_row) * kTile;
             const int n = (int)min((int64_t)kTile, cols - t0);
             const T* src = x + row * ld + t0;
             // stage: thread t owns slice t (16 elements = 4 chunks)
-            {
-                const int s = threadIdx.x;
-                uint32_t u[kSlice];
-                load_slice_guarded(src + s * kSlice, 1, max(0, min(kSlice, n - s * kSlice)), u);
+            const int s = threadIdx.x;
+            uint32_t u[kSlice];
+            load_slice_guarded(src + s * kSlice, 1, max(0, min(kSlice, n - s * kSlice)), u);
 #pragma unroll
-                for (int v = 0; v < 4; ++v) sm.x[swz4(4 * s + v)] = make_uint4(u[4 * v], u[4 * v + 1], u[4 * v + 2], u[4 * v + 3]);
-                // exponent pyramid levels 1..4 from the slice, signal energy of the slice
-                uint32_t e[kSlice];
+            for (int v = 0; v < 4; ++v) tl.x[swz4(4 * s + v)] = make_uint4(u[4 * v], u[4 * v + 1], u[4 * v + 2], u[4 * v + 3]);
+            // exponent pyramid levels 1..4 from the slice
+            uint32_t e[kSlice];
 #pragma unroll
-                for (int i = 0; i < kSlice; ++i) e[i] = u[i] >> 23 & 0xFFu;
+            for (int i = 0; i < kSlice; ++i) e[i] = u[i] >> 23 & 0xFFu;
 #pragma unroll
-                for (int l = 1; l <= 4; ++l) {
+            for (int l = 1; l <= 4; ++l) {
 #pragma unroll
-                    for (int j = 0; j < (kSlice >> l); ++j) {
-                        e[j] = max(e[2 * j], e[2 * j + 1]);
-                        sm.lv[lv_off(l) + s * (kSlice >> l) + j] = (uint8_t)e[j];
-                    }
+                for (int j = 0; j < (kSlice >> l); ++j) {
+                    e[j] = max(e[2 * j], e[2 * j + 1]);
+                    tl.lv[lv_off(l) + s * (kSlice >> l) + j] = (uint8_t)e[j];
                 }
-                // levels 5..9 inside the warp (a warp covers 512 consecutive elements), level 10 below
-                uint32_t v = e[0];
+            }
+            // levels 5..9 inside the warp (a warp covers 512 consecutive elements), level 10 below
+            uint32_t v = e[0];
 #pragma unroll
-                for (int l = 5; l <= 9; ++l) {
-                    v = max(v, __shfl_xor_sync(0xFFFFFFFFu, v, 1 << (l - 5)));
-                    if ((lane & ((1 << (l - 4)) - 1)) == 0) sm.lv[lv_off(l) + (s >> (l - 4))] = (uint8_t)v;
-                }
-                // signal energy: sum x^2 normalised by the slice exponent, widened once
+            for (int l = 5; l <= 9; ++l) {
+                v = max(v, __shfl_xor_sync(0xFFFFFFFFu, v, 1 << (l - 5)));
+                if ((lane & ((1 << (l - 4)) - 1)) == 0) tl.lv[lv_off(l) + (s >> (l - 4))] = (uint8_t)v;
+            }
+            // signal energy: sum x^2 normalised by the slice exponent, widened once (first family group only)
+            if (group == 0) {
                 const uint32_t F23 = e[0] << 23;
                 const float K = __uint_as_float(max(0x7F000000u - F23, 0x00400000u));
                 float ps = 0.f;
@@ -291,40 +299,39 @@ sweep_kernel(const T* x, int64_t rows, int64_t cols, int64_t ld, const SweepCfg*
                     }
                     sg = (double)ps * __hiloint2double((int)((F23 >> 2) + 0x30100000u), 0);
                 }
-                sg = warp_sum(sg);
-                if (lane == 0) sm.sig_warp[warp] = sg;
+                sig_acc += sg;  // per thread; reduced once at the end of the kernel
             }
-            __syncthreads();
-            if (threadIdx.x < kTile / 1024)
-                sm.lv[lv_off(10) + threadIdx.x] = max(sm.lv[lv_off(9) + 2 * threadIdx.x], sm.lv[lv_off(9) + 2 * threadIdx.x + 1]);
-            if (threadIdx.x == 0 && group == 0) {
-#pragma unroll
-                for (int w = 0; w < kSweepWarps; ++w) sig_acc += sm.sig_warp[w];
-            }
-            __syncthreads();
-            loaded_tile = tile;
         }
-        // All warps work on the same family at the same time (one slice per thread), so the whole CTA
-        // runs one instantiation of the slice code at a time and stays inside the instruction cache.
+        __syncthreads();
+        if (threadIdx.x < ntiles * (kTile / 1024)) {
+            SweepTile& tl = sm.t[threadIdx.x / (kTile / 1024)];
+            const int i = threadIdx.x % (kTile / 1024);
+            tl.lv[lv_off(10) + i] = max(tl.lv[lv_off(9) + 2 * i], tl.lv[lv_off(9) + 2 * i + 1]);
+        }
+        __syncthreads();
+        // All warps work on the same family at the same time (one slice per thread and tile), so the
+        // whole CTA runs one instantiation of the slice code at a time and stays inside the
+        // instruction cache; a lane's sums over the unit's tiles are reduced once per family.
         for (int fi = group * kFamGroup; fi < min(n_fam, (group + 1) * kFamGroup); ++fi) {
             const SweepCfg c = fams[fi];
             double* e2 = &sm.fam_acc[warp][0][lane];  // this lane's sums, member mi at e2[32 * mi]
             for (int mi = 0; mi < c.nm; ++mi) e2[32 * mi] = 0.0;
-            {
+            for (int ti = 0; ti < ntiles; ++ti) {
+                const SweepTile& tl = sm.t[ti];
                 const int s = threadIdx.x;  // kTileSlices == kSweepThreads
                 uint32_t u[kSlice];
 #pragma unroll
                 for (int v = 0; v < 4; ++v) {
-                    const uint4 w = sm.x[swz4(4 * s + v)];
+                    const uint4 w = tl.x[swz4(4 * s + v)];
                     u[4 * v] = w.x; u[4 * v + 1] = w.y; u[4 * v + 2] = w.z; u[4 * v + 3] = w.w;
                 }
                 if (c.kind == BDR_SCALE_POW2) {
                     switch (c.k1t) {
-                        case 1: pow2_slice_k2<1>(u, sm, s, c, e2); break;
-                        case 2: pow2_slice_k2<2>(u, sm, s, c, e2); break;
-                        case 4: pow2_slice_k2<4>(u, sm, s, c, e2); break;
-                        case 8: pow2_slice_k2<8>(u, sm, s, c, e2); break;
-                        default: pow2_slice_k2<16>(u, sm, s, c, e2); break;
+                        case 1: pow2_slice_k2<1>(u, tl, s, c, e2); break;
+                        case 2: pow2_slice_k2<2>(u, tl, s, c, e2); break;
+                        case 4: pow2_slice_k2<4>(u, tl, s, c, e2); break;
+                        case 8: pow2_slice_k2<8>(u, tl, s, c, e2); break;
+                        default: pow2_slice_k2<16>(u, tl, s, c, e2); break;
                     }
                 } else if (c.kind == BDR_SCALE_FP32_INT) {
                     int_slice(u, amax, c, e2[0]);
@@ -338,6 +345,17 @@ sweep_kernel(const T* x, int64_t rows, int64_t cols, int64_t ld, const SweepCfg*
                 const double t = warp_sum(e2[32 * mi]);
                 if (lane == 0) atomicAdd(&acc[c.idx[mi]], t);  // eight warps share the slot
             }
+        }
+    }
+    // signal energy: every thread holds a partial sum
+    {
+        const double sg = warp_sum(sig_acc);
+        if (lane == 0) sm.sig_warp[warp] = sg;
+        __syncthreads();
+        sig_acc = 0.0;
+        if (threadIdx.x == 0) {
+#pragma unroll
+            for (int w = 0; w < kSweepWarps; ++w) sig_acc += sm.sig_warp[w];
         }
     }
     __syncthreads();
@@ -451,11 +469,11 @@ static int sweep_launch(const SweepCfg* host_fams, int n_fam, int n, bool need_a
         }
         const int tiles_per_row = (int)((cols + kTile - 1) / kTile);
         const int n_groups = (n_fam + kFamGroup - 1) / kFamGroup;
-        const int64_t units = rows * tiles_per_row * n_groups;
+        const int64_t units = (rows * tiles_per_row + kTilesPerUnit - 1) / kTilesPerUnit * n_groups;
         const size_t smem = sizeof(SweepSmem) + (size_t)n * sizeof(double);
         auto kern = sweep_kernel<T>;
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return BDR_ERR_CUDA;
-        const int grid = (int)max((int64_t)1, min(units, (int64_t)sm_count() * 4));
+        const int grid = (int)max((int64_t)1, min(units, (int64_t)sm_count() * 2));
         kern<<<grid, kSweepThreads, smem, st>>>(x, rows, cols, ld, dcfg, n_fam, n, n_groups, tiles_per_row, units, err, sig, amax);
     }
     qsnr_finalize_kernel<<<(n + 127) / 128, 128, 0, st>>>(err, sig, n, out_db);
