@@ -49,11 +49,12 @@ def build(force: bool = False, verbose: bool = False) -> str:
     hdr = _newest_header()
     jobs = []
     objs = []
+    extra = os.environ.get("BDR_NVCC_EXTRA", "").split()  # extra nvcc flags, e.g. experiment macros
     for s in srcs:
         o = os.path.join(OBJ, os.path.basename(s)[:-3] + ".o")
         objs.append(o)
         if force or not os.path.exists(o) or os.path.getmtime(o) < max(_included_sources(s), hdr):
-            jobs.append([_nvcc(), *NVCC_FLAGS, "-c", s, "-o", o] + (["-Xptxas", "-v"] if verbose else []))
+            jobs.append([_nvcc(), *NVCC_FLAGS, *extra, "-c", s, "-o", o] + (["-Xptxas", "-v"] if verbose else []))
 
     def run(cmd):
         r = subprocess.run(cmd, capture_output=True, text=True)

@@ -37,8 +37,9 @@ template <int W> struct ChunkPlanes {
 constexpr int kMaxPk = 3;  // packed-chunk buffers (TMA runs up to kPk-1 chunks ahead of the decoders)
 template <int WA, int WB> struct PairSmem {
     static constexpr int kPackedBytes = ChunkPlanes<WA>::kBytes + ChunkPlanes<WB>::kBytes;  // one buffer
-    // three packed buffers when two operand stages still fit beside them, else two
-    static constexpr int kPk = (224 * 1024 - 3 * kPackedBytes - 1024) / kPairStageBytes >= 2 ? 3 : 2;
+    // a third packed buffer only when four operand stages still fit beside it: the MMA round trip
+    // (decoders -> leader's barrier -> MMA -> multicast commit -> decoders) is long, so stages come first
+    static constexpr int kPk = (224 * 1024 - 3 * kPackedBytes - 1024) / kPairStageBytes >= 4 ? 3 : 2;
     static constexpr int kBudget = 224 * 1024 - kPk * kPackedBytes - 1024;
     static constexpr int kStages = kBudget / kPairStageBytes >= 4 ? 4 : kBudget / kPairStageBytes;
     static_assert(kStages >= 2, "operand stages do not fit");
