@@ -18,32 +18,33 @@
 namespace bdr {
 
 constexpr int kPairRows = 128;                  // rows of A and of the B half per CTA
-constexpr int kChunkK = 256;                    // K elements per bulk-copy chunk (4 K steps)
-constexpr int kStepsPerChunk = kChunkK / kBK;   // 4
+constexpr int kChunkK = 256;                    // K elements per exponent / microexponent tile (16 bytes per row)
+constexpr int kEChunkK = 128;                   // K elements per code tile (two K steps): small, so more operand stages fit
+constexpr int kStepsPerEChunk = kEChunkK / kBK; // 2
 constexpr int kPairDecodeWarps = 16;            // two threads per row: each decodes two of the row's four blocks per K step
 constexpr int kLoaderWarp = 16, kMmaWarp = 17;
 constexpr int kPairThreads = 18 * 32;
 constexpr int kPairStageBytes = 2 * kPairRows * kBK * 2;  // A 16 KB + B half 16 KB
 
-// Packed bytes of one chunk (256 K elements) for 128 rows, as the TMA writes them: dense row-major
-// arrays [128][codes], [128][16 exponent bytes], [128][16 microexponent bytes].
+// Packed bytes as the TMA writes them, dense row-major, for the 128 rows of one operand:
+// codes of one 128-element K chunk [128][16 W bytes], and per 256-element K chunk the exponent and
+// microexponent bytes [128][16] each.
 template <int W> struct ChunkPlanes {
-    static constexpr int kElemRow = kChunkK * W / 8;  // 96 / 160 / 256 bytes of codes per row
-    static constexpr int kElems = 0;
-    static constexpr int kExps = kPairRows * kElemRow;
-    static constexpr int kMicro = kExps + kPairRows * 16;
-    static constexpr int kBytes = kMicro + kPairRows * 16;  // a multiple of 128
+    static constexpr int kElemRow = kEChunkK * W / 8;      // 48 / 80 / 128 bytes of codes per row
+    static constexpr int kBytes = kPairRows * kElemRow;    // a multiple of 128
 };
-constexpr int kMaxPk = 3;  // packed-chunk buffers (TMA runs up to kPk-1 chunks ahead of the decoders)
+constexpr int kXmPlane = kPairRows * 16;                   // one exponent or microexponent tile
+constexpr int kXmBytes = 4 * kXmPlane;                     // A exps | A micro | B exps | B micro
+constexpr int kMaxPk = 2;                                  // code-chunk buffers (and exponent buffers)
 template <int WA, int WB> struct PairSmem {
-    static constexpr int kPackedBytes = ChunkPlanes<WA>::kBytes + ChunkPlanes<WB>::kBytes;  // one buffer
-    // a third packed buffer only when four operand stages still fit beside it: the MMA round trip
-    // (decoders -> leader's barrier -> MMA -> multicast commit -> decoders) is long, so stages come first
-    static constexpr int kPk = (224 * 1024 - 3 * kPackedBytes - 1024) / kPairStageBytes >= 4 ? 3 : 2;
-    static constexpr int kBudget = 224 * 1024 - kPk * kPackedBytes - 1024;
-    static constexpr int kStages = kBudget / kPairStageBytes >= 4 ? 4 : kBudget / kPairStageBytes;
+    static constexpr int kPk = kMaxPk;
+    static constexpr int kPackedBytes = ChunkPlanes<WA>::kBytes + ChunkPlanes<WB>::kBytes;  // one code buffer
+    static constexpr int kBudget = 224 * 1024 - kPk * kPackedBytes - 2 * kXmBytes - 1024;
+    // the MMA round trip (decoders -> leader's barrier -> MMA -> multicast commit -> decoders) is long:
+    // as many operand stages as fit
+    static constexpr int kStages = kBudget / kPairStageBytes >= 6 ? 6 : kBudget / kPairStageBytes;
     static_assert(kStages >= 2, "operand stages do not fit");
-    static constexpr size_t kBytes = (size_t)kStages * kPairStageBytes + kPk * kPackedBytes + 1024 /*bookkeeping*/ + 1024 /*alignment*/;
+    static constexpr size_t kBytes = (size_t)kStages * kPairStageBytes + kPk * kPackedBytes + 2 * kXmBytes + 1024 /*bookkeeping*/ + 1024 /*alignment*/;
 };
 
 struct PairMaps {  // tensor maps of the three planes of A and of B (uint8 elements, rows x row bytes)
@@ -51,7 +52,7 @@ struct PairMaps {  // tensor maps of the three planes of A and of B (uint8 eleme
 };
 
 struct PairBars {
-    uint64_t full[4], empty[4], accum, pk_full[kMaxPk], pk_empty[kMaxPk];
+    uint64_t full[6], empty[6], accum, pk_full[kMaxPk], pk_empty[kMaxPk];
     uint32_t tmem_base;
     int failed;
 };
@@ -120,23 +121,23 @@ __device__ __forceinline__ void umma2_bf16(uint32_t tmem_d, uint64_t desc_a, uin
 // D = fp32, A = B = bf16, both K-major, N = 256, M = 256 (128 rows per CTA)
 constexpr uint32_t kPairInstrDesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(256 >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
 
-// pk0 / pk1: shared-memory addresses of this operand's ChunkPlanes in the two packed buffers.
-// `half` selects which two of the row's four 16-element blocks of a K step this thread decodes.
+// pk0: shared-memory address of this operand's codes in code buffer 0 (buffers are pk_stride apart);
+// xm0: address of this operand's exponent tile in exponent buffer 0 (its microexponents follow at
+// +kXmPlane; buffers are kXmBytes apart).  `half` selects which two of the row's four 16-element
+// blocks of a K step this thread decodes.
 template <int W>
-__device__ __forceinline__ bool pair_decode_rows(uint32_t pk0, uint32_t pk_stride, int n_pk, int r, int half, uint32_t tile_off,
+__device__ __forceinline__ bool pair_decode_rows(uint32_t pk0, uint32_t pk_stride, uint32_t xm0, int r, int half, uint32_t tile_off,
                                                  uint32_t stages_addr, int n_stages, PairBars& bars, int nk, int lane) {
     constexpr int NW = 2 * kSlice * W / 32;  // code words of two blocks: 3 / 5 / 8
-    constexpr int NLD = (NW + 1) / 2;        // 8-byte loads that cover them (the run starts 4-byte aligned)
     for (int kk = 0; kk < nk; ++kk) {
-        const int chunk = kk / kStepsPerChunk, ks = kk % kStepsPerChunk, buf = chunk % n_pk;
+        const int ech = kk / kStepsPerEChunk, ks = kk % kStepsPerEChunk, buf = ech % kMaxPk;
         if (ks == 0) {
-            bool ok = mbar_wait(&bars.pk_full[buf], (chunk / n_pk) & 1);
+            bool ok = mbar_wait(&bars.pk_full[buf], (ech / kMaxPk) & 1);
             ok = __all_sync(0xFFFFFFFFu, ok);
             if (!ok) return false;
         }
-        const uint32_t pk = pk0 + buf * pk_stride;
         // the two blocks' codes: 4W bytes starting at byte ks*8W + half*4W of the row (4-byte aligned)
-        const uint32_t ebase = pk + ChunkPlanes<W>::kElems + r * ChunkPlanes<W>::kElemRow + ks * (kBK * W / 8) + half * (4 * W);
+        const uint32_t ebase = pk0 + buf * pk_stride + r * ChunkPlanes<W>::kElemRow + ks * (kBK * W / 8) + half * (4 * W);
         uint32_t w[NW + 1];
         if ((4 * W) % 8 == 0) {
 #pragma unroll
@@ -146,8 +147,10 @@ __device__ __forceinline__ bool pair_decode_rows(uint32_t pk0, uint32_t pk_strid
             for (int i = 0; i < NW; ++i) w[i] = ld_shared_b32(ebase + 4 * i);
         }
         w[NW] = 0;
-        const uint32_t exps2 = (ld_shared_b32(pk + ChunkPlanes<W>::kExps + r * 16 + 4 * ks) >> (16 * half)) & 0xFFFFu;
-        const uint32_t micro2 = (ld_shared_b32(pk + ChunkPlanes<W>::kMicro + r * 16 + 4 * ks) >> (16 * half)) & 0xFFFFu;
+        // exponent / microexponent bytes of this K step: 4 bytes each within the row's 16 (256 K elements)
+        const uint32_t xm = xm0 + ((kk / 4) & 1) * kXmBytes + r * 16 + 4 * (kk & 3);
+        const uint32_t exps2 = (ld_shared_b32(xm) >> (16 * half)) & 0xFFFFu;
+        const uint32_t micro2 = (ld_shared_b32(xm + kXmPlane) >> (16 * half)) & 0xFFFFu;
         const int stage = kk % n_stages;
         if (kk >= n_stages) {
             bool ok = mbar_wait(&bars.empty[stage], ((kk / n_stages) - 1) & 1);
@@ -171,7 +174,7 @@ __device__ __forceinline__ bool pair_decode_rows(uint32_t pk0, uint32_t pk_strid
         __syncwarp();
         if (lane == 0) {
             mbar_arrive_cluster(&bars.full[stage], 0);                            // the leader CTA counts both CTAs' decoders
-            if (ks == kStepsPerChunk - 1) mbar_arrive(&bars.pk_empty[buf]);       // this warp is done with the packed buffer
+            if (ks == kStepsPerEChunk - 1) mbar_arrive(&bars.pk_empty[buf]);      // this warp is done with the code buffer
         }
     }
     return true;
@@ -185,17 +188,18 @@ mx_gemm_pair_kernel(const __grid_constant__ PairMaps maps, int64_t M, int64_t N,
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     uint8_t* stages = reinterpret_cast<uint8_t*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     constexpr int kPk = SM::kPk;
-    uint8_t* pk_base = stages + kStages * kPairStageBytes;  // kPk packed buffers of SM::kPackedBytes each
-    PairBars& bars = *reinterpret_cast<PairBars*>(pk_base + kPk * SM::kPackedBytes);
+    uint8_t* pk_base = stages + kStages * kPairStageBytes;        // kPk code buffers of SM::kPackedBytes each
+    uint8_t* xm_base = pk_base + kPk * SM::kPackedBytes;          // two exponent / microexponent buffers
+    PairBars& bars = *reinterpret_cast<PairBars*>(xm_base + 2 * kXmBytes);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = cluster_ctarank();
     const int64_t m0 = ((int64_t)(blockIdx.x >> 1) * 2 + rank) * kPairRows;  // this CTA's rows of A and C
     const int64_t n0 = (int64_t)blockIdx.y * 256;                             // the pair's columns
     const int64_t nb0 = n0 + (int64_t)rank * kPairRows;                       // this CTA's half of the B tile
-    const int nk = (int)(K / kBK), nchunks = (int)(K / kChunkK);
+    const int nk = (int)(K / kBK), nchunks = (int)(K / kEChunkK);
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < 4; ++s) { mbar_init(&bars.full[s], 2 * kPairDecodeWarps); mbar_init(&bars.empty[s], 1); }
+        for (int s = 0; s < 6; ++s) { mbar_init(&bars.full[s], 2 * kPairDecodeWarps); mbar_init(&bars.empty[s], 1); }
         mbar_init(&bars.accum, 1);
         for (int i = 0; i < kMaxPk; ++i) { mbar_init(&bars.pk_full[i], 1); mbar_init(&bars.pk_empty[i], kPairDecodeWarps); }
         bars.failed = 0;
@@ -216,9 +220,10 @@ mx_gemm_pair_kernel(const __grid_constant__ PairMaps maps, int64_t M, int64_t N,
         const int r = is_a ? row256 : row256 - kPairRows;
         const uint32_t tile_off = (uint32_t)((is_a ? 0 : kPairRows * kBK * 2) + (r >> 3) * 1024 + (r & 7) * 128);
         bool ok;
-        if (is_a) ok = pair_decode_rows<WA>(smem_u32(pk_base), SM::kPackedBytes, kPk, r, half, tile_off, smem_u32(stages), kStages, bars, nk, lane);
-        else ok = pair_decode_rows<WB>(smem_u32(pk_base) + ChunkPlanes<WA>::kBytes, SM::kPackedBytes, kPk, r, half, tile_off,
-                                       smem_u32(stages), kStages, bars, nk, lane);
+        if (is_a) ok = pair_decode_rows<WA>(smem_u32(pk_base), SM::kPackedBytes, smem_u32(xm_base), r, half, tile_off, smem_u32(stages),
+                                            kStages, bars, nk, lane);
+        else ok = pair_decode_rows<WB>(smem_u32(pk_base) + ChunkPlanes<WA>::kBytes, SM::kPackedBytes, smem_u32(xm_base) + 2 * kXmPlane, r,
+                                       half, tile_off, smem_u32(stages), kStages, bars, nk, lane);
         if (!ok) bars.failed = 1;
 
         // ---------------- epilogue: this CTA's 128 x 256 block of C ----------------
@@ -241,7 +246,7 @@ mx_gemm_pair_kernel(const __grid_constant__ PairMaps maps, int64_t M, int64_t N,
         }
         tc_fence_before();
     } else if (warp == kLoaderWarp) {
-        // ---------------- loader: six TMA tile loads per chunk (256 K elements x 128 rows per plane) ----------------
+        // ---------------- loader: TMA tile loads, codes per 128 K elements, exponents per 256 ----------------
         if (lane == 0) {
             bool ok = true;
             for (int ch = 0; ch < nchunks; ++ch) {
@@ -252,13 +257,18 @@ mx_gemm_pair_kernel(const __grid_constant__ PairMaps maps, int64_t M, int64_t N,
                 }
                 uint8_t* pa = pk_base + (size_t)buf * SM::kPackedBytes;
                 uint8_t* pb = pa + ChunkPlanes<WA>::kBytes;
-                mbar_expect_tx(&bars.pk_full[buf], (uint32_t)SM::kPackedBytes);
-                tma_load_2d(pa + ChunkPlanes<WA>::kElems, &maps.a_elems, ch * ChunkPlanes<WA>::kElemRow, (int)m0, &bars.pk_full[buf]);
-                tma_load_2d(pa + ChunkPlanes<WA>::kExps, &maps.a_exps, ch * 16, (int)m0, &bars.pk_full[buf]);
-                tma_load_2d(pa + ChunkPlanes<WA>::kMicro, &maps.a_micro, ch * 16, (int)m0, &bars.pk_full[buf]);
-                tma_load_2d(pb + ChunkPlanes<WB>::kElems, &maps.b_elems, ch * ChunkPlanes<WB>::kElemRow, (int)nb0, &bars.pk_full[buf]);
-                tma_load_2d(pb + ChunkPlanes<WB>::kExps, &maps.b_exps, ch * 16, (int)nb0, &bars.pk_full[buf]);
-                tma_load_2d(pb + ChunkPlanes<WB>::kMicro, &maps.b_micro, ch * 16, (int)nb0, &bars.pk_full[buf]);
+                const bool with_xm = (ch & 1) == 0;  // exponent tiles cover two code chunks and ride on the even one's barrier
+                mbar_expect_tx(&bars.pk_full[buf], (uint32_t)(SM::kPackedBytes + (with_xm ? kXmBytes : 0)));
+                tma_load_2d(pa, &maps.a_elems, ch * ChunkPlanes<WA>::kElemRow, (int)m0, &bars.pk_full[buf]);
+                tma_load_2d(pb, &maps.b_elems, ch * ChunkPlanes<WB>::kElemRow, (int)nb0, &bars.pk_full[buf]);
+                if (with_xm) {
+                    // buffer (ch/2)&1 was last read during code chunk ch-3, which pk_empty above has confirmed done
+                    uint8_t* xm = xm_base + (size_t)((ch >> 1) & 1) * kXmBytes;
+                    tma_load_2d(xm, &maps.a_exps, (ch >> 1) * 16, (int)m0, &bars.pk_full[buf]);
+                    tma_load_2d(xm + kXmPlane, &maps.a_micro, (ch >> 1) * 16, (int)m0, &bars.pk_full[buf]);
+                    tma_load_2d(xm + 2 * kXmPlane, &maps.b_exps, (ch >> 1) * 16, (int)nb0, &bars.pk_full[buf]);
+                    tma_load_2d(xm + 3 * kXmPlane, &maps.b_micro, (ch >> 1) * 16, (int)nb0, &bars.pk_full[buf]);
+                }
             }
             if (!ok) bars.failed = 1;
         }
