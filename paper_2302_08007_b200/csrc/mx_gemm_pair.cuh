@@ -21,7 +21,7 @@ constexpr int kPairRows = 128;                  // rows of A and of the B half p
 constexpr int kChunkK = 256;                    // K elements per exponent / microexponent tile (16 bytes per row)
 constexpr int kEChunkK = 128;                   // K elements per code tile (two K steps): small, so more operand stages fit
 constexpr int kStepsPerEChunk = kEChunkK / kBK; // 2
-constexpr int kPairDecodeWarps = 16;            // two threads per row: each decodes two of the row's four blocks per K step
+constexpr int kPairDecodeWarps = 16;            // two threads per row: one decodes the even K steps, the other the odd ones
 constexpr int kLoaderWarp = 16, kMmaWarp = 17;
 constexpr int kPairThreads = 18 * 32;
 constexpr int kPairStageBytes = 2 * kPairRows * kBK * 2;  // A 16 KB + B half 16 KB
@@ -126,31 +126,25 @@ constexpr uint32_t kPairInstrDesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint3
 // +kXmPlane; buffers are kXmBytes apart).  `half` selects which two of the row's four 16-element
 // blocks of a K step this thread decodes.
 template <int W>
-__device__ __forceinline__ bool pair_decode_rows(uint32_t pk0, uint32_t pk_stride, uint32_t xm0, int r, int half, uint32_t tile_off,
+__device__ __forceinline__ bool pair_decode_rows(uint32_t pk0, uint32_t pk_stride, uint32_t xm0, int r, int group, uint32_t tile_off,
                                                  uint32_t stages_addr, int n_stages, PairBars& bars, int nk, int lane) {
-    constexpr int NW = 2 * kSlice * W / 32;  // code words of two blocks: 3 / 5 / 8
-    for (int kk = 0; kk < nk; ++kk) {
+    constexpr int NW = kBK * W / 32;  // code words of one K step (four blocks): 6 / 10 / 16
+    // Decode group `group` (warps 0-7 or 8-15) takes every second K step, so while one group sits in
+    // its barrier / fence phase the other one is decoding and the SM keeps issuing.
+    for (int kk = group; kk < nk; kk += 2) {
         const int ech = kk / kStepsPerEChunk, ks = kk % kStepsPerEChunk, buf = ech % kMaxPk;
-        if (ks == 0) {
+        {
             bool ok = mbar_wait(&bars.pk_full[buf], (ech / kMaxPk) & 1);
             ok = __all_sync(0xFFFFFFFFu, ok);
             if (!ok) return false;
         }
-        // the two blocks' codes: 4W bytes starting at byte ks*8W + half*4W of the row (4-byte aligned)
-        const uint32_t ebase = pk0 + buf * pk_stride + r * ChunkPlanes<W>::kElemRow + ks * (kBK * W / 8) + half * (4 * W);
-        uint32_t w[NW + 1];
-        if ((4 * W) % 8 == 0) {
+        const uint32_t ebase = pk0 + buf * pk_stride + r * ChunkPlanes<W>::kElemRow + ks * (kBK * W / 8);  // 8-byte aligned
+        uint32_t w[NW];
 #pragma unroll
-            for (int i = 0; i < NW / 2; ++i) { const uint2 v = ld_shared_v2(ebase + 8 * i); w[2 * i] = v.x; w[2 * i + 1] = v.y; }
-        } else {
-#pragma unroll
-            for (int i = 0; i < NW; ++i) w[i] = ld_shared_b32(ebase + 4 * i);
-        }
-        w[NW] = 0;
+        for (int i = 0; i < NW / 2; ++i) { const uint2 v = ld_shared_v2(ebase + 8 * i); w[2 * i] = v.x; w[2 * i + 1] = v.y; }
         // exponent / microexponent bytes of this K step: 4 bytes each within the row's 16 (256 K elements)
         const uint32_t xm = xm0 + ((kk / 4) & 1) * kXmBytes + r * 16 + 4 * (kk & 3);
-        const uint32_t exps2 = (ld_shared_b32(xm) >> (16 * half)) & 0xFFFFu;
-        const uint32_t micro2 = (ld_shared_b32(xm + kXmPlane) >> (16 * half)) & 0xFFFFu;
+        const uint32_t exps4 = ld_shared_b32(xm), micro4 = ld_shared_b32(xm + kXmPlane);
         const int stage = kk % n_stages;
         if (kk >= n_stages) {
             bool ok = mbar_wait(&bars.empty[stage], ((kk / n_stages) - 1) & 1);
@@ -158,23 +152,20 @@ __device__ __forceinline__ bool pair_decode_rows(uint32_t pk0, uint32_t pk_strid
             if (!ok) return false;
         }
         const uint32_t tile = stages_addr + stage * kPairStageBytes + tile_off;
-        constexpr int M = W - 1;
-        const int ea = (int)(exps2 & 0xFFu) - (M - 1), eb = (int)(exps2 >> 8) - (M - 1);
-        const bool safe = __all_sync(0xFFFFFFFFu, ea >= 2 && ea <= 247 && eb >= 2 && eb <= 247);  // warp-uniform decoder choice
+        const bool safe = __all_sync(0xFFFFFFFFu, exps_safe<W>(exps4));  // warp-uniform decoder choice
 #pragma unroll
-        for (int bb = 0; bb < 2; ++bb) {
+        for (int bb = 0; bb < kBK / kSlice; ++bb) {
             uint32_t o[8];
-            if (safe) decode_block_bf16<W, NW + 1, true>(w, bb * kSlice * W, (exps2 >> (8 * bb)) & 0xFFu, (micro2 >> (8 * bb)) & 0xFFu, o);
-            else decode_block_bf16<W, NW + 1, false>(w, bb * kSlice * W, (exps2 >> (8 * bb)) & 0xFFu, (micro2 >> (8 * bb)) & 0xFFu, o);
-            const int chunk16 = 2 * (2 * half + bb);  // 16-byte chunk of the block's first 8 elements within the 128-byte row
-            st_shared_v4(tile + ((chunk16 ^ (r & 7)) << 4), o[0], o[1], o[2], o[3]);
-            st_shared_v4(tile + (((chunk16 + 1) ^ (r & 7)) << 4), o[4], o[5], o[6], o[7]);
+            if (safe) decode_block_bf16<W, NW, true>(w, bb * kSlice * W, (exps4 >> (8 * bb)) & 0xFFu, (micro4 >> (8 * bb)) & 0xFFu, o);
+            else decode_block_bf16<W, NW, false>(w, bb * kSlice * W, (exps4 >> (8 * bb)) & 0xFFu, (micro4 >> (8 * bb)) & 0xFFu, o);
+            st_shared_v4(tile + (((2 * bb) ^ (r & 7)) << 4), o[0], o[1], o[2], o[3]);
+            st_shared_v4(tile + (((2 * bb + 1) ^ (r & 7)) << 4), o[4], o[5], o[6], o[7]);
         }
         fence_proxy_async();  // generic-proxy stores -> visible to the tensor core's (async proxy) reads
         __syncwarp();
         if (lane == 0) {
-            mbar_arrive_cluster(&bars.full[stage], 0);                            // the leader CTA counts both CTAs' decoders
-            if (ks == kStepsPerEChunk - 1) mbar_arrive(&bars.pk_empty[buf]);      // this warp is done with the code buffer
+            mbar_arrive_cluster(&bars.full[stage], 0);   // the leader CTA counts both CTAs' decoders
+            mbar_arrive(&bars.pk_empty[buf]);            // each warp reads a code chunk once (its K step of the two)
         }
     }
     return true;
@@ -199,7 +190,7 @@ mx_gemm_pair_kernel(const __grid_constant__ PairMaps maps, int64_t M, int64_t N,
     const int nk = (int)(K / kBK), nchunks = (int)(K / kEChunkK);
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < 6; ++s) { mbar_init(&bars.full[s], 2 * kPairDecodeWarps); mbar_init(&bars.empty[s], 1); }
+        for (int s = 0; s < 6; ++s) { mbar_init(&bars.full[s], kPairDecodeWarps); mbar_init(&bars.empty[s], 1); }  // 8 warps x 2 CTAs per K step
         mbar_init(&bars.accum, 1);
         for (int i = 0; i < kMaxPk; ++i) { mbar_init(&bars.pk_full[i], 1); mbar_init(&bars.pk_empty[i], kPairDecodeWarps); }
         bars.failed = 0;
@@ -214,7 +205,7 @@ mx_gemm_pair_kernel(const __grid_constant__ PairMaps maps, int64_t M, int64_t N,
 
     if (warp < kPairDecodeWarps) {
         // ---------------- decoders: threads t and t+256 share row t (A rows 0-127, then the B half's 128 rows) ----------------
-        const int half = warp >> 3;                 // warps 0-7: blocks 0,1 of each K step; warps 8-15: blocks 2,3
+        const int half = warp >> 3;                 // warps 0-7: even K steps; warps 8-15: odd K steps
         const int row256 = (int)threadIdx.x & 255;  // consecutive lanes hold consecutive rows (conflict-free swizzled stores)
         const bool is_a = row256 < kPairRows;
         const int r = is_a ? row256 : row256 - kPairRows;
