@@ -21,9 +21,12 @@ constexpr int kPairRows = 128;                  // rows of A and of the B half p
 constexpr int kChunkK = 256;                    // K elements per exponent / microexponent tile (16 bytes per row)
 constexpr int kEChunkK = 128;                   // K elements per code tile (two K steps): small, so more operand stages fit
 constexpr int kStepsPerEChunk = kEChunkK / kBK; // 2
-constexpr int kPairDecodeWarps = 16;            // two threads per row: one decodes the even K steps, the other the odd ones
-constexpr int kLoaderWarp = 16, kMmaWarp = 17;
-constexpr int kPairThreads = 18 * 32;
+constexpr int kDecodeGroups = 2;                // decode groups of 8 warps (one thread per row); group g takes K steps g, g+2, ...
+constexpr int kGroupWarps = 2 * kPairRows / 32; // 8
+constexpr int kPairDecodeWarps = kDecodeGroups * kGroupWarps;
+constexpr int kEpilogueWarps2 = 16;             // warps that drain the accumulator (4 lane groups x 4 column quarters)
+constexpr int kLoaderWarp = kPairDecodeWarps, kMmaWarp = kPairDecodeWarps + 1;
+constexpr int kPairThreads = (kPairDecodeWarps + 2) * 32;
 constexpr int kPairStageBytes = 2 * kPairRows * kBK * 2;  // A 16 KB + B half 16 KB
 
 // Packed bytes as the TMA writes them, dense row-major, for the 128 rows of one operand:
@@ -129,9 +132,9 @@ template <int W>
 __device__ __forceinline__ bool pair_decode_rows(uint32_t pk0, uint32_t pk_stride, uint32_t xm0, int r, int group, uint32_t tile_off,
                                                  uint32_t stages_addr, int n_stages, PairBars& bars, int nk, int lane) {
     constexpr int NW = kBK * W / 32;  // code words of one K step (four blocks): 6 / 10 / 16
-    // Decode group `group` (warps 0-7 or 8-15) takes every second K step, so while one group sits in
-    // its barrier / fence phase the other one is decoding and the SM keeps issuing.
-    for (int kk = group; kk < nk; kk += 2) {
+    // Decode group `group` takes every kDecodeGroups-th K step, so while one group sits in its
+    // barrier / fence phase the others are decoding and the SM keeps issuing.
+    for (int kk = group; kk < nk; kk += kDecodeGroups) {
         const int ech = kk / kStepsPerEChunk, ks = kk % kStepsPerEChunk, buf = ech % kMaxPk;
         {
             bool ok = mbar_wait(&bars.pk_full[buf], (ech / kMaxPk) & 1);
@@ -190,9 +193,9 @@ mx_gemm_pair_kernel(const __grid_constant__ PairMaps maps, int64_t M, int64_t N,
     const int nk = (int)(K / kBK), nchunks = (int)(K / kEChunkK);
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < 6; ++s) { mbar_init(&bars.full[s], kPairDecodeWarps); mbar_init(&bars.empty[s], 1); }  // 8 warps x 2 CTAs per K step
+        for (int s = 0; s < 6; ++s) { mbar_init(&bars.full[s], 2 * kGroupWarps); mbar_init(&bars.empty[s], 1); }  // 8 warps x 2 CTAs per K step
         mbar_init(&bars.accum, 1);
-        for (int i = 0; i < kMaxPk; ++i) { mbar_init(&bars.pk_full[i], 1); mbar_init(&bars.pk_empty[i], kPairDecodeWarps); }
+        for (int i = 0; i < kMaxPk; ++i) { mbar_init(&bars.pk_full[i], 1); mbar_init(&bars.pk_empty[i], kStepsPerEChunk * kGroupWarps); }  // each K step of the chunk is read by one group
         bars.failed = 0;
         fence_barrier_init();
     }
@@ -205,7 +208,7 @@ mx_gemm_pair_kernel(const __grid_constant__ PairMaps maps, int64_t M, int64_t N,
 
     if (warp < kPairDecodeWarps) {
         // ---------------- decoders: threads t and t+256 share row t (A rows 0-127, then the B half's 128 rows) ----------------
-        const int half = warp >> 3;                 // warps 0-7: even K steps; warps 8-15: odd K steps
+        const int half = warp / kGroupWarps;        // decode group
         const int row256 = (int)threadIdx.x & 255;  // consecutive lanes hold consecutive rows (conflict-free swizzled stores)
         const bool is_a = row256 < kPairRows;
         const int r = is_a ? row256 : row256 - kPairRows;
@@ -218,9 +221,11 @@ mx_gemm_pair_kernel(const __grid_constant__ PairMaps maps, int64_t M, int64_t N,
         if (!ok) bars.failed = 1;
 
         // ---------------- epilogue: this CTA's 128 x 256 block of C ----------------
-        bool done = ok && mbar_wait(&bars.accum, 0);
+        bool done = ok && warp < kEpilogueWarps2 && mbar_wait(&bars.accum, 0);
         done = __all_sync(0xFFFFFFFFu, done);
-        if (done) {
+        if (warp >= kEpilogueWarps2) {
+            // the remaining decode warps have no accumulator lanes to drain
+        } else if (done) {
             tc_fence_after();
             const int lane_base = (warp & 3) * 32, col_base = (warp >> 2) * 64;  // 16 warps: 4 lane groups x 4 column quarters
             float* crow = c + (m0 + lane_base + lane) * ldc + n0 + col_base;
