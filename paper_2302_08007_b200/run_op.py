@@ -13,9 +13,47 @@ from . import synth
 FORMATS = {"MX4": bdr.MX4, "MX6": bdr.MX6, "MX9": bdr.MX9}
 
 
+def _timed(fn, reps):
+    fn()
+    torch.cuda.synchronize()
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+    ev[0].record()
+    for _ in range(reps):
+        fn()
+    ev[1].record()
+    torch.cuda.synchronize()
+    return ev[0].elapsed_time(ev[1]) / reps
+
+
+def run_gemm(a, cfg):
+    """C[rows, rows] = A[rows, cols] * B[rows, cols]^T with both operands packed in --fmt along K = cols."""
+    M = N = a.rows
+    K = a.cols
+    A = torch.from_numpy(synth.normal_matrix(M, K, seed=0, stream=10)).cuda()
+    B = torch.from_numpy(synth.normal_matrix(N, K, seed=0, stream=11, sigma=0.02)).cuda()
+    pa, pb = bdr.alloc_planes(cfg, M, K), bdr.alloc_planes(cfg, N, K)
+    bdr.bdr_pack(cfg, A, pa)
+    bdr.bdr_pack(cfg, B, pb)
+    c = torch.empty((M, N), dtype=torch.float32, device="cuda")
+    ms = _timed(lambda: bdr.mx_gemm(cfg, pa, cfg, pb, M, N, K, c), a.reps)
+    print("mx_gemm %s %dx%dx%d: %.4f ms per launch, %.1f TFLOP/s, status %d" % (
+        a.fmt, M, N, K, ms, 2.0 * M * N * K / ms / 1e9, bdr.mx_gemm_status()))
+
+
+def run_sweep(a):
+    """The 457-configuration QSNR sweep over rows*cols fp32 values ~ N(0,1) (one row)."""
+    from . import sweep
+    cfgs = [c for _, c in sweep.sweep_configs()]
+    x = torch.from_numpy(synth.normal(a.rows * a.cols, seed=0)).cuda().reshape(1, -1)
+    out = torch.empty(len(cfgs), dtype=torch.float64, device="cuda")
+    ws = torch.empty(bdr.bdr_qsnr_workspace_bytes(len(cfgs)), dtype=torch.uint8, device="cuda")
+    ms = _timed(lambda: bdr.bdr_qsnr(cfgs, x, out, ws), a.reps)
+    print("bdr_qsnr %d configs x %d values: %.4f ms per call, %.0f configs/s" % (len(cfgs), x.numel(), ms, len(cfgs) / ms * 1e3))
+
+
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--op", default="pack", choices=["quant_dequant", "pack", "unpack"])
+    ap.add_argument("--op", default="pack", choices=["quant_dequant", "pack", "unpack", "gemm", "sweep"])
     ap.add_argument("--fmt", default="MX6", choices=list(FORMATS))
     ap.add_argument("--axis", type=int, default=1)
     ap.add_argument("--dtype", default="bf16", choices=["bf16", "f32"])
@@ -26,6 +64,10 @@ def main():
     ap.add_argument("--no-y", action="store_true", help="quant_dequant: only the QSNR sums")
     a = ap.parse_args()
     cfg = FORMATS[a.fmt]
+    if a.op == "gemm":
+        return run_gemm(a, cfg)
+    if a.op == "sweep":
+        return run_sweep(a)
     x = torch.from_numpy(synth.outlier_channel_matrix(a.rows, a.cols, seed=0, stream=3)).cuda()
     if a.dtype == "bf16":
         x = x.to(torch.bfloat16)
