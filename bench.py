@@ -31,9 +31,21 @@ FORMATS = (("MX4", 2), ("MX6", 4), ("MX9", 7))  # name, m  (k1=16, d1=8, k2=2, d
 METRIC = "MX quant-dequant GB/s"
 FALLBACK_HBM_GBS = 6650.0
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch from the committed ncu captures
-# (profiles/*.md), scaled to the 8192 x 8192 launch; None where no capture exists yet.
-NCU_TRAFFIC_BYTES: dict[str, float | None] = {}
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch of each of the step's kernels on the
+# bench workload itself (8192 x 8192 bf16), from the committed ncu capture
+# profiles/step_kernels_dram_traffic.md.  Writes that still sit in L2 when a kernel ends are not
+# counted by those counters, which is why some figures are below the algorithmic bytes.
+NCU_TRAFFIC_BYTES: dict[str, float | None] = {
+    "quant_dequant_MX4_row": 217688576, "quant_dequant_MX4_col": 221876480,
+    "quant_dequant_MX6_row": 216988160, "quant_dequant_MX6_col": 221636352,
+    "quant_dequant_MX9_row": 216802304, "quant_dequant_MX9_col": 222077952,
+    "pack_MX4_row": 150532096, "pack_MX4_col": 148491520,
+    "pack_MX6_row": 159283968, "pack_MX6_col": 157008640,
+    "pack_MX9_row": 173592832, "pack_MX9_col": 172875264,
+    "unpack_MX4_row": 108700416, "unpack_MX4_col": 107778816,
+    "unpack_MX6_row": 125882112, "unpack_MX6_col": 124492032,
+    "unpack_MX9_row": 153894656, "unpack_MX9_col": 150398976,
+}
 
 
 def bits_per_element(m: int) -> float:
