@@ -71,11 +71,19 @@ typedef enum {
     BDR_ERR_SIZE = -5,        /* negative size, ld < cols, size over the stated maximum               */
     BDR_ERR_WORKSPACE = -6,   /* workspace missing or too small                                       */
     BDR_ERR_CUDA = -7,        /* a CUDA call or kernel launch failed                                  */
-    BDR_ERR_TIMEOUT = -8      /* a bounded device-side wait ran out (reported by mx_gemm_status)      */
+    BDR_ERR_TIMEOUT = -8      /* a bounded device-side wait ran out (see bdr_device_status, mx_gemm_status) */
 } bdr_status_t;
 
 /* Text for a status code (host; never NULL). */
 const char* bdr_strerror(int status);
+
+/* Kernels that stage data with asynchronous bulk copies wait for them with a bounded number of
+ * polls.  A wait that runs out makes the warp stop early (its part of the output is then
+ * incomplete) and leaves BDR_ERR_TIMEOUT in a sticky per-device word.  This host call returns
+ * that word for the current device: BDR_OK, BDR_ERR_TIMEOUT, or BDR_ERR_CUDA if it cannot be read.
+ * It synchronises with the device (one word is copied back), so call it after the work of
+ * interest, not between launches. */
+int bdr_device_status(void);
 
 /* Section III bits-per-element formula realised as plane sizes (host only).  ld_out / bytes_out
  * (host arrays of 3: exps, micro, elems) receive the default line pitches (rounded up to 16 bytes)

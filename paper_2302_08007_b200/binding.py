@@ -19,7 +19,7 @@ SCALE_POW2, SCALE_FP32_INT, SCALE_FP32_FP, SCALE_FP32_VSQ = 0, 1, 2, 3
 ROUND_NEAREST_EVEN, ROUND_NEAREST_AWAY = 0, 1
 F32, BF16 = 0, 1
 
-EXPORTS = ("bdr_strerror", "bdr_packed_sizes", "bdr_quant_dequant", "bdr_pack", "bdr_unpack",
+EXPORTS = ("bdr_strerror", "bdr_device_status", "bdr_packed_sizes", "bdr_quant_dequant", "bdr_pack", "bdr_unpack",
            "bdr_qsnr_workspace_bytes", "bdr_qsnr", "bdr_qsnr_static_max_cfgs", "bdr_qsnr_static", "mx_gemm",
            "mx_gemm_status")
 
@@ -105,6 +105,8 @@ def lib():
                                       C.c_void_p, C.c_void_p]
         L.mx_gemm_status.restype = C.c_int
         L.mx_gemm_status.argtypes = []
+        L.bdr_device_status.restype = C.c_int
+        L.bdr_device_status.argtypes = []
         for fn in (L.bdr_packed_sizes, L.bdr_quant_dequant, L.bdr_pack, L.bdr_unpack, L.bdr_qsnr, L.mx_gemm):
             fn.restype = C.c_int
         _lib = L
@@ -231,6 +233,11 @@ def mx_gemm(cfg_a: Config, a: Planes, cfg_b: Config, b: Planes, M: int, N: int, 
     _check(lib().mx_gemm(C.addressof(ca), C.addressof(pa), C.addressof(cb), C.addressof(pb), M, N, K, _ptr(c),
                          c.stride(0), _stream(stream)), "mx_gemm")
     return c
+
+
+def bdr_device_status() -> int:
+    """Sticky per-device status of the kernels' bounded waits (0 = ok); synchronises."""
+    return int(lib().bdr_device_status())
 
 
 def mx_gemm_status() -> int:

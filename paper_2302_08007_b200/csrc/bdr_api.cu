@@ -1,10 +1,29 @@
 // C-ABI entry points: argument validation on the host, then dispatch to the kernels.
 #include <mutex>
 
+#include <type_traits>
+
+#include "bdr_async.cuh"
 #include "bdr_device.cuh"
 #include "bdr_host.h"
 
 namespace bdr {
+
+__device__ int g_device_status = 0;  // sticky: the first bounded wait that runs out leaves BDR_ERR_TIMEOUT here
+
+int* device_status_word() {
+    static int* cached[64];
+    static std::mutex mu;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    std::lock_guard<std::mutex> lock(mu);
+    if (!cached[dev]) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_device_status) != cudaSuccess) return nullptr;
+        cached[dev] = static_cast<int*>(p);
+    }
+    return cached[dev];
+}
 
 int sm_count() {
     static int cached[64];
@@ -80,6 +99,11 @@ static int quant_dispatch(const QParams& qp, const T* x, T* y, int64_t rows, int
     if (rows == 0 || cols == 0) return BDR_OK;
     int rc = BDR_ERR_UNSUPPORTED;
     if (axis == 1) {
+        if constexpr (std::is_same<T, __nv_bfloat16>::value) {
+            if (out) { if (tight) rc = pack_rowwise_mx_x2(x, y, rows, cols, ld, *out, qp, sums, st); }
+            else rc = quant_rowwise_mx_x2(x, y, rows, cols, ld, qp, sums, st);
+            if (rc != BDR_ERR_UNSUPPORTED) return rc;
+        }
         if (out) { if (tight) rc = pack_rowwise_mx<T>(x, y, rows, cols, ld, *out, qp, sums, st); }
         else rc = quant_rowwise<T>(x, y, rows, cols, ld, qp, sums, st);
     } else {
@@ -108,6 +132,13 @@ const char* bdr_strerror(int status) {
         case BDR_ERR_TIMEOUT: return "bounded device-side wait ran out";
     }
     return "unknown status";
+}
+
+int bdr_device_status(void) {
+    int* word = device_status_word();
+    int v = 0;
+    if (!word || cudaMemcpy(&v, word, sizeof(v), cudaMemcpyDeviceToHost) != cudaSuccess) return BDR_ERR_CUDA;
+    return v;
 }
 
 int bdr_packed_sizes(const bdr_config_t* cfg, int64_t rows, int64_t cols, int axis, int64_t ld_out[3],

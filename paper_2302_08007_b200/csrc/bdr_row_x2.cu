@@ -1,0 +1,296 @@
+// Row-direction (axis 1) kernels for bf16 tensors in the Table II family (k1 = 16, k2 = 2, d2 = 1,
+// m <= 7, ties-to-even), built on the packed bf16x2 quantizer: two elements per instruction, so the
+// kernels stay bound by HBM rather than by instruction issue.  Thread mapping, prefetch ring and
+// coalesced stores are those of the generic row kernels: a lane owns two adjacent 16-element blocks
+// (64 bytes) of a warp's contiguous 2 KB run per iteration.
+#include "bdr_async.cuh"
+#include "bdr_x2.cuh"
+#include "bdr_host.h"
+
+namespace bdr {
+
+using bf16 = __nv_bfloat16;
+constexpr int kX2SPT = 2;
+
+__device__ __forceinline__ double pow4_weight(uint32_t F) {  // 2^(2F-254)
+    return __hiloint2double((int)((F << 21) + 0x30100000u), 0);
+}
+
+__device__ __forceinline__ void words_of(const uint4& v0, const uint4& v1, uint32_t (&w)[8]) {
+    w[0] = v0.x; w[1] = v0.y; w[2] = v0.z; w[3] = v0.w;
+    w[4] = v1.x; w[5] = v1.y; w[6] = v1.z; w[7] = v1.w;
+}
+
+// Per-warp pipeline.  A warp streams runs of 2048 elements (4 KB) through two stages in shared memory:
+// lane 0 refills a stage with one bulk copy as soon as the warp has consumed it, so two runs per warp
+// (and with ~20 warps per SM well over 100 KB per SM) are in flight.  A run is handled as two halves
+// of 1024 elements; in each a lane owns 64 consecutive bytes (two blocks).  Dequantized values go
+// straight from registers to global memory (one 32-byte store per block); the packed planes of a
+// run are collected per warp in a small double-buffered staging area and leave with one bulk store
+// each (256 W code bytes, 128 exponent bytes, 128 microexponent bytes).
+constexpr int kX2Threads = 128;
+constexpr int kX2Warps = kX2Threads / 32;
+constexpr int kX2Stages = 2;
+constexpr int kX2Sub = 2;                                    // halves per run
+constexpr int kSubElems = 32 * kX2SPT * kSlice;              // 1024
+constexpr int kX2RunElems = kX2Sub * kSubElems;              // 2048
+constexpr int kRunBytes = kX2RunElems * 2;
+constexpr int kX2RingBytes = kX2Warps * kX2Stages * kRunBytes;
+constexpr int kX2BarBytes = 128;  // kX2Warps * kX2Stages barriers of 8 bytes, padded
+static_assert(kX2Warps * kX2Stages * 8 <= kX2BarBytes, "barrier area");
+
+template <int W> struct X2PackStage {
+    static constexpr int kElemBytes = kX2RunElems / 8 * W;
+    static constexpr int kExpBytes = kX2RunElems / 16;
+    static constexpr int kMicroBytes = kX2RunElems / 16;
+    static constexpr int kBytes = W > 0 ? kElemBytes + kExpBytes + kMicroBytes : 0;  // a multiple of 128
+};
+
+// Where run `wi` starts.  A contiguous tensor is one long row (flat); otherwise a row holds
+// runs_per_row runs and rows are ld elements apart.
+struct RunIndex {
+    FastDiv runs_per_row;
+    int64_t ld;
+    int flat;
+    __device__ __forceinline__ void split(uint32_t wi, int64_t& row, int64_t& pos) const {
+        if (flat) {
+            row = 0;
+            pos = wi;
+        } else {
+            const uint32_t r = fastdiv(wi, runs_per_row);
+            row = r;
+            pos = wi - r * runs_per_row.d;
+        }
+    }
+    __device__ __forceinline__ int64_t elem_offset(uint32_t wi) const {
+        int64_t row, pos;
+        split(wi, row, pos);
+        return row * ld + pos * kX2RunElems;
+    }
+};
+
+__device__ __forceinline__ void stg256(void* p, const uint32_t (&v)[8]) {
+    asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(p), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]),
+                 "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7])
+                 : "memory");
+}
+
+// W = 0: quantize-dequantize (any m <= 7, from qp); W = m + 1: also write the packed planes.
+template <int W, bool SUMS, bool YOUT>
+__global__ void __launch_bounds__(kX2Threads)
+row_mx_x2_kernel(const bf16* x, bf16* y, RunIndex ri, uint32_t total, bdr_planes_t out, QParams qp, double* sums, int* status) {
+    using PS = X2PackStage<W>;
+    constexpr bool PACK = W > 0;
+    constexpr bool kPackOnly = PACK && !SUMS && !YOUT;
+    constexpr int S = kX2Stages;
+    constexpr int NCW = PACK ? (16 * W + 31) / 32 : 1;  // words of one block's codes (the last one half full when W is odd)
+    extern __shared__ __align__(128) uint8_t smem[];  // ring [warp][stage][4 KB], barriers, staging [warp][2]
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const uint32_t ring0 = async::smem_u32(smem) + warp * S * kRunBytes;
+    const uint32_t bars = async::smem_u32(smem) + kX2RingBytes + warp * S * 8;
+    const uint32_t stage0 = async::smem_u32(smem) + kX2RingBytes + kX2BarBytes + warp * 2 * PS::kBytes;
+    const int m = PACK ? W - 1 : qp.m;
+    const x2::Consts k = x2::make_consts(m);
+    const uint32_t stride = gridDim.x * kX2Warps;
+    const uint32_t w0 = blockIdx.x * kX2Warps + warp;
+    if (lane == 0) {
+#pragma unroll
+        for (int s = 0; s < S; ++s) async::mbar_init(bars + 8 * s, 1);
+        async::fence_barrier_init();
+#pragma unroll
+        for (int s = 0; s < S; ++s) {
+            const uint32_t wi = w0 + s * stride;
+            if (wi < total) {
+                async::mbar_expect_tx(bars + 8 * s, kRunBytes);
+                async::bulk_load(ring0 + s * kRunBytes, x + ri.elem_offset(wi), kRunBytes, bars + 8 * s);
+            }
+        }
+    }
+    int st = 0;
+    uint32_t phase = 0, half = 0;
+    double e2 = 0.0, s2 = 0.0;
+    for (uint32_t wi = w0; wi < total; wi += stride) {
+        __syncwarp();  // lane 0 has finished the previous iteration's hand-over (staging half is free)
+        if (!async::mbar_wait(bars + 8 * st, phase)) {
+            async::report_timeout(status);
+            break;
+        }
+        const uint32_t stage = stage0 + half * PS::kBytes;
+        bf16* yrun = nullptr;
+        if constexpr (YOUT) yrun = y + ri.elem_offset(wi) + lane * 32;
+#pragma unroll
+        for (int sub = 0; sub < kX2Sub; ++sub) {
+            const uint32_t mine = ring0 + st * kRunBytes + sub * (kSubElems * 2) + lane * 64;
+            uint32_t cw[kX2SPT][NCW], Fs[kX2SPT], mbs[kX2SPT];
+#pragma unroll
+            for (int s = 0; s < kX2SPT; ++s) {
+                const uint4 v0 = async::lds128(mine + 32 * s), v1 = async::lds128(mine + 32 * s + 16);
+                uint32_t w[8], yw[8];
+                words_of(v0, v1, w);
+                x2::PairView pv;
+                uint32_t aw[8], F;
+                if constexpr (kPackOnly) {
+                    F = x2::pair_view(w, pv);
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) aw[j] = x2::habs2(w[j]);
+                    F = x2::block_exponent(aw);
+                }
+                if (F - x2::kMinF <= (uint32_t)(x2::kMaxF - x2::kMinF)) {
+                    if constexpr (kPackOnly) {
+                        x2::pack_pair_view<PACK ? W : 8>(pv, F, cw[s], mbs[s]);
+                        Fs[s] = F;
+                    } else {
+                        float pe = 0.f, ps = 0.f;
+                        uint32_t code2[8];
+                        x2::quantize_block_row<SUMS, YOUT, PACK>(w, aw, F, m, k, yw, code2, mbs[s], pe, ps);
+                        if constexpr (PACK) {
+                            x2::pack_block<PACK ? W : 8>(code2, cw[s]);
+                            Fs[s] = F;
+                        }
+                        if constexpr (SUMS) {
+                            const double wgt = pow4_weight(F);
+                            e2 = fma((double)pe, wgt, e2);
+                            s2 = fma((double)ps, wgt, s2);
+                        }
+                    }
+                } else {
+                    const x2::SlowOut o = x2::quantize_block_slow<W, SUMS>(v0, v1, qp);
+                    if constexpr (PACK) {
+#pragma unroll
+                        for (int i = 0; i < NCW; ++i) cw[s][i] = o.cw[i];
+                        Fs[s] = o.F;
+                        mbs[s] = o.micro;
+                    }
+                    if constexpr (SUMS) { e2 += o.e2; s2 += o.s2; }
+                    if constexpr (YOUT) {
+                        yw[0] = o.y[0].x; yw[1] = o.y[0].y; yw[2] = o.y[0].z; yw[3] = o.y[0].w;
+                        yw[4] = o.y[1].x; yw[5] = o.y[1].y; yw[6] = o.y[1].z; yw[7] = o.y[1].w;
+                    }
+                }
+                if constexpr (YOUT) stg256(yrun + sub * kSubElems + 16 * s, yw);
+            }
+            if constexpr (PACK) {
+                // the lane's 32 codes as W words: block 1 follows block 0 at bit 16 W
+                const uint32_t dst = stage + sub * (kSubElems / 8 * W) + lane * 4 * W;
+                if constexpr (W == 8) {
+                    async::sts128(dst, make_uint4(cw[0][0], cw[0][1], cw[0][2], cw[0][3]));
+                    async::sts128(dst + 16, make_uint4(cw[1][0], cw[1][1], cw[1][2], cw[1][3]));
+                } else {
+#pragma unroll
+                    for (int i = 0; i < W / 2; ++i) async::sts32(dst + 4 * i, cw[0][i]);
+                    async::sts32(dst + 4 * (W / 2), cw[0][W / 2] | (cw[1][0] << 16));
+#pragma unroll
+                    for (int i = 0; i < W / 2; ++i) async::sts32(dst + 4 * (W / 2 + 1 + i), __byte_perm(cw[1][i], cw[1][i + 1], 0x5432));
+                }
+                async::sts16(stage + PS::kElemBytes + sub * (kSubElems / 16) + 2 * lane, Fs[0] | (Fs[1] << 8));
+                async::sts16(stage + PS::kElemBytes + PS::kExpBytes + sub * (kSubElems / 16) + 2 * lane, mbs[0] | (mbs[1] << 8));
+            }
+        }
+        if constexpr (PACK) async::fence_proxy_async();
+        __syncwarp();  // every lane has consumed stage st (and filled the staging half)
+        if (lane == 0) {
+            if constexpr (PACK) {
+                int64_t row, pos;
+                ri.split(wi, row, pos);
+                const int64_t blk0 = pos * (kX2RunElems / 16);  // first block of the run within its row
+                async::bulk_store(out.elems + row * out.ld_elems + blk0 * 2 * W, stage, PS::kElemBytes);
+                async::bulk_store(out.exps + row * out.ld_exps + blk0, stage + PS::kElemBytes, PS::kExpBytes);
+                async::bulk_store(out.micro + row * out.ld_micro + blk0, stage + PS::kElemBytes + PS::kExpBytes, PS::kMicroBytes);
+                async::bulk_commit();
+                async::bulk_wait_read<1>();  // the other staging half (used next) has been read out
+            }
+            const uint32_t next = wi + S * stride;
+            if (next < total) {
+                async::mbar_expect_tx(bars + 8 * st, kRunBytes);
+                async::bulk_load(ring0 + st * kRunBytes, x + ri.elem_offset(next), kRunBytes, bars + 8 * st);
+            }
+        }
+        half ^= 1;
+        if (++st == S) { st = 0; phase ^= 1; }
+    }
+    if (PACK && lane == 0) async::bulk_wait_all();
+    if (SUMS) block_accumulate_sums(e2, s2, sums);
+}
+
+// ---- host launchers --------------------------------------------------------------------------------
+static bool x2_config(const QParams& qp) {
+    return qp.k1 == 16 && qp.k2 == 2 && qp.d2 == 1 && qp.m <= 7 && qp.rounding == BDR_ROUND_NEAREST_EVEN;
+}
+
+// One wave of resident CTAs: every warp then streams many runs through its prefetch ring instead of
+// paying the ring's start-up again in a second, partly filled wave.
+template <typename K>
+static int x2_grid(K kern, size_t smem, int64_t total_warps, int& blocks_per_sm) {
+    if (blocks_per_sm == 0) {
+        int n = 0;
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, kern, kX2Threads, smem) != cudaSuccess || n < 1) n = 2;
+        blocks_per_sm = n;
+    }
+    const int64_t need = (total_warps + kX2Threads / 32 - 1) / (kX2Threads / 32);
+    return (int)max((int64_t)1, min(need, (int64_t)sm_count() * blocks_per_sm));
+}
+
+template <int W, bool SUMS, bool YOUT>
+static int launch_x2(const bf16* x, bf16* y, int64_t rows, int64_t cols, int64_t ld, const bdr_planes_t* out, const QParams& qp,
+                     double* sums, cudaStream_t st) {
+    const int64_t rpr = cols / kX2RunElems, total = rows * rpr;
+    if (total == 0) return BDR_OK;
+    if (total >= (1ll << 31) - (1ll << 24)) return BDR_ERR_UNSUPPORTED;  // 32-bit run indices (incl. look-ahead)
+    auto kern = row_mx_x2_kernel<W, SUMS, YOUT>;
+    const size_t smem = kX2RingBytes + kX2BarBytes + kX2Warps * 2 * X2PackStage<W>::kBytes;
+    static bool attr_done = false;  // per instantiation; the attribute is idempotent, so a race is harmless
+    if (!attr_done) {
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return BDR_ERR_CUDA;
+        attr_done = true;
+    }
+    int* status = device_status_word();
+    if (!status) return BDR_ERR_CUDA;
+    static int blocks_per_sm = 0;
+    bdr_planes_t pl = {};
+    if (out) pl = *out;
+    const RunIndex ri{make_fastdiv((uint32_t)rpr), ld, rows == 1 ? 1 : 0};
+    kern<<<x2_grid(kern, smem, total, blocks_per_sm), kX2Threads, smem, st>>>(x, y, ri, (uint32_t)total, pl, qp, sums, status);
+    return cudaGetLastError() == cudaSuccess ? BDR_OK : BDR_ERR_CUDA;
+}
+
+template <int W>
+static int x2_flags(const bf16* x, bf16* y, int64_t rows, int64_t cols, int64_t ld, const bdr_planes_t* out, const QParams& qp,
+                    double* sums, cudaStream_t st) {
+    if (sums) return y ? launch_x2<W, true, true>(x, y, rows, cols, ld, out, qp, sums, st)
+                       : launch_x2<W, true, false>(x, y, rows, cols, ld, out, qp, sums, st);
+    if (y) return launch_x2<W, false, true>(x, y, rows, cols, ld, out, qp, sums, st);
+    if constexpr (W > 0) return launch_x2<W, false, false>(x, y, rows, cols, ld, out, qp, sums, st);
+    return BDR_ERR_NULL;
+}
+
+// Shapes: whole 2048-element runs, 16-byte aligned (a contiguous tensor counts as one long row).
+static bool x2_shape(const void* x, const void* y, int64_t& rows, int64_t& cols, int64_t& ld) {
+    if ((((uintptr_t)x | (uintptr_t)y) % 32) || (ld * 2) % 32) return false;
+    if (ld == cols && cols % 16 == 0) {
+        cols *= rows;
+        ld = cols;
+        rows = 1;
+    }
+    return cols % kX2RunElems == 0;
+}
+
+int quant_rowwise_mx_x2(const bf16* x, bf16* y, int64_t rows, int64_t cols, int64_t ld, const QParams& qp, double* sums,
+                        cudaStream_t st) {
+    if (!x2_config(qp) || !x2_shape(x, y, rows, cols, ld)) return BDR_ERR_UNSUPPORTED;
+    return x2_flags<0>(x, y, rows, cols, ld, nullptr, qp, sums, st);
+}
+
+// The caller guarantees tight planes (line pitch = the line's natural bytes).
+int pack_rowwise_mx_x2(const bf16* x, bf16* y, int64_t rows, int64_t cols, int64_t ld, const bdr_planes_t& out,
+                       const QParams& qp, double* sums, cudaStream_t st) {
+    if (!x2_config(qp) || !x2_shape(x, y, rows, cols, ld)) return BDR_ERR_UNSUPPORTED;
+    switch (qp.m) {
+        case 2: return x2_flags<3>(x, y, rows, cols, ld, &out, qp, sums, st);
+        case 4: return x2_flags<5>(x, y, rows, cols, ld, &out, qp, sums, st);
+        case 7: return x2_flags<8>(x, y, rows, cols, ld, &out, qp, sums, st);
+    }
+    return BDR_ERR_UNSUPPORTED;
+}
+
+}  // namespace bdr

@@ -1,0 +1,290 @@
+// Packed bf16x2 arithmetic for the Table II family (k1 = 16, k2 = 2, d2 = 1, m <= 7) on bf16 tensors.
+//
+// A bf16 tensor arrives as 32-bit words that hold two elements each.  Everything the quantizer of
+// the Appendix needs is done on both halves of a word at once with the bf16x2 instructions:
+//   a  = |x| * 2^(127-F)                 exact (power-of-two scaling), a < 2
+//   r  = min(a + C, C + (2^m-1) ulp)     C = 2^(7-(m-1)-tau): the bf16 adder (8-bit significand) rounds
+//                                        a to a multiple of 2^(-(m-1)-tau) = ulp(C), nearest-even,
+//                                        and leaves q in the seven mantissa bits of r
+//   aq = r - C, Q(x) = aq * 2^(F-127)    exact
+// C is a power of two (not 1.5 * 2^k as in the fp32 formulation) because a >= 0: a + C stays inside
+// C's binade except for the single value 2C, which the clamp removes.  The Eq. 3 terms (aq - a, a)
+// are exact bf16 values; they are widened to fp32, squared and summed there.
+// Valid for 16 <= F <= 250 (every constant and result a normal number) and ties-to-even; callers
+// send other blocks (tiny, huge, Inf/NaN, ties-away) to the fp32 / integer formulation.
+#pragma once
+
+#include "bdr_device.cuh"
+
+namespace bdr {
+namespace x2 {
+
+__device__ __forceinline__ uint32_t hmul2(uint32_t a, uint32_t b) {
+    uint32_t d;
+    asm("mul.rn.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+    return d;
+}
+__device__ __forceinline__ uint32_t hadd2(uint32_t a, uint32_t b) {
+    uint32_t d;
+    asm("add.rn.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+    return d;
+}
+__device__ __forceinline__ uint32_t hsub2(uint32_t a, uint32_t b) {
+    uint32_t d;
+    asm("sub.rn.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+    return d;
+}
+__device__ __forceinline__ uint32_t hmin2(uint32_t a, uint32_t b) {
+    uint32_t d;
+    asm("min.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+    return d;
+}
+__device__ __forceinline__ uint32_t hfma2(uint32_t a, uint32_t b, uint32_t c) {
+    uint32_t d;
+    asm("fma.rn.bf16x2 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+    return d;
+}
+__device__ __forceinline__ uint32_t habs2(uint32_t a) {
+    uint32_t d;
+    asm("abs.bf16x2 %0, %1;" : "=r"(d) : "r"(a));
+    return d;
+}
+// Maximum that keeps NaNs (either operand NaN -> NaN), so a block with Inf/NaN reports exponent 255.
+__device__ __forceinline__ uint32_t hmax2_nan(uint32_t a, uint32_t b) {
+    uint32_t d;
+    asm("max.NaN.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+    return d;
+}
+// Two independent fp32 multiply-adds in one instruction: (d0, d1) += (a0 * a0, a1 * a1).
+__device__ __forceinline__ void ffma2_sq(float& d0, float& d1, float a0, float a1) {
+    asm("{.reg .b64 ra, rc; mov.b64 ra, {%2, %3}; mov.b64 rc, {%0, %1}; fma.rn.f32x2 rc, ra, ra, rc; mov.b64 {%0, %1}, rc;}"
+        : "+f"(d0), "+f"(d1)
+        : "f"(a0), "f"(a1));
+}
+
+constexpr uint32_t kAbs2 = 0x7FFF7FFFu, kSign2 = 0x80008000u;
+constexpr int kMinF = 16, kMaxF = 250;
+
+// constants of one mantissa width
+struct Consts {
+    uint32_t C0, C1;  // 2^(7-(m-1)) and half of it, in both halves
+    uint32_t QM;      // 2^m - 1 in both halves
+};
+__host__ __device__ __forceinline__ Consts make_consts(int m) {
+    Consts k;
+    const uint32_t e0 = (uint32_t)(127 + 7 - (m - 1));
+    k.C0 = (e0 << 7) * 0x10001u;
+    k.C1 = ((e0 - 1) << 7) * 0x10001u;
+    k.QM = ((1u << m) - 1u) * 0x10001u;
+    return k;
+}
+
+// Biased shared exponent of a block given as |x| words (row direction: all 16 halves are one block).
+// For non-negative bf16 the float maximum is the maximum of the bit patterns.
+__device__ __forceinline__ uint32_t block_exponent(const uint32_t (&aw)[8]) {
+    uint32_t mx = hmax2_nan(hmax2_nan(aw[0], aw[1]), hmax2_nan(aw[2], aw[3]));
+    mx = hmax2_nan(mx, hmax2_nan(hmax2_nan(aw[4], aw[5]), hmax2_nan(aw[6], aw[7])));
+    return max(mx & 0xFFFFu, mx >> 16) >> 7;
+}
+
+// Row direction: one block = eight words, sub-block j = word j.
+//   yw     dequantized words (YOUT)
+//   code2  per word, the two codes (sign << m | q) in bits [0, m] and [16, 16 + m] (CODE)
+//   micro  the eight sub-block shifts, bit j = tau of word j (CODE)
+//   pe, ps this block's Eq. 3 sums in the normalised domain (SUMS); scale by 2^(2F-254)
+template <bool SUMS, bool YOUT, bool CODE>
+__device__ __forceinline__ void quantize_block_row(const uint32_t (&w)[8], const uint32_t (&aw)[8], uint32_t F, int m,
+                                                   const Consts& k, uint32_t (&yw)[8], uint32_t (&code2)[8],
+                                                   uint32_t& micro, float& pe, float& ps) {
+    const uint32_t s2 = ((254u - F) << 7) * 0x10001u;  // 2^(127-F)
+    const uint32_t si2 = (F << 7) * 0x10001u;          // 2^(F-127)
+    float pe0 = 0.f, pe1 = 0.f, ps0 = 0.f, ps1 = 0.f;
+    uint32_t macc = 0;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        const uint32_t a2 = hmul2(aw[j], s2);
+        // a half is >= 1.0 (0x3F80) exactly when adding 0x0080 carries into bit 14
+        const bool top = ((a2 + 0x00800080u) & 0x40004000u) != 0;  // tau = 0
+        uint32_t r2;
+        if constexpr (SUMS) {
+            // tau picks the constant; aq and a stay in the block's normalised domain for the sums
+            const uint32_t C2 = top ? k.C0 : k.C1;
+            r2 = hmin2(hadd2(a2, C2), C2 + k.QM);
+            const uint32_t aq2 = hsub2(r2, C2);
+            if constexpr (YOUT) yw[j] = hmul2(aq2, si2) | (w[j] & kSign2);
+            const uint32_t d2 = hsub2(aq2, a2);  // exact
+            ffma2_sq(pe0, pe1, __uint_as_float(d2 << 16), __uint_as_float(d2 & 0xFFFF0000u));
+            ffma2_sq(ps0, ps1, __uint_as_float(a2 << 16), __uint_as_float(a2 & 0xFFFF0000u));
+            if constexpr (CODE) macc |= (r2 << (j + 1)) & (0x100u << j);  // bit 7 of r: lowest exponent bit of C
+        } else {
+            // tau doubles the operand instead (exact), so the constant and the clamp are fixed
+            const uint32_t g2 = top ? 0x3F803F80u : 0x40004000u;  // 1.0 or 2.0
+            r2 = hmin2(hfma2(a2, g2, k.C0), k.C0 + k.QM);
+            if constexpr (YOUT) yw[j] = hmul2(hsub2(r2, k.C0), top ? si2 : si2 - 0x00800080u) | (w[j] & kSign2);
+            if constexpr (CODE) macc |= (g2 << (j + 2)) & (0x10000u << j);  // bit 14 of 2.0
+        }
+        if constexpr (CODE) code2[j] = (r2 & 0x007F007Fu) | ((w[j] >> (15 - m)) & (0x00010001u << m));
+    }
+    if constexpr (SUMS) { pe = pe0 + pe1; ps = ps0 + ps1; }
+    if constexpr (CODE) {
+        if constexpr (SUMS) {
+            const uint32_t e0 = (uint32_t)(127 + 7 - (m - 1));  // exponent of C0: tau = bit ^ (e0 & 1)
+            micro = ((macc >> 8) ^ ((e0 & 1u) ? 0xFFu : 0u)) & 0xFFu;
+        } else {
+            micro = (macc >> 16) & 0xFFu;
+        }
+    }
+}
+
+// The sixteen W-bit codes of a block, from code2[], as the little-endian bit stream (W = m + 1).
+template <int W>
+__device__ __forceinline__ void pack_block(const uint32_t (&code2)[8], uint32_t (&cw)[(16 * W + 31) / 32]) {
+    if constexpr (W == 8) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) cw[i] = __byte_perm(code2[2 * i], code2[2 * i + 1], 0x6420);
+    } else {
+        uint32_t f[8];  // the two codes of a word side by side: 2W bits
+#pragma unroll
+        for (int j = 0; j < 8; ++j) f[j] = (code2[j] | (code2[j] >> (16 - W))) & ((1u << (2 * W)) - 1u);
+        if constexpr (W == 3) {
+            const uint32_t lo = f[0] + (f[1] << 6) + (f[2] << 12) + (f[3] << 18);
+            const uint32_t hi = f[4] + (f[5] << 6) + (f[6] << 12) + (f[7] << 18);
+            cw[0] = lo | (hi << 24);
+            cw[1] = hi >> 8;
+        } else {
+            static_assert(W == 5, "code widths of Table II");
+            const uint32_t g0 = f[0] + (f[1] << 10) + (f[2] << 20);
+            const uint32_t g1 = f[3] + (f[4] << 10) + (f[5] << 20);
+            const uint32_t g2 = f[6] + (f[7] << 10);
+            cw[0] = g0 | (g1 << 30);
+            cw[1] = (g1 >> 2) | (g2 << 28);
+            cw[2] = g2 >> 4;
+        }
+    }
+}
+
+// ---- packing without dequantized output or sums: fewest integer-pipe instructions ----------------------
+// The integer/logic pipe issues at half the rate of the FMA pipe, so this route keeps per-element work
+// on packed floating-point instructions wherever it can:
+//   * words are regrouped so that the two elements of a sub-block sit in the SAME half of two words
+//     (A = {x0, x2}, B = {x1, x3} from {x0, x1}, {x2, x3}); one packed maximum then yields both
+//     sub-block maxima of the pair, and everything after it treats the halves independently;
+//   * tau as arithmetic: u = relu(256 pm - 255) is 0 for pm < 1 and >= 1 otherwise (pm is the scaled
+//     sub-block maximum, a bf16 below 2), so g = 2 - min(u, 1) is the factor 2^tau that lines the
+//     sub-block up with the fixed constant C0;
+//   * the sign joins the magnitude arithmetically (m <= 6): with the constant raised by 1.0 = 2^(m-1)
+//     units, r - sgn(x) has mantissa q for x >= 0 and 2^m + q for x < 0, i.e. the code itself.
+// Words of the regrouped block: pair i (i = 0..3) covers elements 4i .. 4i+3.
+__device__ __forceinline__ uint32_t hfma2_relu(uint32_t a, uint32_t b, uint32_t c) {
+    uint32_t d;
+    asm("fma.rn.relu.bf16x2 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+    return d;
+}
+
+struct PairView {
+    uint32_t A[4], B[4];    // regrouped words
+    uint32_t aA[4], aB[4];  // their magnitudes
+    uint32_t pm[4];         // sub-block maxima: low half sub-block 2i, high half sub-block 2i+1
+};
+
+__device__ __forceinline__ uint32_t pair_view(const uint32_t (&w)[8], PairView& v) {  // returns F
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        v.A[i] = __byte_perm(w[2 * i], w[2 * i + 1], 0x5410);
+        v.B[i] = __byte_perm(w[2 * i], w[2 * i + 1], 0x7632);
+        v.aA[i] = habs2(v.A[i]);
+        v.aB[i] = habs2(v.B[i]);
+        v.pm[i] = hmax2_nan(v.aA[i], v.aB[i]);
+    }
+    const uint32_t mx = hmax2_nan(hmax2_nan(v.pm[0], v.pm[1]), hmax2_nan(v.pm[2], v.pm[3]));
+    return max(mx & 0xFFFFu, mx >> 16) >> 7;
+}
+
+template <int W>
+__device__ __forceinline__ void pack_pair_view(const PairView& v, uint32_t F, uint32_t (&cw)[(16 * W + 31) / 32], uint32_t& micro) {
+    constexpr int M = W - 1;
+    constexpr uint32_t e0 = (uint32_t)(127 + 7 - (M - 1));
+    constexpr bool kSignTrick = M <= 6;
+    constexpr uint32_t C0 = ((e0 << 7) + (kSignTrick ? (1u << (M - 1)) : 0u)) * 0x10001u;  // C0 (+ 1.0 = 2^(m-1) units)
+    constexpr uint32_t Cmax = C0 + ((1u << M) - 1u) * 0x10001u;
+    const uint32_t s2 = ((254u - F) << 7) * 0x10001u;  // 2^(127-F)
+    uint32_t macc = 0, f4[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const uint32_t u = hfma2_relu(hmul2(v.pm[i], s2), 0x43804380u, 0xC37FC37Fu);  // relu(256 pm - 255)
+        const uint32_t g = hsub2(0x40004000u, hmin2(u, 0x3F803F80u));                 // 2^tau per half
+        macc += g << (2 * i);
+        uint32_t rA = hmin2(hfma2(hmul2(v.aA[i], s2), g, C0), Cmax);
+        uint32_t rB = hmin2(hfma2(hmul2(v.aB[i], s2), g, C0), Cmax);
+        if constexpr (kSignTrick) {
+            rA = hsub2(rA, (v.A[i] & kSign2) | 0x3F803F80u);  // -/+ 1.0
+            rB = hsub2(rB, (v.B[i] & kSign2) | 0x3F803F80u);
+            constexpr uint32_t kCode = ((1u << W) - 1u) * 0x10001u;
+            const uint32_t comb = (rA & kCode) + ((rB & kCode) << W);  // halves: codes 4i, 4i+1 | codes 4i+2, 4i+3
+            f4[i] = (comb | (comb >> (16 - 2 * W))) & ((1u << (4 * W)) - 1u);
+        } else {
+            // W = 8: byte 0 / 2 of each word = sign bit over the seven magnitude bits; bytes 1 / 3 are not used
+            const uint32_t cA = ((v.A[i] >> 8) & 0x00800080u) | (rA & ~0x00800080u);
+            const uint32_t cB = ((v.B[i] >> 8) & 0x00800080u) | (rB & ~0x00800080u);
+            f4[i] = __byte_perm(cA, cB, 0x6240);
+        }
+    }
+    if constexpr (W == 8) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) cw[i] = f4[i];
+    } else if constexpr (W == 3) {
+        cw[0] = f4[0] + (f4[1] << 12) + (f4[2] << 24);
+        cw[1] = (f4[2] >> 8) + (f4[3] << 4);
+    } else {
+        static_assert(W == 3 || W == 5 || W == 8, "code widths of Table II");
+        cw[0] = f4[0] + (f4[1] << 20);
+        cw[1] = (f4[1] >> 12) + (f4[2] << 8) + (f4[3] << 28);
+        cw[2] = f4[3] >> 4;
+    }
+    // g is 0x3F80 + 0x80 tau per half: remove the constant part, then bit 7+2i = tau of sub-block 2i and
+    // bit 23+2i = tau of sub-block 2i+1
+    const uint32_t t = macc - 0x3F803F80u * 0x55u;
+    micro = ((t >> 7) & 0x55u) | ((t >> 22) & 0xAAu);
+}
+
+// Slow route for one block (exponent outside the packed range, Inf/NaN, ties-away): the fp32 /
+// integer formulation on widened values.  Kept out of line so the hot loop stays small.
+struct SlowOut {
+    uint4 y[2];
+    uint32_t cw[4];
+    uint32_t F, micro;
+    double e2, s2;
+};
+template <int W, bool SUMS>
+__device__ __noinline__ SlowOut quantize_block_slow(uint4 w0, uint4 w1, QParams qp) {
+    SlowOut o;
+    const uint4 w[2] = {w0, w1};
+    uint32_t u[kSlice], yb[kSlice], rq[kSlice], cb[kSlice / 2], tau[kSlice / 2], fj[kSlice / 2], fb[1];
+    SliceWords<__nv_bfloat16>::expand(w, u);
+    subblock_exponents<2>(u, fj);
+    uint32_t F = 0;
+#pragma unroll
+    for (int j = 0; j < kSlice / 2; ++j) F = max(F, fj[j]);
+    fb[0] = F;
+    o.e2 = 0.0;
+    o.s2 = 0.0;
+    quantize_slice<2, kSlice, SUMS, true, true>(u, fj, fb, qp, yb, rq, cb, tau, o.e2, o.s2);
+    slice_to_words(yb, o.y, (const __nv_bfloat16*)nullptr);
+    o.F = F >> 23;
+    uint32_t mb = 0;
+#pragma unroll
+    for (int j = 0; j < kSlice / 2; ++j) mb |= tau[j] << j;
+    o.micro = mb;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) o.cw[i] = 0;
+    if constexpr (W > 0) {
+        uint32_t words[(kSlice * W + 31) / 32];
+        pack_words<W, kSlice, 2>(u, rq, cb, words);
+#pragma unroll
+        for (int i = 0; i < (kSlice * W + 31) / 32; ++i) o.cw[i] = words[i];
+    }
+    return o;
+}
+
+}  // namespace x2
+}  // namespace bdr

@@ -192,3 +192,17 @@ def test_argument_errors_are_reported_not_launched():
         bdr.bdr_pack(bdr.MX6, x, small)
     assert e.value.status == -5
     torch.cuda.synchronize()
+
+
+@pytest.mark.gpu
+def test_bounded_waits_never_ran_out():
+    # bulk-copy kernels (1024-element runs of bf16) report a wait that ran out through a sticky status word
+    cfg = bdr.MX6
+    x = H.make_input("normal", 64, 4096, "bf16", seed=5)
+    xd = H.host_to_device(x, "bf16")
+    y = torch.empty_like(xd)
+    bdr.bdr_quant_dequant(cfg, xd, y)
+    planes = bdr.alloc_planes(cfg, 64, 4096, 1)
+    bdr.bdr_pack(cfg, xd, planes, y_dq=y)
+    torch.cuda.synchronize()
+    assert bdr.bdr_device_status() == 0
