@@ -11,6 +11,27 @@ namespace bdr {
 
 __device__ int g_device_status = 0;  // sticky: the first bounded wait that runs out leaves BDR_ERR_TIMEOUT here
 
+bool make_tensor_map_u16(CUtensorMap* out, const void* base, int64_t rows, int64_t cols, int64_t ld, int box_cols, int box_rows) {
+    typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                      const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                      CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+    static EncodeTiledFn fn = nullptr;
+    static std::once_flag once;
+    std::call_once(once, [] {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess && q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    });
+    if (!fn) return false;
+    const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
+    const cuuint32_t box[2] = {(cuuint32_t)box_cols, (cuuint32_t)box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    return fn(out, CU_TENSOR_MAP_DATA_TYPE_UINT16, 2, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+              CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 int* device_status_word() {
     static int* cached[64];
     static std::mutex mu;
@@ -107,6 +128,10 @@ static int quant_dispatch(const QParams& qp, const T* x, T* y, int64_t rows, int
         if (out) { if (tight) rc = pack_rowwise_mx<T>(x, y, rows, cols, ld, *out, qp, sums, st); }
         else rc = quant_rowwise<T>(x, y, rows, cols, ld, qp, sums, st);
     } else {
+        if constexpr (std::is_same<T, __nv_bfloat16>::value) {
+            if (!out || tight) rc = quant_colwise_mx_x2(x, y, rows, cols, ld, out, qp, sums, st);
+            if (rc != BDR_ERR_UNSUPPORTED) return rc;
+        }
         if (!out || tight) rc = quant_colwise_mx<T>(x, y, rows, cols, ld, out, qp, sums, st);
     }
     if (rc == BDR_ERR_UNSUPPORTED) rc = quant_general<T>(x, y, rows, cols, ld, axis, out, qp, sums, st);

@@ -6,6 +6,7 @@
 // (read back by bdr_device_status) and the caller leaves its loop.
 #pragma once
 
+#include <cuda.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -53,6 +54,13 @@ __device__ __forceinline__ void bulk_load(uint32_t smem_dst, const void* gsrc, u
 __device__ __forceinline__ void bulk_store(void* gdst, uint32_t smem_src, uint32_t bytes) {
     asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(gdst), "r"(smem_src), "r"(bytes) : "memory");
 }
+// 2-D tile of a tensor map -> shared (dense, row after row); x is the element index along the contiguous
+// dimension (x * element size must be a multiple of 16 bytes), y the row; completes on `bar`
+__device__ __forceinline__ void tma_load_2d(uint32_t smem_dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(smem_dst),
+                 "l"(map), "r"(x), "r"(y), "r"(bar)
+                 : "memory");
+}
 __device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 // all but the N most recent groups of this thread have finished READING shared memory
 template <int N>
@@ -80,6 +88,11 @@ __device__ __forceinline__ void sts16(uint32_t addr, uint32_t v) {
 __device__ __forceinline__ void report_timeout(int* status) { atomicCAS(status, 0, (int)BDR_ERR_TIMEOUT); }
 
 }  // namespace async
+
+// cuTensorMapEncodeTiled for a row-major [rows, cols] matrix of 16-bit elements with a pitch of ld elements and
+// a box of box_cols x box_rows (host; bdr_api.cu).  The library does not link libcuda: the entry point
+// comes from the runtime.  False if the driver refuses the map.
+bool make_tensor_map_u16(CUtensorMap* out, const void* base, int64_t rows, int64_t cols, int64_t ld, int box_cols, int box_rows);
 
 // Device address of the library's sticky status word on the current device (host; bdr_api.cu).
 int* device_status_word();

@@ -1,0 +1,279 @@
+// Column-direction (axis 0) kernels for bf16 tensors in the Table II family (k1 = 16, k2 = 2, d2 = 1,
+// m <= 7, ties-to-even) on packed bf16x2 arithmetic: a 32-bit word holds one row of two adjacent
+// columns, and the two halves are quantized as two independent blocks by the same instructions.
+//
+// A CTA (eight warps) owns tiles of 128 columns x 256 rows (16 block rows).  Warp w takes block rows 2w
+// and 2w+1 of every tile; each arrives as one 2-D TMA box of 16 rows x 128 columns (4 KB) in the
+// warp's own two-stage ring, so the box of the next tile is in flight while the current one is worked
+// on.  A lane owns four adjacent columns (8 bytes of every row).  Dequantized values go straight
+// from registers to global memory (8 bytes per lane and row, 256 contiguous bytes per warp and row).
+// The packed planes are column-major -- the transposed layout the backward-pass GEMMs read -- so codes
+// are first staged per tile in shared memory as [block-row pair][column] items; after a CTA barrier
+// the tile's columns are gathered and each column's 16 blocks leave as one contiguous run (32 W code
+// bytes, 16 exponent bytes, 16 microexponent bytes).
+#include <algorithm>
+
+#include "bdr_async.cuh"
+#include "bdr_x2.cuh"
+#include "bdr_host.h"
+
+namespace bdr {
+
+using bf16 = __nv_bfloat16;
+
+constexpr int kCThreads = 256;
+constexpr int kCWarps = kCThreads / 32;
+constexpr int kCTileCols = 128;
+constexpr int kCTileBlocks = 2 * kCWarps;  // 16 block rows = 256 rows
+constexpr int kCTileRows = kCTileBlocks * kSlice;
+constexpr int kCBoxBytes = kSlice * kCTileCols * 2;  // 4 KB
+constexpr int kCRingBytes = kCWarps * 2 * kCBoxBytes;
+constexpr int kCBarBytes = 128;
+
+template <int W> struct CStage {
+    // codes: W even: [block row 16][column 128] items of 2W bytes, columns XOR-swizzled by the block row;
+    //        W odd:  [block-row pair 8][column 128] items of 4W bytes (W words)
+    static constexpr int kElemBytes = kCTileBlocks * kCTileCols * 2 * W;
+    static constexpr int kExpBytes = kCTileBlocks * kCTileCols;  // [block row][column]
+    static constexpr int kBytes = W > 0 ? kElemBytes + 2 * kExpBytes : 0;
+};
+
+__device__ __forceinline__ uint2 lds64(uint32_t addr) {
+    uint2 v;
+    asm volatile("ld.shared.v2.b32 {%0, %1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(addr) : "memory");
+    return v;
+}
+__device__ __forceinline__ uint32_t lds32(uint32_t addr) {
+    uint32_t v;
+    asm volatile("ld.shared.b32 %0, [%1];" : "=r"(v) : "r"(addr) : "memory");
+    return v;
+}
+__device__ __forceinline__ uint32_t lds8(uint32_t addr) {
+    uint32_t v;
+    asm volatile("ld.shared.u8 %0, [%1];" : "=r"(v) : "r"(addr) : "memory");
+    return v;
+}
+__device__ __forceinline__ double pow4_weight_col(uint32_t F) { return __hiloint2double((int)((F << 21) + 0x30100000u), 0); }
+
+// W = 0: quantize-dequantize / sums only (any m <= 7, from qp); W = m + 1: also write the packed planes.
+template <int W, bool SUMS, bool YOUT>
+__global__ void __launch_bounds__(kCThreads, 2)
+col_mx_x2_kernel(const __grid_constant__ CUtensorMap xmap, bf16* y, int64_t ld, int n_col_tiles, int n_tiles, bdr_planes_t out,
+                 QParams qp, double* sums, int* status) {
+    using CS = CStage<W>;
+    constexpr bool PACK = W > 0;
+    constexpr int NCW = PACK ? (16 * W + 31) / 32 : 1;
+    extern __shared__ __align__(128) uint8_t smem[];  // ring [warp][2][4 KB], barriers, staging
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const uint32_t ring0 = async::smem_u32(smem) + warp * 2 * kCBoxBytes;
+    const uint32_t bars = async::smem_u32(smem) + kCRingBytes + warp * 16;
+    const uint32_t st_elems = async::smem_u32(smem) + kCRingBytes + kCBarBytes;
+    const uint32_t st_exps = st_elems + CS::kElemBytes, st_micro = st_exps + CS::kExpBytes;
+    const int m = PACK ? W - 1 : qp.m;
+
+    auto issue = [&](int t, int i) {  // box of block row 2*warp+i of tile t into stage i (lane 0 only)
+        const int rt = t / n_col_tiles, ct = t - rt * n_col_tiles;
+        async::mbar_expect_tx(bars + 8 * i, kCBoxBytes);
+        async::tma_load_2d(ring0 + i * kCBoxBytes, &xmap, ct * kCTileCols, rt * kCTileRows + (2 * warp + i) * kSlice, bars + 8 * i);
+    };
+    if (lane == 0) {
+        async::mbar_init(bars, 1);
+        async::mbar_init(bars + 8, 1);
+        async::fence_barrier_init();
+        if ((int)blockIdx.x < n_tiles) {
+            issue(blockIdx.x, 0);
+            issue(blockIdx.x, 1);
+        }
+    }
+    __syncwarp();
+    uint32_t phase = 0;
+    double e2 = 0.0, s2 = 0.0;
+    bool failed = false;
+    for (int t = blockIdx.x; t < n_tiles; t += gridDim.x) {
+        const int rt = t / n_col_tiles, ct = t - rt * n_col_tiles;
+        uint32_t cw0[4][NCW];  // codes of block row 2*warp (odd W: held until the pair is complete)
+#pragma unroll
+        for (int i = 0; i < 2; ++i) {
+            const int bl = 2 * warp + i;
+            if (!failed && !async::mbar_wait(bars + 8 * i, phase)) {
+                async::report_timeout(status);
+                failed = true;
+            }
+            uint32_t wc[2][16];
+            const uint32_t mine = ring0 + i * kCBoxBytes + lane * 8;
+#pragma unroll
+            for (int r = 0; r < kSlice; ++r) {
+                const uint2 v = lds64(mine + r * (kCTileCols * 2));
+                wc[0][r] = v.x;
+                wc[1][r] = v.y;
+            }
+            __syncwarp();  // every lane has read stage i
+            if (lane == 0 && !failed && t + (int)gridDim.x < n_tiles) issue(t + gridDim.x, i);
+            uint32_t Fb[4], Mb[4];
+#pragma unroll
+            for (int c = 0; c < 2; ++c) {  // the lane's two word columns
+                uint32_t aw[16], pm[8], yw[16], cl[NCW], ch[NCW], F2;
+                x2::WordColOut o;
+                if (x2::wordcol_exponents(wc[c], aw, pm, F2)) {
+                    x2::quantize_wordcol<W, SUMS, YOUT>(wc[c], aw, pm, F2, m, yw, cl, ch, o);
+                    if constexpr (SUMS) {
+                        const double wl = pow4_weight_col((F2 >> 7) & 0xFFu), wh = pow4_weight_col(F2 >> 23);
+                        e2 = fma((double)o.pe_lo, wl, e2);
+                        e2 = fma((double)o.pe_hi, wh, e2);
+                        s2 = fma((double)o.ps_lo, wl, s2);
+                        s2 = fma((double)o.ps_hi, wh, s2);
+                    }
+                } else {
+                    x2::WordCol in;
+#pragma unroll
+                    for (int r = 0; r < 16; ++r) in.w[r] = wc[c][r];
+                    const x2::WordColSlow so = x2::quantize_wordcol_slow<W, SUMS>(in, qp);
+#pragma unroll
+                    for (int r = 0; r < 16; ++r) yw[r] = so.y[r];
+#pragma unroll
+                    for (int k = 0; k < NCW; ++k) { cl[k] = so.cl[k]; ch[k] = so.ch[k]; }
+                    o.F2 = so.F2;
+                    o.micro_lo = so.micro_lo;
+                    o.micro_hi = so.micro_hi;
+                    if constexpr (SUMS) { e2 += so.e2; s2 += so.s2; }
+                }
+                if constexpr (YOUT) {
+#pragma unroll
+                    for (int r = 0; r < 16; ++r) wc[c][r] = yw[r];  // reuse the input registers for the output rows
+                }
+                if constexpr (PACK) {
+                    Fb[2 * c] = (o.F2 >> 7) & 0xFFu;
+                    Fb[2 * c + 1] = o.F2 >> 23;
+                    Mb[2 * c] = o.micro_lo;
+                    Mb[2 * c + 1] = o.micro_hi;
+                    if constexpr (W % 2 == 0) {
+                        // 2W bytes = one 16-byte item per (block row, column); columns swizzled by the block row
+                        const uint32_t rowb = st_elems + bl * (kCTileCols * 16);
+                        const int col = 4 * lane + 2 * c;
+                        async::sts128(rowb + ((col ^ (bl & 7)) * 16), make_uint4(cl[0], cl[1], cl[2], cl[3]));
+                        async::sts128(rowb + (((col + 1) ^ (bl & 7)) * 16), make_uint4(ch[0], ch[1], ch[2], ch[3]));
+                    } else if (i == 0) {
+#pragma unroll
+                        for (int k = 0; k < NCW; ++k) { cw0[2 * c][k] = cl[k]; cw0[2 * c + 1][k] = ch[k]; }
+                    } else {
+                        // the pair's 32 codes of a column as W words: block row 2w+1 follows 2w at bit 16 W
+                        const uint32_t item = st_elems + ((warp * kCTileCols + 4 * lane + 2 * c) * W) * 4;
+#pragma unroll
+                        for (int h = 0; h < 2; ++h) {
+                            const uint32_t(&a)[NCW] = cw0[2 * c + h];
+                            const uint32_t(&b)[NCW] = h ? ch : cl;
+                            const uint32_t dst = item + h * W * 4;
+#pragma unroll
+                            for (int k = 0; k < W / 2; ++k) async::sts32(dst + 4 * k, a[k]);
+                            async::sts32(dst + 4 * (W / 2), a[W / 2] | (b[0] << 16));
+#pragma unroll
+                            for (int k = 0; k < W / 2; ++k) async::sts32(dst + 4 * (W / 2 + 1 + k), __byte_perm(b[k], b[k + 1], 0x5432));
+                        }
+                    }
+                }
+            }
+            if constexpr (YOUT) {
+                bf16* py = y + ((int64_t)rt * kCTileRows + bl * kSlice) * ld + (int64_t)ct * kCTileCols + 4 * lane;
+#pragma unroll
+                for (int r = 0; r < kSlice; ++r) *reinterpret_cast<uint2*>(py + r * ld) = make_uint2(wc[0][r], wc[1][r]);
+            }
+            if constexpr (PACK) {
+                async::sts32(st_exps + bl * kCTileCols + 4 * lane, Fb[0] | (Fb[1] << 8) | (Fb[2] << 16) | (Fb[3] << 24));
+                async::sts32(st_micro + bl * kCTileCols + 4 * lane, Mb[0] | (Mb[1] << 8) | (Mb[2] << 16) | (Mb[3] << 24));
+            }
+        }
+        phase ^= 1;
+        if constexpr (PACK) {
+            __syncthreads();
+            // codes: column c of the tile owns 32 W contiguous bytes of its plane line = 2W vectors of 16 bytes
+            const int64_t blk0 = (int64_t)rt * kCTileBlocks;  // first block of the tile within a column
+            for (int idx = threadIdx.x; idx < kCTileCols * 2 * W; idx += kCThreads) {
+                const int c = idx / (2 * W), v = idx - c * (2 * W);
+                uint4 q;
+                if constexpr (W % 2 == 0) {
+                    // vector v covers bytes 16v .. 16v+15 of the run: W = 8 -> exactly block row v
+                    q = async::lds128(st_elems + v * (kCTileCols * 16) + ((c ^ (v & 7)) * 16));
+                } else {
+                    uint32_t x4[4];
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) {
+                        const int wd = 4 * v + k, pair = wd / W, kk = wd - pair * W;
+                        x4[k] = lds32(st_elems + ((pair * kCTileCols + c) * W + kk) * 4);
+                    }
+                    q = make_uint4(x4[0], x4[1], x4[2], x4[3]);
+                }
+                *reinterpret_cast<uint4*>(out.elems + ((int64_t)ct * kCTileCols + c) * out.ld_elems + blk0 * 2 * W + v * 16) = q;
+            }
+            // exponents and microexponents: 16 bytes per column each
+            for (int idx = threadIdx.x; idx < kCTileCols * 2; idx += kCThreads) {
+                const int c = idx & (kCTileCols - 1), which = idx / kCTileCols;
+                const uint32_t src = (which ? st_micro : st_exps) + c;
+                uint32_t x4[4] = {0, 0, 0, 0};
+#pragma unroll
+                for (int b = 0; b < 16; ++b) x4[b >> 2] |= lds8(src + b * kCTileCols) << ((b & 3) * 8);
+                uint8_t* base = which ? out.micro + ((int64_t)ct * kCTileCols + c) * out.ld_micro
+                                      : out.exps + ((int64_t)ct * kCTileCols + c) * out.ld_exps;
+                *reinterpret_cast<uint4*>(base + blk0) = make_uint4(x4[0], x4[1], x4[2], x4[3]);
+            }
+            __syncthreads();
+        }
+    }
+    if (SUMS) block_accumulate_sums(e2, s2, sums);
+}
+
+// ---- host side ----------------------------------------------------------------------------------------
+template <int W, bool SUMS, bool YOUT>
+static int launch_col_x2(const bf16* x, bf16* y, int64_t rows, int64_t cols, int64_t ld, const bdr_planes_t* out,
+                         const QParams& qp, double* sums, cudaStream_t st) {
+    auto kern = col_mx_x2_kernel<W, SUMS, YOUT>;
+    const size_t smem = kCRingBytes + kCBarBytes + CStage<W>::kBytes;
+    static bool attr_done = false;  // per instantiation; the attribute is idempotent, so a race is harmless
+    static int blocks_per_sm = 0;
+    if (!attr_done) {
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return BDR_ERR_CUDA;
+        int n = 0;
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, kern, kCThreads, smem) != cudaSuccess || n < 1) n = 1;
+        blocks_per_sm = n;
+        attr_done = true;
+    }
+    int* status = device_status_word();
+    if (!status) return BDR_ERR_CUDA;
+    CUtensorMap xmap;
+    if (!make_tensor_map_u16(&xmap, x, rows, cols, ld, kCTileCols, kSlice)) return BDR_ERR_CUDA;
+    const int n_ct = (int)(cols / kCTileCols);
+    const int64_t n_tiles = (int64_t)n_ct * (rows / kCTileRows);
+    bdr_planes_t pl = {};
+    if (out) pl = *out;
+    const int grid = (int)std::min<int64_t>(n_tiles, (int64_t)sm_count() * blocks_per_sm);
+    kern<<<grid, kCThreads, smem, st>>>(xmap, y, ld, n_ct, (int)n_tiles, pl, qp, sums, status);
+    return cudaGetLastError() == cudaSuccess ? BDR_OK : BDR_ERR_CUDA;
+}
+
+template <int W>
+static int col_x2_flags(const bf16* x, bf16* y, int64_t rows, int64_t cols, int64_t ld, const bdr_planes_t* out,
+                        const QParams& qp, double* sums, cudaStream_t st) {
+    if (sums) return y ? launch_col_x2<W, true, true>(x, y, rows, cols, ld, out, qp, sums, st)
+                       : launch_col_x2<W, true, false>(x, y, rows, cols, ld, out, qp, sums, st);
+    if (y) return launch_col_x2<W, false, true>(x, y, rows, cols, ld, out, qp, sums, st);
+    if constexpr (W > 0) return launch_col_x2<W, false, false>(x, y, rows, cols, ld, out, qp, sums, st);
+    return BDR_ERR_NULL;
+}
+
+// Fast path: whole tiles of 256 rows x 128 columns, 16-byte aligned rows; planes (if any) tight.
+// BDR_ERR_UNSUPPORTED sends the caller to the generic column kernels.
+int quant_colwise_mx_x2(const bf16* x, bf16* y, int64_t rows, int64_t cols, int64_t ld, const bdr_planes_t* out,
+                        const QParams& qp, double* sums, cudaStream_t st) {
+    if (qp.k1 != 16 || qp.k2 != 2 || qp.d2 != 1 || qp.m > 7 || qp.rounding != BDR_ROUND_NEAREST_EVEN) return BDR_ERR_UNSUPPORTED;
+    if (rows % kCTileRows != 0 || cols % kCTileCols != 0) return BDR_ERR_UNSUPPORTED;
+    if (((uintptr_t)x % 16) || ((uintptr_t)y % 8) || (ld * 2) % 16) return BDR_ERR_UNSUPPORTED;
+    if ((int64_t)(cols / kCTileCols) * (rows / kCTileRows) >= (1ll << 30) || rows >= (1ll << 31) || cols >= (1ll << 31)) return BDR_ERR_UNSUPPORTED;
+    if (!out) return col_x2_flags<0>(x, y, rows, cols, ld, out, qp, sums, st);
+    switch (qp.m) {
+        case 2: return col_x2_flags<3>(x, y, rows, cols, ld, out, qp, sums, st);
+        case 4: return col_x2_flags<5>(x, y, rows, cols, ld, out, qp, sums, st);
+        case 7: return col_x2_flags<8>(x, y, rows, cols, ld, out, qp, sums, st);
+    }
+    return BDR_ERR_UNSUPPORTED;
+}
+
+}  // namespace bdr

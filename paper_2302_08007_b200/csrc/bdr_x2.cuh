@@ -286,5 +286,189 @@ __device__ __noinline__ SlowOut quantize_block_slow(uint4 w0, uint4 w1, QParams 
     return o;
 }
 
+// ---- column direction ---------------------------------------------------------------------------------
+// A "word column" is sixteen words w[r], r = 0..15: rows r of two adjacent columns (low half = the even
+// column).  Each half is a block of its own, so everything runs on both halves independently: packed
+// maxima give the two shared exponents, F2 holds them in place (bits 14..7 of each half), and the
+// sub-block of rows 2j, 2j+1 has its maximum in pm[j].
+struct WordColOut {
+    uint32_t F2;           // shared exponents, (F << 7) per half
+    uint32_t micro_lo, micro_hi;
+    float pe_lo, pe_hi, ps_lo, ps_hi;  // Eq. 3 sums of the two blocks in their normalised domains
+};
+
+__device__ __forceinline__ bool wordcol_exponents(const uint32_t (&w)[16], uint32_t (&aw)[16], uint32_t (&pm)[8], uint32_t& F2) {
+#pragma unroll
+    for (int r = 0; r < 16; ++r) aw[r] = habs2(w[r]);
+#pragma unroll
+    for (int j = 0; j < 8; ++j) pm[j] = hmax2_nan(aw[2 * j], aw[2 * j + 1]);
+    const uint32_t mx = hmax2_nan(hmax2_nan(hmax2_nan(pm[0], pm[1]), hmax2_nan(pm[2], pm[3])),
+                                  hmax2_nan(hmax2_nan(pm[4], pm[5]), hmax2_nan(pm[6], pm[7])));
+    F2 = mx & 0x7F807F80u;
+    const uint32_t f_lo = (F2 >> 7) & 0xFFu, f_hi = F2 >> 23;
+    return (f_lo - kMinF <= (uint32_t)(kMaxF - kMinF)) && (f_hi - kMinF <= (uint32_t)(kMaxF - kMinF));
+}
+
+// code streams of the two columns from the sixteen per-row code words (code of the even column in the
+// low half, W clean bits; for W = 8 only bytes 0 and 2 need to be clean)
+template <int W>
+__device__ __forceinline__ void wordcol_streams(const uint32_t (&code)[16], uint32_t (&cl)[(16 * W + 31) / 32],
+                                                uint32_t (&ch)[(16 * W + 31) / 32]) {
+    if constexpr (W == 8) {
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const uint32_t p = __byte_perm(code[4 * k], code[4 * k + 1], 0x6240);      // rows 4k, 4k+1: low column | high column
+            const uint32_t q = __byte_perm(code[4 * k + 2], code[4 * k + 3], 0x6240);  // rows 4k+2, 4k+3
+            cl[k] = __byte_perm(p, q, 0x5410);
+            ch[k] = __byte_perm(p, q, 0x7632);
+        }
+    } else {
+        uint32_t t[8];  // rows 2j, 2j+1 side by side in each half: 2W bits
+#pragma unroll
+        for (int j = 0; j < 8; ++j) t[j] = code[2 * j] + (code[2 * j + 1] << W);
+        if constexpr (W == 3) {
+            uint32_t lo[4], hi[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const uint32_t q4 = t[2 * i] + (t[2 * i + 1] << 6);  // rows 4i .. 4i+3: 12 bits per half
+                lo[i] = q4 & 0xFFFFu;
+                hi[i] = q4 >> 16;
+            }
+            cl[0] = lo[0] + (lo[1] << 12) + (lo[2] << 24);
+            cl[1] = (lo[2] >> 8) + (lo[3] << 4);
+            ch[0] = hi[0] + (hi[1] << 12) + (hi[2] << 24);
+            ch[1] = (hi[2] >> 8) + (hi[3] << 4);
+        } else {
+            static_assert(W == 3 || W == 5 || W == 8, "code widths of Table II");
+            uint32_t lo[8], hi[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) { lo[j] = t[j] & 0xFFFFu; hi[j] = t[j] >> 16; }
+            cl[0] = lo[0] + (lo[1] << 10) + (lo[2] << 20) + (lo[3] << 30);
+            cl[1] = (lo[3] >> 2) + (lo[4] << 8) + (lo[5] << 18) + (lo[6] << 28);
+            cl[2] = (lo[6] >> 4) + (lo[7] << 6);
+            ch[0] = hi[0] + (hi[1] << 10) + (hi[2] << 20) + (hi[3] << 30);
+            ch[1] = (hi[3] >> 2) + (hi[4] << 8) + (hi[5] << 18) + (hi[6] << 28);
+            ch[2] = (hi[6] >> 4) + (hi[7] << 6);
+        }
+    }
+}
+
+// Fast path of one word column (the caller has checked both exponents with wordcol_exponents).
+//   W > 0: code streams cl / ch and the micro bytes; YOUT: dequantized words; SUMS: the four partial sums.
+template <int W, bool SUMS, bool YOUT>
+__device__ __forceinline__ void quantize_wordcol(const uint32_t (&w)[16], const uint32_t (&aw)[16], const uint32_t (&pm)[8],
+                                                 uint32_t F2, int m, uint32_t (&yw)[16],
+                                                 uint32_t (&cl)[W > 0 ? (16 * W + 31) / 32 : 1],
+                                                 uint32_t (&ch)[W > 0 ? (16 * W + 31) / 32 : 1], WordColOut& o) {
+    constexpr bool PACK = W > 0;
+    constexpr bool kPackOnly = PACK && !SUMS && !YOUT;
+    constexpr bool kSignTrick = kPackOnly && W - 1 <= 6;
+    const uint32_t e0 = (uint32_t)(127 + 7 - (m - 1));
+    const uint32_t C0 = ((e0 << 7) + (kSignTrick ? (1u << (m - 1)) : 0u)) * 0x10001u;
+    const uint32_t QM = ((1u << m) - 1u) * 0x10001u;
+    const uint32_t s2 = 0x7F007F00u - F2;  // 2^(127-F) per half
+    uint32_t code[16];
+    uint32_t macc = 0;
+    float pe0 = 0.f, pe1 = 0.f, ps0 = 0.f, ps1 = 0.f;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        const uint32_t u = hfma2_relu(hmul2(pm[j], s2), 0x43804380u, 0xC37FC37Fu);  // relu(256 pm - 255): 0 iff tau = 1
+        const uint32_t v = hmin2(u, 0x3F803F80u);                                   // 1.0 (tau = 0) or 0.0
+        if constexpr (kPackOnly) {
+            const uint32_t g = hsub2(0x40004000u, v);  // 2^tau
+            macc += g << j;
+#pragma unroll
+            for (int r = 2 * j; r < 2 * j + 2; ++r) {
+                uint32_t r2 = hmin2(hfma2(hmul2(aw[r], s2), g, C0), C0 + QM);
+                if constexpr (kSignTrick) {
+                    r2 = hsub2(r2, (w[r] & kSign2) | 0x3F803F80u);
+                    code[r] = r2 & (((1u << W) - 1u) * 0x10001u);
+                } else {
+                    code[r] = ((w[r] >> 8) & 0x00800080u) | (r2 & ~0x00800080u);  // bytes 1 and 3 hold leftovers
+                }
+            }
+        } else {
+            const uint32_t ginv = hfma2(v, 0x3F003F00u, 0x3F003F00u);  // 2^-tau
+            const uint32_t C2 = hmul2(C0, ginv);
+            macc += ginv << j;
+#pragma unroll
+            for (int r = 2 * j; r < 2 * j + 2; ++r) {
+                const uint32_t a2 = hmul2(aw[r], s2);
+                const uint32_t r2 = hmin2(hadd2(a2, C2), C2 + QM);
+                const uint32_t aq2 = hsub2(r2, C2);
+                if constexpr (YOUT) yw[r] = hmul2(aq2, F2) | (w[r] & kSign2);
+                if constexpr (SUMS) {
+                    const uint32_t d2 = hsub2(aq2, a2);  // exact
+                    ffma2_sq(pe0, pe1, __uint_as_float(d2 << 16), __uint_as_float(d2 & 0xFFFF0000u));
+                    ffma2_sq(ps0, ps1, __uint_as_float(a2 << 16), __uint_as_float(a2 & 0xFFFF0000u));
+                }
+                if constexpr (PACK) {
+                    if constexpr (W == 8) code[r] = ((w[r] >> 8) & 0x00800080u) | (r2 & 0x007F007Fu);
+                    else code[r] = (r2 & (((1u << (W - 1)) - 1u) * 0x10001u)) | ((w[r] >> (16 - W)) & (0x00010001u << (W - 1)));
+                }
+            }
+        }
+    }
+    o.F2 = F2;
+    if constexpr (SUMS) { o.pe_lo = pe0; o.pe_hi = pe1; o.ps_lo = ps0; o.ps_hi = ps1; }
+    if constexpr (PACK) {
+        wordcol_streams<PACK ? W : 8>(code, cl, ch);
+        // per half the accumulated factors are 0x3F80 + 0x80 tau (2^tau) or 0x3F80 - 0x80 tau (2^-tau), shifted by j
+        const uint32_t t = kPackOnly ? macc - 0x3F803F80u * 255u : 0x3F803F80u * 255u - macc;
+        o.micro_lo = (t >> 7) & 0xFFu;
+        o.micro_hi = (t >> 23) & 0xFFu;
+    }
+}
+
+// Slow route for one word column: the fp32 / integer formulation on each of the two blocks.
+struct WordCol {
+    uint32_t w[16];
+};
+struct WordColSlow {
+    uint32_t y[16];
+    uint32_t cl[4], ch[4];
+    uint32_t F2, micro_lo, micro_hi;
+    double e2, s2;
+};
+template <int W, bool SUMS>
+__device__ __noinline__ WordColSlow quantize_wordcol_slow(WordCol in, QParams qp) {
+    WordColSlow o;
+    o.e2 = 0.0;
+    o.s2 = 0.0;
+    uint32_t Fs[2], ms[2], yb[2][kSlice];
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+        uint32_t u[kSlice], rq[kSlice], cb[kSlice / 2], tau[kSlice / 2], fj[kSlice / 2], fb[1];
+#pragma unroll
+        for (int r = 0; r < kSlice; ++r) u[r] = h ? (in.w[r] & 0xFFFF0000u) : (in.w[r] << 16);
+        subblock_exponents<2>(u, fj);
+        uint32_t F = 0;
+#pragma unroll
+        for (int j = 0; j < kSlice / 2; ++j) F = max(F, fj[j]);
+        fb[0] = F;
+        quantize_slice<2, kSlice, SUMS, true, true>(u, fj, fb, qp, yb[h], rq, cb, tau, o.e2, o.s2);
+        Fs[h] = F >> 23;
+        uint32_t mb = 0;
+#pragma unroll
+        for (int j = 0; j < kSlice / 2; ++j) mb |= tau[j] << j;
+        ms[h] = mb;
+        uint32_t* dst = h ? o.ch : o.cl;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) dst[i] = 0;
+        if constexpr (W > 0) {
+            uint32_t words[(kSlice * W + 31) / 32];
+            pack_words<W, kSlice, 2>(u, rq, cb, words);
+#pragma unroll
+            for (int i = 0; i < (kSlice * W + 31) / 32; ++i) dst[i] = words[i];
+        }
+    }
+#pragma unroll
+    for (int r = 0; r < kSlice; ++r) o.y[r] = (yb[0][r] >> 16) | (yb[1][r] & 0xFFFF0000u);
+    o.F2 = (Fs[0] << 7) | (Fs[1] << 23);
+    o.micro_lo = ms[0];
+    o.micro_hi = ms[1];
+    return o;
+}
+
 }  // namespace x2
 }  // namespace bdr

@@ -75,16 +75,21 @@ def main():
     planes = bdr.alloc_planes(cfg, a.rows, a.cols, a.axis)
     sums = None if a.no_sums else torch.zeros(2, dtype=torch.float64, device="cuda")
     bdr.bdr_pack(cfg, x, planes, axis=a.axis)
-    torch.cuda.synchronize()
-    ev = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
-    ev[0].record()
-    for _ in range(a.reps):
+
+    def once():
         if a.op == "quant_dequant":
             bdr.bdr_quant_dequant(cfg, x, None if a.no_y else y, axis=a.axis, qsnr_sums=sums)
         elif a.op == "pack":
             bdr.bdr_pack(cfg, x, planes, axis=a.axis, qsnr_sums=sums)
         else:
             bdr.bdr_unpack(cfg, planes, y, axis=a.axis)
+
+    once()  # first call of this kernel variant: attribute set-up
+    torch.cuda.synchronize()
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+    ev[0].record()
+    for _ in range(a.reps):
+        once()
     ev[1].record()
     torch.cuda.synchronize()
     print("%s %s axis=%d %s %dx%d: %.4f ms per launch" % (a.op, a.fmt, a.axis, a.dtype, a.rows, a.cols,
