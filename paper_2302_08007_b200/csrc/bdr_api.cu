@@ -234,6 +234,9 @@ int bdr_unpack(const bdr_config_t* cfg, const bdr_planes_t* in, void* y, bdr_dty
                        : unpack_colwise_mx<float>(*in, (float*)y, rows, cols, ld, qp, st);
         if (rc == BDR_ERR_UNSUPPORTED) rc = unpack_general<float>(*in, (float*)y, rows, cols, ld, axis, qp, st);
     } else {
+        rc = BDR_ERR_UNSUPPORTED;
+        if (axis == 1) rc = unpack_rowwise_mx_x2(*in, (__nv_bfloat16*)y, rows, cols, ld, qp, st);
+        if (rc != BDR_ERR_UNSUPPORTED) return rc;
         rc = axis == 1 ? unpack_rowwise_mx<__nv_bfloat16>(*in, (__nv_bfloat16*)y, rows, cols, ld, qp, st)
                        : unpack_colwise_mx<__nv_bfloat16>(*in, (__nv_bfloat16*)y, rows, cols, ld, qp, st);
         if (rc == BDR_ERR_UNSUPPORTED) rc = unpack_general<__nv_bfloat16>(*in, (__nv_bfloat16*)y, rows, cols, ld, axis, qp, st);

@@ -470,5 +470,79 @@ __device__ __noinline__ WordColSlow quantize_wordcol_slow(WordCol in, QParams qp
     return o;
 }
 
+// ---- decoding -----------------------------------------------------------------------------------------
+// value = q * 2^p, p = F - 127 - tau - (m - 1).  The bf16 number 128 + q is built by ORing q into the
+// mantissa of 128.0, and fma(128 + q, 2^p, -128 * 2^p) is exactly q * 2^p, two elements at a time.
+// Needs every scale normal: kMinF <= F <= kMaxDecodeF; other blocks (and NaN blocks) go the slow way.
+constexpr int kMaxDecodeF = 240;
+
+// The two codes of sub-block j of a little-endian stream of W-bit codes, in bits [0, W) and [16, 16 + W)
+// (other bits hold leftovers that the callers mask away).
+template <int W, int NW>
+__device__ __forceinline__ uint32_t code_pair(const uint32_t (&s)[NW], int j) {
+    if constexpr (W == 8) {
+        return __byte_perm(s[j >> 1], 0u, (j & 1) ? 0x4342 : 0x4140);
+    } else {
+        const int bit = 2 * W * j, wi = bit >> 5, sh = bit & 31;
+        uint32_t f = sh == 0 ? s[wi] : (sh + 2 * W > 32 ? __funnelshift_r(s[wi], s[wi + 1], sh) : s[wi] >> sh);
+        f &= (1u << (2 * W)) - 1u;
+        return f * (1u + (1u << (16 - W)));  // no carries: 3W <= 16
+    }
+}
+
+// Row direction: the W words s[] hold two adjacent blocks (32 codes); F0 / F1 their exponents, mb their
+// microexponent bytes (block 0 in bits 0..7).  Both exponents must be in the fast range.
+template <int W>
+__device__ __forceinline__ void decode_two_blocks_row(const uint32_t (&s)[W], uint32_t F0, uint32_t F1, uint32_t mb,
+                                                      uint32_t (&yw)[16]) {
+    constexpr int M = W - 1;
+    constexpr uint32_t kQ2 = ((1u << M) - 1u) * 0x10001u;
+#pragma unroll
+    for (int b = 0; b < 2; ++b) {
+        const uint32_t F = b ? F1 : F0, mbb = b ? mb >> 8 : mb;
+        const uint32_t sc0 = ((F - (uint32_t)(M - 1)) << 7) * 0x10001u;  // 2^p for tau = 0
+        const uint32_t nb0 = sc0 + 0x83808380u;                          // -128 * 2^p
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const uint32_t c2 = code_pair<W, W>(s, 8 * b + j);
+            const uint32_t t = ((mbb << (7 - j)) & 0x80u) * 0x10001u;  // tau lowers both exponents by one
+            yw[8 * b + j] = hfma2((c2 & kQ2) | 0x43004300u, sc0 - t, nb0 - t) | ((c2 << (15 - M)) & kSign2);
+        }
+    }
+}
+
+// Slow route: the fp32 decoder on each block, then back to packed bf16.
+template <int W> struct TwoBlocks {
+    uint32_t s[W];
+};
+struct TwoBlocksOut {
+    uint32_t y[16];
+};
+template <int W>
+__device__ __noinline__ TwoBlocksOut decode_two_blocks_slow(TwoBlocks<W> in, uint32_t F0, uint32_t F1, uint32_t mb) {
+    TwoBlocksOut o;
+    constexpr int NW = (kSlice * W + 31) / 32;
+#pragma unroll
+    for (int b = 0; b < 2; ++b) {
+        uint32_t words[NW + 1], yb[kSlice];
+#pragma unroll
+        for (int i = 0; i <= NW; ++i) words[i] = 0;
+#pragma unroll
+        for (int i = 0; i < NW; ++i) {
+            if (b == 0) {
+                words[i] = in.s[i];
+            } else if constexpr (W % 2 == 0) {
+                words[i] = in.s[W / 2 + i];
+            } else {
+                words[i] = __byte_perm(in.s[W / 2 + i], W / 2 + i + 1 < W ? in.s[W / 2 + i + 1] : 0u, 0x5432);
+            }
+        }
+        decode_slice_impl<W, false>(words, (int)(b ? F1 : F0), b ? (mb >> 8) & 0xFFu : mb & 0xFFu, yb);
+#pragma unroll
+        for (int k = 0; k < 8; ++k) o.y[8 * b + k] = (yb[2 * k] >> 16) | (yb[2 * k + 1] & 0xFFFF0000u);
+    }
+    return o;
+}
+
 }  // namespace x2
 }  // namespace bdr
