@@ -235,7 +235,8 @@ int bdr_unpack(const bdr_config_t* cfg, const bdr_planes_t* in, void* y, bdr_dty
         if (rc == BDR_ERR_UNSUPPORTED) rc = unpack_general<float>(*in, (float*)y, rows, cols, ld, axis, qp, st);
     } else {
         rc = BDR_ERR_UNSUPPORTED;
-        if (axis == 1) rc = unpack_rowwise_mx_x2(*in, (__nv_bfloat16*)y, rows, cols, ld, qp, st);
+        rc = axis == 1 ? unpack_rowwise_mx_x2(*in, (__nv_bfloat16*)y, rows, cols, ld, qp, st)
+                       : unpack_colwise_mx_x2(*in, (__nv_bfloat16*)y, rows, cols, ld, qp, st);
         if (rc != BDR_ERR_UNSUPPORTED) return rc;
         rc = axis == 1 ? unpack_rowwise_mx<__nv_bfloat16>(*in, (__nv_bfloat16*)y, rows, cols, ld, qp, st)
                        : unpack_colwise_mx<__nv_bfloat16>(*in, (__nv_bfloat16*)y, rows, cols, ld, qp, st);

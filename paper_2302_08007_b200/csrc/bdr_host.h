@@ -45,6 +45,8 @@ int unpack_general(const bdr_planes_t& in, T* y, int64_t rows, int64_t cols, int
 
 int unpack_rowwise_mx_x2(const bdr_planes_t& in, __nv_bfloat16* y, int64_t rows, int64_t cols, int64_t ld, const QParams& qp,
                          cudaStream_t st);  // bdr_unpack_x2.cu
+int unpack_colwise_mx_x2(const bdr_planes_t& in, __nv_bfloat16* y, int64_t rows, int64_t cols, int64_t ld, const QParams& qp,
+                         cudaStream_t st);  // bdr_unpack_col_x2.cu
 
 // unpack fast paths for k1 = 16, k2 = 2 (bdr_unpack.cu)
 template <typename T>

@@ -1,0 +1,156 @@
+// Column-direction (axis 0) unpack to bf16 for the Table II family on packed bf16x2 arithmetic: the
+// mirror image of the column packing kernel in bdr_col_x2.cu.  A CTA (eight warps) owns tiles of 128
+// columns x 256 rows.  The packed planes are column-major, so a tile's input is, per column, one run
+// of 32 W code bytes, 16 exponent bytes and 16 microexponent bytes; all threads fetch these runs with
+// coalesced 16-byte cp.async copies into a double-buffered staging area (the next tile is in flight
+// while the current one is decoded).  Warp w then decodes block rows 2w and 2w+1: a lane owns four
+// adjacent columns, decodes two columns at a time in the two halves of a word and writes 8 bytes per
+// row, i.e. 256 contiguous bytes per warp and row.
+#include <algorithm>
+
+#include "bdr_async.cuh"
+#include "bdr_x2.cuh"
+#include "bdr_host.h"
+
+namespace bdr {
+
+using bf16 = __nv_bfloat16;
+
+constexpr int kUCThreads = 256;
+constexpr int kUCWarps = kUCThreads / 32;
+constexpr int kUCTileCols = 128;
+constexpr int kUCTileBlocks = 2 * kUCWarps;  // 16 block rows
+constexpr int kUCTileRows = kUCTileBlocks * kSlice;
+
+template <int W> struct UCStage {
+    static constexpr int kPitch = kUCTileBlocks * 2 * W + 16;  // code bytes of one column, padded so columns spread over banks
+    static constexpr int kElemBytes = kUCTileCols * kPitch;
+    static constexpr int kExpBytes = kUCTileCols * 16;
+    static constexpr int kBytes = kElemBytes + 2 * kExpBytes;
+};
+
+__device__ __forceinline__ uint32_t uc_lds32(uint32_t addr) {
+    uint32_t v;
+    asm volatile("ld.shared.b32 %0, [%1];" : "=r"(v) : "r"(addr) : "memory");
+    return v;
+}
+__device__ __forceinline__ uint32_t uc_lds16(uint32_t addr) {
+    uint16_t v;
+    asm volatile("ld.shared.u16 %0, [%1];" : "=h"(v) : "r"(addr) : "memory");
+    return v;
+}
+__device__ __forceinline__ void uc_cp16(uint32_t smem_dst, const void* gsrc) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_dst), "l"(gsrc) : "memory");
+}
+
+template <int W>
+__global__ void __launch_bounds__(kUCThreads, 2)
+unpack_col_x2_kernel(bdr_planes_t in, bf16* y, int64_t ld, int n_col_tiles, int n_tiles) {
+    using ST = UCStage<W>;
+    extern __shared__ __align__(128) uint8_t smem[];  // two staging buffers: codes | exponents | microexponents
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const uint32_t base = async::smem_u32(smem);
+    auto fetch = [&](int t, int buf) {
+        const int rt = t / n_col_tiles, ct = t - rt * n_col_tiles;
+        const int64_t blk0 = (int64_t)rt * kUCTileBlocks;
+        const uint32_t b = base + buf * ST::kBytes;
+        for (int idx = threadIdx.x; idx < kUCTileCols * 2 * W; idx += kUCThreads) {
+            const int c = idx / (2 * W), v = idx - c * (2 * W);
+            uc_cp16(b + c * ST::kPitch + v * 16, in.elems + ((int64_t)ct * kUCTileCols + c) * in.ld_elems + blk0 * 2 * W + v * 16);
+        }
+        for (int idx = threadIdx.x; idx < kUCTileCols * 2; idx += kUCThreads) {
+            const int c = idx & (kUCTileCols - 1), which = idx / kUCTileCols;
+            const uint8_t* src = which ? in.micro + ((int64_t)ct * kUCTileCols + c) * in.ld_micro
+                                       : in.exps + ((int64_t)ct * kUCTileCols + c) * in.ld_exps;
+            uc_cp16(b + ST::kElemBytes + which * ST::kExpBytes + c * 16, src + blk0);
+        }
+    };
+    int buf = 0;
+    if ((int)blockIdx.x < n_tiles) fetch(blockIdx.x, 0);
+    cp_async_commit();
+    for (int t = blockIdx.x; t < n_tiles; t += gridDim.x) {
+        if (t + (int)gridDim.x < n_tiles) fetch(t + gridDim.x, buf ^ 1);
+        cp_async_commit();
+        cp_async_wait<1>();
+        __syncthreads();  // the tile's bytes were fetched by all threads
+        const int rt = t / n_col_tiles, ct = t - rt * n_col_tiles;
+        const uint32_t b = base + buf * ST::kBytes;
+        uint32_t s[4][W], Fp[4], mp[4];  // the lane's four columns: pair streams, exponent and microexponent byte pairs
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            const int col = 4 * lane + c;
+            const uint32_t src = b + col * ST::kPitch + warp * 4 * W;
+            if constexpr (W == 8) {
+                const uint4 a0 = async::lds128(src), a1 = async::lds128(src + 16);
+                s[c][0] = a0.x; s[c][1] = a0.y; s[c][2] = a0.z; s[c][3] = a0.w;
+                s[c][4] = a1.x; s[c][5] = a1.y; s[c][6] = a1.z; s[c][7] = a1.w;
+            } else {
+#pragma unroll
+                for (int k = 0; k < W; ++k) s[c][k] = uc_lds32(src + 4 * k);
+            }
+            Fp[c] = uc_lds16(b + ST::kElemBytes + col * 16 + 2 * warp);
+            mp[c] = uc_lds16(b + ST::kElemBytes + ST::kExpBytes + col * 16 + 2 * warp);
+        }
+#pragma unroll
+        for (int i = 0; i < 2; ++i) {  // block rows 2*warp and 2*warp + 1
+            uint32_t yw[2][16];
+#pragma unroll
+            for (int c = 0; c < 2; ++c) {
+                const uint32_t F_lo = (Fp[2 * c] >> (8 * i)) & 0xFFu, F_hi = (Fp[2 * c + 1] >> (8 * i)) & 0xFFu;
+                const uint32_t m_lo = (mp[2 * c] >> (8 * i)) & 0xFFu, m_hi = (mp[2 * c + 1] >> (8 * i)) & 0xFFu;
+                if ((F_lo - x2::kMinF <= (uint32_t)(x2::kMaxDecodeF - x2::kMinF)) && (F_hi - x2::kMinF <= (uint32_t)(x2::kMaxDecodeF - x2::kMinF))) {
+                    x2::decode_wordcol<W>(s[2 * c], s[2 * c + 1], i, (F_lo << 7) | (F_hi << 23), m_lo | (m_hi << 16), yw[c]);
+                } else {
+                    x2::TwoBlocks<W> lo, hi;
+#pragma unroll
+                    for (int k = 0; k < W; ++k) { lo.s[k] = s[2 * c][k]; hi.s[k] = s[2 * c + 1][k]; }
+                    const x2::TwoBlocksOut o = x2::decode_wordcol_slow<W>(lo, hi, i, F_lo, F_hi, m_lo, m_hi);
+#pragma unroll
+                    for (int r = 0; r < 16; ++r) yw[c][r] = o.y[r];
+                }
+            }
+            bf16* py = y + ((int64_t)rt * kUCTileRows + (2 * warp + i) * kSlice) * ld + (int64_t)ct * kUCTileCols + 4 * lane;
+#pragma unroll
+            for (int r = 0; r < kSlice; ++r) *reinterpret_cast<uint2*>(py + r * ld) = make_uint2(yw[0][r], yw[1][r]);
+        }
+        __syncthreads();  // everyone is done with this buffer before it is refilled
+        buf ^= 1;
+    }
+}
+
+template <int W>
+static int launch_unpack_col_x2(const bdr_planes_t& in, bf16* y, int64_t rows, int64_t cols, int64_t ld, cudaStream_t st) {
+    auto kern = unpack_col_x2_kernel<W>;
+    const size_t smem = 2 * UCStage<W>::kBytes;
+    static bool attr_done = false;  // per instantiation; the attribute is idempotent, so a race is harmless
+    static int blocks_per_sm = 0;
+    if (!attr_done) {
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return BDR_ERR_CUDA;
+        int n = 0;
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, kern, kUCThreads, smem) != cudaSuccess || n < 1) n = 1;
+        blocks_per_sm = n;
+        attr_done = true;
+    }
+    const int n_ct = (int)(cols / kUCTileCols);
+    const int64_t n_tiles = (int64_t)n_ct * (rows / kUCTileRows);
+    const int grid = (int)std::min<int64_t>(n_tiles, (int64_t)sm_count() * blocks_per_sm);
+    kern<<<grid, kUCThreads, smem, st>>>(in, y, ld, n_ct, (int)n_tiles);
+    return cudaGetLastError() == cudaSuccess ? BDR_OK : BDR_ERR_CUDA;
+}
+
+// Whole tiles of 256 rows x 128 columns, 8-byte aligned output rows.
+int unpack_colwise_mx_x2(const bdr_planes_t& in, bf16* y, int64_t rows, int64_t cols, int64_t ld, const QParams& qp,
+                         cudaStream_t st) {
+    if (qp.k1 != 16 || qp.k2 != 2 || qp.d2 != 1) return BDR_ERR_UNSUPPORTED;
+    if (rows % kUCTileRows != 0 || cols % kUCTileCols != 0 || rows == 0 || cols == 0) return BDR_ERR_UNSUPPORTED;
+    if (((uintptr_t)y % 8) || (ld * 2) % 8) return BDR_ERR_UNSUPPORTED;
+    if ((int64_t)(cols / kUCTileCols) * (rows / kUCTileRows) >= (1ll << 30)) return BDR_ERR_UNSUPPORTED;
+    switch (qp.m) {
+        case 2: return launch_unpack_col_x2<3>(in, y, rows, cols, ld, st);
+        case 4: return launch_unpack_col_x2<5>(in, y, rows, cols, ld, st);
+        case 7: return launch_unpack_col_x2<8>(in, y, rows, cols, ld, st);
+    }
+    return BDR_ERR_UNSUPPORTED;
+}
+
+}  // namespace bdr

@@ -544,5 +544,66 @@ __device__ __noinline__ TwoBlocksOut decode_two_blocks_slow(TwoBlocks<W> in, uin
     return o;
 }
 
+// Column direction: sl[] / sh[] are the streams of the even / odd column over a pair of block rows (32 codes
+// each, block row i at bit 16 W i).  Decodes block row i of both columns into the sixteen row words.
+// F2 = the two exponents as (F << 7) per half, mm = the two microexponent bytes (odd column in bits 16..23).
+template <int W>
+__device__ __forceinline__ uint32_t code_pair_col(const uint32_t (&sl)[W], const uint32_t (&sh)[W], int idx /* 0..31 */) {
+    if constexpr (W == 8) {
+        const int x = idx & 3;
+        return __byte_perm(sl[idx >> 2], sh[idx >> 2], ((4 + x) << 12) | ((4 + x) << 8) | (x << 4) | x);  // bytes 1, 3: leftovers
+    } else {
+        const int bit = W * idx, wi = bit >> 5, sft = bit & 31;
+        uint32_t lo = sft == 0 ? sl[wi] : (sft + W > 32 ? __funnelshift_r(sl[wi], sl[wi + 1], sft) : sl[wi] >> sft);
+        const uint32_t hi = sft == 0 ? sh[wi] : (sft + W > 32 ? __funnelshift_r(sh[wi], sh[wi + 1], sft) : sh[wi] >> sft);
+        lo &= (1u << W) - 1u;
+        return lo + (hi << 16);  // bits above 16 + W hold leftovers
+    }
+}
+
+template <int W>
+__device__ __forceinline__ void decode_wordcol(const uint32_t (&sl)[W], const uint32_t (&sh)[W], int i, uint32_t F2, uint32_t mm,
+                                               uint32_t (&yw)[16]) {
+    constexpr int M = W - 1;
+    constexpr uint32_t kQ2 = ((1u << M) - 1u) * 0x10001u;
+    const uint32_t sc0 = F2 - ((uint32_t)(M - 1) << 7) * 0x10001u;  // 2^p for tau = 0, per half
+    const uint32_t nb0 = sc0 + 0x83808380u;                         // -128 * 2^p
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        const uint32_t t = (mm << (7 - j)) & 0x00800080u;
+        const uint32_t sc = sc0 - t, nb = nb0 - t;
+#pragma unroll
+        for (int r = 2 * j; r < 2 * j + 2; ++r) {
+            const uint32_t c2 = code_pair_col<W>(sl, sh, 16 * i + r);
+            yw[r] = hfma2((c2 & kQ2) | 0x43004300u, sc, nb) | ((c2 << (15 - M)) & kSign2);
+        }
+    }
+}
+
+// Slow route for block row i of a word column.
+template <int W>
+__device__ __noinline__ TwoBlocksOut decode_wordcol_slow(TwoBlocks<W> lo, TwoBlocks<W> hi, int i, uint32_t F_lo, uint32_t F_hi,
+                                                         uint32_t m_lo, uint32_t m_hi) {
+    TwoBlocksOut o;
+    constexpr int NW = (kSlice * W + 31) / 32;
+    uint32_t yb[2][kSlice];
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+        const uint32_t* s = h ? hi.s : lo.s;
+        uint32_t words[NW + 1];
+#pragma unroll
+        for (int k = 0; k <= NW; ++k) words[k] = 0;
+#pragma unroll
+        for (int k = 0; k < NW; ++k) {
+            const uint32_t a0 = s[k], b0 = (W % 2 == 0) ? s[(W / 2 + k) % W] : __byte_perm(s[(W / 2 + k) % W], W / 2 + k + 1 < W ? s[(W / 2 + k + 1) % W] : 0u, 0x5432);
+            words[k] = i ? b0 : a0;
+        }
+        decode_slice_impl<W, false>(words, (int)(h ? F_hi : F_lo), h ? m_hi : m_lo, yb[h]);
+    }
+#pragma unroll
+    for (int r = 0; r < kSlice; ++r) o.y[r] = (yb[0][r] >> 16) | (yb[1][r] & 0xFFFF0000u);
+    return o;
+}
+
 }  // namespace x2
 }  // namespace bdr
