@@ -162,6 +162,20 @@ int mx_gemm(const bdr_config_t* cfg_a /*host*/, const bdr_planes_t* a /*host str
             const bdr_config_t* cfg_b /*host*/, const bdr_planes_t* b /*host struct*/, int64_t M, int64_t N,
             int64_t K, float* c, int64_t ldc, void* stream);
 
+/* mx_gemm in two phases, for callers that can lend scratch memory: both operands are first decoded to
+ * bf16 in `workspace` (once each, by the unpack kernels), then multiplied by a tensor-core kernel that
+ * streams the bf16 operands with TMA.  mx_gemm decodes inside the GEMM and so repeats the decode of an
+ * operand row for every tile of the other dimension; for large M and N this entry point is the faster
+ * one.  Same result as mx_gemm (only the summation order is unspecified), same format rules.
+ * Needs M and N multiples of 256, K a multiple of 64, and a 256-byte aligned workspace of at least
+ * mx_gemm_workspace_bytes(M, N, K) = 2 (M + N) K bytes (rounded up to 256), whose contents are
+ * overwritten; BDR_ERR_WORKSPACE if it is missing or too small.  Values below bf16's subnormal range
+ * (|v| < 2^-133) are truncated toward zero. */
+int64_t mx_gemm_workspace_bytes(int64_t M, int64_t N, int64_t K);
+int mx_gemm_ws(const bdr_config_t* cfg_a /*host*/, const bdr_planes_t* a /*host struct*/,
+               const bdr_config_t* cfg_b /*host*/, const bdr_planes_t* b /*host struct*/, int64_t M, int64_t N,
+               int64_t K, float* c, int64_t ldc, void* workspace, int64_t workspace_bytes, void* stream);
+
 /* BDR_OK, or BDR_ERR_TIMEOUT if any mx_gemm launch on the current device gave up a bounded wait
  * (sticky).  Host call; synchronises with the device (it copies one word back). */
 int mx_gemm_status(void);

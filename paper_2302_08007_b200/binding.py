@@ -21,7 +21,7 @@ F32, BF16 = 0, 1
 
 EXPORTS = ("bdr_strerror", "bdr_device_status", "bdr_packed_sizes", "bdr_quant_dequant", "bdr_pack", "bdr_unpack",
            "bdr_qsnr_workspace_bytes", "bdr_qsnr", "bdr_qsnr_static_max_cfgs", "bdr_qsnr_static", "mx_gemm",
-           "mx_gemm_status")
+           "mx_gemm_workspace_bytes", "mx_gemm_ws", "mx_gemm_status")
 
 
 class BdrError(RuntimeError):
@@ -103,6 +103,11 @@ def lib():
         L.bdr_qsnr_static.restype = C.c_int
         L.bdr_qsnr_static.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_int, C.c_int64, C.c_int64, C.c_int64, C.c_int,
                                       C.c_void_p, C.c_void_p]
+        L.mx_gemm_workspace_bytes.restype = C.c_int64
+        L.mx_gemm_workspace_bytes.argtypes = [C.c_int64, C.c_int64, C.c_int64]
+        L.mx_gemm_ws.restype = C.c_int
+        L.mx_gemm_ws.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_int64, C.c_int64,
+                                 C.c_void_p, C.c_int64, C.c_void_p, C.c_int64, C.c_void_p]
         L.mx_gemm_status.restype = C.c_int
         L.mx_gemm_status.argtypes = []
         L.bdr_device_status.restype = C.c_int
@@ -232,6 +237,21 @@ def mx_gemm(cfg_a: Config, a: Planes, cfg_b: Config, b: Planes, M: int, N: int, 
     ca, cb, pa, pb = cfg_a.c(), cfg_b.c(), a.c(), b.c()
     _check(lib().mx_gemm(C.addressof(ca), C.addressof(pa), C.addressof(cb), C.addressof(pb), M, N, K, _ptr(c),
                          c.stride(0), _stream(stream)), "mx_gemm")
+    return c
+
+
+def mx_gemm_workspace_bytes(M: int, N: int, K: int) -> int:
+    return int(lib().mx_gemm_workspace_bytes(M, N, K))
+
+
+def mx_gemm_ws(cfg_a: Config, a: Planes, cfg_b: Config, b: Planes, M: int, N: int, K: int, c: torch.Tensor,
+               workspace: torch.Tensor, stream=None):
+    """mx_gemm in two phases: decode both operands once into `workspace` (uint8 device tensor of at least
+    mx_gemm_workspace_bytes(M, N, K) bytes), then a TMA-fed tensor-core GEMM."""
+    ca, cb, pa, pb = cfg_a.c(), cfg_b.c(), a.c(), b.c()
+    _check(lib().mx_gemm_ws(C.addressof(ca), C.addressof(pa), C.addressof(cb), C.addressof(pb), M, N, K, _ptr(c),
+                            c.stride(0), _ptr(workspace), workspace.numel() * workspace.element_size(), _stream(stream)),
+           "mx_gemm_ws")
     return c
 
 

@@ -15,6 +15,8 @@
 // returns.
 #include <cuda.h>
 
+#include <algorithm>
+
 #include "bdr_device.cuh"
 #include "bdr_host.h"
 
@@ -362,6 +364,7 @@ mx_gemm_kernel(bdr_planes_t a, bdr_planes_t b, int64_t M, int64_t N, int64_t K, 
 }  // namespace bdr
 
 #include "mx_gemm_pair.cuh"
+#include "mx_gemm_dense.cuh"
 
 namespace bdr {
 
@@ -430,6 +433,52 @@ int mx_gemm(const bdr_config_t* cfg_a, const bdr_planes_t* a, const bdr_config_t
         case 7: return gemm_pick_b<8>(cfg_b->m, *a, *b, M, N, K, c, ldc, st);
     }
     return BDR_ERR_UNSUPPORTED;
+}
+
+int64_t mx_gemm_workspace_bytes(int64_t M, int64_t N, int64_t K) {
+    if (M < 0 || N < 0 || K < 0) return 0;
+    return ((M + N) * K * 2 + 255) / 256 * 256;
+}
+
+int mx_gemm_ws(const bdr_config_t* cfg_a, const bdr_planes_t* a, const bdr_config_t* cfg_b, const bdr_planes_t* b, int64_t M,
+               int64_t N, int64_t K, float* c, int64_t ldc, void* workspace, int64_t workspace_bytes, void* stream) {
+    if (!cfg_a || !cfg_b || !a || !b || !c) return BDR_ERR_NULL;
+    for (const bdr_config_t* cf : {cfg_a, cfg_b}) {
+        if (cf->scale_kind != BDR_SCALE_POW2) return BDR_ERR_UNSUPPORTED;
+        if (cf->d1 != 8 || cf->k1 < 1 || cf->k2 < 1 || cf->k1 % cf->k2 != 0 || cf->d2 < 0 || cf->d2 > 3 || cf->m < 1 || cf->m > 8)
+            return BDR_ERR_BAD_CONFIG;
+        if (cf->k1 != 16 || cf->k2 != 2 || cf->d2 != 1 || (cf->m != 2 && cf->m != 4 && cf->m != 7)) return BDR_ERR_UNSUPPORTED;
+    }
+    if (M < 0 || N < 0 || K < 0 || ldc < N) return BDR_ERR_SIZE;
+    if (M == 0 || N == 0) return BDR_OK;
+    if (M % 256 || N % 256 || K % kBK || K == 0) return BDR_ERR_UNSUPPORTED;
+    if (M >= (1ll << 31) || N >= (1ll << 31) || K >= (1ll << 31) || (M / 256) * (N / 256) >= (1ll << 30)) return BDR_ERR_UNSUPPORTED;
+    for (const bdr_planes_t* p : {a, b}) {
+        if (!p->exps || !p->micro || !p->elems) return BDR_ERR_NULL;
+        if (((uintptr_t)p->exps | (uintptr_t)p->micro | (uintptr_t)p->elems) % 16) return BDR_ERR_MISALIGNED;
+        if ((p->ld_exps | p->ld_micro | p->ld_elems) % 16) return BDR_ERR_MISALIGNED;
+    }
+    if (a->ld_exps < K / 16 || a->ld_micro < K / 16 || a->ld_elems < K * (cfg_a->m + 1) / 8) return BDR_ERR_SIZE;
+    if (b->ld_exps < K / 16 || b->ld_micro < K / 16 || b->ld_elems < K * (cfg_b->m + 1) / 8) return BDR_ERR_SIZE;
+    if ((uintptr_t)c % 16 || ldc % 4) return BDR_ERR_MISALIGNED;
+    if (!workspace || workspace_bytes < mx_gemm_workspace_bytes(M, N, K)) return BDR_ERR_WORKSPACE;
+    if ((uintptr_t)workspace % 256) return BDR_ERR_MISALIGNED;
+    cudaStream_t st = (cudaStream_t)stream;
+    __nv_bfloat16* wa = static_cast<__nv_bfloat16*>(workspace);
+    __nv_bfloat16* wb = wa + M * K;
+    const bdr_config_t* cfs[2] = {cfg_a, cfg_b};
+    const bdr_planes_t* pls[2] = {a, b};
+    __nv_bfloat16* outs[2] = {wa, wb};
+    const int64_t rows[2] = {M, N};
+    for (int i = 0; i < 2; ++i) {  // phase 1: both operands to bf16, once
+        QParams qp;
+        qp.k1 = 16; qp.k2 = 2; qp.d2 = 1; qp.m = cfs[i]->m; qp.rounding = cfs[i]->rounding; qp.beta = 1; qp.qmax = (1u << cfs[i]->m) - 1u;
+        int rc = unpack_rowwise_mx_x2(*pls[i], outs[i], rows[i], K, K, qp, st);
+        if (rc == BDR_ERR_UNSUPPORTED) rc = unpack_rowwise_mx<__nv_bfloat16>(*pls[i], outs[i], rows[i], K, K, qp, st);
+        if (rc == BDR_ERR_UNSUPPORTED) rc = unpack_general<__nv_bfloat16>(*pls[i], outs[i], rows[i], K, K, 1, qp, st);
+        if (rc != BDR_OK) return rc;
+    }
+    return launch_gemm_dense(wa, wb, M, N, K, c, ldc, st);  // phase 2
 }
 
 int mx_gemm_status(void) {

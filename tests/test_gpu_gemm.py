@@ -121,3 +121,84 @@ def test_gemm_argument_errors():
         bdr.mx_gemm(bdr.MX6, pa, bdr.MX6, pb, 128, 256, 128, c)                       # planes too narrow for K
     assert e.value.status == -5
     torch.cuda.synchronize()
+
+
+# ---- two-phase entry point (decode once into a workspace, then a TMA-fed tensor-core GEMM) ----------------
+def gpu_gemm_ws(cfg_a, a_host, cfg_b, b_host):
+    M, K = a_host.shape
+    N = b_host.shape[0]
+    a, b = torch.from_numpy(a_host).cuda(), torch.from_numpy(b_host).cuda()
+    pa, pb = bdr.alloc_planes(cfg_a, M, K), bdr.alloc_planes(cfg_b, N, K)
+    bdr.bdr_pack(cfg_a, a, pa)
+    bdr.bdr_pack(cfg_b, b, pb)
+    ws = torch.empty(bdr.mx_gemm_workspace_bytes(M, N, K), dtype=torch.uint8, device="cuda")
+    c = torch.full((M, N), float("nan"), dtype=torch.float32, device="cuda")
+    bdr.mx_gemm_ws(cfg_a, pa, cfg_b, pb, M, N, K, c, ws)
+    torch.cuda.synchronize()
+    assert bdr.mx_gemm_status() == 0 and bdr.bdr_device_status() == 0
+    return c.cpu().numpy()
+
+
+def test_ws_exact_case_small_integers():
+    rng = np.random.default_rng(1)
+    a = rng.integers(-8, 9, (256, 128)).astype(np.float32)
+    b = rng.integers(-8, 9, (256, 128)).astype(np.float32)
+    a[:, ::16] = 8.0
+    b[:, ::16] = -8.0
+    c = gpu_gemm_ws(bdr.MX9, a, bdr.MX9, b)
+    assert np.array_equal(c.astype(np.int64), a.astype(np.int64) @ b.astype(np.int64).T)
+
+
+@pytest.mark.parametrize("fa,fb", [("MX6", "MX6"), ("MX9", "MX4"), ("MX4", "MX9")])
+def test_ws_random_operands_match_the_oracle(fa, fb):
+    M, N, K = 512, 768, 1088                             # six tiles, 17 K steps (ring wraps several times)
+    a = synth.normal_matrix(M, K, seed=7, stream=1)
+    b = synth.outlier_channel_matrix(N, K, seed=7, stream=2, gain=20.0, dist="normal", sigma=0.02)
+    c = gpu_gemm_ws(FMT[fa], a, FMT[fb], b)
+    ref = oracle_gemm(FMT[fa], a, FMT[fb], b)
+    assert rel_frob(c, ref) <= 1e-5
+
+
+def test_ws_more_tiles_than_clusters_and_extreme_scales():
+    # 24 x 16 = 384 tiles: every cluster walks over several tiles and both accumulator buffers are reused
+    M, N, K = 6144, 4096, 64
+    a = synth.normal_matrix(M, K, seed=8, stream=1)
+    b = synth.normal_matrix(N, K, seed=8, stream=2, sigma=0.02)
+    c = gpu_gemm_ws(bdr.MX6, a, bdr.MX6, b)
+    ref = oracle_gemm(bdr.MX6, a, bdr.MX6, b)
+    assert rel_frob(c, ref) <= 1e-5
+    for scale in (1e-30, 1e25):
+        b2 = synth.normal_matrix(256, 128, seed=3, sigma=0.02) * np.float32(scale)
+        a2 = synth.outlier_channel_matrix(256, 128, seed=2, gain=50.0)
+        c2 = gpu_gemm_ws(bdr.MX6, a2, bdr.MX9, b2)
+        assert rel_frob(c2, oracle_gemm(bdr.MX6, a2, bdr.MX9, b2)) <= 1e-5, scale
+
+
+def test_ws_config4_shape_on_sampled_entries():
+    M = N = K = 4096
+    a = synth.normal_matrix(M, K, seed=0, stream=10)
+    b = synth.normal_matrix(N, K, seed=0, stream=11, sigma=0.02)
+    c = gpu_gemm_ws(bdr.MX6, a, bdr.MX6, b)
+    aq, _ = orc.quant_dequant(orc.MX6, a, nthreads=8)
+    bq, _ = orc.quant_dequant(orc.MX6, b, nthreads=8)
+    rng = np.random.default_rng(5)
+    ri, ci = rng.integers(0, M, 4096), rng.integers(0, N, 4096)
+    ref = orc.gemm_nt_f64_sampled(aq, bq, ri, ci)
+    got = c[ri, ci].astype(np.float64)
+    assert np.linalg.norm(got - ref) / np.linalg.norm(ref) <= 1e-5
+    assert np.isfinite(c).all()
+    assert rel_frob(c[-256:], orc.gemm_nt_f64(aq[-256:], bq, nthreads=8)) <= 1e-5
+
+
+def test_ws_argument_errors():
+    pa, pb = bdr.alloc_planes(bdr.MX6, 256, 64), bdr.alloc_planes(bdr.MX6, 256, 64)
+    c = torch.empty((256, 256), device="cuda")
+    small = torch.empty(1024, dtype=torch.uint8, device="cuda")
+    with pytest.raises(bdr.BdrError) as e:
+        bdr.mx_gemm_ws(bdr.MX6, pa, bdr.MX6, pb, 256, 256, 64, c, small)               # workspace too small
+    assert e.value.status == -6
+    ws = torch.empty(bdr.mx_gemm_workspace_bytes(256, 256, 64), dtype=torch.uint8, device="cuda")
+    with pytest.raises(bdr.BdrError) as e:
+        bdr.mx_gemm_ws(bdr.MX6, pa, bdr.MX6, pb, 128, 256, 64, c, ws)                  # M must be a multiple of 256
+    assert e.value.status == -3
+    torch.cuda.synchronize()
