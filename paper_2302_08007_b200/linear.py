@@ -25,18 +25,24 @@ class LinearBuffers:
     y: torch.Tensor        # [tokens, out] float32
     dx: torch.Tensor       # [tokens, in] float32
     dw: torch.Tensor       # [out, in] float32
+    workspace: torch.Tensor | None = None  # uint8 scratch for the two-phase GEMM (largest of the three products)
 
 
 ORDER = (("x", 1), ("x", 0), ("w", 1), ("w", 0), ("dy", 1), ("dy", 0))
 
 
-def alloc(cfg: bdr.Config, tokens: int, d_in: int, d_out: int, device="cuda") -> LinearBuffers:
+def alloc(cfg: bdr.Config, tokens: int, d_in: int, d_out: int, device="cuda", two_phase: bool = True) -> LinearBuffers:
     shapes = {"x": (tokens, d_in), "w": (d_out, d_in), "dy": (tokens, d_out)}
     planes = {(n, ax): bdr.alloc_planes(cfg, *shapes[n], ax, device=device) for n, ax in ORDER}
+    ws = None
+    if two_phase and tokens % 256 == 0 and d_in % 256 == 0 and d_out % 256 == 0:
+        nbytes = max(bdr.mx_gemm_workspace_bytes(tokens, d_out, d_in), bdr.mx_gemm_workspace_bytes(tokens, d_in, d_out),
+                     bdr.mx_gemm_workspace_bytes(d_out, d_in, tokens))
+        ws = torch.empty(nbytes, dtype=torch.uint8, device=device)
     return LinearBuffers(planes, torch.zeros((6, 2), dtype=torch.float64, device=device),
                          torch.empty((tokens, d_out), dtype=torch.float32, device=device),
                          torch.empty((tokens, d_in), dtype=torch.float32, device=device),
-                         torch.empty((d_out, d_in), dtype=torch.float32, device=device))
+                         torch.empty((d_out, d_in), dtype=torch.float32, device=device), ws)
 
 
 def step(cfg: bdr.Config, x: torch.Tensor, w: torch.Tensor, dy: torch.Tensor, buf: LinearBuffers, stream=None):
@@ -48,9 +54,16 @@ def step(cfg: bdr.Config, x: torch.Tensor, w: torch.Tensor, dy: torch.Tensor, bu
     for i, (n, ax) in enumerate(ORDER):
         bdr.bdr_pack(cfg, src[n], buf.planes[(n, ax)], axis=ax, qsnr_sums=buf.sums[i], stream=stream)
     p = buf.planes
-    bdr.mx_gemm(cfg, p[("x", 1)], cfg, p[("w", 1)], tokens, d_out, d_in, buf.y, stream=stream)      # Y  = X W^T
-    bdr.mx_gemm(cfg, p[("dy", 1)], cfg, p[("w", 0)], tokens, d_in, d_out, buf.dx, stream=stream)    # dX = dY W
-    bdr.mx_gemm(cfg, p[("dy", 0)], cfg, p[("x", 0)], d_out, d_in, tokens, buf.dw, stream=stream)    # dW = dY^T X
+
+    def gemm(a, b, M, N, K, c):
+        if buf.workspace is not None:
+            bdr.mx_gemm_ws(cfg, a, cfg, b, M, N, K, c, buf.workspace, stream=stream)
+        else:
+            bdr.mx_gemm(cfg, a, cfg, b, M, N, K, c, stream=stream)
+
+    gemm(p[("x", 1)], p[("w", 1)], tokens, d_out, d_in, buf.y)      # Y  = X W^T
+    gemm(p[("dy", 1)], p[("w", 0)], tokens, d_in, d_out, buf.dx)    # dX = dY W
+    gemm(p[("dy", 0)], p[("x", 0)], d_out, d_in, tokens, buf.dw)    # dW = dY^T X
     return buf.y, buf.dx, buf.dw
 
 

@@ -19,21 +19,23 @@ def _inputs(tokens, d_in, d_out, seed):
     return to_bf16(x), to_bf16(w), to_bf16(dy)
 
 
-def _run(cfg, x, w, dy):
+def _run(cfg, x, w, dy, two_phase=True):
     dev = lambda a: torch.from_numpy(a).to(torch.bfloat16).cuda()
-    buf = linear.alloc(cfg, x.shape[0], x.shape[1], w.shape[0])
+    buf = linear.alloc(cfg, x.shape[0], x.shape[1], w.shape[0], two_phase=two_phase)
+    assert (buf.workspace is not None) == two_phase
     y, dx, dw = linear.step(cfg, dev(x), dev(w), dev(dy), buf)
     torch.cuda.synchronize()
     assert bdr.mx_gemm_status() == 0
     return y.cpu().numpy(), dx.cpu().numpy(), dw.cpu().numpy(), linear.qsnr_db(buf), buf
 
 
+@pytest.mark.parametrize("two_phase", [True, False], ids=["mx_gemm_ws", "mx_gemm"])
 @pytest.mark.parametrize("fmt", ["MX9", "MX6"])
-def test_linear_step_small_shapes_full_oracle(fmt):
+def test_linear_step_small_shapes_full_oracle(fmt, two_phase):
     cfg = {"MX9": bdr.MX9, "MX6": bdr.MX6}[fmt]
     o = H.to_orc(cfg)
     x, w, dy = _inputs(512, 256, 768, seed=5)
-    y, dx, dw, q, buf = _run(cfg, x, w, dy)
+    y, dx, dw, q, buf = _run(cfg, x, w, dy, two_phase)
     qd = lambda a, ax: orc.quant_dequant(o, a, axis=ax)
     (xr, sxr), (xc, sxc) = qd(x, 1), qd(x, 0)
     (wr, swr), (wc, swc) = qd(w, 1), qd(w, 0)
