@@ -221,7 +221,9 @@ __device__ __forceinline__ void pack_pair_view(const PairView& v, uint32_t F, ui
             rB = hsub2(rB, (v.B[i] & kSign2) | 0x3F803F80u);
             constexpr uint32_t kCode = ((1u << W) - 1u) * 0x10001u;
             const uint32_t comb = (rA & kCode) + ((rB & kCode) << W);  // halves: codes 4i, 4i+1 | codes 4i+2, 4i+3
-            f4[i] = (comb | (comb >> (16 - 2 * W))) & ((1u << (4 * W)) - 1u);
+            // the two halves side by side: 4 codes, 4W bits
+            if constexpr (3 * W <= 10) f4[i] = (comb | (comb >> (16 - 2 * W))) & ((1u << (4 * W)) - 1u);  // shifted low half falls off
+            else f4[i] = (comb & ((1u << (2 * W)) - 1u)) | ((comb >> (16 - 2 * W)) & (((1u << (2 * W)) - 1u) << (2 * W)));
         } else {
             // W = 8: byte 0 / 2 of each word = sign bit over the seven magnitude bits; bytes 1 / 3 are not used
             const uint32_t cA = ((v.A[i] >> 8) & 0x00800080u) | (rA & ~0x00800080u);

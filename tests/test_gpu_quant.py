@@ -206,3 +206,97 @@ def test_bounded_waits_never_ran_out():
     bdr.bdr_pack(cfg, xd, planes, y_dq=y)
     torch.cuda.synchronize()
     assert bdr.bdr_device_status() == 0
+
+
+# ---- bf16 fast paths (packed bf16x2 arithmetic): every output combination, exponent-range boundaries ----
+def _boundary_input(rows, cols, seed):
+    """bf16-exact values whose 16-element blocks (in both directions: the tile is constant over 16 x 16
+    patches) have their largest exponent field at and around the limits of the packed-arithmetic range."""
+    rng = np.random.default_rng(seed)
+    fields = np.array([1, 8, 14, 15, 16, 17, 18, 100, 127, 200, 238, 239, 240, 241, 242, 248, 249, 250, 251, 252, 254])
+    pr, pc = rows // 16, cols // 16
+    f = fields[rng.integers(0, len(fields), (pr, pc))]
+    scale = np.ldexp(1.0, (f - 127).astype(np.int64)).astype(np.float64)       # 2^(F-127) per patch
+    scale = np.kron(scale, np.ones((16, 16)))
+    mant = 1.0 + rng.integers(0, 128, (rows, cols)) / 128.0                         # 8-bit significands in [1, 2)
+    down = np.ldexp(1.0, -rng.integers(0, 12, (rows, cols)).astype(np.int64))        # most elements below the block maximum
+    sign = np.where(rng.random((rows, cols)) < 0.5, -1.0, 1.0)
+    x = sign * mant * down * scale
+    x[::16, ::16] = np.abs(mant[::16, ::16] * scale[::16, ::16])                       # one element per patch carries the exponent
+    x[1::16, 3::16] = 0.0
+    x[2::16, 5::16] = -0.0
+    x = x.astype(np.float32)
+    x = synth.bf16_bits_to_f32(synth.f32_to_bf16_bits(x)).reshape(rows, cols)
+    return np.where(np.isfinite(x), x, np.float32(1.0)).astype(np.float32)
+
+
+@pytest.mark.parametrize("axis", [1, 0])
+@pytest.mark.parametrize("name", list(MX))
+def test_bf16_fast_paths_every_output_combination(name, axis):
+    cfg = MX[name]
+    rows, cols = 256, 2048
+    for kind in ("laplace_outliers", "boundary", "edge"):
+        x = _boundary_input(rows, cols, seed=77) if kind == "boundary" else H.make_input(kind, rows, cols, "bf16", seed=33)
+        want, so = orc.quant_dequant(H.to_orc(cfg), x, axis=axis)
+        want_planes = orc.pack(H.to_orc(cfg), x, axis=axis)
+        xd = H.host_to_device(x, "bf16")
+        for with_y in (False, True):
+            for with_sums in (False, True):
+                what = "%s axis=%d %s y=%s sums=%s" % (name, axis, kind, with_y, with_sums)
+                y = torch.full_like(xd, 5.0) if with_y else None
+                sums = torch.zeros(2, dtype=torch.float64, device="cuda") if with_sums else None
+                planes = bdr.alloc_planes(cfg, rows, cols, axis)
+                for p in (planes.exps, planes.micro, planes.elems):
+                    p.fill_(0xA5)
+                bdr.bdr_pack(cfg, xd, planes, axis=axis, y_dq=y, qsnr_sums=sums)
+                torch.cuda.synchronize()
+                H.assert_planes_equal(H.planes_to_host(planes), want_planes, what)
+                if with_y:
+                    H.assert_bits_equal(H.device_to_host_f32(y), want, what + " y_dq")
+                if with_sums:
+                    H.assert_qsnr_close(sums.cpu().numpy(), so, what)
+                if with_y or with_sums:
+                    y2 = torch.full_like(xd, 5.0) if with_y else None
+                    s2 = torch.zeros(2, dtype=torch.float64, device="cuda") if with_sums else None
+                    bdr.bdr_quant_dequant(cfg, xd, y2, axis=axis, qsnr_sums=s2)
+                    torch.cuda.synchronize()
+                    if with_y:
+                        H.assert_bits_equal(H.device_to_host_f32(y2), want, what + " quant_dequant")
+                    if with_sums:
+                        H.assert_qsnr_close(s2.cpu().numpy(), so, what + " quant_dequant")
+        back = torch.full_like(xd, 7.0)
+        bdr.bdr_unpack(cfg, planes, back, axis=axis)
+        torch.cuda.synchronize()
+        H.assert_bits_equal(H.device_to_host_f32(back), want, "%s axis=%d %s unpack" % (name, axis, kind))
+    assert bdr.bdr_device_status() == 0
+
+
+@pytest.mark.parametrize("m", [1, 3, 5, 6])
+def test_bf16_quant_dequant_other_mantissa_widths(m):
+    # the packed-arithmetic quantize-dequantize kernels take any m <= 7 of the k1 = 16, k2 = 2, d2 = 1 family
+    cfg = Cfg(16, 8, 2, 1, m)
+    x = _boundary_input(256, 2048, seed=m)
+    for axis in (1, 0):
+        y, sums = run_quant(cfg, x, "bf16", axis=axis)
+        want, so = orc.quant_dequant(H.to_orc(cfg), x, axis=axis)
+        H.assert_bits_equal(y, want, "%s axis=%d" % (cfg, axis))
+        H.assert_qsnr_close(sums, so, "%s axis=%d" % (cfg, axis))
+
+
+def test_bf16_fast_paths_with_a_row_pitch():
+    # rows of 2048 elements that are 2112 elements apart: the run index splits into (row, position)
+    rows, cols, ld = 5, 2048, 2112
+    x = H.make_input("laplace_outliers", rows, cols, "bf16", seed=12)
+    for cfg in (bdr.MX4, bdr.MX9):
+        y, sums = run_quant(cfg, x, "bf16", ld=ld)
+        want, so = orc.quant_dequant(H.to_orc(cfg), x)
+        H.assert_bits_equal(y, want, "%s pitch" % (cfg,))
+        H.assert_qsnr_close(sums, so)
+        xd = H.host_to_device(x, "bf16", ld)
+        planes = bdr.alloc_planes(cfg, rows, cols, 1)
+        bdr.bdr_pack(cfg, xd, planes)
+        back = H.host_to_device(np.zeros_like(x), "bf16", ld)
+        bdr.bdr_unpack(cfg, planes, back)
+        torch.cuda.synchronize()
+        H.assert_planes_equal(H.planes_to_host(planes), orc.pack(H.to_orc(cfg), x), "%s pitch" % (cfg,))
+        H.assert_bits_equal(H.device_to_host_f32(back), want, "%s pitch unpack" % (cfg,))
