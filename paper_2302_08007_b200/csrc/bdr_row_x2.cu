@@ -143,12 +143,7 @@ row_mx_x2_kernel(const bf16* x, bf16* y, RunIndex ri, uint32_t total, bdr_planes
                     } else {
                         float pe = 0.f, ps = 0.f;
                         uint32_t code2[8];
-#ifdef BDR_X2_NOMATH
-                        for (int j = 0; j < 8; ++j) yw[j] = w[j] + 1;
-                        pe = __uint_as_float(w[0]); ps = __uint_as_float(w[1]);
-#else
                         x2::quantize_block_row<SUMS, YOUT, PACK>(w, aw, F, m, k, yw, code2, mbs[s], pe, ps);
-#endif
                         if constexpr (PACK) {
                             x2::pack_block<PACK ? W : 8>(code2, cw[s]);
                             Fs[s] = F;
