@@ -21,23 +21,29 @@ __device__ __forceinline__ void words_of(const uint4& v0, const uint4& v1, uint3
     w[4] = v1.x; w[5] = v1.y; w[6] = v1.z; w[7] = v1.w;
 }
 
-// Per-warp pipeline.  A warp streams runs of 2048 elements (4 KB) through two stages in shared memory:
-// lane 0 refills a stage with one bulk copy as soon as the warp has consumed it, so two runs per warp
-// (and with ~20 warps per SM well over 100 KB per SM) are in flight.  A run is handled as two halves
-// of 1024 elements; in each a lane owns 64 consecutive bytes (two blocks).  Dequantized values go
-// straight from registers to global memory (one 32-byte store per block); the packed planes of a
-// run are collected per warp in a small double-buffered staging area and leave with one bulk store
-// each (256 W code bytes, 128 exponent bytes, 128 microexponent bytes).
+// Per-warp pipeline.  A warp streams runs of 2048 elements (4 KB) through a small ring in shared memory:
+// lane 0 keeps two runs in flight with one bulk copy each (with ~16-24 warps per SM, well over 100 KB per
+// SM).  A run is handled as two halves of 1024 elements; in each a lane owns 64 consecutive bytes (two
+// blocks).  Dequantized values are written back over the run's input in its stage and leave with one
+// bulk store of 4 KB (measured: faster than 32-byte stores from registers); the packed planes of a run
+// are collected per warp in a small double-buffered staging area and leave with one bulk store each
+// (256 W code bytes, 128 exponent bytes, 128 microexponent bytes).  Bulk stores are grouped per run;
+// "all but the latest group have been read" frees what the previous run used.
 constexpr int kX2Threads = 128;
 constexpr int kX2Warps = kX2Threads / 32;
-constexpr int kX2Stages = 2;
+constexpr int kX2Ahead = 2;  // runs in flight per warp
 constexpr int kX2Sub = 2;                                    // halves per run
 constexpr int kSubElems = 32 * kX2SPT * kSlice;              // 1024
 constexpr int kX2RunElems = kX2Sub * kSubElems;              // 2048
 constexpr int kRunBytes = kX2RunElems * 2;
-constexpr int kX2RingBytes = kX2Warps * kX2Stages * kRunBytes;
-constexpr int kX2BarBytes = 128;  // kX2Warps * kX2Stages barriers of 8 bytes, padded
-static_assert(kX2Warps * kX2Stages * 8 <= kX2BarBytes, "barrier area");
+// Stages per warp: with dequantized output the results are written back into the stage they came from and
+// leave with a bulk store, so a third stage is needed while that store drains.
+template <bool YOUT> struct X2Ring {
+    static constexpr int kStages = YOUT ? kX2Ahead + 1 : kX2Ahead;
+    static constexpr int kBytes = kX2Warps * kStages * kRunBytes;
+};
+constexpr int kX2BarBytes = 128;  // barriers of 8 bytes, padded
+static_assert(kX2Warps * (kX2Ahead + 1) * 8 <= kX2BarBytes, "barrier area");
 
 template <int W> struct X2PackStage {
     static constexpr int kElemBytes = kX2RunElems / 8 * W;
@@ -69,12 +75,6 @@ struct RunIndex {
     }
 };
 
-__device__ __forceinline__ void stg256(void* p, const uint32_t (&v)[8]) {
-    asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(p), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]),
-                 "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7])
-                 : "memory");
-}
-
 // W = 0: quantize-dequantize (any m <= 7, from qp); W = m + 1: also write the packed planes.
 template <int W, bool SUMS, bool YOUT>
 __global__ void __launch_bounds__(kX2Threads)
@@ -82,7 +82,8 @@ row_mx_x2_kernel(const bf16* x, bf16* y, RunIndex ri, uint32_t total, bdr_planes
     using PS = X2PackStage<W>;
     constexpr bool PACK = W > 0;
     constexpr bool kPackOnly = PACK && !SUMS && !YOUT;
-    constexpr int S = kX2Stages;
+    constexpr int S = X2Ring<YOUT>::kStages;
+    constexpr int kX2RingBytes = X2Ring<YOUT>::kBytes;
     constexpr int NCW = PACK ? (16 * W + 31) / 32 : 1;  // words of one block's codes (the last one half full when W is odd)
     extern __shared__ __align__(128) uint8_t smem[];  // ring [warp][stage][4 KB], barriers, staging [warp][2]
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -98,7 +99,7 @@ row_mx_x2_kernel(const bf16* x, bf16* y, RunIndex ri, uint32_t total, bdr_planes
         for (int s = 0; s < S; ++s) async::mbar_init(bars + 8 * s, 1);
         async::fence_barrier_init();
 #pragma unroll
-        for (int s = 0; s < S; ++s) {
+        for (int s = 0; s < kX2Ahead; ++s) {
             const uint32_t wi = w0 + s * stride;
             if (wi < total) {
                 async::mbar_expect_tx(bars + 8 * s, kRunBytes);
@@ -116,8 +117,6 @@ row_mx_x2_kernel(const bf16* x, bf16* y, RunIndex ri, uint32_t total, bdr_planes
             break;
         }
         const uint32_t stage = stage0 + half * PS::kBytes;
-        bf16* yrun = nullptr;
-        if constexpr (YOUT) yrun = y + ri.elem_offset(wi) + lane * 32;
 #pragma unroll
         for (int sub = 0; sub < kX2Sub; ++sub) {
             const uint32_t mine = ring0 + st * kRunBytes + sub * (kSubElems * 2) + lane * 64;
@@ -168,7 +167,10 @@ row_mx_x2_kernel(const bf16* x, bf16* y, RunIndex ri, uint32_t total, bdr_planes
                         yw[4] = o.y[1].x; yw[5] = o.y[1].y; yw[6] = o.y[1].z; yw[7] = o.y[1].w;
                     }
                 }
-                if constexpr (YOUT) stg256(yrun + sub * kSubElems + 16 * s, yw);
+                if constexpr (YOUT) {  // back into the stage, over the block's input
+                    async::sts128(mine + 32 * s, make_uint4(yw[0], yw[1], yw[2], yw[3]));
+                    async::sts128(mine + 32 * s + 16, make_uint4(yw[4], yw[5], yw[6], yw[7]));
+                }
             }
             if constexpr (PACK) {
                 // the lane's 32 codes as W words: block 1 follows block 0 at bit 16 W
@@ -187,9 +189,16 @@ row_mx_x2_kernel(const bf16* x, bf16* y, RunIndex ri, uint32_t total, bdr_planes
                 async::sts16(stage + PS::kElemBytes + PS::kExpBytes + sub * (kSubElems / 16) + 2 * lane, mbs[0] | (mbs[1] << 8));
             }
         }
-        if constexpr (PACK) async::fence_proxy_async();
+        if constexpr (PACK || YOUT) async::fence_proxy_async();
         __syncwarp();  // every lane has consumed stage st (and filled the staging half)
         if (lane == 0) {
+            if constexpr (YOUT) {
+                async::bulk_store(y + ri.elem_offset(wi), ring0 + st * kRunBytes, kRunBytes);
+                if constexpr (!PACK) {
+                    async::bulk_commit();
+                    async::bulk_wait_read<1>();  // the previous run's store has left its stage, which is refilled below
+                }
+            }
             if constexpr (PACK) {
                 int64_t row, pos;
                 ri.split(wi, row, pos);
@@ -200,16 +209,17 @@ row_mx_x2_kernel(const bf16* x, bf16* y, RunIndex ri, uint32_t total, bdr_planes
                 async::bulk_commit();
                 async::bulk_wait_read<1>();  // the other staging half (used next) has been read out
             }
-            const uint32_t next = wi + S * stride;
+            const uint32_t next = wi + kX2Ahead * stride;
+            const int nst = st + kX2Ahead >= S ? st + kX2Ahead - S : st + kX2Ahead;  // YOUT: the previous run's stage; else this one
             if (next < total) {
-                async::mbar_expect_tx(bars + 8 * st, kRunBytes);
-                async::bulk_load(ring0 + st * kRunBytes, x + ri.elem_offset(next), kRunBytes, bars + 8 * st);
+                async::mbar_expect_tx(bars + 8 * nst, kRunBytes);
+                async::bulk_load(ring0 + nst * kRunBytes, x + ri.elem_offset(next), kRunBytes, bars + 8 * nst);
             }
         }
         half ^= 1;
         if (++st == S) { st = 0; phase ^= 1; }
     }
-    if (PACK && lane == 0) async::bulk_wait_all();
+    if ((PACK || YOUT) && lane == 0) async::bulk_wait_all();
     if (SUMS) block_accumulate_sums(e2, s2, sums);
 }
 
@@ -238,7 +248,7 @@ static int launch_x2(const bf16* x, bf16* y, int64_t rows, int64_t cols, int64_t
     if (total == 0) return BDR_OK;
     if (total >= (1ll << 31) - (1ll << 24)) return BDR_ERR_UNSUPPORTED;  // 32-bit run indices (incl. look-ahead)
     auto kern = row_mx_x2_kernel<W, SUMS, YOUT>;
-    const size_t smem = kX2RingBytes + kX2BarBytes + kX2Warps * 2 * X2PackStage<W>::kBytes;
+    const size_t smem = X2Ring<YOUT>::kBytes + kX2BarBytes + kX2Warps * 2 * X2PackStage<W>::kBytes;
     static bool attr_done = false;  // per instantiation; the attribute is idempotent, so a race is harmless
     if (!attr_done) {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return BDR_ERR_CUDA;
