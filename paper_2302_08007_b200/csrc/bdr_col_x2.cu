@@ -27,8 +27,13 @@ constexpr int kCTileCols = 128;
 constexpr int kCTileBlocks = 2 * kCWarps;  // 16 block rows = 256 rows
 constexpr int kCTileRows = kCTileBlocks * kSlice;
 constexpr int kCBoxBytes = kSlice * kCTileCols * 2;  // 4 KB
-constexpr int kCRingBytes = kCWarps * 2 * kCBoxBytes;
-constexpr int kCBarBytes = 128;
+// Stages per warp: two boxes are kept in flight; with dequantized output the results are written back into
+// the box they came from and leave with one TMA tile store, so a third stage is needed while it drains.
+template <bool YOUT> struct CRing {
+    static constexpr int kStages = YOUT ? 3 : 2;
+    static constexpr int kBytes = kCWarps * kStages * kCBoxBytes;
+};
+constexpr int kCBarBytes = 256;
 
 template <int W> struct CStage {
     // codes: W even: [block row 16][column 128] items of 2W bytes, columns XOR-swizzled by the block row;
@@ -53,40 +58,51 @@ __device__ __forceinline__ uint32_t lds8(uint32_t addr) {
     asm volatile("ld.shared.u8 %0, [%1];" : "=r"(v) : "r"(addr) : "memory");
     return v;
 }
+__device__ __forceinline__ void sts64(uint32_t addr, uint32_t a, uint32_t b) {
+    asm volatile("st.shared.v2.b32 [%0], {%1, %2};" ::"r"(addr), "r"(a), "r"(b) : "memory");
+}
+// shared (dense box) -> 2-D tile of a tensor map; joins the issuing thread's current bulk group
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, int x, int y, uint32_t smem_src) {
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];" ::"l"(map), "r"(x), "r"(y), "r"(smem_src)
+                 : "memory");
+}
 __device__ __forceinline__ double pow4_weight_col(uint32_t F) { return __hiloint2double((int)((F << 21) + 0x30100000u), 0); }
 
 // W = 0: quantize-dequantize / sums only (any m <= 7, from qp); W = m + 1: also write the packed planes.
 template <int W, bool SUMS, bool YOUT>
 __global__ void __launch_bounds__(kCThreads, 2)
-col_mx_x2_kernel(const __grid_constant__ CUtensorMap xmap, bf16* y, int64_t ld, int n_col_tiles, int n_tiles, bdr_planes_t out,
-                 QParams qp, double* sums, int* status) {
+col_mx_x2_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ CUtensorMap ymap, int n_col_tiles, int n_tiles,
+                 bdr_planes_t out, QParams qp, double* sums, int* status) {
     using CS = CStage<W>;
     constexpr bool PACK = W > 0;
     constexpr int NCW = PACK ? (16 * W + 31) / 32 : 1;
-    extern __shared__ __align__(128) uint8_t smem[];  // ring [warp][2][4 KB], barriers, staging
+    constexpr int S = CRing<YOUT>::kStages;
+    constexpr int kCRingBytes = CRing<YOUT>::kBytes;
+    extern __shared__ __align__(128) uint8_t smem[];  // ring [warp][stage][4 KB], barriers, staging
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const uint32_t ring0 = async::smem_u32(smem) + warp * 2 * kCBoxBytes;
-    const uint32_t bars = async::smem_u32(smem) + kCRingBytes + warp * 16;
+    const uint32_t ring0 = async::smem_u32(smem) + warp * S * kCBoxBytes;
+    const uint32_t bars = async::smem_u32(smem) + kCRingBytes + warp * 32;
     const uint32_t st_elems = async::smem_u32(smem) + kCRingBytes + kCBarBytes;
     const uint32_t st_exps = st_elems + CS::kElemBytes, st_micro = st_exps + CS::kExpBytes;
     const int m = PACK ? W - 1 : qp.m;
 
-    auto issue = [&](int t, int i) {  // box of block row 2*warp+i of tile t into stage i (lane 0 only)
+    auto issue = [&](int t, int i, int stg) {  // box of block row 2*warp+i of tile t into stage stg (lane 0 only)
         const int rt = t / n_col_tiles, ct = t - rt * n_col_tiles;
-        async::mbar_expect_tx(bars + 8 * i, kCBoxBytes);
-        async::tma_load_2d(ring0 + i * kCBoxBytes, &xmap, ct * kCTileCols, rt * kCTileRows + (2 * warp + i) * kSlice, bars + 8 * i);
+        async::mbar_expect_tx(bars + 8 * stg, kCBoxBytes);
+        async::tma_load_2d(ring0 + stg * kCBoxBytes, &xmap, ct * kCTileCols, rt * kCTileRows + (2 * warp + i) * kSlice, bars + 8 * stg);
     };
     if (lane == 0) {
-        async::mbar_init(bars, 1);
-        async::mbar_init(bars + 8, 1);
+#pragma unroll
+        for (int k = 0; k < S; ++k) async::mbar_init(bars + 8 * k, 1);
         async::fence_barrier_init();
         if ((int)blockIdx.x < n_tiles) {
-            issue(blockIdx.x, 0);
-            issue(blockIdx.x, 1);
+            issue(blockIdx.x, 0, 0);
+            issue(blockIdx.x, 1, 1);
         }
     }
     __syncwarp();
     uint32_t phase = 0;
+    int stg = 0;  // stage of the current step; steps alternate between the tile's two block rows
     double e2 = 0.0, s2 = 0.0;
     bool failed = false;
     for (int t = blockIdx.x; t < n_tiles; t += gridDim.x) {
@@ -95,20 +111,22 @@ col_mx_x2_kernel(const __grid_constant__ CUtensorMap xmap, bf16* y, int64_t ld, 
 #pragma unroll
         for (int i = 0; i < 2; ++i) {
             const int bl = 2 * warp + i;
-            if (!failed && !async::mbar_wait(bars + 8 * i, phase)) {
+            if (!failed && !async::mbar_wait(bars + 8 * stg, phase)) {
                 async::report_timeout(status);
                 failed = true;
             }
             uint32_t wc[2][16];
-            const uint32_t mine = ring0 + i * kCBoxBytes + lane * 8;
+            const uint32_t mine = ring0 + stg * kCBoxBytes + lane * 8;
 #pragma unroll
             for (int r = 0; r < kSlice; ++r) {
                 const uint2 v = lds64(mine + r * (kCTileCols * 2));
                 wc[0][r] = v.x;
                 wc[1][r] = v.y;
             }
-            __syncwarp();  // every lane has read stage i
-            if (lane == 0 && !failed && t + (int)gridDim.x < n_tiles) issue(t + gridDim.x, i);
+            if constexpr (!YOUT) {
+                __syncwarp();  // every lane has read the stage: refill it with the same block row of the next tile
+                if (lane == 0 && !failed && t + (int)gridDim.x < n_tiles) issue(t + gridDim.x, i, stg);
+            }
             uint32_t Fb[4], Mb[4];
 #pragma unroll
             for (int c = 0; c < 2; ++c) {  // the lane's two word columns
@@ -173,16 +191,25 @@ col_mx_x2_kernel(const __grid_constant__ CUtensorMap xmap, bf16* y, int64_t ld, 
                 }
             }
             if constexpr (YOUT) {
-                bf16* py = y + ((int64_t)rt * kCTileRows + bl * kSlice) * ld + (int64_t)ct * kCTileCols + 4 * lane;
+                // results over the box's input, then one tile store; the stage of the previous step (whose store
+                // has been read out by then) takes the box two steps ahead
 #pragma unroll
-                for (int r = 0; r < kSlice; ++r) *reinterpret_cast<uint2*>(py + r * ld) = make_uint2(wc[0][r], wc[1][r]);
+                for (int r = 0; r < kSlice; ++r) sts64(mine + r * (kCTileCols * 2), wc[0][r], wc[1][r]);
+                async::fence_proxy_async();
+                __syncwarp();
+                if (lane == 0) {
+                    tma_store_2d(&ymap, ct * kCTileCols, rt * kCTileRows + bl * kSlice, ring0 + stg * kCBoxBytes);
+                    async::bulk_commit();
+                    async::bulk_wait_read<1>();
+                    if (!failed && t + (int)gridDim.x < n_tiles) issue(t + gridDim.x, i, stg + 2 >= S ? stg + 2 - S : stg + 2);
+                }
             }
             if constexpr (PACK) {
                 async::sts32(st_exps + bl * kCTileCols + 4 * lane, Fb[0] | (Fb[1] << 8) | (Fb[2] << 16) | (Fb[3] << 24));
                 async::sts32(st_micro + bl * kCTileCols + 4 * lane, Mb[0] | (Mb[1] << 8) | (Mb[2] << 16) | (Mb[3] << 24));
             }
+            if (++stg == S) { stg = 0; phase ^= 1; }
         }
-        phase ^= 1;
         if constexpr (PACK) {
             __syncthreads();
             // codes: column c of the tile owns 32 W contiguous bytes of its plane line = 2W vectors of 16 bytes
@@ -218,6 +245,7 @@ col_mx_x2_kernel(const __grid_constant__ CUtensorMap xmap, bf16* y, int64_t ld, 
             __syncthreads();
         }
     }
+    if (YOUT && lane == 0) async::bulk_wait_all();
     if (SUMS) block_accumulate_sums(e2, s2, sums);
 }
 
@@ -226,7 +254,7 @@ template <int W, bool SUMS, bool YOUT>
 static int launch_col_x2(const bf16* x, bf16* y, int64_t rows, int64_t cols, int64_t ld, const bdr_planes_t* out,
                          const QParams& qp, double* sums, cudaStream_t st) {
     auto kern = col_mx_x2_kernel<W, SUMS, YOUT>;
-    const size_t smem = kCRingBytes + kCBarBytes + CStage<W>::kBytes;
+    const size_t smem = CRing<YOUT>::kBytes + kCBarBytes + CStage<W>::kBytes;
     static bool attr_done = false;  // per instantiation; the attribute is idempotent, so a race is harmless
     static int blocks_per_sm = 0;
     if (!attr_done) {
@@ -238,14 +266,15 @@ static int launch_col_x2(const bf16* x, bf16* y, int64_t rows, int64_t cols, int
     }
     int* status = device_status_word();
     if (!status) return BDR_ERR_CUDA;
-    CUtensorMap xmap;
+    CUtensorMap xmap, ymap;
     if (!make_tensor_map_u16(&xmap, x, rows, cols, ld, kCTileCols, kSlice)) return BDR_ERR_CUDA;
+    if (!make_tensor_map_u16(&ymap, y ? y : x, rows, cols, ld, kCTileCols, kSlice)) return BDR_ERR_CUDA;
     const int n_ct = (int)(cols / kCTileCols);
     const int64_t n_tiles = (int64_t)n_ct * (rows / kCTileRows);
     bdr_planes_t pl = {};
     if (out) pl = *out;
     const int grid = (int)std::min<int64_t>(n_tiles, (int64_t)sm_count() * blocks_per_sm);
-    kern<<<grid, kCThreads, smem, st>>>(xmap, y, ld, n_ct, (int)n_tiles, pl, qp, sums, status);
+    kern<<<grid, kCThreads, smem, st>>>(xmap, ymap, n_ct, (int)n_tiles, pl, qp, sums, status);
     return cudaGetLastError() == cudaSuccess ? BDR_OK : BDR_ERR_CUDA;
 }
 
@@ -265,7 +294,7 @@ int quant_colwise_mx_x2(const bf16* x, bf16* y, int64_t rows, int64_t cols, int6
                         const QParams& qp, double* sums, cudaStream_t st) {
     if (qp.k1 != 16 || qp.k2 != 2 || qp.d2 != 1 || qp.m > 7 || qp.rounding != BDR_ROUND_NEAREST_EVEN) return BDR_ERR_UNSUPPORTED;
     if (rows % kCTileRows != 0 || cols % kCTileCols != 0) return BDR_ERR_UNSUPPORTED;
-    if (((uintptr_t)x % 16) || ((uintptr_t)y % 8) || (ld * 2) % 16) return BDR_ERR_UNSUPPORTED;
+    if ((((uintptr_t)x | (uintptr_t)y) % 16) || (ld * 2) % 16) return BDR_ERR_UNSUPPORTED;
     if ((int64_t)(cols / kCTileCols) * (rows / kCTileRows) >= (1ll << 30) || rows >= (1ll << 31) || cols >= (1ll << 31)) return BDR_ERR_UNSUPPORTED;
     if (!out) return col_x2_flags<0>(x, y, rows, cols, ld, out, qp, sums, st);
     switch (qp.m) {
