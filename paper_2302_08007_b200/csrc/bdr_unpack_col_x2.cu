@@ -24,6 +24,9 @@ constexpr int kUCTileRows = kUCTileBlocks * kSlice;
 
 template <int W> struct UCStage {
     static constexpr int kPitch = kUCTileBlocks * 2 * W + 16;  // code bytes of one column, padded so columns spread over banks
+    // Column c is kept in row (c % 4) * 32 + c / 4: the lanes of a warp (four adjacent columns each) then read
+    // from 32 consecutive rows, i.e. from different banks, when they fetch "their k-th column".
+    __host__ __device__ static constexpr int row_of(int c) { return (c & 3) * 32 + (c >> 2); }
     static constexpr int kElemBytes = kUCTileCols * kPitch;
     static constexpr int kExpBytes = kUCTileCols * 16;
     static constexpr int kBytes = kElemBytes + 2 * kExpBytes;
@@ -56,13 +59,13 @@ unpack_col_x2_kernel(bdr_planes_t in, bf16* y, int64_t ld, int n_col_tiles, int 
         const uint32_t b = base + buf * ST::kBytes;
         for (int idx = threadIdx.x; idx < kUCTileCols * 2 * W; idx += kUCThreads) {
             const int c = idx / (2 * W), v = idx - c * (2 * W);
-            uc_cp16(b + c * ST::kPitch + v * 16, in.elems + ((int64_t)ct * kUCTileCols + c) * in.ld_elems + blk0 * 2 * W + v * 16);
+            uc_cp16(b + ST::row_of(c) * ST::kPitch + v * 16, in.elems + ((int64_t)ct * kUCTileCols + c) * in.ld_elems + blk0 * 2 * W + v * 16);
         }
         for (int idx = threadIdx.x; idx < kUCTileCols * 2; idx += kUCThreads) {
             const int c = idx & (kUCTileCols - 1), which = idx / kUCTileCols;
             const uint8_t* src = which ? in.micro + ((int64_t)ct * kUCTileCols + c) * in.ld_micro
                                        : in.exps + ((int64_t)ct * kUCTileCols + c) * in.ld_exps;
-            uc_cp16(b + ST::kElemBytes + which * ST::kExpBytes + c * 16, src + blk0);
+            uc_cp16(b + ST::kElemBytes + which * ST::kExpBytes + ST::row_of(c) * 16, src + blk0);
         }
     };
     int buf = 0;
@@ -79,7 +82,7 @@ unpack_col_x2_kernel(bdr_planes_t in, bf16* y, int64_t ld, int n_col_tiles, int 
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
             const int col = 4 * lane + c;
-            const uint32_t src = b + col * ST::kPitch + warp * 4 * W;
+            const uint32_t src = b + ST::row_of(col) * ST::kPitch + warp * 4 * W;
             if constexpr (W == 8) {
                 const uint4 a0 = async::lds128(src), a1 = async::lds128(src + 16);
                 s[c][0] = a0.x; s[c][1] = a0.y; s[c][2] = a0.z; s[c][3] = a0.w;
@@ -88,8 +91,8 @@ unpack_col_x2_kernel(bdr_planes_t in, bf16* y, int64_t ld, int n_col_tiles, int 
 #pragma unroll
                 for (int k = 0; k < W; ++k) s[c][k] = uc_lds32(src + 4 * k);
             }
-            Fp[c] = uc_lds16(b + ST::kElemBytes + col * 16 + 2 * warp);
-            mp[c] = uc_lds16(b + ST::kElemBytes + ST::kExpBytes + col * 16 + 2 * warp);
+            Fp[c] = uc_lds16(b + ST::kElemBytes + ST::row_of(col) * 16 + 2 * warp);
+            mp[c] = uc_lds16(b + ST::kElemBytes + ST::kExpBytes + ST::row_of(col) * 16 + 2 * warp);
         }
 #pragma unroll
         for (int i = 0; i < 2; ++i) {  // block rows 2*warp and 2*warp + 1
