@@ -36,15 +36,15 @@ FALLBACK_HBM_GBS = 6650.0
 # profiles/step_kernels_dram_traffic.md.  Writes that still sit in L2 when a kernel ends are not
 # counted by those counters, which is why some figures are below the algorithmic bytes.
 NCU_TRAFFIC_BYTES: dict[str, float | None] = {
-    "quant_dequant_MX4_row": 217688576, "quant_dequant_MX4_col": 221876480,
-    "quant_dequant_MX6_row": 216988160, "quant_dequant_MX6_col": 221636352,
-    "quant_dequant_MX9_row": 216802304, "quant_dequant_MX9_col": 222077952,
-    "pack_MX4_row": 150532096, "pack_MX4_col": 148491520,
-    "pack_MX6_row": 159283968, "pack_MX6_col": 157008640,
-    "pack_MX9_row": 173592832, "pack_MX9_col": 172875264,
-    "unpack_MX4_row": 108700416, "unpack_MX4_col": 107778816,
-    "unpack_MX6_row": 125882112, "unpack_MX6_col": 124492032,
-    "unpack_MX9_row": 153894656, "unpack_MX9_col": 150398976,
+    "quant_dequant_MX4_row": 217599232, "quant_dequant_MX4_col": 219747328,
+    "quant_dequant_MX6_row": 216175360, "quant_dequant_MX6_col": 217719808,
+    "quant_dequant_MX9_row": 216229120, "quant_dequant_MX9_col": 217433088,
+    "pack_MX4_row": 148824576, "pack_MX4_col": 147020544,
+    "pack_MX6_row": 157561856, "pack_MX6_col": 154361088,
+    "pack_MX9_row": 173053952, "pack_MX9_col": 168261120,
+    "unpack_MX4_row": 111511040, "unpack_MX4_col": 108894464,
+    "unpack_MX6_row": 128527872, "unpack_MX6_col": 126017024,
+    "unpack_MX9_row": 154410752, "unpack_MX9_col": 151516928,
 }
 
 
