@@ -300,3 +300,17 @@ def test_bf16_fast_paths_with_a_row_pitch():
         torch.cuda.synchronize()
         H.assert_planes_equal(H.planes_to_host(planes), orc.pack(H.to_orc(cfg), x), "%s pitch" % (cfg,))
         H.assert_bits_equal(H.device_to_host_f32(back), want, "%s pitch unpack" % (cfg,))
+
+
+@pytest.mark.parametrize("axis", [1, 0])
+def test_bf16_fast_paths_in_place(axis):
+    # y may alias x: the run (row direction) or the box (column direction) is loaded whole before it is written back
+    x = H.make_input("laplace_outliers", 512, 2048, "bf16", seed=8)
+    for cfg in (bdr.MX4, bdr.MX9):
+        want, so = orc.quant_dequant(H.to_orc(cfg), x, axis=axis)
+        xd = H.host_to_device(x, "bf16")
+        sums = torch.zeros(2, dtype=torch.float64, device="cuda")
+        bdr.bdr_quant_dequant(cfg, xd, xd, axis=axis, qsnr_sums=sums)
+        torch.cuda.synchronize()
+        H.assert_bits_equal(H.device_to_host_f32(xd), want, "%s axis=%d in place" % (cfg, axis))
+        H.assert_qsnr_close(sums.cpu().numpy(), so)
