@@ -7,7 +7,9 @@
  * leaves every result on the device.  `stream` is a cudaStream_t passed as void* (NULL = the
  * legacy default stream).  Return value: BDR_OK (0) or a negative bdr_status_t; all argument
  * validation happens on the host before anything is launched, so a failing call has queued no work
- * (BDR_ERR_CUDA reports a failed launch).
+ * (BDR_ERR_CUDA reports a failed launch).  The first call of an entry point on a device sets kernel
+ * attributes and may look up the address of a library-owned status word: make that call outside stream
+ * capture; later calls can be captured into CUDA graphs.
  *
  * Layout conventions
  *   A tensor is a row-major 2-D array [rows, cols] with a row pitch of `ld` ELEMENTS (ld >= cols).
@@ -97,8 +99,11 @@ int bdr_packed_sizes(const bdr_config_t* cfg /*host*/, int64_t rows, int64_t col
  *   x, y          [rows, ld] of `dt`; y may alias x; y may be NULL when only the sums are wanted
  *   qsnr_sums_dev NULL, or 2 doubles that this call ADDS {sum (Q(x)-x)^2, sum x^2} to (Eq. 3);
  *                 the caller zeroes them
- * POW2 kind only.  Fast path: axis 1, 16-byte aligned x/y, ld*sizeof(dt) and cols multiples of
- * what a 16-element slice needs; anything else runs a slower general kernel with the same result. */
+ * POW2 kind only.  Every shape, pitch and alignment is accepted; which kernel runs only changes the speed,
+ * never the result.  Fastest: bf16 tensors in the Table II family (k1 = 16, k2 = 2, d2 = 1, m <= 7,
+ * ties-to-even) with 32-byte aligned rows of whole 2048-element runs (axis 1; a contiguous tensor counts
+ * as one long row) or whole tiles of 256 rows x 128 columns (axis 0); next, fp32 or bf16 with 16-byte
+ * aligned rows of whole 16-element slices; anything else takes a slower general kernel. */
 int bdr_quant_dequant(const bdr_config_t* cfg /*host*/, const void* x, void* y, bdr_dtype_t dt,
                       int64_t rows, int64_t cols, int64_t ld, int axis, double* qsnr_sums_dev,
                       void* stream);
