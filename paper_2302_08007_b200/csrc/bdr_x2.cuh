@@ -9,7 +9,7 @@
 //   aq = r - C, Q(x) = aq * 2^(F-127)    exact
 // C is a power of two (not 1.5 * 2^k as in the fp32 formulation) because a >= 0: a + C stays inside
 // C's binade except for the single value 2C, which the clamp removes.  The Eq. 3 terms (aq - a, a)
-// are exact bf16 values; they are widened to fp32, squared and summed there.
+// are exact bf16 values; they are squared and summed in fp32 (mixed-precision multiply-add).
 // Valid for 16 <= F <= 250 (every constant and result a normal number) and ties-to-even; callers
 // send other blocks (tiny, huge, Inf/NaN, ties-away) to the fp32 / integer formulation.
 #pragma once
@@ -55,11 +55,13 @@ __device__ __forceinline__ uint32_t hmax2_nan(uint32_t a, uint32_t b) {
     asm("max.NaN.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
     return d;
 }
-// Two independent fp32 multiply-adds in one instruction: (d0, d1) += (a0 * a0, a1 * a1).
-__device__ __forceinline__ void ffma2_sq(float& d0, float& d1, float a0, float a1) {
-    asm("{.reg .b64 ra, rc; mov.b64 ra, {%2, %3}; mov.b64 rc, {%0, %1}; fma.rn.f32x2 rc, ra, ra, rc; mov.b64 {%0, %1}, rc;}"
+// (d0, d1) += (lo * lo, hi * hi) for the two bf16 halves of w, with the mixed-precision multiply-add
+// (bf16 operands, fp32 addend and result): the products are exact, each sum is rounded once, and no
+// widening instructions are needed.
+__device__ __forceinline__ void fma_sq_halves(float& d0, float& d1, uint32_t w) {
+    asm("{.reg .b16 lo, hi; mov.b32 {lo, hi}, %2; fma.rn.f32.bf16 %0, lo, lo, %0; fma.rn.f32.bf16 %1, hi, hi, %1;}"
         : "+f"(d0), "+f"(d1)
-        : "f"(a0), "f"(a1));
+        : "r"(w));
 }
 
 constexpr uint32_t kAbs2 = 0x7FFF7FFFu, kSign2 = 0x80008000u;
@@ -113,8 +115,8 @@ __device__ __forceinline__ void quantize_block_row(const uint32_t (&w)[8], const
             const uint32_t aq2 = hsub2(r2, C2);
             if constexpr (YOUT) yw[j] = hmul2(aq2, si2) | (w[j] & kSign2);
             const uint32_t d2 = hsub2(aq2, a2);  // exact
-            ffma2_sq(pe0, pe1, __uint_as_float(d2 << 16), __uint_as_float(d2 & 0xFFFF0000u));
-            ffma2_sq(ps0, ps1, __uint_as_float(a2 << 16), __uint_as_float(a2 & 0xFFFF0000u));
+            fma_sq_halves(pe0, pe1, d2);
+            fma_sq_halves(ps0, ps1, a2);
             if constexpr (CODE) macc |= (r2 << (j + 1)) & (0x100u << j);  // bit 7 of r: lowest exponent bit of C
         } else {
             // tau doubles the operand instead (exact), so the constant and the clamp are fixed
@@ -401,8 +403,8 @@ __device__ __forceinline__ void quantize_wordcol(const uint32_t (&w)[16], const 
                 if constexpr (YOUT) yw[r] = hmul2(aq2, F2) | (w[r] & kSign2);
                 if constexpr (SUMS) {
                     const uint32_t d2 = hsub2(aq2, a2);  // exact
-                    ffma2_sq(pe0, pe1, __uint_as_float(d2 << 16), __uint_as_float(d2 & 0xFFFF0000u));
-                    ffma2_sq(ps0, ps1, __uint_as_float(a2 << 16), __uint_as_float(a2 & 0xFFFF0000u));
+                    fma_sq_halves(pe0, pe1, d2);
+                    fma_sq_halves(ps0, ps1, a2);
                 }
                 if constexpr (PACK) {
                     if constexpr (W == 8) code[r] = ((w[r] >> 8) & 0x00800080u) | (r2 & 0x007F007Fu);
