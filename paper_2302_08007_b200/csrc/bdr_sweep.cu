@@ -60,6 +60,23 @@ __device__ __forceinline__ float round_to_int(float t, int rounding) {  // 0 <= 
 }
 
 // ---- POW2 kind: error energy of one slice for every mantissa width of a family -----------------------
+// packed fp32 arithmetic: two independent operations per instruction
+__device__ __forceinline__ void add_f32x2(float& d0, float& d1, float a0, float a1, float b0, float b1) {
+    asm("{.reg .b64 ra, rb, rd; mov.b64 ra, {%2, %3}; mov.b64 rb, {%4, %5}; add.rn.f32x2 rd, ra, rb; mov.b64 {%0, %1}, rd;}"
+        : "=f"(d0), "=f"(d1)
+        : "f"(a0), "f"(a1), "f"(b0), "f"(b1));
+}
+__device__ __forceinline__ void sub_f32x2(float& d0, float& d1, float a0, float a1, float b0, float b1) {
+    asm("{.reg .b64 ra, rb, rd; mov.b64 ra, {%2, %3}; mov.b64 rb, {%4, %5}; sub.rn.f32x2 rd, ra, rb; mov.b64 {%0, %1}, rd;}"
+        : "=f"(d0), "=f"(d1)
+        : "f"(a0), "f"(a1), "f"(b0), "f"(b1));
+}
+__device__ __forceinline__ void fma_f32x2(float& d0, float& d1, float a0, float a1, float b0, float b1) {  // d += a * b
+    asm("{.reg .b64 ra, rb, rd; mov.b64 ra, {%2, %3}; mov.b64 rb, {%4, %5}; mov.b64 rd, {%0, %1}; fma.rn.f32x2 rd, ra, rb, rd; mov.b64 {%0, %1}, rd;}"
+        : "+f"(d0), "+f"(d1)
+        : "f"(a0), "f"(a1), "f"(b0), "f"(b1));
+}
+
 template <int K2, int K1S>
 __device__ __forceinline__ void pow2_slice(const uint32_t (&u)[kSlice], const SweepTile& sm, int s, const SweepCfg& c,
                                            double* lane_acc /* member mi at lane_acc[32 * mi] */) {
@@ -123,16 +140,27 @@ __device__ __forceinline__ void pow2_slice(const uint32_t (&u)[kSlice], const Sw
             const uint32_t c_base = ((uint32_t)(127 + 23 - (m - 1)) << 23) | 0x400000u;
             const uint32_t qmax = (1u << m) - 1u;
             float pe = 0.f;
+            if constexpr (K1S >= 2) {
+                // two elements per instruction (packed fp32 add / subtract / multiply-add); only the clamp is scalar
+                float pe0 = 0.f, pe1 = 0.f;
 #pragma unroll
-            for (int jj = 0; jj < K1S / K2; ++jj) {
-                const uint32_t c_bits = c_base - dm[jj];
-                const float C = __uint_as_float(c_bits), Cmax = __uint_as_float(c_bits + qmax);
-#pragma unroll
-                for (int i = 0; i < K2; ++i) {
-                    const float ai = a[jj * K2 + i];
-                    const float de = __fsub_rn(__fsub_rn(fminf(__fadd_rn(ai, C), Cmax), C), ai);  // exact
-                    pe = fmaf(de, de, pe);
+                for (int k = 0; k < K1S / 2; ++k) {
+                    const uint32_t cb0 = c_base - dm[(2 * k) / K2], cb1 = c_base - dm[(2 * k + 1) / K2];
+                    const float C0 = __uint_as_float(cb0), C1 = __uint_as_float(cb1);
+                    float r0, r1;
+                    add_f32x2(r0, r1, a[2 * k], a[2 * k + 1], C0, C1);
+                    r0 = fminf(r0, __uint_as_float(cb0 + qmax));
+                    r1 = fminf(r1, __uint_as_float(cb1 + qmax));
+                    sub_f32x2(r0, r1, r0, r1, C0, C1);
+                    sub_f32x2(r0, r1, r0, r1, a[2 * k], a[2 * k + 1]);  // exact
+                    fma_f32x2(pe0, pe1, r0, r1, r0, r1);
                 }
+                pe = pe0 + pe1;
+            } else {
+                const uint32_t c_bits = c_base - dm[0];
+                const float C = __uint_as_float(c_bits), Cmax = __uint_as_float(c_bits + qmax);
+                const float de = __fsub_rn(__fsub_rn(fminf(__fadd_rn(a[0], C), Cmax), C), a[0]);  // exact
+                pe = de * de;
             }
             lane_acc[32 * mi] = fma((double)pe, w, lane_acc[32 * mi]);
         }
