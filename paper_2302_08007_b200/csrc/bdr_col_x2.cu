@@ -86,10 +86,26 @@ col_mx_x2_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant
     const uint32_t st_exps = st_elems + CS::kElemBytes, st_micro = st_exps + CS::kExpBytes;
     const int m = PACK ? W - 1 : qp.m;
 
-    auto issue = [&](int t, int i, int stg) {  // box of block row 2*warp+i of tile t into stage stg (lane 0 only)
-        const int rt = t / n_col_tiles, ct = t - rt * n_col_tiles;
+    // Where the warp's i-th box (i = 0, 1) of the CTA's t-th work unit sits.  When planes are written, a unit is
+    // a tile of 256 rows x 128 columns and warp w owns block rows 2w, 2w+1 (a column's 16 blocks are staged
+    // together).  Without planes nothing ties the warps together, so the eight warps take eight adjacent
+    // column groups of the same 32 rows: the CTA then touches 2 KB of every row at a time instead of 256 bytes.
+    auto box_origin = [&](int t, int i, int& col0, int& row0) {
+        if constexpr (PACK) {
+            const int rt = t / n_col_tiles, ct = t - rt * n_col_tiles;
+            col0 = ct * kCTileCols;
+            row0 = rt * kCTileRows + (2 * warp + i) * kSlice;
+        } else {
+            const int g = t * kCWarps + warp, bp = g / n_col_tiles, ct = g - bp * n_col_tiles;
+            col0 = ct * kCTileCols;
+            row0 = (2 * bp + i) * kSlice;
+        }
+    };
+    auto issue = [&](int t, int i, int stg) {  // lane 0 only
+        int col0, row0;
+        box_origin(t, i, col0, row0);
         async::mbar_expect_tx(bars + 8 * stg, kCBoxBytes);
-        async::tma_load_2d(ring0 + stg * kCBoxBytes, &xmap, ct * kCTileCols, rt * kCTileRows + (2 * warp + i) * kSlice, bars + 8 * stg);
+        async::tma_load_2d(ring0 + stg * kCBoxBytes, &xmap, col0, row0, bars + 8 * stg);
     };
     if (lane == 0) {
 #pragma unroll
@@ -198,7 +214,9 @@ col_mx_x2_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant
                 async::fence_proxy_async();
                 __syncwarp();
                 if (lane == 0) {
-                    tma_store_2d(&ymap, ct * kCTileCols, rt * kCTileRows + bl * kSlice, ring0 + stg * kCBoxBytes);
+                    int col0, row0;
+                    box_origin(t, i, col0, row0);
+                    tma_store_2d(&ymap, col0, row0, ring0 + stg * kCBoxBytes);
                     async::bulk_commit();
                     async::bulk_wait_read<1>();
                     if (!failed && t + (int)gridDim.x < n_tiles) issue(t + gridDim.x, i, stg + 2 >= S ? stg + 2 - S : stg + 2);
