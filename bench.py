@@ -36,15 +36,15 @@ FALLBACK_HBM_GBS = 6650.0
 # profiles/step_kernels_dram_traffic.md.  Writes that still sit in L2 when a kernel ends are not
 # counted by those counters, which is why some figures are below the algorithmic bytes.
 NCU_TRAFFIC_BYTES: dict[str, float | None] = {
-    "quant_dequant_MX4_row": 217599232, "quant_dequant_MX4_col": 219747328,
-    "quant_dequant_MX6_row": 216175360, "quant_dequant_MX6_col": 217719808,
-    "quant_dequant_MX9_row": 216229120, "quant_dequant_MX9_col": 217433088,
-    "pack_MX4_row": 148824576, "pack_MX4_col": 147020544,
-    "pack_MX6_row": 157561856, "pack_MX6_col": 154361088,
-    "pack_MX9_row": 173053952, "pack_MX9_col": 168261120,
-    "unpack_MX4_row": 111511040, "unpack_MX4_col": 108894464,
-    "unpack_MX6_row": 128527872, "unpack_MX6_col": 126017024,
-    "unpack_MX9_row": 154410752, "unpack_MX9_col": 151516928,
+    "quant_dequant_MX4_row": 215910144, "quant_dequant_MX4_col": 217317376,
+    "quant_dequant_MX6_row": 216769536, "quant_dequant_MX6_col": 217431552,
+    "quant_dequant_MX9_row": 217173504, "quant_dequant_MX9_col": 217409024,
+    "pack_MX4_row": 148965888, "pack_MX4_col": 146423552,
+    "pack_MX6_row": 157351168, "pack_MX6_col": 154226432,
+    "pack_MX9_row": 173277696, "pack_MX9_col": 167642368,
+    "unpack_MX4_row": 111672320, "unpack_MX4_col": 109009664,
+    "unpack_MX6_row": 128769792, "unpack_MX6_col": 126806784,
+    "unpack_MX9_row": 154996992, "unpack_MX9_col": 151483904,
 }
 
 
