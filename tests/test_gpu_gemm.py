@@ -202,3 +202,31 @@ def test_ws_argument_errors():
         bdr.mx_gemm_ws(bdr.MX6, pa, bdr.MX6, pb, 128, 256, 64, c, ws)                  # M must be a multiple of 256
     assert e.value.status == -3
     torch.cuda.synchronize()
+
+
+def test_padded_plane_pitches_unpack_and_ws_gemm():
+    # planes whose line pitch exceeds the natural bytes: the general pack kernel fills them, the bf16 row unpack
+    # reads them run by run, and the two-phase GEMM decodes from them
+    M, N, K = 256, 256, 2048
+    a = synth.normal_matrix(M, K, seed=11, stream=1)
+    b = synth.normal_matrix(N, K, seed=11, stream=2, sigma=0.02)
+
+    def padded(cfg, rows):
+        p = bdr.alloc_planes(cfg, rows, K)
+        wide = lambda t: torch.zeros((rows, t.shape[1] + 32), dtype=torch.uint8, device="cuda")[:, :t.shape[1]]
+        return bdr.Planes(wide(p.exps), wide(p.micro), wide(p.elems))
+
+    pa, pb = padded(bdr.MX6, M), padded(bdr.MX9, N)
+    ad, bd = torch.from_numpy(a).cuda(), torch.from_numpy(b).cuda()
+    bdr.bdr_pack(bdr.MX6, ad, pa)
+    bdr.bdr_pack(bdr.MX9, bd, pb)
+    back = torch.empty((M, K), dtype=torch.bfloat16, device="cuda")
+    bdr.bdr_unpack(bdr.MX6, pa, back)
+    aq, _ = orc.quant_dequant(orc.MX6, a)
+    H.assert_bits_equal(H.device_to_host_f32(back), aq, "unpack from padded planes")
+    ws = torch.empty(bdr.mx_gemm_workspace_bytes(M, N, K), dtype=torch.uint8, device="cuda")
+    c = torch.empty((M, N), dtype=torch.float32, device="cuda")
+    bdr.mx_gemm_ws(bdr.MX6, pa, bdr.MX9, pb, M, N, K, c, ws)
+    torch.cuda.synchronize()
+    assert rel_frob(c.cpu().numpy(), oracle_gemm(bdr.MX6, a, bdr.MX9, b)) <= 1e-5
+    assert bdr.mx_gemm_status() == 0 and bdr.bdr_device_status() == 0
