@@ -134,8 +134,8 @@ __device__ __forceinline__ void pow2_slice(const uint32_t (&u)[kSlice], const Sw
         for (int i = 0; i < K1S; ++i) a[i] = __fmul_rn(fabsf(__uint_as_float(u[b * K1S + i])), K);
 #pragma unroll
         for (int jj = 0; jj < K1S / K2; ++jj) dm[jj] = min(F23 - ej[b * (K1S / K2) + jj], beta23);
-#pragma unroll 1
-        for (int mi = 0; mi < c.nm; ++mi) {  // not unrolled: keeps the instruction footprint of the 15 shapes small
+#pragma unroll 2
+        for (int mi = 0; mi < c.nm; ++mi) {  // barely unrolled: keeps the instruction footprint of the 15 shapes small
             const int m = c.m(mi);
             const uint32_t c_base = ((uint32_t)(127 + 23 - (m - 1)) << 23) | 0x400000u;
             const uint32_t qmax = (1u << m) - 1u;
