@@ -2,15 +2,16 @@
 // m <= 7, ties-to-even) on packed bf16x2 arithmetic: a 32-bit word holds one row of two adjacent
 // columns, and the two halves are quantized as two independent blocks by the same instructions.
 //
-// A CTA (eight warps) owns tiles of 128 columns x 256 rows (16 block rows).  Warp w takes block rows 2w
-// and 2w+1 of every tile; each arrives as one 2-D TMA box of 16 rows x 128 columns (4 KB) in the
-// warp's own two-stage ring, so the box of the next tile is in flight while the current one is worked
-// on.  A lane owns four adjacent columns (8 bytes of every row).  Dequantized values go straight
-// from registers to global memory (8 bytes per lane and row, 256 contiguous bytes per warp and row).
-// The packed planes are column-major -- the transposed layout the backward-pass GEMMs read -- so codes
-// are first staged per tile in shared memory as [block-row pair][column] items; after a CTA barrier
-// the tile's columns are gathered and each column's 16 blocks leave as one contiguous run (32 W code
-// bytes, 16 exponent bytes, 16 microexponent bytes).
+// A CTA has eight warps; a warp works on boxes of 16 rows x 128 columns (4 KB), each fetched with one 2-D TMA
+// tile load into the warp's own ring, two boxes in flight; a lane owns four adjacent columns (8 bytes
+// of every row).  Dequantized values are written back over the box in shared memory and leave with one
+// TMA tile store (a third stage covers the time that store needs to drain).
+// When planes are written, a CTA owns tiles of 128 columns x 256 rows and warp w takes block rows 2w and
+// 2w+1 of every tile.  The packed planes are column-major -- the transposed layout the backward-pass
+// GEMMs read -- so codes are first staged per tile in shared memory as [block-row pair][column] items;
+// after a CTA barrier the tile's columns are gathered and each column's 16 blocks leave as one
+// contiguous run (32 W code bytes, 16 exponent bytes, 16 microexponent bytes).  Without planes the
+// eight warps of a CTA take eight adjacent column groups of the same 32 rows instead.
 #include <algorithm>
 
 #include "bdr_async.cuh"
