@@ -505,12 +505,13 @@ __device__ __forceinline__ void decode_two_blocks_row(const uint32_t (&s)[W], ui
     for (int b = 0; b < 2; ++b) {
         const uint32_t F = b ? F1 : F0, mbb = b ? mb >> 8 : mb;
         const uint32_t sc0 = ((F - (uint32_t)(M - 1)) << 7) * 0x10001u;  // 2^p for tau = 0
-        const uint32_t nb0 = sc0 + 0x83808380u;                          // -128 * 2^p
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
             const uint32_t c2 = code_pair<W, W>(s, 8 * b + j);
-            const uint32_t t = ((mbb << (7 - j)) & 0x80u) * 0x10001u;  // tau lowers both exponents by one
-            yw[8 * b + j] = hfma2((c2 & kQ2) | 0x43004300u, sc0 - t, nb0 - t) | ((c2 << (15 - M)) & kSign2);
+            // tau lowers the exponent by one: sc0 - 0x0080 per half, as one multiply-add; the constant term
+            // -128 * 2^p is a packed multiply (both on the FMA pipe, the integer pipe is the busy one)
+            const uint32_t sc = ((mbb << (7 - j)) & 0x80u) * 0xFFFEFFFFu + sc0;
+            yw[8 * b + j] = hfma2((c2 & kQ2) | 0x43004300u, sc, hmul2(sc, 0xC300C300u)) | ((c2 << (15 - M)) & kSign2);
         }
     }
 }
@@ -571,11 +572,10 @@ __device__ __forceinline__ void decode_wordcol(const uint32_t (&sl)[W], const ui
     constexpr int M = W - 1;
     constexpr uint32_t kQ2 = ((1u << M) - 1u) * 0x10001u;
     const uint32_t sc0 = F2 - ((uint32_t)(M - 1) << 7) * 0x10001u;  // 2^p for tau = 0, per half
-    const uint32_t nb0 = sc0 + 0x83808380u;                         // -128 * 2^p
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
         const uint32_t t = (mm << (7 - j)) & 0x00800080u;
-        const uint32_t sc = sc0 - t, nb = nb0 - t;
+        const uint32_t sc = sc0 - t, nb = hmul2(sc, 0xC300C300u);  // 2^p and -128 * 2^p
 #pragma unroll
         for (int r = 2 * j; r < 2 * j + 2; ++r) {
             const uint32_t c2 = code_pair_col<W>(sl, sh, 16 * i + r);
