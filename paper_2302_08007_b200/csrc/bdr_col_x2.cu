@@ -44,31 +44,6 @@ template <int W> struct CStage {
     static constexpr int kBytes = W > 0 ? kElemBytes + 2 * kExpBytes : 0;
 };
 
-__device__ __forceinline__ uint2 lds64(uint32_t addr) {
-    uint2 v;
-    asm volatile("ld.shared.v2.b32 {%0, %1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(addr) : "memory");
-    return v;
-}
-__device__ __forceinline__ uint32_t lds32(uint32_t addr) {
-    uint32_t v;
-    asm volatile("ld.shared.b32 %0, [%1];" : "=r"(v) : "r"(addr) : "memory");
-    return v;
-}
-__device__ __forceinline__ uint32_t lds8(uint32_t addr) {
-    uint32_t v;
-    asm volatile("ld.shared.u8 %0, [%1];" : "=r"(v) : "r"(addr) : "memory");
-    return v;
-}
-__device__ __forceinline__ void sts64(uint32_t addr, uint32_t a, uint32_t b) {
-    asm volatile("st.shared.v2.b32 [%0], {%1, %2};" ::"r"(addr), "r"(a), "r"(b) : "memory");
-}
-// shared (dense box) -> 2-D tile of a tensor map; joins the issuing thread's current bulk group
-__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, int x, int y, uint32_t smem_src) {
-    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];" ::"l"(map), "r"(x), "r"(y), "r"(smem_src)
-                 : "memory");
-}
-__device__ __forceinline__ double pow4_weight_col(uint32_t F) { return __hiloint2double((int)((F << 21) + 0x30100000u), 0); }
-
 // W = 0: quantize-dequantize / sums only (any m <= 7, from qp); W = m + 1: also write the packed planes.
 template <int W, bool SUMS, bool YOUT>
 __global__ void __launch_bounds__(kCThreads, 2)
@@ -136,7 +111,7 @@ col_mx_x2_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant
             const uint32_t mine = ring0 + stg * kCBoxBytes + lane * 8;
 #pragma unroll
             for (int r = 0; r < kSlice; ++r) {
-                const uint2 v = lds64(mine + r * (kCTileCols * 2));
+                const uint2 v = async::lds64(mine + r * (kCTileCols * 2));
                 wc[0][r] = v.x;
                 wc[1][r] = v.y;
             }
@@ -152,7 +127,7 @@ col_mx_x2_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant
                 if (x2::wordcol_exponents(wc[c], aw, pm, F2)) {
                     x2::quantize_wordcol<W, SUMS, YOUT>(wc[c], aw, pm, F2, m, yw, cl, ch, o);
                     if constexpr (SUMS) {
-                        const double wl = pow4_weight_col((F2 >> 7) & 0xFFu), wh = pow4_weight_col(F2 >> 23);
+                        const double wl = x2::pow4_weight((F2 >> 7) & 0xFFu), wh = x2::pow4_weight(F2 >> 23);
                         e2 = fma((double)o.pe_lo, wl, e2);
                         e2 = fma((double)o.pe_hi, wh, e2);
                         s2 = fma((double)o.ps_lo, wl, s2);
@@ -211,13 +186,13 @@ col_mx_x2_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant
                 // results over the box's input, then one tile store; the stage of the previous step (whose store
                 // has been read out by then) takes the box two steps ahead
 #pragma unroll
-                for (int r = 0; r < kSlice; ++r) sts64(mine + r * (kCTileCols * 2), wc[0][r], wc[1][r]);
+                for (int r = 0; r < kSlice; ++r) async::sts64(mine + r * (kCTileCols * 2), wc[0][r], wc[1][r]);
                 async::fence_proxy_async();
                 __syncwarp();
                 if (lane == 0) {
                     int col0, row0;
                     box_origin(t, i, col0, row0);
-                    tma_store_2d(&ymap, col0, row0, ring0 + stg * kCBoxBytes);
+                    async::tma_store_2d(&ymap, col0, row0, ring0 + stg * kCBoxBytes);
                     async::bulk_commit();
                     async::bulk_wait_read<1>();
                     if (!failed && t + (int)gridDim.x < n_tiles) issue(t + gridDim.x, i, stg + 2 >= S ? stg + 2 - S : stg + 2);
@@ -244,7 +219,7 @@ col_mx_x2_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant
 #pragma unroll
                     for (int k = 0; k < 4; ++k) {
                         const int wd = 4 * v + k, pair = wd / W, kk = wd - pair * W;
-                        x4[k] = lds32(st_elems + ((pair * kCTileCols + c) * W + kk) * 4);
+                        x4[k] = async::lds32(st_elems + ((pair * kCTileCols + c) * W + kk) * 4);
                     }
                     q = make_uint4(x4[0], x4[1], x4[2], x4[3]);
                 }
@@ -256,7 +231,7 @@ col_mx_x2_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant
                 const uint32_t src = (which ? st_micro : st_exps) + c;
                 uint32_t x4[4] = {0, 0, 0, 0};
 #pragma unroll
-                for (int b = 0; b < 16; ++b) x4[b >> 2] |= lds8(src + b * kCTileCols) << ((b & 3) * 8);
+                for (int b = 0; b < 16; ++b) x4[b >> 2] |= async::lds8(src + b * kCTileCols) << ((b & 3) * 8);
                 uint8_t* base = which ? out.micro + ((int64_t)ct * kCTileCols + c) * out.ld_micro
                                       : out.exps + ((int64_t)ct * kCTileCols + c) * out.ld_exps;
                 *reinterpret_cast<uint4*>(base + blk0) = make_uint4(x4[0], x4[1], x4[2], x4[3]);

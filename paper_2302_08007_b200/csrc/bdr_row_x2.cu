@@ -12,10 +12,6 @@ namespace bdr {
 using bf16 = __nv_bfloat16;
 constexpr int kX2SPT = 2;
 
-__device__ __forceinline__ double pow4_weight(uint32_t F) {  // 2^(2F-254)
-    return __hiloint2double((int)((F << 21) + 0x30100000u), 0);
-}
-
 __device__ __forceinline__ void words_of(const uint4& v0, const uint4& v1, uint32_t (&w)[8]) {
     w[0] = v0.x; w[1] = v0.y; w[2] = v0.z; w[3] = v0.w;
     w[4] = v1.x; w[5] = v1.y; w[6] = v1.z; w[7] = v1.w;
@@ -52,22 +48,7 @@ template <int W> struct X2PackStage {
     static constexpr int kBytes = W > 0 ? kElemBytes + kExpBytes + kMicroBytes : 0;  // a multiple of 128
 };
 
-// Where run `wi` starts.  A contiguous tensor is one long row (flat); otherwise a row holds
-// runs_per_row runs and rows are ld elements apart.
-struct RunIndex {
-    FastDiv runs_per_row;
-    int64_t ld;
-    int flat;
-    __device__ __forceinline__ void split(uint32_t wi, int64_t& row, int64_t& pos) const {
-        if (flat) {
-            row = 0;
-            pos = wi;
-        } else {
-            const uint32_t r = fastdiv(wi, runs_per_row);
-            row = r;
-            pos = wi - r * runs_per_row.d;
-        }
-    }
+struct RunIndex : x2::RunIndex {
     __device__ __forceinline__ int64_t elem_offset(uint32_t wi) const {
         int64_t row, pos;
         split(wi, row, pos);
@@ -148,7 +129,7 @@ row_mx_x2_kernel(const bf16* x, bf16* y, RunIndex ri, uint32_t total, bdr_planes
                             Fs[s] = F;
                         }
                         if constexpr (SUMS) {
-                            const double wgt = pow4_weight(F);
+                            const double wgt = x2::pow4_weight(F);
                             e2 = fma((double)pe, wgt, e2);
                             s2 = fma((double)ps, wgt, s2);
                         }
@@ -259,7 +240,10 @@ static int launch_x2(const bf16* x, bf16* y, int64_t rows, int64_t cols, int64_t
     static int blocks_per_sm = 0;
     bdr_planes_t pl = {};
     if (out) pl = *out;
-    const RunIndex ri{make_fastdiv((uint32_t)rpr), ld, rows == 1 ? 1 : 0};
+    RunIndex ri;
+    ri.runs_per_row = make_fastdiv((uint32_t)rpr);
+    ri.ld = ld;
+    ri.flat = rows == 1 ? 1 : 0;
     kern<<<x2_grid(kern, smem, total, blocks_per_sm), kX2Threads, smem, st>>>(x, y, ri, (uint32_t)total, pl, qp, sums, status);
     return cudaGetLastError() == cudaSuccess ? BDR_OK : BDR_ERR_CUDA;
 }

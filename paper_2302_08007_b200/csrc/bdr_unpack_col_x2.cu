@@ -32,16 +32,6 @@ template <int W> struct UCStage {
     static constexpr int kBytes = kElemBytes + 2 * kExpBytes;
 };
 
-__device__ __forceinline__ uint32_t uc_lds32(uint32_t addr) {
-    uint32_t v;
-    asm volatile("ld.shared.b32 %0, [%1];" : "=r"(v) : "r"(addr) : "memory");
-    return v;
-}
-__device__ __forceinline__ uint32_t uc_lds16(uint32_t addr) {
-    uint16_t v;
-    asm volatile("ld.shared.u16 %0, [%1];" : "=h"(v) : "r"(addr) : "memory");
-    return v;
-}
 __device__ __forceinline__ void uc_cp16(uint32_t smem_dst, const void* gsrc) {
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_dst), "l"(gsrc) : "memory");
 }
@@ -89,10 +79,10 @@ unpack_col_x2_kernel(bdr_planes_t in, bf16* y, int64_t ld, int n_col_tiles, int 
                 s[c][4] = a1.x; s[c][5] = a1.y; s[c][6] = a1.z; s[c][7] = a1.w;
             } else {
 #pragma unroll
-                for (int k = 0; k < W; ++k) s[c][k] = uc_lds32(src + 4 * k);
+                for (int k = 0; k < W; ++k) s[c][k] = async::lds32(src + 4 * k);
             }
-            Fp[c] = uc_lds16(b + ST::kElemBytes + ST::row_of(col) * 16 + 2 * warp);
-            mp[c] = uc_lds16(b + ST::kElemBytes + ST::kExpBytes + ST::row_of(col) * 16 + 2 * warp);
+            Fp[c] = async::lds16(b + ST::kElemBytes + ST::row_of(col) * 16 + 2 * warp);
+            mp[c] = async::lds16(b + ST::kElemBytes + ST::kExpBytes + ST::row_of(col) * 16 + 2 * warp);
         }
 #pragma unroll
         for (int i = 0; i < 2; ++i) {  // block rows 2*warp and 2*warp + 1

@@ -24,37 +24,7 @@ template <int W> struct UStage {
     static constexpr int kBytes = kElemBytes + 2 * kExpBytes;  // a multiple of 128
 };
 
-struct URunIndex {
-    FastDiv runs_per_row;
-    int64_t ld;
-    int flat;
-    __device__ __forceinline__ void split(uint32_t wi, int64_t& row, int64_t& pos) const {
-        if (flat) {
-            row = 0;
-            pos = wi;
-        } else {
-            const uint32_t r = fastdiv(wi, runs_per_row);
-            row = r;
-            pos = wi - r * runs_per_row.d;
-        }
-    }
-};
-
-__device__ __forceinline__ void ustg256(void* p, const uint32_t* v) {
-    asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(p), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]),
-                 "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7])
-                 : "memory");
-}
-__device__ __forceinline__ uint32_t ulds32(uint32_t addr) {
-    uint32_t v;
-    asm volatile("ld.shared.b32 %0, [%1];" : "=r"(v) : "r"(addr) : "memory");
-    return v;
-}
-__device__ __forceinline__ uint32_t ulds16(uint32_t addr) {
-    uint16_t v;
-    asm volatile("ld.shared.u16 %0, [%1];" : "=h"(v) : "r"(addr) : "memory");
-    return v;
-}
+using URunIndex = x2::RunIndex;
 
 template <int W>
 __global__ void __launch_bounds__(kUThreads)
@@ -104,10 +74,10 @@ unpack_row_x2_kernel(bdr_planes_t in, bf16* y, URunIndex ri, uint32_t total, int
                 s[sub][4] = b.x; s[sub][5] = b.y; s[sub][6] = b.z; s[sub][7] = b.w;
             } else {
 #pragma unroll
-                for (int k = 0; k < W; ++k) s[sub][k] = ulds32(src + 4 * k);
+                for (int k = 0; k < W; ++k) s[sub][k] = async::lds32(src + 4 * k);
             }
-            Fw[sub] = ulds16(stage + US::kElemBytes + sub * (kUHalfElems / 16) + 2 * lane);
-            mw[sub] = ulds16(stage + US::kElemBytes + US::kExpBytes + sub * (kUHalfElems / 16) + 2 * lane);
+            Fw[sub] = async::lds16(stage + US::kElemBytes + sub * (kUHalfElems / 16) + 2 * lane);
+            mw[sub] = async::lds16(stage + US::kElemBytes + US::kExpBytes + sub * (kUHalfElems / 16) + 2 * lane);
         }
         __syncwarp();  // every lane has read stage st
         if (lane == 0 && wi + S * stride < total) load(wi + S * stride, st);
@@ -128,8 +98,8 @@ unpack_row_x2_kernel(bdr_planes_t in, bf16* y, URunIndex ri, uint32_t total, int
 #pragma unroll
                 for (int k = 0; k < 16; ++k) yw[k] = o.y[k];
             }
-            ustg256(yrun + sub * kUHalfElems, yw);
-            ustg256(yrun + sub * kUHalfElems + 16, yw + 8);
+            async::stg256(yrun + sub * kUHalfElems, yw);
+            async::stg256(yrun + sub * kUHalfElems + 16, yw + 8);
         }
         if (++st == S) { st = 0; phase ^= 1; }
     }
@@ -155,7 +125,10 @@ static int launch_unpack_x2(const bdr_planes_t& in, bf16* y, int64_t rows, int64
     if (!status) return BDR_ERR_CUDA;
     const int64_t need = (total + kUWarps - 1) / kUWarps;
     const int grid = (int)max((int64_t)1, min(need, (int64_t)sm_count() * blocks_per_sm));
-    const URunIndex ri{make_fastdiv((uint32_t)rpr), ld, flat ? 1 : 0};
+    URunIndex ri;
+    ri.runs_per_row = make_fastdiv((uint32_t)rpr);
+    ri.ld = ld;
+    ri.flat = flat ? 1 : 0;
     kern<<<grid, kUThreads, smem, st>>>(in, y, ri, (uint32_t)total, status);
     return cudaGetLastError() == cudaSuccess ? BDR_OK : BDR_ERR_CUDA;
 }

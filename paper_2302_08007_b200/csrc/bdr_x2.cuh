@@ -64,6 +64,27 @@ __device__ __forceinline__ void fma_sq_halves(float& d0, float& d1, uint32_t w) 
         : "r"(w));
 }
 
+// 2^(2F-254) as a double: the factor that takes a block's Eq. 3 sums out of its normalised domain
+__device__ __forceinline__ double pow4_weight(uint32_t F) { return __hiloint2double((int)((F << 21) + 0x30100000u), 0); }
+
+// Where run `wi` of kRun elements starts.  A contiguous tensor is one long row (flat); otherwise a row holds
+// runs_per_row runs and rows are ld elements apart.
+struct RunIndex {
+    FastDiv runs_per_row;
+    int64_t ld;
+    int flat;
+    __device__ __forceinline__ void split(uint32_t wi, int64_t& row, int64_t& pos) const {
+        if (flat) {
+            row = 0;
+            pos = wi;
+        } else {
+            const uint32_t r = fastdiv(wi, runs_per_row);
+            row = r;
+            pos = wi - r * runs_per_row.d;
+        }
+    }
+};
+
 constexpr uint32_t kAbs2 = 0x7FFF7FFFu, kSign2 = 0x80008000u;
 constexpr int kMinF = 16, kMaxF = 250;
 
