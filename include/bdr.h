@@ -102,7 +102,8 @@ int bdr_packed_sizes(const bdr_config_t* cfg /*host*/, int64_t rows, int64_t col
  * POW2 kind only.  Every shape, pitch and alignment is accepted; which kernel runs only changes the speed,
  * never the result.  Fastest: bf16 tensors in the Table II family (k1 = 16, k2 = 2, d2 = 1, m <= 7,
  * ties-to-even) with 32-byte aligned rows of whole 2048-element runs (axis 1; a contiguous tensor counts
- * as one long row) or whole tiles of 256 rows x 128 columns (axis 0); next, fp32 or bf16 with 16-byte
+ * as one long row) or whole tiles of 256 rows x 128 columns (axis 0); along axis 1 the same kernel also
+ * takes k1 = 32 .. 1024 (powers of two) and formats without shifts (d2 = 0); next, fp32 or bf16 with 16-byte
  * aligned rows of whole 16-element slices; anything else takes a slower general kernel. */
 int bdr_quant_dequant(const bdr_config_t* cfg /*host*/, const void* x, void* y, bdr_dtype_t dt,
                       int64_t rows, int64_t cols, int64_t ld, int axis, double* qsnr_sums_dev,

@@ -72,7 +72,8 @@ row_mx_x2_kernel(const bf16* x, bf16* y, RunIndex ri, uint32_t total, bdr_planes
     const uint32_t bars = async::smem_u32(smem) + kX2RingBytes + warp * S * 8;
     const uint32_t stage0 = async::smem_u32(smem) + kX2RingBytes + kX2BarBytes + warp * 2 * PS::kBytes;
     const int m = PACK ? W - 1 : qp.m;
-    const x2::Consts k = x2::make_consts(m);
+    const x2::Consts k = x2::make_consts(m, PACK ? 1 : qp.d2);
+    const int group_lanes = qp.k1 >> 5;  // lanes that share a block when k1 >= 64 (1 when the lane's two blocks form one)
     const uint32_t stride = gridDim.x * kX2Warps;
     const uint32_t w0 = blockIdx.x * kX2Warps + warp;
     if (lane == 0) {
@@ -101,7 +102,56 @@ row_mx_x2_kernel(const bf16* x, bf16* y, RunIndex ri, uint32_t total, bdr_planes
 #pragma unroll
         for (int sub = 0; sub < kX2Sub; ++sub) {
             const uint32_t mine = ring0 + st * kRunBytes + sub * (kSubElems * 2) + lane * 64;
-            uint32_t cw[kX2SPT][NCW], Fs[kX2SPT], mbs[kX2SPT];
+            if constexpr (!PACK) {
+                // quantize-dequantize: blocks of 16 .. 1024 elements.  The two 16-element blocks of the lane give
+                // their exponents first; wider blocks take the maximum over the lane's pair and, from 64
+                // elements on, over the k1 / 32 adjacent lanes that share the block.
+                uint4 vv[kX2SPT][2];
+                uint32_t w[kX2SPT][8], aw[kX2SPT][8], Fb[kX2SPT];
+#pragma unroll
+                for (int s = 0; s < kX2SPT; ++s) {
+                    vv[s][0] = async::lds128(mine + 32 * s);
+                    vv[s][1] = async::lds128(mine + 32 * s + 16);
+                    words_of(vv[s][0], vv[s][1], w[s]);
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) aw[s][j] = x2::habs2(w[s][j]);
+                    Fb[s] = x2::block_exponent(aw[s]);
+                }
+                if (group_lanes > 0) {  // the same for every thread
+                    uint32_t F = max(Fb[0], Fb[1]);
+                    for (int o = group_lanes >> 1; o > 0; o >>= 1) F = max(F, __shfl_xor_sync(0xFFFFFFFFu, F, o));
+                    Fb[0] = F;
+                    Fb[1] = F;
+                }
+#pragma unroll
+                for (int s = 0; s < kX2SPT; ++s) {
+                    uint32_t yw[8];
+                    const uint32_t F = Fb[s];
+                    if (F - x2::kMinF <= (uint32_t)(x2::kMaxF - x2::kMinF)) {
+                        float pe = 0.f, ps = 0.f;
+                        uint32_t code2[8], micro;
+                        x2::quantize_block_row<SUMS, YOUT, false>(w[s], aw[s], F, m, k, yw, code2, micro, pe, ps);
+                        if constexpr (SUMS) {
+                            const double wgt = x2::pow4_weight(F);
+                            e2 = fma((double)pe, wgt, e2);
+                            s2 = fma((double)ps, wgt, s2);
+                        }
+                    } else {
+                        const x2::SlowOut o = x2::quantize_block_slow<0, SUMS>(vv[s][0], vv[s][1], qp, F);
+                        if constexpr (SUMS) { e2 += o.e2; s2 += o.s2; }
+                        if constexpr (YOUT) {
+                            yw[0] = o.y[0].x; yw[1] = o.y[0].y; yw[2] = o.y[0].z; yw[3] = o.y[0].w;
+                            yw[4] = o.y[1].x; yw[5] = o.y[1].y; yw[6] = o.y[1].z; yw[7] = o.y[1].w;
+                        }
+                    }
+                    if constexpr (YOUT) {  // back into the stage, over the block's input
+                        async::sts128(mine + 32 * s, make_uint4(yw[0], yw[1], yw[2], yw[3]));
+                        async::sts128(mine + 32 * s + 16, make_uint4(yw[4], yw[5], yw[6], yw[7]));
+                    }
+                }
+            }
+            [[maybe_unused]] uint32_t cw[kX2SPT][NCW], Fs[kX2SPT], mbs[kX2SPT];
+            if constexpr (PACK) {
 #pragma unroll
             for (int s = 0; s < kX2SPT; ++s) {
                 const uint4 v0 = async::lds128(mine + 32 * s), v1 = async::lds128(mine + 32 * s + 16);
@@ -152,6 +202,7 @@ row_mx_x2_kernel(const bf16* x, bf16* y, RunIndex ri, uint32_t total, bdr_planes
                     async::sts128(mine + 32 * s, make_uint4(yw[0], yw[1], yw[2], yw[3]));
                     async::sts128(mine + 32 * s + 16, make_uint4(yw[4], yw[5], yw[6], yw[7]));
                 }
+            }
             }
             if constexpr (PACK) {
                 // the lane's 32 codes as W words: block 1 follows block 0 at bit 16 W
@@ -205,8 +256,13 @@ row_mx_x2_kernel(const bf16* x, bf16* y, RunIndex ri, uint32_t total, bdr_planes
 }
 
 // ---- host launchers --------------------------------------------------------------------------------
-static bool x2_config(const QParams& qp) {
-    return qp.k1 == 16 && qp.k2 == 2 && qp.d2 == 1 && qp.m <= 7 && qp.rounding == BDR_ROUND_NEAREST_EVEN;
+// packing: the Table II family; quantize-dequantize: blocks of 16 .. 1024 elements with one-bit shifts per pair of
+// elements, or without shifts (d2 = 0, where k2 does not matter)
+static bool x2_config(const QParams& qp, bool pack) {
+    if (qp.m > 7 || qp.rounding != BDR_ROUND_NEAREST_EVEN) return false;
+    if (pack) return qp.k1 == 16 && qp.k2 == 2 && qp.d2 == 1;
+    const bool k1_ok = qp.k1 >= 16 && qp.k1 <= 1024 && (qp.k1 & (qp.k1 - 1)) == 0;
+    return k1_ok && ((qp.k2 == 2 && qp.d2 == 1) || qp.d2 == 0);
 }
 
 // One wave of resident CTAs: every warp then streams many runs through its prefetch ring instead of
@@ -258,10 +314,11 @@ static int x2_flags(const bf16* x, bf16* y, int64_t rows, int64_t cols, int64_t 
     return BDR_ERR_NULL;
 }
 
-// Shapes: whole 2048-element runs, 16-byte aligned (a contiguous tensor counts as one long row).
-static bool x2_shape(const void* x, const void* y, int64_t& rows, int64_t& cols, int64_t& ld) {
+// Shapes: whole 2048-element runs, 32-byte aligned (a contiguous tensor whose rows hold whole blocks counts as
+// one long row).
+static bool x2_shape(const void* x, const void* y, int64_t& rows, int64_t& cols, int64_t& ld, int k1 = 16) {
     if ((((uintptr_t)x | (uintptr_t)y) % 32) || (ld * 2) % 32) return false;
-    if (ld == cols && cols % 16 == 0) {
+    if (ld == cols && cols % k1 == 0) {
         cols *= rows;
         ld = cols;
         rows = 1;
@@ -271,14 +328,14 @@ static bool x2_shape(const void* x, const void* y, int64_t& rows, int64_t& cols,
 
 int quant_rowwise_mx_x2(const bf16* x, bf16* y, int64_t rows, int64_t cols, int64_t ld, const QParams& qp, double* sums,
                         cudaStream_t st) {
-    if (!x2_config(qp) || !x2_shape(x, y, rows, cols, ld)) return BDR_ERR_UNSUPPORTED;
+    if (!x2_config(qp, false) || !x2_shape(x, y, rows, cols, ld, qp.k1)) return BDR_ERR_UNSUPPORTED;
     return x2_flags<0>(x, y, rows, cols, ld, nullptr, qp, sums, st);
 }
 
 // The caller guarantees tight planes (line pitch = the line's natural bytes).
 int pack_rowwise_mx_x2(const bf16* x, bf16* y, int64_t rows, int64_t cols, int64_t ld, const bdr_planes_t& out,
                        const QParams& qp, double* sums, cudaStream_t st) {
-    if (!x2_config(qp) || !x2_shape(x, y, rows, cols, ld)) return BDR_ERR_UNSUPPORTED;
+    if (!x2_config(qp, true) || !x2_shape(x, y, rows, cols, ld)) return BDR_ERR_UNSUPPORTED;
     switch (qp.m) {
         case 2: return x2_flags<3>(x, y, rows, cols, ld, &out, qp, sums, st);
         case 4: return x2_flags<5>(x, y, rows, cols, ld, &out, qp, sums, st);

@@ -90,15 +90,19 @@ constexpr int kMinF = 16, kMaxF = 250;
 
 // constants of one mantissa width
 struct Consts {
-    uint32_t C0, C1;  // 2^(7-(m-1)) and half of it, in both halves
+    uint32_t C0, C1;  // 2^(7-(m-1)) and the constant of a shifted sub-block (half of it; the same when d2 = 0)
     uint32_t QM;      // 2^m - 1 in both halves
+    uint32_t G1;      // factor of a shifted sub-block: 2.0 (1.0 when d2 = 0)
+    uint32_t SID;     // what a shifted sub-block takes off the exponent of 2^(F-127): 0x0080 per half (0 when d2 = 0)
 };
-__host__ __device__ __forceinline__ Consts make_consts(int m) {
+__host__ __device__ __forceinline__ Consts make_consts(int m, int d2 = 1) {
     Consts k;
     const uint32_t e0 = (uint32_t)(127 + 7 - (m - 1));
     k.C0 = (e0 << 7) * 0x10001u;
-    k.C1 = ((e0 - 1) << 7) * 0x10001u;
+    k.C1 = d2 ? ((e0 - 1) << 7) * 0x10001u : k.C0;
     k.QM = ((1u << m) - 1u) * 0x10001u;
+    k.G1 = d2 ? 0x40004000u : 0x3F803F80u;
+    k.SID = d2 ? 0x00800080u : 0u;
     return k;
 }
 
@@ -141,9 +145,9 @@ __device__ __forceinline__ void quantize_block_row(const uint32_t (&w)[8], const
             if constexpr (CODE) macc |= (r2 << (j + 1)) & (0x100u << j);  // bit 7 of r: lowest exponent bit of C
         } else {
             // tau doubles the operand instead (exact), so the constant and the clamp are fixed
-            const uint32_t g2 = top ? 0x3F803F80u : 0x40004000u;  // 1.0 or 2.0
+            const uint32_t g2 = top ? 0x3F803F80u : k.G1;  // 1.0 or 2.0
             r2 = hmin2(hfma2(a2, g2, k.C0), k.C0 + k.QM);
-            if constexpr (YOUT) yw[j] = hmul2(hsub2(r2, k.C0), top ? si2 : si2 - 0x00800080u) | (w[j] & kSign2);
+            if constexpr (YOUT) yw[j] = hmul2(hsub2(r2, k.C0), top ? si2 : si2 - k.SID) | (w[j] & kSign2);
             if constexpr (CODE) macc |= (g2 << (j + 2)) & (0x10000u << j);  // bit 14 of 2.0
         }
         if constexpr (CODE) code2[j] = (r2 & 0x007F007Fu) | ((w[j] >> (15 - m)) & (0x00010001u << m));
@@ -280,8 +284,9 @@ struct SlowOut {
     uint32_t F, micro;
     double e2, s2;
 };
+// F_ext: the shared exponent when the block is wider than these sixteen elements (k1 > 16), else 0.
 template <int W, bool SUMS>
-__device__ __noinline__ SlowOut quantize_block_slow(uint4 w0, uint4 w1, QParams qp) {
+__device__ __noinline__ SlowOut quantize_block_slow(uint4 w0, uint4 w1, QParams qp, uint32_t F_ext = 0) {
     SlowOut o;
     const uint4 w[2] = {w0, w1};
     uint32_t u[kSlice], yb[kSlice], rq[kSlice], cb[kSlice / 2], tau[kSlice / 2], fj[kSlice / 2], fb[1];
@@ -290,6 +295,7 @@ __device__ __noinline__ SlowOut quantize_block_slow(uint4 w0, uint4 w1, QParams 
     uint32_t F = 0;
 #pragma unroll
     for (int j = 0; j < kSlice / 2; ++j) F = max(F, fj[j]);
+    if (qp.k1 > kSlice) F = F_ext << 23;
     fb[0] = F;
     o.e2 = 0.0;
     o.s2 = 0.0;

@@ -283,6 +283,27 @@ def test_bf16_quant_dequant_other_mantissa_widths(m):
         H.assert_qsnr_close(sums, so, "%s axis=%d" % (cfg, axis))
 
 
+@pytest.mark.parametrize("k1", [16, 32, 64, 256, 1024])
+@pytest.mark.parametrize("k2,d2", [(2, 1), (1, 0), (8, 0)])
+def test_bf16_rowwise_wider_blocks_and_no_shifts(k1, k2, d2):
+    # the packed-arithmetic row kernel also takes blocks of up to 1024 elements (the exponent is a maximum over
+    # the lanes that share the block) and formats without microexponents (BFP / MSFP)
+    for m in (1, 4, 7):
+        cfg = Cfg(k1, 8, k2, d2, m)
+        cases = [("boundary", _boundary_input(64, 2048, seed=k1 + m), None),
+                 ("laplace_outliers", H.make_input("laplace_outliers", 6, 4096, "bf16", seed=k1), None),
+                 ("normal pitch", H.make_input("normal", 3, 2048, "bf16", seed=m), 2080),
+                 ("edge", H.make_input("edge", 4, 1024, "bf16", seed=3), None)]
+        for what, x, ld in cases:
+            y, sums = run_quant(cfg, x, "bf16", ld=ld)
+            want, so = orc.quant_dequant(H.to_orc(cfg), x)
+            H.assert_bits_equal(y, want, "%s %s" % (cfg, what))
+            H.assert_qsnr_close(sums, so, "%s %s" % (cfg, what))
+            _, sums_only = run_quant(cfg, x, "bf16", ld=ld, want_y=False)
+            H.assert_qsnr_close(sums_only, so, "%s %s sums only" % (cfg, what))
+    assert bdr.bdr_device_status() == 0
+
+
 def test_bf16_fast_paths_with_a_row_pitch():
     # rows of 2048 elements that are 2112 elements apart: the run index splits into (row, position)
     rows, cols, ld = 5, 2048, 2112
