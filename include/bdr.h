@@ -182,6 +182,35 @@ int mx_gemm_ws(const bdr_config_t* cfg_a /*host*/, const bdr_planes_t* a /*host 
                const bdr_config_t* cfg_b /*host*/, const bdr_planes_t* b /*host struct*/, int64_t M, int64_t N,
                int64_t K, float* c, int64_t ldc, void* workspace, int64_t workspace_bytes, void* stream);
 
+/* mx_gemm for MX4 / MX6 operands (k1 = 16, k2 = 2, d2 = 1, m in {2, 4}; A and B may differ) on the 8-bit
+ * block-scaled tensor-core path, which runs at twice the bf16 rate.  (The paper has no counterpart: it maps
+ * the format onto the scaled 8-bit matrix instruction of the target GPU.  A decoded element
+ * q * 2^(E - tau - m + 1), Section III, has at most four significant bits, so it is an exact E4M3 number
+ * once the exponent of the larger of two neighbouring 16-element blocks is taken out as the 32-element
+ * scale.)  Phase 1 re-encodes both operands into `workspace`, phase 2 multiplies them; every product is
+ * exact and accumulation is fp32, so the result agrees with mx_gemm up to summation order.  Operands
+ * that cannot be represented (neighbouring block exponents more than about 12 apart with non-zero
+ * elements in the smaller block, block exponents below 16, Inf/NaN blocks) are detected on the device
+ * in phase 1; the call then computes C with mx_gemm's kernel instead, without host involvement.
+ * Needs M, N and K multiples of 256 and a 256-byte aligned workspace of at least
+ * mx_gemm_f8_workspace_bytes(M, N, K) bytes (about (M + N) K * 33 / 32), whose contents are overwritten. */
+int64_t mx_gemm_f8_workspace_bytes(int64_t M, int64_t N, int64_t K);
+int mx_gemm_f8(const bdr_config_t* cfg_a /*host*/, const bdr_planes_t* a /*host struct*/,
+               const bdr_config_t* cfg_b /*host*/, const bdr_planes_t* b /*host struct*/, int64_t M, int64_t N,
+               int64_t K, float* c, int64_t ldc, void* workspace, int64_t workspace_bytes, void* stream);
+
+/* Phase 1 of mx_gemm_f8 on its own: packed planes of an MX4 / MX6 operand [rows, K] (axis-1 planes) ->
+ *   out      rows * K bytes (device), row-major E4M3 elements
+ *   scales   rows * K / 32 bytes (device): for every 128 rows x 128 K a 512-byte atom holding the scale
+ *            exponent (value 2^(byte - 127)) of row r, K group g (32 elements) at (r % 32) * 16 + (r / 32) * 4 + g;
+ *            atoms ordered [K / 128][rows / 128]
+ *   inexact_dev  one int (device): set to 1 if some element is not representable (then its byte holds
+ *            the nearest E4M3 value); never cleared by this call
+ * so that element = E4M3(out) * 2^(scale - 127) exactly.  rows and K multiples of 128; 16-byte aligned
+ * pointers. */
+int bdr_reencode_e4m3(const bdr_config_t* cfg /*host*/, const bdr_planes_t* in /*host struct*/, int64_t rows, int64_t K,
+                      uint8_t* out, uint8_t* scales, int* inexact_dev, void* stream);
+
 /* BDR_OK, or BDR_ERR_TIMEOUT if any mx_gemm launch on the current device gave up a bounded wait
  * (sticky).  Host call; synchronises with the device (it copies one word back). */
 int mx_gemm_status(void);

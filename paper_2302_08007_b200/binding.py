@@ -21,7 +21,8 @@ F32, BF16 = 0, 1
 
 EXPORTS = ("bdr_strerror", "bdr_device_status", "bdr_packed_sizes", "bdr_quant_dequant", "bdr_pack", "bdr_unpack",
            "bdr_qsnr_workspace_bytes", "bdr_qsnr", "bdr_qsnr_static_max_cfgs", "bdr_qsnr_static", "mx_gemm",
-           "mx_gemm_workspace_bytes", "mx_gemm_ws", "mx_gemm_status")
+           "mx_gemm_workspace_bytes", "mx_gemm_ws", "mx_gemm_f8_workspace_bytes", "mx_gemm_f8", "bdr_reencode_e4m3",
+           "mx_gemm_status")
 
 
 class BdrError(RuntimeError):
@@ -108,6 +109,12 @@ def lib():
         L.mx_gemm_ws.restype = C.c_int
         L.mx_gemm_ws.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_int64, C.c_int64,
                                  C.c_void_p, C.c_int64, C.c_void_p, C.c_int64, C.c_void_p]
+        L.mx_gemm_f8_workspace_bytes.restype = C.c_int64
+        L.mx_gemm_f8_workspace_bytes.argtypes = [C.c_int64, C.c_int64, C.c_int64]
+        L.mx_gemm_f8.restype = C.c_int
+        L.mx_gemm_f8.argtypes = L.mx_gemm_ws.argtypes
+        L.bdr_reencode_e4m3.restype = C.c_int
+        L.bdr_reencode_e4m3.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
         L.mx_gemm_status.restype = C.c_int
         L.mx_gemm_status.argtypes = []
         L.bdr_device_status.restype = C.c_int
@@ -253,6 +260,31 @@ def mx_gemm_ws(cfg_a: Config, a: Planes, cfg_b: Config, b: Planes, M: int, N: in
                             c.stride(0), _ptr(workspace), workspace.numel() * workspace.element_size(), _stream(stream)),
            "mx_gemm_ws")
     return c
+
+
+def mx_gemm_f8_workspace_bytes(M: int, N: int, K: int) -> int:
+    return int(lib().mx_gemm_f8_workspace_bytes(M, N, K))
+
+
+def mx_gemm_f8(cfg_a: Config, a: Planes, cfg_b: Config, b: Planes, M: int, N: int, K: int, c: torch.Tensor,
+               workspace: torch.Tensor, stream=None):
+    """mx_gemm for MX4 / MX6 operands on the block-scaled 8-bit tensor-core path: exact re-encoding to E4M3 with
+    one scale per 32 elements into `workspace` (at least mx_gemm_f8_workspace_bytes(M, N, K) bytes), then the GEMM."""
+    ca, cb, pa, pb = cfg_a.c(), cfg_b.c(), a.c(), b.c()
+    _check(lib().mx_gemm_f8(C.addressof(ca), C.addressof(pa), C.addressof(cb), C.addressof(pb), M, N, K, _ptr(c),
+                            c.stride(0), _ptr(workspace), workspace.numel() * workspace.element_size(), _stream(stream)),
+           "mx_gemm_f8")
+    return c
+
+
+def bdr_reencode_e4m3(cfg: Config, planes: Planes, rows: int, K: int, out: torch.Tensor, scales: torch.Tensor,
+                      inexact: torch.Tensor, stream=None):
+    """Packed MX4 / MX6 operand -> E4M3 bytes `out` [rows, K], scale atoms `scales` (rows * K / 32 bytes) and the
+    int32 flag `inexact` (set to 1, never cleared, if an element is not representable)."""
+    cc, pp = cfg.c(), planes.c()
+    _check(lib().bdr_reencode_e4m3(C.addressof(cc), C.addressof(pp), rows, K, _ptr(out), _ptr(scales), _ptr(inexact),
+                                   _stream(stream)), "bdr_reencode_e4m3")
+    return out, scales
 
 
 def bdr_device_status() -> int:

@@ -85,7 +85,7 @@ __device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t desc_a, uint
         : "memory");
 }
 // 32 lanes x 32 consecutive fp32 columns of the accumulator -> 32 registers per thread.
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+__device__ __forceinline__ void tmem_ld32_nowait(uint32_t taddr, uint32_t (&r)[32]) {
     asm volatile(
         "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
         "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
@@ -96,7 +96,11 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
           "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
         : "r"(taddr)
         : "memory");
-    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+    tmem_ld32_nowait(taddr, r);
+    tmem_ld_wait();
 }
 
 // Shared-memory matrix descriptor: K-major operand, 128-byte swizzle, rows of 64 bf16 (128 bytes),
@@ -271,7 +275,8 @@ __device__ __forceinline__ bool decode_rows(const bdr_planes_t& pl, int64_t grow
 
 template <int WA, int WB>
 __global__ void __launch_bounds__(kGemmThreads, 1)
-mx_gemm_kernel(bdr_planes_t a, bdr_planes_t b, int64_t M, int64_t N, int64_t K, float* c, int64_t ldc) {
+mx_gemm_kernel(bdr_planes_t a, bdr_planes_t b, int64_t M, int64_t N, int64_t K, float* c, int64_t ldc, const int* gate) {
+    if (gate && *gate == 0) return;  // a fall-back launch that is not needed (the same for every thread of the grid)
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     // tiles first (1024-byte aligned for the swizzle), bookkeeping after them
     uint8_t* tiles = reinterpret_cast<uint8_t*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
@@ -365,12 +370,13 @@ mx_gemm_kernel(bdr_planes_t a, bdr_planes_t b, int64_t M, int64_t N, int64_t K, 
 
 #include "mx_gemm_pair.cuh"
 #include "mx_gemm_dense.cuh"
+#include "mx_gemm_f8.cuh"
 
 namespace bdr {
 
 template <int WA, int WB>
 static int launch_gemm(const bdr_planes_t& a, const bdr_planes_t& b, int64_t M, int64_t N, int64_t K, float* c, int64_t ldc,
-                       cudaStream_t st) {
+                       const int* gate, cudaStream_t st) {
     auto kern = mx_gemm_kernel<WA, WB>;
     const size_t smem = (size_t)kStages * kStageBytes + 256 + (size_t)(kBM + kBN) * RingStride<WA, WB>::value + 1024;
     static bool attr_done = false;
@@ -379,22 +385,22 @@ static int launch_gemm(const bdr_planes_t& a, const bdr_planes_t& b, int64_t M, 
         attr_done = true;
     }
     const dim3 grid((unsigned)(N / kBN), (unsigned)(M / kBM));
-    kern<<<grid, kGemmThreads, smem, st>>>(a, b, M, N, K, c, ldc);
+    kern<<<grid, kGemmThreads, smem, st>>>(a, b, M, N, K, c, ldc, gate);
     return cudaGetLastError() == cudaSuccess ? BDR_OK : BDR_ERR_CUDA;
 }
 
 template <int WA>
 static int gemm_pick_b(int mb, const bdr_planes_t& a, const bdr_planes_t& b, int64_t M, int64_t N, int64_t K, float* c,
-                       int64_t ldc, cudaStream_t st) {
+                       int64_t ldc, const int* gate, cudaStream_t st) {
     // 2-CTA kernel when the shape allows whole 256-row pairs and 256-element K chunks
     const bool pair = M % 256 == 0 && K % kChunkK == 0 && M / 128 <= 0x7FFFFFFF && N / 256 <= 65535;
     switch (mb) {
-        case 2: { const int rc = pair ? launch_gemm_pair<WA, 3>(a, b, M, N, K, c, ldc, st) : BDR_ERR_UNSUPPORTED;
-                  return rc == BDR_ERR_UNSUPPORTED ? launch_gemm<WA, 3>(a, b, M, N, K, c, ldc, st) : rc; }
-        case 4: { const int rc = pair ? launch_gemm_pair<WA, 5>(a, b, M, N, K, c, ldc, st) : BDR_ERR_UNSUPPORTED;
-                  return rc == BDR_ERR_UNSUPPORTED ? launch_gemm<WA, 5>(a, b, M, N, K, c, ldc, st) : rc; }
-        case 7: { const int rc = pair ? launch_gemm_pair<WA, 8>(a, b, M, N, K, c, ldc, st) : BDR_ERR_UNSUPPORTED;
-                  return rc == BDR_ERR_UNSUPPORTED ? launch_gemm<WA, 8>(a, b, M, N, K, c, ldc, st) : rc; }
+        case 2: { const int rc = pair ? launch_gemm_pair<WA, 3>(a, b, M, N, K, c, ldc, gate, st) : BDR_ERR_UNSUPPORTED;
+                  return rc == BDR_ERR_UNSUPPORTED ? launch_gemm<WA, 3>(a, b, M, N, K, c, ldc, gate, st) : rc; }
+        case 4: { const int rc = pair ? launch_gemm_pair<WA, 5>(a, b, M, N, K, c, ldc, gate, st) : BDR_ERR_UNSUPPORTED;
+                  return rc == BDR_ERR_UNSUPPORTED ? launch_gemm<WA, 5>(a, b, M, N, K, c, ldc, gate, st) : rc; }
+        case 7: { const int rc = pair ? launch_gemm_pair<WA, 8>(a, b, M, N, K, c, ldc, gate, st) : BDR_ERR_UNSUPPORTED;
+                  return rc == BDR_ERR_UNSUPPORTED ? launch_gemm<WA, 8>(a, b, M, N, K, c, ldc, gate, st) : rc; }
     }
     return BDR_ERR_UNSUPPORTED;
 }
@@ -403,10 +409,9 @@ static int gemm_pick_b(int mb, const bdr_planes_t& a, const bdr_planes_t& b, int
 
 using namespace bdr;
 
-extern "C" {
-
-int mx_gemm(const bdr_config_t* cfg_a, const bdr_planes_t* a, const bdr_config_t* cfg_b, const bdr_planes_t* b, int64_t M,
-            int64_t N, int64_t K, float* c, int64_t ldc, void* stream) {
+// mx_gemm with an optional device-side gate: with gate != nullptr the kernel runs only if *gate != 0
+static int mx_gemm_gated(const bdr_config_t* cfg_a, const bdr_planes_t* a, const bdr_config_t* cfg_b, const bdr_planes_t* b, int64_t M,
+                         int64_t N, int64_t K, float* c, int64_t ldc, const int* gate, void* stream) {
     if (!cfg_a || !cfg_b || !a || !b || !c) return BDR_ERR_NULL;
     for (const bdr_config_t* cf : {cfg_a, cfg_b}) {
         if (cf->scale_kind != BDR_SCALE_POW2) return BDR_ERR_UNSUPPORTED;
@@ -428,11 +433,80 @@ int mx_gemm(const bdr_config_t* cfg_a, const bdr_planes_t* a, const bdr_config_t
     if ((uintptr_t)c % 16 || ldc % 4) return BDR_ERR_MISALIGNED;
     cudaStream_t st = (cudaStream_t)stream;
     switch (cfg_a->m) {
-        case 2: return gemm_pick_b<3>(cfg_b->m, *a, *b, M, N, K, c, ldc, st);
-        case 4: return gemm_pick_b<5>(cfg_b->m, *a, *b, M, N, K, c, ldc, st);
-        case 7: return gemm_pick_b<8>(cfg_b->m, *a, *b, M, N, K, c, ldc, st);
+        case 2: return gemm_pick_b<3>(cfg_b->m, *a, *b, M, N, K, c, ldc, gate, st);
+        case 4: return gemm_pick_b<5>(cfg_b->m, *a, *b, M, N, K, c, ldc, gate, st);
+        case 7: return gemm_pick_b<8>(cfg_b->m, *a, *b, M, N, K, c, ldc, gate, st);
     }
     return BDR_ERR_UNSUPPORTED;
+}
+
+extern "C" {
+
+int mx_gemm(const bdr_config_t* cfg_a, const bdr_planes_t* a, const bdr_config_t* cfg_b, const bdr_planes_t* b, int64_t M,
+            int64_t N, int64_t K, float* c, int64_t ldc, void* stream) {
+    return mx_gemm_gated(cfg_a, a, cfg_b, b, M, N, K, c, ldc, nullptr, stream);
+}
+
+// Workspace of mx_gemm_f8: both operands as E4M3 bytes, their scale atoms, and the flag word.
+int64_t mx_gemm_f8_workspace_bytes(int64_t M, int64_t N, int64_t K) {
+    if (M < 0 || N < 0 || K < 0) return 0;
+    return ((M + N) * K + (M + N) * K / 32 + 255) / 256 * 256 + 256;
+}
+
+int mx_gemm_f8(const bdr_config_t* cfg_a, const bdr_planes_t* a, const bdr_config_t* cfg_b, const bdr_planes_t* b, int64_t M,
+               int64_t N, int64_t K, float* c, int64_t ldc, void* workspace, int64_t workspace_bytes, void* stream) {
+    if (!cfg_a || !cfg_b || !a || !b || !c) return BDR_ERR_NULL;
+    for (const bdr_config_t* cf : {cfg_a, cfg_b}) {
+        if (cf->scale_kind != BDR_SCALE_POW2) return BDR_ERR_UNSUPPORTED;
+        if (cf->d1 != 8 || cf->k1 < 1 || cf->k2 < 1 || cf->k1 % cf->k2 != 0 || cf->d2 < 0 || cf->d2 > 3 || cf->m < 1 || cf->m > 8)
+            return BDR_ERR_BAD_CONFIG;
+        if (cf->k1 != 16 || cf->k2 != 2 || cf->d2 != 1 || (cf->m != 2 && cf->m != 4)) return BDR_ERR_UNSUPPORTED;
+    }
+    if (M < 0 || N < 0 || K < 0 || ldc < N) return BDR_ERR_SIZE;
+    if (M == 0 || N == 0) return BDR_OK;
+    if (M % 256 || N % 256 || K % 256 || K == 0) return BDR_ERR_UNSUPPORTED;
+    if (M >= (1ll << 31) || N >= (1ll << 31) || K >= (1ll << 31) || (M / 256) * (N / 256) >= (1ll << 30)) return BDR_ERR_UNSUPPORTED;
+    if (!workspace || workspace_bytes < mx_gemm_f8_workspace_bytes(M, N, K)) return BDR_ERR_WORKSPACE;
+    if ((uintptr_t)workspace % 256) return BDR_ERR_MISALIGNED;
+    cudaStream_t st = (cudaStream_t)stream;
+    uint8_t* wa = static_cast<uint8_t*>(workspace);
+    uint8_t* wb = wa + M * K;
+    uint8_t* sfa = wb + N * K;
+    uint8_t* sfb = sfa + M * K / 32;
+    int* flag = reinterpret_cast<int*>(wa + mx_gemm_f8_workspace_bytes(M, N, K) - 256);
+    // the fall-back's argument checks run first, so that nothing is launched for a call that would fail later
+    for (const bdr_planes_t* p : {a, b}) {
+        if (!p->exps || !p->micro || !p->elems) return BDR_ERR_NULL;
+        if (((uintptr_t)p->exps | (uintptr_t)p->micro | (uintptr_t)p->elems) % 16) return BDR_ERR_MISALIGNED;
+        if ((p->ld_exps | p->ld_micro | p->ld_elems) % 16) return BDR_ERR_MISALIGNED;
+    }
+    if (a->ld_exps < K / 16 || a->ld_micro < K / 16 || a->ld_elems < K * (cfg_a->m + 1) / 8) return BDR_ERR_SIZE;
+    if (b->ld_exps < K / 16 || b->ld_micro < K / 16 || b->ld_elems < K * (cfg_b->m + 1) / 8) return BDR_ERR_SIZE;
+    if ((uintptr_t)c % 16 || ldc % 4) return BDR_ERR_MISALIGNED;
+    if (cudaMemsetAsync(flag, 0, sizeof(int), st) != cudaSuccess) return BDR_ERR_CUDA;
+    int rc = reencode_rowwise_e4m3(*a, cfg_a->m, *b, cfg_b->m, M, N, K, wa, wb, sfa, sfb, flag, st);  // phase 1
+    if (rc != BDR_OK) return rc;
+    rc = launch_gemm_f8(wa, wb, sfa, sfb, M, N, K, c, ldc, flag, st);                                  // phase 2, if exact
+    if (rc != BDR_OK) return rc;
+    return mx_gemm_gated(cfg_a, a, cfg_b, b, M, N, K, c, ldc, flag, stream);                           // else the bf16 kernel
+}
+
+int bdr_reencode_e4m3(const bdr_config_t* cfg, const bdr_planes_t* in, int64_t rows, int64_t K, uint8_t* out, uint8_t* scales,
+                      int* inexact_dev, void* stream) {
+    if (!cfg || !in || !out || !scales || !inexact_dev) return BDR_ERR_NULL;
+    if (cfg->scale_kind != BDR_SCALE_POW2) return BDR_ERR_UNSUPPORTED;
+    if (cfg->d1 != 8 || cfg->k1 < 1 || cfg->k2 < 1 || cfg->k1 % cfg->k2 != 0 || cfg->d2 < 0 || cfg->d2 > 3 || cfg->m < 1 || cfg->m > 8)
+        return BDR_ERR_BAD_CONFIG;
+    if (cfg->k1 != 16 || cfg->k2 != 2 || cfg->d2 != 1 || (cfg->m != 2 && cfg->m != 4)) return BDR_ERR_UNSUPPORTED;
+    if (rows < 0 || K < 0) return BDR_ERR_SIZE;
+    if (rows == 0 || K == 0) return BDR_OK;
+    if (rows % 128 || K % 128) return BDR_ERR_UNSUPPORTED;
+    if (!in->exps || !in->micro || !in->elems) return BDR_ERR_NULL;
+    if (((uintptr_t)in->exps | (uintptr_t)in->micro | (uintptr_t)in->elems | (uintptr_t)out | (uintptr_t)scales) % 16) return BDR_ERR_MISALIGNED;
+    if ((in->ld_exps | in->ld_micro | in->ld_elems) % 4) return BDR_ERR_MISALIGNED;
+    if (in->ld_exps < K / 16 || in->ld_micro < K / 16 || in->ld_elems < K * (cfg->m + 1) / 8) return BDR_ERR_SIZE;
+    const bdr_planes_t none = {};
+    return reencode_rowwise_e4m3(*in, cfg->m, none, cfg->m, rows, 0, K, out, nullptr, scales, nullptr, inexact_dev, (cudaStream_t)stream);
 }
 
 int64_t mx_gemm_workspace_bytes(int64_t M, int64_t N, int64_t K) {

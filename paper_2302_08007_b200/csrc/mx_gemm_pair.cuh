@@ -176,7 +176,8 @@ __device__ __forceinline__ bool pair_decode_rows(uint32_t pk0, uint32_t pk_strid
 
 template <int WA, int WB>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kPairThreads, 1)
-mx_gemm_pair_kernel(const __grid_constant__ PairMaps maps, int64_t M, int64_t N, int64_t K, float* c, int64_t ldc) {
+mx_gemm_pair_kernel(const __grid_constant__ PairMaps maps, int64_t M, int64_t N, int64_t K, float* c, int64_t ldc, const int* gate) {
+    if (gate && *gate == 0) return;  // a fall-back launch that is not needed (the same for every thread of the grid)
     using SM = PairSmem<WA, WB>;
     constexpr int kStages = SM::kStages;
     extern __shared__ __align__(1024) uint8_t smem_raw[];
@@ -330,7 +331,7 @@ static bool make_plane_map(CUtensorMap* out, const uint8_t* base, int64_t rows, 
 
 template <int WA, int WB>
 int launch_gemm_pair(const bdr_planes_t& a, const bdr_planes_t& b, int64_t M, int64_t N, int64_t K, float* c, int64_t ldc,
-                     cudaStream_t st) {
+                     const int* gate, cudaStream_t st) {
     auto kern = mx_gemm_pair_kernel<WA, WB>;
     const size_t smem = PairSmem<WA, WB>::kBytes;
     static bool attr_done = false;
@@ -347,7 +348,7 @@ int launch_gemm_pair(const bdr_planes_t& a, const bdr_planes_t& b, int64_t M, in
                     make_plane_map(&maps.b_micro, b.micro, N, K / 16, b.ld_micro, 16);
     if (!ok) return BDR_ERR_UNSUPPORTED;  // caller falls back to the single-CTA kernel
     const dim3 grid((unsigned)(M / 128), (unsigned)(N / 256));  // x: CTAs (two per 256-row pair), y: column tiles
-    kern<<<grid, kPairThreads, smem, st>>>(maps, M, N, K, c, ldc);
+    kern<<<grid, kPairThreads, smem, st>>>(maps, M, N, K, c, ldc, gate);
     return cudaGetLastError() == cudaSuccess ? BDR_OK : BDR_ERR_CUDA;
 }
 

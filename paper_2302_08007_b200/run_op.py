@@ -35,13 +35,16 @@ def run_gemm(a, cfg):
     bdr.bdr_pack(cfg, A, pa)
     bdr.bdr_pack(cfg, B, pb)
     c = torch.empty((M, N), dtype=torch.float32, device="cuda")
-    if a.ws:
+    if a.f8:
+        ws = torch.empty(bdr.mx_gemm_f8_workspace_bytes(M, N, K), dtype=torch.uint8, device="cuda")
+        ms = _timed(lambda: bdr.mx_gemm_f8(cfg, pa, cfg, pb, M, N, K, c, ws), a.reps)
+    elif a.ws:
         ws = torch.empty(bdr.mx_gemm_workspace_bytes(M, N, K), dtype=torch.uint8, device="cuda")
         ms = _timed(lambda: bdr.mx_gemm_ws(cfg, pa, cfg, pb, M, N, K, c, ws), a.reps)
     else:
         ms = _timed(lambda: bdr.mx_gemm(cfg, pa, cfg, pb, M, N, K, c), a.reps)
     print("%s %s %dx%dx%d: %.4f ms per launch, %.1f TFLOP/s, status %d" % (
-        "mx_gemm_ws" if a.ws else "mx_gemm", a.fmt, M, N, K, ms, 2.0 * M * N * K / ms / 1e9, bdr.mx_gemm_status()))
+        "mx_gemm_f8" if a.f8 else "mx_gemm_ws" if a.ws else "mx_gemm", a.fmt, M, N, K, ms, 2.0 * M * N * K / ms / 1e9, bdr.mx_gemm_status()))
 
 
 def run_sweep(a):
@@ -66,6 +69,7 @@ def main():
     ap.add_argument("--reps", type=int, default=3)
     ap.add_argument("--no-sums", action="store_true")
     ap.add_argument("--ws", action="store_true", help="gemm: the two-phase entry point (mx_gemm_ws)")
+    ap.add_argument("--f8", action="store_true", help="gemm: the block-scaled 8-bit entry point (mx_gemm_f8; MX4 / MX6)")
     ap.add_argument("--no-y", action="store_true", help="quant_dequant: only the QSNR sums")
     a = ap.parse_args()
     cfg = FORMATS[a.fmt]
