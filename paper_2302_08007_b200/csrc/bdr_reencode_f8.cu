@@ -23,7 +23,7 @@ namespace bdr {
 
 constexpr int kF8Threads = 128;
 constexpr int kF8Warps = kF8Threads / 32;
-constexpr int kF8Rows = 4;                               // rows per warp, all in flight at once
+constexpr int kF8Rows = 2;                               // rows per warp, all in flight at once
 constexpr int kF8StripRows = kF8Warps * kF8Rows;        // rows per CTA (divides 128)
 
 __device__ __forceinline__ uint32_t cvt_e4m3x2(uint32_t h2) {
@@ -40,6 +40,15 @@ __device__ __forceinline__ uint32_t f16x2_mul(uint32_t a, uint32_t b) {
     uint32_t d;
     asm("mul.f16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
     return d;
+}
+
+// bits [pos, pos + len) of x with a left and a right shift (kept apart from the optimiser, which would turn them
+// into a shift and a mask, two operations of the integer pipe; the left shift can go to the multiplier)
+__device__ __forceinline__ uint32_t field_of(uint32_t x, int pos, int len) {
+    uint32_t t, f;
+    asm("shl.b32 %0, %1, %2;" : "=r"(t) : "r"(x), "r"(32 - pos - len));
+    asm("shr.u32 %0, %1, %2;" : "=r"(f) : "r"(t), "r"(32 - len));
+    return f;
 }
 
 // One 16-element block: W code words (LSB-first stream of 16 (m+1)-bit codes starting at bit 0 of w[0])
@@ -122,17 +131,28 @@ __device__ __forceinline__ uint32_t reencode_group(const uint32_t (&w)[W], uint3
 #pragma unroll
         for (int b = 0; b < 2; ++b) {
             const uint32_t Fp = (uint32_t)(14 - (S - (b ? F1 : F0))), mbb = b ? m2 >> 8 : m2;
-            const uint32_t sc0 = ((Fp - (uint32_t)(M - 1)) << 7) * 0x10001u;  // scale for tau = 0, both halves
+            const uint32_t sc0 = ((Fp - (uint32_t)(M - 1)) << 7) * 0x10001u;  // scale 2^p for tau = 0, both halves
             uint32_t v[8];
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
-                const uint32_t c2 = x2::code_pair<W, W>(w, 8 * b + j);
-                const uint32_t sc = ((mbb << (7 - j)) & 0x80u) * 0xFFFEFFFFu + sc0;   // tau lowers the exponent by one
-                const uint32_t y = x2::hfma2((c2 & kQ2) | 0x43004300u, sc, x2::hmul2(sc, 0xC300C300u));  // (128 + q) sc - 128 sc
-                v[j] = ((y >> 4) & 0x007F007Fu) | ((c2 << (7 - M)) & 0x00800080u);    // bytes 0 and 2
+                // the pair's 2 W code bits (a field inside one word comes out with a left and a right shift, no
+                // mask), copied three times by one multiply: code 0 ends up with its magnitude at bits 0.. and
+                // its sign at bit 15, code 1 with its magnitude at bits 16.. and its sign at bit 31
+                const int bit = 2 * W * (8 * b + j), wi = bit >> 5, sh = bit & 31;
+                uint32_t f;
+                if (sh + 2 * W > 32) f = __funnelshift_r(w[wi], w[wi + 1], sh) & ((1u << (2 * W)) - 1u);
+                else f = field_of(w[wi], sh, 2 * W);
+                const uint32_t c3 = f * (1u + (1u << (16 - W)) + (1u << (32 - 2 * W)));
+                // tau lowers the exponent by one: sc0 - 0x0080 per half, as one multiply-add; the constant term
+                // -128 * 2^p is a packed multiply (both on the FMA pipe, the integer pipe is the busy one)
+                const uint32_t sc = ((mbb << (7 - j)) & 0x80u) * 0xFFFEFFFFu + sc0;
+                const uint32_t y = x2::hfma2((c3 & kQ2) | 0x43004300u, sc, x2::hmul2(sc, 0xC300C300u));  // (128 + q) 2^p - 128 2^p
+                // bits 4..10 of each half move to bits 8..14 (a multiply) and the sign bits join them: the E4M3
+                // bytes are bytes 1 and 3
+                v[j] = y * 16u + (c3 & x2::kSign2);
             }
 #pragma unroll
-            for (int k = 0; k < 4; ++k) o[4 * b + k] = __byte_perm(v[2 * k], v[2 * k + 1], 0x6420);
+            for (int k = 0; k < 4; ++k) o[4 * b + k] = __byte_perm(v[2 * k], v[2 * k + 1], 0x7531);
         }
     } else {
         GroupWords<W> in;
