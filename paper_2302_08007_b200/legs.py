@@ -67,13 +67,17 @@ def gemm_leg(args) -> dict:
     ms_f8 = _time(lambda: bdr.mx_gemm_f8(bdr.MX6, pa, bdr.MX6, pb, M, N, K, c, ws8), reps=20, warmup=3)
     f8_exact = int(ws8[-256:-252].view(torch.int32).item()) == 0
     tf = lambda t: 2.0 * M * N * K / (t * 1e-3) / 1e12
-    return {"mx_gemm": {"metric": "MX-GEMM TFLOP/s", "value": tf(ms), "unit": "TFLOP/s", "ms": ms, "shape": [M, N, K],
-                        "format": "MX6 x MX6", "bound": "tensor",
-                        "entry_point": "mx_gemm_ws (both operands decoded once to a bf16 workspace, then a TMA-fed "
-                                       "tcgen05 GEMM; the time covers both phases)",
+    ws_name = ("mx_gemm_ws (both operands decoded once to a bf16 workspace, then a TMA-fed tcgen05 GEMM; the time "
+               "covers both phases)")
+    f8_name = ("mx_gemm_f8 (both operands re-encoded exactly to E4M3 with one E8M0 scale per 32 elements, then a "
+               "block-scaled tcgen05 GEMM; the time covers both phases and the gated fall-back launch)")
+    best_f8 = f8_exact and ms_f8 < ms
+    return {"mx_gemm": {"metric": "MX-GEMM TFLOP/s", "value": tf(ms_f8 if best_f8 else ms), "unit": "TFLOP/s",
+                        "ms": ms_f8 if best_f8 else ms, "shape": [M, N, K], "format": "MX6 x MX6", "bound": "tensor",
+                        "entry_point": f8_name if best_f8 else ws_name,
+                        "mx_gemm_ws": {"value": tf(ms), "unit": "TFLOP/s", "ms": ms},
+                        "mx_gemm_f8": {"value": tf(ms_f8), "unit": "TFLOP/s", "ms": ms_f8, "ran_on_8bit_path": f8_exact},
                         "fused_mx_gemm": {"value": tf(ms_fused), "unit": "TFLOP/s", "ms": ms_fused},
-                        "mx_gemm_f8": {"value": tf(ms_f8), "unit": "TFLOP/s", "ms": ms_f8, "ran_on_8bit_path": f8_exact,
-                                       "note": "E4M3 re-encoding + block-scaled tcgen05 GEMM, both phases timed"},
                         "status": bdr.mx_gemm_status()}}
 
 
