@@ -129,7 +129,8 @@ static int quant_dispatch(const QParams& qp, const T* x, T* y, int64_t rows, int
         else rc = quant_rowwise<T>(x, y, rows, cols, ld, qp, sums, st);
     } else {
         if constexpr (std::is_same<T, __nv_bfloat16>::value) {
-            if (!out || tight) rc = quant_colwise_mx_x2(x, y, rows, cols, ld, out, qp, sums, st);
+            if (!out) rc = quant_colwise_qd_x2(x, y, rows, cols, ld, qp, sums, st);
+            if (rc == BDR_ERR_UNSUPPORTED && (!out || tight)) rc = quant_colwise_mx_x2(x, y, rows, cols, ld, out, qp, sums, st);
             if (rc != BDR_ERR_UNSUPPORTED) return rc;
         }
         if (!out || tight) rc = quant_colwise_mx<T>(x, y, rows, cols, ld, out, qp, sums, st);

@@ -27,6 +27,8 @@ int quant_rowwise_mx_x2(const __nv_bfloat16* x, __nv_bfloat16* y, int64_t rows, 
 int pack_rowwise_mx_x2(const __nv_bfloat16* x, __nv_bfloat16* y, int64_t rows, int64_t cols, int64_t ld,
                        const bdr_planes_t& out, const QParams& qp, double* sums, cudaStream_t st);
 
+int quant_colwise_qd_x2(const __nv_bfloat16* x, __nv_bfloat16* y, int64_t rows, int64_t cols, int64_t ld, const QParams& qp,
+                        double* sums, cudaStream_t st);
 int quant_colwise_mx_x2(const __nv_bfloat16* x, __nv_bfloat16* y, int64_t rows, int64_t cols, int64_t ld,
                         const bdr_planes_t* out, const QParams& qp, double* sums, cudaStream_t st);  // bdr_col_x2.cu
 
