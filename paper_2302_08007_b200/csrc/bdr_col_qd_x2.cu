@@ -161,7 +161,7 @@ static int launch_col_qd(const bf16* x, bf16* y, int64_t rows, int64_t cols, int
     return cudaGetLastError() == cudaSuccess ? BDR_OK : BDR_ERR_CUDA;
 }
 
-constexpr int kQCols = 1024;
+constexpr int kQCols = 512;
 
 // Fast path without planes: whole slabs of 16 rows x kQCols columns, 16-byte aligned rows.
 // BDR_ERR_UNSUPPORTED sends the caller to the tile kernel and the generic column kernels.
