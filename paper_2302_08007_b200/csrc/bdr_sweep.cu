@@ -134,34 +134,45 @@ __device__ __forceinline__ void pow2_slice(const uint32_t (&u)[kSlice], const Sw
         for (int i = 0; i < K1S; ++i) a[i] = __fmul_rn(fabsf(__uint_as_float(u[b * K1S + i])), K);
 #pragma unroll
         for (int jj = 0; jj < K1S / K2; ++jj) dm[jj] = min(F23 - ej[b * (K1S / K2) + jj], beta23);
+        if constexpr (K1S >= 2) {
+            // Two elements per instruction (packed fp32 add / subtract / multiply-add; only the clamp is scalar).
+            // The shift moves into the operand: at = a * 2^tau is rounded with the constant of tau = 0, so the
+            // constant and the clamp are the same for the whole block, and the error comes back to a's scale
+            // with one multiply-add, a - (r - C) * 2^-tau (exact).
+            float at[K1S], sj[K1S / K2];
+#pragma unroll
+            for (int jj = 0; jj < K1S / K2; ++jj) sj[jj] = __uint_as_float(0xBF800000u - dm[jj]);  // -2^-tau
+#pragma unroll
+            for (int i = 0; i < K1S; ++i) at[i] = __fmul_rn(a[i], __uint_as_float(0x3F800000u + dm[i / K2]));
 #pragma unroll 2
-        for (int mi = 0; mi < c.nm; ++mi) {  // barely unrolled: keeps the instruction footprint of the 15 shapes small
-            const int m = c.m(mi);
-            const uint32_t c_base = ((uint32_t)(127 + 23 - (m - 1)) << 23) | 0x400000u;
-            const uint32_t qmax = (1u << m) - 1u;
-            float pe = 0.f;
-            if constexpr (K1S >= 2) {
-                // two elements per instruction (packed fp32 add / subtract / multiply-add); only the clamp is scalar
+            for (int mi = 0; mi < c.nm; ++mi) {  // barely unrolled: keeps the instruction footprint of the 15 shapes small
+                const int m = c.m(mi);
+                const uint32_t c_base = ((uint32_t)(127 + 23 - (m - 1)) << 23) | 0x400000u;
+                const float C = __uint_as_float(c_base), Cmax = __uint_as_float(c_base + (1u << m) - 1u);
                 float pe0 = 0.f, pe1 = 0.f;
 #pragma unroll
                 for (int k = 0; k < K1S / 2; ++k) {
-                    const uint32_t cb0 = c_base - dm[(2 * k) / K2], cb1 = c_base - dm[(2 * k + 1) / K2];
-                    const float C0 = __uint_as_float(cb0), C1 = __uint_as_float(cb1);
-                    float r0, r1;
-                    add_f32x2(r0, r1, a[2 * k], a[2 * k + 1], C0, C1);
-                    r0 = fminf(r0, __uint_as_float(cb0 + qmax));
-                    r1 = fminf(r1, __uint_as_float(cb1 + qmax));
-                    sub_f32x2(r0, r1, r0, r1, C0, C1);
-                    sub_f32x2(r0, r1, r0, r1, a[2 * k], a[2 * k + 1]);  // exact
-                    fma_f32x2(pe0, pe1, r0, r1, r0, r1);
+                    float r0, r1, e0 = a[2 * k], e1 = a[2 * k + 1];
+                    add_f32x2(r0, r1, at[2 * k], at[2 * k + 1], C, C);
+                    r0 = fminf(r0, Cmax);
+                    r1 = fminf(r1, Cmax);
+                    sub_f32x2(r0, r1, r0, r1, C, C);
+                    fma_f32x2(e0, e1, r0, r1, sj[(2 * k) / K2], sj[(2 * k + 1) / K2]);  // exact
+                    fma_f32x2(pe0, pe1, e0, e1, e0, e1);
                 }
-                pe = pe0 + pe1;
-            } else {
-                const uint32_t c_bits = c_base - dm[0];
-                const float C = __uint_as_float(c_bits), Cmax = __uint_as_float(c_bits + qmax);
-                const float de = __fsub_rn(__fsub_rn(fminf(__fadd_rn(a[0], C), Cmax), C), a[0]);  // exact
-                pe = de * de;
+                lane_acc[32 * mi] = fma((double)(pe0 + pe1), w, lane_acc[32 * mi]);
             }
+            continue;
+        }
+#pragma unroll 2
+        for (int mi = 0; mi < c.nm; ++mi) {
+            const int m = c.m(mi);
+            const uint32_t c_base = ((uint32_t)(127 + 23 - (m - 1)) << 23) | 0x400000u;
+            const uint32_t qmax = (1u << m) - 1u;
+            const uint32_t c_bits = c_base - dm[0];
+            const float C = __uint_as_float(c_bits), Cmax = __uint_as_float(c_bits + qmax);
+            const float de = __fsub_rn(__fsub_rn(fminf(__fadd_rn(a[0], C), Cmax), C), a[0]);  // exact
+            const float pe = de * de;
             lane_acc[32 * mi] = fma((double)pe, w, lane_acc[32 * mi]);
         }
     }
