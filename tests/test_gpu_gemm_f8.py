@@ -192,3 +192,35 @@ def test_f8_argument_errors():
         bdr.mx_gemm_f8(bdr.MX6, pa, bdr.MX6, pa, 256, 256, 128, c, ws)                 # K must be a multiple of 256
     assert e.value.status == -3
     torch.cuda.synchronize()
+
+
+@pytest.mark.parametrize("seed", range(12))
+def test_f8_random_exponent_structure(seed):
+    # block exponents drawn at random per 16-element block (spread chosen per case from "always representable" to
+    # "often not"), some blocks all zero, some rows scaled as a whole; whatever path the call takes on the device,
+    # the product must match the oracle, and the re-encoding must be exact whenever it says so
+    rng = np.random.default_rng(100 + seed)
+    M, N, K = 256, 256 * int(rng.integers(1, 3)), 256 * int(rng.integers(1, 5))
+    fa, fb = (bdr.MX6, bdr.MX4)[int(rng.integers(2))], (bdr.MX6, bdr.MX4)[int(rng.integers(2))]
+    spread = int(rng.choice([0, 3, 8, 12, 16, 24]))
+
+    def operand(rows):
+        mant = rng.standard_normal((rows, K))
+        e = rng.integers(-spread, 1, (rows, K // 16)) if spread else np.zeros((rows, K // 16), np.int64)
+        x = mant * np.repeat(np.ldexp(1.0, e), 16, axis=1)
+        x *= np.ldexp(1.0, rng.integers(-20, 20, (rows, 1)))
+        x[np.repeat(rng.random((rows, K // 16)) < 0.05, 16, axis=1)] = 0.0
+        return x.astype(np.float32)
+
+    a, b = operand(M), operand(N)
+    c, flag = gpu_gemm_f8(fa, a, fb, b)
+    assert rel_frob(c, oracle_gemm(fa, a, fb, b)) <= 1e-5, (seed, flag)
+    for cfg, x in ((fa, a), (fb, b)):
+        got, inexact, _, _ = _reencode(cfg, x)
+        want, _ = orc.quant_dequant(H.to_orc(cfg), x)
+        if not inexact:
+            assert np.array_equal(got, want.astype(np.float64)), seed
+        else:
+            assert flag == 1, seed
+    if spread <= 8:
+        assert flag == 0, seed
