@@ -46,8 +46,14 @@ int unpack_general(const bdr_planes_t& in, T* y, int64_t rows, int64_t cols, int
                    cudaStream_t st);
 
 // Packed MX4 / MX6 operands -> E4M3 bytes plus one power-of-two scale byte per 32 elements (bdr_reencode_f8.cu)
+struct ZeroTiles {   // `count` tiles of 256 x 256 floats of c (row pitch ldc, tiles_n tiles per row of tiles), from tile0 on
+    float* c;
+    int64_t ldc;
+    int tiles_n, tile0, count;
+};
 int reencode_rowwise_e4m3(const bdr_planes_t& a, int m_a, const bdr_planes_t& b, int m_b, int64_t M, int64_t N, int64_t K,
-                          uint8_t* out_a, uint8_t* out_b, uint8_t* sf_a, uint8_t* sf_b, int* inexact, cudaStream_t st);
+                          uint8_t* out_a, uint8_t* out_b, uint8_t* sf_a, uint8_t* sf_b, int* inexact, const ZeroTiles& z,
+                          cudaStream_t st);
 int unpack_rowwise_mx_x2(const bdr_planes_t& in, __nv_bfloat16* y, int64_t rows, int64_t cols, int64_t ld, const QParams& qp,
                          cudaStream_t st);  // bdr_unpack_x2.cu
 int unpack_colwise_mx_x2(const bdr_planes_t& in, __nv_bfloat16* y, int64_t rows, int64_t cols, int64_t ld, const QParams& qp,

@@ -207,12 +207,25 @@ __device__ __forceinline__ void reencode_rows(const bdr_planes_t& in, int64_t K,
     if (__any_sync(0xFFFFFFFFu, bad) && lane == 0) atomicExch(inexact, 1);
 }
 
-// grid (row strips of A + row strips of B, K segments): a CTA's warps take kF8Rows consecutive rows each
+// grid (row strips of A + row strips of B + tiles of C to clear, K segments): a CTA's warps take kF8Rows
+// consecutive rows each
 template <int WA, int WB>
 __global__ void __launch_bounds__(kF8Threads)
-reencode_e4m3_kernel(bdr_planes_t a, bdr_planes_t b, int a_strips, int64_t M, int64_t N, int64_t K, uint8_t* out_a, uint8_t* out_b,
-                     uint8_t* sf_a, uint8_t* sf_b, int* inexact) {
+reencode_e4m3_kernel(bdr_planes_t a, bdr_planes_t b, int a_strips, int b_strips, int64_t M, int64_t N, int64_t K, uint8_t* out_a,
+                     uint8_t* out_b, uint8_t* sf_a, uint8_t* sf_b, int* inexact, ZeroTiles z) {
     const int warp = threadIdx.x >> 5;
+    if ((int)blockIdx.x >= a_strips + b_strips) {
+        // extra CTAs: clear the 256 x 256 tiles of C that the GEMM kernel accumulates into
+        const int t = z.tile0 + ((int)blockIdx.x - a_strips - b_strips);
+        const int tm = t / z.tiles_n, tn = t - tm * z.tiles_n;
+        const int rows_per = (256 + (int)gridDim.y - 1) / (int)gridDim.y;
+        const int r0 = (int)blockIdx.y * rows_per, r1 = min(256, r0 + rows_per);
+        for (int idx = r0 * 64 + (int)threadIdx.x; idx < r1 * 64; idx += kF8Threads) {  // 64 chunks of 16 bytes per row
+            const int r = idx >> 6, ch = idx & 63;
+            *reinterpret_cast<uint4*>(z.c + ((int64_t)tm * 256 + r) * z.ldc + (int64_t)tn * 256 + ch * 4) = make_uint4(0, 0, 0, 0);
+        }
+        return;
+    }
     if ((int)blockIdx.x < a_strips) {
         const int64_t row0 = ((int64_t)blockIdx.x * kF8Warps + warp) * kF8Rows;
         reencode_rows<WA>(a, K, row0, blockIdx.y, out_a, sf_a, M / 128, inexact);
@@ -224,26 +237,27 @@ reencode_e4m3_kernel(bdr_planes_t a, bdr_planes_t b, int a_strips, int64_t M, in
 
 template <int WA, int WB>
 static int launch_reencode(const bdr_planes_t& a, const bdr_planes_t& b, int64_t M, int64_t N, int64_t K, uint8_t* out_a, uint8_t* out_b,
-                           uint8_t* sf_a, uint8_t* sf_b, int* inexact, cudaStream_t st) {
+                           uint8_t* sf_a, uint8_t* sf_b, int* inexact, const ZeroTiles& z, cudaStream_t st) {
     const int a_strips = (int)(M / kF8StripRows), b_strips = (int)(N / kF8StripRows);
-    const dim3 grid((unsigned)(a_strips + b_strips), (unsigned)((K + 1023) / 1024));
+    const dim3 grid((unsigned)(a_strips + b_strips + z.count), (unsigned)((K + 1023) / 1024));
     if (grid.x == 0) return BDR_OK;
-    reencode_e4m3_kernel<WA, WB><<<grid, kF8Threads, 0, st>>>(a, b, a_strips, M, N, K, out_a, out_b, sf_a, sf_b, inexact);
+    reencode_e4m3_kernel<WA, WB><<<grid, kF8Threads, 0, st>>>(a, b, a_strips, b_strips, M, N, K, out_a, out_b, sf_a, sf_b, inexact, z);
     return cudaGetLastError() == cudaSuccess ? BDR_OK : BDR_ERR_CUDA;
 }
 
 // Operand A [M, K] and operand B [N, K] (either may have zero rows) in one launch.  M and N are multiples of
 // 128, K a multiple of 128; m_a, m_b in {2, 4}; outputs 32-byte aligned, K bytes per row; scale atoms as
 // described above, M * K / 32 and N * K / 32 bytes.  *inexact is set to 1 (never cleared) when an
-// element cannot be represented.
+// element cannot be represented.  z.count tiles of 256 x 256 floats of z.c are cleared on the side.
 int reencode_rowwise_e4m3(const bdr_planes_t& a, int m_a, const bdr_planes_t& b, int m_b, int64_t M, int64_t N, int64_t K,
-                          uint8_t* out_a, uint8_t* out_b, uint8_t* sf_a, uint8_t* sf_b, int* inexact, cudaStream_t st) {
+                          uint8_t* out_a, uint8_t* out_b, uint8_t* sf_a, uint8_t* sf_b, int* inexact, const ZeroTiles& z,
+                          cudaStream_t st) {
     if (M % 128 || N % 128 || K % 128 || K <= 0) return BDR_ERR_UNSUPPORTED;
-    if ((M + N) / kF8StripRows > 0x7FFFFFFF || (K + 1023) / 1024 > 65535) return BDR_ERR_UNSUPPORTED;
-    if (m_a == 2 && m_b == 2) return launch_reencode<3, 3>(a, b, M, N, K, out_a, out_b, sf_a, sf_b, inexact, st);
-    if (m_a == 2 && m_b == 4) return launch_reencode<3, 5>(a, b, M, N, K, out_a, out_b, sf_a, sf_b, inexact, st);
-    if (m_a == 4 && m_b == 2) return launch_reencode<5, 3>(a, b, M, N, K, out_a, out_b, sf_a, sf_b, inexact, st);
-    if (m_a == 4 && m_b == 4) return launch_reencode<5, 5>(a, b, M, N, K, out_a, out_b, sf_a, sf_b, inexact, st);
+    if ((M + N) / kF8StripRows + z.count > 0x7FFFFFFF || (K + 1023) / 1024 > 65535) return BDR_ERR_UNSUPPORTED;
+    if (m_a == 2 && m_b == 2) return launch_reencode<3, 3>(a, b, M, N, K, out_a, out_b, sf_a, sf_b, inexact, z, st);
+    if (m_a == 2 && m_b == 4) return launch_reencode<3, 5>(a, b, M, N, K, out_a, out_b, sf_a, sf_b, inexact, z, st);
+    if (m_a == 4 && m_b == 2) return launch_reencode<5, 3>(a, b, M, N, K, out_a, out_b, sf_a, sf_b, inexact, z, st);
+    if (m_a == 4 && m_b == 4) return launch_reencode<5, 5>(a, b, M, N, K, out_a, out_b, sf_a, sf_b, inexact, z, st);
     return BDR_ERR_UNSUPPORTED;
 }
 

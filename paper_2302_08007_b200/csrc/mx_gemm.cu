@@ -484,9 +484,11 @@ int mx_gemm_f8(const bdr_config_t* cfg_a, const bdr_planes_t* a, const bdr_confi
     if (b->ld_exps < K / 16 || b->ld_micro < K / 16 || b->ld_elems < K * (cfg_b->m + 1) / 8) return BDR_ERR_SIZE;
     if ((uintptr_t)c % 16 || ldc % 4) return BDR_ERR_MISALIGNED;
     if (cudaMemsetAsync(flag, 0, sizeof(int), st) != cudaSuccess) return BDR_ERR_CUDA;
-    int rc = reencode_rowwise_e4m3(*a, cfg_a->m, *b, cfg_b->m, M, N, K, wa, wb, sfa, sfb, flag, st);  // phase 1
+    const F8Plan plan = plan_gemm_f8(M, N, K);
+    const ZeroTiles z = {c, ldc, plan.tiles_n, plan.tiles_full, plan.split_tiles()};
+    int rc = reencode_rowwise_e4m3(*a, cfg_a->m, *b, cfg_b->m, M, N, K, wa, wb, sfa, sfb, flag, z, st);  // phase 1
     if (rc != BDR_OK) return rc;
-    rc = launch_gemm_f8(wa, wb, sfa, sfb, M, N, K, c, ldc, flag, st);                                  // phase 2, if exact
+    rc = launch_gemm_f8(wa, wb, sfa, sfb, M, N, K, plan, c, ldc, flag, st);                               // phase 2, if exact
     if (rc != BDR_OK) return rc;
     return mx_gemm_gated(cfg_a, a, cfg_b, b, M, N, K, c, ldc, flag, stream);                           // else the bf16 kernel
 }
@@ -506,7 +508,8 @@ int bdr_reencode_e4m3(const bdr_config_t* cfg, const bdr_planes_t* in, int64_t r
     if ((in->ld_exps | in->ld_micro | in->ld_elems) % 4) return BDR_ERR_MISALIGNED;
     if (in->ld_exps < K / 16 || in->ld_micro < K / 16 || in->ld_elems < K * (cfg->m + 1) / 8) return BDR_ERR_SIZE;
     const bdr_planes_t none = {};
-    return reencode_rowwise_e4m3(*in, cfg->m, none, cfg->m, rows, 0, K, out, nullptr, scales, nullptr, inexact_dev, (cudaStream_t)stream);
+    const ZeroTiles z = {nullptr, 0, 1, 0, 0};
+    return reencode_rowwise_e4m3(*in, cfg->m, none, cfg->m, rows, 0, K, out, nullptr, scales, nullptr, inexact_dev, z, (cudaStream_t)stream);
 }
 
 int64_t mx_gemm_workspace_bytes(int64_t M, int64_t N, int64_t K) {

@@ -14,7 +14,10 @@
 //     the scale-factor id in the instruction descriptor;
 //   * tensor memory holds one 256-column accumulator plus 12 scale columns per stage, so the epilogue
 //     does not overlap the next tile's main loop through a second buffer; instead each epilogue warp
-//     pulls its 32 x 128 block into registers, releases the accumulator, and only then stores.
+//     pulls its 32 x 128 block into registers, releases the accumulator, and only then stores;
+//   * when the last round of tiles would keep at most half of the clusters busy, each of its tiles is
+//     computed as two halves of the K range by two clusters that add (red.global.add) into a tile the
+//     re-encoding launch has cleared.
 // The kernel returns at once when *gate is non-zero (the operands were not representable).
 // Every wait is bounded.  (textually included by mx_gemm.cu after mx_gemm_dense.cuh)
 #pragma once
@@ -70,6 +73,11 @@ __device__ __forceinline__ void umma2_mxf8(uint32_t tmem_d, uint64_t desc_a, uin
         ::"r"(tmem_d), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate), "r"(tmem_sfa), "r"(tmem_sfb)
         : "memory");
 }
+__device__ __forceinline__ void red_add_v4(float* p, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+    asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(p), "f"(__uint_as_float(a)), "f"(__uint_as_float(b)),
+                 "f"(__uint_as_float(c)), "f"(__uint_as_float(d))
+                 : "memory");
+}
 __device__ __forceinline__ void bulk_load_g2s(void* smem_dst, const void* gsrc, uint32_t bytes, uint64_t* bar) {
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(smem_u32(smem_dst)),
                  "l"(gsrc), "r"(bytes), "r"(smem_u32(bar))
@@ -78,7 +86,7 @@ __device__ __forceinline__ void bulk_load_g2s(void* smem_dst, const void* gsrc, 
 
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kFThreads, 1)
 mxf8_gemm_pair_kernel(const __grid_constant__ F8Maps maps, const uint8_t* sf_a, const uint8_t* sf_b, int tiles_m, int tiles_n, int nk,
-                      float* c, int64_t ldc, const int* gate) {
+                      int tiles_full, int n_items, float* c, int64_t ldc, const int* gate) {
     if (gate && *gate != 0) return;  // the same for every thread of the grid
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     uint8_t* stages = reinterpret_cast<uint8_t*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
@@ -86,7 +94,13 @@ mxf8_gemm_pair_kernel(const __grid_constant__ F8Maps maps, const uint8_t* sf_a, 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = cluster_ctarank();
     const int cluster_id = blockIdx.x >> 1, n_clusters = gridDim.x >> 1;
-    const int n_tiles = tiles_m * tiles_n;
+    // Work items: the first tiles_full tiles with their whole K range (a multiple of the cluster count: whole
+    // rounds), then every remaining tile as two items of half the K range each, which add their results into a
+    // zeroed C tile -- so a last round that would keep less than half of the clusters busy takes half as long.
+    auto item_of = [&](int i, int& t, int& k0, int& cnt, bool& add) {
+        if (i < tiles_full) { t = i; k0 = 0; cnt = nk; add = false; }
+        else { const int j = i - tiles_full; t = tiles_full + (j >> 1); cnt = nk >> 1; k0 = (j & 1) * cnt; add = true; }
+    };
     const int64_t row_tiles_a = (int64_t)tiles_m * 2, row_tiles_b = (int64_t)tiles_n * 2;  // 128-row tiles of the scale atoms
 
     if (threadIdx.x == 0) {
@@ -113,10 +127,13 @@ mxf8_gemm_pair_kernel(const __grid_constant__ F8Maps maps, const uint8_t* sf_a, 
             uint64_t* const my_full = rank == 0 ? bars.full : bars.full_local;
             bool ok = true;
             uint32_t it = 0;  // running K-step count across tiles
-            for (int t = cluster_id; t < n_tiles && ok; t += n_clusters) {
+            for (int i = cluster_id; i < n_items && ok; i += n_clusters) {
+                int t, k0, cnt;
+                bool add;
+                item_of(i, t, k0, cnt, add);
                 const int tm = t / tiles_n, tn = t - tm * tiles_n;
                 const int row_a = (tm * 2 + (int)rank) * kPairRows, row_b = (tn * 2 + (int)rank) * kPairRows;
-                for (int kk = 0; kk < nk; ++kk, ++it) {
+                for (int kk = k0; kk < k0 + cnt; ++kk, ++it) {
                     const int stage = it % kFStages;
                     if (it >= kFStages) {
                         ok = mbar_wait(&bars.empty[stage], ((it / kFStages) - 1) & 1);
@@ -142,13 +159,16 @@ mxf8_gemm_pair_kernel(const __grid_constant__ F8Maps maps, const uint8_t* sf_a, 
             if (rank == 0) {
                 // ---------------- MMA issuer (leader CTA) ----------------
                 int tcount = 0;
-                for (int t = cluster_id; t < n_tiles && ok; t += n_clusters, ++tcount) {
+                for (int i = cluster_id; i < n_items && ok; i += n_clusters, ++tcount) {
+                    int t, k0, cnt;
+                    bool add;
+                    item_of(i, t, k0, cnt, add);
                     if (tcount >= 1) {  // the epilogues of both CTAs hold the previous tile in registers
                         ok = mbar_wait_cluster(&bars.tmem_empty, (tcount - 1) & 1);
                         if (!ok) break;
                         tc_fence_after();
                     }
-                    for (int kk = 0; kk < nk; ++kk, ++it) {
+                    for (int kk = 0; kk < cnt; ++kk, ++it) {
                         const int stage = it % kFStages;
                         ok = mbar_wait_cluster(&bars.full[stage], (it / kFStages) & 1);
                         if (!ok) break;
@@ -169,8 +189,11 @@ mxf8_gemm_pair_kernel(const __grid_constant__ F8Maps maps, const uint8_t* sf_a, 
                 }
             } else {
                 // ---------------- relay (peer CTA): "my half of the stage has landed" ----------------
-                for (int t = cluster_id; t < n_tiles && ok; t += n_clusters) {
-                    for (int kk = 0; kk < nk; ++kk, ++it) {
+                for (int i = cluster_id; i < n_items && ok; i += n_clusters) {
+                    int t, k0, cnt;
+                    bool add;
+                    item_of(i, t, k0, cnt, add);
+                    for (int kk = 0; kk < cnt; ++kk, ++it) {
                         const int stage = it % kFStages;
                         ok = mbar_wait(&bars.full_local[stage], (it / kFStages) & 1);
                         if (!ok) break;
@@ -189,7 +212,10 @@ mxf8_gemm_pair_kernel(const __grid_constant__ F8Maps maps, const uint8_t* sf_a, 
         const int col_base = (ew >> 2) * 128;      // two warps share a lane quarter: 128 columns each
         bool ok = true;
         int tcount = 0;
-        for (int t = cluster_id; t < n_tiles; t += n_clusters, ++tcount) {
+        for (int i = cluster_id; i < n_items; i += n_clusters, ++tcount) {
+            int t, k0, cnt;
+            bool add;
+            item_of(i, t, k0, cnt, add);
             ok = ok && mbar_wait(&bars.tmem_full, tcount & 1);
             ok = __all_sync(0xFFFFFFFFu, ok);
             if (!ok) break;
@@ -204,11 +230,19 @@ mxf8_gemm_pair_kernel(const __grid_constant__ F8Maps maps, const uint8_t* sf_a, 
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive_cluster(&bars.tmem_empty, 0);  // the next tile may overwrite the accumulator
+            if (!add) {
 #pragma unroll
-            for (int q = 0; q < 4; ++q)
+                for (int q = 0; q < 4; ++q)
 #pragma unroll
-                for (int j = 0; j < 8; ++j)
-                    *reinterpret_cast<uint4*>(crow + 32 * q + 4 * j) = make_uint4(v[q][4 * j], v[q][4 * j + 1], v[q][4 * j + 2], v[q][4 * j + 3]);
+                    for (int j = 0; j < 8; ++j)
+                        *reinterpret_cast<uint4*>(crow + 32 * q + 4 * j) = make_uint4(v[q][4 * j], v[q][4 * j + 1], v[q][4 * j + 2], v[q][4 * j + 3]);
+            } else {  // half of the K range: add to the zeroed tile (two terms, so the order does not matter)
+#pragma unroll
+                for (int q = 0; q < 4; ++q)
+#pragma unroll
+                    for (int j = 0; j < 8; ++j)
+                        red_add_v4(crow + 32 * q + 4 * j, v[q][4 * j], v[q][4 * j + 1], v[q][4 * j + 2], v[q][4 * j + 3]);
+            }
         }
         if (!ok) bars.failed = 1;
         tc_fence_before();
@@ -233,10 +267,30 @@ static bool make_f8_map(CUtensorMap* out, const void* base, int64_t rows, int64_
               CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// How the tiles of an M x N product are handed out: n_clusters clusters, tiles_full tiles with their whole K
+// range, the remaining tiles (fewer than half the cluster count) in two halves of K each.
+struct F8Plan {
+    int tiles_m, tiles_n, n_clusters, tiles_full, n_items;
+    int split_tiles() const { return tiles_m * tiles_n - tiles_full; }
+};
+static F8Plan plan_gemm_f8(int64_t M, int64_t N, int64_t K) {
+    F8Plan p;
+    p.tiles_m = (int)(M / 256);
+    p.tiles_n = (int)(N / 256);
+    const int T = p.tiles_m * p.tiles_n, cmax = sm_count() / 2;
+    p.n_clusters = std::min(T, cmax);
+    const int rest = T % cmax;
+    const bool split = rest > 0 && 2 * rest <= cmax && (K / kFBK) % 2 == 0;
+    p.tiles_full = split ? T - rest : T;
+    p.n_items = p.tiles_full + 2 * (T - p.tiles_full);
+    if (split) p.n_clusters = std::min(p.n_items, cmax);
+    return p;
+}
+
 // a_e4m3 [M, K], b_e4m3 [N, K] bytes, contiguous; scale atoms ordered [K / 128][rows / 128][512];
-// M, N multiples of 256, K a multiple of 128
+// M, N multiples of 256, K a multiple of 128.  The tiles plan.tiles_full .. of C must hold zeros.
 static int launch_gemm_f8(const uint8_t* a_e4m3, const uint8_t* b_e4m3, const uint8_t* sf_a, const uint8_t* sf_b, int64_t M, int64_t N,
-                          int64_t K, float* c, int64_t ldc, const int* gate, cudaStream_t st) {
+                          int64_t K, const F8Plan& plan, float* c, int64_t ldc, const int* gate, cudaStream_t st) {
     static bool attr_done = false;
     if (!attr_done) {
         if (cudaFuncSetAttribute(mxf8_gemm_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kFSmemBytes) != cudaSuccess)
@@ -245,10 +299,8 @@ static int launch_gemm_f8(const uint8_t* a_e4m3, const uint8_t* b_e4m3, const ui
     }
     F8Maps maps;
     if (!make_f8_map(&maps.a, a_e4m3, M, K) || !make_f8_map(&maps.b, b_e4m3, N, K)) return BDR_ERR_CUDA;
-    const int tiles_m = (int)(M / 256), tiles_n = (int)(N / 256);
-    const int64_t n_tiles = (int64_t)tiles_m * tiles_n;
-    const int n_clusters = (int)std::min<int64_t>(n_tiles, sm_count() / 2);
-    mxf8_gemm_pair_kernel<<<2 * n_clusters, kFThreads, kFSmemBytes, st>>>(maps, sf_a, sf_b, tiles_m, tiles_n, (int)(K / kFBK), c, ldc, gate);
+    mxf8_gemm_pair_kernel<<<2 * plan.n_clusters, kFThreads, kFSmemBytes, st>>>(maps, sf_a, sf_b, plan.tiles_m, plan.tiles_n, (int)(K / kFBK),
+                                                                              plan.tiles_full, plan.n_items, c, ldc, gate);
     return cudaGetLastError() == cudaSuccess ? BDR_OK : BDR_ERR_CUDA;
 }
 

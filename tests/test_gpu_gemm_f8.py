@@ -147,6 +147,17 @@ def test_f8_more_tiles_than_clusters():
     assert rel_frob(c, oracle_gemm(bdr.MX6, a, bdr.MX6, b)) <= 1e-5
 
 
+def test_f8_whole_rounds_only():
+    # 64 tiles on 74 clusters: more than half of the clusters are busy in the only round, so no tile's K range is
+    # split in two (the other tests have few tiles, or a sparse last round, and take the split path)
+    M, N, K = 2048, 2048, 256
+    a = synth.normal_matrix(M, K, seed=11, stream=1)
+    b = synth.normal_matrix(N, K, seed=11, stream=2, sigma=0.02)
+    c, flag = gpu_gemm_f8(bdr.MX4, a, bdr.MX6, b)
+    assert flag == 0
+    assert rel_frob(c, oracle_gemm(bdr.MX4, a, bdr.MX6, b)) <= 1e-5
+
+
 def test_f8_falls_back_when_the_operands_are_not_representable():
     M, N, K = 256, 256, 512
     a = synth.normal_matrix(M, K, seed=9, stream=1)
