@@ -36,15 +36,15 @@ FALLBACK_HBM_GBS = 6650.0
 # profiles/step_kernels_dram_traffic.md.  Writes that still sit in L2 when a kernel ends are not
 # counted by those counters, which is why some figures are below the algorithmic bytes.
 NCU_TRAFFIC_BYTES: dict[str, float | None] = {
-    "quant_dequant_MX4_row": 215910144, "quant_dequant_MX4_col": 217317376,
-    "quant_dequant_MX6_row": 216769536, "quant_dequant_MX6_col": 217431552,
-    "quant_dequant_MX9_row": 217173504, "quant_dequant_MX9_col": 217409024,
-    "pack_MX4_row": 148965888, "pack_MX4_col": 146423552,
-    "pack_MX6_row": 157351168, "pack_MX6_col": 154226432,
-    "pack_MX9_row": 173277696, "pack_MX9_col": 167642368,
-    "unpack_MX4_row": 111672320, "unpack_MX4_col": 109009664,
-    "unpack_MX6_row": 128769792, "unpack_MX6_col": 126806784,
-    "unpack_MX9_row": 154996992, "unpack_MX9_col": 151483904,
+    "quant_dequant_MX4_row": 217483776, "quant_dequant_MX4_col": 216174336,
+    "quant_dequant_MX6_row": 216457216, "quant_dequant_MX6_col": 215976192,
+    "quant_dequant_MX9_row": 216821760, "quant_dequant_MX9_col": 216307200,
+    "pack_MX4_row": 148817664, "pack_MX4_col": 147564288,
+    "pack_MX6_row": 157307904, "pack_MX6_col": 155158784,
+    "pack_MX9_row": 173331712, "pack_MX9_col": 168369664,
+    "unpack_MX4_row": 112468736, "unpack_MX4_col": 109030656,
+    "unpack_MX6_row": 128452352, "unpack_MX6_col": 128861440,
+    "unpack_MX9_row": 154516736, "unpack_MX9_col": 153580800,
 }
 
 
