@@ -8,10 +8,12 @@
 //   * a K step is 128 elements (128-byte rows, 128-byte swizzle), four MMAs of K = 32;
 //   * every stage also carries the scale atoms of its K chunk -- 512 bytes for this CTA's 128 rows of A
 //     and 1024 bytes for all 256 rows of the B tile (each CTA's tensor memory needs the scales of every
-//     column it accumulates) -- fetched with plain bulk copies on the stage's barrier; the MMA thread
-//     copies them to tensor memory (tcgen05.cp, 32 lanes x 128 bits replicated over the four lane
-//     quarters) right before the stage's MMAs; the MMA picks the scale byte of its K = 32 slice with
-//     the scale-factor id in the instruction descriptor;
+//     column it accumulates) -- fetched with plain bulk copies on the stage's barrier; a warp of its own in
+//     the leader CTA copies them to the tensor memory of both CTAs (tcgen05.cp, 32 lanes x 128 bits
+//     replicated over the four lane quarters) as soon as the stage has landed and commits to a
+//     "scales ready" barrier that the MMA thread waits on (issued from the MMA thread itself the three copies
+//     per K step cost 17 % of the kernel: they serialise with its MMAs; from another thread they overlap);
+//     the MMA picks the scale byte of its K = 32 slice with the scale-factor id in the instruction descriptor;
 //   * tensor memory holds one 256-column accumulator plus 12 scale columns per stage, so the epilogue
 //     does not overlap the next tile's main loop through a second buffer; instead each epilogue warp
 //     pulls its 32 x 128 block into registers, releases the accumulator, and only then stores;
@@ -31,13 +33,14 @@ constexpr int kFSfaBytes = 512, kFSfbBytes = 1024;
 constexpr int kFStageBytes = kFTileBytes + 2048;            // tiles, then scales of A, then scales of B (1024-byte multiple)
 constexpr int kFTxBytes = kFTileBytes + kFSfaBytes + kFSfbBytes;
 constexpr int kFEpiWarps = 8;
-constexpr int kFThreads = (2 + kFEpiWarps) * 32;
+constexpr int kFThreads = (3 + kFEpiWarps) * 32;            // producer, MMA / relay, 8 epilogue warps, scale copier
+constexpr int kFCopyWarp = 2 + kFEpiWarps;
 constexpr size_t kFSmemBytes = (size_t)kFStages * kFStageBytes + 1024 /*bookkeeping*/ + 1024 /*alignment*/;
 constexpr uint32_t kFSfCol0 = 256;                          // first scale column in tensor memory
 constexpr uint32_t kFSfColsPerStage = 12;                   // 4 (A: 128 rows) + 8 (B: 256 rows)
 
 struct F8Bars {
-    uint64_t full[kFStages], full_local[kFStages], empty[kFStages], tmem_full, tmem_empty;
+    uint64_t full[kFStages], full_local[kFStages], empty[kFStages], sf_ready[kFStages], tmem_full, tmem_empty;
     uint32_t tmem_base;
     int failed;
 };
@@ -63,6 +66,12 @@ __device__ __forceinline__ uint64_t make_sf_desc(uint32_t smem_addr) {
 }
 __device__ __forceinline__ void sf_copy2(uint32_t tmem_dst, uint64_t desc) {
     asm volatile("tcgen05.cp.cta_group::2.32x128b.warpx4 [%0], %1;" ::"r"(tmem_dst), "l"(desc) : "memory");
+}
+__device__ __forceinline__ void umma_commit2_leader(uint64_t* bar) {  // arrives on the leader CTA's barrier only
+    const uint16_t mask = 1;
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                 ::"r"(smem_u32(bar)), "h"(mask)
+                 : "memory");
 }
 __device__ __forceinline__ void umma2_mxf8(uint32_t tmem_d, uint64_t desc_a, uint64_t desc_b, uint32_t idesc, uint32_t accumulate,
                                            uint32_t tmem_sfa, uint32_t tmem_sfb) {
@@ -107,7 +116,8 @@ mxf8_gemm_pair_kernel(const __grid_constant__ F8Maps maps, const uint8_t* sf_a, 
         for (int s = 0; s < kFStages; ++s) {
             mbar_init(&bars.full[s], 2);        // leader: its own bytes (arrive.expect_tx) + the peer's relay
             mbar_init(&bars.full_local[s], 1);  // peer: its own bytes
-            mbar_init(&bars.empty[s], 1);       // multicast commit of the copies and MMAs that read the stage
+            mbar_init(&bars.empty[s], 1);       // multicast commit of the MMAs that read the stage
+            mbar_init(&bars.sf_ready[s], 1);    // leader: commit of the stage's scale copies
         }
         mbar_init(&bars.tmem_full, 1);                  // multicast commit after a tile's last K step
         mbar_init(&bars.tmem_empty, 2 * kFEpiWarps);    // leader: every epilogue warp of both CTAs
@@ -170,14 +180,11 @@ mxf8_gemm_pair_kernel(const __grid_constant__ F8Maps maps, const uint8_t* sf_a, 
                     }
                     for (int kk = 0; kk < cnt; ++kk, ++it) {
                         const int stage = it % kFStages;
-                        ok = mbar_wait_cluster(&bars.full[stage], (it / kFStages) & 1);
+                        ok = mbar_wait_cluster(&bars.sf_ready[stage], (it / kFStages) & 1);  // data landed, scales copied
                         if (!ok) break;
                         tc_fence_after();
                         const uint32_t sa = smem_u32(stages + stage * kFStageBytes);
                         const uint32_t tsfa = tmem_base + kFSfCol0 + (uint32_t)stage * kFSfColsPerStage, tsfb = tsfa + 4;
-                        sf_copy2(tsfa, make_sf_desc(sa + kFTileBytes));
-                        sf_copy2(tsfb, make_sf_desc(sa + kFTileBytes + kFSfaBytes));
-                        sf_copy2(tsfb + 4, make_sf_desc(sa + kFTileBytes + kFSfaBytes + 512));
                         const uint64_t da = make_smem_desc(sa), db = make_smem_desc(sa + kPairRows * kFBK);
 #pragma unroll
                         for (int k = 0; k < kFBK / 32; ++k)  // 32 bytes of K per MMA; scale byte k of the columns
@@ -199,6 +206,33 @@ mxf8_gemm_pair_kernel(const __grid_constant__ F8Maps maps, const uint8_t* sf_a, 
                         if (!ok) break;
                         mbar_arrive_cluster(&bars.full[stage], 0);
                     }
+                }
+            }
+            if (!ok) bars.failed = 1;
+        }
+        __syncwarp();
+        tc_fence_before();
+    } else if (warp == kFCopyWarp) {
+        // ---------------- scale copier (leader CTA): shared memory -> tensor memory of both CTAs ----------------
+        if (lane == 0 && rank == 0) {
+            bool ok = true;
+            uint32_t it = 0;
+            for (int i = cluster_id; i < n_items && ok; i += n_clusters) {
+                int t, k0, cnt;
+                bool add;
+                item_of(i, t, k0, cnt, add);
+                for (int kk = 0; kk < cnt; ++kk, ++it) {
+                    const int stage = it % kFStages;
+                    // (the stage's previous MMAs are done: the producer refilled it only after their commit)
+                    ok = mbar_wait_cluster(&bars.full[stage], (it / kFStages) & 1);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const uint32_t sf = smem_u32(stages + stage * kFStageBytes) + kFTileBytes;
+                    const uint32_t tsfa = tmem_base + kFSfCol0 + (uint32_t)stage * kFSfColsPerStage;
+                    sf_copy2(tsfa, make_sf_desc(sf));
+                    sf_copy2(tsfa + 4, make_sf_desc(sf + kFSfaBytes));
+                    sf_copy2(tsfa + 8, make_sf_desc(sf + kFSfaBytes + 512));
+                    umma_commit2_leader(&bars.sf_ready[stage]);
                 }
             }
             if (!ok) bars.failed = 1;
