@@ -204,8 +204,9 @@ int mx_gemm_f8(const bdr_config_t* cfg_a /*host*/, const bdr_planes_t* a /*host 
  *   scales   rows * K / 32 bytes (device): for every 128 rows x 128 K a 512-byte atom holding the scale
  *            exponent (value 2^(byte - 127)) of row r, K group g (32 elements) at (r % 32) * 16 + (r / 32) * 4 + g;
  *            atoms ordered [K / 128][rows / 128]
- *   inexact_dev  one int (device): set to 1 if some element is not representable (then its byte holds
- *            the nearest E4M3 value); never cleared by this call
+ *   inexact_dev  one int (device): set to 1 if some element is not representable, if a block with an
+ *            exponent field below 16 holds a non-zero element, or if a block has the exponent field 255
+ *            (the bytes of `out` are then unspecified); never cleared by this call
  * so that element = E4M3(out) * 2^(scale - 127) exactly.  rows and K multiples of 128; 16-byte aligned
  * pointers. */
 int bdr_reencode_e4m3(const bdr_config_t* cfg /*host*/, const bdr_planes_t* in /*host struct*/, int64_t rows, int64_t K,

@@ -6,6 +6,7 @@ import pytest
 import torch
 
 from oracle import oracle as orc
+from oracle import reencode as orc_re
 from paper_2302_08007_b200 import binding as bdr
 from paper_2302_08007_b200 import synth
 from tests import helpers as H
@@ -30,6 +31,12 @@ def _reencode(cfg, x_host):
     flag = torch.zeros(1, dtype=torch.int32, device="cuda")
     bdr.bdr_reencode_e4m3(cfg, p, rows, K, out, sf, flag)
     torch.cuda.synchronize()
+    # bytes, scale bytes and the flag against the oracle's re-encoding (bytes are unspecified once the flag is up)
+    want_out, want_sf, want_flag = orc_re.reencode_e4m3(H.to_orc(cfg), x_host)
+    assert int(flag.item()) == int(want_flag)
+    if not want_flag:
+        assert np.array_equal(out.cpu().numpy(), want_out)
+    assert np.array_equal(sf.cpu().numpy(), want_sf)
     vals = out.view(torch.float8_e4m3fn).to(torch.float32).cpu().numpy().astype(np.float64)
     # scale of (row r, group g): atom [g // 4][r // 128], byte (r % 32) * 16 + ((r % 128) // 32) * 4 + g % 4
     sfh = sf.cpu().numpy().reshape(K // 128, rows // 128, 32, 4, 4)          # [chunk][row tile][r % 32][(r % 128) // 32][g % 4]

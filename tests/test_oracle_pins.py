@@ -447,3 +447,43 @@ def test_multithreaded_oracle_is_the_same_function():
         a, sa = orc.quant_dequant(orc.MX6, x, axis=axis)
         b, sb = orc.quant_dequant(orc.MX6, x, axis=axis, nthreads=4)
         assert np.array_equal(a, b) and sa == sb
+
+
+# ---- re-encoding onto E4M3 + power-of-two block scales (library extension; oracle/reencode.py) ----------------
+def test_e4m3_byte_table_matches_the_library_cast():
+    torch = pytest.importorskip("torch")
+    from oracle import reencode as R
+    lib_vals = torch.arange(256, dtype=torch.uint8).view(torch.float8_e4m3fn).to(torch.float32).numpy().astype(np.float64)
+    table = R.e4m3_value_table()
+    assert np.array_equal(table[:0x7F], lib_vals[:0x7F]) and np.isnan(table[0x7F]) and np.isnan(lib_vals[0x7F])
+    both = np.concatenate([lib_vals[:0x7F], -lib_vals[:0x7F]])
+    got, hit = R.e4m3_bytes(both)
+    assert hit.all() and np.array_equal(got, np.concatenate([np.arange(0x7F), 0x80 + np.arange(0x7F)]).astype(np.uint8))
+    _, hit = R.e4m3_bytes(np.array([17.0, 2.0 ** -10, 3.0 * 2.0 ** -10, 449.0, 0.3]))     # five significant bits, below the
+    assert not hit.any()                                                                  # finest step, above the range
+
+
+def test_reencoding_reconstructs_the_decoded_operand_and_knows_its_limits():
+    from oracle import reencode as R
+    rng = np.random.default_rng(8)
+    table = R.e4m3_value_table()
+    for cfg, m in ((orc.MX6, 4), (orc.MX4, 2)):
+        x = rng.standard_normal((128, 256)).astype(np.float32)
+        x[:, 64:80] = 0.0                                            # an all-zero block beside a normal one
+        out, scales, inexact = R.reencode_e4m3(cfg, x)
+        assert not inexact
+        y, _ = orc.quant_dequant(cfg, x)
+        sb = scales.reshape(2, 1, 32, 4, 4).transpose(1, 3, 2, 0, 4).reshape(128, 8).astype(np.int64)
+        val = np.where(out & 0x80, -1.0, 1.0) * table[out & 0x7F] * np.repeat(np.ldexp(1.0, sb - 127), 32, axis=1)
+        assert np.array_equal(val, y.astype(np.float64))
+        # scale byte = larger block exponent of the pair minus 7
+        F, _, _ = orc.encode(cfg, x)
+        assert np.array_equal(sb, F.astype(np.int64).reshape(128, 8, 2).max(axis=2) - 7)
+        # neighbouring blocks d binades apart, every magnitude in [1, 2) * 2^F (so tau = 0): exact up to d = 16 - (m - 1)
+        for d, want_inexact in ((16 - (m - 1), False), (17 - (m - 1), True)):
+            z = ((1.0 + rng.integers(0, 8, (128, 128)) / 8.0) * np.where(rng.random((128, 128)) < 0.5, -1, 1)).astype(np.float32)
+            z[:, 16:32] *= np.float32(2.0 ** -d)
+            assert R.reencode_e4m3(cfg, z)[2] == want_inexact, (m, d)
+    tiny = np.full((128, 128), 1.0, np.float32)
+    tiny[3, 0:16] = np.float32(1e-38)                                # block exponent below 16
+    assert R.reencode_e4m3(orc.MX6, tiny)[2]
