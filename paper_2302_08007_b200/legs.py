@@ -92,6 +92,15 @@ def linear_leg(args) -> dict:
     buf = linear.alloc(bdr.MX9, tokens, d_in, d_out)
     ms = _time(lambda: linear.step(bdr.MX9, x, w, dy, buf), reps=3)
     flops = 3 * 2.0 * tokens * d_in * d_out
-    return {"linear_layer": {"workload": "MX9 linear layer fwd+bwd: 6 quantize+pack (+QSNR), 3 mx_gemm", "ms": ms,
-                             "gemm_tflops_incl_quantization": flops / (ms * 1e-3) / 1e12,
-                             "qsnr_db": linear.qsnr_db(buf), "mx_gemm_status": bdr.mx_gemm_status()}}
+    out = {"linear_layer": {"workload": "MX9 linear layer fwd+bwd: 6 quantize+pack (+QSNR), 3 mx_gemm", "ms": ms,
+                            "gemm_tflops_incl_quantization": flops / (ms * 1e-3) / 1e12,
+                            "qsnr_db": linear.qsnr_db(buf), "mx_gemm_status": bdr.mx_gemm_status()}}
+    del buf
+    # the same step in MX6 (the paper's inference / fine-tuning format): the three products take the 8-bit path
+    buf6 = linear.alloc(bdr.MX6, tokens, d_in, d_out)
+    ms6 = _time(lambda: linear.step(bdr.MX6, x, w, dy, buf6), reps=3)
+    nb = bdr.mx_gemm_f8_workspace_bytes(d_out, d_in, tokens)   # the flag word of the step's last product (dW)
+    out["linear_layer"]["mx6"] = {"ms": ms6, "gemm_tflops_incl_quantization": flops / (ms6 * 1e-3) / 1e12,
+                                  "ran_on_8bit_path": int(buf6.workspace[nb - 256:nb - 252].view(torch.int32).item()) == 0,
+                                  "qsnr_db": linear.qsnr_db(buf6)}
+    return out

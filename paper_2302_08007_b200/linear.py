@@ -36,8 +36,9 @@ def alloc(cfg: bdr.Config, tokens: int, d_in: int, d_out: int, device="cuda", tw
     planes = {(n, ax): bdr.alloc_planes(cfg, *shapes[n], ax, device=device) for n, ax in ORDER}
     ws = None
     if two_phase and tokens % 256 == 0 and d_in % 256 == 0 and d_out % 256 == 0:
-        nbytes = max(bdr.mx_gemm_workspace_bytes(tokens, d_out, d_in), bdr.mx_gemm_workspace_bytes(tokens, d_in, d_out),
-                     bdr.mx_gemm_workspace_bytes(d_out, d_in, tokens))
+        # formats with at most four significant bits take the 8-bit block-scaled GEMM, the others the bf16 one
+        size = bdr.mx_gemm_f8_workspace_bytes if cfg.m <= 4 else bdr.mx_gemm_workspace_bytes
+        nbytes = max(size(tokens, d_out, d_in), size(tokens, d_in, d_out), size(d_out, d_in, tokens))
         ws = torch.empty(nbytes, dtype=torch.uint8, device=device)
     return LinearBuffers(planes, torch.zeros((6, 2), dtype=torch.float64, device=device),
                          torch.empty((tokens, d_out), dtype=torch.float32, device=device),
@@ -56,7 +57,9 @@ def step(cfg: bdr.Config, x: torch.Tensor, w: torch.Tensor, dy: torch.Tensor, bu
     p = buf.planes
 
     def gemm(a, b, M, N, K, c):
-        if buf.workspace is not None:
+        if buf.workspace is not None and cfg.m <= 4:
+            bdr.mx_gemm_f8(cfg, a, cfg, b, M, N, K, c, buf.workspace[:bdr.mx_gemm_f8_workspace_bytes(M, N, K)], stream=stream)
+        elif buf.workspace is not None:
             bdr.mx_gemm_ws(cfg, a, cfg, b, M, N, K, c, buf.workspace, stream=stream)
         else:
             bdr.mx_gemm(cfg, a, cfg, b, M, N, K, c, stream=stream)

@@ -29,7 +29,7 @@ def _run(cfg, x, w, dy, two_phase=True):
     return y.cpu().numpy(), dx.cpu().numpy(), dw.cpu().numpy(), linear.qsnr_db(buf), buf
 
 
-@pytest.mark.parametrize("two_phase", [True, False], ids=["mx_gemm_ws", "mx_gemm"])
+@pytest.mark.parametrize("two_phase", [True, False], ids=["with_workspace", "no_workspace"])
 @pytest.mark.parametrize("fmt", ["MX9", "MX6"])
 def test_linear_step_small_shapes_full_oracle(fmt, two_phase):
     cfg = {"MX9": bdr.MX9, "MX6": bdr.MX6}[fmt]
