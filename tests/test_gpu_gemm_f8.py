@@ -154,6 +154,23 @@ def test_f8_more_tiles_than_clusters():
     assert rel_frob(c, oracle_gemm(bdr.MX6, a, bdr.MX6, b)) <= 1e-5
 
 
+def test_f8_padded_output_pitch_keeps_the_padding():
+    # C is a view of a wider buffer: the split tiles are cleared and accumulated with the view's pitch, and the
+    # columns beside the view stay untouched
+    M, N, K = 512, 256, 512
+    a = synth.normal_matrix(M, K, seed=21, stream=1)
+    b = synth.normal_matrix(N, K, seed=21, stream=2, sigma=0.02)
+    pa, pb = _pack(bdr.MX6, a), _pack(bdr.MX6, b)
+    ws = torch.empty(bdr.mx_gemm_f8_workspace_bytes(M, N, K), dtype=torch.uint8, device="cuda")
+    wide = torch.full((M, N + 64), 7.0, dtype=torch.float32, device="cuda")
+    bdr.mx_gemm_f8(bdr.MX6, pa, bdr.MX6, pb, M, N, K, wide[:, :N], ws)
+    torch.cuda.synchronize()
+    assert bdr.mx_gemm_status() == 0
+    got = wide.cpu().numpy()
+    assert (got[:, N:] == 7.0).all()
+    assert rel_frob(got[:, :N], oracle_gemm(bdr.MX6, a, bdr.MX6, b)) <= 1e-5
+
+
 def test_f8_whole_rounds_only():
     # 64 tiles on 74 clusters: more than half of the clusters are busy in the only round, so no tile's K range is
     # split in two (the other tests have few tiles, or a sparse last round, and take the split path)
