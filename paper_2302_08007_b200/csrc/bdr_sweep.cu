@@ -191,27 +191,91 @@ __device__ __forceinline__ void pow2_slice_k2(const uint32_t (&u)[kSlice], const
 }
 
 // ---- FP32-scaled comparator kinds (one FP32 scale for the whole tensor) -----------------------------
-__device__ __forceinline__ void add_err(float deq_mag, uint32_t ubits, double& e2) {
-    const double d = (double)deq_mag - (double)__uint_as_float(ubits & 0x7FFFFFFFu);
-    e2 = fma(d, d, e2);
+// x / s for many x and one s.  With r = RN(1 / s): q0 = RN(x r), e = x - q0 s (exact in one fused multiply-add),
+// q = RN(q0 + e r) is the correctly rounded quotient (Markstein), as long as nothing leaves the normal range
+// and the significand of s is not all ones; outside these conditions the plain IEEE division is used.
+// Quotients below 2^-26 may come out inexact (their residual can be subnormal); every caller rounds them
+// to zero anyway.
+struct Divisor {
+    float s, r;
+    bool fast;
+};
+__device__ __forceinline__ Divisor make_divisor(float s) {
+    Divisor d;
+    d.s = s;
+    d.r = __frcp_rn(s);
+    const uint32_t b = __float_as_uint(s);
+    d.fast = (b & 0x7FFFFFu) != 0x7FFFFFu && b >= 0x0D800000u /*2^-100*/ && b <= 0x71800000u /*2^100*/;
+    return d;
+}
+template <bool FAST>
+__device__ __forceinline__ float divide(float x, const Divisor& d) {
+    if constexpr (FAST) {
+        const float q0 = __fmul_rn(x, d.r);
+        return __fmaf_rn(__fmaf_rn(-q0, d.s, x), d.r, q0);
+    } else {
+        return __fdiv_rn(x, d.s);
+    }
+}
+template <bool RNE>
+__device__ __forceinline__ float round_int(float t) {  // 0 <= t < 2^22
+    if constexpr (RNE) return __fsub_rn(__fadd_rn(t, 8388608.0f), 8388608.0f);
+    else return floorf(__fadd_rn(t, 0.5f));
 }
 
-// Eq. 1: s = max / (2^(b-1) - 1) with m = b-1;  Eq. 2: q = RoundToInt(x / s);  descale s * q.
+// |deq| - |x| is exact in fp32: either deq = 0, or the two are within a factor of two of each other (a value and
+// its rounding to a grid with at least one significant bit).  The square goes to the fp64 accumulator directly:
+// unlike on the power-of-two path the values are not normalised, so fp32 squares could overflow or vanish.
+__device__ __forceinline__ void add_err(float deq_mag, float ax, double& e2) {
+    const double d = (double)__fsub_rn(deq_mag, ax);
+    e2 = fma(d, d, e2);
+}
+__device__ __forceinline__ void all_zero_slice(const uint32_t (&u)[kSlice], double& e2) {  // scale 0: everything quantizes to 0
+#pragma unroll
+    for (int i = 0; i < kSlice; ++i) add_err(0.f, __uint_as_float(u[i] & 0x7FFFFFFFu), e2);
+}
+// The tie rule and the kind of division are the same for the whole slice: chosen once, outside the element loop.
+#define BDR_SLICE_DISPATCH(FN, ...)                                             \
+    do {                                                                        \
+        if (c.rounding == BDR_ROUND_NEAREST_EVEN) {                             \
+            if (dv.fast) FN<true, true>(__VA_ARGS__); else FN<true, false>(__VA_ARGS__);   \
+        } else {                                                                \
+            if (dv.fast) FN<false, true>(__VA_ARGS__); else FN<false, false>(__VA_ARGS__); \
+        }                                                                       \
+    } while (0)
+
+// Eq. 2: q = RoundToInt(x / s), clamped;  descale s * q.
+template <bool RNE, bool FAST>
+__device__ __forceinline__ void int_elements(const uint32_t (&u)[kSlice], const Divisor& dv, float qmax, double& e2) {
+#pragma unroll
+    for (int i = 0; i < kSlice; ++i) {
+        const float ax = __uint_as_float(u[i] & 0x7FFFFFFFu);
+        add_err(__fmul_rn(fminf(round_int<RNE>(divide<FAST>(ax, dv)), qmax), dv.s), ax, e2);
+    }
+}
+// Eq. 1: s = max / (2^(b-1) - 1) with m = b-1.
 __device__ __forceinline__ void int_slice(const uint32_t (&u)[kSlice], float amax, const SweepCfg& c, double& e2) {
     const float qmax = (float)((1 << c.m(0)) - 1);
     const float s = __fdiv_rn(amax, qmax);
-#pragma unroll
-    for (int i = 0; i < kSlice; ++i) {
-        float mag = 0.f;
-        if (s > 0.f) {
-            const float t = __fdiv_rn(__uint_as_float(u[i] & 0x7FFFFFFFu), s);
-            mag = __fmul_rn(fminf(round_to_int(t, c.rounding), qmax), s);
-        }
-        add_err(mag, u[i], e2);
-    }
+    if (!(s > 0.f)) return all_zero_slice(u, e2);
+    const Divisor dv = make_divisor(s);
+    BDR_SLICE_DISPATCH(int_elements, u, dv, qmax, e2);
 }
 
 // Scalar float with d2 exponent bits and m explicit mantissa bits under an FP32 tensor scale.
+template <bool RNE, bool FAST>
+__device__ __forceinline__ void fp_elements(const uint32_t (&u)[kSlice], const Divisor& dv, float fmax, int ef_min, int cm, double& e2) {
+#pragma unroll
+    for (int i = 0; i < kSlice; ++i) {
+        const float ax = __uint_as_float(u[i] & 0x7FFFFFFFu);
+        const float a = divide<FAST>(ax, dv);
+        const int ef = max((int)(__float_as_uint(a) >> 23), ef_min);
+        const float step = __uint_as_float((uint32_t)(ef - cm) << 23);
+        const float inv_step = __uint_as_float((uint32_t)(254 - (ef - cm)) << 23);
+        const float q = round_int<RNE>(__fmul_rn(a, inv_step));
+        add_err(__fmul_rn(fminf(__fmul_rn(q, step), fmax), dv.s), ax, e2);
+    }
+}
 __device__ __forceinline__ void fp_slice(const uint32_t (&u)[kSlice], float amax, const SweepCfg& c, double& e2) {
     const int cm = c.m(0);
     const int bias = (1 << (c.d2 - 1)) - 1;
@@ -219,20 +283,10 @@ __device__ __forceinline__ void fp_slice(const uint32_t (&u)[kSlice], float amax
                            ? 448.0f
                            : __uint_as_float(((uint32_t)((1 << c.d2) - 2 - bias + 127) << 23) | (0x7FFFFFu & ~(0x7FFFFFu >> cm)));
     const float s = __fdiv_rn(amax, fmax);
+    if (!(s > 0.f)) return all_zero_slice(u, e2);
+    const Divisor dv = make_divisor(s);
     const int ef_min = 1 - bias + 127;
-#pragma unroll
-    for (int i = 0; i < kSlice; ++i) {
-        float mag = 0.f;
-        if (s > 0.f) {
-            const float a = fabsf(__fdiv_rn(__uint_as_float(u[i]), s));
-            const int ef = max((int)(__float_as_uint(a) >> 23), ef_min);
-            const float step = __uint_as_float((uint32_t)(ef - cm) << 23);
-            const float inv_step = __uint_as_float((uint32_t)(254 - (ef - cm)) << 23);
-            const float q = round_to_int(__fmul_rn(a, inv_step), c.rounding);
-            mag = fabsf(__fmul_rn(fminf(__fmul_rn(q, step), fmax), s));
-        }
-        add_err(mag, u[i], e2);
-    }
+    BDR_SLICE_DISPATCH(fp_elements, u, dv, fmax, ef_min, cm, e2);
 }
 
 // VSQ: FP32 scale gamma for the tensor, unsigned d2-bit integer sub-scale per 16-element vector.
@@ -247,25 +301,44 @@ __device__ __forceinline__ void vsq_slice(const uint32_t (&u)[kSlice], float ama
     float uu = 0.f;
     if (gamma > 0.f) uu = fminf(round_to_int(__fdiv_rn(sv, gamma), c.rounding), umax);
     const float eff = __fmul_rn(uu, gamma);
-#pragma unroll
-    for (int i = 0; i < kSlice; ++i) {
-        float mag = 0.f;
-        if (eff > 0.f) {
-            const float t = __fdiv_rn(__uint_as_float(u[i] & 0x7FFFFFFFu), eff);
-            mag = __fmul_rn(fminf(round_to_int(t, c.rounding), qmax), eff);
-        }
-        add_err(mag, u[i], e2);
-    }
+    if (!(eff > 0.f)) return all_zero_slice(u, e2);
+    const Divisor dv = make_divisor(eff);
+    BDR_SLICE_DISPATCH(int_elements, u, dv, qmax, e2);
 }
 
 // ---- kernels ----------------------------------------------------------------------------------------------
+// Largest magnitude of the tensor (as fp32 bits).  A contiguous, 16-byte aligned tensor is read with 16-byte
+// loads, four in flight per thread; anything else element by element.
 template <typename T>
 __global__ void amax_kernel(const T* x, int64_t rows, int64_t cols, int64_t ld, uint32_t* amax_bits) {
     uint32_t m = 0;
     const int64_t total = rows * cols;
-    for (int64_t g = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; g < total; g += (int64_t)gridDim.x * blockDim.x) {
-        const int64_t r = g / cols;
-        m = max(m, Elem<T>::load_bits(x + r * ld + (g - r * cols)) & 0x7FFFFFFFu);
+    constexpr int kPer = 16 / (int)sizeof(T);
+    const int64_t tid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x, nthr = (int64_t)gridDim.x * blockDim.x;
+    if ((ld == cols || rows == 1) && (reinterpret_cast<uintptr_t>(x) % 16) == 0) {
+        const uint4* v = reinterpret_cast<const uint4*>(x);
+        const int64_t nv = total / kPer;
+        auto take = [&](const uint4& q) {
+            if constexpr (sizeof(T) == 4) {
+                m = max(max(m, q.x & 0x7FFFFFFFu), max(q.y & 0x7FFFFFFFu, max(q.z & 0x7FFFFFFFu, q.w & 0x7FFFFFFFu)));
+            } else {  // two bf16 per word: the high half is already in place, the low half moves up
+                const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+                for (int k = 0; k < 4; ++k) m = max(m, max(w[k] & 0x7FFF0000u, (w[k] << 16) & 0x7FFF0000u));
+            }
+        };
+        int64_t g = tid;
+        for (; g + 3 * nthr < nv; g += 4 * nthr) {
+            const uint4 a = __ldg(v + g), b = __ldg(v + g + nthr), c = __ldg(v + g + 2 * nthr), d = __ldg(v + g + 3 * nthr);
+            take(a); take(b); take(c); take(d);
+        }
+        for (; g < nv; g += nthr) take(__ldg(v + g));
+        for (int64_t e = nv * kPer + tid; e < total; e += nthr) m = max(m, Elem<T>::load_bits(x + e) & 0x7FFFFFFFu);
+    } else {
+        for (int64_t g = tid; g < total; g += nthr) {
+            const int64_t r = g / cols;
+            m = max(m, Elem<T>::load_bits(x + r * ld + (g - r * cols)) & 0x7FFFFFFFu);
+        }
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) m = max(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
