@@ -36,15 +36,15 @@ FALLBACK_HBM_GBS = 6650.0
 # profiles/step_kernels_dram_traffic.md.  Writes that still sit in L2 when a kernel ends are not
 # counted by those counters, which is why some figures are below the algorithmic bytes.
 NCU_TRAFFIC_BYTES: dict[str, float | None] = {
-    "quant_dequant_MX4_row": 217483776, "quant_dequant_MX4_col": 216174336,
-    "quant_dequant_MX6_row": 216457216, "quant_dequant_MX6_col": 215976192,
-    "quant_dequant_MX9_row": 216821760, "quant_dequant_MX9_col": 216307200,
-    "pack_MX4_row": 148817664, "pack_MX4_col": 147564288,
-    "pack_MX6_row": 157307904, "pack_MX6_col": 155158784,
-    "pack_MX9_row": 173331712, "pack_MX9_col": 168369664,
-    "unpack_MX4_row": 112468736, "unpack_MX4_col": 109030656,
-    "unpack_MX6_row": 128452352, "unpack_MX6_col": 128861440,
-    "unpack_MX9_row": 154516736, "unpack_MX9_col": 153580800,
+    "quant_dequant_MX4_row": 217033472, "quant_dequant_MX4_col": 217938688,
+    "quant_dequant_MX6_row": 216496640, "quant_dequant_MX6_col": 216127232,
+    "quant_dequant_MX9_row": 216842752, "quant_dequant_MX9_col": 217294848,
+    "pack_MX4_row": 149412096, "pack_MX4_col": 146696448,
+    "pack_MX6_row": 157221888, "pack_MX6_col": 154196480,
+    "pack_MX9_row": 173520128, "pack_MX9_col": 168751104,
+    "unpack_MX4_row": 111391232, "unpack_MX4_col": 108662528,
+    "unpack_MX6_row": 128986112, "unpack_MX6_col": 126326016,
+    "unpack_MX9_row": 154794496, "unpack_MX9_col": 151429632,
 }
 
 
