@@ -78,8 +78,31 @@ unpack_col_x2_kernel(bdr_planes_t in, bf16* y, int64_t ld, int n_col_tiles, int 
                 s[c][0] = a0.x; s[c][1] = a0.y; s[c][2] = a0.z; s[c][3] = a0.w;
                 s[c][4] = a1.x; s[c][5] = a1.y; s[c][6] = a1.z; s[c][7] = a1.w;
             } else {
+                // W words at word offset W * warp of the column's row.  The row pitch is a multiple of 16 bytes, so
+                // 32-bit loads at the same offset would put the 32 lanes (32 rows) on only eight banks; instead
+                // the two aligned 16-byte chunks that contain the words are loaded (conflict-free) and the W
+                // words are picked out: they start at word (W * warp) mod 4 of the eight, the same for the warp.
+                const uint32_t first = b + ST::row_of(col) * ST::kPitch + (((W * warp) >> 2) << 4);
+                const uint4 a0 = async::lds128(first), a1 = async::lds128(first + 16);
+                const uint32_t L[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
+                switch ((W * warp) & 3) {
+                    case 0:
 #pragma unroll
-                for (int k = 0; k < W; ++k) s[c][k] = async::lds32(src + 4 * k);
+                        for (int k = 0; k < W; ++k) s[c][k] = L[k];
+                        break;
+                    case 1:
+#pragma unroll
+                        for (int k = 0; k < W; ++k) s[c][k] = L[(1 + k) & 7];
+                        break;
+                    case 2:
+#pragma unroll
+                        for (int k = 0; k < W; ++k) s[c][k] = L[(2 + k) & 7];
+                        break;
+                    default:
+#pragma unroll
+                        for (int k = 0; k < W; ++k) s[c][k] = L[(3 + k) & 7];
+                        break;
+                }
             }
             Fp[c] = async::lds16(b + ST::kElemBytes + ST::row_of(col) * 16 + 2 * warp);
             mp[c] = async::lds16(b + ST::kElemBytes + ST::kExpBytes + ST::row_of(col) * 16 + 2 * warp);
