@@ -213,6 +213,9 @@ template <int WA, int WB>
 __global__ void __launch_bounds__(kF8Threads)
 reencode_e4m3_kernel(bdr_planes_t a, bdr_planes_t b, int a_strips, int b_strips, int64_t M, int64_t N, int64_t K, uint8_t* out_a,
                      uint8_t* out_b, uint8_t* sf_a, uint8_t* sf_b, int* inexact, ZeroTiles z) {
+    // a kernel launched behind this one as a programmatic dependent may begin its own set-up now (it still
+    // waits for this grid to finish before it reads what is written here); without such a launch: no effect
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int warp = threadIdx.x >> 5;
     if ((int)blockIdx.x >= a_strips + b_strips) {
         // extra CTAs: clear the 256 x 256 tiles of C that the GEMM kernel accumulates into

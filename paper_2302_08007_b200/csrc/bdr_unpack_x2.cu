@@ -31,6 +31,9 @@ __global__ void __launch_bounds__(kUThreads)
 unpack_row_x2_kernel(bdr_planes_t in, bf16* y, URunIndex ri, uint32_t total, int* status) {
     using US = UStage<W>;
     constexpr int S = kUStages;
+    // a kernel launched behind this one as a programmatic dependent (the second phase of mx_gemm_ws) may begin its
+    // set-up now; it still waits for this grid to finish before it reads y.  Without such a launch: no effect
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     extern __shared__ __align__(128) uint8_t smem[];  // ring [warp][stage][codes | exponents | microexponents], barriers
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const uint32_t ring0 = async::smem_u32(smem) + warp * S * US::kBytes;

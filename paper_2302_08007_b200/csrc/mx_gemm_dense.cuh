@@ -69,6 +69,10 @@ bf16_gemm_pair_kernel(const __grid_constant__ DenseMaps maps, int tiles_m, int t
     tc_fence_after();
     const uint32_t tmem_base = bars.tmem_base;
 
+    // Nothing above touched global memory: under a programmatic dependent launch it overlaps the tail of the
+    // unpack kernel that writes operand B.  From here on the operands are needed.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+
     if (warp == 0) {
         // ---------------- TMA producer ----------------
         if (lane == 0) {
@@ -201,8 +205,20 @@ static int launch_gemm_dense(const void* a_bf16, const void* b_bf16, int64_t M, 
     const int tiles_m = (int)(M / 256), tiles_n = (int)(N / 256);
     const int64_t n_tiles = (int64_t)tiles_m * tiles_n;
     const int n_clusters = (int)std::min<int64_t>(n_tiles, sm_count() / 2);
-    bf16_gemm_pair_kernel<<<2 * n_clusters, kDThreads, kDSmemBytes, st>>>(maps, tiles_m, tiles_n, (int)(K / kBK), c, ldc);
-    return cudaGetLastError() == cudaSuccess ? BDR_OK : BDR_ERR_CUDA;
+    // programmatic dependent launch: set-up may overlap the tail of the kernel before it in the stream; the kernel
+    // waits (griddepcontrol.wait) before it reads anything
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(2 * n_clusters));
+    cfg.blockDim = dim3(kDThreads);
+    cfg.dynamicSmemBytes = kDSmemBytes;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    const cudaError_t e = cudaLaunchKernelEx(&cfg, bf16_gemm_pair_kernel, maps, tiles_m, tiles_n, (int)(K / kBK), c, ldc);
+    return e == cudaSuccess && cudaGetLastError() == cudaSuccess ? BDR_OK : BDR_ERR_CUDA;
 }
 
 }  // namespace bdr

@@ -20,7 +20,7 @@
 //   * when the last round of tiles would keep at most half of the clusters busy, each of its tiles is
 //     computed as two halves of the K range by two clusters that add (red.global.add) into a tile the
 //     re-encoding launch has cleared.
-// The kernel returns at once when *gate is non-zero (the operands were not representable).
+// The kernel does nothing when *gate is non-zero (the operands were not representable).
 // Every wait is bounded.  (textually included by mx_gemm.cu after mx_gemm_dense.cuh)
 #pragma once
 
@@ -96,7 +96,6 @@ __device__ __forceinline__ void bulk_load_g2s(void* smem_dst, const void* gsrc, 
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kFThreads, 1)
 mxf8_gemm_pair_kernel(const __grid_constant__ F8Maps maps, const uint8_t* sf_a, const uint8_t* sf_b, int tiles_m, int tiles_n, int nk,
                       int tiles_full, int n_items, float* c, int64_t ldc, const int* gate) {
-    if (gate && *gate != 0) return;  // the same for every thread of the grid
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     uint8_t* stages = reinterpret_cast<uint8_t*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     F8Bars& bars = *reinterpret_cast<F8Bars*>(stages + kFStages * kFStageBytes);
@@ -131,7 +130,14 @@ mxf8_gemm_pair_kernel(const __grid_constant__ F8Maps maps, const uint8_t* sf_a, 
     tc_fence_after();
     const uint32_t tmem_base = bars.tmem_base;
 
-    if (warp == 0) {
+    // Everything above touched no global memory: under a programmatic dependent launch it overlaps the tail of the
+    // re-encoding kernel.  From here on the operands, the cleared tiles of C and the gate are needed.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    const bool open = !(gate && *gate != 0);  // the same for every thread of the grid
+
+    if (!open) {
+        // the operands were not representable: nothing to do but to give the tensor memory back
+    } else if (warp == 0) {
         // ---------------- producer: operand tiles by TMA, scale atoms by bulk copy ----------------
         if (lane == 0) {
             uint64_t* const my_full = rank == 0 ? bars.full : bars.full_local;
@@ -333,9 +339,21 @@ static int launch_gemm_f8(const uint8_t* a_e4m3, const uint8_t* b_e4m3, const ui
     }
     F8Maps maps;
     if (!make_f8_map(&maps.a, a_e4m3, M, K) || !make_f8_map(&maps.b, b_e4m3, N, K)) return BDR_ERR_CUDA;
-    mxf8_gemm_pair_kernel<<<2 * plan.n_clusters, kFThreads, kFSmemBytes, st>>>(maps, sf_a, sf_b, plan.tiles_m, plan.tiles_n, (int)(K / kFBK),
-                                                                              plan.tiles_full, plan.n_items, c, ldc, gate);
-    return cudaGetLastError() == cudaSuccess ? BDR_OK : BDR_ERR_CUDA;
+    // programmatic dependent launch: the kernel may start while the re-encoding kernel before it in the stream is
+    // draining; it waits (griddepcontrol.wait) before it reads anything that kernel wrote
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(2 * plan.n_clusters));
+    cfg.blockDim = dim3(kFThreads);
+    cfg.dynamicSmemBytes = kFSmemBytes;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    const cudaError_t e = cudaLaunchKernelEx(&cfg, mxf8_gemm_pair_kernel, maps, sf_a, sf_b, plan.tiles_m, plan.tiles_n, (int)(K / kFBK),
+                                             plan.tiles_full, plan.n_items, c, ldc, gate);
+    return e == cudaSuccess && cudaGetLastError() == cudaSuccess ? BDR_OK : BDR_ERR_CUDA;
 }
 
 }  // namespace bdr
