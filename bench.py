@@ -36,15 +36,15 @@ FALLBACK_HBM_GBS = 6650.0
 # profiles/step_kernels_dram_traffic.md.  Writes that still sit in L2 when a kernel ends are not
 # counted by those counters, which is why some figures are below the algorithmic bytes.
 NCU_TRAFFIC_BYTES: dict[str, float | None] = {
-    "quant_dequant_MX4_row": 217033472, "quant_dequant_MX4_col": 217938688,
-    "quant_dequant_MX6_row": 216496640, "quant_dequant_MX6_col": 216127232,
-    "quant_dequant_MX9_row": 216842752, "quant_dequant_MX9_col": 217294848,
-    "pack_MX4_row": 149412096, "pack_MX4_col": 146696448,
-    "pack_MX6_row": 157221888, "pack_MX6_col": 154196480,
-    "pack_MX9_row": 173520128, "pack_MX9_col": 168751104,
-    "unpack_MX4_row": 111391232, "unpack_MX4_col": 108662528,
-    "unpack_MX6_row": 128986112, "unpack_MX6_col": 126326016,
-    "unpack_MX9_row": 154794496, "unpack_MX9_col": 151429632,
+    "quant_dequant_MX4_row": 216804096, "quant_dequant_MX4_col": 216572928,
+    "quant_dequant_MX6_row": 216876800, "quant_dequant_MX6_col": 216743168,
+    "quant_dequant_MX9_row": 216424704, "quant_dequant_MX9_col": 216255232,
+    "pack_MX4_row": 149431296, "pack_MX4_col": 146424832,
+    "pack_MX6_row": 157652224, "pack_MX6_col": 154688512,
+    "pack_MX9_row": 173349120, "pack_MX9_col": 168726784,
+    "unpack_MX4_row": 113256704, "unpack_MX4_col": 108517888,
+    "unpack_MX6_row": 128259584, "unpack_MX6_col": 126010880,
+    "unpack_MX9_row": 154560000, "unpack_MX9_col": 151881984,
 }
 
 
