@@ -30,6 +30,7 @@ ROWS, COLS = 8192, 8192
 FORMATS = (("MX4", 2), ("MX6", 4), ("MX9", 7))  # name, m  (k1=16, d1=8, k2=2, d2=1: Table II)
 METRIC = "MX quant-dequant GB/s"
 FALLBACK_HBM_GBS = 6650.0
+FALLBACK_BF16_TFLOPS = 1590.0
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of each of the step's kernels on the
 # bench workload itself (8192 x 8192 bf16), from the committed ncu capture
@@ -405,6 +406,18 @@ def secondary_legs(args, bdr, synth, torch) -> dict:
             out.update(fn(args))
         except bdr.BdrError as e:
             out[fn.__name__] = {"unavailable": str(e)}
+    # tensor roofline of the GEMM line: the measured cuBLAS bf16 burst figure (the call is timed alone); an 8-bit
+    # contraction takes that figure times the nominal 8-bit : bf16 ratio of 2
+    g = out.get("mx_gemm")
+    if isinstance(g, dict) and "value" in g:
+        _, src, peaks = measured_peaks()
+        bf16_peak = float(peaks.get("bf16_tflops", FALLBACK_BF16_TFLOPS))
+        f8 = g["entry_point"].startswith("mx_gemm_f8")
+        peak = bf16_peak * (2.0 if f8 else 1.0)
+        g["roofline"] = {"bound": "tensor", "dtype": "e4m3 x e4m3, e8m0 block scales, fp32 accumulate" if f8 else "bf16, fp32 accumulate",
+                         "achieved": g["value"], "peak": peak, "unit": "TFLOP/s", "frac": g["value"] / peak,
+                         "peak_source": ("measured bf16" if "bf16_tflops" in peaks else "fallback bf16") + (" x 2 (nominal 8-bit ratio)" if f8 else ""),
+                         "frac_of_bf16_peak": g["value"] / bf16_peak}
     return out
 
 
