@@ -212,6 +212,13 @@ int mx_gemm_f8(const bdr_config_t* cfg_a /*host*/, const bdr_planes_t* a /*host 
 int bdr_reencode_e4m3(const bdr_config_t* cfg /*host*/, const bdr_planes_t* in /*host struct*/, int64_t rows, int64_t K,
                       uint8_t* out, uint8_t* scales, int* inexact_dev, void* stream);
 
+/* Phase 2 of mx_gemm_f8 on its own, for operands that were re-encoded earlier (weights that do not change
+ * between calls, say): C = A B^T from E4M3 bytes a [M, K], b [N, K] (row-major, contiguous) and their scale
+ * atoms as bdr_reencode_e4m3 writes them.  The caller has checked that no re-encoding raised `inexact`.
+ * M, N, K multiples of 256; 16-byte aligned pointers; device memory; fp32 accumulate and output. */
+int mx_gemm_e4m3(const uint8_t* a, const uint8_t* scales_a, const uint8_t* b, const uint8_t* scales_b, int64_t M,
+                 int64_t N, int64_t K, float* c, int64_t ldc, void* stream);
+
 /* BDR_OK, or BDR_ERR_TIMEOUT if any mx_gemm launch on the current device gave up a bounded wait
  * (sticky).  Host call; synchronises with the device (it copies one word back). */
 int mx_gemm_status(void);

@@ -21,7 +21,7 @@ F32, BF16 = 0, 1
 
 EXPORTS = ("bdr_strerror", "bdr_device_status", "bdr_packed_sizes", "bdr_quant_dequant", "bdr_pack", "bdr_unpack",
            "bdr_qsnr_workspace_bytes", "bdr_qsnr", "bdr_qsnr_static_max_cfgs", "bdr_qsnr_static", "mx_gemm",
-           "mx_gemm_workspace_bytes", "mx_gemm_ws", "mx_gemm_f8_workspace_bytes", "mx_gemm_f8", "bdr_reencode_e4m3",
+           "mx_gemm_workspace_bytes", "mx_gemm_ws", "mx_gemm_f8_workspace_bytes", "mx_gemm_f8", "bdr_reencode_e4m3", "mx_gemm_e4m3",
            "mx_gemm_status")
 
 
@@ -115,6 +115,9 @@ def lib():
         L.mx_gemm_f8.argtypes = L.mx_gemm_ws.argtypes
         L.bdr_reencode_e4m3.restype = C.c_int
         L.bdr_reencode_e4m3.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+        L.mx_gemm_e4m3.restype = C.c_int
+        L.mx_gemm_e4m3.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_int64, C.c_int64, C.c_void_p,
+                                   C.c_int64, C.c_void_p]
         L.mx_gemm_status.restype = C.c_int
         L.mx_gemm_status.argtypes = []
         L.bdr_device_status.restype = C.c_int
@@ -285,6 +288,14 @@ def bdr_reencode_e4m3(cfg: Config, planes: Planes, rows: int, K: int, out: torch
     _check(lib().bdr_reencode_e4m3(C.addressof(cc), C.addressof(pp), rows, K, _ptr(out), _ptr(scales), _ptr(inexact),
                                    _stream(stream)), "bdr_reencode_e4m3")
     return out, scales
+
+
+def mx_gemm_e4m3(a: torch.Tensor, scales_a: torch.Tensor, b: torch.Tensor, scales_b: torch.Tensor, M: int, N: int, K: int,
+                 c: torch.Tensor, stream=None):
+    """C = A B^T from operands re-encoded earlier with bdr_reencode_e4m3 (E4M3 bytes [rows, K] and scale atoms)."""
+    _check(lib().mx_gemm_e4m3(_ptr(a), _ptr(scales_a), _ptr(b), _ptr(scales_b), M, N, K, _ptr(c), c.stride(0), _stream(stream)),
+           "mx_gemm_e4m3")
+    return c
 
 
 def bdr_device_status() -> int:

@@ -493,6 +493,24 @@ int mx_gemm_f8(const bdr_config_t* cfg_a, const bdr_planes_t* a, const bdr_confi
     return mx_gemm_gated(cfg_a, a, cfg_b, b, M, N, K, c, ldc, flag, stream);                           // else the bf16 kernel
 }
 
+int mx_gemm_e4m3(const uint8_t* a, const uint8_t* scales_a, const uint8_t* b, const uint8_t* scales_b, int64_t M, int64_t N, int64_t K,
+                 float* c, int64_t ldc, void* stream) {
+    if (!a || !scales_a || !b || !scales_b || !c) return BDR_ERR_NULL;
+    if (M < 0 || N < 0 || K < 0 || ldc < N) return BDR_ERR_SIZE;
+    if (M == 0 || N == 0) return BDR_OK;
+    if (M % 256 || N % 256 || K % 256 || K == 0) return BDR_ERR_UNSUPPORTED;
+    if (M >= (1ll << 31) || N >= (1ll << 31) || K >= (1ll << 31) || (M / 256) * (N / 256) >= (1ll << 30)) return BDR_ERR_UNSUPPORTED;
+    if (((uintptr_t)a | (uintptr_t)b | (uintptr_t)scales_a | (uintptr_t)scales_b | (uintptr_t)c) % 16 || ldc % 4) return BDR_ERR_MISALIGNED;
+    cudaStream_t st = (cudaStream_t)stream;
+    const F8Plan plan = plan_gemm_f8(M, N, K);
+    if (plan.split_tiles() > 0) {
+        const ZeroTiles z = {c, ldc, plan.tiles_n, plan.tiles_full, plan.split_tiles()};
+        zero_tiles_kernel<<<dim3((unsigned)z.count, 4), 256, 0, st>>>(z);
+        if (cudaGetLastError() != cudaSuccess) return BDR_ERR_CUDA;
+    }
+    return launch_gemm_f8(a, b, scales_a, scales_b, M, N, K, plan, c, ldc, nullptr, st);
+}
+
 int bdr_reencode_e4m3(const bdr_config_t* cfg, const bdr_planes_t* in, int64_t rows, int64_t K, uint8_t* out, uint8_t* scales,
                       int* inexact_dev, void* stream) {
     if (!cfg || !in || !out || !scales || !inexact_dev) return BDR_ERR_NULL;

@@ -296,6 +296,17 @@ mxf8_gemm_pair_kernel(const __grid_constant__ F8Maps maps, const uint8_t* sf_a, 
     if (threadIdx.x == 0 && bars.failed) atomicExch(&g_gemm_status, (int)BDR_ERR_TIMEOUT);
 }
 
+// Clears `z.count` tiles of 256 x 256 floats (for callers of the GEMM kernel that do not come through the re-encoding
+// launch, which clears them on the side); grid (z.count, 4), 256 threads.
+__global__ void zero_tiles_kernel(ZeroTiles z) {
+    const int t = z.tile0 + (int)blockIdx.x;
+    const int tm = t / z.tiles_n, tn = t - tm * z.tiles_n;
+    for (int idx = (int)blockIdx.y * 64 * 64 + (int)threadIdx.x; idx < ((int)blockIdx.y + 1) * 64 * 64; idx += 256) {
+        const int r = idx >> 6, ch = idx & 63;  // 64 rows per block, 64 chunks of 16 bytes per row
+        *reinterpret_cast<uint4*>(z.c + ((int64_t)tm * 256 + r) * z.ldc + (int64_t)tn * 256 + ch * 4) = make_uint4(0, 0, 0, 0);
+    }
+}
+
 static bool make_f8_map(CUtensorMap* out, const void* base, int64_t rows, int64_t K) {
     EncodeTiledFn fn = encode_tiled_fn();
     if (!fn) return false;

@@ -171,6 +171,28 @@ def test_f8_padded_output_pitch_keeps_the_padding():
     assert rel_frob(got[:, :N], oracle_gemm(bdr.MX6, a, bdr.MX6, b)) <= 1e-5
 
 
+def test_gemm_from_operands_re_encoded_earlier():
+    # weights re-encoded once, activations per call: the GEMM kernel on its own
+    M, N, K = 512, 1024, 768
+    a = synth.outlier_channel_matrix(M, K, seed=31, stream=1, gain=20.0)
+    b = synth.normal_matrix(N, K, seed=31, stream=2, sigma=0.02)
+    enc = []
+    for cfg, x in ((bdr.MX6, a), (bdr.MX4, b)):
+        rows = x.shape[0]
+        out = torch.empty((rows, K), dtype=torch.uint8, device="cuda")
+        sf = torch.empty(rows * K // 32, dtype=torch.uint8, device="cuda")
+        flag = torch.zeros(1, dtype=torch.int32, device="cuda")
+        bdr.bdr_reencode_e4m3(cfg, _pack(cfg, x), rows, K, out, sf, flag)
+        assert int(flag.item()) == 0
+        enc += [out, sf]
+    for _ in range(2):                                       # the second call finds C full of the first call's result
+        c = torch.full((M, N), 3.0, dtype=torch.float32, device="cuda")
+        bdr.mx_gemm_e4m3(enc[0], enc[1], enc[2], enc[3], M, N, K, c)
+        torch.cuda.synchronize()
+        assert bdr.mx_gemm_status() == 0
+        assert rel_frob(c.cpu().numpy(), oracle_gemm(bdr.MX6, a, bdr.MX4, b)) <= 1e-5
+
+
 def test_f8_whole_rounds_only():
     # 64 tiles on 74 clusters: more than half of the clusters are busy in the only round, so no tile's K range is
     # split in two (the other tests have few tiles, or a sparse last round, and take the split path)
