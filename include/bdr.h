@@ -168,6 +168,15 @@ int mx_gemm(const bdr_config_t* cfg_a /*host*/, const bdr_planes_t* a /*host str
             const bdr_config_t* cfg_b /*host*/, const bdr_planes_t* b /*host struct*/, int64_t M, int64_t N,
             int64_t K, float* c, int64_t ldc, void* stream);
 
+/* Lends the library scratch memory on the current device (or takes it back: workspace = NULL).  While it is
+ * lent, mx_gemm uses it to compute the same product through the faster two-phase kernels (mx_gemm_f8 when
+ * both formats have m <= 4, else mx_gemm_ws) whenever M, N and K are multiples of 256 and the memory is large
+ * enough (mx_gemm_f8_workspace_bytes / mx_gemm_workspace_bytes); otherwise mx_gemm works without scratch as
+ * before.  The memory stays the caller's: 256-byte aligned device memory that must outlive every mx_gemm call
+ * issued while it is lent; its contents are overwritten by those calls, which therefore have to be ordered
+ * with respect to each other (one stream, or events).  Host call, no device work. */
+int bdr_set_workspace(void* workspace, int64_t workspace_bytes);
+
 /* mx_gemm in two phases, for callers that can lend scratch memory: both operands are first decoded to
  * bf16 in `workspace` (once each, by the unpack kernels), then multiplied by a tensor-core kernel that
  * streams the bf16 operands with TMA.  mx_gemm decodes inside the GEMM and so repeats the decode of an

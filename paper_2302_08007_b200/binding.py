@@ -21,7 +21,7 @@ F32, BF16 = 0, 1
 
 EXPORTS = ("bdr_strerror", "bdr_device_status", "bdr_packed_sizes", "bdr_quant_dequant", "bdr_pack", "bdr_unpack",
            "bdr_qsnr_workspace_bytes", "bdr_qsnr", "bdr_qsnr_static_max_cfgs", "bdr_qsnr_static", "mx_gemm",
-           "mx_gemm_workspace_bytes", "mx_gemm_ws", "mx_gemm_f8_workspace_bytes", "mx_gemm_f8", "bdr_reencode_e4m3", "mx_gemm_e4m3",
+           "mx_gemm_workspace_bytes", "mx_gemm_ws", "mx_gemm_f8_workspace_bytes", "mx_gemm_f8", "bdr_reencode_e4m3", "mx_gemm_e4m3", "bdr_set_workspace",
            "mx_gemm_status")
 
 
@@ -115,6 +115,8 @@ def lib():
         L.mx_gemm_f8.argtypes = L.mx_gemm_ws.argtypes
         L.bdr_reencode_e4m3.restype = C.c_int
         L.bdr_reencode_e4m3.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+        L.bdr_set_workspace.restype = C.c_int
+        L.bdr_set_workspace.argtypes = [C.c_void_p, C.c_int64]
         L.mx_gemm_e4m3.restype = C.c_int
         L.mx_gemm_e4m3.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_int64, C.c_int64, C.c_void_p,
                                    C.c_int64, C.c_void_p]
@@ -288,6 +290,14 @@ def bdr_reencode_e4m3(cfg: Config, planes: Planes, rows: int, K: int, out: torch
     _check(lib().bdr_reencode_e4m3(C.addressof(cc), C.addressof(pp), rows, K, _ptr(out), _ptr(scales), _ptr(inexact),
                                    _stream(stream)), "bdr_reencode_e4m3")
     return out, scales
+
+
+def bdr_set_workspace(workspace: torch.Tensor | None):
+    """Lends mx_gemm scratch memory on the current device (None takes it back).  The tensor must stay alive while lent."""
+    if workspace is None:
+        _check(lib().bdr_set_workspace(None, 0), "bdr_set_workspace")
+    else:
+        _check(lib().bdr_set_workspace(_ptr(workspace), workspace.numel() * workspace.element_size()), "bdr_set_workspace")
 
 
 def mx_gemm_e4m3(a: torch.Tensor, scales_a: torch.Tensor, b: torch.Tensor, scales_b: torch.Tensor, M: int, N: int, K: int,

@@ -442,8 +442,40 @@ static int mx_gemm_gated(const bdr_config_t* cfg_a, const bdr_planes_t* a, const
 
 extern "C" {
 
+// Scratch memory lent to mx_gemm by the caller (bdr_set_workspace), per device.
+struct LentWorkspace { void* ptr; int64_t bytes; };
+static LentWorkspace g_lent[64] = {};
+
+int bdr_set_workspace(void* workspace, int64_t workspace_bytes) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return BDR_ERR_CUDA;
+    if (workspace && ((uintptr_t)workspace % 256 || workspace_bytes < 0)) return BDR_ERR_MISALIGNED;
+    g_lent[dev].ptr = workspace;
+    g_lent[dev].bytes = workspace ? workspace_bytes : 0;
+    return BDR_OK;
+}
+
+int mx_gemm_ws(const bdr_config_t*, const bdr_planes_t*, const bdr_config_t*, const bdr_planes_t*, int64_t, int64_t, int64_t, float*,
+               int64_t, void*, int64_t, void*);
+int mx_gemm_f8(const bdr_config_t*, const bdr_planes_t*, const bdr_config_t*, const bdr_planes_t*, int64_t, int64_t, int64_t, float*,
+               int64_t, void*, int64_t, void*);
+int64_t mx_gemm_workspace_bytes(int64_t, int64_t, int64_t);
+int64_t mx_gemm_f8_workspace_bytes(int64_t, int64_t, int64_t);
+
 int mx_gemm(const bdr_config_t* cfg_a, const bdr_planes_t* a, const bdr_config_t* cfg_b, const bdr_planes_t* b, int64_t M,
             int64_t N, int64_t K, float* c, int64_t ldc, void* stream) {
+    // with scratch memory lent by the caller the two-phase kernels are the faster way to the same product
+    int dev = 0;
+    if (cfg_a && cfg_b && M > 0 && N > 0 && M % 256 == 0 && N % 256 == 0 && K % 256 == 0 && cudaGetDevice(&dev) == cudaSuccess && dev >= 0 &&
+        dev < 64 && g_lent[dev].ptr) {
+        const LentWorkspace w = g_lent[dev];
+        int rc = BDR_ERR_UNSUPPORTED;
+        if (cfg_a->m <= 4 && cfg_b->m <= 4 && w.bytes >= mx_gemm_f8_workspace_bytes(M, N, K))
+            rc = mx_gemm_f8(cfg_a, a, cfg_b, b, M, N, K, c, ldc, w.ptr, w.bytes, stream);
+        else if (w.bytes >= mx_gemm_workspace_bytes(M, N, K))
+            rc = mx_gemm_ws(cfg_a, a, cfg_b, b, M, N, K, c, ldc, w.ptr, w.bytes, stream);
+        if (rc != BDR_ERR_UNSUPPORTED && rc != BDR_ERR_WORKSPACE) return rc;
+    }
     return mx_gemm_gated(cfg_a, a, cfg_b, b, M, N, K, c, ldc, nullptr, stream);
 }
 

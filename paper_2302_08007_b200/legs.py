@@ -75,6 +75,12 @@ def gemm_leg(args) -> dict:
         bdr.bdr_reencode_e4m3(bdr.MX6, planes, rows, K, e8, sf, flag)
         enc += [e8, sf]
     ms_pre = _time(lambda: bdr.mx_gemm_e4m3(enc[0], enc[1], enc[2], enc[3], M, N, K, c), reps=20, warmup=3)
+    # the plain mx_gemm call while scratch memory is lent to the library (it then takes the 8-bit path itself)
+    bdr.bdr_set_workspace(ws8)
+    try:
+        ms_lent = _time(lambda: bdr.mx_gemm(bdr.MX6, pa, bdr.MX6, pb, M, N, K, c), reps=20, warmup=3)
+    finally:
+        bdr.bdr_set_workspace(None)
     tf = lambda t: 2.0 * M * N * K / (t * 1e-3) / 1e12
     ws_name = ("mx_gemm_ws (both operands decoded once to a bf16 workspace, then a TMA-fed tcgen05 GEMM; the time "
                "covers both phases)")
@@ -86,7 +92,9 @@ def gemm_leg(args) -> dict:
                         "entry_point": f8_name if best_f8 else ws_name,
                         "mx_gemm_ws": {"value": tf(ms), "unit": "TFLOP/s", "ms": ms},
                         "mx_gemm_f8": {"value": tf(ms_f8), "unit": "TFLOP/s", "ms": ms_f8, "ran_on_8bit_path": f8_exact},
-                        "fused_mx_gemm": {"value": tf(ms_fused), "unit": "TFLOP/s", "ms": ms_fused},
+                        "fused_mx_gemm": {"value": tf(ms_fused), "unit": "TFLOP/s", "ms": ms_fused,
+                                          "note": "mx_gemm without scratch memory (decode inside the GEMM)"},
+                        "mx_gemm_with_lent_workspace": {"value": tf(ms_lent), "unit": "TFLOP/s", "ms": ms_lent},
                         "mx_gemm_e4m3": {"value": tf(ms_pre), "unit": "TFLOP/s", "ms": ms_pre,
                                          "note": "operands re-encoded ahead of time (not the headline: the re-encoding is not timed)",
                                          "exact": int(flag.item()) == 0},

@@ -230,3 +230,30 @@ def test_padded_plane_pitches_unpack_and_ws_gemm():
     torch.cuda.synchronize()
     assert rel_frob(c.cpu().numpy(), oracle_gemm(bdr.MX6, a, bdr.MX9, b)) <= 1e-5
     assert bdr.mx_gemm_status() == 0 and bdr.bdr_device_status() == 0
+
+
+def test_mx_gemm_uses_a_lent_workspace_and_gives_it_back():
+    # the same call, with and without scratch memory lent to the library: same product (up to summation order);
+    # the scratch is touched only while it is lent
+    M, N, K = 512, 256, 768
+    a = synth.normal_matrix(M, K, seed=13, stream=1)
+    b = synth.normal_matrix(N, K, seed=13, stream=2, sigma=0.02)
+    nbytes = max(bdr.mx_gemm_f8_workspace_bytes(M, N, K), bdr.mx_gemm_workspace_bytes(M, N, K))
+    ws = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+    try:
+        for fa, fb in ((bdr.MX6, bdr.MX4), (bdr.MX9, bdr.MX6)):
+            ref = oracle_gemm(fa, a, fb, b)
+            ws.fill_(0xAB)
+            bdr.bdr_set_workspace(ws)
+            c = gpu_gemm(fa, a, fb, b)
+            assert rel_frob(c, ref) <= 1e-5
+            assert int((ws != 0xAB).sum().item()) > M * K // 2           # the two-phase kernels ran
+            ws.fill_(0xAB)
+            bdr.bdr_set_workspace(None)
+            c = gpu_gemm(fa, a, fb, b)
+            assert rel_frob(c, ref) <= 1e-5
+            assert int((ws != 0xAB).sum().item()) == 0                    # back to the kernel without scratch
+        bdr.bdr_set_workspace(ws[:1024])                                 # too small: the call still works
+        assert rel_frob(gpu_gemm(bdr.MX6, a, bdr.MX6, b), oracle_gemm(bdr.MX6, a, bdr.MX6, b)) <= 1e-5
+    finally:
+        bdr.bdr_set_workspace(None)
