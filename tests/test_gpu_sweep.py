@@ -85,3 +85,16 @@ def test_sweep_degenerate_tensors_and_errors():
         bdr.bdr_qsnr([bdr.Config(16, 8, 3, 1, 4)], x, out, ws)
     assert e.value.status == -2
     torch.cuda.synchronize()
+
+
+def test_full_size_sweep_on_sampled_configurations():
+    # the benchmark's sweep workload itself: all 457 configurations over 2^24 values in one call (the launch
+    # bench.py times); the oracle recomputes every 12th configuration and all comparators one by one
+    cfgs = [c for _, c in sweep.sweep_configs()]
+    x = synth.sweep_distribution("normal_outliers", 1 << 24, seed=0).reshape(1, -1)
+    got = run_sweep(cfgs, x)
+    picked = list(range(0, 441, 12)) + list(range(441, 457))
+    for i in picked:
+        want = orc.qsnr(H.to_orc(cfgs[i]), x, nthreads=16)
+        assert abs(got[i] - want) <= H.QSNR_REL_TOL * max(abs(want), 1e-3), (i, cfgs[i], got[i], want)
+    assert np.isfinite(got).all()
