@@ -107,21 +107,34 @@ col_mx_x2_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant
                 async::report_timeout(status);
                 failed = true;
             }
+            // Packing with sums is the variant with the most live registers: there the second word column is
+            // loaded only when the first is done (and the stage is refilled after that), which keeps 16 registers free.
+            constexpr bool kLate = PACK && SUMS && !YOUT;
             uint32_t wc[2][16];
             const uint32_t mine = ring0 + stg * kCBoxBytes + lane * 8;
+            if constexpr (!kLate) {
 #pragma unroll
-            for (int r = 0; r < kSlice; ++r) {
-                const uint2 v = async::lds64(mine + r * (kCTileCols * 2));
-                wc[0][r] = v.x;
-                wc[1][r] = v.y;
-            }
-            if constexpr (!YOUT) {
-                __syncwarp();  // every lane has read the stage: refill it with the same block row of the next tile
-                if (lane == 0 && !failed && t + (int)gridDim.x < n_tiles) issue(t + gridDim.x, i, stg);
+                for (int r = 0; r < kSlice; ++r) {
+                    const uint2 v = async::lds64(mine + r * (kCTileCols * 2));
+                    wc[0][r] = v.x;
+                    wc[1][r] = v.y;
+                }
+                if constexpr (!YOUT) {
+                    __syncwarp();  // every lane has read the stage: refill it with the same block row of the next tile
+                    if (lane == 0 && !failed && t + (int)gridDim.x < n_tiles) issue(t + gridDim.x, i, stg);
+                }
             }
             uint32_t Fb[4], Mb[4];
 #pragma unroll
             for (int c = 0; c < 2; ++c) {  // the lane's two word columns
+                if constexpr (kLate) {
+#pragma unroll
+                    for (int r = 0; r < kSlice; ++r) wc[c][r] = async::lds32(mine + 4 * c + r * (kCTileCols * 2));
+                    if (c == 1) {
+                        __syncwarp();
+                        if (lane == 0 && !failed && t + (int)gridDim.x < n_tiles) issue(t + gridDim.x, i, stg);
+                    }
+                }
                 uint32_t aw[16], pm[8], yw[16], cl[NCW], ch[NCW], F2;
                 x2::WordColOut o;
                 if (x2::wordcol_exponents(wc[c], aw, pm, F2)) {
