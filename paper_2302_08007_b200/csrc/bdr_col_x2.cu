@@ -107,9 +107,10 @@ col_mx_x2_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant
                 async::report_timeout(status);
                 failed = true;
             }
-            // Packing with sums is the variant with the most live registers: there the second word column is
-            // loaded only when the first is done (and the stage is refilled after that), which keeps 16 registers free.
-            constexpr bool kLate = PACK && SUMS && !YOUT;
+            // Packing with sums or with dequantized output are the variants with the most live registers: there the
+            // second word column is loaded only when the first is done (and, without output, the stage is refilled
+            // after that), which keeps 16 registers free.
+            constexpr bool kLate = PACK && (SUMS || YOUT);
             uint32_t wc[2][16];
             const uint32_t mine = ring0 + stg * kCBoxBytes + lane * 8;
             if constexpr (!kLate) {
@@ -130,9 +131,11 @@ col_mx_x2_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant
                 if constexpr (kLate) {
 #pragma unroll
                     for (int r = 0; r < kSlice; ++r) wc[c][r] = async::lds32(mine + 4 * c + r * (kCTileCols * 2));
-                    if (c == 1) {
-                        __syncwarp();
-                        if (lane == 0 && !failed && t + (int)gridDim.x < n_tiles) issue(t + gridDim.x, i, stg);
+                    if constexpr (!YOUT) {
+                        if (c == 1) {
+                            __syncwarp();
+                            if (lane == 0 && !failed && t + (int)gridDim.x < n_tiles) issue(t + gridDim.x, i, stg);
+                        }
                     }
                 }
                 uint32_t aw[16], pm[8], yw[16], cl[NCW], ch[NCW], F2;
@@ -160,7 +163,10 @@ col_mx_x2_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant
                     o.micro_hi = so.micro_hi;
                     if constexpr (SUMS) { e2 += so.e2; s2 += so.s2; }
                 }
-                if constexpr (YOUT) {
+                if constexpr (YOUT && kLate) {  // results over the word column's input right away
+#pragma unroll
+                    for (int r = 0; r < 16; ++r) async::sts32(mine + 4 * c + r * (kCTileCols * 2), yw[r]);
+                } else if constexpr (YOUT) {
 #pragma unroll
                     for (int r = 0; r < 16; ++r) wc[c][r] = yw[r];  // reuse the input registers for the output rows
                 }
@@ -198,8 +204,10 @@ col_mx_x2_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant
             if constexpr (YOUT) {
                 // results over the box's input, then one tile store; the stage of the previous step (whose store
                 // has been read out by then) takes the box two steps ahead
+                if constexpr (!kLate) {
 #pragma unroll
-                for (int r = 0; r < kSlice; ++r) async::sts64(mine + r * (kCTileCols * 2), wc[0][r], wc[1][r]);
+                    for (int r = 0; r < kSlice; ++r) async::sts64(mine + r * (kCTileCols * 2), wc[0][r], wc[1][r]);
+                }
                 async::fence_proxy_async();
                 __syncwarp();
                 if (lane == 0) {
