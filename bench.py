@@ -37,15 +37,15 @@ FALLBACK_BF16_TFLOPS = 1590.0
 # profiles/step_kernels_dram_traffic.md.  Writes that still sit in L2 when a kernel ends are not
 # counted by those counters, which is why some figures are below the algorithmic bytes.
 NCU_TRAFFIC_BYTES: dict[str, float | None] = {
-    "quant_dequant_MX4_row": 216804096, "quant_dequant_MX4_col": 216572928,
-    "quant_dequant_MX6_row": 216876800, "quant_dequant_MX6_col": 216743168,
-    "quant_dequant_MX9_row": 216424704, "quant_dequant_MX9_col": 216255232,
-    "pack_MX4_row": 149431296, "pack_MX4_col": 146424832,
-    "pack_MX6_row": 157652224, "pack_MX6_col": 154688512,
-    "pack_MX9_row": 173349120, "pack_MX9_col": 168726784,
-    "unpack_MX4_row": 113256704, "unpack_MX4_col": 108517888,
-    "unpack_MX6_row": 128259584, "unpack_MX6_col": 126010880,
-    "unpack_MX9_row": 154560000, "unpack_MX9_col": 151881984,
+    "quant_dequant_MX4_row": 216616960, "quant_dequant_MX4_col": 216386048,
+    "quant_dequant_MX6_row": 216921600, "quant_dequant_MX6_col": 216279296,
+    "quant_dequant_MX9_row": 218355200, "quant_dequant_MX9_col": 216524800,
+    "pack_MX4_row": 148879104, "pack_MX4_col": 146531584,
+    "pack_MX6_row": 157287936, "pack_MX6_col": 154167808,
+    "pack_MX9_row": 173157376, "pack_MX9_col": 168432640,
+    "unpack_MX4_row": 111313664, "unpack_MX4_col": 108342528,
+    "unpack_MX6_row": 130237440, "unpack_MX6_col": 126141952,
+    "unpack_MX9_row": 154232832, "unpack_MX9_col": 151379968,
 }
 
 
