@@ -24,10 +24,12 @@
 //   the sign bit of the input is kept even when the magnitude quantizes to zero; any Inf/NaN in a
 //   block turns the whole block into quiet NaNs with exponent byte 0xFF.
 //
-// Parity pins: every POW2 function here is pinned by tests (closed forms, invariants, brute force,
-// textbook special cases).  The VSQ kind is "parity unpinned" beyond its two reductions (equal
-// per-vector maxima => per-tensor INT; it never exceeds the INT code range): the paper gives no
-// formula for it.
+// Parity pins: every function here is pinned by tests (closed forms, invariants, brute force,
+// textbook special cases, hand-worked examples).  The VSQ kind, for which the paper gives the
+// principle but no formula, is pinned by hand-worked groups (sub-scales that round up, round down,
+// tie, reach the top code and flush to zero; both tie rules; per-group first-level scale) and by its
+// reductions (equal per-vector maxima => per-tensor INT; a 16-bit sub-scale => INT with one FP32
+// scale per vector, within a derived bound).
 //
 // Build: g++ -O2 -std=c++17 -ffp-contract=off -fPIC -shared bdr_oracle.cpp -o liboracle_bdr.so -lpthread
 

@@ -497,9 +497,9 @@ __global__ void qsnr_finalize_kernel(const double* err_sums, const double* sig_s
 }
 
 // workspace layout: [n] error sums | signal sum | amax bits (+pad to 16) | [n] SweepCfg
-static size_t ws_cfg_offset(int n) { return (((size_t)n + 1) * 8 + 16 + 15) / 16 * 16; }
+static constexpr size_t ws_cfg_offset(int n) { return (((size_t)n + 1) * 8 + 16 + 15) / 16 * 16; }
 
-int64_t sweep_workspace_bytes(int n) { return (int64_t)((ws_cfg_offset(n) + (size_t)n * sizeof(SweepCfg) + 255) / 256 * 256); }
+constexpr int64_t sweep_workspace_bytes(int n) { return (int64_t)((ws_cfg_offset(n) + (size_t)n * sizeof(SweepCfg) + 255) / 256 * 256); }
 
 static bool is_pow2i(int v) { return v > 0 && (v & (v - 1)) == 0; }
 
@@ -598,7 +598,8 @@ static int sweep_launch(const SweepCfg* host_fams, int n_fam, int n, bool need_a
 // code the array's name is only a stand-in symbol, not a device address, so the address a kernel can
 // use is looked up once per device with cudaGetSymbolAddress (below) while that device is current.
 constexpr int kStaticMaxCfgs = 512;
-constexpr size_t kStaticScratchBytes = 20736;  // = sweep_workspace_bytes(512)
+constexpr size_t kStaticScratchBytes = 20736;
+static_assert(kStaticScratchBytes == (size_t)sweep_workspace_bytes(kStaticMaxCfgs), "the built-in scratch holds exactly the documented maximum");
 static __device__ __align__(256) unsigned char g_qsnr_static_scratch[kStaticScratchBytes];
 
 // Device address of the built-in scratch on the current device (set up on first use per device).

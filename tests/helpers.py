@@ -11,6 +11,8 @@ from paper_2302_08007_b200 import synth
 
 # QSNR tolerance from the target statement: 1e-6 dB relative.
 QSNR_REL_TOL = 1e-6
+# Relative bound on the fused sums of Eq. 3 (derivation in assert_qsnr_close): 16 fp32 roundings per partial sum.
+SUM_REL_TOL = 1.01 * 2.0 ** -20
 
 
 def to_orc(cfg: bdr.Config) -> orc.Config:
@@ -70,8 +72,13 @@ def assert_qsnr_close(sums_gpu, sums_orc, what: str = ""):
     if math.isnan(e_o) or math.isnan(s_o):
         assert math.isnan(e_g) or math.isnan(s_g), what
         return
-    # the signal sum is only an ingredient of QSNR; its own accuracy is bounded loosely
-    assert s_g == np.float64(s_o) or abs(s_g - s_o) <= 2e-6 * abs(s_o), (what, s_g, s_o)
+    # Both sums are sums of non-negative terms.  The kernels form each term in fp32 in the block-normalised
+    # domain (one rounding, relative 2^-24, for the square of an fp32 input; exact for bf16 inputs and for the
+    # error terms), add at most 16 of them in fp32 (at most 15 additions, each relative 2^-24 on a partial sum
+    # of non-negative terms) and continue in fp64 after an exact power-of-two rescaling.  A sum of non-negative
+    # terms inherits the worst relative error of its parts: (1 + 2^-24)^16 - 1 < 2^-20.  The fp64 part adds
+    # at most a few 2^-53 per addition and is covered by the 1 % slack.
+    assert s_g == np.float64(s_o) or abs(s_g - s_o) <= SUM_REL_TOL * abs(s_o), (what, s_g, s_o)
     q_g, q_o = orc.qsnr_db(e_g, s_g), orc.qsnr_db(e_o, s_o)
     if math.isinf(q_o) or math.isnan(q_o):
         assert (math.isinf(q_g) and math.isinf(q_o)) or (math.isnan(q_g) and math.isnan(q_o)), (what, q_g, q_o)

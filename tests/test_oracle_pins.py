@@ -429,6 +429,71 @@ def test_vsq_reductions():
     assert qs == sorted(qs) or max(qs) - min(qs) < 1.0
 
 
+def _vsq_cases():
+    """tests/golden/vsq_blocks.txt -> [(name, rounding, k1, m, d2, gammas, [(u, x, q, Q), ...])]."""
+    def expand(field):
+        out = []
+        for tok in field.split():
+            out += [0.0] * int(tok[1:]) if tok[0] == "z" else [float(tok)]
+        assert len(out) == 16, field
+        return out
+    cases = []
+    for row in _golden_rows("vsq_blocks.txt"):
+        if row.startswith("case"):
+            _, name, rnd, k1, m, d2, gam = row.split()
+            cases.append((name, int(rnd), int(k1), int(m), int(d2), [float(g) for g in gam.split(",")], []))
+        else:
+            u, xs, qs, Qs = [f.strip() for f in row[3:].split("|")]
+            cases[-1][-1].append((int(u), expand(xs), expand(qs), expand(Qs)))
+    return cases
+
+
+def test_vsq_hand_worked_groups():
+    # vectors with different maxima: an integer sub-scale that rounds up, one that rounds down (and makes its
+    # largest element clamp), an exact tie in the sub-scale under both tie rules, the top code, an all-zero
+    # vector, a vector flushed by u = 0, ties and clamps of the elements, and the scope of the first-level scale
+    names = set()
+    for name, rnd, k1, m, d2, gammas, vecs in _vsq_cases():
+        names.add(name)
+        x = np.array([v for _, xs, _, _ in vecs for v in xs], dtype=np.float32)
+        want = np.array([v for _, _, _, Qs in vecs for v in Qs], dtype=np.float32)
+        # the file is consistent with itself: Q = sign(x) * q * u * gamma, every product exact
+        for i, (u, xs, qs, Qs) in enumerate(vecs):
+            g = gammas[0] if k1 == 0 else gammas[i * 16 // k1]
+            assert u <= 2 ** d2 - 1 and max(qs) <= 2 ** m - 1
+            assert [abs(v) for v in Qs] == [q * u * g for q in qs], (name, i)
+            assert [math.copysign(1, a) for a in Qs] == [math.copysign(1, a) for a in xs], (name, i)
+        y, _ = orc.quant_dequant(Cfg(k1, 32, 16, d2, m, orc.FP32_VSQ, rnd), x)
+        assert y.view(np.uint32).tolist() == want.view(np.uint32).tolist(), (name, y.tolist(), want.tolist())
+    assert names == {"d4_even", "d4_away", "d6_even", "d6_away", "group32"}
+
+
+def test_vsq_with_a_wide_sub_scale_approaches_int_with_one_fp32_scale_per_vector():
+    # d2 = 16: u_v = RN(s_v / gamma) with gamma = s_max / 65535, so the effective scale u_v * gamma differs from
+    # the vector's ideal scale s_v = amax_v / qmax by |delta| <= 0.5 / u_v (+ fp32 rounding).  With every vector
+    # maximum within a factor 4 of the largest, u_v >= 16383 and |delta| <= 3.1e-5.  An element keeps its code q
+    # unless |x|/s_v lies within qmax * |delta| of a half-integer; then |Q' - Q| <= q * s_v * |delta| <=
+    # 7 * 3.1e-5 * s_v = 2.2e-4 s_v (m = 3); the rare element whose code flips moves by one step s_v (1 + delta).
+    rng = np.random.default_rng(77)
+    x = synth.normal(4096 * 16, 77).reshape(-1, 16)
+    x = (x / np.abs(x).max(axis=1, keepdims=True) * rng.uniform(0.25, 1.0, (4096, 1))).astype(np.float32)
+    m = 3
+    qmax = 2 ** m - 1
+    yv, (ev, sv) = orc.quant_dequant(Cfg(0, 32, 16, 16, m, orc.FP32_VSQ), x.ravel())
+    yi, (ei, si) = orc.quant_dequant(Cfg(16, 32, 1, 0, m, orc.FP32_INT), x.ravel())
+    s_v = (np.abs(x).max(axis=1, keepdims=True) / qmax).astype(np.float64)
+    diff = np.abs(yv.reshape(-1, 16).astype(np.float64) - yi.reshape(-1, 16)) / s_v
+    same_code = diff <= qmax * 3.2e-5
+    flipped = ~same_code
+    assert flipped.mean() < 2 * qmax * 3.2e-5 * 2            # half-integers are hit with probability ~2 q |delta|
+    assert np.all(diff[flipped] <= 1.0 + 1e-3)
+    # RMS error ~ s/sqrt(12); per-element change <= 2.2e-4 s (same code) => |dQSNR| <= 20 log10(1 + 8e-4) < 0.01 dB
+    # for those, plus the flipped ones (error stays about half a step): bound the total by 0.02 dB
+    assert sv == si and abs(orc.qsnr_db(ev, sv) - orc.qsnr_db(ei, si)) < 0.02
+    # and the narrow sub-scales are measurably worse on the same data (the reduction is not vacuous)
+    assert orc.qsnr(Cfg(0, 32, 16, 4, m, orc.FP32_VSQ), x.ravel()) < orc.qsnr_db(ei, si) - 0.1
+
+
 # ---- GEMM reference ---------------------------------------------------------------------------------------------
 def test_gemm_reference_is_the_plain_definition():
     rng = np.random.default_rng(80)

@@ -5,13 +5,16 @@ step, where that framework's pool owns the GPU's memory and a cudaMalloc would b
 stall the device.  For them the library carries its own small scratch array.  This test calls the
 entry point through the C ABI twice in a row (the scratch keeps the previous call's contents, so the
 second call proves it is cleared) and checks both results against the ordinary bdr_qsnr, within the
-QSNR tolerance the other tests use.  It lives in a file that pytest collects last.
+QSNR tolerance the other tests use, and a sample of them (every 12th grid point and every comparator) against
+the CPU oracle, so that the expected values do not come from the library alone.  A further call uses exactly
+as many configurations as the scratch holds.  It lives in a file that pytest collects last.
 """
 import math
 
 import pytest
 import torch
 
+from oracle import oracle as orc
 from paper_2302_08007_b200 import binding as bdr
 from paper_2302_08007_b200 import sweep, synth
 from tests import helpers as H
@@ -37,8 +40,30 @@ def test_static_scratch_sweep_matches_workspace_sweep_twice_in_a_row():
         bdr.bdr_qsnr(cfgs, x, want, ws)
         bdr.bdr_qsnr_static(cfgs, x, got)
         torch.cuda.synchronize()
-        for cfg, g, w in zip(cfgs, got.cpu().tolist(), want.cpu().tolist()):
+        got_h = got.cpu().tolist()
+        for cfg, g, w in zip(cfgs, got_h, want.cpu().tolist()):
             assert _close(g, w), (cfg, g, w)
+        x_h = x.cpu().numpy()
+        for i in list(range(0, 441, 12)) + list(range(441, len(cfgs))):
+            w = orc.qsnr(H.to_orc(cfgs[i]), x_h)
+            assert _close(got_h[i], w), ("oracle", cfgs[i], got_h[i], w)
+
+
+def test_static_scratch_sweep_with_exactly_as_many_configurations_as_it_holds():
+    n = bdr.bdr_qsnr_static_max_cfgs()
+    base = [c for _, c in sweep.sweep_configs()]
+    cfgs = (base + base)[:n]                           # repeats are legal: every entry has its own accumulators
+    assert len(cfgs) == n
+    x_h = synth.sweep_distribution("student_t3", 1 << 15, seed=9).reshape(1, -1)
+    x = torch.from_numpy(x_h).cuda()
+    got = torch.full((n,), -1.0, dtype=torch.float64, device="cuda")
+    bdr.bdr_qsnr_static(cfgs, x, got)
+    torch.cuda.synchronize()
+    got_h = got.cpu().tolist()
+    for i in (0, 5, 440, 441, 456, 457, n - 1):         # first, last and the entries around the repeat
+        w = orc.qsnr(H.to_orc(cfgs[i]), x_h)
+        assert _close(got_h[i], w), (i, cfgs[i], got_h[i], w)
+    assert got_h[457:n] == got_h[:n - 457]              # the second copy of a configuration gives the same number
 
 
 def test_static_scratch_sweep_rejects_more_configurations_than_it_holds():
