@@ -5,10 +5,11 @@ One "step" = one pass of the whole quantization path over one 8192 x 8192 bf16 a
 (Laplace(0,1), 1% outlier columns x50): for each of MX4 / MX6 / MX9 and each direction (row-wise,
 column-wise) a quantize-dequantize with fused QSNR sums, a quantize+pack, and an unpack+dequantize
 -- 18 kernel launches.  `value` is the algorithmic bytes those 18 operations
-must move divided by the device time (GB/s); the MX-GEMM and design-sweep legs are measured
-separately after the timed steps and reported in the same JSON line.
+must move divided by the device time (GB/s); the MX-GEMM, design-sweep, linear-layer and small-vector legs are
+measured separately after the timed steps and reported in the same JSON line.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+    python bench.py --only pack --fmt MX6 --axis 0 [--rows R --cols C --reps N]     # one operation, for profilers
 """
 from __future__ import annotations
 
@@ -213,6 +214,10 @@ def run_reference(args):
 # ---------------------------------------------------------------------------------------------------
 # GPU arm
 # ---------------------------------------------------------------------------------------------------
+N_SETS = 3   # buffer sets rotated so that no launch finds its input in L2 (126 MB)
+REPEATS = 10  # the K-step timed region is measured this many times; the headline is the median
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -232,30 +237,38 @@ def run_ours(args):
     x_bits = synth.f32_to_bf16_bits(x_host)
     del x_host
     x_pinned = torch.from_numpy(x_bits.view(np.int16)).view(torch.bfloat16).pin_memory()
-    x = x_pinned.cuda()
-    n_elems = x.numel()
+    n_elems = x_pinned.numel()
 
     cfgs = {name: bdr.Config(16, 8, 2, 1, m) for name, m in FORMATS}
-    y = torch.empty_like(x)
-    planes = {(name, axis): bdr.alloc_planes(cfgs[name], ROWS, COLS, axis) for name, _ in FORMATS for axis in (1, 0)}
-    ops = [(name, m, axis, op) for name, m in FORMATS for axis in (1, 0) for op in ("quant_dequant", "pack", "unpack")]
+    # N_SETS copies of (x, y, planes).  Operation j of step s reads x[(s + j) % N_SETS] and writes y[(s + j) % N_SETS];
+    # the packs of step s write plane set s % N_SETS and its unpacks read plane set (s + 1) % N_SETS, which was
+    # written two steps (7.7 GB of traffic) earlier.  So no launch reads what one of the two launches before it
+    # read or wrote, and every byte a kernel reads comes from HBM, not from the 126 MB L2.
+    xs = [x_pinned.cuda() for _ in range(N_SETS)]
+    ys = [torch.empty_like(xs[0]) for _ in range(N_SETS)]
+    plane_sets = [{(name, axis): bdr.alloc_planes(cfgs[name], ROWS, COLS, axis) for name, _ in FORMATS for axis in (1, 0)}
+                  for _ in range(N_SETS)]
+    ops = [(name, m, axis, op) for op in ("quant_dequant", "pack", "unpack") for name, m in FORMATS for axis in (1, 0)]
     sums = torch.zeros((len(ops), 2), dtype=torch.float64, device="cuda")
-    sums_host = torch.empty((len(ops), 2), dtype=torch.float64).pin_memory()
-
     sum_views = [sums[i] for i in range(len(ops))]  # made once: no tensor indexing on the launch path
 
-    def run_op(i, name, axis, op, src=None):
-        src = x if src is None else src
+    def run_op(j, s, x_override=None, y_override=None, planes_override=None):
+        name, _m, axis, op = ops[j]
+        k = (s + j) % N_SETS
+        src = xs[k] if x_override is None else x_override
+        dst = ys[k] if y_override is None else y_override
         if op == "quant_dequant":
-            bdr.bdr_quant_dequant(cfgs[name], src, y, axis=axis, qsnr_sums=sum_views[i])
+            bdr.bdr_quant_dequant(cfgs[name], src, dst, axis=axis, qsnr_sums=sum_views[j])
         elif op == "pack":
-            bdr.bdr_pack(cfgs[name], src, planes[(name, axis)], axis=axis)
+            pl = plane_sets[s % N_SETS] if planes_override is None else planes_override
+            bdr.bdr_pack(cfgs[name], src, pl[(name, axis)], axis=axis)
         else:
-            bdr.bdr_unpack(cfgs[name], planes[(name, axis)], y, axis=axis)
+            pl = plane_sets[(s + 1) % N_SETS] if planes_override is None else planes_override
+            bdr.bdr_unpack(cfgs[name], pl[(name, axis)], dst, axis=axis)
 
-    def step_direct(src=None):
-        for i, (name, _m, axis, op) in enumerate(ops):
-            run_op(i, name, axis, op, src)
+    def step_direct(s):
+        for j in range(len(ops)):
+            run_op(j, s)
 
     def capture(fn):
         """One CUDA graph of fn's launches (the library allocates nothing and never synchronises, so its
@@ -267,105 +280,151 @@ def run_ours(args):
             fn()
         return g.replay
 
+    for s in range(N_SETS):   # every plane set is filled before anything reads it
+        step_direct(s)
+    torch.cuda.synchronize()
     use_graph = not args.no_graph
-    step = capture(step_direct) if use_graph else step_direct
+    if use_graph:
+        graphs = [capture(lambda s=s: step_direct(s)) for s in range(N_SETS)]
+        step = lambda s: graphs[s % N_SETS]()
+    else:
+        step = step_direct
 
     def barrier():
         if world > 1:
             dist.barrier()
         torch.cuda.synchronize()
 
-    for _ in range(args.warmup):
-        step()
+    for s in range(args.warmup):
+        step(s)
     barrier()
 
     sampler = ClockSampler(local_rank)
     if rank == 0:
         sampler.start()
         time.sleep(0.3)
-    sums.zero_()
-    barrier()
-    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    ev0.record()
-    for _ in range(args.steps):
-        step()
-    ev1.record()
-    barrier()
-    ms = ev0.elapsed_time(ev1)
+    times = []
+    for _rep in range(REPEATS):   # each repetition: exactly K steps between barrier + synchronize
+        sums.zero_()
+        barrier()
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        ev0.record()
+        for s in range(args.steps):
+            step(s)
+        ev1.record()
+        barrier()
+        times.append(max_over_ranks(ev0.elapsed_time(ev1), world) / args.steps)
     clocks = sampler.stop() if rank == 0 else {}
-    ms = max_over_ranks(ms, world)
-    ms_per_step = ms / args.steps
+    ms_per_step = float(np.median(times))
+    ms_best = float(min(times))
     value = aggregate_value(step_bytes(n_elems), world, ms_per_step)
-    qsnr = {}
-    sums_np = (sums / args.steps).cpu().numpy()
-    for i, (name, _m, axis, op) in enumerate(ops):
-        if op == "quant_dequant":
-            qsnr["%s_axis%d" % (name, axis)] = float(-10.0 * np.log10(sums_np[i, 0] / sums_np[i, 1]))
+    db = bdr.bdr_qsnr_from_sums(sums, torch.empty(len(ops), dtype=torch.float64, device="cuda")).cpu().numpy()
+    qsnr = {"%s_axis%d" % (name, axis): float(db[j]) for j, (name, _m, axis, op) in enumerate(ops) if op == "quant_dequant"}
 
     # ---- per-kernel timing on the launching stream (roofline of the dominant kernel) ----
+    # one graph of N_SETS launches of the operation, one per buffer set, replayed: consecutive launches never touch
+    # the same buffers, so inputs (also the 34-76 MB of planes an unpack reads) come from HBM
     kernels = {}
-    reps = max(5, args.steps)
-    for i, (name, m, axis, op) in enumerate(ops):
-        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        one = (lambda i=i, name=name, axis=axis, op=op: run_op(i, name, axis, op))
-        launch = capture(one) if use_graph else one
+    reps = max(5, min(args.steps, 20))
+    for j, (name, m, axis, op) in enumerate(ops):
+        def rot(j=j):
+            for s in range(N_SETS):
+                run_op(j, s, planes_override=plane_sets[s])
+        launch = capture(rot) if use_graph else rot
         launch()
         torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         a.record()
         for _ in range(reps):
             launch()
         b.record()
         torch.cuda.synchronize()
-        dur_ms = a.elapsed_time(b) / reps
+        dur_ms = a.elapsed_time(b) / (reps * N_SETS)
         key = "%s_%s_%s" % (op, name, "row" if axis == 1 else "col")
         kernels[key] = {"ms": dur_ms, "GBps": op_bytes(op, m, n_elems) / (dur_ms * 1e-3) / 1e9}
-    peak, peak_kind, _ = measured_peaks()
+    peak, peak_kind, peaks = measured_peaks()
     dom = max(kernels, key=lambda k: kernels[k]["ms"])
     for k in kernels.values():
         k["frac"] = k["GBps"] / peak
     roofline = {"bound": "hbm", "kernel": dom, "achieved": kernels[dom]["GBps"], "peak": peak, "unit": "GB/s",
                 "frac": kernels[dom]["GBps"] / peak, "peak_source": peak_kind,
-                "traffic": NCU_TRAFFIC_BYTES.get(dom)}
+                "traffic": NCU_TRAFFIC_BYTES.get(dom),
+                "achieved_kind": "algorithmic bytes / CUDA-event time, rotating %d buffer sets" % N_SETS}
 
-    # ---- end to end through the C ABI with host buffers: H2D of the step's input, D2H of its result ----
-    # Two device buffers and a copy stream: the host-to-device copy of step i+1 overlaps the kernels of step i
-    # (every step still copies its whole input from pinned host memory and reads its result back).
-    e2e_steps = max(2, min(args.steps, 6))
-    xin = [x, torch.empty_like(x)]
-    copy_stream = torch.cuda.Stream()
+    # ---- end to end through the C ABI with host buffers ----
+    # Every step copies its input from pinned host memory, runs the 18 C-ABI calls, and copies back to pinned host
+    # memory what the caller of each call receives: the dequantized tensor of every quantize-dequantize and unpack,
+    # the three planes of every pack, and the QSNR sums.  Copy streams in both directions overlap the kernels.
+    e2e_steps = max(2, min(args.steps, 3))
+    xin = [torch.empty_like(xs[0]) for _ in range(2)]
+    y_dev = [torch.empty_like(xs[0]) for _ in range(len(ops))]            # one output tensor per operation
+    y_host = [torch.empty((ROWS, COLS), dtype=torch.bfloat16).pin_memory() if ops[j][3] != "pack" else None for j in range(len(ops))]
+    e2e_planes = plane_sets[0]
+    planes_host = {k: tuple(torch.empty(t.shape, dtype=torch.uint8).pin_memory() for t in (p.exps, p.micro, p.elems))
+                   for k, p in e2e_planes.items()}
+    sums_host = torch.empty((len(ops), 2), dtype=torch.float64).pin_memory()
+    h2d, d2h = torch.cuda.Stream(), torch.cuda.Stream()
     main_stream = torch.cuda.current_stream()
     copied = [torch.cuda.Event() for _ in range(e2e_steps)]
     consumed = [torch.cuda.Event() for _ in range(e2e_steps)]
+    drained = [torch.cuda.Event() for _ in range(e2e_steps)]
+    d2h_bytes = 0
     barrier()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
-    copy_stream.wait_event(e0)
+    h2d.wait_event(e0)
+    d2h.wait_event(e0)
 
     def enqueue_copy(i):
-        with torch.cuda.stream(copy_stream):
+        with torch.cuda.stream(h2d):
             if i >= 2:
-                copy_stream.wait_event(consumed[i - 2])  # the buffer's previous contents have been used
+                h2d.wait_event(consumed[i - 2])  # the buffer's previous contents have been used
             xin[i % 2].copy_(x_pinned, non_blocking=True)
-            copied[i].record(copy_stream)
+            copied[i].record(h2d)
 
     enqueue_copy(0)
     for i in range(e2e_steps):
         if i + 1 < e2e_steps:
             enqueue_copy(i + 1)
         main_stream.wait_event(copied[i])
-        step_direct(xin[i % 2])  # the calls a user makes, one C-ABI call per operation
+        if i >= 1:
+            main_stream.wait_event(drained[i - 1])   # the previous step's results have left the output buffers
+        for j, (name, _m, axis, op) in enumerate(ops):   # the calls a user makes, one C-ABI call per operation
+            run_op(j, 0, x_override=xin[i % 2], y_override=y_dev[j], planes_override=e2e_planes)
+            done = torch.cuda.Event()
+            done.record(main_stream)
+            with torch.cuda.stream(d2h):
+                d2h.wait_event(done)
+                if op == "pack":
+                    p = e2e_planes[(name, axis)]
+                    for src_t, dst_t in zip((p.exps, p.micro, p.elems), planes_host[(name, axis)]):
+                        dst_t.copy_(src_t, non_blocking=True)
+                        d2h_bytes += src_t.numel() if i == 0 else 0
+                else:
+                    y_host[j].copy_(y_dev[j], non_blocking=True)
+                    d2h_bytes += y_dev[j].numel() * 2 if i == 0 else 0
         consumed[i].record(main_stream)
-        sums_host.copy_(sums, non_blocking=True)
+        with torch.cuda.stream(d2h):
+            d2h.wait_event(consumed[i])
+            sums_host.copy_(sums, non_blocking=True)
+            drained[i].record(d2h)
+    main_stream.wait_event(drained[e2e_steps - 1])
     e1.record()
     barrier()
-    e2e_ms = e0.elapsed_time(e1)
-    e2e_ms = max_over_ranks(e2e_ms, world)
+    d2h_bytes += sums.numel() * 8
+    e2e_ms = max_over_ranks(e0.elapsed_time(e1), world)
     e2e = {"value": aggregate_value(step_bytes(n_elems), world, e2e_ms / e2e_steps), "unit": "GB/s",
-           "h2d_bytes_per_step": x.numel() * x.element_size(), "d2h_bytes_per_step": sums.numel() * 8,
-           "steps": e2e_steps, "overlap": "H2D copy of the next step on a second stream, double-buffered input"}
+           "h2d_bytes_per_step": n_elems * 2, "d2h_bytes_per_step": d2h_bytes, "ms_per_step": e2e_ms / e2e_steps,
+           "steps": e2e_steps,
+           "returns": "dequantized tensor of each quantize-dequantize and unpack, three planes of each pack, QSNR sums",
+           "overlap": "host-to-device copy of the next step and device-to-host copies of finished operations on their own streams",
+           "bound": "PCIe: %.2f GB cross the bus per step" % ((n_elems * 2 + d2h_bytes) / 1e9)}
+    del y_dev, y_host, planes_host, xin
 
     extra = {}
     if rank == 0:
+        args.peaks = peaks
+        args.cpu_legs = world == 1
         extra = secondary_legs(args, bdr, synth, torch)
 
     cpu_baseline = None
@@ -374,9 +433,9 @@ def run_ours(args):
         orc.build()
         cores = len(os.sched_getaffinity(0))
         sample_rows = 4096
-        xs = cpu_sample(x_bits, sample_rows)
-        sec = oracle_step(xs, cores)
-        cpu_baseline = {"value": step_bytes(xs.size) / sec / 1e9, "unit": "GB/s", "cores": cores, "kind": "oracle",
+        xs_cpu = cpu_sample(x_bits, sample_rows)
+        sec = oracle_step(xs_cpu, cores)
+        cpu_baseline = {"value": step_bytes(xs_cpu.size) / sec / 1e9, "unit": "GB/s", "cores": cores, "kind": "oracle",
                         "sample": "first %d of %d rows, all 18 operations once (%.1f s)" % (sample_rows, ROWS, sec)}
 
     if rank == 0:
@@ -385,9 +444,12 @@ def run_ours(args):
                 "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
                 "config": {"workload": "C3: 8192x8192 bf16 Laplace(0,1), 1% outlier columns x50; MX4/MX6/MX9 x "
                                        "row/column x (quant-dequant+QSNR, pack, unpack)",
-                           "l2": "inputs larger than L2 (134 MB tensor, >=168 MB streamed per launch)",
+                           "l2": "inputs larger than L2 and rotated: %d sets of (x, y, planes); no launch reads what either "
+                                 "of the two launches before it read or wrote" % N_SETS,
                            "launch": "direct" if args.no_graph else "one CUDA graph of the 18 launches per step",
                            "replicas": "independent tensor per rank, no collective"},
+                "repeats": REPEATS, "ms_per_step_best": ms_best, "ms_per_step_all": times,
+                "value_kind": "median of %d repetitions of the %d-step timed region" % (REPEATS, args.steps),
                 "frac_of_hbm_peak": value / world / peak, "roofline": roofline, "kernels": kernels,
                 "cpu_baseline": cpu_baseline, "e2e": e2e, "gpu_launches": len(ops) * args.steps, "clocks": clocks,
                 "qsnr_db": qsnr}
@@ -398,10 +460,10 @@ def run_ours(args):
 
 
 def secondary_legs(args, bdr, synth, torch) -> dict:
-    """MX-GEMM TFLOP/s and design-sweep configs/s, when those entry points are built."""
-    from paper_2302_08007_b200 import legs
+    """MX-GEMM TFLOP/s, design-sweep configs/s, the linear-layer step and the small-vector latency case."""
+    import bench_legs as legs
     out = {}
-    for fn in (legs.gemm_leg, legs.sweep_leg, legs.linear_leg):
+    for fn in (legs.c1_leg, legs.gemm_leg, legs.sweep_leg, legs.linear_leg):
         try:
             out.update(fn(args))
         except bdr.BdrError as e:
@@ -424,12 +486,25 @@ def secondary_legs(args, bdr, synth, torch) -> dict:
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-graph", action="store_true", help="launch every kernel from Python instead of replaying a CUDA graph of the step")
+    ap.add_argument("--only", default=None, choices=["quant_dequant", "pack", "unpack", "pack2", "gemm", "gemm_ws", "gemm_f8", "sweep"],
+                    help="run one operation a few times on a seeded tensor and print its time (for profilers); no JSON line")
+    ap.add_argument("--fmt", default="MX6", choices=["MX4", "MX6", "MX9"])
+    ap.add_argument("--axis", type=int, default=1)
+    ap.add_argument("--dtype", default="bf16", choices=["bf16", "f32"])
+    ap.add_argument("--rows", type=int, default=8192)
+    ap.add_argument("--cols", type=int, default=8192)
+    ap.add_argument("--reps", type=int, default=3)
+    ap.add_argument("--no-sums", action="store_true", help="--only quant_dequant / pack: without the fused QSNR sums")
+    ap.add_argument("--no-y", action="store_true", help="--only quant_dequant: only the QSNR sums")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.only:
+        import bench_legs
+        return bench_legs.run_only(args)
     if args.impl == "reference":
         run_reference(args)
     else:

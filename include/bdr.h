@@ -87,6 +87,17 @@ const char* bdr_strerror(int status);
  * interest, not between launches. */
 int bdr_device_status(void);
 
+/* Self-tests of the library's failure handling.  (The paper has no counterpart.)
+ * bdr_selftest_bounded_wait queues a one-warp kernel that waits, with the same bounded wait the streaming
+ * kernels use (cut down to a few hundred polls, well under a millisecond), on a barrier that nothing
+ * completes.  The wait runs out by design; the kernel then reports BDR_ERR_TIMEOUT into `status_dev` (one
+ * int of device memory that the caller zeroed: NOT the library's own sticky word, which stays clean) and
+ * ends normally, so the context stays usable.  It shows that a wait that gives up is reported and does not
+ * hang the GPU.  bdr_selftest_host checks, without any CUDA call, the per-device bookkeeping that decides when
+ * a kernel's launch attributes are set (once per device, not once per process); BDR_OK when it holds. */
+int bdr_selftest_bounded_wait(int* status_dev, void* stream);
+int bdr_selftest_host(void);
+
 /* Section III bits-per-element formula realised as plane sizes (host only).  ld_out / bytes_out
  * (host arrays of 3: exps, micro, elems) receive the default line pitches (rounded up to 16 bytes)
  * and total plane sizes for a [rows, cols] tensor quantized along `axis`. */
@@ -121,18 +132,29 @@ int bdr_pack(const bdr_config_t* cfg /*host*/, const void* x, bdr_dtype_t dt, in
 int bdr_unpack(const bdr_config_t* cfg /*host*/, const bdr_planes_t* in /*host struct*/, void* y, bdr_dtype_t dt,
                int64_t rows, int64_t cols, int64_t ld, int axis, void* stream);
 
+/* Eq. 3 from accumulated sums: qsnr_db_dev[i] = -10 log10(sums_dev[2i] / sums_dev[2i+1]) for n pairs
+ * {sum (Q(x)-x)^2, sum x^2} as bdr_quant_dequant / bdr_pack accumulate them (device pointers, 8-byte aligned;
+ * a zero error sum over a non-zero signal gives +inf, a zero signal NaN).  The sums stay usable: they are
+ * only read. */
+int bdr_qsnr_from_sums(const double* sums_dev, int n, double* qsnr_db_dev, void* stream);
+
 /* Bytes of device scratch that bdr_qsnr needs for n_cfgs configurations (host only). */
 int64_t bdr_qsnr_workspace_bytes(int n_cfgs);
 
 /* The design-space sweep of Section IV: QSNR (Eq. 3, in dB, ratio of whole-tensor sums) of one
  * tensor under n_cfgs configurations, reading the tensor once per group of configurations.
- *   cfgs         host array; POW2 entries as above; FP32_INT / FP32_FP (d2 = 4,m = 3 or d2 = 5,m = 2)
- *                / FP32_VSQ entries need k1 = 0 (per-tensor FP32 scale from the current amax)
+ *   cfgs         host array.  POW2 entries as above, with k2 <= 16 whenever d2 > 0 (BDR_ERR_UNSUPPORTED beyond).
+ *                FP32_INT (1 <= m <= 15), FP32_FP (a scalar float with d2 = 2..5 exponent bits and m = 1..7
+ *                explicit mantissa bits, bias 2^(d2-1)-1, gradual underflow, top exponent reserved except
+ *                for d2 = 4, m = 3, which is E4M3 with maximum 448; E5M2 is d2 = 5, m = 2) and FP32_VSQ
+ *                (k2 = 16, 1 <= d2 <= 16, 1 <= m <= 15) entries need k1 = 0: one FP32 scale for the whole
+ *                tensor, from the current amax
  *   qsnr_db_dev  n_cfgs doubles, written (not accumulated)
  *   workspace    device scratch of at least bdr_qsnr_workspace_bytes(n_cfgs) bytes, 16-byte aligned;
  *                contents are overwritten
- * 1 <= n_cfgs <= 4096.  axis must be 1 (rows are the lines); column-direction QSNR of a single
- * configuration comes from bdr_quant_dequant's fused sums. */
+ * 1 <= n_cfgs <= 4096.  axis 1: rows are the lines; axis 0: columns are the lines (blocks and VSQ vectors
+ * run down a column; the loads are strided, so this direction reads slower, which matters little to a
+ * kernel that is bound by arithmetic). */
 int bdr_qsnr(const bdr_config_t* cfgs /*host*/, int n_cfgs, const void* x, bdr_dtype_t dt, int64_t rows,
              int64_t cols, int64_t ld, int axis, double* qsnr_db_dev, void* workspace, int64_t workspace_bytes,
              void* stream);

@@ -22,7 +22,7 @@ F32, BF16 = 0, 1
 EXPORTS = ("bdr_strerror", "bdr_device_status", "bdr_packed_sizes", "bdr_quant_dequant", "bdr_pack", "bdr_unpack",
            "bdr_qsnr_workspace_bytes", "bdr_qsnr", "bdr_qsnr_static_max_cfgs", "bdr_qsnr_static", "mx_gemm",
            "mx_gemm_workspace_bytes", "mx_gemm_ws", "mx_gemm_f8_workspace_bytes", "mx_gemm_f8", "bdr_reencode_e4m3", "mx_gemm_e4m3", "bdr_set_workspace",
-           "mx_gemm_status")
+           "mx_gemm_status", "bdr_selftest_bounded_wait", "bdr_selftest_host", "bdr_qsnr_from_sums")
 
 
 class BdrError(RuntimeError):
@@ -124,6 +124,12 @@ def lib():
         L.mx_gemm_status.argtypes = []
         L.bdr_device_status.restype = C.c_int
         L.bdr_device_status.argtypes = []
+        L.bdr_selftest_bounded_wait.restype = C.c_int
+        L.bdr_selftest_bounded_wait.argtypes = [C.c_void_p, C.c_void_p]
+        L.bdr_selftest_host.restype = C.c_int
+        L.bdr_selftest_host.argtypes = []
+        L.bdr_qsnr_from_sums.restype = C.c_int
+        L.bdr_qsnr_from_sums.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p]
         for fn in (L.bdr_packed_sizes, L.bdr_quant_dequant, L.bdr_pack, L.bdr_unpack, L.bdr_qsnr, L.mx_gemm):
             fn.restype = C.c_int
         _lib = L
@@ -311,6 +317,28 @@ def mx_gemm_e4m3(a: torch.Tensor, scales_a: torch.Tensor, b: torch.Tensor, scale
 def bdr_device_status() -> int:
     """Sticky per-device status of the kernels' bounded waits (0 = ok); synchronises."""
     return int(lib().bdr_device_status())
+
+
+def bdr_qsnr_from_sums(sums: torch.Tensor, out_db: torch.Tensor, stream=None) -> torch.Tensor:
+    """Eq. 3 in dB for every {error, signal} pair of `sums` ([n, 2] or [2] float64, device) into out_db ([n] float64)."""
+    assert sums.dtype == torch.float64 and out_db.dtype == torch.float64 and sums.is_contiguous() and out_db.is_contiguous()
+    n = sums.numel() // 2
+    assert sums.numel() == 2 * n and out_db.numel() >= n
+    _check(lib().bdr_qsnr_from_sums(C.c_void_p(sums.data_ptr()), n, C.c_void_p(out_db.data_ptr()), _stream(stream)),
+           "bdr_qsnr_from_sums")
+    return out_db
+
+
+def bdr_selftest_bounded_wait(status_word) -> None:
+    """Queues the kernel whose bounded wait runs out by design; it leaves BDR_ERR_TIMEOUT (-8) in `status_word`,
+    one zeroed int32 on the device."""
+    assert status_word.dtype == torch.int32 and status_word.numel() == 1 and status_word.is_cuda
+    _check(lib().bdr_selftest_bounded_wait(C.c_void_p(status_word.data_ptr()), _stream(None)), "bdr_selftest_bounded_wait")
+
+
+def bdr_selftest_host() -> int:
+    """Host-only check of the per-device launch bookkeeping (0 = ok); makes no CUDA call."""
+    return int(lib().bdr_selftest_host())
 
 
 def mx_gemm_status() -> int:

@@ -32,6 +32,20 @@ bool make_tensor_map_u16(CUtensorMap* out, const void* base, int64_t rows, int64
               CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// One warp arms a barrier that nothing will ever complete and waits on it with the kernels' own bounded wait,
+// cut down to a few hundred polls (well under a millisecond): the wait runs out, the warp reports it the way
+// the streaming kernels do, and the kernel ends normally.
+__global__ void bounded_wait_selftest_kernel(int* status) {
+    __shared__ __align__(8) uint64_t bar;
+    const uint32_t b = async::smem_u32(&bar);
+    if (threadIdx.x == 0) {
+        async::mbar_init(b, 1);
+        async::fence_barrier_init();
+    }
+    __syncwarp();
+    if (threadIdx.x == 0 && !async::mbar_wait<256>(b, 0)) async::report_timeout(status);
+}
+
 int* device_status_word() {
     static int* cached[64];
     static std::mutex mu;
@@ -165,6 +179,30 @@ int bdr_device_status(void) {
     int v = 0;
     if (!word || cudaMemcpy(&v, word, sizeof(v), cudaMemcpyDeviceToHost) != cudaSuccess) return BDR_ERR_CUDA;
     return v;
+}
+
+int bdr_selftest_bounded_wait(int* status_dev, void* stream) {
+    if (!status_dev) return BDR_ERR_NULL;
+    if ((uintptr_t)status_dev % 4) return BDR_ERR_MISALIGNED;
+    bounded_wait_selftest_kernel<<<1, 32, 0, (cudaStream_t)stream>>>(status_dev);
+    return cudaGetLastError() == cudaSuccess ? BDR_OK : BDR_ERR_CUDA;
+}
+
+int bdr_selftest_host(void) {
+    // PerDevice: the set-up runs once per device, a failed set-up is not remembered, bad indices are refused
+    static PerDevice once;
+    int runs[kMaxDevices] = {};
+    auto setup_for = [&](int dev) { return [&runs, dev]() -> int { ++runs[dev]; return 10 + dev; }; };
+    const int order[] = {0, 1, 0, 63, 1, 0, 63};
+    for (int dev : order)
+        if (once.get(dev, setup_for(dev)) != 10 + dev) return BDR_ERR_CUDA;
+    if (runs[0] != 1 || runs[1] != 1 || runs[63] != 1 || runs[2] != 0) return BDR_ERR_CUDA;
+    int failures = 0;
+    if (once.get(2, [&]() -> int { ++failures; return 0; }) != 0) return BDR_ERR_CUDA;  // fails: nothing is remembered ...
+    if (once.get(2, [&]() -> int { ++failures; return 7; }) != 7) return BDR_ERR_CUDA;  // ... so the next call sets up again
+    if (once.get(2, [&]() -> int { ++failures; return 9; }) != 7 || failures != 2) return BDR_ERR_CUDA;
+    if (once.get(-1, setup_for(0)) != -1 || once.get(kMaxDevices, setup_for(0)) != -1 || runs[0] != 1) return BDR_ERR_CUDA;
+    return BDR_OK;
 }
 
 int bdr_packed_sizes(const bdr_config_t* cfg, int64_t rows, int64_t cols, int axis, int64_t ld_out[3],

@@ -226,11 +226,8 @@ static int launch_col(const T* x, T* y, int64_t rows, int64_t cols, int64_t ld, 
     if (out) pl = *out;
     auto kern = quant_colwise_mx_kernel<T, W, SUMS, YOUT>;
     const size_t smem = ColRing<T>::kBytes + (W > 0 ? sizeof(ColStage<W>) : 16);
-    static bool attr_done = false;
-    if (!attr_done) {
-        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return BDR_ERR_CUDA;
-        attr_done = true;
-    }
+    static PerDevice once;  // per instantiation
+    if (kernel_setup(once, kern, kColThreads, smem) < 1) return BDR_ERR_CUDA;
     kern<<<grid, kColThreads, smem, st>>>(x, y, rows, cols, ld, pl, qp, sums);
     return cudaGetLastError() == cudaSuccess ? BDR_OK : BDR_ERR_CUDA;
 }

@@ -142,15 +142,9 @@ template <int QCOLS, bool SUMS, bool YOUT>
 static int launch_col_qd(const bf16* x, bf16* y, int64_t rows, int64_t cols, int64_t ld, const QParams& qp, double* sums, cudaStream_t st) {
     using SL = QSlab<QCOLS>;
     auto kern = col_qd_x2_kernel<QCOLS, SUMS, YOUT>;
-    static bool attr_done = false;  // per instantiation; the attribute is idempotent, so a race is harmless
-    static int blocks_per_sm = 0;
-    if (!attr_done) {
-        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SL::kSmem) != cudaSuccess) return BDR_ERR_CUDA;
-        int n = 0;
-        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, kern, SL::kThreads, SL::kSmem) != cudaSuccess || n < 1) n = 1;
-        blocks_per_sm = n;
-        attr_done = true;
-    }
+    static PerDevice once;  // per instantiation
+    const int blocks_per_sm = kernel_setup(once, kern, SL::kThreads, SL::kSmem);
+    if (blocks_per_sm < 1) return BDR_ERR_CUDA;
     int* status = device_status_word();
     if (!status) return BDR_ERR_CUDA;
     const int n_cs = (int)(cols / QCOLS);

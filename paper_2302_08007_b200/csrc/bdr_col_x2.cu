@@ -270,15 +270,9 @@ static int launch_col_x2(const bf16* x, bf16* y, int64_t rows, int64_t cols, int
                          const QParams& qp, double* sums, cudaStream_t st) {
     auto kern = col_mx_x2_kernel<W, SUMS, YOUT>;
     const size_t smem = CRing<YOUT>::kBytes + kCBarBytes + CStage<W>::kBytes;
-    static bool attr_done = false;  // per instantiation; the attribute is idempotent, so a race is harmless
-    static int blocks_per_sm = 0;
-    if (!attr_done) {
-        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return BDR_ERR_CUDA;
-        int n = 0;
-        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, kern, kCThreads, smem) != cudaSuccess || n < 1) n = 1;
-        blocks_per_sm = n;
-        attr_done = true;
-    }
+    static PerDevice once;  // per instantiation
+    const int blocks_per_sm = kernel_setup(once, kern, kCThreads, smem);
+    if (blocks_per_sm < 1) return BDR_ERR_CUDA;
     int* status = device_status_word();
     if (!status) return BDR_ERR_CUDA;
     CUtensorMap xmap, ymap;

@@ -5,6 +5,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <atomic>
+
 #include "bdr.h"
 
 namespace bdr {
@@ -12,6 +14,47 @@ namespace bdr {
 struct QParams;
 
 int sm_count();  // SMs of the current device (cached per device)
+
+constexpr int kMaxDevices = 64;
+
+// A positive integer remembered per device by one call site (a zero-initialised static object).
+// cudaFuncSetAttribute and the occupancy query apply to the device that is current, so the launchers keep
+// one of these per kernel instantiation: the set-up runs the first time each device launches the kernel,
+// not the first time the process does.  The set-up is idempotent, so two threads that race on the first
+// call of a device both run it and store the same value.
+class PerDevice {
+    std::atomic<int> v_[kMaxDevices];
+
+   public:
+    // value remembered for `dev`, running `setup` (returns > 0, or <= 0 on failure, which is not remembered)
+    // when there is none yet; -1 when `dev` is out of range
+    template <typename F>
+    int get(int dev, F&& setup) {
+        if (dev < 0 || dev >= kMaxDevices) return -1;
+        int v = v_[dev].load(std::memory_order_acquire);
+        if (v > 0) return v;
+        v = setup();
+        if (v > 0) v_[dev].store(v, std::memory_order_release);
+        return v;
+    }
+};
+
+inline int current_device() {
+    int dev = -1;
+    return cudaGetDevice(&dev) == cudaSuccess ? dev : -1;
+}
+
+// Per-device set-up of one kernel: raises its dynamic shared-memory limit to `smem` and returns how many of
+// its CTAs fit on an SM (>= 1); <= 0 when the attribute could not be set on the current device.
+template <typename K>
+int kernel_setup(PerDevice& once, K kern, int threads, size_t smem) {
+    return once.get(current_device(), [&]() -> int {
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return 0;
+        int n = 0;
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, kern, threads, smem) != cudaSuccess || n < 1) n = 1;
+        return n;
+    });
+}
 
 // axis-1 kernels (bdr_row.cu); BDR_ERR_UNSUPPORTED = not covered, use the general kernel
 template <typename T>

@@ -267,11 +267,8 @@ static int launch_quant_row_flags(const T* x, T* y, int64_t rows, int64_t cols, 
     if (total >= (1ll << 31) - (1ll << 24)) return BDR_ERR_UNSUPPORTED;  // 32-bit unit indices (incl. prefetch look-ahead)
     auto kern = quant_rowwise_kernel<T, K2, K1S, SPT, SUMS, YOUT>;
     const size_t smem = Ring<T, SPT>::kBytes;
-    static bool attr_done = false;  // per instantiation; the attribute is idempotent, so a race is harmless
-    if (!attr_done) {
-        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return BDR_ERR_CUDA;
-        attr_done = true;
-    }
+    static PerDevice once;  // per instantiation
+    if (kernel_setup(once, kern, kThreads, smem) < 1) return BDR_ERR_CUDA;
     kern<<<grid_for(total, kThreads), kThreads, smem, st>>>(x, y, rows, cols, ld, make_fastdiv((uint32_t)upr), (uint32_t)total, group, qp,
                                                             vec_ok, all_full, sums);
     return cudaGetLastError() == cudaSuccess ? BDR_OK : BDR_ERR_CUDA;
@@ -331,11 +328,8 @@ static int launch_pack_row(const T* x, T* y, int64_t rows, int64_t cols, int64_t
     if (total >= (1ll << 31) - (1ll << 24)) return BDR_ERR_UNSUPPORTED;
     auto kern = pack_rowwise_mx_kernel<T, W, SUMS, YDQ>;
     const size_t smem = Ring<T, kPackSPT>::kBytes + (kThreads / 32) * PackStage<W>::kBytes;
-    static bool attr_done = false;
-    if (!attr_done) {
-        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return BDR_ERR_CUDA;
-        attr_done = true;
-    }
+    static PerDevice once;  // per instantiation
+    if (kernel_setup(once, kern, kThreads, smem) < 1) return BDR_ERR_CUDA;
     kern<<<grid_for(total, kThreads / 32), kThreads, smem, st>>>(x, y, make_fastdiv((uint32_t)(cols / 1024)), (uint32_t)total, ld, out, qp, sums);
     return cudaGetLastError() == cudaSuccess ? BDR_OK : BDR_ERR_CUDA;
 }

@@ -96,6 +96,19 @@ row_mx_x2_kernel(const bf16* x, bf16* y, RunIndex ri, uint32_t total, bdr_planes
         __syncwarp();  // lane 0 has finished the previous iteration's hand-over (staging half is free)
         if (!async::mbar_wait(bars + 8 * st, phase)) {
             async::report_timeout(status);
+            // Nothing more is issued.  The loads queued for this and the next kX2Ahead - 1 runs may still be on
+            // their way into this CTA's shared memory: give each of them one further bounded wait, so that the
+            // CTA does not knowingly leave with a copy in flight (if one still does not land, the CTA leaves
+            // all the same: the wait must end).
+            if (lane == 0) {
+                for (int s = 0; s < kX2Ahead; ++s) {
+                    if ((uint64_t)wi + (uint64_t)s * stride >= total) break;
+                    int ds = st + s;
+                    uint32_t dp = phase;
+                    if (ds >= S) { ds -= S; dp ^= 1; }
+                    async::mbar_wait(bars + 8 * ds, dp);
+                }
+            }
             break;
         }
         const uint32_t stage = stage0 + half * PS::kBytes;
@@ -267,13 +280,7 @@ static bool x2_config(const QParams& qp, bool pack) {
 
 // One wave of resident CTAs: every warp then streams many runs through its prefetch ring instead of
 // paying the ring's start-up again in a second, partly filled wave.
-template <typename K>
-static int x2_grid(K kern, size_t smem, int64_t total_warps, int& blocks_per_sm) {
-    if (blocks_per_sm == 0) {
-        int n = 0;
-        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, kern, kX2Threads, smem) != cudaSuccess || n < 1) n = 2;
-        blocks_per_sm = n;
-    }
+static int x2_grid(int64_t total_warps, int blocks_per_sm) {
     const int64_t need = (total_warps + kX2Threads / 32 - 1) / (kX2Threads / 32);
     return (int)max((int64_t)1, min(need, (int64_t)sm_count() * blocks_per_sm));
 }
@@ -286,21 +293,18 @@ static int launch_x2(const bf16* x, bf16* y, int64_t rows, int64_t cols, int64_t
     if (total >= (1ll << 31) - (1ll << 24)) return BDR_ERR_UNSUPPORTED;  // 32-bit run indices (incl. look-ahead)
     auto kern = row_mx_x2_kernel<W, SUMS, YOUT>;
     const size_t smem = X2Ring<YOUT>::kBytes + kX2BarBytes + kX2Warps * 2 * X2PackStage<W>::kBytes;
-    static bool attr_done = false;  // per instantiation; the attribute is idempotent, so a race is harmless
-    if (!attr_done) {
-        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return BDR_ERR_CUDA;
-        attr_done = true;
-    }
+    static PerDevice once;  // per instantiation
+    const int blocks_per_sm = kernel_setup(once, kern, kX2Threads, smem);
+    if (blocks_per_sm < 1) return BDR_ERR_CUDA;
     int* status = device_status_word();
     if (!status) return BDR_ERR_CUDA;
-    static int blocks_per_sm = 0;
     bdr_planes_t pl = {};
     if (out) pl = *out;
     RunIndex ri;
     ri.runs_per_row = make_fastdiv((uint32_t)rpr);
     ri.ld = ld;
     ri.flat = rows == 1 ? 1 : 0;
-    kern<<<x2_grid(kern, smem, total, blocks_per_sm), kX2Threads, smem, st>>>(x, y, ri, (uint32_t)total, pl, qp, sums, status);
+    kern<<<x2_grid(total, blocks_per_sm), kX2Threads, smem, st>>>(x, y, ri, (uint32_t)total, pl, qp, sums, status);
     return cudaGetLastError() == cudaSuccess ? BDR_OK : BDR_ERR_CUDA;
 }
 

@@ -1,18 +1,23 @@
 // bdr_qsnr: the design-space sweep of Section IV -- QSNR (Eq. 3) of one tensor under many
-// configurations, reading the tensor once per group of 64 configurations.
+// configurations, reading the tensor once per group of 16 families of configurations.
 //
-// A CTA stages a tile of 4096 consecutive elements of a row in shared memory (fp32 bit patterns)
-// together with a pyramid of block-maximum exponent bytes for block sizes 2, 4, ..., 1024 (every k1
-// and k2 of the grid is one of its levels).  Then each warp takes configurations round-robin; for
-// one configuration its lanes walk the tile's 16-element slices, evaluate sum (Q(x)-x)^2 with the
-// same slice quantizer as the quantize kernels, and the warp adds the tile's total to a per-CTA
-// accumulator in shared memory.  Only at the end does a CTA touch the global sums (one atomic per
-// configuration), so the tensor is read from HBM once per 64 configurations and the kernel is
-// bound by plain ALU throughput.
+// The host merges configurations that differ only in the mantissa width m into families of up to
+// eight members (same k1, k2, d2, kind and tie rule).  A work unit of a CTA is four tiles of 4096
+// consecutive elements of a line (a row, or a column for axis 0) held in shared memory as fp32 bit
+// patterns, each with a pyramid of block-maximum exponent bytes for block sizes 2, 4, ..., 1024 (every k1
+// and k2 of the grid is one of its levels).  All warps of the CTA then work on the same family at the
+// same time, one 16-element slice per thread and tile: exponents and shifts are computed once per slice,
+// the loop over the family's mantissa widths only changes the rounding constant and the clamp, and
+// sum (Q(x)-x)^2 is formed as in the quantize kernels.  A lane's sums are reduced once per family into
+// per-CTA accumulators in shared memory; only at the end does a CTA touch the global sums (one atomic
+// per configuration), so the tensor is read from HBM once per 16 families and the kernel is bound by
+// plain ALU throughput.
 //
 // The comparator kinds of Table I (INT with an FP32 max-scale, Eq. 1-2; FP8-like scalar floats;
-// VSQ) are evaluated in the same loop with IEEE single operations (division included), so their
-// dequantized values match a plain CPU implementation bit for bit.
+// VSQ) are evaluated in the same loop; their divisions are exact IEEE single divisions (computed by a
+// multiply, a residual and a correction with the correctly rounded reciprocal, or by the divide
+// instruction where that shortcut is not safe), so their dequantized values match a plain CPU
+// implementation bit for bit.
 #include <mutex>
 #include <vector>
 
@@ -347,8 +352,12 @@ __global__ void amax_kernel(const T* x, int64_t rows, int64_t cols, int64_t ld, 
 
 template <typename T>
 __global__ void __launch_bounds__(kSweepThreads)
-sweep_kernel(const T* x, int64_t rows, int64_t cols, int64_t ld, const SweepCfg* fams, int n_fam, int n_cfg, int n_groups,
-             int tiles_per_row, int64_t total_units, double* err_sums, double* sig_sum, const uint32_t* amax_bits) {
+sweep_kernel(const T* x, int64_t n_lines, int64_t len, int64_t line_stride, int64_t elem_stride, const SweepCfg* fams, int n_fam,
+             int n_cfg, int n_groups, int tiles_per_line, int64_t total_units, double* err_sums, double* sig_sum,
+             const uint32_t* amax_bits) {
+    // A line is a row (elem_stride 1, line_stride = the row pitch) or a column (elem_stride = the row pitch,
+    // line_stride 1).  Tiles are numbered line by line for rows; for columns the tiles at the same position of
+    // adjacent columns are neighbours, so that the four tiles of a unit share the 32-byte sectors they touch.
     extern __shared__ __align__(16) uint8_t dyn[];
     SweepSmem& sm = *reinterpret_cast<SweepSmem*>(dyn);
     double* acc = reinterpret_cast<double*>(dyn + sizeof(SweepSmem));  // [n_cfg]
@@ -356,7 +365,8 @@ sweep_kernel(const T* x, int64_t rows, int64_t cols, int64_t ld, const SweepCfg*
     for (int c = threadIdx.x; c < n_cfg; c += kSweepThreads) acc[c] = 0.0;
     double sig_acc = 0.0;
     const float amax = __uint_as_float(*amax_bits);
-    const int64_t total_tiles = rows * tiles_per_row;
+    const int64_t total_tiles = n_lines * tiles_per_line;
+    const bool by_column = elem_stride != 1;
     for (int64_t unit = blockIdx.x; unit < total_units; unit += gridDim.x) {
         const int64_t tgroup = unit / n_groups;              // kTilesPerUnit consecutive tiles
         const int group = (int)(unit - tgroup * n_groups);   // kFamGroup consecutive families
@@ -366,14 +376,22 @@ sweep_kernel(const T* x, int64_t rows, int64_t cols, int64_t ld, const SweepCfg*
         for (int ti = 0; ti < ntiles; ++ti) {
             SweepTile& tl = sm.t[ti];
             const int64_t tile = tile0 + ti;
-            const int64_t row = tile / tiles_per_row;
-            const int64_t t0 = (tile - row * tiles_per_row) * kTile;
-            const int n = (int)min((int64_t)kTile, cols - t0);
-            const T* src = x + row * ld + t0;
+            int64_t line, tpos;
+            if (by_column) {
+                tpos = tile / n_lines;
+                line = tile - tpos * n_lines;
+            } else {
+                line = tile / tiles_per_line;
+                tpos = tile - line * tiles_per_line;
+            }
+            const int64_t t0 = tpos * kTile;
+            const int n = (int)min((int64_t)kTile, len - t0);
+            const T* src = x + line * line_stride + t0 * elem_stride;
             // stage: thread t owns slice t (16 elements = 4 chunks)
             const int s = threadIdx.x;
             uint32_t u[kSlice];
-            load_slice_guarded(src + s * kSlice, 1, max(0, min(kSlice, n - s * kSlice)), u);
+            if (by_column) load_slice_guarded(src + (int64_t)s * kSlice * elem_stride, elem_stride, max(0, min(kSlice, n - s * kSlice)), u);
+            else load_slice_guarded(src + s * kSlice, 1, max(0, min(kSlice, n - s * kSlice)), u);
 #pragma unroll
             for (int v = 0; v < 4; ++v) tl.x[swz4(4 * s + v)] = make_uint4(u[4 * v], u[4 * v + 1], u[4 * v + 2], u[4 * v + 3]);
             // exponent pyramid levels 1..4 from the slice
@@ -496,6 +514,18 @@ __global__ void qsnr_finalize_kernel(const double* err_sums, const double* sig_s
     out_db[i] = q;
 }
 
+// The same for n independent {error, signal} pairs, as the quantize kernels accumulate them.
+__global__ void qsnr_pairs_kernel(const double* sums, int n, double* out_db) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n) return;
+    const double e = sums[2 * i], s = sums[2 * i + 1];
+    double q;
+    if (s == 0.0 || s != s || e != e) q = __longlong_as_double(0x7FF8000000000000ll);
+    else if (e == 0.0) q = __longlong_as_double(0x7FF0000000000000ll);
+    else q = -10.0 * log10(e / s);
+    out_db[i] = q;
+}
+
 // workspace layout: [n] error sums | signal sum | amax bits (+pad to 16) | [n] SweepCfg
 static constexpr size_t ws_cfg_offset(int n) { return (((size_t)n + 1) * 8 + 16 + 15) / 16 * 16; }
 
@@ -561,7 +591,7 @@ static void build_families(const std::vector<SweepCfg>& singles, std::vector<Swe
 
 template <typename T>
 static int sweep_launch(const SweepCfg* host_fams, int n_fam, int n, bool need_amax, const T* x, int64_t rows, int64_t cols,
-                        int64_t ld, double* out_db, uint8_t* ws, cudaStream_t st) {
+                        int64_t ld, int axis, double* out_db, uint8_t* ws, cudaStream_t st) {
     double* err = reinterpret_cast<double*>(ws);
     double* sig = err + n;
     uint32_t* amax = reinterpret_cast<uint32_t*>(sig + 1);
@@ -579,14 +609,17 @@ static int sweep_launch(const SweepCfg* host_fams, int n_fam, int n, bool need_a
             const int grid = (int)max((int64_t)1, min((total + 1023) / 1024, (int64_t)sm_count() * 8));
             amax_kernel<T><<<grid, 256, 0, st>>>(x, rows, cols, ld, amax);
         }
-        const int tiles_per_row = (int)((cols + kTile - 1) / kTile);
+        const int64_t n_lines = axis == 1 ? rows : cols, len = axis == 1 ? cols : rows;
+        const int tiles_per_line = (int)((len + kTile - 1) / kTile);
         const int n_groups = (n_fam + kFamGroup - 1) / kFamGroup;
-        const int64_t units = (rows * tiles_per_row + kTilesPerUnit - 1) / kTilesPerUnit * n_groups;
+        const int64_t units = (n_lines * tiles_per_line + kTilesPerUnit - 1) / kTilesPerUnit * n_groups;
         const size_t smem = sizeof(SweepSmem) + (size_t)n * sizeof(double);
         auto kern = sweep_kernel<T>;
+        // set on every call: the size depends on the number of configurations, and the attribute is per device
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return BDR_ERR_CUDA;
         const int grid = (int)max((int64_t)1, min(units, (int64_t)sm_count() * 2));
-        kern<<<grid, kSweepThreads, smem, st>>>(x, rows, cols, ld, dcfg, n_fam, n, n_groups, tiles_per_row, units, err, sig, amax);
+        kern<<<grid, kSweepThreads, smem, st>>>(x, n_lines, len, axis == 1 ? ld : 1, axis == 1 ? 1 : ld, dcfg, n_fam, n, n_groups,
+                                                tiles_per_line, units, err, sig, amax);
     }
     qsnr_finalize_kernel<<<(n + 127) / 128, 128, 0, st>>>(err, sig, n, out_db);
     return cudaGetLastError() == cudaSuccess ? BDR_OK : BDR_ERR_CUDA;
@@ -645,14 +678,23 @@ int bdr_qsnr(const bdr_config_t* cfgs, int n_cfgs, const void* x, bdr_dtype_t dt
     }
     build_families(singles, &table);
     const int n_fam = (int)table.size();
-    if (axis != 1) return BDR_ERR_UNSUPPORTED;  // the sweep walks rows; column-wise QSNR comes from bdr_quant_dequant's sums
     if (!workspace || workspace_bytes < sweep_workspace_bytes(n_cfgs)) return BDR_ERR_WORKSPACE;
     if ((uintptr_t)workspace % 16) return BDR_ERR_MISALIGNED;
     cudaStream_t st = (cudaStream_t)stream;
     if (dt == BDR_F32)
-        return sweep_launch<float>(table.data(), n_fam, n_cfgs, need_amax, (const float*)x, rows, cols, ld, qsnr_db_dev, (uint8_t*)workspace, st);
-    return sweep_launch<__nv_bfloat16>(table.data(), n_fam, n_cfgs, need_amax, (const __nv_bfloat16*)x, rows, cols, ld, qsnr_db_dev,
+        return sweep_launch<float>(table.data(), n_fam, n_cfgs, need_amax, (const float*)x, rows, cols, ld, axis, qsnr_db_dev,
+                                   (uint8_t*)workspace, st);
+    return sweep_launch<__nv_bfloat16>(table.data(), n_fam, n_cfgs, need_amax, (const __nv_bfloat16*)x, rows, cols, ld, axis, qsnr_db_dev,
                                        (uint8_t*)workspace, st);
+}
+
+int bdr_qsnr_from_sums(const double* sums_dev, int n, double* qsnr_db_dev, void* stream) {
+    if (!sums_dev || !qsnr_db_dev) return BDR_ERR_NULL;
+    if (n < 0) return BDR_ERR_SIZE;
+    if ((uintptr_t)sums_dev % 8 || (uintptr_t)qsnr_db_dev % 8) return BDR_ERR_MISALIGNED;
+    if (n == 0) return BDR_OK;
+    qsnr_pairs_kernel<<<(n + 127) / 128, 128, 0, (cudaStream_t)stream>>>(sums_dev, n, qsnr_db_dev);
+    return cudaGetLastError() == cudaSuccess ? BDR_OK : BDR_ERR_CUDA;
 }
 
 int bdr_qsnr_static_max_cfgs(void) { return kStaticMaxCfgs; }

@@ -138,15 +138,9 @@ template <int W>
 static int launch_unpack_col_x2(const bdr_planes_t& in, bf16* y, int64_t rows, int64_t cols, int64_t ld, cudaStream_t st) {
     auto kern = unpack_col_x2_kernel<W>;
     const size_t smem = 2 * UCStage<W>::kBytes;
-    static bool attr_done = false;  // per instantiation; the attribute is idempotent, so a race is harmless
-    static int blocks_per_sm = 0;
-    if (!attr_done) {
-        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return BDR_ERR_CUDA;
-        int n = 0;
-        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, kern, kUCThreads, smem) != cudaSuccess || n < 1) n = 1;
-        blocks_per_sm = n;
-        attr_done = true;
-    }
+    static PerDevice once;  // per instantiation
+    const int blocks_per_sm = kernel_setup(once, kern, kUCThreads, smem);
+    if (blocks_per_sm < 1) return BDR_ERR_CUDA;
     const int n_ct = (int)(cols / kUCTileCols);
     const int64_t n_tiles = (int64_t)n_ct * (rows / kUCTileRows);
     const int grid = (int)std::min<int64_t>(n_tiles, (int64_t)sm_count() * blocks_per_sm);

@@ -115,15 +115,9 @@ static int launch_unpack_x2(const bdr_planes_t& in, bf16* y, int64_t rows, int64
     if (total >= (1ll << 31) - (1ll << 24)) return BDR_ERR_UNSUPPORTED;
     auto kern = unpack_row_x2_kernel<W>;
     const size_t smem = kUWarps * kUStages * UStage<W>::kBytes + kUBarBytes;
-    static bool attr_done = false;  // per instantiation; the attribute is idempotent, so a race is harmless
-    static int blocks_per_sm = 0;
-    if (!attr_done) {
-        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return BDR_ERR_CUDA;
-        int n = 0;
-        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, kern, kUThreads, smem) != cudaSuccess || n < 1) n = 2;
-        blocks_per_sm = n;
-        attr_done = true;
-    }
+    static PerDevice once;  // per instantiation
+    const int blocks_per_sm = kernel_setup(once, kern, kUThreads, smem);
+    if (blocks_per_sm < 1) return BDR_ERR_CUDA;
     int* status = device_status_word();
     if (!status) return BDR_ERR_CUDA;
     const int64_t need = (total + kUWarps - 1) / kUWarps;

@@ -1,21 +1,26 @@
 // mx_gemm: C[M,N] = deq(A)[M,K] * deq(B)[N,K]^T with both operands given as packed MX planes
 // quantized along K (Section V: both inputs of a tensor operation are MX-quantized along the
-// reduction dimension).  The packed bytes are decoded to bf16 inside the kernel -- every MX value
-// with m <= 7 is exact in bf16 -- and multiplied on the 5th-generation tensor cores
-// (tcgen05.mma, kind::f16, fp32 accumulation in tensor memory).
-//
-// One CTA computes a 128 x 256 tile of C.  Warps 0-11 are decoders, one thread per tile row (128 A
-// rows + 256 B rows): per 64-wide K step a thread reads its row's packed codes / exponents /
-// microexponents from global memory (the operands live in L2) one step ahead of use, rebuilds bf16
-// values with packed bf16x2 arithmetic and stores them in shared memory in the K-major,
-// 128-byte-swizzled layout the tensor core reads.  Warp 12 issues the MMAs (4 x K=16 per stage) and
-// signals stage reuse / accumulator completion through tcgen05.commit on mbarriers.  After the last
-// K step warps 0-7 read the accumulator from tensor memory (tcgen05.ld) and store C.  Every wait is bounded: if one runs out the kernel
-// records BDR_ERR_TIMEOUT in a status word, skips the remaining work, frees its tensor memory and
-// returns.
+// reduction dimension).  The packed bytes are decoded to bf16 -- every MX value with m <= 7 is exact in
+// bf16 -- and multiplied on the 5th-generation tensor cores (tcgen05.mma, fp32 accumulation in tensor
+// memory).  This file holds the shared PTX wrappers, the packed-byte decoder, the C-ABI entry points and the
+// kernels, the last three as textually included headers:
+//   * mx_gemm_kernel (below): one CTA per 128 x 256 tile of C, for shapes the paired kernel does not take.
+//     Warps 0-11 decode, one thread per tile row (128 A rows + 256 B rows): per 64-wide K step a thread reads
+//     its row's packed codes / exponents / microexponents from global memory one step ahead of use, rebuilds
+//     bf16 values with packed bf16x2 arithmetic and stores them in shared memory in the K-major,
+//     128-byte-swizzled layout the tensor core reads.  Warp 12 issues the MMAs (kind::f16, 4 x K=16 per stage)
+//     and signals stage reuse / accumulator completion through tcgen05.commit on mbarriers; warps 0-7 then
+//     read the accumulator from tensor memory (tcgen05.ld) and store C.
+//   * mx_gemm_pair.cuh: the same decode-inside-the-GEMM scheme for a cluster of two CTAs on a 256 x 256 tile
+//     (cta_group::2), packed planes brought in by TMA; what mx_gemm runs when M and K are multiples of 256.
+//   * mx_gemm_dense.cuh: bf16 x bf16 persistent kernel for operands decoded once into a workspace (mx_gemm_ws).
+//   * mx_gemm_f8.cuh: E4M3 x E4M3 block-scaled kernel for operands re-encoded into a workspace (mx_gemm_f8).
+// Every wait is bounded: if one runs out the kernel records BDR_ERR_TIMEOUT in a status word, skips the
+// remaining work, frees its tensor memory and returns.
 #include <cuda.h>
 
 #include <algorithm>
+#include <mutex>
 
 #include "bdr_device.cuh"
 #include "bdr_host.h"
@@ -379,11 +384,8 @@ static int launch_gemm(const bdr_planes_t& a, const bdr_planes_t& b, int64_t M, 
                        const int* gate, cudaStream_t st) {
     auto kern = mx_gemm_kernel<WA, WB>;
     const size_t smem = (size_t)kStages * kStageBytes + 256 + (size_t)(kBM + kBN) * RingStride<WA, WB>::value + 1024;
-    static bool attr_done = false;
-    if (!attr_done) {
-        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return BDR_ERR_CUDA;
-        attr_done = true;
-    }
+    static PerDevice once;  // per instantiation
+    if (kernel_setup(once, kern, kGemmThreads, smem) < 1) return BDR_ERR_CUDA;
     const dim3 grid((unsigned)(N / kBN), (unsigned)(M / kBM));
     kern<<<grid, kGemmThreads, smem, st>>>(a, b, M, N, K, c, ldc, gate);
     return cudaGetLastError() == cudaSuccess ? BDR_OK : BDR_ERR_CUDA;
@@ -444,12 +446,14 @@ extern "C" {
 
 // Scratch memory lent to mx_gemm by the caller (bdr_set_workspace), per device.
 struct LentWorkspace { void* ptr; int64_t bytes; };
-static LentWorkspace g_lent[64] = {};
+static LentWorkspace g_lent[kMaxDevices] = {};
+static std::mutex g_lent_mu;  // bdr_set_workspace on one thread, mx_gemm on another
 
 int bdr_set_workspace(void* workspace, int64_t workspace_bytes) {
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return BDR_ERR_CUDA;
+    const int dev = current_device();
+    if (dev < 0 || dev >= kMaxDevices) return BDR_ERR_CUDA;
     if (workspace && ((uintptr_t)workspace % 256 || workspace_bytes < 0)) return BDR_ERR_MISALIGNED;
+    std::lock_guard<std::mutex> lock(g_lent_mu);
     g_lent[dev].ptr = workspace;
     g_lent[dev].bytes = workspace ? workspace_bytes : 0;
     return BDR_OK;
@@ -465,10 +469,15 @@ int64_t mx_gemm_f8_workspace_bytes(int64_t, int64_t, int64_t);
 int mx_gemm(const bdr_config_t* cfg_a, const bdr_planes_t* a, const bdr_config_t* cfg_b, const bdr_planes_t* b, int64_t M,
             int64_t N, int64_t K, float* c, int64_t ldc, void* stream) {
     // with scratch memory lent by the caller the two-phase kernels are the faster way to the same product
-    int dev = 0;
-    if (cfg_a && cfg_b && M > 0 && N > 0 && M % 256 == 0 && N % 256 == 0 && K % 256 == 0 && cudaGetDevice(&dev) == cudaSuccess && dev >= 0 &&
-        dev < 64 && g_lent[dev].ptr) {
-        const LentWorkspace w = g_lent[dev];
+    LentWorkspace w = {};
+    if (cfg_a && cfg_b && M > 0 && N > 0 && M % 256 == 0 && N % 256 == 0 && K % 256 == 0) {
+        const int dev = current_device();
+        if (dev >= 0 && dev < kMaxDevices) {
+            std::lock_guard<std::mutex> lock(g_lent_mu);
+            w = g_lent[dev];
+        }
+    }
+    if (w.ptr) {
         int rc = BDR_ERR_UNSUPPORTED;
         if (cfg_a->m <= 4 && cfg_b->m <= 4 && w.bytes >= mx_gemm_f8_workspace_bytes(M, N, K))
             rc = mx_gemm_f8(cfg_a, a, cfg_b, b, M, N, K, c, ldc, w.ptr, w.bytes, stream);

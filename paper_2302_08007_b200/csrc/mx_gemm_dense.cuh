@@ -194,12 +194,11 @@ static bool make_dense_map(CUtensorMap* out, const void* base, int64_t rows, int
 // a_bf16 [M, K], b_bf16 [N, K], both contiguous; M, N multiples of 256, K a multiple of 64
 static int launch_gemm_dense(const void* a_bf16, const void* b_bf16, int64_t M, int64_t N, int64_t K, float* c, int64_t ldc,
                              cudaStream_t st) {
-    static bool attr_done = false;
-    if (!attr_done) {
-        if (cudaFuncSetAttribute(bf16_gemm_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kDSmemBytes) != cudaSuccess)
-            return BDR_ERR_CUDA;
-        attr_done = true;
-    }
+    static PerDevice once;
+    if (once.get(current_device(), [&]() -> int {  // no occupancy query: cluster kernel, one CTA per SM
+            return cudaFuncSetAttribute(bf16_gemm_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kDSmemBytes) == cudaSuccess ? 1 : 0;
+        }) < 1)
+        return BDR_ERR_CUDA;
     DenseMaps maps;
     if (!make_dense_map(&maps.a, a_bf16, M, K) || !make_dense_map(&maps.b, b_bf16, N, K)) return BDR_ERR_CUDA;
     const int tiles_m = (int)(M / 256), tiles_n = (int)(N / 256);

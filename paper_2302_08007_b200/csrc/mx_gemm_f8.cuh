@@ -342,12 +342,11 @@ static F8Plan plan_gemm_f8(int64_t M, int64_t N, int64_t K) {
 // M, N multiples of 256, K a multiple of 128.  The tiles plan.tiles_full .. of C must hold zeros.
 static int launch_gemm_f8(const uint8_t* a_e4m3, const uint8_t* b_e4m3, const uint8_t* sf_a, const uint8_t* sf_b, int64_t M, int64_t N,
                           int64_t K, const F8Plan& plan, float* c, int64_t ldc, const int* gate, cudaStream_t st) {
-    static bool attr_done = false;
-    if (!attr_done) {
-        if (cudaFuncSetAttribute(mxf8_gemm_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kFSmemBytes) != cudaSuccess)
-            return BDR_ERR_CUDA;
-        attr_done = true;
-    }
+    static PerDevice once;
+    if (once.get(current_device(), [&]() -> int {  // no occupancy query: cluster kernel, one CTA per SM
+            return cudaFuncSetAttribute(mxf8_gemm_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kFSmemBytes) == cudaSuccess ? 1 : 0;
+        }) < 1)
+        return BDR_ERR_CUDA;
     F8Maps maps;
     if (!make_f8_map(&maps.a, a_e4m3, M, K) || !make_f8_map(&maps.b, b_e4m3, N, K)) return BDR_ERR_CUDA;
     // programmatic dependent launch: the kernel may start while the re-encoding kernel before it in the stream is

@@ -334,11 +334,11 @@ int launch_gemm_pair(const bdr_planes_t& a, const bdr_planes_t& b, int64_t M, in
                      const int* gate, cudaStream_t st) {
     auto kern = mx_gemm_pair_kernel<WA, WB>;
     const size_t smem = PairSmem<WA, WB>::kBytes;
-    static bool attr_done = false;
-    if (!attr_done) {
-        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return BDR_ERR_CUDA;
-        attr_done = true;
-    }
+    static PerDevice once;  // per instantiation
+    if (once.get(current_device(), [&]() -> int {  // no occupancy query: cluster kernel, one CTA per SM
+            return cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) == cudaSuccess ? 1 : 0;
+        }) < 1)
+        return BDR_ERR_CUDA;
     PairMaps maps;
     const bool ok = make_plane_map(&maps.a_elems, a.elems, M, K * WA / 8, a.ld_elems, ChunkPlanes<WA>::kElemRow) &&
                     make_plane_map(&maps.a_exps, a.exps, M, K / 16, a.ld_exps, 16) &&

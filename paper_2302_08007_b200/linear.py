@@ -71,6 +71,6 @@ def step(cfg: bdr.Config, x: torch.Tensor, w: torch.Tensor, dy: torch.Tensor, bu
 
 
 def qsnr_db(buf: LinearBuffers) -> dict:
-    s = buf.sums.cpu()
-    return {"%s_%s" % (n, "row" if ax == 1 else "col"): float(-10.0 * torch.log10(s[i, 0] / s[i, 1]))
-            for i, (n, ax) in enumerate(ORDER)}
+    """Eq. 3 of the six quantized operands, from the sums the last step accumulated."""
+    db = bdr.bdr_qsnr_from_sums(buf.sums, torch.empty(6, dtype=torch.float64, device=buf.sums.device)).cpu()
+    return {"%s_%s" % (n, "row" if ax == 1 else "col"): float(db[i]) for i, (n, ax) in enumerate(ORDER)}

@@ -64,3 +64,9 @@ def test_validation_happens_on_the_host():
     assert L.bdr_unpack(C.addressof(ok), None, dummy, 0, 1, 16, 16, 1, None) == -1
     with pytest.raises(bdr.BdrError):
         bdr.bdr_packed_sizes(bdr.Config(16, 8, 5, 1, 4), 4, 64)
+
+
+def test_per_device_launch_bookkeeping():
+    # kernel attributes are per device: the library keeps "set up" flags per device, not per process.  The
+    # self-test drives that bookkeeping with fake set-up functions for devices 0, 1, 2 and 63 (no CUDA call).
+    assert bdr.bdr_selftest_host() == 0

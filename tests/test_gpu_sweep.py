@@ -13,18 +13,18 @@ from tests import helpers as H
 pytestmark = pytest.mark.gpu
 
 
-def run_sweep(cfgs, x_host, dtype="f32", ld=None):
+def run_sweep(cfgs, x_host, dtype="f32", ld=None, axis=1):
     x = H.host_to_device(x_host, dtype, ld)
     out = torch.full((len(cfgs),), -1.0, dtype=torch.float64, device="cuda")
     ws = torch.empty(bdr.bdr_qsnr_workspace_bytes(len(cfgs)), dtype=torch.uint8, device="cuda")
-    bdr.bdr_qsnr(cfgs, x, out, ws)
+    bdr.bdr_qsnr(cfgs, x, out, ws, axis=axis)
     torch.cuda.synchronize()
     return out.cpu().numpy()
 
 
-def check(cfgs, got, x, what=""):
+def check(cfgs, got, x, what="", axis=1):
     for cfg, g in zip(cfgs, got):
-        want = orc.qsnr(H.to_orc(cfg), x)
+        want = orc.qsnr(H.to_orc(cfg), x, axis=axis)
         if math.isnan(want) or math.isinf(want):
             assert (math.isnan(g) and math.isnan(want)) or g == want, (what, cfg, g, want)
         else:
@@ -49,6 +49,27 @@ def test_sweep_ragged_rows_pitch_and_bf16():
     check(cfgs, run_sweep(cfgs, x, ld=5008), x, "ragged")
     xb = H.make_input("laplace_outliers", 3, 4096 + 512, "bf16", seed=4)
     check(cfgs, run_sweep(cfgs, xb, dtype="bf16"), xb, "bf16")
+
+
+def test_sweep_along_columns():
+    # axis 0: the lines are columns (the reduction dimension of half of a training step's operands, Section V);
+    # blocks, sub-blocks and VSQ vectors run down a column.  Every configuration against the oracle on a
+    # matrix whose outlier channels are columns, then ragged shapes with a pitch, bf16, and columns longer
+    # than one 4096-element tile.
+    cfgs = [c for _, c in sweep.sweep_configs()]
+    x = synth.outlier_channel_matrix(1024, 64, seed=11, gain=50.0)
+    got = run_sweep(cfgs, x, axis=0)
+    check(cfgs, got, x, "columns", axis=0)
+    rows_dir = run_sweep(cfgs, x, axis=1)
+    assert np.abs(got[:441] - rows_dir[:441]).max() > 0.1       # the direction matters on this input
+    some = cfgs[::7] + [c for _, c in sweep.comparators()]
+    xr = synth.normal_with_outliers(5000 * 7, seed=12).reshape(5000, 7)   # 5000 is not a multiple of 16; 2 tiles per column
+    check(some, run_sweep(some, xr, ld=12, axis=0), xr, "ragged columns", axis=0)
+    xb = H.make_input("laplace_outliers", 4096 + 512, 6, "bf16", seed=13)
+    check(some, run_sweep(some, xb, dtype="bf16", axis=0), xb, "bf16 columns", axis=0)
+    one = synth.normal(777, 14).reshape(777, 1)
+    check(some, run_sweep(some, one, axis=0), one, "single column", axis=0)
+    check(some, run_sweep(some, one.reshape(1, 777), axis=0), one.reshape(1, 777), "columns of one element", axis=0)
 
 
 def test_sweep_extra_configs_edge_values_and_ties_away():
@@ -79,8 +100,8 @@ def test_sweep_degenerate_tensors_and_errors():
     assert e.value.status == -6
     ws = torch.empty(bdr.bdr_qsnr_workspace_bytes(1), dtype=torch.uint8, device="cuda")
     with pytest.raises(bdr.BdrError) as e:
-        bdr.bdr_qsnr([bdr.MX6], x, out, ws, axis=0)
-    assert e.value.status == -3
+        bdr.bdr_qsnr([bdr.MX6], x, out, ws, axis=2)
+    assert e.value.status == -2
     with pytest.raises(bdr.BdrError) as e:
         bdr.bdr_qsnr([bdr.Config(16, 8, 3, 1, 4)], x, out, ws)
     assert e.value.status == -2

@@ -385,6 +385,58 @@ def test_fp8_casts_match_library_casts():
     assert orc.minifloat_round(np.array([1e9], dtype=np.float32), 5, 2).tolist() == [57344.0]
 
 
+def test_minifloat_rounding_by_nearest_value_search_over_the_explicit_code_set():
+    # every (exponent bits, mantissa bits) shape the FP32_FP kind accepts, not only the two FP8 formats that have a
+    # library cast: enumerate the format's finite values (bias 2^(eb-1)-1, gradual underflow, top exponent
+    # reserved as in IEEE -- except E4M3, whose top exponent is finite up to 448), then find the nearest one to
+    # each input with exact rationals; ties go to the even mantissa code (or away from zero); beyond the largest
+    # value the cast saturates.
+    for eb, mb in ((2, 1), (3, 2), (2, 3), (4, 3), (5, 2), (3, 4), (4, 1), (5, 7)):
+        bias = (1 << (eb - 1)) - 1
+        codes = []                                                   # (value, mantissa code) in ascending order
+        top = (1 << eb) - 1 if (eb, mb) != (4, 3) else (1 << eb)
+        for e in range(0, top):
+            for f in range(1 << mb):
+                if (eb, mb) == (4, 3) and e == 15 and f == 7:
+                    continue                                          # the one NaN code of E4M3
+                val = Fraction(f, 1 << mb) * Fraction(2) ** (1 - bias) if e == 0 else \
+                    (1 + Fraction(f, 1 << mb)) * Fraction(2) ** (e - bias)
+                codes.append((val, f))
+        vals = [v for v, _ in codes]
+        assert vals == sorted(vals) and len(set(vals)) == len(vals)
+        fmax = vals[-1]
+        if (eb, mb) == (4, 3):
+            assert fmax == 448
+        if (eb, mb) == (5, 2):
+            assert fmax == 57344
+        rng = np.random.default_rng(1000 + 10 * eb + mb)
+        xs = np.concatenate([
+            rng.normal(size=300).astype(np.float32) * np.float32(float(fmax) / 3),
+            (rng.normal(size=300) * float(vals[1 << mb]) * 2).astype(np.float32),      # around the subnormal range
+            np.array([float((a + b) / 2) for (a, _), (b, _) in zip(codes[:-1], codes[1:])], dtype=np.float32),  # exact ties
+            np.array([float(fmax) * 1.5, -float(fmax) * 4, 0.0, float(vals[1]) / 2, float(vals[1]) / 4], dtype=np.float32)])
+        for rnd in (orc.RNE, orc.RNA):
+            got = orc.minifloat_round(xs, eb, mb, rnd)
+            for x, g in zip(xs.tolist(), got.tolist()):
+                a = abs(Fraction(x))
+                if a >= fmax:
+                    want = fmax
+                else:
+                    import bisect
+                    hi = bisect.bisect_right(vals, a)                 # vals[hi-1] <= a < vals[hi]
+                    lo_v, hi_v = vals[hi - 1], vals[hi]
+                    if a - lo_v < hi_v - a:
+                        want = lo_v
+                    elif a - lo_v > hi_v - a:
+                        want = hi_v
+                    elif rnd == orc.RNA:
+                        want = hi_v
+                    else:
+                        want = lo_v if codes[hi - 1][1] % 2 == 0 else hi_v
+                assert Fraction(abs(g)) == want, (eb, mb, rnd, x, g, float(want))
+                assert math.copysign(1, g) == math.copysign(1, x)
+
+
 def test_fp8_kind_is_scale_then_cast():
     import torch
     x = synth.normal(4096, 72)
