@@ -127,6 +127,20 @@ int bdr_pack(const bdr_config_t* cfg /*host*/, const void* x, bdr_dtype_t dt, in
              int64_t ld, int axis, const bdr_planes_t* out /*host struct of device pointers*/, void* y_dq,
              double* qsnr_sums_dev, void* stream);
 
+/* bdr_pack along both directions at once: out_rows receives exactly what bdr_pack(axis = 1) writes and out_cols
+ * exactly what bdr_pack(axis = 0) writes (the planes of the transposed tensor), from ONE read of x.  Section V,
+ * Fig. 8: every tensor of a training step is an operand of one matrix product in the forward pass and of one in
+ * the backward pass, reduced over different dimensions, so it is quantized along both ("transpose, then quantize"
+ * for the second copy).  The optional sums are those of bdr_pack for the two directions (each 2 doubles, added to;
+ * pass both or neither for the single-read kernel).
+ * Single-read kernel: bf16, Table II formats (k1 = 16, k2 = 2, d2 = 1, m in {2, 4, 7}), ties-to-even, rows a
+ * multiple of 256, cols a multiple of 256, 16-byte aligned rows, planes with their natural pitches; its algorithmic
+ * traffic is 2 + 2 bits/8 bytes per element against 2 (2 + bits/8) for two calls.  Anything else is served by one
+ * pass per direction, with the same bytes as result. */
+int bdr_pack2(const bdr_config_t* cfg /*host*/, const void* x, bdr_dtype_t dt, int64_t rows, int64_t cols, int64_t ld,
+              const bdr_planes_t* out_rows /*host struct*/, const bdr_planes_t* out_cols /*host struct*/,
+              double* qsnr_sums_rows_dev, double* qsnr_sums_cols_dev, void* stream);
+
 /* Decode packed planes to values (-1)^s * q * 2^(F-127-tau-(m-1)) of dtype `dt` in a [rows, ld]
  * tensor; the inverse of bdr_pack's planes -> Q(x). */
 int bdr_unpack(const bdr_config_t* cfg /*host*/, const bdr_planes_t* in /*host struct*/, void* y, bdr_dtype_t dt,

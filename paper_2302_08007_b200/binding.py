@@ -22,7 +22,7 @@ F32, BF16 = 0, 1
 EXPORTS = ("bdr_strerror", "bdr_device_status", "bdr_packed_sizes", "bdr_quant_dequant", "bdr_pack", "bdr_unpack",
            "bdr_qsnr_workspace_bytes", "bdr_qsnr", "bdr_qsnr_static_max_cfgs", "bdr_qsnr_static", "mx_gemm",
            "mx_gemm_workspace_bytes", "mx_gemm_ws", "mx_gemm_f8_workspace_bytes", "mx_gemm_f8", "bdr_reencode_e4m3", "mx_gemm_e4m3", "bdr_set_workspace",
-           "mx_gemm_status", "bdr_selftest_bounded_wait", "bdr_selftest_host", "bdr_qsnr_from_sums")
+           "mx_gemm_status", "bdr_selftest_bounded_wait", "bdr_selftest_host", "bdr_qsnr_from_sums", "bdr_pack2")
 
 
 class BdrError(RuntimeError):
@@ -93,6 +93,9 @@ def lib():
                                C.c_void_p, C.c_void_p, C.c_void_p]
         L.bdr_unpack.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int64, C.c_int64, C.c_int64, C.c_int,
                                  C.c_void_p]
+        L.bdr_pack2.restype = C.c_int
+        L.bdr_pack2.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int64, C.c_int64, C.c_int64, C.c_void_p, C.c_void_p,
+                                C.c_void_p, C.c_void_p, C.c_void_p]
         L.bdr_qsnr_workspace_bytes.restype = C.c_int64
         L.bdr_qsnr_workspace_bytes.argtypes = [C.c_int]
         L.bdr_qsnr.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_int, C.c_int64, C.c_int64, C.c_int64, C.c_int,
@@ -211,6 +214,16 @@ def bdr_pack(cfg: Config, x: torch.Tensor, planes: Planes, axis: int = 1, y_dq: 
     _check(lib().bdr_pack(C.addressof(c), _ptr(x2), _dt(x2), x2.shape[0], x2.shape[1], x2.stride(0), axis,
                           C.addressof(p), _ptr(y2), _ptr(qsnr_sums), _stream(stream)), "bdr_pack")
     return planes
+
+
+def bdr_pack2(cfg: Config, x: torch.Tensor, planes_rows: Planes, planes_cols: Planes, qsnr_sums_rows: torch.Tensor | None = None,
+              qsnr_sums_cols: torch.Tensor | None = None, stream=None):
+    """Both packed copies of x -- quantized along its rows (axis 1) and along its columns (axis 0) -- from one read."""
+    x2 = _as2d(x)
+    c, pr, pc = cfg.c(), planes_rows.c(), planes_cols.c()
+    _check(lib().bdr_pack2(C.addressof(c), _ptr(x2), _dt(x2), x2.shape[0], x2.shape[1], x2.stride(0), C.addressof(pr),
+                           C.addressof(pc), _ptr(qsnr_sums_rows), _ptr(qsnr_sums_cols), _stream(stream)), "bdr_pack2")
+    return planes_rows, planes_cols
 
 
 def bdr_unpack(cfg: Config, planes: Planes, y: torch.Tensor, axis: int = 1, stream=None) -> torch.Tensor:

@@ -259,6 +259,34 @@ int bdr_pack(const bdr_config_t* cfg, const void* x, bdr_dtype_t dt, int64_t row
                                          tight, qsnr_sums_dev, st);
 }
 
+int bdr_pack2(const bdr_config_t* cfg, const void* x, bdr_dtype_t dt, int64_t rows, int64_t cols, int64_t ld,
+              const bdr_planes_t* out_rows, const bdr_planes_t* out_cols, double* qsnr_sums_rows_dev, double* qsnr_sums_cols_dev,
+              void* stream) {
+    QParams qp;
+    int rc = check_pow2_config(cfg, &qp);
+    if (rc) return rc;
+    if ((rc = check_tensor(x, dt, rows, cols, ld, 1))) return rc;
+    if (rows == 0 || cols == 0) return BDR_OK;
+    if ((rc = check_planes(cfg, out_rows, cols))) return rc;
+    if ((rc = check_planes(cfg, out_cols, rows))) return rc;
+    if ((qsnr_sums_rows_dev && (uintptr_t)qsnr_sums_rows_dev % 8) || (qsnr_sums_cols_dev && (uintptr_t)qsnr_sums_cols_dev % 8)) return BDR_ERR_MISALIGNED;
+    const bool tight_r = planes_tight(cfg, out_rows, cols), tight_c = planes_tight(cfg, out_cols, rows);
+    cudaStream_t st = (cudaStream_t)stream;
+    if (dt == BDR_BF16 && tight_r && tight_c) {
+        rc = pack2_mx_x2((const __nv_bfloat16*)x, rows, cols, ld, *out_rows, *out_cols, qp, qsnr_sums_rows_dev, qsnr_sums_cols_dev, st);
+        if (rc != BDR_ERR_UNSUPPORTED) return rc;
+    }
+    // any other shape, dtype or configuration: one pass per direction (the same bytes, the tensor is read twice)
+    if (dt == BDR_F32) {
+        rc = quant_dispatch<float>(qp, (const float*)x, nullptr, rows, cols, ld, 1, out_rows, tight_r, qsnr_sums_rows_dev, st);
+        if (rc) return rc;
+        return quant_dispatch<float>(qp, (const float*)x, nullptr, rows, cols, ld, 0, out_cols, tight_c, qsnr_sums_cols_dev, st);
+    }
+    rc = quant_dispatch<__nv_bfloat16>(qp, (const __nv_bfloat16*)x, nullptr, rows, cols, ld, 1, out_rows, tight_r, qsnr_sums_rows_dev, st);
+    if (rc) return rc;
+    return quant_dispatch<__nv_bfloat16>(qp, (const __nv_bfloat16*)x, nullptr, rows, cols, ld, 0, out_cols, tight_c, qsnr_sums_cols_dev, st);
+}
+
 int bdr_unpack(const bdr_config_t* cfg, const bdr_planes_t* in, void* y, bdr_dtype_t dt, int64_t rows, int64_t cols,
                int64_t ld, int axis, void* stream) {
     QParams qp;

@@ -75,6 +75,10 @@ int quant_colwise_qd_x2(const __nv_bfloat16* x, __nv_bfloat16* y, int64_t rows, 
 int quant_colwise_mx_x2(const __nv_bfloat16* x, __nv_bfloat16* y, int64_t rows, int64_t cols, int64_t ld,
                         const bdr_planes_t* out, const QParams& qp, double* sums, cudaStream_t st);  // bdr_col_x2.cu
 
+// both directions from one read of the tensor (bdr_pack2_x2.cu)
+int pack2_mx_x2(const __nv_bfloat16* x, int64_t rows, int64_t cols, int64_t ld, const bdr_planes_t& rout, const bdr_planes_t& cout_,
+                const QParams& qp, double* sums_row, double* sums_col, cudaStream_t st);
+
 // axis-0 fast path for k1 = 16, k2 = 2 (bdr_col.cu)
 template <typename T>
 int quant_colwise_mx(const T* x, T* y, int64_t rows, int64_t cols, int64_t ld, const bdr_planes_t* out,

@@ -47,13 +47,13 @@ def alloc(cfg: bdr.Config, tokens: int, d_in: int, d_out: int, device="cuda", tw
 
 
 def step(cfg: bdr.Config, x: torch.Tensor, w: torch.Tensor, dy: torch.Tensor, buf: LinearBuffers, stream=None):
-    """Six quantizations (with fused QSNR sums) and three MX GEMMs.  Returns (Y, dX, dW)."""
+    """Six quantizations (three dual-direction calls, with fused QSNR sums) and three MX GEMMs.  Returns (Y, dX, dW)."""
     tokens, d_in = x.shape
     d_out = w.shape[0]
     src = {"x": x, "w": w, "dy": dy}
     buf.sums.zero_()
-    for i, (n, ax) in enumerate(ORDER):
-        bdr.bdr_pack(cfg, src[n], buf.planes[(n, ax)], axis=ax, qsnr_sums=buf.sums[i], stream=stream)
+    for i, n in enumerate(("x", "w", "dy")):   # each tensor is read once and packed along both directions
+        bdr.bdr_pack2(cfg, src[n], buf.planes[(n, 1)], buf.planes[(n, 0)], buf.sums[2 * i], buf.sums[2 * i + 1], stream=stream)
     p = buf.planes
 
     def gemm(a, b, M, N, K, c):
