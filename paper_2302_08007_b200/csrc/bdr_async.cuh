@@ -127,8 +127,10 @@ __device__ __forceinline__ void report_timeout(int* status) { atomicCAS(status, 
 
 // cuTensorMapEncodeTiled for a row-major [rows, cols] matrix of 16-bit elements with a pitch of ld elements and
 // a box of box_cols x box_rows (host; bdr_api.cu).  The library does not link libcuda: the entry point
-// comes from the runtime.  False if the driver refuses the map.
-bool make_tensor_map_u16(CUtensorMap* out, const void* base, int64_t rows, int64_t cols, int64_t ld, int box_cols, int box_rows);
+// comes from the runtime.  False if the driver refuses the map.  swizzle128 (box rows of exactly 128 bytes): the
+// 16-byte chunk c of box row r lands at chunk c ^ (r & 7) of that row in shared memory (destination 1 KB aligned).
+bool make_tensor_map_u16(CUtensorMap* out, const void* base, int64_t rows, int64_t cols, int64_t ld, int box_cols, int box_rows,
+                         bool swizzle128 = false);
 
 // Device address of the library's sticky status word on the current device (host; bdr_api.cu).
 int* device_status_word();

@@ -5,8 +5,9 @@
 // each reducing over a different dimension, so each tensor is quantized along both.
 //
 // A CTA of eight warps owns tiles of 256 rows x 128 columns; warp w takes block rows 2w and 2w+1 of a tile,
-// each a box of 16 rows x 128 columns (4 KB) fetched with one 2-D TMA tile load into the warp's own ring.
-// A box is used twice while it sits in shared memory:
+// each a box of 16 rows x 128 columns (4 KB) fetched as two 2-D TMA tile loads of 64 columns (128-byte rows,
+// 128-byte swizzle: 16-byte chunk c of row r sits at chunk c ^ (r & 7), which makes both access patterns below
+// free of bank conflicts) into the warp's own ring.  A box is used twice while it sits in shared memory:
 //   * column direction: a lane owns four adjacent columns (8 bytes of every row) = two word columns, i.e. four
 //     blocks of 16 rows; codes are staged per tile as [block-row pair][column] items and, after a CTA barrier,
 //     each column's 16 blocks leave as one contiguous run of the column-major planes;
@@ -59,7 +60,7 @@ pack2_x2_kernel(const __grid_constant__ CUtensorMap xmap, int n_col_tiles, int n
     constexpr int NCW = (16 * W + 31) / 32;
     constexpr int S = kP2Stages;
     constexpr int M = W - 1;
-    extern __shared__ __align__(128) uint8_t smem[];  // ring [warp][stage][4 KB], barriers, column staging, row staging
+    extern __shared__ __align__(1024) uint8_t smem[];  // ring [warp][stage][4 KB] (1 KB aligned: swizzle atoms), barriers, column staging, row staging
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const uint32_t ring0 = async::smem_u32(smem) + warp * S * kP2BoxBytes;
     const uint32_t bars = async::smem_u32(smem) + kP2RingBytes + warp * 32;
@@ -71,7 +72,9 @@ pack2_x2_kernel(const __grid_constant__ CUtensorMap xmap, int n_col_tiles, int n
     auto issue = [&](int t, int i, int stg) {  // lane 0 only: box i of tile t into stage stg
         const int rt = t / n_col_tiles, ct = t - rt * n_col_tiles;
         async::mbar_expect_tx(bars + 8 * stg, kP2BoxBytes);
-        async::tma_load_2d(ring0 + stg * kP2BoxBytes, &xmap, ct * kP2TileCols, rt * kP2TileRows + (2 * warp + i) * kSlice, bars + 8 * stg);
+        const int row0 = rt * kP2TileRows + (2 * warp + i) * kSlice;
+        async::tma_load_2d(ring0 + stg * kP2BoxBytes, &xmap, ct * kP2TileCols, row0, bars + 8 * stg);
+        async::tma_load_2d(ring0 + stg * kP2BoxBytes + kP2BoxBytes / 2, &xmap, ct * kP2TileCols + kP2TileCols / 2, row0, bars + 8 * stg);
     };
     if (lane == 0) {
 #pragma unroll
@@ -100,13 +103,27 @@ pack2_x2_kernel(const __grid_constant__ CUtensorMap xmap, int n_col_tiles, int n
             const uint32_t box = ring0 + stg * kP2BoxBytes;
             // ---- column direction: the lane's two word columns ------------------------------------------------
             {
-                const uint32_t mine = box + lane * 8;
+                // the lane's 8 bytes of row r: half box lane / 16, chunk (lane % 16) / 2 of the row, swizzled by the row
+                const uint32_t mine = box + (lane >> 4) * (kP2BoxBytes / 2) + (lane & 1) * 8;
+                const uint32_t chunk = ((lane & 15) >> 1) << 4;
                 uint32_t Fb[4], Mb[4];
+                [[maybe_unused]] uint32_t wboth[2][16];
+                if constexpr (!SUMS) {  // both word columns with one load per row (the sums variant has no registers to spare)
+#pragma unroll
+                    for (int r = 0; r < kSlice; ++r) {
+                        const uint2 v2 = async::lds64(mine + r * 128 + (chunk ^ ((r & 7) << 4)));
+                        wboth[0][r] = v2.x;
+                        wboth[1][r] = v2.y;
+                    }
+                }
 #pragma unroll
                 for (int c = 0; c < 2; ++c) {
                     uint32_t wc[16];
 #pragma unroll
-                    for (int r = 0; r < kSlice; ++r) wc[r] = async::lds32(mine + 4 * c + r * (kP2TileCols * 2));
+                    for (int r = 0; r < kSlice; ++r) {
+                        if constexpr (!SUMS) wc[r] = wboth[c][r];
+                        else wc[r] = async::lds32(mine + 4 * c + r * 128 + (chunk ^ ((r & 7) << 4)));
+                    }
                     uint32_t aw[16], pm[8], yw[16], cl[NCW], ch[NCW], F2;
                     x2::WordColOut o;
                     if (x2::wordcol_exponents(wc, aw, pm, F2)) {
@@ -167,10 +184,11 @@ pack2_x2_kernel(const __grid_constant__ CUtensorMap xmap, int n_col_tiles, int n
 #pragma unroll
             for (int k = 0; k < 2; ++k) {
                 const int it = lane + 32 * k, row = it >> 2, pair = it & 3;
-                const uint32_t src = box + row * (kP2TileCols * 2) + pair * 64;
+                const uint32_t src = box + (pair >> 1) * (kP2BoxBytes / 2) + row * 128;
+                const uint32_t c0 = (uint32_t)(pair & 1) << 6, sw = (uint32_t)(row & 7) << 4;
                 uint4 v[4];
 #pragma unroll
-                for (int g = 0; g < 4; ++g) v[g] = async::lds128(src + 16 * g);
+                for (int g = 0; g < 4; ++g) v[g] = async::lds128(src + ((c0 + 16 * g) ^ sw));
                 if (k == 1) {
                     __syncwarp();  // every lane has read the box for the last time: refill the stage with box i of the next tile
                     if (lane == 0 && !failed && t + (int)gridDim.x < n_tiles) issue(t + gridDim.x, i, stg);
@@ -291,7 +309,7 @@ static int launch_pack2(const bf16* x, int64_t rows, int64_t cols, int64_t ld, c
     int* status = device_status_word();
     if (!status) return BDR_ERR_CUDA;
     CUtensorMap xmap;
-    if (!make_tensor_map_u16(&xmap, x, rows, cols, ld, kP2TileCols, kSlice)) return BDR_ERR_CUDA;
+    if (!make_tensor_map_u16(&xmap, x, rows, cols, ld, kP2TileCols / 2, kSlice, true)) return BDR_ERR_CUDA;
     const int n_ct = (int)(cols / kP2TileCols);
     const int64_t n_tiles = (int64_t)n_ct * (rows / kP2TileRows);
     const int grid = (int)std::min<int64_t>(n_tiles, (int64_t)sm_count() * blocks_per_sm);
