@@ -305,3 +305,45 @@ def run_only(a) -> None:
     ms = _time(once, reps)
     print("%s %s axis=%d %s %dx%d: %.4f ms per launch, status %d" % (a.only, a.fmt, a.axis, a.dtype, a.rows, a.cols, ms,
                                                                    bdr.bdr_device_status()))
+
+
+def paper_sweep_leg(args) -> dict:
+    """Section IV-B/C as the paper sets it up: 16,384 vectors of 1,024 values ~ N(0, |N(0,1)|) (one variance per vector),
+    the 457 configurations, the FP32 kinds scaled by the maximum over a window of past chunks (delayed scaling), and the
+    QSNR-versus-cost frontier with cost = bits per element / packing efficiency of a 256-element tile in 64-byte lines."""
+    n_vec, length, chunks, window = 16384, 1024, 8, 4
+    named = sweep.sweep_configs()
+    cfgs = [c for _, c in named]
+    x = torch.from_numpy(synth.variable_variance_vectors(n_vec, length, seed=0)).cuda()
+    out = torch.empty(len(cfgs), dtype=torch.float64, device="cuda")
+    ws = torch.empty(bdr.bdr_qsnr_workspace_bytes(len(cfgs)), dtype=torch.uint8, device="cuda")
+    ms = _time(lambda: bdr.bdr_qsnr(cfgs, x, out, ws), reps=3)
+    q_now = out.cpu().numpy().copy()
+    # delayed scaling: chunk t is quantized with the largest maximum of chunks t - window .. t - 1
+    per = n_vec // chunks
+    hist = torch.zeros(chunks, dtype=torch.float32, device="cuda")
+    for t in range(chunks):
+        bdr.bdr_amax(x[t * per:(t + 1) * per], hist[t:t + 1])
+    comp = [c for _, c in sweep.comparators()]
+    outc = torch.empty(len(comp), dtype=torch.float64, device="cuda")
+    wsc = torch.empty(bdr.bdr_qsnr_workspace_bytes(len(comp)), dtype=torch.uint8, device="cuda")
+    delayed = np.zeros(len(comp))
+    for t in range(1, chunks):
+        bdr.bdr_qsnr_delayed(comp, x[t * per:(t + 1) * per], hist[max(0, t - window):t], outc, wsc)
+        delayed += outc.cpu().numpy()
+    delayed /= chunks - 1                                  # mean of per-chunk dB, as the paper averages per-vector QSNR
+    q = q_now.copy()
+    q[441:] = delayed
+    pts = [(n, sweep.bits_per_element(c) / bdr.bdr_tile_packing_efficiency(c), float(v)) for (n, c), v in zip(named, q)]
+    front = sweep.pareto_frontier(pts)
+    names = [n for n, _ in named]
+    show = {"MX9": "bdr_k1=16_k2=2_d2=1_m=7", "MX6": "bdr_k1=16_k2=2_d2=1_m=4", "MX4": "bdr_k1=16_k2=2_d2=1_m=2",
+            "MSFP16": "bdr_k1=16_k2=1_d2=0_m=7", "MSFP12": "bdr_k1=16_k2=1_d2=0_m=3", "INT8": "int8", "FP8_E4M3": "fp8_e4m3",
+            "FP8_E5M2": "fp8_e5m2"}
+    return {"paper_sweep": {"workload": "16,384 x 1,024 fp32 ~ N(0,|N(0,1)|), 457 configurations in one bdr_qsnr call",
+                            "ms": ms, "configs_per_s": len(cfgs) / (ms * 1e-3),
+                            "qsnr_db": {k: float(q[names.index(v)]) for k, v in show.items()},
+                            "qsnr_db_current_amax": {k: float(q_now[names.index(v)]) for k, v in show.items() if names.index(v) >= 441},
+                            "delayed_scaling": "FP32 kinds: maximum over the %d previous chunks of %d vectors, mean of per-chunk dB" % (window, per),
+                            "packing_efficiency_256_in_64B": {k: bdr.bdr_tile_packing_efficiency(cfgs[names.index(v)]) for k, v in show.items()},
+                            "frontier": [{"name": n, "bits_over_packing_efficiency": c, "qsnr_db": v} for n, c, v in front]}}

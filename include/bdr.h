@@ -173,6 +173,24 @@ int bdr_qsnr(const bdr_config_t* cfgs /*host*/, int n_cfgs, const void* x, bdr_d
              int64_t cols, int64_t ld, int axis, double* qsnr_db_dev, void* workspace, int64_t workspace_bytes,
              void* stream);
 
+/* The sweep with a first-level maximum that comes from elsewhere (Section IV-B, Fig. 7 caption: the INT, FP and VSQ
+ * points take their FP32 first-level scale from the absolute maximum over a window of PAST vectors, "delayed
+ * scaling").  amax_window_dev holds n_window >= 1 non-negative floats on the device (the maxima of earlier tensors,
+ * e.g. written by bdr_amax); the FP32_* entries derive their scale from the largest of them instead of from x, and
+ * values of x beyond it saturate at the top code.  POW2 entries are unaffected.  Everything else as bdr_qsnr. */
+int bdr_qsnr_delayed(const bdr_config_t* cfgs /*host*/, int n_cfgs, const void* x, bdr_dtype_t dt, int64_t rows,
+                     int64_t cols, int64_t ld, int axis, const float* amax_window_dev, int n_window,
+                     double* qsnr_db_dev, void* workspace, int64_t workspace_bytes, void* stream);
+
+/* Eq. 1's maximum: *amax_dev = max(*amax_dev, max |x|) over a [rows, ld] tensor (one float on the device; the
+ * caller zeroes it, or leaves an earlier maximum in it to extend a window). */
+int bdr_amax(const void* x, bdr_dtype_t dt, int64_t rows, int64_t cols, int64_t ld, float* amax_dev, void* stream);
+
+/* Section IV-B, memory footprint (host only): the fraction of the fetched bits that are payload when a tile of
+ * tile_elems elements ((m+1) + d1/k1 + d2/k2 bits each, Section III) is stored in whole memory lines of line_bytes
+ * bytes; the paper's setting is a 256-element tile and a 64-byte interface.  Negative for a bad argument. */
+double bdr_tile_packing_efficiency(const bdr_config_t* cfg /*host*/, int64_t tile_elems, int64_t line_bytes);
+
 /* The same sweep as bdr_qsnr for callers that cannot hand over scratch memory.  (The paper has no
  * counterpart; this is a convenience of this library.)  Think of a monitoring hook that runs inside
  * another framework's training step, or a serving loop with a fixed memory plan: all device memory

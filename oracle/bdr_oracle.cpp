@@ -374,13 +374,19 @@ double orc_qsnr_db(double err2, double sig2) {
 // Quantize-dequantize.  x, y: fp32 [rows, ld] row-major (only cols columns used).  sums (nullable)
 // receives {sum (Q-x)^2, sum x^2} in fp64 over the tensor.  nthreads > 1 splits lines over
 // std::threads (the blocks are independent); the arithmetic is the same.
-int orc_quant_dequant_mt(const orc_config* c, const float* x, float* y, int64_t rows, int64_t cols, int64_t ld,
-                         int axis, double* sums, int alt, int nthreads) {
+// first_level_amax (nullable): for the FP32-scaled kinds with one scale per tensor (k1 = 0), the maximum that
+// the first-level scale is derived from when it does not come from the tensor itself -- Section IV-B, Fig. 7
+// caption: the INT / FP / VSQ points use the absolute maximum over a window of PAST vectors ("delayed
+// scaling"); values beyond it saturate at the top code.  NULL: the current tensor's own maximum.
+static int quant_dequant_impl(const orc_config* c, const float* x, float* y, int64_t rows, int64_t cols, int64_t ld,
+                              int axis, double* sums, int alt, int nthreads, const float* first_level_amax) {
     if (!config_ok(c) || !x || !y || rows < 0 || cols < 0 || ld < cols || (axis != 0 && axis != 1)) return ORC_BAD;
     if (alt && c->scale_kind != ORC_POW2) return ORC_BAD;
+    if (first_level_amax && (c->scale_kind == ORC_POW2 || c->k1 != 0 || !(*first_level_amax >= 0.f))) return ORC_BAD;
     LineView v = make_view(rows, cols, ld, axis);
     float tensor_amax = 0.f;
-    if (c->scale_kind != ORC_POW2 && c->k1 == 0)
+    if (first_level_amax) tensor_amax = *first_level_amax;
+    else if (c->scale_kind != ORC_POW2 && c->k1 == 0)
         for (int64_t r = 0; r < rows; ++r) tensor_amax = std::fmax(tensor_amax, absmax(x + r * ld, 1, cols));
     if (nthreads <= 1) {
         quantize_lines(*c, x, y, v, 0, v.nlines, tensor_amax, alt != 0);
@@ -406,6 +412,27 @@ int orc_quant_dequant_mt(const orc_config* c, const float* x, float* y, int64_t 
         sums[1] = s2;
     }
     return ORC_OK;
+}
+
+int orc_quant_dequant_mt(const orc_config* c, const float* x, float* y, int64_t rows, int64_t cols, int64_t ld,
+                         int axis, double* sums, int alt, int nthreads) {
+    return quant_dequant_impl(c, x, y, rows, cols, ld, axis, sums, alt, nthreads, nullptr);
+}
+
+int orc_quant_dequant_scaled(const orc_config* c, const float* x, float* y, int64_t rows, int64_t cols, int64_t ld,
+                             int axis, double* sums, float first_level_amax, int nthreads) {
+    return quant_dequant_impl(c, x, y, rows, cols, ld, axis, sums, 0, nthreads, &first_level_amax);
+}
+
+// Section IV-B, memory footprint: how well a tile of `tile_elems` elements packs into memory lines of
+// `line_bytes` bytes -- the tile's bits (bits per element of Section III x elements) over the bits of the
+// whole lines it occupies.
+double orc_tile_packing_efficiency(const orc_config* c, int64_t tile_elems, int64_t line_bytes) {
+    if (!config_ok(c) || tile_elems < 1 || line_bytes < 1) return -1.0;
+    const double bits = orc_bits_per_element(c) * (double)tile_elems;
+    const double line_bits = 8.0 * (double)line_bytes;
+    const double lines = std::ceil(bits / line_bits);
+    return bits / (lines * line_bits);
 }
 
 int orc_quant_dequant(const orc_config* c, const float* x, float* y, int64_t rows, int64_t cols, int64_t ld,

@@ -67,6 +67,8 @@ def lib():
         _lib.orc_theorem1_bound_db.argtypes = [C.c_void_p, C.c_int64]
         _lib.orc_qsnr_db.restype = C.c_double
         _lib.orc_qsnr_db.argtypes = [C.c_double, C.c_double]
+        _lib.orc_tile_packing_efficiency.restype = C.c_double
+        _lib.orc_tile_packing_efficiency.argtypes = [C.c_void_p, C.c_int64, C.c_int64]
     return _lib
 
 
@@ -102,23 +104,33 @@ def config_check(cfg: Config) -> int:
     return lib().orc_config_check(C.byref(c))
 
 
-def quant_dequant(cfg: Config, x, axis: int = 1, alt: bool = False, nthreads: int = 1):
-    """Returns (y fp32 with x's 2-D shape, (sum_err2, sum_sig2))."""
+def tile_packing_efficiency(cfg: Config, tile_elems: int = 256, line_bytes: int = 64) -> float:
+    c = cfg.c()
+    return lib().orc_tile_packing_efficiency(C.cast(C.byref(c), C.c_void_p), tile_elems, line_bytes)
+
+
+def quant_dequant(cfg: Config, x, axis: int = 1, alt: bool = False, nthreads: int = 1, amax: float | None = None):
+    """Returns (y fp32 with x's 2-D shape, (sum_err2, sum_sig2)).  amax: the first-level maximum of the FP32-scaled
+    kinds when it comes from elsewhere (a window of past tensors) instead of from x itself."""
     x = _f32(x)
     x2 = x.reshape(1, -1) if x.ndim == 1 else x
     rows, cols = x2.shape
     y = np.empty_like(x2)
     sums = np.zeros(2, dtype=np.float64)
     c = cfg.c()
-    rc = lib().orc_quant_dequant_mt(C.byref(c), _p(x2), _p(y), _i64(rows), _i64(cols), _i64(cols), C.c_int(axis),
-                                    _p(sums), C.c_int(int(alt)), C.c_int(nthreads))
+    if amax is not None:
+        rc = lib().orc_quant_dequant_scaled(C.byref(c), _p(x2), _p(y), _i64(rows), _i64(cols), _i64(cols), C.c_int(axis),
+                                            _p(sums), C.c_float(float(amax)), C.c_int(nthreads))
+    else:
+        rc = lib().orc_quant_dequant_mt(C.byref(c), _p(x2), _p(y), _i64(rows), _i64(cols), _i64(cols), C.c_int(axis),
+                                            _p(sums), C.c_int(int(alt)), C.c_int(nthreads))
     if rc != 0:
         raise ValueError("oracle rejected the configuration or arguments")
     return y.reshape(x.shape), (float(sums[0]), float(sums[1]))
 
 
-def qsnr(cfg: Config, x, axis: int = 1, nthreads: int = 1) -> float:
-    _, (e2, s2) = quant_dequant(cfg, x, axis, nthreads=nthreads)
+def qsnr(cfg: Config, x, axis: int = 1, nthreads: int = 1, amax: float | None = None) -> float:
+    _, (e2, s2) = quant_dequant(cfg, x, axis, nthreads=nthreads, amax=amax)
     return qsnr_db(e2, s2)
 
 

@@ -22,7 +22,7 @@ F32, BF16 = 0, 1
 EXPORTS = ("bdr_strerror", "bdr_device_status", "bdr_packed_sizes", "bdr_quant_dequant", "bdr_pack", "bdr_unpack",
            "bdr_qsnr_workspace_bytes", "bdr_qsnr", "bdr_qsnr_static_max_cfgs", "bdr_qsnr_static", "mx_gemm",
            "mx_gemm_workspace_bytes", "mx_gemm_ws", "mx_gemm_f8_workspace_bytes", "mx_gemm_f8", "bdr_reencode_e4m3", "mx_gemm_e4m3", "bdr_set_workspace",
-           "mx_gemm_status", "bdr_selftest_bounded_wait", "bdr_selftest_host", "bdr_qsnr_from_sums", "bdr_pack2")
+           "mx_gemm_status", "bdr_selftest_bounded_wait", "bdr_selftest_host", "bdr_qsnr_from_sums", "bdr_pack2", "bdr_qsnr_delayed", "bdr_amax", "bdr_tile_packing_efficiency")
 
 
 class BdrError(RuntimeError):
@@ -93,6 +93,13 @@ def lib():
                                C.c_void_p, C.c_void_p, C.c_void_p]
         L.bdr_unpack.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int64, C.c_int64, C.c_int64, C.c_int,
                                  C.c_void_p]
+        L.bdr_qsnr_delayed.restype = C.c_int
+        L.bdr_qsnr_delayed.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_int, C.c_int64, C.c_int64, C.c_int64, C.c_int,
+                                       C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p]
+        L.bdr_amax.restype = C.c_int
+        L.bdr_amax.argtypes = [C.c_void_p, C.c_int, C.c_int64, C.c_int64, C.c_int64, C.c_void_p, C.c_void_p]
+        L.bdr_tile_packing_efficiency.restype = C.c_double
+        L.bdr_tile_packing_efficiency.argtypes = [C.c_void_p, C.c_int64, C.c_int64]
         L.bdr_pack2.restype = C.c_int
         L.bdr_pack2.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int64, C.c_int64, C.c_int64, C.c_void_p, C.c_void_p,
                                 C.c_void_p, C.c_void_p, C.c_void_p]
@@ -246,6 +253,32 @@ def bdr_qsnr(cfgs, x: torch.Tensor, out_db: torch.Tensor, workspace: torch.Tenso
                           _ptr(out_db), _ptr(workspace), workspace.numel() * workspace.element_size(),
                           _stream(stream)), "bdr_qsnr")
     return out_db
+
+
+def bdr_qsnr_delayed(cfgs, x: torch.Tensor, amax_window: torch.Tensor, out_db: torch.Tensor, workspace: torch.Tensor,
+                     axis: int = 1, stream=None):
+    """bdr_qsnr with the FP32 kinds' first-level maximum taken from `amax_window` (float32 device tensor of earlier
+    maxima) instead of from x."""
+    assert amax_window.dtype == torch.float32 and amax_window.is_contiguous() and amax_window.is_cuda
+    x2 = _as2d(x)
+    arr = (_Config * len(cfgs))(*[c.c() for c in cfgs])
+    _check(lib().bdr_qsnr_delayed(C.addressof(arr), len(cfgs), _ptr(x2), _dt(x2), x2.shape[0], x2.shape[1], x2.stride(0), axis,
+                                  _ptr(amax_window), amax_window.numel(), _ptr(out_db), _ptr(workspace),
+                                  workspace.numel() * workspace.element_size(), _stream(stream)), "bdr_qsnr_delayed")
+    return out_db
+
+
+def bdr_amax(x: torch.Tensor, amax: torch.Tensor, stream=None) -> torch.Tensor:
+    """amax[0] = max(amax[0], max |x|); amax: one float32 on the device, zeroed by the caller."""
+    assert amax.dtype == torch.float32 and amax.numel() == 1 and amax.is_cuda
+    x2 = _as2d(x)
+    _check(lib().bdr_amax(_ptr(x2), _dt(x2), x2.shape[0], x2.shape[1], x2.stride(0), _ptr(amax), _stream(stream)), "bdr_amax")
+    return amax
+
+
+def bdr_tile_packing_efficiency(cfg: Config, tile_elems: int = 256, line_bytes: int = 64) -> float:
+    c = cfg.c()
+    return float(lib().bdr_tile_packing_efficiency(C.addressof(c), tile_elems, line_bytes))
 
 
 def bdr_qsnr_static_max_cfgs() -> int:

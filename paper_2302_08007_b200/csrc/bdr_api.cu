@@ -226,6 +226,17 @@ int bdr_packed_sizes(const bdr_config_t* cfg, int64_t rows, int64_t cols, int ax
     return BDR_OK;
 }
 
+double bdr_tile_packing_efficiency(const bdr_config_t* c, int64_t tile_elems, int64_t line_bytes) {
+    if (!c || tile_elems < 1 || line_bytes < 1 || c->m < 1 || c->k1 < 0 || c->k2 < 0 || c->d1 < 0 || c->d2 < 0) return -1.0;
+    // integer arithmetic in units of 1 / (k1 k2) bit, so that no rounding decides the number of lines
+    const int64_t k1 = c->k1 > 0 ? c->k1 : 1, k2 = c->k2 > 0 ? c->k2 : 1;
+    const int64_t unit = k1 * k2;
+    const int64_t per_elem = (int64_t)(c->m + 1) * unit + (c->k1 > 0 ? (int64_t)c->d1 * k2 : 0) + (c->k2 > 0 ? (int64_t)c->d2 * k1 : 0);
+    const int64_t bits = per_elem * tile_elems, line = line_bytes * 8 * unit;
+    const int64_t lines = (bits + line - 1) / line;
+    return (double)bits / (double)(lines * line);
+}
+
 int bdr_quant_dequant(const bdr_config_t* cfg, const void* x, void* y, bdr_dtype_t dt, int64_t rows, int64_t cols,
                       int64_t ld, int axis, double* qsnr_sums_dev, void* stream) {
     QParams qp;

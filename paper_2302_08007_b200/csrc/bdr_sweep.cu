@@ -228,11 +228,12 @@ __device__ __forceinline__ float round_int(float t) {  // 0 <= t < 2^22
     else return floorf(__fadd_rn(t, 0.5f));
 }
 
-// |deq| - |x| is exact in fp32: either deq = 0, or the two are within a factor of two of each other (a value and
-// its rounding to a grid with at least one significant bit).  The square goes to the fp64 accumulator directly:
-// unlike on the power-of-two path the values are not normalised, so fp32 squares could overflow or vanish.
+// |deq| - |x| is formed in fp64, where it is exact: with a first-level maximum that comes from elsewhere (delayed
+// scaling) a value can saturate far below its magnitude, and then the fp32 difference would round.  The square goes
+// to the fp64 accumulator directly: unlike on the power-of-two path the values are not normalised, so fp32 squares
+// could overflow or vanish.
 __device__ __forceinline__ void add_err(float deq_mag, float ax, double& e2) {
-    const double d = (double)__fsub_rn(deq_mag, ax);
+    const double d = (double)deq_mag - (double)ax;
     e2 = fma(d, d, e2);
 }
 __device__ __forceinline__ void all_zero_slice(const uint32_t (&u)[kSlice], double& e2) {  // scale 0: everything quantizes to 0
@@ -348,6 +349,18 @@ __global__ void amax_kernel(const T* x, int64_t rows, int64_t cols, int64_t ld, 
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) m = max(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
     if ((threadIdx.x & 31) == 0) atomicMax(amax_bits, m);
+}
+
+// First-level maximum from a window of earlier maxima (delayed scaling): the largest of n non-negative floats.
+__global__ void window_amax_kernel(const float* window, int n, uint32_t* amax_bits) {
+    uint32_t m = 0;
+    for (int i = threadIdx.x; i < n; i += 32) {
+        const uint32_t b = __float_as_uint(window[i]);
+        if (b <= 0x7F800000u) m = max(m, b);  // negative values and NaNs are not maxima of magnitudes: ignored
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) m = max(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
+    if (threadIdx.x == 0) *amax_bits = m;
 }
 
 template <typename T>
@@ -590,8 +603,16 @@ static void build_families(const std::vector<SweepCfg>& singles, std::vector<Swe
 }
 
 template <typename T>
+static int amax_launch(const T* x, int64_t rows, int64_t cols, int64_t ld, uint32_t* amax_bits, cudaStream_t st) {
+    const int64_t total = rows * cols;
+    const int grid = (int)max((int64_t)1, min((total + 1023) / 1024, (int64_t)sm_count() * 8));
+    amax_kernel<T><<<grid, 256, 0, st>>>(x, rows, cols, ld, amax_bits);
+    return cudaGetLastError() == cudaSuccess ? BDR_OK : BDR_ERR_CUDA;
+}
+
+template <typename T>
 static int sweep_launch(const SweepCfg* host_fams, int n_fam, int n, bool need_amax, const T* x, int64_t rows, int64_t cols,
-                        int64_t ld, int axis, double* out_db, uint8_t* ws, cudaStream_t st) {
+                        int64_t ld, int axis, const float* amax_window, int n_window, double* out_db, uint8_t* ws, cudaStream_t st) {
     double* err = reinterpret_cast<double*>(ws);
     double* sig = err + n;
     uint32_t* amax = reinterpret_cast<uint32_t*>(sig + 1);
@@ -605,9 +626,8 @@ static int sweep_launch(const SweepCfg* host_fams, int n_fam, int n, bool need_a
     }
     if (rows > 0 && cols > 0) {
         if (need_amax) {
-            const int64_t total = rows * cols;
-            const int grid = (int)max((int64_t)1, min((total + 1023) / 1024, (int64_t)sm_count() * 8));
-            amax_kernel<T><<<grid, 256, 0, st>>>(x, rows, cols, ld, amax);
+            if (amax_window) window_amax_kernel<<<1, 32, 0, st>>>(amax_window, n_window, amax);
+            else amax_launch<T>(x, rows, cols, ld, amax, st);
         }
         const int64_t n_lines = axis == 1 ? rows : cols, len = axis == 1 ? cols : rows;
         const int tiles_per_line = (int)((len + kTile - 1) / kTile);
@@ -659,8 +679,9 @@ extern "C" {
 
 int64_t bdr_qsnr_workspace_bytes(int n_cfgs) { return n_cfgs < 1 ? 0 : sweep_workspace_bytes(n_cfgs); }
 
-int bdr_qsnr(const bdr_config_t* cfgs, int n_cfgs, const void* x, bdr_dtype_t dt, int64_t rows, int64_t cols, int64_t ld,
-             int axis, double* qsnr_db_dev, void* workspace, int64_t workspace_bytes, void* stream) {
+static int qsnr_impl(const bdr_config_t* cfgs, int n_cfgs, const void* x, bdr_dtype_t dt, int64_t rows, int64_t cols, int64_t ld,
+                     int axis, const float* amax_window, int n_window, double* qsnr_db_dev, void* workspace, int64_t workspace_bytes,
+                     void* stream) {
     constexpr int kMaxCfgs = 4096;  // per-CTA accumulators live in shared memory
     if (!cfgs || !qsnr_db_dev) return BDR_ERR_NULL;
     if (n_cfgs < 1 || n_cfgs > kMaxCfgs) return BDR_ERR_SIZE;
@@ -682,10 +703,38 @@ int bdr_qsnr(const bdr_config_t* cfgs, int n_cfgs, const void* x, bdr_dtype_t dt
     if ((uintptr_t)workspace % 16) return BDR_ERR_MISALIGNED;
     cudaStream_t st = (cudaStream_t)stream;
     if (dt == BDR_F32)
-        return sweep_launch<float>(table.data(), n_fam, n_cfgs, need_amax, (const float*)x, rows, cols, ld, axis, qsnr_db_dev,
-                                   (uint8_t*)workspace, st);
-    return sweep_launch<__nv_bfloat16>(table.data(), n_fam, n_cfgs, need_amax, (const __nv_bfloat16*)x, rows, cols, ld, axis, qsnr_db_dev,
-                                       (uint8_t*)workspace, st);
+        return sweep_launch<float>(table.data(), n_fam, n_cfgs, need_amax, (const float*)x, rows, cols, ld, axis, amax_window, n_window,
+                                   qsnr_db_dev, (uint8_t*)workspace, st);
+    return sweep_launch<__nv_bfloat16>(table.data(), n_fam, n_cfgs, need_amax, (const __nv_bfloat16*)x, rows, cols, ld, axis, amax_window,
+                                       n_window, qsnr_db_dev, (uint8_t*)workspace, st);
+}
+
+int bdr_qsnr(const bdr_config_t* cfgs, int n_cfgs, const void* x, bdr_dtype_t dt, int64_t rows, int64_t cols, int64_t ld,
+             int axis, double* qsnr_db_dev, void* workspace, int64_t workspace_bytes, void* stream) {
+    return qsnr_impl(cfgs, n_cfgs, x, dt, rows, cols, ld, axis, nullptr, 0, qsnr_db_dev, workspace, workspace_bytes, stream);
+}
+
+int bdr_qsnr_delayed(const bdr_config_t* cfgs, int n_cfgs, const void* x, bdr_dtype_t dt, int64_t rows, int64_t cols, int64_t ld,
+                     int axis, const float* amax_window_dev, int n_window, double* qsnr_db_dev, void* workspace,
+                     int64_t workspace_bytes, void* stream) {
+    if (!amax_window_dev) return BDR_ERR_NULL;
+    if (n_window < 1) return BDR_ERR_SIZE;
+    if ((uintptr_t)amax_window_dev % 4) return BDR_ERR_MISALIGNED;
+    return qsnr_impl(cfgs, n_cfgs, x, dt, rows, cols, ld, axis, amax_window_dev, n_window, qsnr_db_dev, workspace, workspace_bytes,
+                     stream);
+}
+
+int bdr_amax(const void* x, bdr_dtype_t dt, int64_t rows, int64_t cols, int64_t ld, float* amax_dev, void* stream) {
+    if (!amax_dev) return BDR_ERR_NULL;
+    if (dt != BDR_F32 && dt != BDR_BF16) return BDR_ERR_UNSUPPORTED;
+    if (rows < 0 || cols < 0 || ld < cols) return BDR_ERR_SIZE;
+    if (rows == 0 || cols == 0) return BDR_OK;
+    if (!x) return BDR_ERR_NULL;
+    if ((uintptr_t)x % (dt == BDR_F32 ? 4 : 2) || (uintptr_t)amax_dev % 4) return BDR_ERR_MISALIGNED;
+    cudaStream_t st = (cudaStream_t)stream;
+    // magnitudes are non-negative floats, whose order is the order of their bit patterns
+    if (dt == BDR_F32) return amax_launch<float>((const float*)x, rows, cols, ld, reinterpret_cast<uint32_t*>(amax_dev), st);
+    return amax_launch<__nv_bfloat16>((const __nv_bfloat16*)x, rows, cols, ld, reinterpret_cast<uint32_t*>(amax_dev), st);
 }
 
 int bdr_qsnr_from_sums(const double* sums_dev, int n, double* qsnr_db_dev, void* stream) {
@@ -707,7 +756,7 @@ int bdr_qsnr_static(const bdr_config_t* cfgs, int n_cfgs, const void* x, bdr_dty
     uint8_t* scratch = nullptr;
     const int rc = static_scratch_ptr(&scratch);  // first call on a device resolves the symbol's address
     if (rc) return rc;
-    return bdr_qsnr(cfgs, n_cfgs, x, dt, rows, cols, ld, axis, qsnr_db_dev, scratch, (int64_t)kStaticScratchBytes, stream);
+    return qsnr_impl(cfgs, n_cfgs, x, dt, rows, cols, ld, axis, nullptr, 0, qsnr_db_dev, scratch, (int64_t)kStaticScratchBytes, stream);
 }
 
 }  // extern "C"

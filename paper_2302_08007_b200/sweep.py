@@ -40,3 +40,21 @@ def comparators() -> list[tuple[str, Config]]:
 def sweep_configs() -> list[tuple[str, Config]]:
     """457 named configurations: the BDR grid first, then the comparators."""
     return bdr_grid() + comparators()
+
+
+def bits_per_element(cfg: Config) -> float:
+    """Section III: (m + 1) + d1/k1 + d2/k2 (a per-tensor scale, k1 = 0, costs nothing per element)."""
+    return (cfg.m + 1) + (cfg.d1 / cfg.k1 if cfg.k1 > 0 else 0.0) + (cfg.d2 / cfg.k2 if cfg.k2 > 0 else 0.0)
+
+
+def pareto_frontier(points):
+    """The QSNR-versus-cost frontier of Section IV-C from (name, cost, qsnr_db) triples: the points that no other
+    point beats or equals on both axes (lower cost, higher QSNR), in order of rising cost.  Here the cost axis is
+    bits per element divided by the tile packing efficiency; the paper's circuit-area factor is not reproducible."""
+    best = []
+    for name, cost, q in sorted(points, key=lambda p: (p[1], -p[2])):
+        if q != q:
+            continue
+        if not best or q > best[-1][2]:
+            best.append((name, cost, q))
+    return best

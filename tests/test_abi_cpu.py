@@ -15,7 +15,7 @@ ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 def _declared_functions():
     text = open(os.path.join(ROOT, "include", "bdr.h")).read()
     text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
-    names = re.findall(r"^\s*(?:const\s+char\s*\*|int64_t|int)\s+(\w+)\s*\(", text, flags=re.M)
+    names = re.findall(r"^\s*(?:const\s+char\s*\*|int64_t|int|double)\s+(\w+)\s*\(", text, flags=re.M)
     return sorted(set(names))
 
 
@@ -70,3 +70,14 @@ def test_per_device_launch_bookkeeping():
     # kernel attributes are per device: the library keeps "set up" flags per device, not per process.  The
     # self-test drives that bookkeeping with fake set-up functions for devices 0, 1, 2 and 63 (no CUDA call).
     assert bdr.bdr_selftest_host() == 0
+
+
+def test_tile_packing_efficiency_agrees_with_the_oracle():
+    C_ = bdr.Config
+    for cfg in (bdr.MX4, bdr.MX6, bdr.MX9, C_(16, 8, 1, 0, 3), C_(64, 8, 8, 2, 5), C_(0, 32, 1, 4, 3, bdr.SCALE_FP32_FP),
+                C_(0, 32, 16, 6, 3, bdr.SCALE_FP32_VSQ)):
+        o = orc.Config(cfg.k1, cfg.d1, cfg.k2, cfg.d2, cfg.m, cfg.scale_kind, cfg.rounding)
+        for tile, line in ((256, 64), (100, 32), (16, 128), (1, 1)):
+            assert bdr.bdr_tile_packing_efficiency(cfg, tile, line) == pytest.approx(orc.tile_packing_efficiency(o, tile, line), rel=1e-15)
+    assert bdr.bdr_tile_packing_efficiency(bdr.MX9) == 0.9
+    assert bdr.bdr_tile_packing_efficiency(bdr.MX9, 0, 64) < 0

@@ -119,3 +119,46 @@ def test_full_size_sweep_on_sampled_configurations():
         want = orc.qsnr(H.to_orc(cfgs[i]), x, nthreads=16)
         assert abs(got[i] - want) <= H.QSNR_REL_TOL * max(abs(want), 1e-3), (i, cfgs[i], got[i], want)
     assert np.isfinite(got).all()
+
+
+def test_first_level_maximum_from_a_window_of_past_tensors():
+    # Fig. 7 caption: INT / FP / VSQ take their FP32 scale from the maximum over a window of past vectors.  bdr_amax
+    # gives each past tensor's maximum (checked against numpy), bdr_qsnr_delayed uses the largest of the window; the
+    # oracle is handed that maximum.  Windows above, equal to and below the current tensor's own maximum (then
+    # values saturate); the power-of-two formats do not depend on it.
+    cfgs = [c for _, c in sweep.comparators()] + [bdr.MX6, bdr.MX9,
+            bdr.Config(0, 32, 1, 0, 7, bdr.SCALE_FP32_INT, bdr.ROUND_NEAREST_AWAY), bdr.Config(0, 32, 16, 6, 3, bdr.SCALE_FP32_VSQ, bdr.ROUND_NEAREST_AWAY)]
+    x = synth.variable_variance_vectors(512, 1024, seed=21)
+    xd = torch.from_numpy(x).cuda()
+    cur = float(np.abs(x).max())
+    past = [synth.variable_variance_vectors(64, 1024, seed=22 + i) * np.float32(sc) for i, sc in enumerate((0.5, 1.5, 0.25))]
+    window = torch.zeros(len(past), dtype=torch.float32, device="cuda")
+    for i, t in enumerate(past):
+        bdr.bdr_amax(torch.from_numpy(t).cuda(), window[i:i + 1])
+    bb = torch.from_numpy(synth.f32_to_bf16_bits(past[0]).view(np.int16)).view(torch.bfloat16).cuda().reshape(64, 1024)
+    a16 = torch.zeros(1, dtype=torch.float32, device="cuda")
+    bdr.bdr_amax(bb[:, :1000], a16)                                    # bf16, a pitch: 1000 of 1024 columns
+    torch.cuda.synchronize()
+    assert window.cpu().tolist() == [float(np.abs(t).max()) for t in past]
+    assert a16.item() == float(np.abs(synth.bf16_bits_to_f32(synth.f32_to_bf16_bits(past[0])).reshape(64, 1024)[:, :1000]).max())
+    ws = torch.empty(bdr.bdr_qsnr_workspace_bytes(len(cfgs)), dtype=torch.uint8, device="cuda")
+    out = torch.empty(len(cfgs), dtype=torch.float64, device="cuda")
+    for win in (window, window[:1], window[2:], torch.tensor([cur], dtype=torch.float32, device="cuda"),
+                torch.tensor([cur * 0.01, 0.0], dtype=torch.float32, device="cuda")):
+        amax = float(win.max().item())
+        bdr.bdr_qsnr_delayed(cfgs, xd, win, out, ws)
+        torch.cuda.synchronize()
+        got = out.cpu().numpy()
+        for cfg, g in zip(cfgs, got):
+            o = H.to_orc(cfg)
+            want = orc.qsnr(o, x, amax=None if cfg.scale_kind == bdr.SCALE_POW2 else amax)
+            assert abs(g - want) <= H.QSNR_REL_TOL * max(abs(want), 1e-3), (cfg, amax, g, want)
+    same = torch.empty(len(cfgs), dtype=torch.float64, device="cuda")
+    bdr.bdr_qsnr(cfgs, xd, same, ws)                                   # window = the tensor's own maximum: plain bdr_qsnr
+    bdr.bdr_qsnr_delayed(cfgs, xd, torch.tensor([cur], dtype=torch.float32, device="cuda"), out, ws)
+    torch.cuda.synchronize()
+    assert torch.allclose(same, out, rtol=1e-12, atol=0)               # the same arithmetic; only the order of the fp64 atomics differs
+    with pytest.raises(bdr.BdrError) as e:
+        bdr.bdr_qsnr_delayed(cfgs, xd, window[:0], out, ws)
+    assert e.value.status == -5
+    torch.cuda.synchronize()

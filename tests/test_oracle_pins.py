@@ -546,6 +546,67 @@ def test_vsq_with_a_wide_sub_scale_approaches_int_with_one_fp32_scale_per_vector
     assert orc.qsnr(Cfg(0, 32, 16, 4, m, orc.FP32_VSQ), x.ravel()) < orc.qsnr_db(ei, si) - 0.1
 
 
+# ---- first-level scale from elsewhere (delayed scaling), packing efficiency -------------------------------------
+def test_supplied_first_level_maximum():
+    import torch
+    x = synth.normal(8192, 90) * np.float32(3.0)
+    cur = float(np.abs(x).max())
+    kinds = [Cfg(0, 32, 1, 0, 7, orc.FP32_INT), Cfg(0, 32, 1, 4, 3, orc.FP32_FP), Cfg(0, 32, 16, 6, 3, orc.FP32_VSQ)]
+    for cfg in kinds:     # the current tensor's own maximum, supplied from outside: the same function
+        a, sa = orc.quant_dequant(cfg, x)
+        b, sb = orc.quant_dequant(cfg, x, amax=cur)
+        assert np.array_equal(a.view(np.uint32), b.view(np.uint32)) and sa == sb
+    # INT8 with a supplied maximum of 127: s = 1, so Eq. 2 is rint(x) and values beyond the maximum saturate
+    xi = (synth.normal(4096, 91) * 80).astype(np.float32)
+    y, _ = orc.quant_dequant(Cfg(0, 32, 1, 0, 7, orc.FP32_INT), xi, amax=127.0)
+    assert np.abs(xi).max() > 200 and np.array_equal(y, np.clip(np.rint(xi), -127, 127))
+    # E4M3 with a supplied maximum of 448: s = 1, the library's saturating cast
+    xf = (synth.normal(4096, 92) * 300).astype(np.float32)
+    y, _ = orc.quant_dequant(Cfg(0, 32, 1, 4, 3, orc.FP32_FP), xf, amax=448.0)
+    want = torch.from_numpy(np.clip(xf, -448, 448)).to(torch.float8_e4m3fn).to(torch.float32).numpy()
+    assert np.abs(xf).max() > 448 and np.array_equal(y.view(np.uint32), want.view(np.uint32))
+    # VSQ: the hand-worked group without its largest vector, with that vector's maximum supplied: same results
+    for name, rnd, k1, m, d2, gammas, vecs in _vsq_cases():
+        if name != "d4_even":
+            continue
+        xs = np.array([v for _, xx, _, _ in vecs[1:] for v in xx], dtype=np.float32)
+        want = np.array([v for _, _, _, Q in vecs[1:] for v in Q], dtype=np.float32)
+        y, _ = orc.quant_dequant(Cfg(0, 32, 16, d2, m, orc.FP32_VSQ, rnd), xs, amax=6.5625)
+        assert y.view(np.uint32).tolist() == want.view(np.uint32).tolist()
+        # a window maximum SMALLER than a vector's own (105/64: gamma = 1/64): (2/7) x 64 = 18.3 clamps at the top
+        # sub-scale 15, scale 15/64; 2.0 / (15/64) = 8.5 saturates at 7; 0.78125 / (15/64) = 3.33 -> 3
+        y, _ = orc.quant_dequant(Cfg(0, 32, 16, d2, m, orc.FP32_VSQ, rnd), xs[:16], amax=1.640625)
+        assert y[0] == np.float32(7 * 15 / 64) and y[1] == np.float32(3 * 15 / 64)
+    # a supplied maximum is refused where it has no meaning
+    with pytest.raises(ValueError):
+        orc.quant_dequant(orc.MX6, x, amax=1.0)
+
+
+def test_tile_packing_efficiency_closed_form():
+    # Section IV-B: a 256-element tile into 64-byte lines.  MX9: 288 bytes in 5 lines = 0.9; MX6 192 B, MX4 128 B and
+    # FP8 256 B fill whole lines; MSFP12 (4.5 bits: 144 B in 3 lines) 0.75
+    assert orc.tile_packing_efficiency(orc.MX9) == 288 / 320
+    assert orc.tile_packing_efficiency(orc.MX6) == 1.0 and orc.tile_packing_efficiency(orc.MX4) == 1.0
+    assert orc.tile_packing_efficiency(Cfg(0, 32, 1, 4, 3, orc.FP32_FP)) == 1.0
+    assert orc.tile_packing_efficiency(Cfg(16, 8, 1, 0, 3)) == 144 / 192
+    for cfg in (orc.MX9, Cfg(64, 8, 8, 2, 5), Cfg(8, 8, 1, 3, 2)):
+        for tile, line in ((256, 64), (100, 32), (16, 128)):
+            bits = orc.bits_per_element(cfg) * tile
+            lines = math.ceil(bits / (8 * line))
+            assert orc.tile_packing_efficiency(cfg, tile, line) == pytest.approx(bits / (lines * 8 * line), rel=1e-15)
+
+
+def test_pareto_frontier_against_brute_force():
+    from paper_2302_08007_b200 import sweep
+    rng = np.random.default_rng(93)
+    pts = [("p%d" % i, float(rng.integers(2, 12)) / 2, float(rng.normal(30, 10))) for i in range(200)]
+    got = sweep.pareto_frontier(pts)
+    brute = [p for p in pts if not any((q[1] <= p[1] and q[2] > p[2]) or (q[1] < p[1] and q[2] >= p[2]) for q in pts)]
+    assert sorted(got) == sorted(brute)
+    assert [g[1] for g in got] == sorted(g[1] for g in got) and [g[2] for g in got] == sorted(g[2] for g in got)
+    assert sweep.bits_per_element(sweep.Config(16, 8, 2, 1, 7)) == 9.0
+
+
 # ---- GEMM reference ---------------------------------------------------------------------------------------------
 def test_gemm_reference_is_the_plain_definition():
     rng = np.random.default_rng(80)
