@@ -567,4 +567,102 @@ void orc_gemm_nt_f64_sampled(const float* a, const float* b, int64_t K, const in
     }
 }
 
+// ---------------------------------------------------------------------------------------------
+// Dot product as the hardware pipeline of Section IV-B (Fig. 6) computes it, C = A B^T with both
+// operands quantized along K in a POW2 format (same k1, k2, d2; the mantissa widths may differ).
+// The paper describes the pipeline in words; the readings taken here (listed in the design notes):
+//   1. Inside a k1-block the integer mantissa products (sign-magnitude) are summed exactly.  The
+//      products of sub-block j are summed first (depth log2 k2), then aligned by the two operands'
+//      shifts: the sub-block sum S_j enters the block sum with weight 2^(2 beta - tau_A,j - tau_B,j)
+//      (the conditional right shift, done on a datapath widened by 2 beta bits so that nothing is
+//      lost).  Block result: an integer D_b, |D_b| < 2^W, W = m_A + m_B + log2 k1 + 2 beta, worth
+//      D_b * 2^(E_A,b + E_B,b - (m_A - 1) - (m_B - 1) - 2 beta).
+//   2. The r/k1 block results of one pass through the pipeline (r consecutive elements of K) are
+//      normalised to the largest block exponent sum e_max = max_b (F_A,b + F_B,b) -- every block takes
+//      part, also one whose result is zero -- and reduced in fixed point: block b is shifted right by
+//      e_max - e_b inside a frame of f magnitude bits whose top bit is the top bit of a W-bit result
+//      at e_max, i.e. A_b = trunc(D_b * 2^(f - W - (e_max - e_b))), truncated toward zero (sign-
+//      magnitude datapath).  The aligned integers are added exactly.
+//   3. The pass's sum leaves the pipeline as an fp32 number (one rounding to nearest even), and
+//      successive passes (K > r) are accumulated in fp32 in order of increasing K.
+//   4. A block with the exponent byte 0xFF (Inf/NaN input) makes the result NaN.
+// ---------------------------------------------------------------------------------------------
+static inline int64_t shift_trunc(int64_t v, int sh) {  // v * 2^sh, truncated toward zero
+    if (sh >= 0) return sh >= 62 ? 0 : v * ((int64_t)1 << sh);  // callers keep |v| 2^sh below 2^62
+    if (-sh >= 63) return 0;
+    const int64_t mag = (v < 0 ? -v : v) >> (-sh);
+    return v < 0 ? -mag : mag;
+}
+
+int orc_gemm_hw(const orc_config* ca, const float* a, int64_t M, const orc_config* cb, const float* b, int64_t N, int64_t K,
+                int r, int f, float* c) {
+    if (!config_ok(ca) || !config_ok(cb) || ca->scale_kind != ORC_POW2 || cb->scale_kind != ORC_POW2) return ORC_BAD;
+    if (ca->k1 != cb->k1 || ca->k2 != cb->k2 || ca->d2 != cb->d2 || ca->rounding != cb->rounding) return ORC_BAD;
+    const int k1 = ca->k1, k2 = ca->k2, beta = (1 << ca->d2) - 1;
+    if (!a || !b || !c || M < 0 || N < 0 || K < 0 || r < k1 || r % k1 != 0 || K % r != 0) return ORC_BAD;
+    int lg = 0;
+    while ((1 << lg) < k1) ++lg;
+    const int W = ca->m + cb->m + lg + 2 * beta;
+    if (f < 1 || f > 40 || W > 40 || r / k1 > 4096) return ORC_BAD;
+    const int nb = (int)(K / k1), nsub = k1 / k2;
+    // encode both operands row by row
+    auto encode_rows = [&](const orc_config& cfg, const float* x, int64_t rows, std::vector<uint8_t>& F, std::vector<uint8_t>& tau,
+                           std::vector<int32_t>& q) {
+        F.assign(rows * nb, 0);
+        tau.assign(rows * nb * nsub, 0);
+        q.assign(rows * K, 0);
+        std::vector<uint16_t> code(k1);
+        for (int64_t i = 0; i < rows; ++i)
+            for (int bb = 0; bb < nb; ++bb) {
+                pow2_block(cfg, x + i * K + (int64_t)bb * k1, 1, k1, &F[i * nb + bb], &tau[(i * nb + bb) * nsub], code.data(), nullptr, 0);
+                for (int e = 0; e < k1; ++e) {
+                    const int32_t mag = code[e] & ((1 << cfg.m) - 1);
+                    q[i * K + (int64_t)bb * k1 + e] = (code[e] >> cfg.m) & 1 ? -mag : mag;
+                }
+            }
+    };
+    std::vector<uint8_t> Fa, Fb, ta, tb;
+    std::vector<int32_t> qa, qb;
+    encode_rows(*ca, a, M, Fa, ta, qa);
+    encode_rows(*cb, b, N, Fb, tb, qb);
+    const int bpr = r / k1;  // blocks per pass
+    std::vector<int64_t> D(bpr);
+    std::vector<int> e(bpr);
+    for (int64_t i = 0; i < M; ++i)
+        for (int64_t j = 0; j < N; ++j) {
+            float acc = 0.f;
+            bool nan = false;
+            for (int64_t p0 = 0; p0 < nb; p0 += bpr) {
+                int emax = 0;
+                for (int bb = 0; bb < bpr; ++bb) {
+                    const int64_t blk = p0 + bb;
+                    const int fa = Fa[i * nb + blk], fb = Fb[j * nb + blk];
+                    if (fa == 255 || fb == 255) nan = true;
+                    int64_t d = 0;
+                    for (int sj = 0; sj < nsub; ++sj) {
+                        int64_t sum = 0;
+                        for (int t = 0; t < k2; ++t) {
+                            const int64_t k = blk * k1 + (int64_t)sj * k2 + t;
+                            sum += (int64_t)qa[i * K + k] * (int64_t)qb[j * K + k];
+                        }
+                        const int sh = 2 * beta - ta[(i * nb + blk) * nsub + sj] - tb[(j * nb + blk) * nsub + sj];
+                        d += sum * ((int64_t)1 << sh);
+                    }
+                    D[bb] = d;
+                    e[bb] = fa + fb;
+                    emax = std::max(emax, e[bb]);
+                }
+                int64_t total = 0;
+                for (int bb = 0; bb < bpr; ++bb) total += shift_trunc(D[bb], f - W - (emax - e[bb]));
+                // value of the frame's unit: 2^(emax - 254 - (mA - 1) - (mB - 1) - 2 beta - (f - W))
+                const int unit = emax - 254 - (ca->m - 1) - (cb->m - 1) - 2 * beta - (f - W);
+                const float pass = (float)total;                       // one rounding to nearest even (|total| < 2^53)
+                const float v = (float)std::ldexp((double)pass, unit);  // exact unless it leaves the fp32 range
+                acc = acc + v;
+            }
+            c[i * N + j] = nan ? std::numeric_limits<float>::quiet_NaN() : acc;
+        }
+    return ORC_OK;
+}
+
 }  // extern "C"

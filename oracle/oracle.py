@@ -213,3 +213,18 @@ def gemm_nt_f64_sampled(a, b, ri, ci):
     out = np.empty(ri.size, dtype=np.float64)
     lib().orc_gemm_nt_f64_sampled(_p(a), _p(b), _i64(a.shape[1]), _p(ri), _p(ci), _i64(ri.size), _p(out))
     return out
+
+
+def gemm_hw(cfg_a: Config, a, cfg_b: Config, b, r: int = 64, f: int = 25):
+    """C = A B^T [M, N] fp32 as the dot-product pipeline of Section IV-B computes it (pass length r, f-bit fixed-point
+    reduction) from the raw fp32 operands A [M, K], B [N, K], which are quantized along K first."""
+    a, b = _f32(a), _f32(b)
+    M, K = a.shape
+    N = b.shape[0]
+    assert b.shape[1] == K
+    c = np.empty((M, N), dtype=np.float32)
+    ca, cb = cfg_a.c(), cfg_b.c()
+    rc = lib().orc_gemm_hw(C.byref(ca), _p(a), _i64(M), C.byref(cb), _p(b), _i64(N), _i64(K), C.c_int(r), C.c_int(f), _p(c))
+    if rc != 0:
+        raise ValueError("oracle rejected the configuration or arguments")
+    return c

@@ -607,6 +607,94 @@ def test_pareto_frontier_against_brute_force():
     assert sweep.bits_per_element(sweep.Config(16, 8, 2, 1, 7)) == 9.0
 
 
+# ---- the dot product as the hardware pipeline computes it (Section IV-B, Fig. 6) --------------------------------
+def _exact_dot_f32(qa, qb):
+    """float32(sum_k qa[k] qb[k]) with the sum formed exactly (rationals), for dequantized fp32 operands."""
+    out = np.empty((qa.shape[0], qb.shape[0]), dtype=np.float32)
+    for i in range(qa.shape[0]):
+        for j in range(qb.shape[0]):
+            out[i, j] = np.float32(float(sum(Fraction(float(x)) * Fraction(float(y)) for x, y in zip(qa[i], qb[j]))))
+    return out
+
+
+def test_hw_dot_hand_worked_passes():
+    cfg = Cfg(4, 8, 2, 1, 3)
+    for row in _golden_rows("hw_dot_blocks.txt"):
+        f, a, b, want = [t.strip() for t in row.split("|")]
+        a = np.array([float(v) for v in a.split()], dtype=np.float32).reshape(1, -1)
+        b = np.array([float(v) for v in b.split()], dtype=np.float32).reshape(1, -1)
+        got = orc.gemm_hw(cfg, a, cfg, b, r=8, f=int(f))
+        assert got.shape == (1, 1) and got[0, 0] == np.float32(float(want)), (row, got)
+
+
+def test_hw_dot_is_the_exact_dot_product_when_nothing_is_shifted_out():
+    rng = np.random.default_rng(95)
+    # (1) MX9, one pass of 64: every block holds an element of magnitude 1.5, so all block exponents are equal and the
+    # 25-bit frame keeps every bit of the 20-bit block results: the pass is the exact dot product, rounded once
+    a = rng.normal(size=(5, 64)).astype(np.float32).clip(-1.4, 1.4)
+    b = rng.normal(size=(4, 64)).astype(np.float32).clip(-1.4, 1.4)
+    a[:, ::16] = 1.5
+    b[:, 5::16] = -1.5
+    qa, qb = orc.quant_dequant(orc.MX9, a)[0], orc.quant_dequant(orc.MX9, b)[0]
+    assert np.array_equal(orc.gemm_hw(orc.MX9, a, orc.MX9, b, r=64, f=25), _exact_dot_f32(qa, qb))
+    # (2) no microexponents (d2 = 0: plain block floating point), m = 7 x m = 4, block exponents up to 3 + 3 binades apart:
+    # W = 7 + 4 + 4 = 15, the frame has 10 spare bits, nothing is lost
+    ca, cb = Cfg(16, 8, 1, 0, 7), Cfg(16, 8, 1, 0, 4)
+    a = (rng.normal(size=(3, 128)) * np.repeat(2.0 ** rng.integers(0, 4, (3, 8)), 16, axis=1)).astype(np.float32)
+    b = (rng.normal(size=(6, 128)) * np.repeat(2.0 ** rng.integers(0, 4, (6, 8)), 16, axis=1)).astype(np.float32)
+    qa, qb = orc.quant_dequant(ca, a)[0], orc.quant_dequant(cb, b)[0]
+    assert np.array_equal(orc.gemm_hw(ca, a, cb, b, r=128, f=25), _exact_dot_f32(qa, qb))
+    # and equals the integer dot product of the codes, block by block
+    Fa, _, codea = orc.encode(ca, a)
+    Fb, _, codeb = orc.encode(cb, b)
+    sa = np.where(codea >> 7 & 1, -1, 1) * (codea & 127).astype(np.int64)
+    sb = np.where(codeb >> 4 & 1, -1, 1) * (codeb & 15).astype(np.int64)
+    i, j = 1, 4
+    D = (sa[i] * sb[j]).reshape(8, 16).sum(axis=1)
+    val = sum(Fraction(int(D[k])) * Fraction(2) ** (int(Fa[i, k]) + int(Fb[j, k]) - 254 - 6 - 3) for k in range(8))
+    assert orc.gemm_hw(ca, a, cb, b, r=128, f=25)[i, j] == np.float32(float(val))
+
+
+def test_hw_dot_truncation_is_bounded_ordered_and_pass_structured():
+    rng = np.random.default_rng(96)
+    a = (rng.normal(size=(4, 64)) * np.repeat(2.0 ** rng.integers(-6, 7, (4, 4)), 16, axis=1)).astype(np.float32)
+    b = (rng.normal(size=(5, 64)) * np.repeat(2.0 ** rng.integers(-6, 7, (5, 4)), 16, axis=1)).astype(np.float32)
+    qa, qb = orc.quant_dequant(orc.MX6, a)[0], orc.quant_dequant(orc.MX6, b)[0]
+    exact = qa.astype(np.float64) @ qb.astype(np.float64).T          # exact in fp64: 64 products of 5-bit numbers
+    Fa, Fb = orc.encode(orc.MX6, a)[0].astype(int), orc.encode(orc.MX6, b)[0].astype(int)
+    W = 4 + 4 + 4 + 2
+    lost = False
+    for f in (6, 10, 14, 25):
+        c = orc.gemm_hw(orc.MX6, a, orc.MX6, b, r=64, f=f).astype(np.float64)
+        emax = (Fa[:, None, :] + Fb[None, :, :]).max(axis=2)
+        unit = 2.0 ** (emax - 254 - 3 - 3 - 2 - (f - W))
+        # each of the 4 blocks loses less than one unit of the frame (toward zero); the largest block loses nothing when f >= W
+        err = np.abs(c - exact)
+        assert np.all(err <= 4 * unit + 2.0 ** -23 * np.abs(exact)), f
+        lost |= bool(np.any(err > 0))
+    assert lost                                                       # the narrow frames do drop bits on this input
+    # blocks of a pass may come in any order: the fixed-point sum is exact
+    perm = np.array([2, 0, 3, 1])
+    idx = (perm[:, None] * 16 + np.arange(16)[None, :]).ravel()
+    assert np.array_equal(orc.gemm_hw(orc.MX6, a[:, idx], orc.MX6, b[:, idx], r=64, f=10), orc.gemm_hw(orc.MX6, a, orc.MX6, b, r=64, f=10))
+    # K = 2 r: two passes, added in fp32 in order
+    a2, b2 = np.concatenate([a, a[::-1]], axis=1), np.concatenate([b, 3 * b], axis=1)
+    p1 = orc.gemm_hw(orc.MX6, a2[:, :64], orc.MX6, b2[:, :64], r=64, f=10)
+    p2 = orc.gemm_hw(orc.MX6, a2[:, 64:], orc.MX6, b2[:, 64:], r=64, f=10)
+    assert np.array_equal(orc.gemm_hw(orc.MX6, a2, orc.MX6, b2, r=64, f=10), p1 + p2)
+    # shorter passes align fewer blocks to a common exponent: r = 16 (one block per pass) loses nothing in the frame
+    one = orc.gemm_hw(orc.MX6, a, orc.MX6, b, r=16, f=14)
+    blocks = sum((qa[:, k:k + 16].astype(np.float64) @ qb[:, k:k + 16].astype(np.float64).T).astype(np.float32) for k in range(0, 64, 16))
+    assert np.array_equal(one, blocks.astype(np.float32))
+    # an Inf/NaN block poisons the outputs of its row only
+    an = a.copy()
+    an[2, 17] = np.inf
+    cn = orc.gemm_hw(orc.MX6, an, orc.MX6, b, r=64, f=25)
+    assert np.isnan(cn[2]).all() and not np.isnan(np.delete(cn, 2, axis=0)).any()
+    with pytest.raises(ValueError):
+        orc.gemm_hw(orc.MX6, a, orc.MX9._replace(k2=4) if hasattr(orc.MX9, "_replace") else Cfg(16, 8, 4, 1, 7), b)
+
+
 # ---- GEMM reference ---------------------------------------------------------------------------------------------
 def test_gemm_reference_is_the_plain_definition():
     rng = np.random.default_rng(80)
