@@ -490,7 +490,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-graph", action="store_true", help="launch every kernel from Python instead of replaying a CUDA graph of the step")
-    ap.add_argument("--only", default=None, choices=["quant_dequant", "pack", "unpack", "pack2", "gemm", "gemm_ws", "gemm_f8", "sweep"],
+    ap.add_argument("--only", default=None, choices=["quant_dequant", "pack", "unpack", "pack2", "gemm", "gemm_ws", "gemm_f8", "gemm_hw", "sweep"],
                     help="run one operation a few times on a seeded tensor and print its time (for profilers); no JSON line")
     ap.add_argument("--fmt", default="MX6", choices=["MX4", "MX6", "MX9"])
     ap.add_argument("--axis", type=int, default=1)

@@ -125,6 +125,7 @@ def gemm_leg(args) -> dict:
         ms_lent = _time(lambda: bdr.mx_gemm(bdr.MX6, pa, bdr.MX6, pb, M, N, K, c), reps=20, warmup=3)
     finally:
         bdr.bdr_set_workspace(None)
+    ms_hw = _time(lambda: bdr.mx_gemm_hw(bdr.MX6, pa, bdr.MX6, pb, M, N, K, c, r=64, f=25), reps=2, warmup=1)
     cpu = gemm_oracle_sample(M, N, K) if getattr(args, "cpu_legs", False) else None
     tf = lambda t: 2.0 * M * N * K / (t * 1e-3) / 1e12
     ws_name = ("mx_gemm_ws (both operands decoded once to a bf16 workspace, then a TMA-fed tcgen05 GEMM; the time "
@@ -143,6 +144,10 @@ def gemm_leg(args) -> dict:
                         "mx_gemm_e4m3": {"value": tf(ms_pre), "unit": "TFLOP/s", "ms": ms_pre,
                                          "note": "operands re-encoded ahead of time (not the headline: the re-encoding is not timed)",
                                          "exact": int(flag.item()) == 0},
+                        "mx_gemm_hw": {"value": tf(ms_hw), "unit": "TFLOP/s", "ms": ms_hw, "bound": "alu",
+                                       "note": "the product as the dot-product pipeline of Section IV-B computes it (r = 64, f = 25): integer "
+                                               "block sums, truncating alignment per block and output; ordinary arithmetic units, bit-exact "
+                                               "with the oracle"},
                         "cpu_baseline": cpu, "status": bdr.mx_gemm_status()}}
 
 
@@ -255,7 +260,7 @@ FORMATS = {"MX4": bdr.MX4, "MX6": bdr.MX6, "MX9": bdr.MX9}
 def run_only(a) -> None:
     cfg = FORMATS[a.fmt]
     reps = a.reps
-    if a.only in ("gemm", "gemm_ws", "gemm_f8"):
+    if a.only in ("gemm", "gemm_ws", "gemm_f8", "gemm_hw"):
         M = N = a.rows
         K = a.cols
         A = torch.from_numpy(synth.normal_matrix(M, K, seed=0, stream=10)).cuda()
@@ -270,6 +275,8 @@ def run_only(a) -> None:
         elif a.only == "gemm_ws":
             ws = torch.empty(bdr.mx_gemm_workspace_bytes(M, N, K), dtype=torch.uint8, device="cuda")
             ms = _time(lambda: bdr.mx_gemm_ws(cfg, pa, cfg, pb, M, N, K, c, ws), reps)
+        elif a.only == "gemm_hw":
+            ms = _time(lambda: bdr.mx_gemm_hw(cfg, pa, cfg, pb, M, N, K, c, r=64, f=25), reps)
         else:
             ms = _time(lambda: bdr.mx_gemm(cfg, pa, cfg, pb, M, N, K, c), reps)
         print("%s %s %dx%dx%d: %.4f ms per call, %.1f TFLOP/s, status %d" % (a.only, a.fmt, M, N, K, ms, 2.0 * M * N * K / ms / 1e9,

@@ -282,6 +282,23 @@ int bdr_reencode_e4m3(const bdr_config_t* cfg /*host*/, const bdr_planes_t* in /
 int mx_gemm_e4m3(const uint8_t* a, const uint8_t* scales_a, const uint8_t* b, const uint8_t* scales_b, int64_t M,
                  int64_t N, int64_t K, float* c, int64_t ldc, void* stream);
 
+/* C = A B^T as the dot-product pipeline of Section IV-B (Fig. 6) computes it, bit for bit, from the same packed
+ * operands as mx_gemm.  The paper describes the pipeline in words; this library's reading: inside a 16-element block
+ * the integer mantissa products are summed exactly, the two products of sub-block j entering with the weight
+ * 2^(2 - tau_A,j - tau_B,j) (the conditional right shifts by the microexponents); the r/16 block results of one pass
+ * (r consecutive elements of K) are aligned to the largest exponent sum F_A + F_B of the pass inside a frame of f
+ * magnitude bits whose top bit is the top bit of a block result at that exponent, truncated toward zero, and added
+ * as integers; the pass's sum is rounded to fp32 (nearest even) and passes are accumulated in fp32 in order of
+ * increasing K.  The paper chooses f = min(25, the format's dynamic range), which is 25 for every format with an
+ * 8-bit shared exponent.  With a frame wide enough for the exponent spread of a pass the result is the exact dot
+ * product of the dequantized operands rounded once per pass; narrower frames drop low bits of the smaller blocks.
+ * Table II formats (A and B may differ), r in {16, 32, 64}, 1 <= f <= 25, M and N multiples of 64, K a multiple of
+ * 64, c 16-byte aligned with ldc a multiple of 4.  A block with the exponent byte 0xFF makes its row's (column's)
+ * outputs NaN.  Runs on the ordinary arithmetic units (the alignment is per block and output), not the tensor cores. */
+int mx_gemm_hw(const bdr_config_t* cfg_a /*host*/, const bdr_planes_t* a /*host struct*/,
+               const bdr_config_t* cfg_b /*host*/, const bdr_planes_t* b /*host struct*/, int64_t M, int64_t N,
+               int64_t K, int r, int f, float* c, int64_t ldc, void* stream);
+
 /* BDR_OK, or BDR_ERR_TIMEOUT if any mx_gemm launch on the current device gave up a bounded wait
  * (sticky).  Host call; synchronises with the device (it copies one word back). */
 int mx_gemm_status(void);

@@ -22,7 +22,7 @@ F32, BF16 = 0, 1
 EXPORTS = ("bdr_strerror", "bdr_device_status", "bdr_packed_sizes", "bdr_quant_dequant", "bdr_pack", "bdr_unpack",
            "bdr_qsnr_workspace_bytes", "bdr_qsnr", "bdr_qsnr_static_max_cfgs", "bdr_qsnr_static", "mx_gemm",
            "mx_gemm_workspace_bytes", "mx_gemm_ws", "mx_gemm_f8_workspace_bytes", "mx_gemm_f8", "bdr_reencode_e4m3", "mx_gemm_e4m3", "bdr_set_workspace",
-           "mx_gemm_status", "bdr_selftest_bounded_wait", "bdr_selftest_host", "bdr_qsnr_from_sums", "bdr_pack2", "bdr_qsnr_delayed", "bdr_amax", "bdr_tile_packing_efficiency")
+           "mx_gemm_status", "bdr_selftest_bounded_wait", "bdr_selftest_host", "bdr_qsnr_from_sums", "bdr_pack2", "bdr_qsnr_delayed", "bdr_amax", "bdr_tile_packing_efficiency", "mx_gemm_hw")
 
 
 class BdrError(RuntimeError):
@@ -100,6 +100,9 @@ def lib():
         L.bdr_amax.argtypes = [C.c_void_p, C.c_int, C.c_int64, C.c_int64, C.c_int64, C.c_void_p, C.c_void_p]
         L.bdr_tile_packing_efficiency.restype = C.c_double
         L.bdr_tile_packing_efficiency.argtypes = [C.c_void_p, C.c_int64, C.c_int64]
+        L.mx_gemm_hw.restype = C.c_int
+        L.mx_gemm_hw.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_int64, C.c_int64, C.c_int, C.c_int,
+                                 C.c_void_p, C.c_int64, C.c_void_p]
         L.bdr_pack2.restype = C.c_int
         L.bdr_pack2.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int64, C.c_int64, C.c_int64, C.c_void_p, C.c_void_p,
                                 C.c_void_p, C.c_void_p, C.c_void_p]
@@ -301,6 +304,15 @@ def mx_gemm(cfg_a: Config, a: Planes, cfg_b: Config, b: Planes, M: int, N: int, 
     ca, cb, pa, pb = cfg_a.c(), cfg_b.c(), a.c(), b.c()
     _check(lib().mx_gemm(C.addressof(ca), C.addressof(pa), C.addressof(cb), C.addressof(pb), M, N, K, _ptr(c),
                          c.stride(0), _stream(stream)), "mx_gemm")
+    return c
+
+
+def mx_gemm_hw(cfg_a: Config, a: Planes, cfg_b: Config, b: Planes, M: int, N: int, K: int, c: torch.Tensor, r: int = 64, f: int = 25,
+               stream=None):
+    """c[M,N] (float32) = the product as the dot-product pipeline of Section IV-B computes it (pass length r, f-bit frame)."""
+    ca, cb, pa, pb = cfg_a.c(), cfg_b.c(), a.c(), b.c()
+    _check(lib().mx_gemm_hw(C.addressof(ca), C.addressof(pa), C.addressof(cb), C.addressof(pb), M, N, K, r, f, _ptr(c),
+                            c.stride(0), _stream(stream)), "mx_gemm_hw")
     return c
 
 
