@@ -717,8 +717,8 @@ int bdr_qsnr(const bdr_config_t* cfgs, int n_cfgs, const void* x, bdr_dtype_t dt
 int bdr_qsnr_delayed(const bdr_config_t* cfgs, int n_cfgs, const void* x, bdr_dtype_t dt, int64_t rows, int64_t cols, int64_t ld,
                      int axis, const float* amax_window_dev, int n_window, double* qsnr_db_dev, void* workspace,
                      int64_t workspace_bytes, void* stream) {
-    if (!amax_window_dev) return BDR_ERR_NULL;
     if (n_window < 1) return BDR_ERR_SIZE;
+    if (!amax_window_dev) return BDR_ERR_NULL;
     if ((uintptr_t)amax_window_dev % 4) return BDR_ERR_MISALIGNED;
     return qsnr_impl(cfgs, n_cfgs, x, dt, rows, cols, ld, axis, amax_window_dev, n_window, qsnr_db_dev, workspace, workspace_bytes,
                      stream);
