@@ -82,10 +82,12 @@ const char* bdr_strerror(int status);
 /* Kernels that stage data with asynchronous bulk copies wait for them with a bounded number of
  * polls.  A wait that runs out makes the warp stop early (its part of the output is then
  * incomplete) and leaves BDR_ERR_TIMEOUT in a sticky per-device word.  This host call returns
- * that word for the current device: BDR_OK, BDR_ERR_TIMEOUT, or BDR_ERR_CUDA if it cannot be read.
- * It synchronises with the device (one word is copied back), so call it after the work of
- * interest, not between launches. */
+ * that word for the current device: BDR_OK, BDR_ERR_TIMEOUT, BDR_ERR_SIZE (an index that bdr_gather_rows found
+ * outside its table), or BDR_ERR_CUDA if it cannot be read.  It synchronises with the device (one word is
+ * copied back), so call it after the work of interest, not between launches.  bdr_device_status_reset
+ * returns the word in the same way and clears it (the first failure sticks until then). */
 int bdr_device_status(void);
+int bdr_device_status_reset(void);
 
 /* Self-tests of the library's failure handling.  (The paper has no counterpart.)
  * bdr_selftest_bounded_wait queues a one-warp kernel that waits, with the same bounded wait the streaming
@@ -145,6 +147,15 @@ int bdr_pack2(const bdr_config_t* cfg /*host*/, const void* x, bdr_dtype_t dt, i
  * tensor; the inverse of bdr_pack's planes -> Q(x). */
 int bdr_unpack(const bdr_config_t* cfg /*host*/, const bdr_planes_t* in /*host struct*/, void* y, bdr_dtype_t dt,
                int64_t rows, int64_t cols, int64_t ld, int axis, void* stream);
+
+/* Rows of a packed table, decoded: y[i, :] = the dequantized row idx_dev[i] of a [n_rows, dim] table stored as axis-1
+ * planes (what bdr_pack(axis = 1) wrote), for i < n_idx.  Section V (inferencing): in memory-bound models such as
+ * recommendation models the embedding tables are kept in MX format as well, so a lookup reads (m+1) + 1 bits per
+ * element instead of 16 or 32.  idx_dev: n_idx int64 indices on the device; y [n_idx, ld] of `dt`.  Any POW2
+ * configuration.  An index outside [0, n_rows) cannot be seen by the host: its output row is filled with quiet
+ * NaNs and BDR_ERR_SIZE is left in the sticky word that bdr_device_status returns. */
+int bdr_gather_rows(const bdr_config_t* cfg /*host*/, const bdr_planes_t* table /*host struct*/, int64_t n_rows, int64_t dim,
+                    const int64_t* idx_dev, int64_t n_idx, void* y, bdr_dtype_t dt, int64_t ld, void* stream);
 
 /* Eq. 3 from accumulated sums: qsnr_db_dev[i] = -10 log10(sums_dev[2i] / sums_dev[2i+1]) for n pairs
  * {sum (Q(x)-x)^2, sum x^2} as bdr_quant_dequant / bdr_pack accumulate them (device pointers, 8-byte aligned;

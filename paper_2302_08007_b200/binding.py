@@ -22,7 +22,7 @@ F32, BF16 = 0, 1
 EXPORTS = ("bdr_strerror", "bdr_device_status", "bdr_packed_sizes", "bdr_quant_dequant", "bdr_pack", "bdr_unpack",
            "bdr_qsnr_workspace_bytes", "bdr_qsnr", "bdr_qsnr_static_max_cfgs", "bdr_qsnr_static", "mx_gemm",
            "mx_gemm_workspace_bytes", "mx_gemm_ws", "mx_gemm_f8_workspace_bytes", "mx_gemm_f8", "bdr_reencode_e4m3", "mx_gemm_e4m3", "bdr_set_workspace",
-           "mx_gemm_status", "bdr_selftest_bounded_wait", "bdr_selftest_host", "bdr_qsnr_from_sums", "bdr_pack2", "bdr_qsnr_delayed", "bdr_amax", "bdr_tile_packing_efficiency", "mx_gemm_hw")
+           "mx_gemm_status", "bdr_selftest_bounded_wait", "bdr_selftest_host", "bdr_qsnr_from_sums", "bdr_pack2", "bdr_qsnr_delayed", "bdr_amax", "bdr_tile_packing_efficiency", "mx_gemm_hw", "bdr_gather_rows", "bdr_device_status_reset")
 
 
 class BdrError(RuntimeError):
@@ -103,6 +103,9 @@ def lib():
         L.mx_gemm_hw.restype = C.c_int
         L.mx_gemm_hw.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_int64, C.c_int64, C.c_int, C.c_int,
                                  C.c_void_p, C.c_int64, C.c_void_p]
+        L.bdr_gather_rows.restype = C.c_int
+        L.bdr_gather_rows.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_int64, C.c_void_p, C.c_int64, C.c_void_p, C.c_int,
+                                      C.c_int64, C.c_void_p]
         L.bdr_pack2.restype = C.c_int
         L.bdr_pack2.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int64, C.c_int64, C.c_int64, C.c_void_p, C.c_void_p,
                                 C.c_void_p, C.c_void_p, C.c_void_p]
@@ -137,6 +140,8 @@ def lib():
         L.mx_gemm_status.argtypes = []
         L.bdr_device_status.restype = C.c_int
         L.bdr_device_status.argtypes = []
+        L.bdr_device_status_reset.restype = C.c_int
+        L.bdr_device_status_reset.argtypes = []
         L.bdr_selftest_bounded_wait.restype = C.c_int
         L.bdr_selftest_bounded_wait.argtypes = [C.c_void_p, C.c_void_p]
         L.bdr_selftest_host.restype = C.c_int
@@ -234,6 +239,15 @@ def bdr_pack2(cfg: Config, x: torch.Tensor, planes_rows: Planes, planes_cols: Pl
     _check(lib().bdr_pack2(C.addressof(c), _ptr(x2), _dt(x2), x2.shape[0], x2.shape[1], x2.stride(0), C.addressof(pr),
                            C.addressof(pc), _ptr(qsnr_sums_rows), _ptr(qsnr_sums_cols), _stream(stream)), "bdr_pack2")
     return planes_rows, planes_cols
+
+
+def bdr_gather_rows(cfg: Config, table: Planes, n_rows: int, idx: torch.Tensor, y: torch.Tensor, stream=None) -> torch.Tensor:
+    """y[i, :] = decoded row idx[i] of a packed [n_rows, dim] table (axis-1 planes); idx int64 on the device."""
+    assert idx.dtype == torch.int64 and idx.is_contiguous() and idx.is_cuda and y.dim() == 2 and y.shape[0] == idx.numel()
+    c, p = cfg.c(), table.c()
+    _check(lib().bdr_gather_rows(C.addressof(c), C.addressof(p), n_rows, y.shape[1], _ptr(idx), idx.numel(), _ptr(y), _dt(y),
+                                 y.stride(0), _stream(stream)), "bdr_gather_rows")
+    return y
 
 
 def bdr_unpack(cfg: Config, planes: Planes, y: torch.Tensor, axis: int = 1, stream=None) -> torch.Tensor:
@@ -375,6 +389,11 @@ def mx_gemm_e4m3(a: torch.Tensor, scales_a: torch.Tensor, b: torch.Tensor, scale
 def bdr_device_status() -> int:
     """Sticky per-device status of the kernels' bounded waits (0 = ok); synchronises."""
     return int(lib().bdr_device_status())
+
+
+def bdr_device_status_reset() -> int:
+    """Returns the sticky per-device status word and clears it; synchronises."""
+    return int(lib().bdr_device_status_reset())
 
 
 def bdr_qsnr_from_sums(sums: torch.Tensor, out_db: torch.Tensor, stream=None) -> torch.Tensor:

@@ -183,6 +183,14 @@ int bdr_device_status(void) {
     return v;
 }
 
+int bdr_device_status_reset(void) {
+    int* word = device_status_word();
+    int v = 0;
+    if (!word || cudaMemcpy(&v, word, sizeof(v), cudaMemcpyDeviceToHost) != cudaSuccess) return BDR_ERR_CUDA;
+    if (v != 0 && cudaMemset(word, 0, sizeof(v)) != cudaSuccess) return BDR_ERR_CUDA;
+    return v;
+}
+
 int bdr_selftest_bounded_wait(int* status_dev, void* stream) {
     if (!status_dev) return BDR_ERR_NULL;
     if ((uintptr_t)status_dev % 4) return BDR_ERR_MISALIGNED;
@@ -298,6 +306,24 @@ int bdr_pack2(const bdr_config_t* cfg, const void* x, bdr_dtype_t dt, int64_t ro
     rc = quant_dispatch<__nv_bfloat16>(qp, (const __nv_bfloat16*)x, nullptr, rows, cols, ld, 1, out_rows, tight_r, qsnr_sums_rows_dev, st);
     if (rc) return rc;
     return quant_dispatch<__nv_bfloat16>(qp, (const __nv_bfloat16*)x, nullptr, rows, cols, ld, 0, out_cols, tight_c, qsnr_sums_cols_dev, st);
+}
+
+int bdr_gather_rows(const bdr_config_t* cfg, const bdr_planes_t* table, int64_t n_rows, int64_t dim, const int64_t* idx_dev,
+                    int64_t n_idx, void* y, bdr_dtype_t dt, int64_t ld, void* stream) {
+    QParams qp;
+    int rc = check_pow2_config(cfg, &qp);
+    if (rc) return rc;
+    if (n_rows < 0 || n_idx < 0) return BDR_ERR_SIZE;
+    if ((rc = check_tensor(y, dt, n_idx, dim, ld, 1))) return rc;
+    if (n_idx == 0 || dim == 0) return BDR_OK;
+    if (!idx_dev) return BDR_ERR_NULL;
+    if ((uintptr_t)idx_dev % 8) return BDR_ERR_MISALIGNED;
+    if ((rc = check_planes(cfg, table, dim))) return rc;
+    int* status = device_status_word();
+    if (!status) return BDR_ERR_CUDA;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (dt == BDR_F32) return gather_rows_general<float>(*table, n_rows, idx_dev, (float*)y, n_idx, dim, ld, qp, status, st);
+    return gather_rows_general<__nv_bfloat16>(*table, n_rows, idx_dev, (__nv_bfloat16*)y, n_idx, dim, ld, qp, status, st);
 }
 
 int bdr_unpack(const bdr_config_t* cfg, const bdr_planes_t* in, void* y, bdr_dtype_t dt, int64_t rows, int64_t cols,

@@ -94,6 +94,50 @@ unpack_general_kernel(bdr_planes_t in, T* y, int64_t nlines, int64_t len, int64_
     }
 }
 
+// Row gather from a packed table (axis-1 planes of [n_rows, len]): output line l is the decoded row idx[l].
+// One thread per element; an index outside the table gives a row of quiet NaNs and leaves BDR_ERR_SIZE in *status.
+template <typename T>
+__global__ void __launch_bounds__(kGenThreads)
+gather_rows_kernel(bdr_planes_t in, int64_t n_rows, const int64_t* idx, T* y, int64_t n_idx, int64_t len, int64_t ld, QParams qp,
+                   int* status) {
+    const int nsub = qp.k1 / qp.k2;
+    const int64_t total = n_idx * len;
+    for (int64_t g = (int64_t)blockIdx.x * kGenThreads + threadIdx.x; g < total; g += (int64_t)gridDim.x * kGenThreads) {
+        const int64_t l = g / len, i = g - l * len;
+        const int64_t line = idx[l];
+        uint32_t yb = 0x7FC00000u;
+        if (line < 0 || line >= n_rows) {
+            if (i == 0) atomicCAS(status, 0, (int)BDR_ERR_SIZE);
+        } else {
+            const int64_t b = i / qp.k1;
+            const int F = in.exps[line * in.ld_exps + b];
+            if (F != 255) {
+                const int64_t j = b * nsub + (i - b * qp.k1) / qp.k2;
+                const int tau = qp.d2 ? (int)get_bits(in.micro + line * in.ld_micro, j * (int64_t)qp.d2, qp.d2) : 0;
+                const uint32_t code = get_bits(in.elems + line * in.ld_elems, i * (int64_t)(qp.m + 1), qp.m + 1);
+                const uint32_t q = code & qp.qmax;
+                const int p = max(F - 127 - tau - (qp.m - 1), -149);
+                yb = __float_as_uint(__fmul_rn(__uint2float_rn(q), __uint_as_float(pow2_bits(p)))) | ((code >> qp.m) << 31);
+            }
+        }
+        Elem<T>::store_bits(y + l * ld + i, yb);
+    }
+}
+
+template <typename T>
+int gather_rows_general(const bdr_planes_t& in, int64_t n_rows, const int64_t* idx, T* y, int64_t n_idx, int64_t len, int64_t ld,
+                        const QParams& qp, int* status, cudaStream_t st) {
+    const int64_t total = n_idx * len;
+    if (total == 0) return BDR_OK;
+    const int grid = (int)max((int64_t)1, min((total + kGenThreads - 1) / kGenThreads, (int64_t)sm_count() * 16));
+    gather_rows_kernel<T><<<grid, kGenThreads, 0, st>>>(in, n_rows, idx, y, n_idx, len, ld, qp, status);
+    return cudaGetLastError() == cudaSuccess ? BDR_OK : BDR_ERR_CUDA;
+}
+template int gather_rows_general<float>(const bdr_planes_t&, int64_t, const int64_t*, float*, int64_t, int64_t, int64_t, const QParams&, int*,
+                                        cudaStream_t);
+template int gather_rows_general<__nv_bfloat16>(const bdr_planes_t&, int64_t, const int64_t*, __nv_bfloat16*, int64_t, int64_t, int64_t,
+                                                const QParams&, int*, cudaStream_t);
+
 template <typename T>
 int quant_general(const T* x, T* y, int64_t rows, int64_t cols, int64_t ld, int axis, const bdr_planes_t* out,
                   const QParams& qp, double* sums, cudaStream_t st) {
