@@ -183,10 +183,10 @@ def linear_leg(args) -> dict:
     tensor = float(peaks.get("bf16_tflops_sustained", peaks.get("bf16_tflops", 1590.0)))   # a kernel inside a long step
 
     def roofline(m_bits, t_ms, tensor_peak, what):
-        # the step's floor: every operand read once per direction and its planes written (2 + bits/8 bytes per element
-        # and direction) at the HBM peak, plus the three products at the tensor peak
+        # the step's floor: every operand read once and both its packed copies written (2 + 2 bits/8 bytes per element:
+        # bdr_pack2) at the HBM peak, plus the three products at the tensor peak
         n_el = tokens * d_in + d_out * d_in + tokens * d_out
-        qbytes = 2 * n_el * (2.0 + (m_bits + 2) / 8.0)
+        qbytes = n_el * (2.0 + 2.0 * (m_bits + 2) / 8.0)
         floor_ms = qbytes / (hbm * 1e9) * 1e3 + flops / (tensor_peak * 1e12) * 1e3
         return {"bound": "tensor", "achieved": flops / (t_ms * 1e-3) / 1e12, "peak": tensor_peak, "unit": "TFLOP/s",
                 "frac": floor_ms / t_ms, "floor_ms": floor_ms, "quantization_bytes": qbytes, "flops": flops,
@@ -297,6 +297,7 @@ def run_only(a) -> None:
     planes = bdr.alloc_planes(cfg, a.rows, a.cols, a.axis)
     planes2 = bdr.alloc_planes(cfg, a.rows, a.cols, 1 - a.axis) if a.only == "pack2" else None
     sums = None if a.no_sums else torch.zeros(2, dtype=torch.float64, device="cuda")
+    sums2 = None if a.no_sums else torch.zeros(2, dtype=torch.float64, device="cuda")
     bdr.bdr_pack(cfg, x, planes, axis=a.axis)
 
     def once():
@@ -305,7 +306,7 @@ def run_only(a) -> None:
         elif a.only == "pack":
             bdr.bdr_pack(cfg, x, planes, axis=a.axis, qsnr_sums=sums)
         elif a.only == "pack2":
-            bdr.bdr_pack2(cfg, x, planes if a.axis == 1 else planes2, planes2 if a.axis == 1 else planes)
+            bdr.bdr_pack2(cfg, x, planes if a.axis == 1 else planes2, planes2 if a.axis == 1 else planes, sums, sums2)
         else:
             bdr.bdr_unpack(cfg, planes, y, axis=a.axis)
 
