@@ -122,6 +122,16 @@ int bdr_quant_dequant(const bdr_config_t* cfg /*host*/, const void* x, void* y, 
                       int64_t rows, int64_t cols, int64_t ld, int axis, double* qsnr_sums_dev,
                       void* stream);
 
+/* Three-level scaling, the extension sketched at the end of Section III: a software FP32 parent scale over groups of
+ * k_parent consecutive elements of a line (the paper: "an even coarser granularity at up to ~1K") above the power-of-two
+ * block scale and the microexponents.  This library's reading: the parent scale maps the group's largest magnitude onto
+ * the largest value a block with exponent 0 can hold, V = (2^m - 1) 2^-(m-1):  s = amax_g / V,  x' = x / s,
+ * y = Q(x') s with Q the two-level quantizer of bdr_quant_dequant (IEEE fp32 division and multiplication).  Arguments
+ * as bdr_quant_dequant.  fp32 tensors, k1 <= 16, k_parent a multiple of 16 (and of k1) up to 1024; a correctness-grade
+ * kernel (one warp per group), meant for fidelity studies. */
+int bdr_quant_dequant_parent(const bdr_config_t* cfg /*host*/, int k_parent, const void* x, void* y, bdr_dtype_t dt,
+                             int64_t rows, int64_t cols, int64_t ld, int axis, double* qsnr_sums_dev, void* stream);
+
 /* Quantize and write the packed planes (layout above); optionally also the dequantized tensor
  * (y_dq, same dtype/pitch as x, may be NULL) and the Eq. 3 sums.  Every byte of every plane line
  * up to its pitch is written (padding bytes are zero). */

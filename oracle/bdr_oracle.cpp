@@ -665,4 +665,49 @@ int orc_gemm_hw(const orc_config* ca, const float* a, int64_t M, const orc_confi
     return ORC_OK;
 }
 
+// Three-level scaling (Section III, last paragraph: an extension the paper only sketches): a software FP32
+// parent scale over groups of k_parent consecutive elements of a line, above the power-of-two block scale and
+// the microexponents.  Reading: the parent scale maps the group's largest magnitude onto the largest value a
+// block with exponent 0 can hold, V = (2^m - 1) 2^-(m-1):  s = fl(amax_g / V),  x' = fl(x / s),
+// Q3(x) = fl(Q(x') s) with Q the two-level quantizer on the group's k1-blocks.  A group of zeros stays zeros.
+int orc_quant_dequant_parent(const orc_config* c, int64_t k_parent, const float* x, float* y, int64_t rows, int64_t cols,
+                             int64_t ld, int axis, double* sums) {
+    if (!config_ok(c) || c->scale_kind != ORC_POW2 || !x || !y || rows < 0 || cols < 0 || ld < cols || (axis != 0 && axis != 1))
+        return ORC_BAD;
+    if (k_parent < c->k1 || k_parent % c->k1 != 0) return ORC_BAD;
+    LineView v = make_view(rows, cols, ld, axis);
+    const float V = (float)((1 << c->m) - 1) * std::ldexp(1.0f, -(c->m - 1));
+    std::vector<float> xs(k_parent), qs(k_parent);
+    for (int64_t l = 0; l < v.nlines; ++l)
+        for (int64_t g0 = 0; g0 < v.len; g0 += k_parent) {
+            const int64_t n = std::min<int64_t>(k_parent, v.len - g0);
+            const float* xg = x + l * v.line_stride + g0 * v.elem_stride;
+            float* yg = y + l * v.line_stride + g0 * v.elem_stride;
+            const float amax = absmax(xg, v.elem_stride, n);
+            const float s = amax / V;
+            if (!(s > 0.f)) {
+                for (int64_t i = 0; i < n; ++i) yg[i * v.elem_stride] = with_sign(0.f, xg[i * v.elem_stride]);
+                continue;
+            }
+            for (int64_t i = 0; i < n; ++i) xs[i] = xg[i * v.elem_stride] / s;
+            for (int64_t b0 = 0; b0 < n; b0 += c->k1) {
+                const int nb = (int)std::min<int64_t>(c->k1, n - b0);
+                pow2_block(*c, xs.data() + b0, 1, nb, nullptr, nullptr, nullptr, qs.data() + b0, 1);
+            }
+            for (int64_t i = 0; i < n; ++i) yg[i * v.elem_stride] = qs[i] * s;
+        }
+    if (sums) {
+        double e2 = 0.0, s2 = 0.0;
+        for (int64_t r = 0; r < rows; ++r)
+            for (int64_t cc = 0; cc < cols; ++cc) {
+                double a = (double)x[r * ld + cc], q = (double)y[r * ld + cc];
+                e2 += (q - a) * (q - a);
+                s2 += a * a;
+            }
+        sums[0] = e2;
+        sums[1] = s2;
+    }
+    return ORC_OK;
+}
+
 }  // extern "C"

@@ -228,3 +228,19 @@ def gemm_hw(cfg_a: Config, a, cfg_b: Config, b, r: int = 64, f: int = 25):
     if rc != 0:
         raise ValueError("oracle rejected the configuration or arguments")
     return c
+
+
+def quant_dequant_parent(cfg: Config, k_parent: int, x, axis: int = 1):
+    """Three-level scaling: an FP32 parent scale per k_parent elements of a line above the two-level quantizer.
+    Returns (y fp32, (sum_err2, sum_sig2))."""
+    x = _f32(x)
+    x2 = x.reshape(1, -1) if x.ndim == 1 else x
+    rows, cols = x2.shape
+    y = np.empty_like(x2)
+    sums = np.zeros(2, dtype=np.float64)
+    c = cfg.c()
+    rc = lib().orc_quant_dequant_parent(C.byref(c), _i64(k_parent), _p(x2), _p(y), _i64(rows), _i64(cols), _i64(cols), C.c_int(axis),
+                                        _p(sums))
+    if rc != 0:
+        raise ValueError("oracle rejected the configuration or arguments")
+    return y.reshape(x.shape), (float(sums[0]), float(sums[1]))

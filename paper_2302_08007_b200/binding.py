@@ -22,7 +22,7 @@ F32, BF16 = 0, 1
 EXPORTS = ("bdr_strerror", "bdr_device_status", "bdr_packed_sizes", "bdr_quant_dequant", "bdr_pack", "bdr_unpack",
            "bdr_qsnr_workspace_bytes", "bdr_qsnr", "bdr_qsnr_static_max_cfgs", "bdr_qsnr_static", "mx_gemm",
            "mx_gemm_workspace_bytes", "mx_gemm_ws", "mx_gemm_f8_workspace_bytes", "mx_gemm_f8", "bdr_reencode_e4m3", "mx_gemm_e4m3", "bdr_set_workspace",
-           "mx_gemm_status", "bdr_selftest_bounded_wait", "bdr_selftest_host", "bdr_qsnr_from_sums", "bdr_pack2", "bdr_qsnr_delayed", "bdr_amax", "bdr_tile_packing_efficiency", "mx_gemm_hw", "bdr_gather_rows", "bdr_device_status_reset")
+           "mx_gemm_status", "bdr_selftest_bounded_wait", "bdr_selftest_host", "bdr_qsnr_from_sums", "bdr_pack2", "bdr_qsnr_delayed", "bdr_amax", "bdr_tile_packing_efficiency", "mx_gemm_hw", "bdr_gather_rows", "bdr_device_status_reset", "bdr_quant_dequant_parent")
 
 
 class BdrError(RuntimeError):
@@ -103,6 +103,9 @@ def lib():
         L.mx_gemm_hw.restype = C.c_int
         L.mx_gemm_hw.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_int64, C.c_int64, C.c_int, C.c_int,
                                  C.c_void_p, C.c_int64, C.c_void_p]
+        L.bdr_quant_dequant_parent.restype = C.c_int
+        L.bdr_quant_dequant_parent.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_int, C.c_int64, C.c_int64, C.c_int64,
+                                               C.c_int, C.c_void_p, C.c_void_p]
         L.bdr_gather_rows.restype = C.c_int
         L.bdr_gather_rows.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_int64, C.c_void_p, C.c_int64, C.c_void_p, C.c_int,
                                       C.c_int64, C.c_void_p]
@@ -239,6 +242,19 @@ def bdr_pack2(cfg: Config, x: torch.Tensor, planes_rows: Planes, planes_cols: Pl
     _check(lib().bdr_pack2(C.addressof(c), _ptr(x2), _dt(x2), x2.shape[0], x2.shape[1], x2.stride(0), C.addressof(pr),
                            C.addressof(pc), _ptr(qsnr_sums_rows), _ptr(qsnr_sums_cols), _stream(stream)), "bdr_pack2")
     return planes_rows, planes_cols
+
+
+def bdr_quant_dequant_parent(cfg: Config, k_parent: int, x: torch.Tensor, y: torch.Tensor | None, axis: int = 1,
+                             qsnr_sums: torch.Tensor | None = None, stream=None):
+    """Three-level scaling: FP32 parent scale per k_parent elements of a line above the two-level quantizer (fp32 tensors)."""
+    x2 = _as2d(x)
+    y2 = _as2d(y) if y is not None else None
+    if y2 is not None and (y2.shape != x2.shape or y2.stride(0) != x2.stride(0) or y2.dtype != x2.dtype):
+        raise ValueError("y must match x in shape, pitch and dtype")
+    c = cfg.c()
+    _check(lib().bdr_quant_dequant_parent(C.addressof(c), k_parent, _ptr(x2), _ptr(y2), _dt(x2), x2.shape[0], x2.shape[1], x2.stride(0),
+                                          axis, _ptr(qsnr_sums), _stream(stream)), "bdr_quant_dequant_parent")
+    return y
 
 
 def bdr_gather_rows(cfg: Config, table: Planes, n_rows: int, idx: torch.Tensor, y: torch.Tensor, stream=None) -> torch.Tensor:

@@ -308,6 +308,20 @@ int bdr_pack2(const bdr_config_t* cfg, const void* x, bdr_dtype_t dt, int64_t ro
     return quant_dispatch<__nv_bfloat16>(qp, (const __nv_bfloat16*)x, nullptr, rows, cols, ld, 0, out_cols, tight_c, qsnr_sums_cols_dev, st);
 }
 
+int bdr_quant_dequant_parent(const bdr_config_t* cfg, int k_parent, const void* x, void* y, bdr_dtype_t dt, int64_t rows, int64_t cols,
+                             int64_t ld, int axis, double* qsnr_sums_dev, void* stream) {
+    QParams qp;
+    int rc = check_pow2_config(cfg, &qp);
+    if (rc) return rc;
+    if (k_parent < cfg->k1 || k_parent % cfg->k1 != 0) return BDR_ERR_BAD_CONFIG;
+    if ((rc = check_tensor(x, dt, rows, cols, ld, axis))) return rc;
+    if (dt != BDR_F32 || cfg->k1 > 16 || k_parent > 1024 || k_parent % 16 != 0) return BDR_ERR_UNSUPPORTED;
+    if (rows == 0 || cols == 0) return BDR_OK;
+    if (!y && !qsnr_sums_dev) return BDR_ERR_NULL;
+    if ((y && (uintptr_t)y % 4) || (qsnr_sums_dev && (uintptr_t)qsnr_sums_dev % 8)) return BDR_ERR_MISALIGNED;
+    return quant_parent_scale((const float*)x, (float*)y, rows, cols, ld, axis, k_parent, qp, qsnr_sums_dev, (cudaStream_t)stream);
+}
+
 int bdr_gather_rows(const bdr_config_t* cfg, const bdr_planes_t* table, int64_t n_rows, int64_t dim, const int64_t* idx_dev,
                     int64_t n_idx, void* y, bdr_dtype_t dt, int64_t ld, void* stream) {
     QParams qp;

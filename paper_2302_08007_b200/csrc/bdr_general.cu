@@ -94,6 +94,87 @@ unpack_general_kernel(bdr_planes_t in, T* y, int64_t nlines, int64_t len, int64_
     }
 }
 
+// Three-level scaling (Section III, last paragraph): an FP32 parent scale per group of k_parent consecutive elements of a
+// line above the two-level quantizer.  One warp per group (k_parent <= 1024): a lane holds the group's 16-element slices
+// lane, lane + 32; group maximum by shuffle; s = amax / V with V = (2^m - 1) 2^-(m-1); x' = x / s (IEEE division); the
+// two-level quantizer on x' (k1 <= 16: the blocks of a slice; the exact integer formulation); y = Q(x') s.
+__global__ void __launch_bounds__(kGenThreads)
+parent_scale_kernel(const float* x, float* y, int64_t nlines, int64_t len, int64_t line_stride, int64_t elem_stride, int k_parent,
+                    QParams qp, double* sums) {
+    const int lane = threadIdx.x & 31;
+    const int64_t warp0 = ((int64_t)blockIdx.x * kGenThreads + threadIdx.x) >> 5, nwarps = ((int64_t)gridDim.x * kGenThreads) >> 5;
+    const int64_t gpl = (len + k_parent - 1) / k_parent, total = nlines * gpl;
+    const float V = (float)qp.qmax * __uint_as_float((uint32_t)(127 - (qp.m - 1)) << 23);
+    double e2 = 0.0, s2 = 0.0;
+    for (int64_t g = warp0; g < total; g += nwarps) {
+        const int64_t line = g / gpl, g0 = (g - line * gpl) * k_parent;
+        const int n = (int)min((int64_t)k_parent, len - g0);
+        const float* xg = x + line * line_stride + g0 * elem_stride;
+        float* yg = y ? y + line * line_stride + g0 * elem_stride : nullptr;
+        uint32_t u[2][kSlice];
+        uint32_t am = 0;
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            const int e0 = (lane + 32 * h) * kSlice;
+            load_slice_guarded(xg + (int64_t)e0 * elem_stride, elem_stride, max(0, min(kSlice, n - e0)), u[h]);
+#pragma unroll
+            for (int i = 0; i < kSlice; ++i) am = max(am, u[h][i] & 0x7FFFFFFFu);
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) am = max(am, __shfl_xor_sync(0xFFFFFFFFu, am, o));
+        const float s = __fdiv_rn(__uint_as_float(am), V);
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            const int e0 = (lane + 32 * h) * kSlice;
+            const int cnt = max(0, min(kSlice, n - e0));
+            if (cnt == 0) continue;
+            uint32_t yb[kSlice];
+            if (!(s > 0.f)) {
+#pragma unroll
+                for (int i = 0; i < kSlice; ++i) yb[i] = u[h][i] & 0x80000000u;
+            } else {
+                uint32_t xs[kSlice];
+#pragma unroll
+                for (int i = 0; i < kSlice; ++i) xs[i] = __float_as_uint(__fdiv_rn(__uint_as_float(u[h][i]), s));
+                for (int b0 = 0; b0 < kSlice; b0 += qp.k1) {        // the slice's k1-blocks (k1 <= 16)
+                    int F = 0;
+                    for (int i = 0; i < qp.k1; ++i) F = max(F, exp_field(xs[b0 + i]));
+                    for (int j0 = b0; j0 < b0 + qp.k1; j0 += qp.k2) {
+                        int Fj = 0;
+                        for (int i = 0; i < qp.k2; ++i) Fj = max(Fj, exp_field(xs[j0 + i]));
+                        const int tau = F == 255 ? 0 : min(F - Fj, qp.beta);
+                        for (int i = 0; i < qp.k2; ++i) {
+                            uint32_t q = 0, yq = 0x7FC00000u;
+                            if (F != 255) quant_elem_exact(xs[j0 + i], F, tau, qp, q, yq);
+                            yb[j0 + i] = __float_as_uint(__fmul_rn(__uint_as_float(yq), s));
+                        }
+                    }
+                }
+            }
+            if (yg) store_slice_guarded(yg + (int64_t)e0 * elem_stride, elem_stride, cnt, yb);
+            if (sums) {
+                for (int i = 0; i < cnt; ++i) {
+                    const double a = (double)__uint_as_float(u[h][i]), d = (double)__uint_as_float(yb[i]) - a;
+                    e2 = fma(d, d, e2);
+                    s2 = fma(a, a, s2);
+                }
+            }
+        }
+    }
+    if (sums) block_accumulate_sums(e2, s2, sums);
+}
+
+int quant_parent_scale(const float* x, float* y, int64_t rows, int64_t cols, int64_t ld, int axis, int k_parent, const QParams& qp,
+                       double* sums, cudaStream_t st) {
+    const int64_t nlines = axis == 1 ? rows : cols, len = axis == 1 ? cols : rows;
+    const int64_t line_stride = axis == 1 ? ld : 1, elem_stride = axis == 1 ? 1 : ld;
+    const int64_t groups = nlines * ((len + k_parent - 1) / k_parent);
+    if (groups == 0) return BDR_OK;
+    const int grid = (int)max((int64_t)1, min((groups * 32 + kGenThreads - 1) / kGenThreads, (int64_t)sm_count() * 16));
+    parent_scale_kernel<<<grid, kGenThreads, 0, st>>>(x, y, nlines, len, line_stride, elem_stride, k_parent, qp, sums);
+    return cudaGetLastError() == cudaSuccess ? BDR_OK : BDR_ERR_CUDA;
+}
+
 // Row gather from a packed table (axis-1 planes of [n_rows, len]): output line l is the decoded row idx[l].
 // One thread per element; an index outside the table gives a row of quiet NaNs and leaves BDR_ERR_SIZE in *status.
 template <typename T>

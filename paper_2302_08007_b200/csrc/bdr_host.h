@@ -92,6 +92,10 @@ template <typename T>
 int unpack_general(const bdr_planes_t& in, T* y, int64_t rows, int64_t cols, int64_t ld, int axis, const QParams& qp,
                    cudaStream_t st);
 
+// FP32 parent scale per k_parent elements above the two-level quantizer, fp32 tensors, k1 <= 16 (bdr_general.cu)
+int quant_parent_scale(const float* x, float* y, int64_t rows, int64_t cols, int64_t ld, int axis, int k_parent, const QParams& qp,
+                       double* sums, cudaStream_t st);
+
 // rows of a packed table selected by device-side indices (bdr_general.cu)
 template <typename T>
 int gather_rows_general(const bdr_planes_t& in, int64_t n_rows, const int64_t* idx, T* y, int64_t n_idx, int64_t len, int64_t ld,

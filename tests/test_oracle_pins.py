@@ -695,6 +695,50 @@ def test_hw_dot_truncation_is_bounded_ordered_and_pass_structured():
         orc.gemm_hw(orc.MX6, a, orc.MX9._replace(k2=4) if hasattr(orc.MX9, "_replace") else Cfg(16, 8, 4, 1, 7), b)
 
 
+# ---- three-level scaling: FP32 parent scale above the block scale (Section III, extension) ---------------------------
+def test_parent_scale_hand_worked_group_and_reductions():
+    # k1 = 4, k2 = 2, d2 = 1, m = 3: V = 7/4.  Group maximum 5.25 -> s = 3 exactly; x/3 = [1.75 1 | -.5 .25] [.2 -.3 | .1 .0333]
+    # block 0: F 127, tau [0 1], q [7 4 | -4 2]: exact.  block 1: F 125 (0.3), units 1/16 and 1/32: 3.2 -> 3, 4.8 -> 5, 3.2 -> 3,
+    # 1.07 -> 1: [.1875 -.3125 | .09375 .03125]; times 3.  (Worked by hand; without the parent scale 5.25 -> 5 and 0.75 -> 1.)
+    cfg = Cfg(4, 8, 2, 1, 3)
+    x = np.array([5.25, 3.0, -1.5, 0.75, 0.6, -0.9, 0.3, 0.1], dtype=np.float32)
+    y, _ = orc.quant_dequant_parent(cfg, 8, x)
+    assert y.tolist() == [5.25, 3.0, -1.5, 0.75, 0.5625, -0.9375, 0.28125, 0.09375]
+    assert orc.quant_dequant(cfg, x)[0].tolist()[:4] == [5.0, 3.0, -1.5, 1.0]
+    # a group maximum of V 2^t makes the parent scale a power of two: the two-level quantizer itself (scale equivariance)
+    for cfg in (orc.MX4, orc.MX6, orc.MX9, Cfg(16, 8, 4, 2, 5)):
+        V = (2 ** cfg.m - 1) * 2.0 ** -(cfg.m - 1)
+        x = synth.normal_matrix(8, 512, 97).clip(-1.7, 1.7)
+        for r in range(8):
+            x[r, 37 * r] = V * 2.0 ** (r - 3)
+            x[r] = np.clip(x[r], -V * 2.0 ** (r - 3), V * 2.0 ** (r - 3))
+        for kp in (512, 128):
+            xx = x.copy()
+            if kp == 128:                                   # every group of 128 needs its own maximum of that form
+                xx[:, ::128] = (V * 2.0 ** (np.arange(8) - 3))[:, None]
+            y3, s3 = orc.quant_dequant_parent(cfg, kp, xx)
+            y2, s2 = orc.quant_dequant(cfg, xx)
+            assert np.array_equal(y3.view(np.uint32), y2.view(np.uint32)) and s3 == s2
+    # the group's largest element comes back within a rounding of the two divisions / multiplications; zeros stay zeros
+    x = synth.variable_variance_vectors(64, 1024, 98)
+    x[5] = 0.0
+    x[5, 3] = -0.0
+    for cfg in (orc.MX4, orc.MX9):
+        y, _ = orc.quant_dequant_parent(cfg, 1024, x)
+        i = np.abs(x).argmax(axis=1)
+        top, got = x[np.arange(64), i], y[np.arange(64), i]
+        ok = top != 0
+        assert np.all(np.abs(got[ok] - top[ok]) <= 4 * np.spacing(np.abs(top[ok])))
+        assert not y[5].any() and np.signbit(y[5, 3])
+    # lines are independent and the column direction is the row direction of the transpose
+    xm = synth.normal_matrix(64, 48, 99)
+    a, sa = orc.quant_dequant_parent(orc.MX6, 32, xm, axis=0)
+    b, sb = orc.quant_dequant_parent(orc.MX6, 32, np.ascontiguousarray(xm.T), axis=1)
+    assert np.array_equal(a, b.T) and sa == pytest.approx(sb, rel=1e-12)
+    with pytest.raises(ValueError):
+        orc.quant_dequant_parent(orc.MX6, 24, xm)
+
+
 # ---- GEMM reference ---------------------------------------------------------------------------------------------
 def test_gemm_reference_is_the_plain_definition():
     rng = np.random.default_rng(80)
