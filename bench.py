@@ -38,15 +38,15 @@ FALLBACK_BF16_TFLOPS = 1590.0
 # profiles/step_kernels_dram_traffic.md.  Writes that still sit in L2 when a kernel ends are not
 # counted by those counters, which is why some figures are below the algorithmic bytes.
 NCU_TRAFFIC_BYTES: dict[str, float | None] = {
-    "quant_dequant_MX4_row": 216616960, "quant_dequant_MX4_col": 216386048,
-    "quant_dequant_MX6_row": 216921600, "quant_dequant_MX6_col": 216279296,
-    "quant_dequant_MX9_row": 218355200, "quant_dequant_MX9_col": 216524800,
-    "pack_MX4_row": 148879104, "pack_MX4_col": 146531584,
-    "pack_MX6_row": 157287936, "pack_MX6_col": 154167808,
-    "pack_MX9_row": 173157376, "pack_MX9_col": 168432640,
-    "unpack_MX4_row": 111313664, "unpack_MX4_col": 108342528,
-    "unpack_MX6_row": 130237440, "unpack_MX6_col": 126141952,
-    "unpack_MX9_row": 154232832, "unpack_MX9_col": 151379968,
+    "quant_dequant_MX4_row": 216465664, "quant_dequant_MX4_col": 216645888,
+    "quant_dequant_MX6_row": 216837632, "quant_dequant_MX6_col": 215354368,
+    "quant_dequant_MX9_row": 216819712, "quant_dequant_MX9_col": 216272128,
+    "pack_MX4_row": 149406720, "pack_MX4_col": 146402560,
+    "pack_MX6_row": 157472768, "pack_MX6_col": 154135808,
+    "pack_MX9_row": 173253888, "pack_MX9_col": 168272128,
+    "unpack_MX4_row": 111284224, "unpack_MX4_col": 108499968,
+    "unpack_MX6_row": 128216832, "unpack_MX6_col": 125247232,
+    "unpack_MX9_row": 154121472, "unpack_MX9_col": 151368960,
 }
 
 
@@ -298,6 +298,18 @@ def run_ours(args):
     for s in range(args.warmup):
         step(s)
     barrier()
+    if args.step_only:   # for a profiler's launch list: nothing but the step's launches
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        ev0.record()
+        for s in range(args.steps):
+            step(s)
+        ev1.record()
+        barrier()
+        if rank == 0:
+            print("step only: %d steps of %d launches, %.4f ms per step" % (args.steps, len(ops), ev0.elapsed_time(ev1) / args.steps))
+        if world > 1:
+            dist.destroy_process_group()
+        return
 
     sampler = ClockSampler(local_rank)
     if rank == 0:
@@ -492,6 +504,7 @@ def main():
     ap.add_argument("--no-graph", action="store_true", help="launch every kernel from Python instead of replaying a CUDA graph of the step")
     ap.add_argument("--only", default=None, choices=["quant_dequant", "pack", "unpack", "pack2", "gemm", "gemm_ws", "gemm_f8", "gemm_hw", "sweep"],
                     help="run one operation a few times on a seeded tensor and print its time (for profilers); no JSON line")
+    ap.add_argument("--step-only", action="store_true", help="run only the warm-up and the timed steps (18 launches each) and print the time; no JSON line")
     ap.add_argument("--fmt", default="MX6", choices=["MX4", "MX6", "MX9"])
     ap.add_argument("--axis", type=int, default=1)
     ap.add_argument("--dtype", default="bf16", choices=["bf16", "f32"])

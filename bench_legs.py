@@ -221,11 +221,11 @@ def c1_leg(args) -> dict:
     call = lambda: bdr.bdr_pack(bdr.MX6, x, planes, axis=1, y_dq=y, qsnr_sums=sums)
     call()
     torch.cuda.synchronize()
-    us_stream = _time(call, reps=500, warmup=20) * 1e3          # back-to-back calls from Python
+    us_stream = _time(call, reps=200, warmup=20) * 1e3          # back-to-back calls from Python
     g = torch.cuda.CUDAGraph()
     with torch.cuda.graph(g):
         call()
-    us_graph = _time(g.replay, reps=500, warmup=20) * 1e3       # the launch alone, replayed
+    us_graph = _time(g.replay, reps=200, warmup=20) * 1e3       # the launch alone, replayed
     lat = []
     for _ in range(50):                                         # one call, then wait for it: what a lone caller sees
         torch.cuda.synchronize()

@@ -143,12 +143,12 @@ mx_gemm_hw_kernel(bdr_planes_t a, bdr_planes_t b, int64_t K, int r, int f, float
                     base[i][j] = fbase - emax[i][j];
                 }
             for (int bb = b0; bb < b0 + bpr; ++bb) {
-                unsigned long long D2[4][2];  // (row i; columns 0, 1) and (row i; columns 2, 3)
-#pragma unroll
-                for (int i = 0; i < 4; ++i) D2[i][0] = D2[i][1] = 0ull;
                 const int swz = (bb >> 1) << 4;  // the half (32 elements) this block belongs to
                 const float* ap = As + (16 * bb) * kHwTile + ((4 * ty) ^ swz);
                 const float* bp = Bs + (16 * bb) * kHwTile + ((4 * tx) ^ swz);
+                unsigned long long D2[4][2];  // (row i; columns 0, 1) and (row i; columns 2, 3)
+#pragma unroll
+                for (int i = 0; i < 4; ++i) D2[i][0] = D2[i][1] = 0ull;
 #pragma unroll
                 for (int kk = 0; kk < 16; ++kk) {
                     const float4 av = *reinterpret_cast<const float4*>(ap + kk * kHwTile);

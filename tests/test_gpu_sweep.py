@@ -162,3 +162,19 @@ def test_first_level_maximum_from_a_window_of_past_tensors():
         bdr.bdr_qsnr_delayed(cfgs, xd, window[:0], out, ws)
     assert e.value.status == -5
     torch.cuda.synchronize()
+
+
+def test_qsnr_from_sums_is_eq3_on_pairs():
+    pairs = np.array([[1.0, 100.0], [3.5e-7, 2.25], [0.0, 4.0], [1.0, 0.0], [0.0, 0.0], [7.0, 7.0], [1e-300, 1e300]], dtype=np.float64)
+    sums = torch.from_numpy(pairs).cuda()
+    out = torch.full((len(pairs),), -1.0, dtype=torch.float64, device="cuda")
+    bdr.bdr_qsnr_from_sums(sums, out)
+    torch.cuda.synchronize()
+    got = out.cpu().numpy()
+    for (e, s_), g in zip(pairs, got):
+        want = orc.qsnr_db(e, s_)
+        if math.isnan(want) or math.isinf(want):
+            assert (math.isnan(g) and math.isnan(want)) or g == want, (e, s_, g, want)
+        else:
+            assert abs(g - want) <= 1e-12 * max(abs(want), 1.0), (e, s_, g, want)
+    assert torch.equal(sums.cpu(), torch.from_numpy(pairs))          # the sums are only read
