@@ -82,3 +82,41 @@ def test_two_phase_gemms_replayed_from_a_graph(entry):
     ref = orc.gemm_nt_f64(aq, bq, nthreads=8)
     got = c.cpu().numpy().astype(np.float64)
     assert np.linalg.norm(got - ref) / np.linalg.norm(ref) <= 1e-5
+
+
+def test_training_flow_calls_replayed_from_a_graph():
+    # both packed copies from one read, Eq. 3 from the fused sums, the hardware-pipeline product and an embedding lookup
+    rows, cols = 512, 512
+    host = [H.make_input(k, rows, cols, "bf16", seed=s) for k, s in (("normal", 5), ("laplace_outliers", 6))]
+    x = _bf16(host[0])
+    pr, pc = bdr.alloc_planes(bdr.MX6, rows, cols, 1), bdr.alloc_planes(bdr.MX6, rows, cols, 0)
+    sums = torch.zeros((2, 2), dtype=torch.float64, device="cuda")
+    db = torch.zeros(2, dtype=torch.float64, device="cuda")
+    c = torch.empty((rows, rows), dtype=torch.float32, device="cuda")
+    idx = torch.tensor([5, 0, 511, 5], dtype=torch.int64, device="cuda")
+    looked_up = torch.empty((4, cols), dtype=torch.bfloat16, device="cuda")
+
+    def step():
+        sums.zero_()
+        bdr.bdr_pack2(bdr.MX6, x, pr, pc, sums[0], sums[1])
+        bdr.bdr_qsnr_from_sums(sums, db)
+        bdr.mx_gemm_hw(bdr.MX6, pr, bdr.MX6, pr, rows, rows, cols, c, r=64, f=12)
+        bdr.bdr_gather_rows(bdr.MX6, pr, rows, idx, looked_up)
+
+    step()
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        step()
+    for h in reversed(host):
+        x.copy_(_bf16(h))
+        g.replay()
+        torch.cuda.synchronize()
+        H.assert_planes_equal(H.planes_to_host(pr), orc.pack(orc.MX6, h, axis=1), "row planes")
+        H.assert_planes_equal(H.planes_to_host(pc), orc.pack(orc.MX6, h, axis=0), "column planes")
+        qd, so = orc.quant_dequant(orc.MX6, h, axis=1)
+        want_db = [orc.qsnr_db(*so), orc.qsnr_db(*orc.quant_dequant(orc.MX6, h, axis=0)[1])]
+        assert np.allclose(db.cpu().numpy(), want_db, rtol=H.QSNR_REL_TOL, atol=0)
+        H.assert_bits_equal(c.cpu().numpy(), orc.gemm_hw(orc.MX6, h, orc.MX6, h, r=64, f=12), "hardware-pipeline product")
+        H.assert_bits_equal(H.device_to_host_f32(looked_up), qd[[5, 0, 511, 5]], "lookup")
+    assert bdr.bdr_device_status() == 0
