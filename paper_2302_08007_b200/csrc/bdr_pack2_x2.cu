@@ -187,15 +187,25 @@ pack2_x2_kernel(const __grid_constant__ CUtensorMap xmap, int n_col_tiles, int n
                 const uint32_t src = box + (pair >> 1) * (kP2BoxBytes / 2) + row * 128;
                 const uint32_t c0 = (uint32_t)(pair & 1) << 6, sw = (uint32_t)(row & 7) << 4;
                 uint4 v[4];
+                if constexpr (!SUMS) {
 #pragma unroll
-                for (int g = 0; g < 4; ++g) v[g] = async::lds128(src + ((c0 + 16 * g) ^ sw));
-                if (k == 1) {
-                    __syncwarp();  // every lane has read the box for the last time: refill the stage with box i of the next tile
-                    if (lane == 0 && !failed && t + (int)gridDim.x < n_tiles) issue(t + gridDim.x, i, stg);
+                    for (int g = 0; g < 4; ++g) v[g] = async::lds128(src + ((c0 + 16 * g) ^ sw));
+                    if (k == 1) {
+                        __syncwarp();  // every lane has read the box for the last time: refill the stage with box i of the next tile
+                        if (lane == 0 && !failed && t + (int)gridDim.x < n_tiles) issue(t + gridDim.x, i, stg);
+                    }
                 }
                 uint32_t cw[2][NCW], Fs[2], mbs[2];
 #pragma unroll
                 for (int s = 0; s < 2; ++s) {
+                    if constexpr (SUMS) {  // the sums variant has no registers to spare: one block's 32 bytes at a time
+                        v[2 * s] = async::lds128(src + ((c0 + 32 * s) ^ sw));
+                        v[2 * s + 1] = async::lds128(src + ((c0 + 32 * s + 16) ^ sw));
+                        if (k == 1 && s == 1) {
+                            __syncwarp();
+                            if (lane == 0 && !failed && t + (int)gridDim.x < n_tiles) issue(t + gridDim.x, i, stg);
+                        }
+                    }
                     uint32_t w[8];
                     p2_words_of(v[2 * s], v[2 * s + 1], w);
                     x2::PairView pv;
