@@ -15,7 +15,12 @@
 //   * QSNR                                                      -- Section IV-A, Eq. 3;
 //   * Theorem 1 bound                                           -- Section IV-C, Theorem 1;
 //   * INT quantization with an FP32 max-scale                   -- Section II, Eq. 1 and Eq. 2;
-//   * FP8 / VSQ as two-level schemes                            -- Section III, Table I.
+//   * FP8 / VSQ as two-level schemes                            -- Section III, Table I;
+//   * a first-level maximum supplied from outside ("delayed scaling") and the packing efficiency of
+//     a tile in fixed-width memory lines                          -- Section IV-B, Fig. 7 caption and the
+//     memory-footprint paragraph;
+//   * the dot product as the hardware pipeline computes it        -- Section IV-B, Fig. 6 and its text;
+//   * an FP32 parent scale above the two levels (three-level)     -- Section III, last paragraph.
 //
 // Readings taken where the paper is silent (all listed in the design notes of the repository):
 //   ties round to even by default (ties-away selectable); a magnitude that would round to 2^m is
@@ -29,7 +34,9 @@
 // principle but no formula, is pinned by hand-worked groups (sub-scales that round up, round down,
 // tie, reach the top code and flush to zero; both tie rules; per-group first-level scale) and by its
 // reductions (equal per-vector maxima => per-tensor INT; a 16-bit sub-scale => INT with one FP32
-// scale per vector, within a derived bound).
+// scale per vector, within a derived bound).  The hardware dot product and the parent scale, which
+// the paper describes in words only, are pinned by hand-worked examples and by the cases in which they
+// must reduce to the exact dot product / the two-level quantizer.
 //
 // Build: g++ -O2 -std=c++17 -ffp-contract=off -fPIC -shared bdr_oracle.cpp -o liboracle_bdr.so -lpthread
 
