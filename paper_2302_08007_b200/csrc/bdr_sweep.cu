@@ -699,6 +699,21 @@ static int qsnr_impl(const bdr_config_t* cfgs, int n_cfgs, const void* x, bdr_dt
     }
     build_families(singles, &table);
     const int n_fam = (int)table.size();
+    // Rows shorter than a tile would leave the 4096-element tiles mostly empty.  When the rows are contiguous and every
+    // configuration's blocks (and VSQ vectors) divide the row length, no block straddles two rows, so the tensor is the
+    // same problem as one long row.
+    if (axis == 1 && rows > 1 && ld == cols && cols > 0) {
+        bool whole = true;
+        for (int i = 0; i < n_cfgs && whole; ++i) {
+            const int64_t g = cfgs[i].scale_kind == BDR_SCALE_POW2 ? cfgs[i].k1 : (cfgs[i].scale_kind == BDR_SCALE_FP32_VSQ ? cfgs[i].k2 : 1);
+            whole = g > 0 && cols % g == 0;
+        }
+        if (whole) {
+            cols *= rows;
+            rows = 1;
+            ld = cols;
+        }
+    }
     if (!workspace || workspace_bytes < sweep_workspace_bytes(n_cfgs)) return BDR_ERR_WORKSPACE;
     if ((uintptr_t)workspace % 16) return BDR_ERR_MISALIGNED;
     cudaStream_t st = (cudaStream_t)stream;

@@ -178,3 +178,14 @@ def test_qsnr_from_sums_is_eq3_on_pairs():
         else:
             assert abs(g - want) <= 1e-12 * max(abs(want), 1.0), (e, s_, g, want)
     assert torch.equal(sums.cpu(), torch.from_numpy(pairs))          # the sums are only read
+
+
+def test_short_contiguous_rows_are_swept_as_one_long_line_without_changing_the_result():
+    # 1,024-element vectors (the paper's sweep workload): every block size of the grid divides the row, so the kernel treats the
+    # contiguous tensor as one long row; a pitch, or a row length some block size does not divide, keeps the rows apart
+    cfgs = [c for _, c in sweep.sweep_configs()]
+    x = synth.variable_variance_vectors(48, 1024, seed=31)
+    check(cfgs, run_sweep(cfgs, x), x, "merged rows")
+    check(cfgs[::9], run_sweep(cfgs[::9], x, ld=1040), x, "pitched rows")
+    x2 = synth.variable_variance_vectors(40, 1536, seed=32)          # 1536 is not a multiple of 1024: blocks of 1024 are ragged per row
+    check(cfgs[::9] + cfgs[430:457], run_sweep(cfgs[::9] + cfgs[430:457], x2), x2, "rows kept apart")
