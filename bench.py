@@ -475,7 +475,7 @@ def secondary_legs(args, bdr, synth, torch) -> dict:
     """MX-GEMM TFLOP/s, design-sweep configs/s, the linear-layer step and the small-vector latency case."""
     import bench_legs as legs
     out = {}
-    for fn in (legs.c1_leg, legs.gemm_leg, legs.sweep_leg, legs.paper_sweep_leg, legs.linear_leg):
+    for fn in (legs.c1_leg, legs.gemm_leg, legs.sweep_leg, legs.paper_sweep_leg, legs.embedding_leg, legs.linear_leg):
         try:
             out.update(fn(args))
         except bdr.BdrError as e:

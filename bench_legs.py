@@ -251,6 +251,38 @@ def c1_leg(args) -> dict:
     return {"c1_vector": out}
 
 
+def embedding_leg(args) -> dict:
+    """Lookups in an MX6-packed embedding table (Section V, inferencing): 2^20 rows of 128 elements, 2^20 random indices,
+    bf16 output.  Algorithmic bytes per lookup: the row's packed bytes (128 x 6 / 8), the 8-byte index and the 256 output bytes."""
+    n_rows, dim, n_idx = 1 << 20, 128, 1 << 20
+    g = torch.Generator(device="cuda").manual_seed(0)
+    table = (torch.randn((n_rows, dim), device="cuda", generator=g) * 0.05).to(torch.bfloat16)
+    planes = bdr.alloc_planes(bdr.MX6, n_rows, dim, 1)
+    bdr.bdr_pack(bdr.MX6, table, planes, axis=1)
+    idx = torch.randint(0, n_rows, (n_idx,), device="cuda", dtype=torch.int64, generator=g)
+    out = torch.empty((n_idx, dim), dtype=torch.bfloat16, device="cuda")
+    ms = _time(lambda: bdr.bdr_gather_rows(bdr.MX6, planes, n_rows, idx, out), reps=10, warmup=2)
+    nbytes = n_idx * (dim * 6 / 8 + 8 + dim * 2)
+    peaks = getattr(args, "peaks", {})
+    hbm = float(peaks.get("hbm_gbs", 6650.0))
+    res = {"workload": "2^20 random lookups in a 2^20 x 128 MX6-packed table, bf16 output", "ms": ms, "value": nbytes / (ms * 1e-3) / 1e9,
+           "unit": "GB/s", "lookups_per_s": n_idx / (ms * 1e-3),
+           "roofline": {"bound": "hbm", "achieved": nbytes / (ms * 1e-3) / 1e9, "peak": hbm, "unit": "GB/s", "frac": nbytes / (ms * 1e-3) / 1e9 / hbm,
+                        "peak_source": "measured" if peaks else "fallback", "traffic": None,
+                        "kind": "algorithmic bytes (packed row + index + output row) / CUDA-event time; random 96 + 8 + 8 byte reads"},
+           "status": bdr.bdr_device_status()}
+    if getattr(args, "cpu_legs", False):
+        from oracle import oracle as orc
+        sample = 4096
+        host = tuple(t[:sample].cpu().numpy() for t in (planes.exps, planes.micro, planes.elems))
+        t0 = time.perf_counter()
+        orc.unpack(orc.MX6, host, sample, dim)
+        sec = time.perf_counter() - t0
+        res["cpu_baseline"] = {"value": sample / sec, "unit": "lookups/s", "cores": 1, "kind": "oracle",
+                               "sample": "decoding %d rows of the table (%.3f s)" % (sample, sec)}
+    return {"embedding_lookup": res}
+
+
 # ---------------------------------------------------------------------------------------------------------------------
 # bench.py --only <op>: one operation, a few launches, for profilers and quick timing
 # ---------------------------------------------------------------------------------------------------------------------

@@ -336,7 +336,13 @@ int bdr_gather_rows(const bdr_config_t* cfg, const bdr_planes_t* table, int64_t 
     int* status = device_status_word();
     if (!status) return BDR_ERR_CUDA;
     cudaStream_t st = (cudaStream_t)stream;
-    if (dt == BDR_F32) return gather_rows_general<float>(*table, n_rows, idx_dev, (float*)y, n_idx, dim, ld, qp, status, st);
+    if (dt == BDR_F32) {
+        rc = gather_rows_mx_x2<float>(*table, n_rows, idx_dev, (float*)y, n_idx, dim, ld, qp, status, st);
+        if (rc != BDR_ERR_UNSUPPORTED) return rc;
+        return gather_rows_general<float>(*table, n_rows, idx_dev, (float*)y, n_idx, dim, ld, qp, status, st);
+    }
+    rc = gather_rows_mx_x2<__nv_bfloat16>(*table, n_rows, idx_dev, (__nv_bfloat16*)y, n_idx, dim, ld, qp, status, st);
+    if (rc != BDR_ERR_UNSUPPORTED) return rc;
     return gather_rows_general<__nv_bfloat16>(*table, n_rows, idx_dev, (__nv_bfloat16*)y, n_idx, dim, ld, qp, status, st);
 }
 

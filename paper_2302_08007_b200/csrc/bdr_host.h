@@ -101,6 +101,11 @@ template <typename T>
 int gather_rows_general(const bdr_planes_t& in, int64_t n_rows, const int64_t* idx, T* y, int64_t n_idx, int64_t len, int64_t ld,
                         const QParams& qp, int* status, cudaStream_t st);
 
+// the same for the Table II formats on packed bf16x2 arithmetic, one thread per 32 elements (bdr_gather_x2.cu)
+template <typename T>
+int gather_rows_mx_x2(const bdr_planes_t& in, int64_t n_rows, const int64_t* idx, T* y, int64_t n_idx, int64_t dim, int64_t ld,
+                      const QParams& qp, int* status, cudaStream_t st);
+
 // Packed MX4 / MX6 operands -> E4M3 bytes plus one power-of-two scale byte per 32 elements (bdr_reencode_f8.cu)
 struct ZeroTiles {   // `count` tiles of 256 x 256 floats of c (row pitch ldc, tiles_n tiles per row of tiles), from tile0 on
     float* c;

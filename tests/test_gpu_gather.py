@@ -17,7 +17,7 @@ pytestmark = pytest.mark.gpu
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
 def test_gathered_rows_equal_the_oracles_dequantized_table_rows(cfg, dtype):
     rng = np.random.default_rng(51)
-    for n_rows, dim, n_idx, ld in ((1000, 128, 4096, None), (37, 100, 64, 104), (5, 16, 1, None)):
+    for n_rows, dim, n_idx, ld in ((1000, 128, 4096, None), (37, 100, 64, 104), (5, 16, 1, None), (300, 96, 777, 104), (64, 1024, 50, None)):
         table = H.make_input("laplace_outliers", n_rows, dim, dtype, seed=n_rows)
         planes = bdr.alloc_planes(cfg, n_rows, dim, 1)
         bdr.bdr_pack(cfg, H.host_to_device(table, dtype), planes, axis=1)
@@ -51,3 +51,23 @@ def test_an_index_outside_the_table_is_reported_and_poisons_only_its_row():
         bdr.bdr_gather_rows(cfg, planes, 64, idx, torch.zeros((5, 128), dtype=torch.float32, device="cuda"))   # planes too short for dim
     assert e.value.status == -5
     torch.cuda.synchronize()
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_lookup_of_rows_with_tiny_huge_and_nonfinite_blocks(dtype):
+    # blocks outside the exponent range of the packed arithmetic (and Inf/NaN blocks) take the out-of-line decoder
+    for name, cfg in (("MX4", bdr.MX4), ("MX6", bdr.MX6), ("MX9", bdr.MX9)):
+        table = np.concatenate([H.make_input(k, 32, 128, dtype, seed=53) for k in ("tiny", "huge", "edge", "normal")])
+        table[100, 40] = np.inf
+        planes = bdr.alloc_planes(cfg, 128, 128, 1)
+        bdr.bdr_pack(cfg, H.host_to_device(table, dtype), planes, axis=1)
+        want = orc.quant_dequant(H.to_orc(cfg), table, axis=1)[0]
+        idx = np.random.default_rng(54).permutation(128)
+        out = H.host_to_device(np.zeros((128, 128), dtype=np.float32), dtype)
+        bdr.bdr_gather_rows(cfg, planes, 128, torch.from_numpy(idx).cuda(), out)
+        torch.cuda.synchronize()
+        got = H.device_to_host_f32(out)
+        nan = np.isnan(want[idx])
+        assert np.array_equal(np.isnan(got), nan) and nan.any()
+        H.assert_bits_equal(got[~nan], want[idx][~nan], "%s %s" % (name, dtype))
+    assert bdr.bdr_device_status() == 0
