@@ -127,8 +127,9 @@ int bdr_quant_dequant(const bdr_config_t* cfg /*host*/, const void* x, void* y, 
  * block scale and the microexponents.  This library's reading: the parent scale maps the group's largest magnitude onto
  * the largest value a block with exponent 0 can hold, V = (2^m - 1) 2^-(m-1):  s = amax_g / V,  x' = x / s,
  * y = Q(x') s with Q the two-level quantizer of bdr_quant_dequant (IEEE fp32 division and multiplication).  Arguments
- * as bdr_quant_dequant.  fp32 tensors, k1 <= 16, k_parent a multiple of 16 (and of k1) up to 1024; a correctness-grade
- * kernel (one warp per group), meant for fidelity studies. */
+ * as bdr_quant_dequant.  fp32 tensors, k1 <= 16, k_parent a multiple of 16 (and of k1) up to 1024.  Fastest (about half
+ * the copy bandwidth): k1 = 16, k_parent a power of two, whole groups along contiguous 16-byte aligned rows (axis 1);
+ * other shapes take one warp per group with element-wise loads. */
 int bdr_quant_dequant_parent(const bdr_config_t* cfg /*host*/, int k_parent, const void* x, void* y, bdr_dtype_t dt,
                              int64_t rows, int64_t cols, int64_t ld, int axis, double* qsnr_sums_dev, void* stream);
 

@@ -164,8 +164,120 @@ parent_scale_kernel(const float* x, float* y, int64_t nlines, int64_t len, int64
     if (sums) block_accumulate_sums(e2, s2, sums);
 }
 
+// The same for the common shape: rows along the contiguous dimension, k1 = 16, groups of 16 * 2^j <= 1024 elements that tile
+// the row, 16-byte aligned rows.  A thread owns one 16-element slice (one block) of a group -- two when the group has 64 slices --
+// loaded and stored with 16-byte accesses; the group maximum goes round the group's lanes by shuffle; x / s is the correctly
+// rounded quotient computed with the rounded reciprocal, a residual and a correction (one reciprocal per group; plain division
+// where that shortcut is not safe); the two-level quantizer is the adder formulation of quantize_slice.
+struct PsDivisor {
+    float s, r;
+    bool fast;
+};
+__device__ __forceinline__ PsDivisor ps_make_divisor(float s) {
+    PsDivisor d;
+    d.s = s;
+    d.r = __frcp_rn(s);
+    const uint32_t b = __float_as_uint(s);
+    d.fast = (b & 0x7FFFFFu) != 0x7FFFFFu && b >= 0x0D800000u /*2^-100*/ && b <= 0x71800000u /*2^100*/;
+    return d;
+}
+// x / d.s, correctly rounded.  Fast route: q0 = RN(x r), e = x - q0 s (exact in one fused multiply-add), q = RN(q0 + e r); valid
+// while nothing leaves the normal range: the residual is a multiple of ulp(q0) ulp(s), so x and q0 are kept above 2^-100 (s lies
+// within 2^+-100, and |x| <= amax makes the quotient smaller than 2); anything else takes the division instruction.
+__device__ __forceinline__ float ps_divide(float x, const PsDivisor& d) {
+    const float q0 = __fmul_rn(x, d.r);
+    const bool ok = d.fast && (__float_as_uint(x) & 0x7FFFFFFFu) >= 0x0D800000u && (__float_as_uint(q0) & 0x7FFFFFFFu) >= 0x0D800000u;
+    if (ok) return __fmaf_rn(__fmaf_rn(-q0, d.s, x), d.r, q0);
+    return __fdiv_rn(x, d.s);
+}
+
+template <int K2>
+__global__ void __launch_bounds__(kGenThreads)
+parent_scale_rows_kernel(const float* x, float* y, int64_t rows, int64_t cols, int64_t ld, int slices_per_group, QParams qp, double* sums) {
+    const int lanes = min(slices_per_group, 32), per_lane = slices_per_group > 32 ? 2 : 1;   // lanes of a group, slices per lane
+    const int64_t spr = cols / kSlice / per_lane;                                              // threads per row
+    const int64_t total = rows * spr;
+    const float V = (float)qp.qmax * __uint_as_float((uint32_t)(127 - (qp.m - 1)) << 23);
+    double e2 = 0.0, s2 = 0.0;
+    const int64_t nthreads = (int64_t)gridDim.x * kGenThreads;
+    const int64_t rounded = (total + 31) / 32 * 32;   // whole warps take part in the shuffles
+    for (int64_t t = (int64_t)blockIdx.x * kGenThreads + threadIdx.x; t < rounded; t += nthreads) {
+        const bool live = t < total;
+        const int64_t row = live ? t / spr : 0, pos = live ? t - row * spr : 0;
+        // with two slices per lane a warp is one group: lane l owns slices l and l + 32 of it
+        const int64_t slice0 = per_lane == 2 ? (pos / 32) * 64 + (pos & 31) : pos;
+        uint32_t u[2][kSlice];
+        uint32_t am = 0;
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            if (h < per_lane && live) {
+                load_slice_vec(x + row * ld + (slice0 + 32 * h) * kSlice, u[h]);
+#pragma unroll
+                for (int i = 0; i < kSlice; ++i) am = max(am, u[h][i] & 0x7FFFFFFFu);
+            }
+        }
+        for (int o = lanes >> 1; o > 0; o >>= 1) am = max(am, __shfl_xor_sync(0xFFFFFFFFu, am, o));
+        if (!live) continue;
+        const float s = __fdiv_rn(__uint_as_float(am), V);
+        const PsDivisor dv = ps_make_divisor(s);
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            if (h >= per_lane) break;
+            uint32_t yb[kSlice];
+            if (!(s > 0.f)) {
+#pragma unroll
+                for (int i = 0; i < kSlice; ++i) yb[i] = u[h][i] & 0x80000000u;
+            } else {
+                uint32_t xs[kSlice], ej[kSlice / K2], fb[1], rq[kSlice], cb[kSlice / K2], tau[kSlice / K2];
+#pragma unroll
+                for (int i = 0; i < kSlice; ++i) xs[i] = __float_as_uint(ps_divide(__uint_as_float(u[h][i]), dv));
+                subblock_exponents<K2>(xs, ej);
+                uint32_t F = 0;
+#pragma unroll
+                for (int j = 0; j < kSlice / K2; ++j) F = max(F, ej[j]);
+                fb[0] = F;
+                double de = 0.0, ds = 0.0;
+                quantize_slice<K2, kSlice, false, true, false>(xs, ej, fb, qp, yb, rq, cb, tau, de, ds);
+#pragma unroll
+                for (int i = 0; i < kSlice; ++i) yb[i] = __float_as_uint(__fmul_rn(__uint_as_float(yb[i]), s));
+            }
+            if (y) store_slice_vec(y + row * ld + (slice0 + 32 * h) * kSlice, yb);
+            if (sums) {
+#pragma unroll
+                for (int i = 0; i < kSlice; ++i) {
+                    const double a = (double)__uint_as_float(u[h][i]), d = (double)__uint_as_float(yb[i]) - a;
+                    e2 = fma(d, d, e2);
+                    s2 = fma(a, a, s2);
+                }
+            }
+        }
+    }
+    if (sums) block_accumulate_sums(e2, s2, sums);
+}
+
+template <int K2>
+static int launch_parent_rows(const float* x, float* y, int64_t rows, int64_t cols, int64_t ld, int k_parent, const QParams& qp, double* sums,
+                              cudaStream_t st) {
+    const int spg = k_parent / kSlice;
+    const int64_t total = rows * (cols / kSlice / (spg > 32 ? 2 : 1));
+    const int grid = (int)max((int64_t)1, min((total + kGenThreads - 1) / kGenThreads, (int64_t)sm_count() * 16));
+    parent_scale_rows_kernel<K2><<<grid, kGenThreads, 0, st>>>(x, y, rows, cols, ld, spg, qp, sums);
+    return cudaGetLastError() == cudaSuccess ? BDR_OK : BDR_ERR_CUDA;
+}
+
 int quant_parent_scale(const float* x, float* y, int64_t rows, int64_t cols, int64_t ld, int axis, int k_parent, const QParams& qp,
                        double* sums, cudaStream_t st) {
+    const bool pow2 = (k_parent & (k_parent - 1)) == 0;
+    if (axis == 1 && qp.k1 == kSlice && pow2 && k_parent >= kSlice && k_parent <= 1024 && cols % k_parent == 0 && ld % 4 == 0 &&
+        ((uintptr_t)x | (uintptr_t)y) % 16 == 0 && rows > 0 && cols > 0) {
+        switch (qp.k2) {
+            case 1: return launch_parent_rows<1>(x, y, rows, cols, ld, k_parent, qp, sums, st);
+            case 2: return launch_parent_rows<2>(x, y, rows, cols, ld, k_parent, qp, sums, st);
+            case 4: return launch_parent_rows<4>(x, y, rows, cols, ld, k_parent, qp, sums, st);
+            case 8: return launch_parent_rows<8>(x, y, rows, cols, ld, k_parent, qp, sums, st);
+            case 16: return launch_parent_rows<16>(x, y, rows, cols, ld, k_parent, qp, sums, st);
+        }
+    }
     const int64_t nlines = axis == 1 ? rows : cols, len = axis == 1 ? cols : rows;
     const int64_t line_stride = axis == 1 ? ld : 1, elem_stride = axis == 1 ? 1 : ld;
     const int64_t groups = nlines * ((len + k_parent - 1) / k_parent);

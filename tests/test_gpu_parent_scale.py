@@ -50,3 +50,24 @@ def test_parent_scale_argument_checks_and_sums_only():
         bdr.bdr_quant_dequant_parent(bdr.MX6, 64, x.to(torch.bfloat16), torch.empty_like(x, dtype=torch.bfloat16))
     assert e.value.status == -3
     torch.cuda.synchronize()
+
+
+@pytest.mark.parametrize("kp", [16, 64, 256, 512, 1024])
+def test_parent_scale_row_kernel_on_groups_with_a_wide_dynamic_range(kp):
+    # whole groups along contiguous rows (the fast kernel): every block of a group scaled by a random power of two over 80
+    # binades, so that the quotients x / s run from about 1 down to far below the block unit, plus zero and tiny groups
+    rng = np.random.default_rng(62 + kp)
+    rows, cols = 33, 4096
+    x = (synth.normal_matrix(rows, cols, seed=63) * np.repeat(2.0 ** rng.integers(-70, 11, (rows, cols // 16)), 16, axis=1)).astype(np.float32)
+    x[3, :kp] = 0.0
+    x[4, :kp] = synth.normal(kp, 64) * np.float32(1e-37)
+    x[5, :kp] = synth.normal(kp, 65) * np.float32(1e30)
+    for cfg in (bdr.MX4, bdr.MX9, C_(16, 8, 8, 2, 5), C_(16, 8, 1, 3, 6)):
+        xd = H.host_to_device(x, "f32")
+        y = torch.zeros_like(xd)
+        sums = torch.zeros(2, dtype=torch.float64, device="cuda")
+        bdr.bdr_quant_dequant_parent(cfg, kp, xd, y, axis=1, qsnr_sums=sums)
+        torch.cuda.synchronize()
+        want, so = orc.quant_dequant_parent(H.to_orc(cfg), kp, x, axis=1)
+        H.assert_bits_equal(H.device_to_host_f32(y), want, "%s k_parent=%d" % (cfg, kp))
+        H.assert_qsnr_close(sums.cpu().numpy(), so, "%s k_parent=%d" % (cfg, kp))
