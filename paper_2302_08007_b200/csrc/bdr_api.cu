@@ -150,6 +150,7 @@ static int quant_dispatch(const QParams& qp, const T* x, T* y, int64_t rows, int
             if (rc != BDR_ERR_UNSUPPORTED) return rc;
         }
         if (!out || tight) rc = quant_colwise_mx<T>(x, y, rows, cols, ld, out, qp, sums, st);
+        if (rc == BDR_ERR_UNSUPPORTED && !out) rc = quant_colwise_any<T>(x, y, rows, cols, ld, qp, sums, st);
     }
     if (rc == BDR_ERR_UNSUPPORTED) rc = quant_general<T>(x, y, rows, cols, ld, axis, out, qp, sums, st);
     return rc;

@@ -84,6 +84,10 @@ template <typename T>
 int quant_colwise_mx(const T* x, T* y, int64_t rows, int64_t cols, int64_t ld, const bdr_planes_t* out,
                      const QParams& qp, double* sums, cudaStream_t st);
 
+// axis-0 quantize-dequantize of every other POW2 configuration with k2 <= 16 (bdr_col_any.cu)
+template <typename T>
+int quant_colwise_any(const T* x, T* y, int64_t rows, int64_t cols, int64_t ld, const QParams& qp, double* sums, cudaStream_t st);
+
 // general kernels: any axis, any POW2 configuration, any alignment (bdr_general.cu)
 template <typename T>
 int quant_general(const T* x, T* y, int64_t rows, int64_t cols, int64_t ld, int axis, const bdr_planes_t* out,

@@ -171,6 +171,32 @@ def test_columnwise_quant_dequant(dtype):
             H.assert_qsnr_close(sums, so)
 
 
+@pytest.mark.parametrize("cfg", ROW_CONFIGS + [Cfg(16, 8, 2, 1, 4, bdr.SCALE_POW2, bdr.ROUND_NEAREST_AWAY),
+                                             Cfg(64, 8, 4, 2, 6, bdr.SCALE_POW2, bdr.ROUND_NEAREST_AWAY)], ids=str)
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_columnwise_quant_dequant_of_every_configuration(cfg, dtype):
+    # blocks run down the columns; every (k1, k2, d2) family of the sweep: block sizes from 1 to 1024 rows, several blocks
+    # per column, a ragged last block (rows not a multiple of k1), ragged column groups, a pitch, in place, sums only
+    for kind, rows, cols, ld in (("laplace_outliers", 2048 + 40, 96, None), ("edge", 1100, 70, 72), ("normal", 48, 130, None)):
+        x = H.make_input(kind, rows, cols, dtype, seed=43)
+        y, sums = run_quant(cfg, x, dtype, axis=0, ld=ld)
+        want, so = orc.quant_dequant(H.to_orc(cfg), x, axis=0)
+        H.assert_bits_equal(y, want, "%s %s %s %dx%d" % (cfg, dtype, kind, rows, cols))
+        H.assert_qsnr_close(sums, so, "%s %s %s" % (cfg, dtype, kind))
+    x = H.make_input("normal", 300, 64, dtype, seed=44)
+    want, so = orc.quant_dequant(H.to_orc(cfg), x, axis=0)
+    y, _ = run_quant(cfg, x, dtype, axis=0, inplace=True)
+    H.assert_bits_equal(y, want, "%s %s in place" % (cfg, dtype))
+    _, sums = run_quant(cfg, x, dtype, axis=0, want_y=False)
+    H.assert_qsnr_close(sums, so, "%s %s sums only" % (cfg, dtype))
+    for kind in ("tiny", "huge"):
+        x = H.make_input(kind, 260, 34, dtype, seed=45)
+        y, sums = run_quant(cfg, x, dtype, axis=0)
+        want, so = orc.quant_dequant(H.to_orc(cfg), x, axis=0)
+        H.assert_bits_equal(y, want, "%s %s %s" % (cfg, dtype, kind))
+        H.assert_qsnr_close(sums, so, "%s %s %s" % (cfg, dtype, kind))
+
+
 # ---- host-side error paths: nothing is launched -----------------------------------------------------------
 def test_argument_errors_are_reported_not_launched():
     x = torch.zeros((4, 64), device="cuda")
