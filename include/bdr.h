@@ -117,7 +117,8 @@ int bdr_packed_sizes(const bdr_config_t* cfg /*host*/, int64_t rows, int64_t col
  * ties-to-even) with 32-byte aligned rows of whole 2048-element runs (axis 1; a contiguous tensor counts
  * as one long row) or whole tiles of 256 rows x 128 columns (axis 0); along axis 1 the same kernel also
  * takes k1 = 32 .. 1024 (powers of two) and formats without shifts (d2 = 0); next, fp32 or bf16 with 16-byte
- * aligned rows of whole 16-element slices; anything else takes a slower general kernel. */
+ * aligned rows of whole 16-element slices (axis 1), and along axis 0 every configuration with k2 <= 16 (bf16: an
+ * even number of columns and an even pitch); anything else takes a slower general kernel. */
 int bdr_quant_dequant(const bdr_config_t* cfg /*host*/, const void* x, void* y, bdr_dtype_t dt,
                       int64_t rows, int64_t cols, int64_t ld, int axis, double* qsnr_sums_dev,
                       void* stream);
