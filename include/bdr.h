@@ -315,8 +315,8 @@ int mx_gemm_e4m3(const uint8_t* a, const uint8_t* scales_a, const uint8_t* b, co
  * increasing K.  The paper chooses f = min(25, the format's dynamic range), which is 25 for every format with an
  * 8-bit shared exponent.  With a frame wide enough for the exponent spread of a pass the result is the exact dot
  * product of the dequantized operands rounded once per pass; narrower frames drop low bits of the smaller blocks.
- * Table II formats (A and B may differ), r in {16, 32, 64}, 1 <= f <= 25, M and N multiples of 64, K a multiple of
- * 64, c 16-byte aligned with ldc a multiple of 4.  A block with the exponent byte 0xFF makes its row's (column's)
+ * Table II formats (A and B may differ), r a power of two from 16 to 1024 that divides K, 1 <= f <= 25, M and N multiples
+ * of 64, K a multiple of 64, c 16-byte aligned with ldc a multiple of 4.  A block with the exponent byte 0xFF makes its row's (column's)
  * outputs NaN.  Runs on the ordinary arithmetic units (the alignment is per block and output), not the tensor cores. */
 int mx_gemm_hw(const bdr_config_t* cfg_a /*host*/, const bdr_planes_t* a /*host struct*/,
                const bdr_config_t* cfg_b /*host*/, const bdr_planes_t* b /*host struct*/, int64_t M, int64_t N,

@@ -74,7 +74,8 @@ __device__ __forceinline__ void hw_decode(const HwItem<W>& it, float* tile, int 
 
 __device__ __forceinline__ bool hw_has_ff_byte(uint32_t w) { return (((w & 0x7F7F7F7Fu) + 0x01010101u) & w & 0x80808080u) != 0; }
 
-template <int WA, int WB>
+// LONG: a pass spans several steps (r > 64) and its state lives across them.
+template <int WA, int WB, bool LONG>
 __global__ void __launch_bounds__(kHwThreads, 2)
 mx_gemm_hw_kernel(bdr_planes_t a, bdr_planes_t b, int64_t K, int r, int f, float* c, int64_t ldc) {
     __shared__ __align__(16) float As[kHwStep * kHwTile], Bs[kHwStep * kHwTile];
@@ -93,6 +94,7 @@ mx_gemm_hw_kernel(bdr_planes_t a, bdr_planes_t b, int64_t K, int r, int f, float
 #pragma unroll
         for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
     bool bad_a[4] = {false, false, false, false}, bad_b[4] = {false, false, false, false};
+    [[maybe_unused]] int emax_p[LONG ? 4 : 1][4], total_p[LONG ? 4 : 1][4];  // state of a pass that spans several steps
     HwItem<WA> ia;
     HwItem<WB> ib;
     if (dutyA) hw_fetch<WA>(a, row0 + drow, 2 * dhalf, ia);
@@ -120,67 +122,48 @@ mx_gemm_hw_kernel(bdr_planes_t a, bdr_planes_t b, int64_t K, int r, int f, float
             bad_a[i] |= hw_has_ff_byte(fa[i]);
             bad_b[i] |= hw_has_ff_byte(fb[i]);
         }
-        for (int p = 0; p < passes; ++p) {
-            const int b0 = p * bpr;
-            int emax[4][4];
+        // one block of 16 elements of K: exact block results D_b, aligned to the pass's largest exponent inside the f-bit frame,
+        // truncated toward zero, added as integers
+        auto do_block = [&](int bb, const int (&base)[4][4], int (&total)[4][4]) {
+            const int swz = (bb >> 1) << 4;  // the half (32 elements) this block belongs to
+            const float* ap = As + (16 * bb) * kHwTile + ((4 * ty) ^ swz);
+            const float* bp = Bs + (16 * bb) * kHwTile + ((4 * tx) ^ swz);
+            unsigned long long D2[4][2];  // (row i; columns 0, 1) and (row i; columns 2, 3)
 #pragma unroll
-            for (int i = 0; i < 4; ++i)
+            for (int i = 0; i < 4; ++i) D2[i][0] = D2[i][1] = 0ull;
 #pragma unroll
-                for (int j = 0; j < 4; ++j) emax[i][j] = 0;
-            for (int bb = b0; bb < b0 + bpr; ++bb) {
+            for (int kk = 0; kk < 16; ++kk) {
+                const float4 av = *reinterpret_cast<const float4*>(ap + kk * kHwTile);
+                const ulonglong2 bv = *reinterpret_cast<const ulonglong2*>(bp + kk * kHwTile);
+                const float ar[4] = {av.x, av.y, av.z, av.w};
 #pragma unroll
-                for (int i = 0; i < 4; ++i)
-#pragma unroll
-                    for (int j = 0; j < 4; ++j)
-                        emax[i][j] = max(emax[i][j], (int)((fa[i] >> (8 * bb)) & 0xFFu) + (int)((fb[j] >> (8 * bb)) & 0xFFu));
+                for (int i = 0; i < 4; ++i) {
+                    const unsigned long long aa = hw_dup(ar[i]);
+                    hw_fma2(D2[i][0], aa, bv.x);
+                    hw_fma2(D2[i][1], aa, bv.y);
+                }
             }
-            int total[4][4], base[4][4];
+            int ea[4], eb[4];
 #pragma unroll
-            for (int i = 0; i < 4; ++i)
+            for (int i = 0; i < 4; ++i) {
+                ea[i] = (int)((fa[i] >> (8 * bb)) & 0xFFu);
+                eb[i] = (int)((fb[i] >> (8 * bb)) & 0xFFu);
+            }
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                float D[4];
+                hw_split(D2[i][0], D[0], D[1]);
+                hw_split(D2[i][1], D[2], D[3]);
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
-                    total[i][j] = 0;
-                    base[i][j] = fbase - emax[i][j];
-                }
-            for (int bb = b0; bb < b0 + bpr; ++bb) {
-                const int swz = (bb >> 1) << 4;  // the half (32 elements) this block belongs to
-                const float* ap = As + (16 * bb) * kHwTile + ((4 * ty) ^ swz);
-                const float* bp = Bs + (16 * bb) * kHwTile + ((4 * tx) ^ swz);
-                unsigned long long D2[4][2];  // (row i; columns 0, 1) and (row i; columns 2, 3)
-#pragma unroll
-                for (int i = 0; i < 4; ++i) D2[i][0] = D2[i][1] = 0ull;
-#pragma unroll
-                for (int kk = 0; kk < 16; ++kk) {
-                    const float4 av = *reinterpret_cast<const float4*>(ap + kk * kHwTile);
-                    const ulonglong2 bv = *reinterpret_cast<const ulonglong2*>(bp + kk * kHwTile);
-                    const float ar[4] = {av.x, av.y, av.z, av.w};
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        const unsigned long long aa = hw_dup(ar[i]);
-                        hw_fma2(D2[i][0], aa, bv.x);
-                        hw_fma2(D2[i][1], aa, bv.y);
-                    }
-                }
-                // align to the pass's largest exponent inside the f-bit frame, truncate toward zero, add
-                int ea[4], eb[4];
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    ea[i] = (int)((fa[i] >> (8 * bb)) & 0xFFu);
-                    eb[i] = (int)((fb[i] >> (8 * bb)) & 0xFFu);
-                }
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    float D[4];
-                    hw_split(D2[i][0], D[0], D[1]);
-                    hw_split(D2[i][1], D[2], D[3]);
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        const int field = base[i][j] + ea[i] + eb[j];  // exponent field of 2^(f - W - (e_max - e))
-                        const float scale = __uint_as_float((uint32_t)max(field, 0) << 23);
-                        total[i][j] += __float2int_rz(D[j] * scale);
-                    }
+                    const int field = base[i][j] + ea[i] + eb[j];  // exponent field of 2^(f - W - (e_max - e))
+                    const float scale = __uint_as_float((uint32_t)max(field, 0) << 23);
+                    total[i][j] += __float2int_rz(D[j] * scale);
                 }
             }
+        };
+        // end of a pass: the integer sum becomes an fp32 number, takes its power of two, joins the fp32 accumulator
+        auto finish_pass = [&](const int (&emax)[4][4], const int (&total)[4][4]) {
 #pragma unroll
             for (int i = 0; i < 4; ++i)
 #pragma unroll
@@ -190,6 +173,65 @@ mx_gemm_hw_kernel(bdr_planes_t a, bdr_planes_t b, int64_t K, int r, int f, float
                     const double v = (double)(float)total[i][j] * __hiloint2double((1023 + unit) << 20, 0);
                     acc[i][j] = __fadd_rn(acc[i][j], (float)v);
                 }
+        };
+        if constexpr (!LONG) {  // whole passes inside the step
+            for (int p = 0; p < passes; ++p) {
+                const int b0 = p * bpr;
+                int emax[4][4], total[4][4], base[4][4];
+#pragma unroll
+                for (int i = 0; i < 4; ++i)
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) emax[i][j] = 0;
+                for (int bb = b0; bb < b0 + bpr; ++bb) {
+#pragma unroll
+                    for (int i = 0; i < 4; ++i)
+#pragma unroll
+                        for (int j = 0; j < 4; ++j)
+                            emax[i][j] = max(emax[i][j], (int)((fa[i] >> (8 * bb)) & 0xFFu) + (int)((fb[j] >> (8 * bb)) & 0xFFu));
+                }
+#pragma unroll
+                for (int i = 0; i < 4; ++i)
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        total[i][j] = 0;
+                        base[i][j] = fbase - emax[i][j];
+                    }
+                for (int bb = b0; bb < b0 + bpr; ++bb) do_block(bb, base, total);
+                finish_pass(emax, total);
+            }
+        } else {  // a pass spans r / 64 steps: its largest exponent sums come from the exponent planes when it starts
+            const int spp = r / kHwStep;
+            if (s % spp == 0) {
+#pragma unroll
+                for (int i = 0; i < 4; ++i)
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        emax_p[i][j] = 0;
+                        total_p[i][j] = 0;
+                    }
+                for (int wd = 0; wd < spp; ++wd) {  // word wd: the four exponent bytes of step s + wd
+                    uint32_t wa[4], wb[4];
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        wa[i] = __ldg(reinterpret_cast<const uint32_t*>(a.exps + (row0 + 4 * ty + i) * a.ld_exps + 4 * (s + wd)));
+                        wb[i] = __ldg(reinterpret_cast<const uint32_t*>(b.exps + (col0 + 4 * tx + i) * b.ld_exps + 4 * (s + wd)));
+                    }
+#pragma unroll
+                    for (int bb = 0; bb < 4; ++bb)
+#pragma unroll
+                        for (int i = 0; i < 4; ++i)
+#pragma unroll
+                            for (int j = 0; j < 4; ++j)
+                                emax_p[i][j] = max(emax_p[i][j], (int)((wa[i] >> (8 * bb)) & 0xFFu) + (int)((wb[j] >> (8 * bb)) & 0xFFu));
+                }
+            }
+            int base[4][4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) base[i][j] = fbase - emax_p[i][j];
+            for (int bb = 0; bb < 4; ++bb) do_block(bb, base, total_p);
+            if (s % spp == spp - 1) finish_pass(emax_p, total_p);
         }
         __syncthreads();  // everyone is done with the step's tiles
     }
@@ -209,7 +251,8 @@ template <int WA, int WB>
 static int launch_hw(const bdr_planes_t& a, const bdr_planes_t& b, int64_t M, int64_t N, int64_t K, int r, int f, float* c, int64_t ldc,
                      cudaStream_t st) {
     const dim3 grid((unsigned)(N / kHwTile), (unsigned)(M / kHwTile));
-    mx_gemm_hw_kernel<WA, WB><<<grid, kHwThreads, 0, st>>>(a, b, K, r, f, c, ldc);
+    if (r > kHwStep) mx_gemm_hw_kernel<WA, WB, true><<<grid, kHwThreads, 0, st>>>(a, b, K, r, f, c, ldc);
+    else mx_gemm_hw_kernel<WA, WB, false><<<grid, kHwThreads, 0, st>>>(a, b, K, r, f, c, ldc);
     return cudaGetLastError() == cudaSuccess ? BDR_OK : BDR_ERR_CUDA;
 }
 
@@ -238,10 +281,10 @@ extern "C" int mx_gemm_hw(const bdr_config_t* cfg_a, const bdr_planes_t* a, cons
         if (cf->k1 != 16 || cf->k2 != 2 || cf->d2 != 1 || (cf->m != 2 && cf->m != 4 && cf->m != 7)) return BDR_ERR_UNSUPPORTED;
     }
     if (M < 0 || N < 0 || K < 0 || ldc < N) return BDR_ERR_SIZE;
-    if (r != 16 && r != 32 && r != 64) return BDR_ERR_UNSUPPORTED;
+    if (r != 16 && r != 32 && r != 64 && r != 128 && r != 256 && r != 512 && r != 1024) return BDR_ERR_UNSUPPORTED;
     if (f < 1 || f > 25) return BDR_ERR_SIZE;
     if (M == 0 || N == 0) return BDR_OK;
-    if (M % kHwTile || N % kHwTile || K % kHwStep || K == 0) return BDR_ERR_UNSUPPORTED;
+    if (M % kHwTile || N % kHwTile || K % kHwStep || K % r || K == 0) return BDR_ERR_UNSUPPORTED;
     for (const bdr_planes_t* p : {a, b}) {
         if (!p->exps || !p->micro || !p->elems) return BDR_ERR_NULL;
         if (((uintptr_t)p->exps | (uintptr_t)p->micro | (uintptr_t)p->elems) % 16) return BDR_ERR_MISALIGNED;

@@ -36,7 +36,7 @@ def spread(rows, K, seed, lo=-6, hi=7):
 @pytest.mark.parametrize("fa,fb", [("MX9", "MX9"), ("MX6", "MX6"), ("MX4", "MX4"), ("MX9", "MX4"), ("MX6", "MX9")])
 def test_bit_exact_against_the_oracle(fa, fb):
     a, b = spread(128, 256, 41), spread(192, 256, 42)
-    for r, f in ((64, 25), (64, 10), (32, 14), (16, 25), (64, 1)):
+    for r, f in ((64, 25), (64, 10), (32, 14), (16, 25), (64, 1), (128, 25), (256, 9)):
         got = run_hw(MX[fa], a, MX[fb], b, r, f)
         want = orc.gemm_hw(H.to_orc(MX[fa]), a, H.to_orc(MX[fb]), b, r=r, f=f)
         H.assert_bits_equal(got, want, "%s x %s r=%d f=%d" % (fa, fb, r, f))
@@ -85,7 +85,7 @@ def test_argument_checks():
     pa = bdr.alloc_planes(bdr.MX6, 64, 64)
     bdr.bdr_pack(bdr.MX6, torch.from_numpy(a).cuda(), pa)
     c = torch.empty((64, 64), dtype=torch.float32, device="cuda")
-    for kw, status in ((dict(r=48), -3), (dict(r=128), -3), (dict(f=0), -5), (dict(f=26), -5)):
+    for kw, status in ((dict(r=48), -3), (dict(r=128), -3), (dict(r=2048), -3), (dict(f=0), -5), (dict(f=26), -5)):   # K = 64: r = 128 does not divide it
         with pytest.raises(bdr.BdrError) as e:
             bdr.mx_gemm_hw(bdr.MX6, pa, bdr.MX6, pa, 64, 64, 64, c, **kw)
         assert e.value.status == status
@@ -96,3 +96,11 @@ def test_argument_checks():
         bdr.mx_gemm_hw(bdr.MX6, pa, bdr.MX6, pa, 32, 64, 64, c)
     assert e.value.status == -3
     torch.cuda.synchronize()
+
+
+def test_passes_longer_than_a_step():
+    # r = 512 and 1024: the blocks of a pass are aligned to a maximum taken over up to 64 blocks
+    a, b = spread(64, 2048, 48, -20, 21), spread(128, 2048, 49, -20, 21)
+    for r, f in ((512, 25), (1024, 16), (1024, 25)):
+        got = run_hw(bdr.MX9, a, bdr.MX6, b, r, f)
+        H.assert_bits_equal(got, orc.gemm_hw(orc.MX9, a, orc.MX6, b, r=r, f=f), "r=%d f=%d" % (r, f))
