@@ -334,14 +334,17 @@ def run_ours(args):
     qsnr = {"%s_axis%d" % (name, axis): float(db[j]) for j, (name, _m, axis, op) in enumerate(ops) if op == "quant_dequant"}
 
     # ---- per-kernel timing on the launching stream (roofline of the dominant kernel) ----
-    # one graph of N_SETS launches of the operation, one per buffer set, replayed: consecutive launches never touch
-    # the same buffers, so inputs (also the 34-76 MB of planes an unpack reads) come from HBM
+    # one graph of ROUNDS x N_SETS launches of the operation, cycling through the buffer sets, replayed: consecutive
+    # launches never touch the same buffers, so inputs (also the 34-76 MB of planes an unpack reads) come from HBM,
+    # and the gap between two graph replays is spread over a dozen launches
     kernels = {}
     reps = max(5, min(args.steps, 20))
+    ROUNDS = 4
     for j, (name, m, axis, op) in enumerate(ops):
         def rot(j=j):
-            for s in range(N_SETS):
-                run_op(j, s, planes_override=plane_sets[s])
+            for _r in range(ROUNDS if use_graph else 1):
+                for s in range(N_SETS):
+                    run_op(j, s, planes_override=plane_sets[s])
         launch = capture(rot) if use_graph else rot
         launch()
         torch.cuda.synchronize()
@@ -351,7 +354,7 @@ def run_ours(args):
             launch()
         b.record()
         torch.cuda.synchronize()
-        dur_ms = a.elapsed_time(b) / (reps * N_SETS)
+        dur_ms = a.elapsed_time(b) / (reps * N_SETS * (ROUNDS if use_graph else 1))
         key = "%s_%s_%s" % (op, name, "row" if axis == 1 else "col")
         kernels[key] = {"ms": dur_ms, "GBps": op_bytes(op, m, n_elems) / (dur_ms * 1e-3) / 1e9}
     peak, peak_kind, peaks = measured_peaks()

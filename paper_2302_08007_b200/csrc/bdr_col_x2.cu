@@ -8,7 +8,7 @@
 // TMA tile store (a third stage covers the time that store needs to drain).
 // When planes are written, a CTA owns tiles of 128 columns x 256 rows and warp w takes block rows 2w and
 // 2w+1 of every tile.  The packed planes are column-major -- the transposed layout the backward-pass
-// GEMMs read -- so codes are first staged per tile in shared memory as [block-row pair][column] items;
+// GEMMs read -- so codes are first staged per tile in shared memory (layouts at CStage);
 // after a CTA barrier the tile's columns are gathered and each column's 16 blocks leave as one
 // contiguous run (32 W code bytes, 16 exponent bytes, 16 microexponent bytes).  Without planes the
 // eight warps of a CTA take eight adjacent column groups of the same 32 rows instead.
@@ -38,8 +38,11 @@ constexpr int kCBarBytes = 256;
 
 template <int W> struct CStage {
     // codes: W even: [block row 16][column 128] items of 2W bytes, columns XOR-swizzled by the block row;
-    //        W odd:  [block-row pair 8][column 128] items of 4W bytes (W words)
-    static constexpr int kElemBytes = kCTileBlocks * kCTileCols * 2 * W;
+    //        W odd:  per column its whole run of 8 W words (block-row pair p at word W p), column c in row
+    //                (c % 4) * 32 + c / 4, rows 8 W + 1 words apart: the lanes of a warp write their k-th columns to
+    //                different banks and the write-out reads a run's words without any index arithmetic
+    static constexpr int kOddPitchWords = 8 * W + 1;
+    static constexpr int kElemBytes = W % 2 ? kCTileCols * kOddPitchWords * 4 : kCTileBlocks * kCTileCols * 2 * W;
     static constexpr int kExpBytes = kCTileBlocks * kCTileCols;  // [block row][column]
     static constexpr int kBytes = W > 0 ? kElemBytes + 2 * kExpBytes : 0;
 };
@@ -186,12 +189,11 @@ col_mx_x2_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant
                         for (int k = 0; k < NCW; ++k) { cw0[2 * c][k] = cl[k]; cw0[2 * c + 1][k] = ch[k]; }
                     } else {
                         // the pair's 32 codes of a column as W words: block row 2w+1 follows 2w at bit 16 W
-                        const uint32_t item = st_elems + ((warp * kCTileCols + 4 * lane + 2 * c) * W) * 4;
 #pragma unroll
                         for (int h = 0; h < 2; ++h) {
                             const uint32_t(&a)[NCW] = cw0[2 * c + h];
                             const uint32_t(&b)[NCW] = h ? ch : cl;
-                            const uint32_t dst = item + h * W * 4;
+                            const uint32_t dst = st_elems + (((2 * c + h) * 32 + lane) * CS::kOddPitchWords + warp * W) * 4;
 #pragma unroll
                             for (int k = 0; k < W / 2; ++k) async::sts32(dst + 4 * k, a[k]);
                             async::sts32(dst + 4 * (W / 2), a[W / 2] | (b[0] << 16));
@@ -236,13 +238,9 @@ col_mx_x2_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant
                     // vector v covers bytes 16v .. 16v+15 of the run: W = 8 -> exactly block row v
                     q = async::lds128(st_elems + v * (kCTileCols * 16) + ((c ^ (v & 7)) * 16));
                 } else {
-                    uint32_t x4[4];
-#pragma unroll
-                    for (int k = 0; k < 4; ++k) {
-                        const int wd = 4 * v + k, pair = wd / W, kk = wd - pair * W;
-                        x4[k] = async::lds32(st_elems + ((pair * kCTileCols + c) * W + kk) * 4);
-                    }
-                    q = make_uint4(x4[0], x4[1], x4[2], x4[3]);
+                    // column c's run is kept whole in row (c % 4) * 32 + c / 4, rows an odd number of words apart
+                    const uint32_t src = st_elems + ((((c & 3) * 32 + (c >> 2)) * CS::kOddPitchWords) + 4 * v) * 4;
+                    q = make_uint4(async::lds32(src), async::lds32(src + 4), async::lds32(src + 8), async::lds32(src + 12));
                 }
                 *reinterpret_cast<uint4*>(out.elems + ((int64_t)ct * kCTileCols + c) * out.ld_elems + blk0 * 2 * W + v * 16) = q;
             }
