@@ -41,12 +41,12 @@ NCU_TRAFFIC_BYTES: dict[str, float | None] = {
     "quant_dequant_MX4_row": 216465664, "quant_dequant_MX4_col": 216645888,
     "quant_dequant_MX6_row": 216837632, "quant_dequant_MX6_col": 215354368,
     "quant_dequant_MX9_row": 216819712, "quant_dequant_MX9_col": 216272128,
-    "pack_MX4_row": 149406720, "pack_MX4_col": 146402560,
-    "pack_MX6_row": 157472768, "pack_MX6_col": 154135808,
-    "pack_MX9_row": 173253888, "pack_MX9_col": 168272128,
-    "unpack_MX4_row": 111284224, "unpack_MX4_col": 108499968,
-    "unpack_MX6_row": 128216832, "unpack_MX6_col": 125247232,
-    "unpack_MX9_row": 154121472, "unpack_MX9_col": 151368960,
+    "pack_MX4_row": 149406720, "pack_MX4_col": 146448384,
+    "pack_MX6_row": 157472768, "pack_MX6_col": 154535680,
+    "pack_MX9_row": 173253888, "pack_MX9_col": 168492800,
+    "unpack_MX4_row": 111284224, "unpack_MX4_col": 109175808,
+    "unpack_MX6_row": 128216832, "unpack_MX6_col": 127134464,
+    "unpack_MX9_row": 154121472, "unpack_MX9_col": 151977728,
 }
 
 
