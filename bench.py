@@ -452,6 +452,11 @@ def run_ours(args):
         sec = oracle_step(xs_cpu, cores)
         cpu_baseline = {"value": step_bytes(xs_cpu.size) / sec / 1e9, "unit": "GB/s", "cores": cores, "kind": "oracle",
                         "sample": "first %d of %d rows, all 18 operations once (%.1f s)" % (sample_rows, ROWS, sec)}
+        one_rows = 512   # the same oracle on one thread, on a sample an eighth as large
+        xs_one = cpu_sample(x_bits, one_rows)
+        sec1 = oracle_step(xs_one, 1)
+        cpu_baseline["single_thread"] = {"value": step_bytes(xs_one.size) / sec1 / 1e9, "unit": "GB/s", "cores": 1,
+                                         "sample": "first %d of %d rows, all 18 operations once (%.1f s)" % (one_rows, ROWS, sec1)}
 
     if rank == 0:
         line = {"metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
