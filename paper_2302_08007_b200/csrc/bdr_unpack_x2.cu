@@ -64,6 +64,18 @@ unpack_row_x2_kernel(bdr_planes_t in, bf16* y, URunIndex ri, uint32_t total, int
     for (uint32_t wi = w0; wi < total; wi += stride) {
         if (!async::mbar_wait(bars + 8 * st, phase)) {
             async::report_timeout(status);
+            // Nothing more is issued.  The copies queued for this and the next S - 1 runs may still be on their way into
+            // this CTA's shared memory: one further bounded wait for each, so that the CTA does not knowingly leave with
+            // a copy in flight (if one still does not land, the CTA leaves all the same: the wait must end).
+            if (lane == 0) {
+                for (int k = 0; k < S; ++k) {
+                    if ((uint64_t)wi + (uint64_t)k * stride >= total) break;
+                    int ds = st + k;
+                    uint32_t dp = phase;
+                    if (ds >= S) { ds -= S; dp ^= 1; }
+                    async::mbar_wait(bars + 8 * ds, dp);
+                }
+            }
             break;
         }
         const uint32_t stage = ring0 + st * US::kBytes;
