@@ -349,6 +349,26 @@ def test_bf16_fast_paths_with_a_row_pitch():
         H.assert_bits_equal(H.device_to_host_f32(back), want, "%s pitch unpack" % (cfg,))
 
 
+def test_bf16_column_fast_paths_with_a_row_pitch():
+    # the tile kernels of the column direction address the tensor through tensor maps built with the caller's pitch
+    rows, cols, ld = 512, 384, 448
+    x = H.make_input("laplace_outliers", rows, cols, "bf16", seed=13)
+    for cfg in (bdr.MX4, bdr.MX6, bdr.MX9):
+        want, so = orc.quant_dequant(H.to_orc(cfg), x, axis=0)
+        y, sums = run_quant(cfg, x, "bf16", axis=0, ld=ld)
+        H.assert_bits_equal(y, want, "%s pitch" % (cfg,))
+        H.assert_qsnr_close(sums, so)
+        xd = H.host_to_device(x, "bf16", ld)
+        planes = bdr.alloc_planes(cfg, rows, cols, 0)
+        bdr.bdr_pack(cfg, xd, planes, axis=0)
+        back = H.host_to_device(np.full_like(x, 3.0), "bf16", ld)
+        bdr.bdr_unpack(cfg, planes, back, axis=0)
+        torch.cuda.synchronize()
+        H.assert_planes_equal(H.planes_to_host(planes), orc.pack(H.to_orc(cfg), x, axis=0), "%s pitch" % (cfg,))
+        H.assert_bits_equal(H.device_to_host_f32(back), want, "%s pitch unpack" % (cfg,))
+    assert bdr.bdr_device_status() == 0
+
+
 @pytest.mark.parametrize("axis", [1, 0])
 def test_bf16_fast_paths_in_place(axis):
     # y may alias x: the run (row direction) or the box (column direction) is loaded whole before it is written back
