@@ -111,10 +111,26 @@ int gather_rows_mx_x2(const bdr_planes_t& in, int64_t n_rows, const int64_t* idx
                       const QParams& qp, int* status, cudaStream_t st);
 
 // Packed MX4 / MX6 operands -> E4M3 bytes plus one power-of-two scale byte per 32 elements (bdr_reencode_f8.cu)
-struct ZeroTiles {   // `count` tiles of 256 x 256 floats of c (row pitch ldc, tiles_n tiles per row of tiles), from tile0 on
+// Order in which the GEMM kernels' clusters walk over the 256 x 256 tiles of C: bands of band_rows tile rows, column by
+// column inside a band (band_rows = 1 is row-major order).  With bands of eight the 74 tiles in flight share eight 256-row
+// panels of A and about ten of B, which stay in L2, and every panel of B is fetched once per band; in row-major order a
+// round of tiles touches every panel of B, and an operand larger than L2 is then read from HBM once per round.
+__host__ __device__ inline void gemm_tile_coords(int t, int tiles_m, int tiles_n, int band_rows, int& tm, int& tn) {
+    const int per_band = band_rows * tiles_n;
+    const int band = t / per_band, r = t - band * per_band;
+    const int left = tiles_m - band * band_rows;
+    const int rows = band_rows < left ? band_rows : left;
+    tn = r / rows;
+    tm = band * band_rows + (r - tn * rows);
+}
+// Bands pay when the operands (bytes as the GEMM reads them) and the tiles of C being written no longer fit in L2 together
+// (126 MB on the target); for operands of 64 MiB (4096^3 in bf16) row-major order measured 3 % faster.
+inline int gemm_band_rows(int64_t operand_bytes) { return operand_bytes > (64ll << 20) ? 8 : 1; }
+
+struct ZeroTiles {   // `count` tiles of 256 x 256 floats of c (row pitch ldc), tiles tile0 .. in the order of gemm_tile_coords
     float* c;
     int64_t ldc;
-    int tiles_n, tile0, count;
+    int tiles_n, tile0, count, tiles_m, band_rows;
 };
 int reencode_rowwise_e4m3(const bdr_planes_t& a, int m_a, const bdr_planes_t& b, int m_b, int64_t M, int64_t N, int64_t K,
                           uint8_t* out_a, uint8_t* out_b, uint8_t* sf_a, uint8_t* sf_b, int* inexact, const ZeroTiles& z,

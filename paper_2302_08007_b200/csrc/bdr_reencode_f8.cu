@@ -220,7 +220,8 @@ reencode_e4m3_kernel(bdr_planes_t a, bdr_planes_t b, int a_strips, int b_strips,
     if ((int)blockIdx.x >= a_strips + b_strips) {
         // extra CTAs: clear the 256 x 256 tiles of C that the GEMM kernel accumulates into
         const int t = z.tile0 + ((int)blockIdx.x - a_strips - b_strips);
-        const int tm = t / z.tiles_n, tn = t - tm * z.tiles_n;
+        int tm, tn;
+        gemm_tile_coords(t, z.tiles_m, z.tiles_n, z.band_rows, tm, tn);
         const int rows_per = (256 + (int)gridDim.y - 1) / (int)gridDim.y;
         const int r0 = (int)blockIdx.y * rows_per, r1 = min(256, r0 + rows_per);
         for (int idx = r0 * 64 + (int)threadIdx.x; idx < r1 * 64; idx += kF8Threads) {  // 64 chunks of 16 bytes per row

@@ -526,7 +526,7 @@ int mx_gemm_f8(const bdr_config_t* cfg_a, const bdr_planes_t* a, const bdr_confi
     if ((uintptr_t)c % 16 || ldc % 4) return BDR_ERR_MISALIGNED;
     if (cudaMemsetAsync(flag, 0, sizeof(int), st) != cudaSuccess) return BDR_ERR_CUDA;
     const F8Plan plan = plan_gemm_f8(M, N, K);
-    const ZeroTiles z = {c, ldc, plan.tiles_n, plan.tiles_full, plan.split_tiles()};
+    const ZeroTiles z = {c, ldc, plan.tiles_n, plan.tiles_full, plan.split_tiles(), plan.tiles_m, plan.band_rows};
     int rc = reencode_rowwise_e4m3(*a, cfg_a->m, *b, cfg_b->m, M, N, K, wa, wb, sfa, sfb, flag, z, st);  // phase 1
     if (rc != BDR_OK) return rc;
     rc = launch_gemm_f8(wa, wb, sfa, sfb, M, N, K, plan, c, ldc, flag, st);                               // phase 2, if exact
@@ -545,7 +545,7 @@ int mx_gemm_e4m3(const uint8_t* a, const uint8_t* scales_a, const uint8_t* b, co
     cudaStream_t st = (cudaStream_t)stream;
     const F8Plan plan = plan_gemm_f8(M, N, K);
     if (plan.split_tiles() > 0) {
-        const ZeroTiles z = {c, ldc, plan.tiles_n, plan.tiles_full, plan.split_tiles()};
+        const ZeroTiles z = {c, ldc, plan.tiles_n, plan.tiles_full, plan.split_tiles(), plan.tiles_m, plan.band_rows};
         zero_tiles_kernel<<<dim3((unsigned)z.count, 4), 256, 0, st>>>(z);
         if (cudaGetLastError() != cudaSuccess) return BDR_ERR_CUDA;
     }
@@ -567,7 +567,7 @@ int bdr_reencode_e4m3(const bdr_config_t* cfg, const bdr_planes_t* in, int64_t r
     if ((in->ld_exps | in->ld_micro | in->ld_elems) % 4) return BDR_ERR_MISALIGNED;
     if (in->ld_exps < K / 16 || in->ld_micro < K / 16 || in->ld_elems < K * (cfg->m + 1) / 8) return BDR_ERR_SIZE;
     const bdr_planes_t none = {};
-    const ZeroTiles z = {nullptr, 0, 1, 0, 0};
+    const ZeroTiles z = {nullptr, 0, 1, 0, 0, 1, 1};
     return reencode_rowwise_e4m3(*in, cfg->m, none, cfg->m, rows, 0, K, out, nullptr, scales, nullptr, inexact_dev, z, (cudaStream_t)stream);
 }
 

@@ -40,7 +40,7 @@ __device__ __forceinline__ void tmem_alloc2_cols(uint32_t* dst_smem, uint32_t nc
 }
 
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kDThreads, 1)
-bf16_gemm_pair_kernel(const __grid_constant__ DenseMaps maps, int tiles_m, int tiles_n, int nk, float* c, int64_t ldc) {
+bf16_gemm_pair_kernel(const __grid_constant__ DenseMaps maps, int tiles_m, int tiles_n, int band_rows, int nk, float* c, int64_t ldc) {
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     uint8_t* stages = reinterpret_cast<uint8_t*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     DenseBars& bars = *reinterpret_cast<DenseBars*>(stages + kDStages * kDStageBytes);
@@ -80,7 +80,8 @@ bf16_gemm_pair_kernel(const __grid_constant__ DenseMaps maps, int tiles_m, int t
             bool ok = true;
             uint32_t it = 0;  // running K-step count across tiles
             for (int t = cluster_id; t < n_tiles && ok; t += n_clusters) {
-                const int tm = t / tiles_n, tn = t - tm * tiles_n;
+                int tm, tn;
+                gemm_tile_coords(t, tiles_m, tiles_n, band_rows, tm, tn);
                 const int row_a = (tm * 2 + (int)rank) * kPairRows, row_b = (tn * 2 + (int)rank) * kPairRows;
                 for (int kk = 0; kk < nk; ++kk, ++it) {
                     const int stage = it % kDStages;
@@ -154,7 +155,8 @@ bf16_gemm_pair_kernel(const __grid_constant__ DenseMaps maps, int tiles_m, int t
             ok = __all_sync(0xFFFFFFFFu, ok);
             if (!ok) break;
             tc_fence_after();
-            const int tm = t / tiles_n, tn = t - tm * tiles_n;
+            int tm, tn;
+            gemm_tile_coords(t, tiles_m, tiles_n, band_rows, tm, tn);
             float* crow = c + ((int64_t)(tm * 2 + (int)rank) * kPairRows + lane_base + lane) * ldc + (int64_t)tn * 256 + col_base;
 #pragma unroll 1
             for (int cc = 0; cc < 128; cc += 32) {
@@ -203,6 +205,7 @@ static int launch_gemm_dense(const void* a_bf16, const void* b_bf16, int64_t M, 
     if (!make_dense_map(&maps.a, a_bf16, M, K) || !make_dense_map(&maps.b, b_bf16, N, K)) return BDR_ERR_CUDA;
     const int tiles_m = (int)(M / 256), tiles_n = (int)(N / 256);
     const int64_t n_tiles = (int64_t)tiles_m * tiles_n;
+    const int band_rows = gemm_band_rows((M + N) * K * 2);
     const int n_clusters = (int)std::min<int64_t>(n_tiles, sm_count() / 2);
     // programmatic dependent launch: set-up may overlap the tail of the kernel before it in the stream; the kernel
     // waits (griddepcontrol.wait) before it reads anything
@@ -216,7 +219,7 @@ static int launch_gemm_dense(const void* a_bf16, const void* b_bf16, int64_t M, 
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    const cudaError_t e = cudaLaunchKernelEx(&cfg, bf16_gemm_pair_kernel, maps, tiles_m, tiles_n, (int)(K / kBK), c, ldc);
+    const cudaError_t e = cudaLaunchKernelEx(&cfg, bf16_gemm_pair_kernel, maps, tiles_m, tiles_n, band_rows, (int)(K / kBK), c, ldc);
     return e == cudaSuccess && cudaGetLastError() == cudaSuccess ? BDR_OK : BDR_ERR_CUDA;
 }
 

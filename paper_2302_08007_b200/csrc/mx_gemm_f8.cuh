@@ -94,7 +94,7 @@ __device__ __forceinline__ void bulk_load_g2s(void* smem_dst, const void* gsrc, 
 }
 
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kFThreads, 1)
-mxf8_gemm_pair_kernel(const __grid_constant__ F8Maps maps, const uint8_t* sf_a, const uint8_t* sf_b, int tiles_m, int tiles_n, int nk,
+mxf8_gemm_pair_kernel(const __grid_constant__ F8Maps maps, const uint8_t* sf_a, const uint8_t* sf_b, int tiles_m, int tiles_n, int band_rows, int nk,
                       int tiles_full, int n_items, float* c, int64_t ldc, const int* gate) {
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     uint8_t* stages = reinterpret_cast<uint8_t*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
@@ -147,7 +147,8 @@ mxf8_gemm_pair_kernel(const __grid_constant__ F8Maps maps, const uint8_t* sf_a, 
                 int t, k0, cnt;
                 bool add;
                 item_of(i, t, k0, cnt, add);
-                const int tm = t / tiles_n, tn = t - tm * tiles_n;
+                int tm, tn;
+                gemm_tile_coords(t, tiles_m, tiles_n, band_rows, tm, tn);
                 const int row_a = (tm * 2 + (int)rank) * kPairRows, row_b = (tn * 2 + (int)rank) * kPairRows;
                 for (int kk = k0; kk < k0 + cnt; ++kk, ++it) {
                     const int stage = it % kFStages;
@@ -260,7 +261,8 @@ mxf8_gemm_pair_kernel(const __grid_constant__ F8Maps maps, const uint8_t* sf_a, 
             ok = __all_sync(0xFFFFFFFFu, ok);
             if (!ok) break;
             tc_fence_after();
-            const int tm = t / tiles_n, tn = t - tm * tiles_n;
+            int tm, tn;
+            gemm_tile_coords(t, tiles_m, tiles_n, band_rows, tm, tn);
             float* crow = c + ((int64_t)(tm * 2 + (int)rank) * kPairRows + lane_base + lane) * ldc + (int64_t)tn * 256 + col_base;
             uint32_t v[4][32];
 #pragma unroll
@@ -300,7 +302,8 @@ mxf8_gemm_pair_kernel(const __grid_constant__ F8Maps maps, const uint8_t* sf_a, 
 // launch, which clears them on the side); grid (z.count, 4), 256 threads.
 __global__ void zero_tiles_kernel(ZeroTiles z) {
     const int t = z.tile0 + (int)blockIdx.x;
-    const int tm = t / z.tiles_n, tn = t - tm * z.tiles_n;
+    int tm, tn;
+    gemm_tile_coords(t, z.tiles_m, z.tiles_n, z.band_rows, tm, tn);
     for (int idx = (int)blockIdx.y * 64 * 64 + (int)threadIdx.x; idx < ((int)blockIdx.y + 1) * 64 * 64; idx += 256) {
         const int r = idx >> 6, ch = idx & 63;  // 64 rows per block, 64 chunks of 16 bytes per row
         *reinterpret_cast<uint4*>(z.c + ((int64_t)tm * 256 + r) * z.ldc + (int64_t)tn * 256 + ch * 4) = make_uint4(0, 0, 0, 0);
@@ -321,13 +324,14 @@ static bool make_f8_map(CUtensorMap* out, const void* base, int64_t rows, int64_
 // How the tiles of an M x N product are handed out: n_clusters clusters, tiles_full tiles with their whole K
 // range, the remaining tiles (fewer than half the cluster count) in two halves of K each.
 struct F8Plan {
-    int tiles_m, tiles_n, n_clusters, tiles_full, n_items;
+    int tiles_m, tiles_n, band_rows, n_clusters, tiles_full, n_items;
     int split_tiles() const { return tiles_m * tiles_n - tiles_full; }
 };
 static F8Plan plan_gemm_f8(int64_t M, int64_t N, int64_t K) {
     F8Plan p;
     p.tiles_m = (int)(M / 256);
     p.tiles_n = (int)(N / 256);
+    p.band_rows = gemm_band_rows((M + N) * K);
     const int T = p.tiles_m * p.tiles_n, cmax = sm_count() / 2;
     p.n_clusters = std::min(T, cmax);
     const int rest = T % cmax;
@@ -361,7 +365,7 @@ static int launch_gemm_f8(const uint8_t* a_e4m3, const uint8_t* b_e4m3, const ui
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    const cudaError_t e = cudaLaunchKernelEx(&cfg, mxf8_gemm_pair_kernel, maps, sf_a, sf_b, plan.tiles_m, plan.tiles_n, (int)(K / kFBK),
+    const cudaError_t e = cudaLaunchKernelEx(&cfg, mxf8_gemm_pair_kernel, maps, sf_a, sf_b, plan.tiles_m, plan.tiles_n, plan.band_rows, (int)(K / kFBK),
                                              plan.tiles_full, plan.n_items, c, ldc, gate);
     return e == cudaSuccess && cudaGetLastError() == cudaSuccess ? BDR_OK : BDR_ERR_CUDA;
 }
