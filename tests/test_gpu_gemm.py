@@ -190,6 +190,25 @@ def test_ws_config4_shape_on_sampled_entries():
     assert rel_frob(c[-256:], orc.gemm_nt_f64(aq[-256:], bq, nthreads=8)) <= 1e-5
 
 
+def test_ws_tiles_walked_in_bands():
+    # operands above 64 MiB: the clusters walk the 9 x 10 tiles in bands of eight tile rows (the last band has one row)
+    # and most clusters take a second tile; every tile must land where it belongs
+    M, N, K = 2304, 2560, 8192
+    a = synth.normal_matrix(M, K, seed=21, stream=1)
+    b = synth.normal_matrix(N, K, seed=21, stream=2, sigma=0.02)
+    c = gpu_gemm_ws(bdr.MX9, a, bdr.MX9, b)
+    assert np.isfinite(c).all()
+    aq, _ = orc.quant_dequant(orc.MX9, a, nthreads=8)
+    bq, _ = orc.quant_dequant(orc.MX9, b, nthreads=8)
+    rng = np.random.default_rng(6)
+    ri, ci = rng.integers(0, M, 8192), rng.integers(0, N, 8192)
+    ref = orc.gemm_nt_f64_sampled(aq, bq, ri, ci)
+    got = c[ri, ci].astype(np.float64)
+    assert np.max(np.abs(got - ref)) <= 1e-4 * np.max(np.abs(ref))      # a misplaced tile is off by the size of an entry
+    assert np.linalg.norm(got - ref) / np.linalg.norm(ref) <= 1e-5
+    assert rel_frob(c[-256:], orc.gemm_nt_f64(aq[-256:], bq, nthreads=8)) <= 1e-5   # the one-row band
+
+
 def test_ws_argument_errors():
     pa, pb = bdr.alloc_planes(bdr.MX6, 256, 64), bdr.alloc_planes(bdr.MX6, 256, 64)
     c = torch.empty((256, 256), device="cuda")

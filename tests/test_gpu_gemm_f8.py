@@ -235,6 +235,26 @@ def test_f8_config4_shape_on_sampled_entries():
     assert rel_frob(c[-256:], orc.gemm_nt_f64(aq[-256:], bq, nthreads=8)) <= 1e-5
 
 
+def test_f8_tiles_walked_in_bands_with_split_tiles():
+    # 8-bit operands above 64 MiB: 9 x 10 tiles in bands of eight tile rows; the 16 tiles of the last round are split
+    # along K and accumulate into tiles that the first phase cleared, addressed in the same banded order
+    M, N, K = 2304, 2560, 16384
+    a = synth.normal_matrix(M, K, seed=22, stream=1)
+    b = synth.normal_matrix(N, K, seed=22, stream=2, sigma=0.02)
+    c, flag = gpu_gemm_f8(bdr.MX6, a, bdr.MX6, b)
+    assert flag == 0
+    assert np.isfinite(c).all()
+    aq, _ = orc.quant_dequant(orc.MX6, a, nthreads=8)
+    bq, _ = orc.quant_dequant(orc.MX6, b, nthreads=8)
+    rng = np.random.default_rng(7)
+    ri, ci = rng.integers(0, M, 8192), rng.integers(0, N, 8192)
+    ref = orc.gemm_nt_f64_sampled(aq, bq, ri, ci)
+    got = c[ri, ci].astype(np.float64)
+    assert np.max(np.abs(got - ref)) <= 1e-4 * np.max(np.abs(ref))
+    assert np.linalg.norm(got - ref) / np.linalg.norm(ref) <= 1e-5
+    assert rel_frob(c[-256:], orc.gemm_nt_f64(aq[-256:], bq, nthreads=8)) <= 1e-5   # the one-row band holds the split tiles
+
+
 def test_f8_argument_errors():
     pa, pb = bdr.alloc_planes(bdr.MX6, 256, 256), bdr.alloc_planes(bdr.MX9, 256, 256)
     c = torch.empty((256, 256), device="cuda")
