@@ -606,6 +606,8 @@ int mx_gemm_ws(const bdr_config_t* cfg_a, const bdr_planes_t* a, const bdr_confi
     const bdr_planes_t* pls[2] = {a, b};
     __nv_bfloat16* outs[2] = {wa, wb};
     const int64_t rows[2] = {M, N};
+    const GemmPlan plan = plan_gemm(M, N, K / kBK, (M + N) * K * 2);
+    if (zero_split_tiles(plan, c, ldc, st) != BDR_OK) return BDR_ERR_CUDA;
     for (int i = 0; i < 2; ++i) {  // phase 1: both operands to bf16, once
         QParams qp;
         qp.k1 = 16; qp.k2 = 2; qp.d2 = 1; qp.m = cfs[i]->m; qp.rounding = cfs[i]->rounding; qp.beta = 1; qp.qmax = (1u << cfs[i]->m) - 1u;
@@ -614,7 +616,7 @@ int mx_gemm_ws(const bdr_config_t* cfg_a, const bdr_planes_t* a, const bdr_confi
         if (rc == BDR_ERR_UNSUPPORTED) rc = unpack_general<__nv_bfloat16>(*pls[i], outs[i], rows[i], K, K, 1, qp, st);
         if (rc != BDR_OK) return rc;
     }
-    return launch_gemm_dense(wa, wb, M, N, K, c, ldc, st);  // phase 2
+    return launch_gemm_dense(wa, wb, M, N, K, plan, c, ldc, st);  // phase 2
 }
 
 int mx_gemm_status(void) {

@@ -82,11 +82,6 @@ __device__ __forceinline__ void umma2_mxf8(uint32_t tmem_d, uint64_t desc_a, uin
         ::"r"(tmem_d), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate), "r"(tmem_sfa), "r"(tmem_sfb)
         : "memory");
 }
-__device__ __forceinline__ void red_add_v4(float* p, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
-    asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(p), "f"(__uint_as_float(a)), "f"(__uint_as_float(b)),
-                 "f"(__uint_as_float(c)), "f"(__uint_as_float(d))
-                 : "memory");
-}
 __device__ __forceinline__ void bulk_load_g2s(void* smem_dst, const void* gsrc, uint32_t bytes, uint64_t* bar) {
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(smem_u32(smem_dst)),
                  "l"(gsrc), "r"(bytes), "r"(smem_u32(bar))
@@ -300,16 +295,6 @@ mxf8_gemm_pair_kernel(const __grid_constant__ F8Maps maps, const uint8_t* sf_a, 
 
 // Clears `z.count` tiles of 256 x 256 floats (for callers of the GEMM kernel that do not come through the re-encoding
 // launch, which clears them on the side); grid (z.count, 4), 256 threads.
-__global__ void zero_tiles_kernel(ZeroTiles z) {
-    const int t = z.tile0 + (int)blockIdx.x;
-    int tm, tn;
-    gemm_tile_coords(t, z.tiles_m, z.tiles_n, z.band_rows, tm, tn);
-    for (int idx = (int)blockIdx.y * 64 * 64 + (int)threadIdx.x; idx < ((int)blockIdx.y + 1) * 64 * 64; idx += 256) {
-        const int r = idx >> 6, ch = idx & 63;  // 64 rows per block, 64 chunks of 16 bytes per row
-        *reinterpret_cast<uint4*>(z.c + ((int64_t)tm * 256 + r) * z.ldc + (int64_t)tn * 256 + ch * 4) = make_uint4(0, 0, 0, 0);
-    }
-}
-
 static bool make_f8_map(CUtensorMap* out, const void* base, int64_t rows, int64_t K) {
     EncodeTiledFn fn = encode_tiled_fn();
     if (!fn) return false;
@@ -323,24 +308,8 @@ static bool make_f8_map(CUtensorMap* out, const void* base, int64_t rows, int64_
 
 // How the tiles of an M x N product are handed out: n_clusters clusters, tiles_full tiles with their whole K
 // range, the remaining tiles (fewer than half the cluster count) in two halves of K each.
-struct F8Plan {
-    int tiles_m, tiles_n, band_rows, n_clusters, tiles_full, n_items;
-    int split_tiles() const { return tiles_m * tiles_n - tiles_full; }
-};
-static F8Plan plan_gemm_f8(int64_t M, int64_t N, int64_t K) {
-    F8Plan p;
-    p.tiles_m = (int)(M / 256);
-    p.tiles_n = (int)(N / 256);
-    p.band_rows = gemm_band_rows((M + N) * K);
-    const int T = p.tiles_m * p.tiles_n, cmax = sm_count() / 2;
-    p.n_clusters = std::min(T, cmax);
-    const int rest = T % cmax;
-    const bool split = rest > 0 && 2 * rest <= cmax && (K / kFBK) % 2 == 0;
-    p.tiles_full = split ? T - rest : T;
-    p.n_items = p.tiles_full + 2 * (T - p.tiles_full);
-    if (split) p.n_clusters = std::min(p.n_items, cmax);
-    return p;
-}
+using F8Plan = GemmPlan;
+static F8Plan plan_gemm_f8(int64_t M, int64_t N, int64_t K) { return plan_gemm(M, N, K / kFBK, (M + N) * K); }
 
 // a_e4m3 [M, K], b_e4m3 [N, K] bytes, contiguous; scale atoms ordered [K / 128][rows / 128][512];
 // M, N multiples of 256, K a multiple of 128.  The tiles plan.tiles_full .. of C must hold zeros.
