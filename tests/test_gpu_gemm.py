@@ -190,6 +190,32 @@ def test_ws_config4_shape_on_sampled_entries():
     assert rel_frob(c[-256:], orc.gemm_nt_f64(aq[-256:], bq, nthreads=8)) <= 1e-5
 
 
+def test_ws_split_tiles_with_a_padded_output_pitch_and_whole_rounds():
+    # two tiles on 74 clusters: both are computed as two halves of K that add into tiles cleared beforehand, with the
+    # pitch of the view C is; the columns beside the view stay untouched.  Called twice: the clearing is per call.
+    M, N, K = 512, 256, 512
+    a = synth.normal_matrix(M, K, seed=23, stream=1)
+    b = synth.normal_matrix(N, K, seed=23, stream=2, sigma=0.02)
+    ta, tb = torch.from_numpy(a).cuda(), torch.from_numpy(b).cuda()
+    pa, pb = bdr.alloc_planes(bdr.MX9, M, K), bdr.alloc_planes(bdr.MX9, N, K)
+    bdr.bdr_pack(bdr.MX9, ta, pa)
+    bdr.bdr_pack(bdr.MX9, tb, pb)
+    ws = torch.empty(bdr.mx_gemm_workspace_bytes(M, N, K), dtype=torch.uint8, device="cuda")
+    wide = torch.full((M, N + 64), 7.0, dtype=torch.float32, device="cuda")
+    ref = oracle_gemm(bdr.MX9, a, bdr.MX9, b)
+    for _ in range(2):
+        bdr.mx_gemm_ws(bdr.MX9, pa, bdr.MX9, pb, M, N, K, wide[:, :N], ws)
+        torch.cuda.synchronize()
+        assert bdr.mx_gemm_status() == 0
+        got = wide.cpu().numpy()
+        assert (got[:, N:] == 7.0).all()
+        assert rel_frob(got[:, :N], ref) <= 1e-5
+    # an odd number of K steps cannot be halved: whole tiles, plain stores
+    K2 = 192
+    a2, b2 = synth.normal_matrix(M, K2, seed=24, stream=1), synth.normal_matrix(N, K2, seed=24, stream=2, sigma=0.02)
+    assert rel_frob(gpu_gemm_ws(bdr.MX6, a2, bdr.MX6, b2), oracle_gemm(bdr.MX6, a2, bdr.MX6, b2)) <= 1e-5
+
+
 def test_ws_tiles_walked_in_bands():
     # operands above 64 MiB: the clusters walk the 9 x 10 tiles in bands of eight tile rows (the last band has one row)
     # and most clusters take a second tile; every tile must land where it belongs
