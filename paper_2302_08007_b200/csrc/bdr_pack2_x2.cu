@@ -67,7 +67,6 @@ pack2_x2_kernel(const __grid_constant__ CUtensorMap xmap, int n_col_tiles, int n
     const uint32_t st_elems = async::smem_u32(smem) + kP2RingBytes + kP2BarBytes;
     const uint32_t st_exps = st_elems + PS::kColElemBytes, st_micro = st_exps + PS::kColExpBytes;
     const uint32_t st_row = st_micro + PS::kColExpBytes + warp * PS::kRowBytes;
-    const x2::Consts kc = x2::make_consts(M, 1);
 
     auto issue = [&](int t, int i, int stg) {  // lane 0 only: box i of tile t into stage stg
         const int rt = t / n_col_tiles, ct = t - rt * n_col_tiles;
@@ -209,22 +208,13 @@ pack2_x2_kernel(const __grid_constant__ CUtensorMap xmap, int n_col_tiles, int n
                     uint32_t w[8];
                     p2_words_of(v[2 * s], v[2 * s + 1], w);
                     x2::PairView pv;
-                    uint32_t aw[8], F;
-                    if constexpr (!SUMS) {
-                        F = x2::pair_view(w, pv);
-                    } else {
-#pragma unroll
-                        for (int j = 0; j < 8; ++j) aw[j] = x2::habs2(w[j]);
-                        F = x2::block_exponent(aw);
-                    }
+                    const uint32_t F = x2::pair_view(w, pv);
                     if (F - x2::kMinF <= (uint32_t)(x2::kMaxF - x2::kMinF)) {
                         if constexpr (!SUMS) {
                             x2::pack_pair_view<W>(pv, F, cw[s], mbs[s]);
                         } else {
-                            float pe = 0.f, ps = 0.f;
-                            uint32_t code2[8], yw[8];
-                            x2::quantize_block_row<true, false, true>(w, aw, F, M, kc, yw, code2, mbs[s], pe, ps);
-                            x2::pack_block<W>(code2, cw[s]);
+                            float pe, ps;
+                            x2::pack_pair_view<W, true>(pv, F, cw[s], mbs[s], &pe, &ps);
                             const double wgt = x2::pow4_weight(F);
                             e2r = fma((double)pe, wgt, e2r);
                             s2r = fma((double)ps, wgt, s2r);

@@ -227,8 +227,9 @@ __device__ __forceinline__ uint32_t pair_view(const uint32_t (&w)[8], PairView& 
     return max(mx & 0xFFFFu, mx >> 16) >> 7;
 }
 
-template <int W>
-__device__ __forceinline__ void pack_pair_view(const PairView& v, uint32_t F, uint32_t (&cw)[(16 * W + 31) / 32], uint32_t& micro) {
+template <int W, bool SUMS = false>
+__device__ __forceinline__ void pack_pair_view(const PairView& v, uint32_t F, uint32_t (&cw)[(16 * W + 31) / 32], uint32_t& micro,
+                                               float* pe = nullptr, float* ps = nullptr) {
     constexpr int M = W - 1;
     constexpr uint32_t e0 = (uint32_t)(127 + 7 - (M - 1));
     constexpr bool kSignTrick = M <= 6;
@@ -236,13 +237,25 @@ __device__ __forceinline__ void pack_pair_view(const PairView& v, uint32_t F, ui
     constexpr uint32_t Cmax = C0 + ((1u << M) - 1u) * 0x10001u;
     const uint32_t s2 = ((254u - F) << 7) * 0x10001u;  // 2^(127-F)
     uint32_t macc = 0, f4[4];
+    [[maybe_unused]] float pe0 = 0.f, pe1 = 0.f, ps0 = 0.f, ps1 = 0.f;
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
         const uint32_t u = hfma2_relu(hmul2(v.pm[i], s2), 0x43804380u, 0xC37FC37Fu);  // relu(256 pm - 255)
-        const uint32_t g = hsub2(0x40004000u, hmin2(u, 0x3F803F80u));                 // 2^tau per half
+        const uint32_t mn = hmin2(u, 0x3F803F80u);                                    // 1 - tau
+        const uint32_t g = hsub2(0x40004000u, mn);                                    // 2^tau per half
         macc += g << (2 * i);
-        uint32_t rA = hmin2(hfma2(hmul2(v.aA[i], s2), g, C0), Cmax);
-        uint32_t rB = hmin2(hfma2(hmul2(v.aB[i], s2), g, C0), Cmax);
+        const uint32_t tA = hmul2(v.aA[i], s2), tB = hmul2(v.aB[i], s2);
+        uint32_t rA = hmin2(hfma2(tA, g, C0), Cmax);
+        uint32_t rB = hmin2(hfma2(tB, g, C0), Cmax);
+        if constexpr (SUMS) {
+            // Eq. 3 sums in the block's normalised domain: the quantized magnitude is (r - C0) 2^-tau, the difference is exact
+            const uint32_t ngi = hfma2(mn, 0xBF00BF00u, 0xBF00BF00u);  // -2^-tau
+            const uint32_t dA = hfma2(hsub2(rA, C0), ngi, tA), dB = hfma2(hsub2(rB, C0), ngi, tB);
+            fma_sq_halves(pe0, pe1, dA);
+            fma_sq_halves(pe0, pe1, dB);
+            fma_sq_halves(ps0, ps1, tA);
+            fma_sq_halves(ps0, ps1, tB);
+        }
         if constexpr (kSignTrick) {
             rA = hsub2(rA, (v.A[i] & kSign2) | 0x3F803F80u);  // -/+ 1.0
             rB = hsub2(rB, (v.B[i] & kSign2) | 0x3F803F80u);
@@ -274,6 +287,7 @@ __device__ __forceinline__ void pack_pair_view(const PairView& v, uint32_t F, ui
     // bit 23+2i = tau of sub-block 2i+1
     const uint32_t t = macc - 0x3F803F80u * 0x55u;
     micro = ((t >> 7) & 0x55u) | ((t >> 22) & 0xAAu);
+    if constexpr (SUMS) { *pe = pe0 + pe1; *ps = ps0 + ps1; }
 }
 
 // Slow route for one block (exponent outside the packed range, Inf/NaN, ties-away): the fp32 /
@@ -392,7 +406,7 @@ __device__ __forceinline__ void quantize_wordcol(const uint32_t (&w)[16], const 
                                                  uint32_t (&cl)[W > 0 ? (16 * W + 31) / 32 : 1],
                                                  uint32_t (&ch)[W > 0 ? (16 * W + 31) / 32 : 1], WordColOut& o) {
     constexpr bool PACK = W > 0;
-    constexpr bool kPackOnly = PACK && !SUMS && !YOUT;
+    constexpr bool kPackOnly = PACK && !YOUT;  // codes (and perhaps sums) only: the formulation with the fixed constant
     constexpr bool kSignTrick = kPackOnly && W - 1 <= 6;
     const uint32_t e0 = (uint32_t)(127 + 7 - (m - 1));
     const uint32_t C0 = ((e0 << 7) + (kSignTrick ? (1u << (m - 1)) : 0u)) * 0x10001u;
@@ -408,9 +422,17 @@ __device__ __forceinline__ void quantize_wordcol(const uint32_t (&w)[16], const 
         if constexpr (kPackOnly) {
             const uint32_t g = hsub2(0x40004000u, v);  // 2^tau
             macc += g << j;
+            [[maybe_unused]] const uint32_t ngi = hfma2(v, 0xBF00BF00u, 0xBF00BF00u);  // -2^-tau
 #pragma unroll
             for (int r = 2 * j; r < 2 * j + 2; ++r) {
-                uint32_t r2 = hmin2(hfma2(hmul2(aw[r], s2), g, C0), C0 + QM);
+                const uint32_t a2 = hmul2(aw[r], s2);
+                uint32_t r2 = hmin2(hfma2(a2, g, C0), C0 + QM);
+                if constexpr (SUMS) {
+                    // the quantized magnitude in the block's normalised domain is (r - C0) 2^-tau; the difference is exact
+                    const uint32_t d2 = hfma2(hsub2(r2, C0), ngi, a2);
+                    fma_sq_halves(pe0, pe1, d2);
+                    fma_sq_halves(ps0, ps1, a2);
+                }
                 if constexpr (kSignTrick) {
                     r2 = hsub2(r2, (w[r] & kSign2) | 0x3F803F80u);
                     code[r] = r2 & (((1u << W) - 1u) * 0x10001u);
