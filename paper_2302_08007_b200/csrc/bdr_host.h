@@ -136,7 +136,7 @@ int reencode_rowwise_e4m3(const bdr_planes_t& a, int m_a, const bdr_planes_t& b,
                           uint8_t* out_a, uint8_t* out_b, uint8_t* sf_a, uint8_t* sf_b, int* inexact, const ZeroTiles& z,
                           cudaStream_t st);
 int unpack_rowwise_mx_x2(const bdr_planes_t& in, __nv_bfloat16* y, int64_t rows, int64_t cols, int64_t ld, const QParams& qp,
-                         cudaStream_t st);  // bdr_unpack_x2.cu
+                         cudaStream_t st, bool chained = false);  // bdr_unpack_x2.cu
 int unpack_colwise_mx_x2(const bdr_planes_t& in, __nv_bfloat16* y, int64_t rows, int64_t cols, int64_t ld, const QParams& qp,
                          cudaStream_t st);  // bdr_unpack_col_x2.cu
 

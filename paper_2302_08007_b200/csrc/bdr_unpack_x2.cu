@@ -118,10 +118,14 @@ unpack_row_x2_kernel(bdr_planes_t in, bf16* y, URunIndex ri, uint32_t total, int
         }
         if (++st == S) { st = 0; phase ^= 1; }
     }
+    // Launched as a programmatic dependent of the kernel before it (the second operand's decode behind the first's in
+    // mx_gemm_ws: the two do not depend on each other, so this one starts while that one drains), this grid must not
+    // finish first: whoever waits for this grid then also has the other one's results.  Otherwise: no effect.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
 }
 
 template <int W>
-static int launch_unpack_x2(const bdr_planes_t& in, bf16* y, int64_t rows, int64_t cols, int64_t ld, bool flat, cudaStream_t st) {
+static int launch_unpack_x2(const bdr_planes_t& in, bf16* y, int64_t rows, int64_t cols, int64_t ld, bool flat, cudaStream_t st, bool chained) {
     const int64_t rpr = cols / kURunElems, total = rows * rpr;
     if (total == 0) return BDR_OK;
     if (total >= (1ll << 31) - (1ll << 24)) return BDR_ERR_UNSUPPORTED;
@@ -138,13 +142,29 @@ static int launch_unpack_x2(const bdr_planes_t& in, bf16* y, int64_t rows, int64
     ri.runs_per_row = make_fastdiv((uint32_t)rpr);
     ri.ld = ld;
     ri.flat = flat ? 1 : 0;
-    kern<<<grid, kUThreads, smem, st>>>(in, y, ri, (uint32_t)total, status);
-    return cudaGetLastError() == cudaSuccess ? BDR_OK : BDR_ERR_CUDA;
+    if (!chained) {
+        kern<<<grid, kUThreads, smem, st>>>(in, y, ri, (uint32_t)total, status);
+        return cudaGetLastError() == cudaSuccess ? BDR_OK : BDR_ERR_CUDA;
+    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3(kUThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    const cudaError_t e = cudaLaunchKernelEx(&cfg, kern, in, y, ri, (uint32_t)total, status);
+    return e == cudaSuccess && cudaGetLastError() == cudaSuccess ? BDR_OK : BDR_ERR_CUDA;
 }
 
 // Whole 2048-element runs, 32-byte aligned output rows; a contiguous tensor with tight planes is one long row.
+// chained: launch as a programmatic dependent of the kernel before it in the stream, which must be another launch of this
+// function whose output this one does not read (see the end of the kernel).
 int unpack_rowwise_mx_x2(const bdr_planes_t& in, bf16* y, int64_t rows, int64_t cols, int64_t ld, const QParams& qp,
-                         cudaStream_t st) {
+                         cudaStream_t st, bool chained) {
     if (qp.k1 != 16 || qp.k2 != 2 || qp.d2 != 1) return BDR_ERR_UNSUPPORTED;
     if (((uintptr_t)y % 32) || (ld * 2) % 32 || cols % 16 != 0) return BDR_ERR_UNSUPPORTED;
     const int W = qp.m + 1;
@@ -157,9 +177,9 @@ int unpack_rowwise_mx_x2(const bdr_planes_t& in, bf16* y, int64_t rows, int64_t 
     flat = rows == 1;
     if (cols % kURunElems != 0) return BDR_ERR_UNSUPPORTED;
     switch (qp.m) {
-        case 2: return launch_unpack_x2<3>(in, y, rows, cols, ld, flat, st);
-        case 4: return launch_unpack_x2<5>(in, y, rows, cols, ld, flat, st);
-        case 7: return launch_unpack_x2<8>(in, y, rows, cols, ld, flat, st);
+        case 2: return launch_unpack_x2<3>(in, y, rows, cols, ld, flat, st, chained);
+        case 4: return launch_unpack_x2<5>(in, y, rows, cols, ld, flat, st, chained);
+        case 7: return launch_unpack_x2<8>(in, y, rows, cols, ld, flat, st, chained);
     }
     return BDR_ERR_UNSUPPORTED;
 }

@@ -608,10 +608,13 @@ int mx_gemm_ws(const bdr_config_t* cfg_a, const bdr_planes_t* a, const bdr_confi
     const int64_t rows[2] = {M, N};
     const GemmPlan plan = plan_gemm(M, N, K / kBK, (M + N) * K * 2);
     if (zero_split_tiles(plan, c, ldc, st) != BDR_OK) return BDR_ERR_CUDA;
+    bool first_fast = false;
     for (int i = 0; i < 2; ++i) {  // phase 1: both operands to bf16, once
         QParams qp;
         qp.k1 = 16; qp.k2 = 2; qp.d2 = 1; qp.m = cfs[i]->m; qp.rounding = cfs[i]->rounding; qp.beta = 1; qp.qmax = (1u << cfs[i]->m) - 1u;
-        int rc = unpack_rowwise_mx_x2(*pls[i], outs[i], rows[i], K, K, qp, st);
+        // the second decode starts while the first drains (it is chained only when the first ran on the same kernel family)
+        int rc = unpack_rowwise_mx_x2(*pls[i], outs[i], rows[i], K, K, qp, st, i == 1 && first_fast);
+        if (i == 0) first_fast = rc == BDR_OK;
         if (rc == BDR_ERR_UNSUPPORTED) rc = unpack_rowwise_mx<__nv_bfloat16>(*pls[i], outs[i], rows[i], K, K, qp, st);
         if (rc == BDR_ERR_UNSUPPORTED) rc = unpack_general<__nv_bfloat16>(*pls[i], outs[i], rows[i], K, K, 1, qp, st);
         if (rc != BDR_OK) return rc;
