@@ -607,7 +607,6 @@ int mx_gemm_ws(const bdr_config_t* cfg_a, const bdr_planes_t* a, const bdr_confi
     __nv_bfloat16* outs[2] = {wa, wb};
     const int64_t rows[2] = {M, N};
     const GemmPlan plan = plan_gemm(M, N, K / kBK, (M + N) * K * 2);
-    if (zero_split_tiles(plan, c, ldc, st) != BDR_OK) return BDR_ERR_CUDA;
     bool first_fast = false;
     for (int i = 0; i < 2; ++i) {  // phase 1: both operands to bf16, once
         QParams qp;
@@ -618,6 +617,8 @@ int mx_gemm_ws(const bdr_config_t* cfg_a, const bdr_planes_t* a, const bdr_confi
         if (rc == BDR_ERR_UNSUPPORTED) rc = unpack_rowwise_mx<__nv_bfloat16>(*pls[i], outs[i], rows[i], K, K, qp, st);
         if (rc == BDR_ERR_UNSUPPORTED) rc = unpack_general<__nv_bfloat16>(*pls[i], outs[i], rows[i], K, K, 1, qp, st);
         if (rc != BDR_OK) return rc;
+        // the tiles that two clusters add into are cleared between the two decodes, as a link of the same chain
+        if (i == 0 && zero_split_tiles(plan, c, ldc, st, true) != BDR_OK) return BDR_ERR_CUDA;
     }
     return launch_gemm_dense(wa, wb, M, N, K, plan, c, ldc, st);  // phase 2
 }

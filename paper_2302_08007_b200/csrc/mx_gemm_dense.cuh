@@ -227,6 +227,7 @@ static bool make_dense_map(CUtensorMap* out, const void* base, int64_t rows, int
 
 // clears `count` tiles of c from tile0 on (tile order of gemm_tile_coords): grid (count, 4), 256 threads
 __global__ void zero_tiles_kernel(ZeroTiles z) {
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");  // see zero_split_tiles
     const int t = z.tile0 + (int)blockIdx.x;
     int tm, tn;
     gemm_tile_coords(t, z.tiles_m, z.tiles_n, z.band_rows, tm, tn);
@@ -234,6 +235,7 @@ __global__ void zero_tiles_kernel(ZeroTiles z) {
         const int r = idx >> 6, ch = idx & 63;  // 64 rows per block, 64 chunks of 16 bytes per row
         *reinterpret_cast<uint4*>(z.c + ((int64_t)tm * 256 + r) * z.ldc + (int64_t)tn * 256 + ch * 4) = make_uint4(0, 0, 0, 0);
     }
+    asm volatile("griddepcontrol.wait;" ::: "memory");  // launched as a programmatic dependent: do not finish before the grid in front
 }
 
 // How the tiles of C are shared out: whole rounds of full tiles, and a last round that would keep at most half of the
@@ -256,11 +258,27 @@ static GemmPlan plan_gemm(int64_t M, int64_t N, int64_t k_steps, int64_t operand
     if (split) p.n_clusters = std::min(p.n_items, cmax);
     return p;
 }
-static int zero_split_tiles(const GemmPlan& plan, float* c, int64_t ldc, cudaStream_t st) {
+// chained: launched as a programmatic dependent of the kernel before it in the stream, whose output it does not touch: it
+// runs while that kernel drains, lets the kernel behind it start at once, and does not finish before the one in front
+// (so whoever waits for the end of such a chain has every link's results).
+static int zero_split_tiles(const GemmPlan& plan, float* c, int64_t ldc, cudaStream_t st, bool chained = false) {
     if (plan.split_tiles() == 0) return BDR_OK;
     const ZeroTiles z = {c, ldc, plan.tiles_n, plan.tiles_full, plan.split_tiles(), plan.tiles_m, plan.band_rows};
-    zero_tiles_kernel<<<dim3((unsigned)z.count, 4), 256, 0, st>>>(z);
-    return cudaGetLastError() == cudaSuccess ? BDR_OK : BDR_ERR_CUDA;
+    if (!chained) {
+        zero_tiles_kernel<<<dim3((unsigned)z.count, 4), 256, 0, st>>>(z);
+        return cudaGetLastError() == cudaSuccess ? BDR_OK : BDR_ERR_CUDA;
+    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)z.count, 4);
+    cfg.blockDim = dim3(256);
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    const cudaError_t e = cudaLaunchKernelEx(&cfg, zero_tiles_kernel, z);
+    return e == cudaSuccess && cudaGetLastError() == cudaSuccess ? BDR_OK : BDR_ERR_CUDA;
 }
 
 // a_bf16 [M, K], b_bf16 [N, K], both contiguous; M, N multiples of 256, K a multiple of 64.  The tiles plan.tiles_full ..
